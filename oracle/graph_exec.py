@@ -1,0 +1,82 @@
+"""CPU fp64 oracle: run an operator graph node by node. TEST INFRASTRUCTURE ONLY.
+
+The graph is the plain-data description the planner receives (tensors = the paper's "edges",
+ops = its "nodes"; Sec. "Design"). The oracle ignores every layout and every arena offset: each
+tensor is one fresh canonical fp64 array, ops run in declaration order (which is a topological
+order of the flow), exactly the unoptimised blueprint the method must stay equal to.
+
+Pinned by tests/test_oracle_models.py against the direct model formulas in oracle/models.py
+and by whole-model invariants (causality, batch independence, permutation equivariance).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from . import ops
+
+# operator codes of the graph description (the C header's fluid_op_kind values)
+(EMBED, LINEAR, ADD, MUL, GELU, SILU, SOFTMAX, LAYERNORM, RMSNORM, ROPE, TRANSPOSE, BMM_QK,
+ BMM_PV, SELECT_LAST_TOKEN) = range(14)
+
+
+def run_op(kind, ins, attrs):
+    """Apply one node to canonical fp64 inputs; returns the list of outputs."""
+    if kind == EMBED:
+        return [ops.embed(ins[0], ins[1], ins[2] if len(ins) > 2 else None)]
+    if kind == LINEAR:
+        return [ops.linear(ins[0], ins[1], ins[2] if len(ins) > 2 else None,
+                           contract=attrs.get("contract", 1))]
+    if kind == ADD:
+        return [ops.add(ins[0], ins[1])]
+    if kind == MUL:
+        return [ops.mul(ins[0], ins[1])]
+    if kind == GELU:
+        return [ops.gelu(ins[0], tanh_form=bool(attrs.get("gelu_tanh", 0)))]
+    if kind == SILU:
+        return [ops.silu(ins[0])]
+    if kind == SOFTMAX:
+        return [ops.softmax(ins[0], causal=bool(attrs.get("causal", 0)),
+                            scale=attrs.get("scale", 1.0))]
+    if kind == LAYERNORM:
+        return [ops.layernorm(ins[0], ins[1], ins[2], eps=attrs.get("eps", 1e-5))]
+    if kind == RMSNORM:
+        return [ops.rmsnorm(ins[0], ins[1], eps=attrs.get("eps", 1e-5))]
+    if kind == ROPE:
+        return [ops.rope(ins[0], base=attrs.get("rope_base", 10000.0),
+                         interleaved=bool(attrs.get("rope_interleaved", 0)))]
+    if kind == TRANSPOSE:
+        return [ops.transpose(ins[0], attrs["perm"])]
+    if kind == BMM_QK:
+        return [ops.bmm_qk(ins[0], ins[1], scale=attrs.get("scale", 1.0))]
+    if kind == BMM_PV:
+        return [ops.bmm_pv(ins[0], ins[1])]
+    if kind == SELECT_LAST_TOKEN:
+        return [ops.select_last_token(ins[0])]
+    raise ValueError(f"unknown op kind {kind}")
+
+
+def run_graph(tensors, op_list, feeds, keep_all=False):
+    """Execute the graph.
+
+    tensors : list of dicts with "dims" (and "kind"); op_list : list of dicts with "kind",
+    "ins", "outs", "attrs"; feeds : {tensor id: array} for every graph input and constant.
+    Returns {tensor id: fp64 array} for every tensor (keep_all) or only those no op consumes
+    plus anything marked as a graph output (kind == 1).
+    """
+    vals = {}
+    for tid, a in feeds.items():
+        a = np.asarray(a)
+        vals[tid] = a if a.dtype.kind in "iu" else a.astype(np.float64)
+    consumed = set()
+    for op in op_list:
+        ins = [vals[i] for i in op["ins"]]
+        outs = run_op(op["kind"], ins, op.get("attrs", {}))
+        for tid, o in zip(op["outs"], outs):
+            assert list(o.shape) == list(tensors[tid]["dims"]), (
+                tensors[tid].get("name"), o.shape, tensors[tid]["dims"])
+            vals[tid] = o
+        consumed.update(op["ins"])
+    if keep_all:
+        return vals
+    return {tid: v for tid, v in vals.items()
+            if tensors[tid].get("kind") == 1 or (tid not in consumed and tid not in feeds)}
