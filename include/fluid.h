@@ -1,0 +1,212 @@
+/*
+ * fluid.h — C-ABI of the planned-arena transformer executor for NVIDIA B200 (sm_100a).
+ *
+ * The two central calls follow the paper's problem statement (FluidML, Sec. "Design"):
+ *   fluid_plan(graph, layout_candidates) -> plan   chooses, on the host, one memory layout per
+ *       tensor ("edge") and one offset per activation inside a single shared arena;
+ *   fluid_run(plan, arena_ptr, inputs, outputs, stream)   executes that blueprint on the GPU.
+ *
+ * Conventions for every call
+ *   - Return value: FLUID_OK (0) or a negative fluid_status_t; fluid_last_error() gives a
+ *     thread-local message for the last failure. Nothing throws or aborts across this boundary.
+ *   - Ownership: the caller owns every device byte (arena, inputs, outputs, constants). The
+ *     library owns only host memory inside fluid_graph_t / fluid_plan_t objects and never allocates
+ *     or frees device memory.
+ *   - "dev" pointers are device addresses; everything else is host memory.
+ *   - A layout of a rank-r tensor is a permutation of its logical dims listed slowest to
+ *     fastest with dense strides; the identity is canonical row-major. For a matrix (0,1) is
+ *     row-major and (1,0) column-major (paper, Sec. "Background", Fig. "matmul").
+ *   - Graph inputs and outputs are dense canonical buffers, passed in declaration order.
+ */
+#ifndef FLUID_H
+#define FLUID_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define FLUID_API __attribute__((visibility("default")))
+#else
+#define FLUID_API
+#endif
+
+#define FLUID_MAX_RANK 5
+#define FLUID_ARENA_ALIGN 1024   /* required alignment of arena_ptr, bytes */
+#define FLUID_ARENA_HEADER 256   /* reserved bytes at arena offset 0 (device status words) */
+#define FLUID_SLOT_ALIGN 256     /* every planned offset and size is a multiple of this */
+
+typedef struct fluid_graph_s fluid_graph_t; /* host object, opaque, library-owned */
+typedef struct fluid_plan_s fluid_plan_t;   /* host object, opaque, library-owned */
+typedef void* fluid_stream;             /* a cudaStream_t (NULL = the legacy default stream) */
+
+typedef enum {
+  FLUID_OK = 0,
+  FLUID_EINVAL = -1,       /* malformed argument, graph or plan */
+  FLUID_EUNSUPPORTED = -2, /* no kernel for this op / layout combination (reported at plan time) */
+  FLUID_EALIGN = -3,       /* a device pointer is not aligned as required */
+  FLUID_ECUDA = -4,        /* a CUDA call or launch failed */
+  FLUID_ENOMEM = -5,       /* host allocation failed */
+  FLUID_ETIMEOUT = -6      /* a bounded device-side wait expired (see fluid_status) */
+} fluid_status_t;
+
+typedef enum { FLUID_F32 = 0, FLUID_BF16 = 1, FLUID_I32 = 2 } fluid_dtype;
+typedef enum { FLUID_INPUT = 0, FLUID_OUTPUT = 1, FLUID_CONST = 2, FLUID_ACT = 3 } fluid_tensor_kind;
+
+/* Primitive operators ("nodes"). Shapes are logical, independent of layout.
+ *  EMBED   (ids[B,S] i32, tok[V,H] [, pos[S,H]]) -> x[B,S,H] = tok[ids] (+ pos)
+ *  LINEAR  (x[..m.., ..k..], w[..k.., ..n..] [, bias[..n..]]) -> y[..m.., ..n..]; contracts the
+ *          last `contract` dims of x with the first `contract` dims of w (the paper's GEMM:
+ *          left (i,k), right (k,j), out (i,j))
+ *  ADD, MUL (a, b) -> elementwise, same shape;  GELU, SILU (x) -> elementwise
+ *  SOFTMAX (s[..., n]) -> over the last dim, after multiplying by `scale`; causal: column j of
+ *          row i (the last two dims) takes part only if j <= i, other outputs are exactly 0
+ *  LAYERNORM (x, gamma, beta) / RMSNORM (x, gamma) -> over the last dim, population variance
+ *  ROPE    (x[B,S,nh,D]) -> rotary embedding with position = index along dim 1
+ *  TRANSPOSE (x) -> y with y dim j = x dim perm[j]
+ *  BMM_QK  (q[B,nh,S,D], kt[B,nh,D,S]) -> scale * q.kt  [B,nh,S,S]
+ *  BMM_PV  (p[B,nh,S,S], v[B,nh,S,D]) -> p.v  [B,nh,S,D]
+ *  SELECT_LAST_TOKEN (x[B,S,H]) -> x[:, S-1, :]  [B,H]
+ */
+typedef enum {
+  FLUID_OP_EMBED = 0, FLUID_OP_LINEAR = 1, FLUID_OP_ADD = 2, FLUID_OP_MUL = 3, FLUID_OP_GELU = 4,
+  FLUID_OP_SILU = 5, FLUID_OP_SOFTMAX = 6, FLUID_OP_LAYERNORM = 7, FLUID_OP_RMSNORM = 8,
+  FLUID_OP_ROPE = 9, FLUID_OP_TRANSPOSE = 10, FLUID_OP_BMM_QK = 11, FLUID_OP_BMM_PV = 12,
+  FLUID_OP_SELECT_LAST_TOKEN = 13, FLUID_OP_COUNT = 14
+} fluid_op_kind;
+
+/* One attribute block serves every operator; unused fields are ignored. */
+typedef struct fluid_op_attrs {
+  int32_t contract;          /* LINEAR: number of contracted dims (>= 1) */
+  int32_t causal;            /* SOFTMAX */
+  int32_t gelu_tanh;         /* GELU: 0 = erf form, 1 = tanh approximation */
+  int32_t rope_interleaved;  /* ROPE: 0 = pairs (i, i+D/2), 1 = pairs (2i, 2i+1) */
+  int32_t perm[8];           /* TRANSPOSE */
+  double scale;              /* BMM_QK, SOFTMAX (0 is read as 1) */
+  double eps;                /* LAYERNORM, RMSNORM */
+  double rope_base;          /* ROPE */
+} fluid_op_attrs;
+
+/* Layout options per tensor (the paper's L(u): "each with a few diverse memory layout
+ * options"). n_cands[t] == 0 means canonical only. perms holds, tensor after tensor, n_cands[t]
+ * permutations of rank(t) ints each; the first candidate of a tensor must be the identity. */
+typedef struct fluid_layout_candidates {
+  int32_t n_tensors;
+  const int32_t* n_cands;
+  const int32_t* perms;
+} fluid_layout_candidates;
+
+/* The paper's external cost function eval(node, layouts) (Algorithm 3): the time of one node
+ * given a layout index for each of its tensors. Return +infinity for an unsupported
+ * combination. node_id is the graph's op id (custom evaluation implies fusion = 0). */
+typedef double (*fluid_eval_fn)(void* user, int32_t node_id, int32_t n_tensors,
+                                const int32_t* tensor_ids, const int32_t* layout_index);
+
+typedef struct fluid_plan_options {
+  int32_t fusion;           /* 1: fold bias/GELU/residual into GEMM epilogues, residual into norms,
+                               SiLU*up into one pass; 0: one step per graph op */
+  int32_t arena_policy;     /* 0: first fit (Algorithm 4 as printed), 1: best fit (its prose) */
+  int32_t no_reuse;         /* 1: one private slice per activation (the naive plan) */
+  int32_t force_canonical;  /* 1: skip the layout search, every tensor canonical */
+  int32_t gemm_path;        /* 0: tensor cores where eligible, 1: SIMT kernel everywhere */
+  int32_t reserved[3];
+  fluid_eval_fn eval;       /* NULL: built-in analytic B200 cost table */
+  void* eval_user;
+} fluid_plan_options;
+
+typedef enum {
+  FLUID_K_EMBED = 0, FLUID_K_NORM = 1, FLUID_K_GEMM_SIMT = 2, FLUID_K_GEMM_TC = 3,
+  FLUID_K_SOFTMAX = 4, FLUID_K_ROPE = 5, FLUID_K_ELTWISE = 6, FLUID_K_PERMUTE = 7,
+  FLUID_K_SELECT_LAST = 8, FLUID_K_COUNT = 9
+} fluid_kernel_id;
+
+typedef struct fluid_step_info {
+  int32_t kernel;        /* fluid_kernel_id */
+  int32_t variant;       /* kernel-specific (GEMM: bit0 A MN-major, bit1 B MN-major, bits 8.. tile N) */
+  int32_t n_ops;         /* graph ops folded into this step */
+  int32_t ops[8];
+  int32_t n_in, n_out;   /* tensors read / written (graph tensor ids) */
+  int32_t in_ids[8];
+  int32_t out_ids[4];
+  double cost;           /* modelled (or user-evaluated) time, seconds */
+  double flops;          /* algorithmic floating-point operations */
+  double bytes;          /* algorithmic bytes moved to and from device memory */
+} fluid_step_info;
+
+/* ---- graph construction (host) --------------------------------------------------------- */
+FLUID_API int fluid_graph_create(fluid_graph_t** g);
+FLUID_API void fluid_graph_destroy(fluid_graph_t* g);
+/* dims: rank ints, logical shape. Returns the tensor id in *tensor_id (ids count from 0). */
+FLUID_API int fluid_graph_add_tensor(fluid_graph_t* g, int dtype, int rank, const int64_t* dims, int kind,
+                           int* tensor_id);
+/* Shapes and dtypes are checked against the operator's definition; attrs may be NULL. */
+FLUID_API int fluid_graph_add_op(fluid_graph_t* g, int op_kind, int n_in, const int* in_ids, int n_out,
+                       const int* out_ids, const fluid_op_attrs* attrs, int* op_id);
+
+/* ---- planning (host only; touches no device) --------------------------------------------
+ * Linearises the graph, splits it into sequences (Algorithms 1-2), runs the per-sequence
+ * dynamic programme over layouts (Eq. 1, Algorithm 3), merges by majority vote, lowers to a
+ * list of kernel steps, computes lifetimes and places every activation with Greedy-by-Size
+ * (Algorithm 4). cands or opts may be NULL (canonical only / defaults). */
+FLUID_API int fluid_plan(const fluid_graph_t* g, const fluid_layout_candidates* cands,
+                      const fluid_plan_options* opts, fluid_plan_t** plan);
+FLUID_API void fluid_plan_destroy(fluid_plan_t* plan);
+FLUID_API void fluid_plan_default_options(fluid_plan_options* opts);
+
+/* Peak bytes of the arena, header included; the caller allocates exactly this much. */
+FLUID_API size_t fluid_plan_arena_bytes(const fluid_plan_t* plan);
+/* Sum of all slices without reuse, and the largest simultaneously-live sum (both + header). */
+FLUID_API size_t fluid_plan_arena_naive_bytes(const fluid_plan_t* plan);
+FLUID_API size_t fluid_plan_arena_live_bound_bytes(const fluid_plan_t* plan);
+/* Total modelled cost of the chosen layouts and of the all-canonical assignment, seconds. */
+FLUID_API double fluid_plan_cost(const fluid_plan_t* plan);
+FLUID_API double fluid_plan_canonical_cost(const fluid_plan_t* plan);
+
+/* Per tensor: chosen layout index and permutation (rank ints); offset/bytes of its arena slice
+ * (offset -1 when it is not arena-resident: input, output, constant, or folded away by fusion);
+ * inclusive step lifetime; alias_of = the tensor whose storage it shares (itself if none).
+ * Any out pointer may be NULL. */
+FLUID_API int fluid_plan_tensor_info(const fluid_plan_t* plan, int tensor_id, int* layout_index, int* perm,
+                           int64_t* offset, int64_t* bytes, int* first_step, int* last_step,
+                           int* alias_of);
+FLUID_API int fluid_plan_num_steps(const fluid_plan_t* plan);
+FLUID_API int fluid_plan_step_info(const fluid_plan_t* plan, int step, fluid_step_info* info);
+/* The sequences of Algorithm 2, as node ids (= op ids when fusion is 0). */
+FLUID_API int fluid_plan_num_sequences(const fluid_plan_t* plan);
+FLUID_API int fluid_plan_sequence(const fluid_plan_t* plan, int index, int* node_ids, int capacity, int* length);
+
+/* ---- constants (weights live outside the arena; the paper keeps them in read-only data) ----
+ * bind: dev_ptr must already hold the tensor in the plan's layout for it and stay valid.
+ * pack: one-time device-side re-layout of a canonical constant into the planned layout. */
+FLUID_API int fluid_plan_bind_constant(fluid_plan_t* plan, int tensor_id, const void* dev_ptr);
+FLUID_API int fluid_pack_constant(const fluid_plan_t* plan, int tensor_id, const void* dev_src_canonical,
+                        void* dev_dst, fluid_stream stream);
+
+/* ---- execution -----------------------------------------------------------------------------
+ * Launches every step of the plan on `stream` and returns without synchronising. arena_ptr:
+ * device, FLUID_ARENA_ALIGN-aligned, fluid_plan_arena_bytes() long. inputs/outputs: host arrays
+ * of device pointers in declaration order, each 16-byte aligned. No device memory is allocated,
+ * freed or copied to the host. Launch errors are reported as FLUID_ECUDA. Runs of one plan that
+ * share an arena must not overlap in time. */
+FLUID_API int fluid_run(fluid_plan_t* plan, void* arena_ptr, const void* const* inputs, void* const* outputs,
+              fluid_stream stream);
+/* As fluid_run, but brackets each step with CUDA events and, after synchronising the stream,
+ * writes per-step milliseconds to step_ms[fluid_plan_num_steps()]. For measurement only. */
+FLUID_API int fluid_run_profiled(fluid_plan_t* plan, void* arena_ptr, const void* const* inputs,
+                       void* const* outputs, fluid_stream stream, float* step_ms);
+/* Synchronises `stream`, reads the arena header and reports in *device_status 0 or the code a
+ * kernel left when one of its bounded waits expired (returns FLUID_ETIMEOUT in that case). */
+FLUID_API int fluid_status(const fluid_plan_t* plan, const void* arena_ptr, fluid_stream stream,
+                 int* device_status);
+
+FLUID_API const char* fluid_last_error(void);
+/* Number of kernel launches issued by this library in this process (for launch accounting). */
+FLUID_API int64_t fluid_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLUID_H */

@@ -21,9 +21,11 @@ implements, so that both produce the same plan bit for bit):
   * Tensors of a node that are not the chain's incoming or outgoing edge (weights, skip
     connections, edges owned by another sequence) are minimised over inside eval's argument and
     reported as that sequence's proposal for them.
-  * Majority vote: most proposals wins; the paper breaks ties at random, this takes the lowest
-    index (any choice is valid; tests check validity and cost, not the pick). After each vote all
-    sequences are re-run with the winners fixed until no edge is proposed two ways.
+  * Majority vote: most proposals wins. The paper breaks ties at random; here a tie goes to the
+    tied layout under which the sequences, re-optimised with it fixed, cost least in total, then
+    to the lowest index (any choice is valid; tests check validity and cost, not the pick).
+    After each vote all sequences are re-run with the winners fixed until no edge is proposed
+    two ways.
   * Not in the paper: if the merged plan costs more than the all-canonical plan, canonical is
     returned (so a plan never loses to doing nothing).
 
@@ -178,7 +180,7 @@ def dp_on_sequence(flow: Flow, seq, ncand, fixed, evalfn):
     l = min(prev, key=lambda k: (prev[k], k))
     cost = prev[l]
     if math.isinf(cost):
-        raise ValueError("no supported layout assignment on a sequence")
+        return None, cost
     proposals = [(edges[-1], l)]
     for i in range(len(seq), 0, -1):
         side, back = backs[i - 1]
@@ -213,6 +215,8 @@ def plan_layouts(ops, ncand, evalfn, const_ids=()):
         votes = {}
         for seq in sequences:
             proposals, _ = dp_on_sequence(flow, seq, ncand, fixed, evalfn)
+            if proposals is None:
+                raise ValueError("no supported layout assignment on a sequence")
             for t, l in proposals:
                 votes.setdefault(t, {})
                 votes[t][l] = votes[t].get(l, 0) + 1
@@ -220,7 +224,19 @@ def plan_layouts(ops, ncand, evalfn, const_ids=()):
         if not conflicted:
             break
         for t in conflicted:
-            fixed[t] = majority(votes[t])
+            top = max(votes[t].values())
+            tied = sorted(l for l, c in votes[t].items() if c == top)
+            if len(tied) == 1:
+                fixed[t] = tied[0]
+                continue
+            best, best_cost = None, None
+            for l in tied:
+                trial = dict(fixed)
+                trial[t] = l
+                c = sum(dp_on_sequence(flow, seq, ncand, trial, evalfn)[1] for seq in sequences)
+                if best is None or c < best_cost:
+                    best, best_cost = l, c
+            fixed[t] = best
     assignment = {t: next(iter(v)) for t, v in votes.items()}
     for t in ncand:
         assignment.setdefault(t, 0)

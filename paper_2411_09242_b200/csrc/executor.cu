@@ -1,0 +1,411 @@
+// fluid_run(): the arena executor. Walks the plan's step list, binds every tensor to
+// arena_ptr + offset (or to a bound constant / caller buffer) and launches one kernel per step on
+// the caller's stream. No allocation, no synchronisation, no copies (the paper's "user only
+// needs to allocate a big block of buffer", Sec. "Evaluation", memory-allocation paragraph).
+#include <atomic>
+#include <cstdio>
+#include <vector>
+
+#include "fluid_internal.h"
+
+namespace fluid {
+
+static std::atomic<int64_t> g_launches{0};
+
+static void perm_strides(const fluid_plan_s* p, int t, int64_t* st) {
+  strides_of(p->graph.tensors[t], p->cands[t][p->layout[t]], st);
+}
+
+// Derive every step's launch payload from the final layouts (host only, no device access).
+int finalize_steps(fluid_plan_s* p) {
+  const auto& T = p->graph.tensors;
+  const int* lo = p->layout.data();
+  for (Step& s : p->steps) {
+    const Node& n = p->nodes[s.node];
+    const TensorDesc& ty = T[n.out];
+    const double es = (double)ty.esize();
+    switch (n.kind) {
+      case N_EMBED: {
+        s.kernel = FLUID_K_EMBED;
+        EmbedParams e{};
+        e.dtype = ty.dtype;
+        e.tokens = int(ty.dims[0] * ty.dims[1]);
+        e.S = (int)ty.dims[1];
+        e.H = (int)ty.dims[2];
+        e.V = (int)T[n.b].dims[0];
+        s.embed = e;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.pos; s.t_ptr[3] = n.out;
+        s.bytes = es * ty.numel() * (n.pos >= 0 ? 3.0 : 2.0) + 4.0 * e.tokens;
+        break;
+      }
+      case N_GEMM: {
+        if (!lower_gemm(p, n, lo, &s.gemm)) {
+          set_error("step for op %d: GEMM cannot be lowered under the chosen layouts", n.ops[0]);
+          return FLUID_EUNSUPPORTED;
+        }
+        const GemmParams& g = s.gemm;
+        s.kernel = gemm_tc_eligible(p, g, &s.tc) ? FLUID_K_GEMM_TC : FLUID_K_GEMM_SIMT;
+        if (s.kernel == FLUID_K_GEMM_TC)
+          s.variant = (s.tc.cfg.a_mn_major ? 1 : 0) | (s.tc.cfg.b_mn_major ? 2 : 0) | (s.tc.cfg.bn << 8);
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.out; s.t_ptr[3] = n.bias; s.t_ptr[4] = n.res;
+        double fl = 2.0 * double(g.batch) * g.M * double(g.N) * g.K;
+        double a = double(g.batch) * g.M * double(g.K), b = double(g.batch) * g.K * double(g.N),
+               c = double(g.batch) * g.M * double(g.N);
+        if (g.causal != CAUSAL_NONE) {
+          const double tri = 0.5 * (1.0 + 1.0 / g.M);
+          fl *= tri;
+          if (g.causal == CAUSAL_SKIP_UPPER) c *= tri;
+          else a *= tri;
+        }
+        s.flops = fl;
+        s.bytes = es * (a + b + c * (g.has_res ? 2.0 : 1.0) + (g.has_bias ? g.N : 0));
+        break;
+      }
+      case N_NORM: {
+        s.kernel = FLUID_K_NORM;
+        NormParams q{};
+        q.dtype = ty.dtype;
+        q.width = (int)ty.dims[ty.rank - 1];
+        q.rows = int(ty.numel() / q.width);
+        q.eps = (float)n.eps;
+        q.rms = n.rms;
+        s.norm = q;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.res; s.t_ptr[2] = n.gamma; s.t_ptr[3] = n.beta; s.t_ptr[4] = n.out;
+        s.bytes = es * ty.numel() * (n.res >= 0 ? 3.0 : 2.0);
+        break;
+      }
+      case N_SOFTMAX: {
+        s.kernel = FLUID_K_SOFTMAX;
+        SoftmaxParams q{};
+        q.dtype = ty.dtype;
+        q.n = (int)ty.dims[ty.rank - 1];
+        q.rows = ty.numel() / q.n;
+        q.rows_per_mat = ty.rank >= 2 ? (int)ty.dims[ty.rank - 2] : 1;
+        q.scale = (float)n.scale;
+        q.causal = n.sm_causal;
+        s.softmax = q;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out;
+        double frac = 1.0;
+        if (q.causal) frac = 0.5 * (1.0 + 1.0 / q.n);
+        s.bytes = es * ty.numel() * 2.0 * frac;
+        break;
+      }
+      case N_ROPE: {
+        s.kernel = FLUID_K_ROPE;
+        RopeParams q{};
+        q.dtype = ty.dtype;
+        int64_t st[FLUID_MAX_RANK];
+        perm_strides(p, n.out, st);
+        for (int i = 0; i < 4; ++i) {
+          q.dims[i] = (int)ty.dims[i];
+          q.st[i] = st[i];
+          q.order[i] = p->cands[n.out][lo[n.out]][i];
+        }
+        q.base = (float)n.rope_base;
+        q.interleaved = n.rope_interleaved;
+        s.rope = q;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out;
+        s.bytes = es * ty.numel() * 2.0;
+        break;
+      }
+      case N_ELTWISE: {
+        s.kernel = FLUID_K_ELTWISE;
+        EltParams q{};
+        q.dtype = ty.dtype;
+        q.n = ty.numel();
+        q.op = n.elt;
+        s.elt = q;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.out;
+        s.bytes = es * ty.numel() * (n.b >= 0 ? 3.0 : 2.0);
+        break;
+      }
+      case N_TRANSPOSE: {
+        s.kernel = FLUID_K_PERMUTE;
+        PermuteParams q{};
+        q.esize = (int)ty.esize();
+        q.rank = ty.rank;
+        int64_t sx[FLUID_MAX_RANK], sy[FLUID_MAX_RANK];
+        perm_strides(p, n.a, sx);
+        perm_strides(p, n.out, sy);
+        q.x_inner = q.y_inner = -1;
+        for (int j = 0; j < 5; ++j) {
+          q.dims[j] = j < ty.rank ? (int)ty.dims[j] : 1;
+          q.xs[j] = j < ty.rank ? sx[n.perm[j]] : 0;
+          q.ys[j] = j < ty.rank ? sy[j] : 0;
+          if (j < ty.rank && q.dims[j] > 1 && q.xs[j] == 1) q.x_inner = j;
+          if (j < ty.rank && q.dims[j] > 1 && q.ys[j] == 1) q.y_inner = j;
+        }
+        s.permute = q;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out;
+        s.bytes = es * ty.numel() * 2.0;
+        break;
+      }
+      case N_SELECT: {
+        s.kernel = FLUID_K_SELECT_LAST;
+        const TensorDesc& tx = T[n.a];
+        PermuteParams q{};
+        q.esize = (int)ty.esize();
+        q.rank = 2;
+        for (int j = 0; j < 5; ++j) { q.dims[j] = 1; q.xs[j] = 0; q.ys[j] = 0; }
+        q.dims[0] = (int)ty.dims[0]; q.dims[1] = (int)ty.dims[1];
+        q.xs[0] = tx.dims[1] * tx.dims[2]; q.xs[1] = 1;
+        q.ys[0] = ty.dims[1]; q.ys[1] = 1;
+        q.x_offset = (tx.dims[1] - 1) * tx.dims[2];
+        q.x_inner = q.y_inner = 1;
+        s.permute = q;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out;
+        s.bytes = es * ty.numel() * 2.0;
+        break;
+      }
+    }
+  }
+  return FLUID_OK;
+}
+
+struct Resolver {
+  const fluid_plan_s* p;
+  char* arena;
+  const void* const* inputs;
+  void* const* outputs;
+  bool ok = true;
+  const void* operator()(int t) {
+    if (t < 0) return nullptr;
+    const int r = p->alias_root[t];
+    const TensorDesc& td = p->graph.tensors[r];
+    switch (td.kind) {
+      case FLUID_INPUT: return inputs[p->input_slot[r]];
+      case FLUID_OUTPUT: return outputs[p->output_slot[r]];
+      case FLUID_CONST:
+        if (!p->const_ptr[r]) {
+          set_error("constant tensor %d is not bound", r);
+          ok = false;
+        }
+        return p->const_ptr[r];
+      default: {
+        const int rec = p->record_of[r];
+        if (rec < 0) {
+          set_error("tensor %d has no storage", r);
+          ok = false;
+          return nullptr;
+        }
+        return arena + p->records[rec].offset;
+      }
+    }
+  }
+};
+
+static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs, void* const* outputs,
+                    cudaStream_t stream, float* step_ms) {
+  if (!p || !arena_ptr) {
+    set_error("null plan or arena");
+    return FLUID_EINVAL;
+  }
+  if (reinterpret_cast<uintptr_t>(arena_ptr) % FLUID_ARENA_ALIGN) {
+    set_error("arena_ptr must be %d-byte aligned", FLUID_ARENA_ALIGN);
+    return FLUID_EALIGN;
+  }
+  const auto& T = p->graph.tensors;
+  std::vector<const void*> key;
+  key.push_back(arena_ptr);
+  for (int t = 0; t < (int)T.size(); ++t) {
+    const void* q = nullptr;
+    if (T[t].kind == FLUID_INPUT) {
+      if (!inputs || !(q = inputs[p->input_slot[t]])) { set_error("input %d is null", p->input_slot[t]); return FLUID_EINVAL; }
+    } else if (T[t].kind == FLUID_OUTPUT) {
+      if (!outputs || !(q = outputs[p->output_slot[t]])) { set_error("output %d is null", p->output_slot[t]); return FLUID_EINVAL; }
+    } else {
+      continue;
+    }
+    if (reinterpret_cast<uintptr_t>(q) & 15) {
+      set_error("input/output pointers must be 16-byte aligned");
+      return FLUID_EALIGN;
+    }
+    key.push_back(q);
+  }
+  Resolver R{p, static_cast<char*>(arena_ptr), inputs, outputs};
+  std::lock_guard<std::mutex> lk(p->mu);
+  // tensor maps hold absolute addresses: (re-)encode when any base address changed
+  if (!p->maps_valid || key != p->bound_key) {
+    for (Step& s : p->steps) {
+      if (s.kernel != FLUID_K_GEMM_TC) continue;
+      const void* a = R(s.t_ptr[0]);
+      const void* b = R(s.t_ptr[1]);
+      if (!R.ok) return FLUID_EINVAL;
+      if (encode_tensor_map(&s.tc.map_a, a, s.tc.a) != 0 || encode_tensor_map(&s.tc.map_b, b, s.tc.b) != 0) {
+        set_error("tensor map encoding failed for the step of op %d", p->nodes[s.node].ops[0]);
+        return FLUID_ECUDA;
+      }
+    }
+    p->bound_key = key;
+    p->maps_valid = true;
+  }
+  std::vector<cudaEvent_t> ev;
+  if (step_ms) {
+    ev.resize(p->steps.size() + 1);
+    for (auto& e : ev) cudaEventCreate(&e);
+    cudaEventRecord(ev[0], stream);
+  }
+  uint32_t* status = reinterpret_cast<uint32_t*>(arena_ptr);
+  {  // the header's status words start every run at zero
+    cudaError_t err = cudaMemsetAsync(arena_ptr, 0, FLUID_ARENA_HEADER, stream);
+    if (err != cudaSuccess) {
+      set_error("clearing the arena header: %s", cudaGetErrorString(err));
+      return FLUID_ECUDA;
+    }
+  }
+  int si = 0;
+  for (Step& s : p->steps) {
+    cudaError_t err = cudaSuccess;
+    switch (s.kernel) {
+      case FLUID_K_EMBED: {
+        EmbedParams q = s.embed;
+        q.ids = static_cast<const int*>(R(s.t_ptr[0])); q.tok = R(s.t_ptr[1]); q.pos = R(s.t_ptr[2]);
+        q.y = const_cast<void*>(R(s.t_ptr[3]));
+        if (R.ok) err = launch_embed(q, stream);
+        break;
+      }
+      case FLUID_K_GEMM_SIMT:
+      case FLUID_K_GEMM_TC: {
+        GemmParams q = s.gemm;
+        q.A = R(s.t_ptr[0]); q.B = R(s.t_ptr[1]); q.C = const_cast<void*>(R(s.t_ptr[2]));
+        q.bias = R(s.t_ptr[3]); q.R = R(s.t_ptr[4]);
+        if (R.ok) err = s.kernel == FLUID_K_GEMM_TC ? launch_gemm_tc(q, s.tc, status, stream) : launch_gemm_simt(q, stream);
+        break;
+      }
+      case FLUID_K_NORM: {
+        NormParams q = s.norm;
+        q.x = R(s.t_ptr[0]); q.res = R(s.t_ptr[1]); q.gamma = R(s.t_ptr[2]); q.beta = R(s.t_ptr[3]);
+        q.y = const_cast<void*>(R(s.t_ptr[4]));
+        if (R.ok) err = launch_norm(q, stream);
+        break;
+      }
+      case FLUID_K_SOFTMAX: {
+        SoftmaxParams q = s.softmax;
+        q.x = R(s.t_ptr[0]); q.y = const_cast<void*>(R(s.t_ptr[1]));
+        if (R.ok) err = launch_softmax(q, stream);
+        break;
+      }
+      case FLUID_K_ROPE: {
+        RopeParams q = s.rope;
+        q.x = R(s.t_ptr[0]); q.y = const_cast<void*>(R(s.t_ptr[1]));
+        if (R.ok) err = launch_rope(q, stream);
+        break;
+      }
+      case FLUID_K_ELTWISE: {
+        EltParams q = s.elt;
+        q.a = R(s.t_ptr[0]); q.b = R(s.t_ptr[1]); q.y = const_cast<void*>(R(s.t_ptr[2]));
+        if (R.ok) err = launch_eltwise(q, stream);
+        break;
+      }
+      case FLUID_K_PERMUTE:
+      case FLUID_K_SELECT_LAST: {
+        PermuteParams q = s.permute;
+        q.x = R(s.t_ptr[0]); q.y = const_cast<void*>(R(s.t_ptr[1]));
+        if (R.ok) err = launch_permute(q, stream);
+        break;
+      }
+    }
+    if (!R.ok) return FLUID_EINVAL;
+    if (err != cudaSuccess) {
+      set_error("step %d (kernel %d): %s", si, s.kernel, cudaGetErrorString(err));
+      return FLUID_ECUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    ++si;
+    if (step_ms) cudaEventRecord(ev[si], stream);
+  }
+  if (step_ms) {
+    cudaError_t err = cudaStreamSynchronize(stream);
+    for (size_t i = 0; i + 1 < ev.size(); ++i) {
+      float ms = 0;
+      cudaEventElapsedTime(&ms, ev[i], ev[i + 1]);
+      step_ms[i] = ms;
+    }
+    for (auto& e : ev) cudaEventDestroy(e);
+    if (err != cudaSuccess) {
+      set_error("stream synchronise: %s", cudaGetErrorString(err));
+      return FLUID_ECUDA;
+    }
+  }
+  return FLUID_OK;
+}
+
+int pack_constant_launch(const fluid_plan_s* p, int t, const void* src, void* dst, void* stream) {
+  const TensorDesc& td = p->graph.tensors[t];
+  PermuteParams q{};
+  q.esize = (int)td.esize();
+  q.rank = td.rank;
+  int64_t sx[FLUID_MAX_RANK], sy[FLUID_MAX_RANK];
+  strides_of(td, identity_perm(), sx);
+  strides_of(td, p->cands[t][p->layout[t]], sy);
+  q.x_inner = q.y_inner = -1;
+  for (int j = 0; j < 5; ++j) {
+    q.dims[j] = j < td.rank ? (int)td.dims[j] : 1;
+    q.xs[j] = j < td.rank ? sx[j] : 0;
+    q.ys[j] = j < td.rank ? sy[j] : 0;
+    if (j < td.rank && q.dims[j] > 1 && q.xs[j] == 1) q.x_inner = j;
+    if (j < td.rank && q.dims[j] > 1 && q.ys[j] == 1) q.y_inner = j;
+  }
+  q.x = src;
+  q.y = dst;
+  cudaError_t err = launch_permute(q, static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) {
+    set_error("pack_constant: %s", cudaGetErrorString(err));
+    return FLUID_ECUDA;
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return FLUID_OK;
+}
+
+}  // namespace fluid
+
+using namespace fluid;
+
+extern "C" {
+
+int fluid_run(fluid_plan_t* plan, void* arena_ptr, const void* const* inputs, void* const* outputs,
+              fluid_stream stream) {
+  return run_impl(plan, arena_ptr, inputs, outputs, static_cast<cudaStream_t>(stream), nullptr);
+}
+
+int fluid_run_profiled(fluid_plan_t* plan, void* arena_ptr, const void* const* inputs, void* const* outputs,
+                       fluid_stream stream, float* step_ms) {
+  if (!step_ms) {
+    set_error("step_ms is null");
+    return FLUID_EINVAL;
+  }
+  return run_impl(plan, arena_ptr, inputs, outputs, static_cast<cudaStream_t>(stream), step_ms);
+}
+
+int fluid_pack_constant(const fluid_plan_t* plan, int tensor_id, const void* dev_src_canonical, void* dev_dst,
+                        fluid_stream stream) {
+  if (!plan || tensor_id < 0 || tensor_id >= (int)plan->graph.tensors.size() || !dev_src_canonical || !dev_dst) {
+    set_error("pack_constant: bad argument");
+    return FLUID_EINVAL;
+  }
+  return pack_constant_launch(plan, tensor_id, dev_src_canonical, dev_dst, stream);
+}
+
+int fluid_status(const fluid_plan_t* plan, const void* arena_ptr, fluid_stream stream, int* device_status) {
+  if (!plan || !arena_ptr || !device_status) {
+    set_error("status: null argument");
+    return FLUID_EINVAL;
+  }
+  uint32_t word = 0;
+  cudaError_t err = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (err == cudaSuccess) err = cudaMemcpy(&word, arena_ptr, sizeof(word), cudaMemcpyDeviceToHost);
+  if (err != cudaSuccess) {
+    set_error("status: %s", cudaGetErrorString(err));
+    return FLUID_ECUDA;
+  }
+  *device_status = (int)word;
+  if (word != 0) {
+    set_error("a device-side wait expired (code 0x%x)", word);
+    return FLUID_ETIMEOUT;
+  }
+  return FLUID_OK;
+}
+
+int64_t fluid_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

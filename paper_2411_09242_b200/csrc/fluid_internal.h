@@ -1,0 +1,136 @@
+// Internal host-side data model of the planner and executor (not part of the C-ABI).
+#pragma once
+
+#include <array>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "fluid.h"
+#include "kernels.h"
+
+namespace fluid {
+
+constexpr double kInf = std::numeric_limits<double>::infinity();
+
+struct TensorDesc {
+  int dtype = FLUID_F32;
+  int rank = 0;
+  int64_t dims[FLUID_MAX_RANK] = {1, 1, 1, 1, 1};
+  int kind = FLUID_ACT;
+  int64_t numel() const {
+    int64_t n = 1;
+    for (int i = 0; i < rank; ++i) n *= dims[i];
+    return n;
+  }
+  int64_t esize() const { return dtype == FLUID_BF16 ? 2 : 4; }
+};
+
+struct OpDesc {
+  int kind = 0;
+  std::vector<int> ins, outs;
+  fluid_op_attrs attrs{};
+};
+
+using Perm = std::array<int8_t, FLUID_MAX_RANK>;
+
+inline Perm identity_perm() { return Perm{0, 1, 2, 3, 4}; }
+
+// Element strides per logical dim for a dense tensor stored with dims ordered `perm`
+// (slowest to fastest).
+inline void strides_of(const TensorDesc& t, const Perm& perm, int64_t* st) {
+  int64_t run = 1;
+  for (int i = t.rank - 1; i >= 0; --i) {
+    st[perm[i]] = run;
+    run *= t.dims[perm[i]];
+  }
+}
+
+// A planning node: one graph op, or several folded into one kernel step.
+enum NodeKind { N_EMBED, N_GEMM, N_NORM, N_SOFTMAX, N_ROPE, N_ELTWISE, N_TRANSPOSE, N_SELECT };
+enum GemmKind { G_LINEAR, G_QK, G_PV };
+
+struct Node {
+  int kind = 0;
+  std::vector<int> ops;        // graph op ids folded into this node, first = anchor
+  std::vector<int> ins, outs;  // distinct external tensors, inputs in role order
+  // role-tagged tensor ids (-1 = absent)
+  int a = -1, b = -1, bias = -1, res = -1, out = -1, gamma = -1, beta = -1, pos = -1;
+  int gemm_kind = G_LINEAR, contract = 1, act = ACT_NONE, causal = CAUSAL_NONE;
+  double scale = 1.0, eps = 1e-5, rope_base = 10000.0;
+  int elt = ELT_ADD, rms = 0, rope_interleaved = 0, sm_causal = 0;
+  int perm[8] = {0, 1, 2, 3, 4, 5, 6, 7};
+};
+
+// One executable step: a kernel id plus the tensors it touches; launch parameters are derived
+// from the plan's layouts when the plan is finalised.
+struct Step {
+  int kernel = 0;
+  int variant = 0;
+  int node = -1;
+  double cost = 0, flops = 0, bytes = 0;
+  // launch payloads (one of these is used, by kernel id)
+  GemmParams gemm{};
+  GemmTcHost tc{};
+  NormParams norm{};
+  SoftmaxParams softmax{};
+  RopeParams rope{};
+  EltParams elt{};
+  PermuteParams permute{};
+  EmbedParams embed{};
+  // tensor ids whose device addresses fill the payload's pointer slots
+  int t_ptr[8] = {-1, -1, -1, -1, -1, -1, -1, -1};
+};
+
+struct ArenaRecord {
+  int root = -1;  // root tensor id
+  int64_t bytes = 0;
+  int first = 0, last = 0;
+  int64_t offset = -1;
+};
+
+}  // namespace fluid
+
+struct fluid_graph_s {
+  std::vector<fluid::TensorDesc> tensors;
+  std::vector<fluid::OpDesc> ops;
+};
+
+struct fluid_plan_s {
+  fluid_graph_s graph;  // private copy
+  fluid_plan_options opts{};
+  std::vector<std::vector<fluid::Perm>> cands;  // per tensor
+  std::vector<fluid::Node> nodes;               // in linear order
+  std::vector<int> node_of_op;
+  std::vector<std::vector<int>> sequences;      // node ids
+  std::vector<int> layout;                      // per tensor: candidate index
+  std::vector<int> alias_root;                  // per tensor: root tensor id
+  std::vector<int> folded;                      // per tensor: 1 if removed by fusion
+  std::vector<fluid::Step> steps;
+  std::vector<fluid::ArenaRecord> records;
+  std::vector<int> record_of;                   // per tensor (root): index in records or -1
+  std::vector<int> first_step, last_step;       // per tensor
+  std::vector<const void*> const_ptr;           // per tensor
+  std::vector<int> input_slot, output_slot;     // per tensor: index in inputs/outputs or -1
+  size_t arena_bytes = 0, naive_bytes = 0, live_bound = 0;
+  double cost = 0, canonical_cost = 0;
+  // executor state: tensor maps are encoded for one set of base addresses and re-encoded when
+  // any of them changes
+  std::mutex mu;
+  std::vector<const void*> bound_key;
+  bool maps_valid = false;
+};
+
+namespace fluid {
+void set_error(const char* fmt, ...);
+int finalize_steps(fluid_plan_s* p);               // executor-side: derive launch payloads
+int pack_constant_launch(const fluid_plan_s* p, int tid, const void* src, void* dst, void* stream);
+double node_cost(const fluid_plan_s* p, const Node& n, const int* layout_of /*per tensor*/);
+bool transpose_is_alias(const fluid_plan_s* p, const Node& n, const int* layout_of);
+// Lower a GEMM-like node under the given layouts; false if the node cannot be expressed.
+bool lower_gemm(const fluid_plan_s* p, const Node& n, const int* layout_of, GemmParams* gp);
+bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& gp, GemmTcHost* tc);
+}  // namespace fluid

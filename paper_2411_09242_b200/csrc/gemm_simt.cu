@@ -1,0 +1,99 @@
+// SIMT GEMM over arbitrarily strided operands (fp32 accumulate, FFMA). It serves the fp32
+// configuration, whose 1e-4 tolerance rules out single-pass tf32 tensor-core products, and any
+// bf16 GEMM whose layout the TMA-fed tensor-core kernel cannot express.
+#include "device_utils.cuh"
+#include "fluid.h"
+#include "kernels.h"
+
+namespace fluid {
+
+constexpr int BM = 64, BN = 64, BK = 16;
+
+__device__ __forceinline__ int64_t split_off(int i, int x0, int64_t s1, int64_t s0) {
+  return (int64_t)(i / x0) * s1 + (int64_t)(i % x0) * s0;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(GemmParams p, int a_k_fast, int b_n_fast) {
+  __shared__ float As[BK][BM + 4];
+  __shared__ float Bs[BK][BN + 4];
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN, bz = blockIdx.z;
+  if (p.causal == CAUSAL_SKIP_UPPER && n0 > m0 + BM - 1) return;
+  int kend = p.K;
+  if (p.causal == CAUSAL_CLIP_K) kend = min(p.K, m0 + BM);
+  const int64_t ab = split_off(bz, p.B0, p.a_s[0], p.a_s[1]);
+  const int64_t bb = split_off(bz, p.B0, p.b_s[0], p.b_s[1]);
+  const int64_t cb = split_off(bz, p.B0, p.c_s[0], p.c_s[1]);
+  const T* A = static_cast<const T*>(p.A) + ab;
+  const T* B = static_cast<const T*>(p.B) + bb;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  float acc[4][4] = {};
+  for (int k0 = 0; k0 < kend; k0 += BK) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int e = tid + 256 * j;
+      const int r = a_k_fast ? e / BK : e % BM, kk = a_k_fast ? e % BK : e / BM;
+      const int m = m0 + r, k = k0 + kk;
+      float v = 0.f;
+      if (m < p.M && k < kend)
+        v = to_f(A[split_off(m, p.M0, p.a_s[2], p.a_s[3]) + split_off(k, p.K0, p.a_s[4], p.a_s[5])]);
+      As[kk][r] = v;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int e = tid + 256 * j;
+      const int c = b_n_fast ? e % BN : e / BK, kk = b_n_fast ? e / BN : e % BK;
+      const int n = n0 + c, k = k0 + kk;
+      float v = 0.f;
+      if (n < p.N && k < kend)
+        v = to_f(B[split_off(k, p.K0, p.b_s[2], p.b_s[3]) + split_off(n, p.N0, p.b_s[4], p.b_s[5])]);
+      Bs[kk][c] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  T* C = static_cast<T*>(p.C) + cb;
+  const T* R = p.has_res ? static_cast<const T*>(p.R) + split_off(bz, p.B0, p.r_s[0], p.r_s[1]) : nullptr;
+  const T* bias = static_cast<const T*>(p.bias);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= p.M) continue;
+    const int64_t cm = split_off(m, p.M0, p.c_s[2], p.c_s[3]);
+    const int64_t rm = R ? split_off(m, p.M0, p.r_s[2], p.r_s[3]) : 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= p.N) continue;
+      float v = acc[i][j] * p.scale;
+      if (p.has_bias) v += to_f(bias[n]);
+      if (p.act == ACT_GELU_ERF) v = gelu_erf(v);
+      else if (p.act == ACT_GELU_TANH) v = gelu_tanh(v);
+      if (R) v += to_f(R[rm + split_off(n, p.N0, p.r_s[4], p.r_s[5])]);
+      C[cm + split_off(n, p.N0, p.c_s[4], p.c_s[5])] = from_f<T>(v);
+    }
+  }
+}
+
+cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t st) {
+  dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, p.batch);
+  const int a_k_fast = p.a_s[5] == 1 || p.a_s[3] != 1;
+  const int b_n_fast = p.b_s[5] == 1 || p.b_s[3] != 1;
+  if (p.dtype == FLUID_BF16) gemm_simt_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(p, a_k_fast, b_n_fast);
+  else gemm_simt_kernel<float><<<grid, 256, 0, st>>>(p, a_k_fast, b_n_fast);
+  return cudaGetLastError();
+}
+
+}  // namespace fluid

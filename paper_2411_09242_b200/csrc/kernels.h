@@ -1,0 +1,151 @@
+// Launch payloads (plain data, visible to host and device) and launch entry points of the
+// sm_100a kernels. Tensor addresses are filled in by the executor from the arena base, the
+// bound constants and the caller's input/output pointers.
+#pragma once
+
+#include <cstdint>
+
+#include <cuda_runtime.h>
+
+namespace fluid {
+
+enum ActKind { ACT_NONE = 0, ACT_GELU_ERF = 1, ACT_GELU_TANH = 2 };
+enum CausalKind { CAUSAL_NONE = 0, CAUSAL_SKIP_UPPER = 1, CAUSAL_CLIP_K = 2 };
+enum EltKind { ELT_ADD = 0, ELT_MUL = 1, ELT_GELU_ERF = 2, ELT_GELU_TANH = 3, ELT_SILU = 4, ELT_SILU_MUL = 5 };
+
+// C[b, m, n] = epilogue(scale * sum_k A[b, m, k] * B[b, k, n]) with every index split in two
+// levels, i = i1 * X0 + i0, and one element stride per level and operand. This one form covers
+// LINEAR over any layout of x / W / y (head-major outputs included) and the batched
+// attention products over any head layout.
+struct GemmParams {
+  const void* A;
+  const void* B;
+  void* C;
+  const void* bias;  // indexed by n, dense
+  const void* R;     // residual, indexed like C with its own strides
+  int dtype;         // FLUID_F32 or FLUID_BF16 (A, B, C, bias, R all share it)
+  int M, N, K, batch;
+  int M0, N0, K0, B0;  // inner extents of the m, n, k and batch index splits
+  int64_t a_s[6];      // strides for b1, b0, m1, m0, k1, k0
+  int64_t b_s[6];      // strides for b1, b0, k1, k0, n1, n0
+  int64_t c_s[6];      // strides for b1, b0, m1, m0, n1, n0
+  int64_t r_s[6];
+  float scale;
+  int act;
+  int causal;  // CAUSAL_SKIP_UPPER: tiles with n > m everywhere are not computed;
+               // CAUSAL_CLIP_K: the k loop stops after the tile holding k = m_max
+  int has_bias, has_res;
+};
+
+// Host-side description of the two TMA tensor maps of a tensor-core GEMM step.
+struct TmaOperand {
+  int rank;
+  uint64_t dims[5];     // elements, fastest first
+  uint64_t strides[5];  // elements; strides[0] == 1
+  uint32_t box[5];
+  int sel[5];           // which index feeds each coordinate: 0 k0, 1 k1, 2 r0, 3 r1, 4 b0, 5 b1
+  int k0, r0, b0;       // inner extents used to split the k, row and batch indices
+  int mn_major;         // 1: the row (m or n) index is the contiguous one
+};
+
+struct GemmTcCfg {
+  int bn;               // tile width (64, 128 or 256); tile height is 128, depth 64
+  int stages;
+  int a_mn_major, b_mn_major;
+  int a_sel[5], b_sel[5];
+  int a_k0, a_r0, a_b0, b_k0, b_r0, b_b0;
+  int a_rank, b_rank;
+};
+
+struct alignas(64) TensorMapStorage {
+  unsigned char bytes[128];
+};
+
+struct GemmTcHost {
+  int eligible;
+  TmaOperand a, b;
+  GemmTcCfg cfg;
+  TensorMapStorage map_a, map_b;
+};
+
+struct NormParams {
+  const void* x;
+  const void* res;    // optional second addend (x + res is normalised)
+  const void* gamma;
+  const void* beta;   // null for RMSNorm
+  void* y;
+  int dtype;
+  int rows, width;
+  float eps;
+  int rms;
+};
+
+struct SoftmaxParams {
+  const void* x;
+  void* y;
+  int dtype;
+  int64_t rows;
+  int n;              // row length
+  int rows_per_mat;   // causal: row index inside its matrix = row % rows_per_mat
+  float scale;
+  int causal;
+};
+
+struct RopeParams {
+  const void* x;
+  void* y;
+  int dtype;
+  int dims[4];        // B, S, nh, D
+  int64_t st[4];      // element strides of x and y (same layout) per logical dim
+  int order[4];       // logical dims, slowest to fastest, in memory
+  float base;
+  int interleaved;
+};
+
+struct EltParams {
+  const void* a;
+  const void* b;
+  void* y;
+  int dtype;
+  int64_t n;
+  int op;
+};
+
+// y[i0..i4] = x[...] for a dense rank-<=5 tensor; dims are the output's logical dims, xs / ys the
+// input / output element strides per output logical dim.
+struct PermuteParams {
+  const void* x;
+  void* y;
+  int esize;
+  int rank;
+  int dims[5];
+  int64_t xs[5], ys[5];
+  int64_t x_offset;   // elements, added to x
+  int x_inner, y_inner;  // output-logical dim that is contiguous in x / in y (-1: none)
+};
+
+struct EmbedParams {
+  const int* ids;
+  const void* tok;
+  const void* pos;    // optional [S, H]
+  void* y;
+  int dtype;
+  int tokens, S, H, V;
+};
+
+// Launchers: enqueue on `stream`, return the CUDA error of the launch.
+cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
+cudaError_t launch_gemm_tc(const GemmParams& p, const GemmTcHost& tc, uint32_t* status,
+                           cudaStream_t stream);
+cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);
+cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t stream);
+cudaError_t launch_rope(const RopeParams& p, cudaStream_t stream);
+cudaError_t launch_eltwise(const EltParams& p, cudaStream_t stream);
+cudaError_t launch_permute(const PermuteParams& p, cudaStream_t stream);
+cudaError_t launch_embed(const EmbedParams& p, cudaStream_t stream);
+
+int encode_tensor_map(TensorMapStorage* out, const void* base, const TmaOperand& op);
+int sm_count();
+bool tc_kernel_available();
+
+}  // namespace fluid

@@ -1,0 +1,1066 @@
+// fluid_plan(): the layout-and-memory planner (host only).
+//
+// Pipeline, in the order the paper's compiler applies it (Sec. "Implementation", "Compiler"):
+// fusion -> linear sequence -> layout reschedule -> memory plan.
+//   linearise        topological order, smallest ready op id first
+//   build_nodes      epilogue / elementwise fusion into planning nodes
+//   split            Algorithms 1 and 2: longest sequence, remove, recurse on connected remains
+//   dp_on_sequence   Eq. 1 / Algorithm 3: cheapest layout per edge of a sequence
+//   merge            majority vote over conflicting proposals, losers re-optimise
+//   lower            elided TRANSPOSEs become aliases, nodes become kernel steps
+//   liveness + Greedy-by-Size  Algorithm 4
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <map>
+#include <new>
+#include <set>
+
+#include "fluid_internal.h"
+
+namespace fluid {
+
+// ---- analytic B200 cost table (the default eval()) ------------------------------------------
+static constexpr double kBw = 6.0e12;        // bytes/s a streaming kernel sustains
+static constexpr double kTcPeak = 1.3e15;    // bf16 tensor-core flop/s under sustained load
+static constexpr double kSimtPeak = 1.5e13;  // flop/s of the SIMT GEMM
+static constexpr double kLaunch = 2.5e-6;    // per-step launch + drain
+
+static const Perm& perm_of(const fluid_plan_s* p, int t, const int* layout_of) { return p->cands[t][layout_of[t]]; }
+
+static bool same_perm(const fluid_plan_s* p, int a, int b, const int* lo) {
+  const TensorDesc& ta = p->graph.tensors[a];
+  const Perm &pa = perm_of(p, a, lo), &pb = perm_of(p, b, lo);
+  for (int i = 0; i < ta.rank; ++i)
+    if (pa[i] != pb[i]) return false;
+  return true;
+}
+
+static bool is_identity(const fluid_plan_s* p, int t, const int* lo) {
+  const Perm& pm = perm_of(p, t, lo);
+  for (int i = 0; i < p->graph.tensors[t].rank; ++i)
+    if (pm[i] != i) return false;
+  return true;
+}
+
+static double tbytes(const fluid_plan_s* p, int t) {
+  const TensorDesc& d = p->graph.tensors[t];
+  return double(d.numel()) * double(d.esize());
+}
+
+bool transpose_is_alias(const fluid_plan_s* p, const Node& n, const int* lo) {
+  const TensorDesc &x = p->graph.tensors[n.a], &y = p->graph.tensors[n.out];
+  if (y.kind == FLUID_OUTPUT) return false;  // the caller's buffer must really be written
+  int64_t sx[FLUID_MAX_RANK], sy[FLUID_MAX_RANK];
+  strides_of(x, perm_of(p, n.a, lo), sx);
+  strides_of(y, perm_of(p, n.out, lo), sy);
+  for (int j = 0; j < y.rank; ++j)
+    if (y.dims[j] > 1 && sy[j] != sx[n.perm[j]]) return false;
+  return true;
+}
+
+// Split `count` consecutive logical dims starting at `first` into (outer, inner) levels.
+static bool two_level(const TensorDesc& t, const int64_t* st, int first, int count, int* x0, int64_t* s1,
+                      int64_t* s0, int64_t* total) {
+  if (count == 1) {
+    *x0 = (int)t.dims[first];
+    *s1 = 0;
+    *s0 = st[first];
+    *total = t.dims[first];
+    return true;
+  }
+  if (count == 2) {
+    *x0 = (int)t.dims[first + 1];
+    *s1 = st[first];
+    *s0 = st[first + 1];
+    *total = t.dims[first] * t.dims[first + 1];
+    return true;
+  }
+  return false;
+}
+
+bool lower_gemm(const fluid_plan_s* p, const Node& n, const int* lo, GemmParams* gp) {
+  const auto& T = p->graph.tensors;
+  const TensorDesc &ta = T[n.a], &tb = T[n.b], &tc = T[n.out];
+  int64_t sa[FLUID_MAX_RANK], sb[FLUID_MAX_RANK], sc[FLUID_MAX_RANK], sr[FLUID_MAX_RANK];
+  strides_of(ta, perm_of(p, n.a, lo), sa);
+  strides_of(tb, perm_of(p, n.b, lo), sb);
+  strides_of(tc, perm_of(p, n.out, lo), sc);
+  if (n.res >= 0) strides_of(T[n.res], perm_of(p, n.res, lo), sr);
+  GemmParams g{};
+  g.dtype = tc.dtype;
+  int64_t M, N, K, tot;
+  int x0;
+  if (n.gemm_kind == G_LINEAR) {
+    const int c = n.contract, mc = ta.rank - c, nc = tb.rank - c;
+    if (!two_level(ta, sa, 0, mc, &g.M0, &g.a_s[2], &g.a_s[3], &M)) return false;
+    if (!two_level(ta, sa, mc, c, &g.K0, &g.a_s[4], &g.a_s[5], &K)) return false;
+    if (!two_level(tb, sb, 0, c, &x0, &g.b_s[2], &g.b_s[3], &tot)) return false;
+    if (!two_level(tb, sb, c, nc, &g.N0, &g.b_s[4], &g.b_s[5], &N)) return false;
+    if (!two_level(tc, sc, 0, mc, &x0, &g.c_s[2], &g.c_s[3], &tot)) return false;
+    if (!two_level(tc, sc, mc, nc, &x0, &g.c_s[4], &g.c_s[5], &tot)) return false;
+    if (n.res >= 0) {
+      two_level(T[n.res], sr, 0, mc, &x0, &g.r_s[2], &g.r_s[3], &tot);
+      two_level(T[n.res], sr, mc, nc, &x0, &g.r_s[4], &g.r_s[5], &tot);
+    }
+    g.batch = 1;
+    g.B0 = 1;
+  } else {
+    // rank-4 operands [B, nh, rows, cols]: batch = (B, nh)
+    g.batch = int(ta.dims[0] * ta.dims[1]);
+    g.B0 = (int)ta.dims[1];
+    g.a_s[0] = sa[0]; g.a_s[1] = sa[1]; g.a_s[2] = 0; g.a_s[3] = sa[2]; g.a_s[4] = 0; g.a_s[5] = sa[3];
+    g.b_s[0] = sb[0]; g.b_s[1] = sb[1]; g.b_s[2] = 0; g.b_s[3] = sb[2]; g.b_s[4] = 0; g.b_s[5] = sb[3];
+    g.c_s[0] = sc[0]; g.c_s[1] = sc[1]; g.c_s[2] = 0; g.c_s[3] = sc[2]; g.c_s[4] = 0; g.c_s[5] = sc[3];
+    M = ta.dims[2];
+    K = ta.dims[3];
+    N = tb.dims[3];
+    g.M0 = (int)M; g.K0 = (int)K; g.N0 = (int)N;
+    if (n.res >= 0) return false;
+  }
+  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return false;
+  g.M = (int)M; g.N = (int)N; g.K = (int)K;
+  g.scale = (float)n.scale;
+  g.act = n.act;
+  g.causal = n.causal;
+  g.has_bias = n.bias >= 0;
+  g.has_res = n.res >= 0;
+  *gp = g;
+  return true;
+}
+
+// ---- TMA operand description for the tensor-core GEMM -------------------------------------------
+// An operand is a set of (extent, stride) levels: row (r1, r0), contraction (k1, k0), batch
+// (b1, b0). Levels whose strides chain are merged; one level must be contiguous (k0: "K-major",
+// r0: "MN-major"); the rest must be 16-byte multiples; tiles may not straddle an unmerged level.
+static bool build_tma_operand(int64_t R, int R0, const int64_t* rs, int64_t K, int K0, const int64_t* ks,
+                              int64_t BATCH, int B0, const int64_t* bs, int tile_rows, TmaOperand* o) {
+  struct Lvl { int64_t n1, n0, s1, s0; bool merged; };
+  auto mk = [](int64_t total, int x0, const int64_t* s) {
+    Lvl l;
+    l.n0 = x0;
+    l.n1 = total / x0;
+    l.s1 = s[0];
+    l.s0 = s[1];
+    l.merged = false;
+    if (l.n1 == 1) {
+      l.merged = true;
+    } else if (l.n0 == 1) {
+      l.n0 = l.n1; l.s0 = l.s1; l.n1 = 1; l.merged = true;
+    } else if (l.s1 == l.n0 * l.s0) {
+      l.n0 = total; l.n1 = 1; l.merged = true;
+    }
+    return l;
+  };
+  Lvl r = mk(R, R0, rs), k = mk(K, K0, ks), b = mk(BATCH, B0, bs);
+  const bool k_major = (k.n0 == 1 && k.n1 == 1) ? (r.s0 != 1) : (k.s0 == 1);
+  const bool mn_major = !k_major && (r.s0 == 1 || (r.n0 == 1 && r.n1 == 1));
+  if (!k_major && !mn_major) return false;
+  if (k.n0 * k.n1 == 1 && !k_major) { /* degenerate K = 1 handled as MN-major */ }
+  auto aligned = [](int64_t n, int64_t s) { return n == 1 || (s % 8 == 0); };
+  if (k_major) {
+    if (!(k.s0 == 1 || k.n0 == 1)) return false;
+    if (!aligned(k.n1, k.s1) || !aligned(r.n0, r.s0) || !aligned(r.n1, r.s1)) return false;
+    if (!k.merged && k.n0 % 64 != 0) return false;
+    if (!r.merged && r.n0 % tile_rows != 0) return false;
+  } else {
+    if (!aligned(r.n1, r.s1) || !aligned(k.n0, k.s0) || !aligned(k.n1, k.s1)) return false;
+    if (!r.merged && r.n0 % 64 != 0) return false;
+    if (!k.merged && k.n0 % 64 != 0) return false;
+  }
+  if (!aligned(b.n0, b.s0) || !aligned(b.n1, b.s1)) return false;
+  TmaOperand t{};
+  t.mn_major = mn_major ? 1 : 0;
+  t.k0 = (int)k.n0; t.r0 = (int)r.n0; t.b0 = (int)b.n0;
+  int d = 0;
+  auto push = [&](int64_t n, int64_t s, uint32_t box, int sel) {
+    t.dims[d] = (uint64_t)n; t.strides[d] = (uint64_t)s; t.box[d] = box; t.sel[d] = sel; ++d;
+  };
+  if (k_major) {
+    push(k.n0, 1, 64, 0);
+    if (k.n1 > 1) push(k.n1, k.s1, 1, 1);
+    push(r.n0, r.n0 == 1 ? 8 : r.s0, (uint32_t)tile_rows, 2);
+  } else {
+    push(r.n0, 1, 64, 2);
+    if (r.n1 > 1) push(r.n1, r.s1, 1, 3);
+    push(k.n0, k.n0 == 1 ? 8 : k.s0, 64, 0);
+    if (k.n1 > 1) push(k.n1, k.s1, 1, 1);
+  }
+  if (k_major && r.n1 > 1) {
+    if (d >= 5) return false;
+    push(r.n1, r.s1, 1, 3);
+  }
+  if (b.n0 > 1) {
+    if (d >= 5) return false;
+    push(b.n0, b.s0, 1, 4);
+  }
+  if (b.n1 > 1) {
+    if (d >= 5) return false;
+    push(b.n1, b.s1, 1, 5);
+  }
+  if (d > 5) return false;
+  t.rank = d;
+  // contiguity of the fastest level
+  if (t.dims[0] > 1 && t.strides[0] != 1) return false;
+  *o = t;
+  return true;
+}
+
+bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& g, GemmTcHost* tc) {
+  GemmTcHost h{};
+  h.eligible = 0;
+  *tc = h;
+  if (!tc_kernel_available() || p->opts.gemm_path == 1 || g.dtype != FLUID_BF16) return false;
+  if (g.K < 8) return false;
+  int bn = 128;
+  if (g.N <= 64) bn = 64;
+  else {
+    const int64_t tiles256 = int64_t((g.M + 127) / 128) * ((g.N + 255) / 256) * g.batch;
+    if (g.N >= 256 && tiles256 >= 120) bn = 256;
+  }
+  const int64_t a_rs[2] = {g.a_s[2], g.a_s[3]}, a_ks[2] = {g.a_s[4], g.a_s[5]}, a_bs[2] = {g.a_s[0], g.a_s[1]};
+  const int64_t b_rs[2] = {g.b_s[4], g.b_s[5]}, b_ks[2] = {g.b_s[2], g.b_s[3]}, b_bs[2] = {g.b_s[0], g.b_s[1]};
+  if (!build_tma_operand(g.M, g.M0, a_rs, g.K, g.K0, a_ks, g.batch, g.B0, a_bs, 128, &h.a)) return false;
+  // an unmerged n level narrower than the tile would be straddled: shrink the tile first
+  while (true) {
+    if (build_tma_operand(g.N, g.N0, b_rs, g.K, g.K0, b_ks, g.batch, g.B0, b_bs, bn, &h.b)) break;
+    if (bn == 64) return false;
+    bn /= 2;
+  }
+  // output / residual vector accesses assume 8-element alignment of every outer stride when the
+  // n index is contiguous; otherwise the epilogue falls back to scalar stores (always legal)
+  h.cfg.bn = bn;
+  h.cfg.stages = bn == 256 ? 4 : (bn == 128 ? 6 : 8);
+  h.cfg.a_mn_major = h.a.mn_major;
+  h.cfg.b_mn_major = h.b.mn_major;
+  for (int i = 0; i < 5; ++i) {
+    h.cfg.a_sel[i] = h.a.sel[i];
+    h.cfg.b_sel[i] = h.b.sel[i];
+  }
+  h.cfg.a_k0 = h.a.k0; h.cfg.a_r0 = h.a.r0; h.cfg.a_b0 = h.a.b0;
+  h.cfg.b_k0 = h.b.k0; h.cfg.b_r0 = h.b.r0; h.cfg.b_b0 = h.b.b0;
+  h.cfg.a_rank = h.a.rank;
+  h.cfg.b_rank = h.b.rank;
+  h.eligible = 1;
+  *tc = h;
+  return true;
+}
+
+static double gemm_flops(const GemmParams& g) {
+  double f = 2.0 * double(g.batch) * g.M * double(g.N) * g.K;
+  if (g.causal != CAUSAL_NONE) f *= 0.5 * (1.0 + 1.0 / std::max(1, g.M));
+  return f;
+}
+
+static double gemm_bytes(const GemmParams& g) {
+  const double es = g.dtype == FLUID_BF16 ? 2.0 : 4.0;
+  double a = double(g.batch) * g.M * double(g.K), b = double(g.batch) * g.K * double(g.N),
+         c = double(g.batch) * g.M * double(g.N);
+  if (g.causal == CAUSAL_SKIP_UPPER) c *= 0.5;
+  if (g.causal == CAUSAL_CLIP_K) a *= 0.5;
+  return es * (a + b + c * (g.has_res ? 2.0 : 1.0) + (g.has_bias ? g.N : 0));
+}
+
+double node_cost(const fluid_plan_s* p, const Node& n, const int* lo) {
+  const auto& T = p->graph.tensors;
+  switch (n.kind) {
+    case N_EMBED: {
+      for (int t : n.ins)
+        if (!is_identity(p, t, lo)) return kInf;
+      if (!is_identity(p, n.out, lo)) return kInf;
+      return kLaunch + 2.0 * tbytes(p, n.out) / kBw;
+    }
+    case N_GEMM: {
+      GemmParams g;
+      if (!lower_gemm(p, n, lo, &g)) return kInf;
+      if (n.bias >= 0 && !is_identity(p, n.bias, lo)) return kInf;
+      if (n.res >= 0) {
+        for (int i = 0; i < 6; ++i)
+          if (g.r_s[i] != g.c_s[i]) return kInf;
+      }
+      GemmTcHost tc;
+      const double fl = gemm_flops(g), by = gemm_bytes(g);
+      if (gemm_tc_eligible(p, g, &tc)) {
+        const double skew = 1.0 + 0.02 * (tc.cfg.a_mn_major + tc.cfg.b_mn_major);
+        const bool c_fast = g.c_s[5] == 1 || g.c_s[3] == 1;
+        return kLaunch + std::max(fl / kTcPeak, by / kBw) * skew * (c_fast ? 1.0 : 1.5);
+      }
+      const bool a_fast = g.a_s[5] == 1 || g.a_s[3] == 1, b_fast = g.b_s[5] == 1 || g.b_s[3] == 1,
+                 c_fast = g.c_s[5] == 1 || g.c_s[3] == 1;
+      const double pen = (a_fast ? 1.0 : 4.0) * (b_fast ? 1.0 : 4.0) * (c_fast ? 1.0 : 2.0);
+      return kLaunch + std::max(fl / kSimtPeak, by / kBw) * pen;
+    }
+    case N_NORM: {
+      const int rank = T[n.out].rank;
+      if (perm_of(p, n.out, lo)[rank - 1] != rank - 1) return kInf;
+      if (!same_perm(p, n.a, n.out, lo)) return kInf;
+      if (n.res >= 0 && !same_perm(p, n.res, n.out, lo)) return kInf;
+      return kLaunch + (2.0 + (n.res >= 0 ? 1.0 : 0.0)) * tbytes(p, n.out) / kBw;
+    }
+    case N_SOFTMAX: {
+      const int rank = T[n.out].rank;
+      const Perm& pm = perm_of(p, n.out, lo);
+      if (pm[rank - 1] != rank - 1 || !same_perm(p, n.a, n.out, lo)) return kInf;
+      if (n.sm_causal && pm[rank - 2] != rank - 2) return kInf;
+      return kLaunch + (n.sm_causal ? 1.5 : 2.0) * tbytes(p, n.out) / kBw;
+    }
+    case N_ROPE:
+      if (!same_perm(p, n.a, n.out, lo)) return kInf;
+      return kLaunch + 2.0 * tbytes(p, n.out) / kBw;
+    case N_ELTWISE: {
+      if (!same_perm(p, n.a, n.out, lo)) return kInf;
+      if (n.b >= 0 && !same_perm(p, n.b, n.out, lo)) return kInf;
+      return kLaunch + (2.0 + (n.b >= 0 ? 1.0 : 0.0)) * tbytes(p, n.out) / kBw;
+    }
+    case N_TRANSPOSE: {
+      if (transpose_is_alias(p, n, lo)) return 0.0;
+      const TensorDesc &x = T[n.a], &y = T[n.out];
+      const Perm &px = perm_of(p, n.a, lo), &py = perm_of(p, n.out, lo);
+      const bool inner_kept = n.perm[py[y.rank - 1]] == px[x.rank - 1];
+      return kLaunch + 2.0 * tbytes(p, n.out) / kBw * (inner_kept ? 1.0 : 1.25);
+    }
+    case N_SELECT:
+      if (!is_identity(p, n.a, lo) || !is_identity(p, n.out, lo)) return kInf;
+      return kLaunch + 2.0 * tbytes(p, n.out) / kBw;
+  }
+  return kInf;
+}
+
+// ---- evaluation wrapper: built-in table or the caller's eval() -----------------------------------
+struct Evaluator {
+  const fluid_plan_s* p;
+  std::vector<int> lo;  // scratch: layout index per tensor
+  double operator()(int node, const std::vector<int>& tids, const std::vector<int>& lidx) {
+    const Node& n = p->nodes[node];
+    if (p->opts.eval) {
+      return p->opts.eval(p->opts.eval_user, n.ops[0], (int)tids.size(), tids.data(), lidx.data());
+    }
+    for (size_t i = 0; i < tids.size(); ++i) lo[tids[i]] = lidx[i];
+    return node_cost(p, n, lo.data());
+  }
+};
+
+static std::vector<int> node_tensors(const Node& n) {
+  std::vector<int> v;
+  auto add = [&](int t) {
+    if (std::find(v.begin(), v.end(), t) == v.end()) v.push_back(t);
+  };
+  for (int t : n.ins) add(t);
+  for (int t : n.outs) add(t);
+  return v;
+}
+
+static double total_cost(fluid_plan_s* p, Evaluator& ev, const std::vector<int>& assign) {
+  double c = 0;
+  for (size_t i = 0; i < p->nodes.size(); ++i) {
+    std::vector<int> tids = node_tensors(p->nodes[i]), l;
+    for (int t : tids) l.push_back(assign[t]);
+    c += ev((int)i, tids, l);
+  }
+  return c;
+}
+
+// ---- P1: graph -> linear sequence ------------------------------------------------------------------
+static bool linearise(const fluid_graph_s& g, std::vector<int>* order) {
+  const int n = (int)g.ops.size();
+  std::vector<int> producer(g.tensors.size(), -1), indeg(n, 0);
+  for (int o = 0; o < n; ++o)
+    for (int t : g.ops[o].outs) producer[t] = o;
+  std::vector<std::set<int>> pred(n);
+  std::vector<std::vector<int>> succ(n);
+  for (int o = 0; o < n; ++o)
+    for (int t : g.ops[o].ins)
+      if (producer[t] >= 0) pred[o].insert(producer[t]);
+  for (int o = 0; o < n; ++o) {
+    indeg[o] = (int)pred[o].size();
+    for (int q : pred[o]) succ[q].push_back(o);
+  }
+  std::set<int> ready;
+  for (int o = 0; o < n; ++o)
+    if (indeg[o] == 0) ready.insert(o);
+  order->clear();
+  while (!ready.empty()) {
+    int v = *ready.begin();
+    ready.erase(ready.begin());
+    order->push_back(v);
+    for (int s : succ[v])
+      if (--indeg[s] == 0) ready.insert(s);
+  }
+  return (int)order->size() == n;
+}
+
+// ---- fusion: graph ops -> planning nodes ----------------------------------------------------------
+static void build_nodes(fluid_plan_s* p, const std::vector<int>& order) {
+  const fluid_graph_s& g = p->graph;
+  const int nops = (int)g.ops.size(), nt = (int)g.tensors.size();
+  const bool fuse = p->opts.fusion != 0;
+  std::vector<int> pos(nops), producer(nt, -1);
+  std::vector<std::vector<int>> consumers(nt);
+  for (int i = 0; i < nops; ++i) pos[order[i]] = i;
+  for (int o = 0; o < nops; ++o) {
+    for (int t : g.ops[o].outs) producer[t] = o;
+    for (int t : g.ops[o].ins) consumers[t].push_back(o);
+  }
+  std::vector<char> absorbed(nops, 0);
+  p->node_of_op.assign(nops, -1);
+  p->folded.assign(nt, 0);
+  auto sole_consumer = [&](int t) -> int {
+    if (g.tensors[t].kind != FLUID_ACT || consumers[t].size() != 1) return -1;
+    int c = consumers[t][0];
+    return absorbed[c] ? -1 : c;
+  };
+  auto available_before = [&](int t, int at_pos) { return producer[t] < 0 || pos[producer[t]] < at_pos; };
+  for (int oi = 0; oi < nops; ++oi) {
+    const int o = order[oi];
+    if (absorbed[o]) continue;
+    const OpDesc& op = g.ops[o];
+    Node n;
+    n.ops.push_back(o);
+    n.out = op.outs[0];
+    n.a = op.ins[0];
+    switch (op.kind) {
+      case FLUID_OP_EMBED:
+        n.kind = N_EMBED; n.b = op.ins[1]; n.pos = op.ins.size() > 2 ? op.ins[2] : -1;
+        break;
+      case FLUID_OP_LINEAR:
+      case FLUID_OP_BMM_QK:
+      case FLUID_OP_BMM_PV: {
+        n.kind = N_GEMM;
+        n.b = op.ins[1];
+        n.gemm_kind = op.kind == FLUID_OP_LINEAR ? G_LINEAR : (op.kind == FLUID_OP_BMM_QK ? G_QK : G_PV);
+        n.contract = op.attrs.contract;
+        n.scale = op.kind == FLUID_OP_BMM_QK ? op.attrs.scale : 1.0;
+        if (op.kind == FLUID_OP_LINEAR && op.ins.size() > 2) n.bias = op.ins[2];
+        if (fuse && op.kind == FLUID_OP_LINEAR) {
+          int c = sole_consumer(n.out);
+          if (c >= 0 && g.ops[c].kind == FLUID_OP_GELU) {
+            n.act = g.ops[c].attrs.gelu_tanh ? ACT_GELU_TANH : ACT_GELU_ERF;
+            absorbed[c] = 1; n.ops.push_back(c); p->folded[n.out] = 1; n.out = g.ops[c].outs[0];
+            c = sole_consumer(n.out);
+          }
+          if (c >= 0 && g.ops[c].kind == FLUID_OP_ADD) {
+            const int other = g.ops[c].ins[0] == n.out ? g.ops[c].ins[1] : g.ops[c].ins[0];
+            if (other != n.out && available_before(other, oi)) {
+              n.res = other;
+              absorbed[c] = 1; n.ops.push_back(c); p->folded[n.out] = 1; n.out = g.ops[c].outs[0];
+            }
+          }
+        }
+        if (fuse && op.kind == FLUID_OP_BMM_QK) {
+          int c = sole_consumer(n.out);
+          if (c >= 0 && g.ops[c].kind == FLUID_OP_SOFTMAX && g.ops[c].attrs.causal &&
+              g.tensors[n.out].dims[2] == g.tensors[n.out].dims[3])
+            n.causal = CAUSAL_SKIP_UPPER;
+        }
+        if (fuse && op.kind == FLUID_OP_BMM_PV) {
+          int pr = producer[n.a];
+          if (pr >= 0 && g.ops[pr].kind == FLUID_OP_SOFTMAX && g.ops[pr].attrs.causal &&
+              g.tensors[n.a].dims[2] == g.tensors[n.a].dims[3])
+            n.causal = CAUSAL_CLIP_K;
+        }
+        break;
+      }
+      case FLUID_OP_ADD:
+      case FLUID_OP_MUL: {
+        n.b = op.ins[1];
+        int c = (fuse && op.kind == FLUID_OP_ADD) ? sole_consumer(n.out) : -1;
+        if (c >= 0 && (g.ops[c].kind == FLUID_OP_LAYERNORM || g.ops[c].kind == FLUID_OP_RMSNORM) &&
+            g.ops[c].ins[0] == n.out && available_before(g.ops[c].ins[1], oi) &&
+            (g.ops[c].ins.size() < 3 || available_before(g.ops[c].ins[2], oi))) {
+          n.kind = N_NORM;
+          n.res = op.ins[1];
+          n.rms = g.ops[c].kind == FLUID_OP_RMSNORM;
+          n.eps = g.ops[c].attrs.eps;
+          n.gamma = g.ops[c].ins[1];
+          n.beta = n.rms ? -1 : g.ops[c].ins[2];
+          absorbed[c] = 1; n.ops.push_back(c); p->folded[n.out] = 1; n.out = g.ops[c].outs[0];
+          n.b = -1;
+        } else {
+          n.kind = N_ELTWISE;
+          n.elt = op.kind == FLUID_OP_ADD ? ELT_ADD : ELT_MUL;
+        }
+        break;
+      }
+      case FLUID_OP_GELU:
+        n.kind = N_ELTWISE; n.elt = op.attrs.gelu_tanh ? ELT_GELU_TANH : ELT_GELU_ERF;
+        break;
+      case FLUID_OP_SILU: {
+        n.kind = N_ELTWISE; n.elt = ELT_SILU;
+        int c = fuse ? sole_consumer(n.out) : -1;
+        if (c >= 0 && g.ops[c].kind == FLUID_OP_MUL) {
+          const int other = g.ops[c].ins[0] == n.out ? g.ops[c].ins[1] : g.ops[c].ins[0];
+          if (other != n.out && available_before(other, oi)) {
+            n.elt = ELT_SILU_MUL; n.b = other;
+            absorbed[c] = 1; n.ops.push_back(c); p->folded[n.out] = 1; n.out = g.ops[c].outs[0];
+          }
+        }
+        break;
+      }
+      case FLUID_OP_SOFTMAX:
+        n.kind = N_SOFTMAX; n.sm_causal = op.attrs.causal; n.scale = op.attrs.scale;
+        break;
+      case FLUID_OP_LAYERNORM:
+      case FLUID_OP_RMSNORM:
+        n.kind = N_NORM; n.rms = op.kind == FLUID_OP_RMSNORM; n.eps = op.attrs.eps;
+        n.gamma = op.ins[1]; n.beta = n.rms ? -1 : op.ins[2];
+        break;
+      case FLUID_OP_ROPE:
+        n.kind = N_ROPE; n.rope_base = op.attrs.rope_base; n.rope_interleaved = op.attrs.rope_interleaved;
+        break;
+      case FLUID_OP_TRANSPOSE:
+        n.kind = N_TRANSPOSE;
+        for (int i = 0; i < 8; ++i) n.perm[i] = op.attrs.perm[i];
+        break;
+      case FLUID_OP_SELECT_LAST_TOKEN:
+        n.kind = N_SELECT;
+        break;
+    }
+    // distinct external inputs in role order
+    auto add_in = [&](int t) {
+      if (t >= 0 && std::find(n.ins.begin(), n.ins.end(), t) == n.ins.end()) n.ins.push_back(t);
+    };
+    if (n.ops.size() == 1) {
+      for (int t : op.ins) add_in(t);
+    } else {
+      add_in(n.a); add_in(n.b); add_in(n.bias); add_in(n.res); add_in(n.gamma); add_in(n.beta); add_in(n.pos);
+    }
+    n.outs.push_back(n.out);
+    for (int o2 : n.ops) p->node_of_op[o2] = (int)p->nodes.size();
+    p->nodes.push_back(n);
+  }
+}
+
+// ---- Algorithms 1 and 2 on the node graph -------------------------------------------------------------
+struct NodeFlow {
+  std::vector<std::vector<int>> pred, succ;  // node indices, pred sorted by anchor op id
+  std::vector<int> anchor;                   // tie-break key: the node's first op id
+};
+
+static NodeFlow make_flow(const fluid_plan_s* p) {
+  NodeFlow f;
+  const int nn = (int)p->nodes.size();
+  std::vector<int> producer(p->graph.tensors.size(), -1);
+  f.pred.resize(nn);
+  f.succ.resize(nn);
+  f.anchor.resize(nn);
+  for (int i = 0; i < nn; ++i) {
+    f.anchor[i] = p->nodes[i].ops[0];
+    for (int t : p->nodes[i].outs) producer[t] = i;
+  }
+  for (int i = 0; i < nn; ++i) {
+    for (int t : p->nodes[i].ins) {
+      int q = producer[t];
+      if (q >= 0 && std::find(f.pred[i].begin(), f.pred[i].end(), q) == f.pred[i].end()) f.pred[i].push_back(q);
+    }
+    std::sort(f.pred[i].begin(), f.pred[i].end(), [&](int x, int y) { return f.anchor[x] < f.anchor[y]; });
+    for (int q : f.pred[i]) f.succ[q].push_back(i);
+  }
+  return f;
+}
+
+// Algorithm 1: longest distances from the sub-flow's sources, then walk back from the farthest node.
+static std::vector<int> find_longest_sequence(const NodeFlow& f, const std::vector<int>& nodes /*linear order*/,
+                                              const std::vector<char>& inside) {
+  std::map<int, int> dist, back;
+  for (int v : nodes) {
+    int best_d = -1, best_p = -1;
+    for (int q : f.pred[v])
+      if (inside[q] && dist[q] > best_d) {
+        best_d = dist[q];
+        best_p = q;
+      }
+    dist[v] = best_p >= 0 ? best_d + 1 : 0;
+    back[v] = best_p;
+  }
+  int end = -1;
+  for (int v : nodes)
+    if (end < 0 || dist[v] > dist[end] || (dist[v] == dist[end] && f.anchor[v] < f.anchor[end])) end = v;
+  std::vector<int> seq;
+  for (int v = end; v >= 0; v = back[v]) seq.push_back(v);
+  std::reverse(seq.begin(), seq.end());
+  return seq;
+}
+
+// Algorithm 2: peel the longest sequence and recurse into each connected component of the rest.
+static void split(const NodeFlow& f, std::vector<int> nodes, std::vector<std::vector<int>>* out) {
+  if (nodes.empty()) return;
+  const int nn = (int)f.pred.size();
+  std::vector<char> inside(nn, 0);
+  for (int v : nodes) inside[v] = 1;
+  std::vector<int> seq = find_longest_sequence(f, nodes, inside);
+  out->push_back(seq);
+  for (int v : seq) inside[v] = 0;
+  std::vector<int> rest;
+  for (int v : nodes)
+    if (inside[v]) rest.push_back(v);
+  std::vector<int> by_anchor = rest;
+  std::sort(by_anchor.begin(), by_anchor.end(), [&](int x, int y) { return f.anchor[x] < f.anchor[y]; });
+  std::vector<char> seen(nn, 0);
+  for (int start : by_anchor) {
+    if (seen[start]) continue;
+    std::vector<int> comp, stack{start};
+    seen[start] = 1;
+    while (!stack.empty()) {
+      int v = stack.back();
+      stack.pop_back();
+      comp.push_back(v);
+      for (int u : f.pred[v])
+        if (inside[u] && !seen[u]) { seen[u] = 1; stack.push_back(u); }
+      for (int u : f.succ[v])
+        if (inside[u] && !seen[u]) { seen[u] = 1; stack.push_back(u); }
+    }
+    std::sort(comp.begin(), comp.end());  // node index order = linear order
+    split(f, comp, out);
+  }
+}
+
+// ---- Eq. 1 / Algorithm 3 ---------------------------------------------------------------------------------
+struct Proposal { int tensor, layout; };
+
+static bool dp_on_sequence(fluid_plan_s* p, Evaluator& ev, const std::vector<int>& seq,
+                           const std::vector<int>& fixed /*per tensor, -1 = free*/, std::vector<Proposal>* props,
+                           double* cost_out = nullptr) {
+  const auto& T = p->graph.tensors;
+  const int n = (int)seq.size();
+  // chain edges e_0 .. e_n
+  std::vector<int> edges(n + 1, -1);
+  for (int t : p->nodes[seq[0]].ins)
+    if (T[t].kind != FLUID_CONST) { edges[0] = t; break; }
+  for (int i = 0; i + 1 < n; ++i) {
+    int best = -1;
+    for (int t : p->nodes[seq[i]].outs)
+      for (int u : p->nodes[seq[i + 1]].ins)
+        if (t == u && (best < 0 || t < best)) best = t;
+    edges[i + 1] = best;
+  }
+  edges[n] = p->nodes[seq[n - 1]].outs[0];
+  auto allowed = [&](int t) {
+    std::vector<int> v;
+    if (t < 0) { v.push_back(0); return v; }
+    if (fixed[t] >= 0) { v.push_back(fixed[t]); return v; }
+    for (int i = 0; i < (int)p->cands[t].size(); ++i) v.push_back(i);
+    return v;
+  };
+  struct Back { int lp = -1; std::vector<int> side_assign; };
+  std::vector<std::map<int, Back>> backs(n);
+  std::vector<std::vector<int>> sides(n);
+  std::map<int, double> prev;
+  for (int l : allowed(edges[0])) prev[l] = 0.0;
+  for (int i = 1; i <= n; ++i) {
+    const int node = seq[i - 1], e_in = edges[i - 1], e_out = edges[i];
+    std::vector<int> tids = node_tensors(p->nodes[node]);
+    std::vector<int>& side = sides[i - 1];
+    for (int t : tids)
+      if (t != e_in && t != e_out) side.push_back(t);
+    std::vector<std::vector<int>> side_opts;
+    for (int s : side) side_opts.push_back(allowed(s));
+    // argument order handed to eval: the node's tensors, inputs then outputs
+    std::vector<int> lidx(tids.size(), 0);
+    auto slot = [&](int t) { return int(std::find(tids.begin(), tids.end(), t) - tids.begin()); };
+    std::map<int, double> cur;
+    for (int l : allowed(e_out)) {
+      double best = kInf;
+      Back arg;
+      for (int lp : allowed(e_in)) {
+        if (std::isinf(prev[lp])) continue;
+        std::vector<int> idx(side.size(), 0);
+        while (true) {
+          for (size_t s = 0; s < side.size(); ++s) lidx[slot(side[s])] = side_opts[s][idx[s]];
+          if (e_in >= 0) lidx[slot(e_in)] = lp;
+          lidx[slot(e_out)] = l;
+          const double c = prev[lp] + ev(node, tids, lidx);
+          if (c < best) {
+            best = c;
+            arg.lp = lp;
+            arg.side_assign.clear();
+            for (size_t s = 0; s < side.size(); ++s) arg.side_assign.push_back(side_opts[s][idx[s]]);
+          }
+          // next combination, last side tensor fastest
+          int s = (int)side.size() - 1;
+          while (s >= 0 && ++idx[s] == (int)side_opts[s].size()) idx[s--] = 0;
+          if (s < 0) break;
+        }
+      }
+      cur[l] = best;
+      backs[i - 1][l] = arg;
+    }
+    prev = cur;
+  }
+  int l = -1;
+  for (auto& kv : prev)
+    if (l < 0 || kv.second < prev[l]) l = kv.first;
+  if (cost_out) *cost_out = l < 0 ? kInf : prev[l];
+  if (l < 0 || std::isinf(prev[l])) return false;
+  props->push_back({edges[n], l});
+  for (int i = n; i >= 1; --i) {
+    const Back& b = backs[i - 1][l];
+    for (size_t s = 0; s < sides[i - 1].size(); ++s) props->push_back({sides[i - 1][s], b.side_assign[s]});
+    if (edges[i - 1] >= 0) props->push_back({edges[i - 1], b.lp});
+    l = b.lp;
+  }
+  return true;
+}
+
+// ---- merge: majority vote, losers re-optimise ------------------------------------------------------------
+static int plan_layouts(fluid_plan_s* p) {
+  const int nt = (int)p->graph.tensors.size();
+  Evaluator ev{p, std::vector<int>(nt, 0)};
+  std::vector<int> canonical(nt, 0);
+  p->canonical_cost = total_cost(p, ev, canonical);
+  p->layout = canonical;
+  p->cost = p->canonical_cost;
+  NodeFlow flow = make_flow(p);
+  std::vector<int> all(p->nodes.size());
+  for (size_t i = 0; i < all.size(); ++i) all[i] = (int)i;
+  p->sequences.clear();
+  split(flow, all, &p->sequences);
+  if (std::isinf(p->canonical_cost)) {
+    set_error("the canonical layout assignment is not executable (an op has no kernel)");
+    return FLUID_EUNSUPPORTED;
+  }
+  if (p->opts.force_canonical) return FLUID_OK;
+  std::vector<int> fixed(nt, -1);
+  std::vector<std::map<int, int>> votes;
+  for (int round = 0; round <= nt + 1; ++round) {
+    votes.assign(nt, {});
+    for (const auto& seq : p->sequences) {
+      std::vector<Proposal> props;
+      if (!dp_on_sequence(p, ev, seq, fixed, &props)) {
+        set_error("no supported layout assignment on a sequence");
+        return FLUID_EUNSUPPORTED;
+      }
+      for (const Proposal& pr : props) votes[pr.tensor][pr.layout]++;
+    }
+    bool conflict = false;
+    for (int t = 0; t < nt; ++t) {
+      if (votes[t].size() <= 1) continue;
+      conflict = true;
+      int top = 0;
+      for (auto& kv : votes[t]) top = std::max(top, kv.second);
+      std::vector<int> tied;
+      for (auto& kv : votes[t])
+        if (kv.second == top) tied.push_back(kv.first);  // ascending layout index
+      if (tied.size() == 1) {
+        fixed[t] = tied[0];
+        continue;
+      }
+      // a tie goes to the layout under which the re-optimised sequences cost least in total
+      int best = -1;
+      double best_cost = 0;
+      for (int l : tied) {
+        std::vector<int> trial = fixed;
+        trial[t] = l;
+        double c = 0;
+        for (const auto& seq : p->sequences) {
+          std::vector<Proposal> scratch;
+          double sc = kInf;
+          dp_on_sequence(p, ev, seq, trial, &scratch, &sc);
+          c += sc;
+        }
+        if (best < 0 || c < best_cost) { best = l; best_cost = c; }
+      }
+      fixed[t] = best;
+    }
+    if (!conflict) break;
+  }
+  std::vector<int> assign(nt, 0);
+  for (int t = 0; t < nt; ++t)
+    if (!votes[t].empty()) assign[t] = votes[t].begin()->first;
+  const double c = total_cost(p, ev, assign);
+  if (c <= p->canonical_cost) {  // never worse than leaving every tensor canonical
+    p->layout = assign;
+    p->cost = c;
+  }
+  return FLUID_OK;
+}
+
+// ---- Algorithm 4: Greedy-by-Size --------------------------------------------------------------------------
+static int64_t round_up(int64_t n, int64_t a) { return (n + a - 1) / a * a; }
+
+static void greedy_by_size(std::vector<ArenaRecord>& recs, int policy, bool no_reuse, size_t* arena_bytes) {
+  std::vector<int> order(recs.size());
+  for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
+  std::sort(order.begin(), order.end(), [&](int x, int y) {
+    if (recs[x].bytes != recs[y].bytes) return recs[x].bytes > recs[y].bytes;
+    if (recs[x].first != recs[y].first) return recs[x].first < recs[y].first;
+    return recs[x].root < recs[y].root;
+  });
+  int64_t arena = FLUID_ARENA_HEADER;
+  std::vector<int> placed;
+  for (int ri : order) {
+    ArenaRecord& r = recs[ri];
+    std::vector<std::pair<int64_t, int64_t>> busy;
+    for (int qi : placed) {
+      const ArenaRecord& q = recs[qi];
+      if (no_reuse || (q.first <= r.last && r.first <= q.last)) busy.push_back({q.offset, q.offset + q.bytes});
+    }
+    std::sort(busy.begin(), busy.end());
+    int64_t cursor = FLUID_ARENA_HEADER, best_off = -1, best_gap = -1;
+    for (auto& b : busy) {
+      const int64_t gap = b.first - cursor;
+      if (gap >= r.bytes) {
+        if (policy == 0) {
+          if (best_off < 0) { best_off = cursor; best_gap = gap; }
+        } else if (best_off < 0 || gap < best_gap) {
+          best_off = cursor; best_gap = gap;
+        }
+      }
+      cursor = std::max(cursor, b.second);
+    }
+    r.offset = best_off >= 0 ? best_off : cursor;
+    arena = std::max(arena, r.offset + r.bytes);
+    placed.push_back(ri);
+  }
+  *arena_bytes = (size_t)arena;
+}
+
+// ---- lowering: nodes -> steps, aliases, lifetimes ----------------------------------------------------------
+static int lower_and_place(fluid_plan_s* p) {
+  const auto& T = p->graph.tensors;
+  const int nt = (int)T.size();
+  p->alias_root.resize(nt);
+  for (int t = 0; t < nt; ++t) p->alias_root[t] = t;
+  p->steps.clear();
+  const int* lo = p->layout.data();
+  Evaluator ev{p, std::vector<int>(nt, 0)};
+  for (int ni = 0; ni < (int)p->nodes.size(); ++ni) {
+    const Node& n = p->nodes[ni];
+    if (n.kind == N_TRANSPOSE && transpose_is_alias(p, n, lo)) {
+      p->alias_root[n.out] = p->alias_root[n.a];
+      continue;
+    }
+    Step s;
+    s.node = ni;
+    std::vector<int> tids = node_tensors(n), l;
+    for (int t : tids) l.push_back(lo[t]);
+    s.cost = ev(ni, tids, l);
+    p->steps.push_back(s);
+  }
+  // lifetimes in step indices, per alias group
+  p->first_step.assign(nt, -1);
+  p->last_step.assign(nt, -1);
+  std::vector<int> gfirst(nt, -1), glast(nt, -1);
+  for (int si = 0; si < (int)p->steps.size(); ++si) {
+    const Node& n = p->nodes[p->steps[si].node];
+    for (int t : n.outs) {
+      int r = p->alias_root[t];
+      if (gfirst[r] < 0) gfirst[r] = si;
+      glast[r] = std::max(glast[r], si);
+    }
+    for (int t : n.ins) {
+      int r = p->alias_root[t];
+      if (gfirst[r] < 0) gfirst[r] = si;  // inputs and constants: alive from first use
+      glast[r] = std::max(glast[r], si);
+    }
+  }
+  for (int t = 0; t < nt; ++t) {
+    p->first_step[t] = gfirst[p->alias_root[t]];
+    p->last_step[t] = glast[p->alias_root[t]];
+  }
+  p->records.clear();
+  p->record_of.assign(nt, -1);
+  for (int t = 0; t < nt; ++t) {
+    if (p->alias_root[t] != t || T[t].kind != FLUID_ACT || p->folded[t] || gfirst[t] < 0) continue;
+    ArenaRecord r;
+    r.root = t;
+    r.bytes = round_up(T[t].numel() * T[t].esize(), FLUID_SLOT_ALIGN);
+    r.first = gfirst[t];
+    r.last = glast[t];
+    p->record_of[t] = (int)p->records.size();
+    p->records.push_back(r);
+  }
+  greedy_by_size(p->records, p->opts.arena_policy, p->opts.no_reuse != 0, &p->arena_bytes);
+  // reference figures: one slice per tensor, and the largest live set
+  int64_t naive = FLUID_ARENA_HEADER, live = 0;
+  for (const ArenaRecord& r : p->records) naive += r.bytes;
+  for (int si = 0; si < (int)p->steps.size(); ++si) {
+    int64_t s = 0;
+    for (const ArenaRecord& r : p->records)
+      if (r.first <= si && si <= r.last) s += r.bytes;
+    live = std::max(live, s);
+  }
+  p->naive_bytes = (size_t)naive;
+  p->live_bound = (size_t)(live + FLUID_ARENA_HEADER);
+  return finalize_steps(p);
+}
+
+}  // namespace fluid
+
+using namespace fluid;
+
+extern "C" {
+
+void fluid_plan_default_options(fluid_plan_options* o) {
+  if (!o) return;
+  std::memset(o, 0, sizeof(*o));
+  o->fusion = 1;
+}
+
+int fluid_plan(const fluid_graph_t* g, const fluid_layout_candidates* cands, const fluid_plan_options* opts,
+               fluid_plan_t** out) {
+  if (!g || !out) {
+    set_error("null argument");
+    return FLUID_EINVAL;
+  }
+  *out = nullptr;
+  if (g->ops.empty()) {
+    set_error("empty graph");
+    return FLUID_EINVAL;
+  }
+  fluid_plan_s* p = new (std::nothrow) fluid_plan_s();
+  if (!p) {
+    set_error("out of host memory");
+    return FLUID_ENOMEM;
+  }
+  p->graph = *g;
+  if (opts) p->opts = *opts;
+  else fluid_plan_default_options(&p->opts);
+  if (p->opts.eval) p->opts.fusion = 0;
+  const int nt = (int)g->tensors.size();
+  // layout candidates
+  p->cands.assign(nt, {});
+  if (cands && cands->n_tensors != nt) {
+    set_error("layout_candidates covers %d tensors, graph has %d", cands->n_tensors, nt);
+    delete p;
+    return FLUID_EINVAL;
+  }
+  size_t cursor = 0;
+  for (int t = 0; t < nt; ++t) {
+    const TensorDesc& td = g->tensors[t];
+    const int nc = cands ? cands->n_cands[t] : 0;
+    if (nc < 0 || nc > 64) {
+      set_error("tensor %d: bad candidate count %d", t, nc);
+      delete p;
+      return FLUID_EINVAL;
+    }
+    for (int c = 0; c < nc; ++c) {
+      Perm pm = identity_perm();
+      int seen = 0;
+      bool ok = true;
+      for (int i = 0; i < td.rank; ++i) {
+        int v = cands->perms[cursor + i];
+        ok = ok && v >= 0 && v < td.rank && !(seen & (1 << v));
+        if (ok) { seen |= 1 << v; pm[i] = (int8_t)v; }
+      }
+      cursor += td.rank;
+      if (ok && c == 0)
+        for (int i = 0; i < td.rank; ++i) ok = ok && pm[i] == i;
+      if (!ok) {
+        set_error("tensor %d: candidate %d is not a permutation (or the first is not the identity)", t, c);
+        delete p;
+        return FLUID_EINVAL;
+      }
+      // the caller's buffers stay canonical whatever the list says
+      if ((td.kind == FLUID_INPUT || td.kind == FLUID_OUTPUT) && c > 0) continue;
+      p->cands[t].push_back(pm);
+    }
+    if (p->cands[t].empty()) p->cands[t].push_back(identity_perm());
+  }
+  // inputs / outputs in declaration order
+  p->input_slot.assign(nt, -1);
+  p->output_slot.assign(nt, -1);
+  p->const_ptr.assign(nt, nullptr);
+  int ni = 0, no = 0;
+  for (int t = 0; t < nt; ++t) {
+    if (g->tensors[t].kind == FLUID_INPUT) p->input_slot[t] = ni++;
+    if (g->tensors[t].kind == FLUID_OUTPUT) p->output_slot[t] = no++;
+  }
+  std::vector<int> order;
+  if (!linearise(p->graph, &order)) {
+    set_error("graph has a cycle");
+    delete p;
+    return FLUID_EINVAL;
+  }
+  build_nodes(p, order);
+  int rc = plan_layouts(p);
+  if (rc == FLUID_OK) rc = lower_and_place(p);
+  if (rc != FLUID_OK) {
+    delete p;
+    return rc;
+  }
+  *out = p;
+  return FLUID_OK;
+}
+
+void fluid_plan_destroy(fluid_plan_t* p) { delete p; }
+
+size_t fluid_plan_arena_bytes(const fluid_plan_t* p) { return p ? p->arena_bytes : 0; }
+size_t fluid_plan_arena_naive_bytes(const fluid_plan_t* p) { return p ? p->naive_bytes : 0; }
+size_t fluid_plan_arena_live_bound_bytes(const fluid_plan_t* p) { return p ? p->live_bound : 0; }
+double fluid_plan_cost(const fluid_plan_t* p) { return p ? p->cost : 0.0; }
+double fluid_plan_canonical_cost(const fluid_plan_t* p) { return p ? p->canonical_cost : 0.0; }
+
+int fluid_plan_tensor_info(const fluid_plan_t* p, int t, int* layout_index, int* perm, int64_t* offset,
+                           int64_t* bytes, int* first_step, int* last_step, int* alias_of) {
+  if (!p || t < 0 || t >= (int)p->graph.tensors.size()) {
+    set_error("bad plan or tensor id");
+    return FLUID_EINVAL;
+  }
+  const TensorDesc& td = p->graph.tensors[t];
+  if (layout_index) *layout_index = p->layout[t];
+  if (perm)
+    for (int i = 0; i < td.rank; ++i) perm[i] = p->cands[t][p->layout[t]][i];
+  const int root = p->alias_root[t];
+  const int rec = p->record_of[root];
+  if (offset) *offset = rec >= 0 ? p->records[rec].offset : -1;
+  if (bytes) *bytes = rec >= 0 ? p->records[rec].bytes : td.numel() * td.esize();
+  if (first_step) *first_step = p->first_step[t];
+  if (last_step) *last_step = p->last_step[t];
+  if (alias_of) *alias_of = root;
+  return FLUID_OK;
+}
+
+int fluid_plan_num_steps(const fluid_plan_t* p) { return p ? (int)p->steps.size() : 0; }
+
+int fluid_plan_step_info(const fluid_plan_t* p, int step, fluid_step_info* info) {
+  if (!p || !info || step < 0 || step >= (int)p->steps.size()) {
+    set_error("bad plan or step index");
+    return FLUID_EINVAL;
+  }
+  const Step& s = p->steps[step];
+  const Node& n = p->nodes[s.node];
+  std::memset(info, 0, sizeof(*info));
+  info->kernel = s.kernel;
+  info->variant = s.variant;
+  info->n_ops = (int)std::min<size_t>(n.ops.size(), 8);
+  for (int i = 0; i < info->n_ops; ++i) info->ops[i] = n.ops[i];
+  info->n_in = (int)std::min<size_t>(n.ins.size(), 8);
+  for (int i = 0; i < info->n_in; ++i) info->in_ids[i] = n.ins[i];
+  info->n_out = (int)std::min<size_t>(n.outs.size(), 4);
+  for (int i = 0; i < info->n_out; ++i) info->out_ids[i] = n.outs[i];
+  info->cost = s.cost;
+  info->flops = s.flops;
+  info->bytes = s.bytes;
+  return FLUID_OK;
+}
+
+int fluid_plan_num_sequences(const fluid_plan_t* p) { return p ? (int)p->sequences.size() : 0; }
+
+int fluid_plan_sequence(const fluid_plan_t* p, int index, int* node_ids, int capacity, int* length) {
+  if (!p || index < 0 || index >= (int)p->sequences.size() || !length) {
+    set_error("bad plan or sequence index");
+    return FLUID_EINVAL;
+  }
+  const auto& s = p->sequences[index];
+  *length = (int)s.size();
+  if (node_ids)
+    for (int i = 0; i < (int)s.size() && i < capacity; ++i) node_ids[i] = p->nodes[s[i]].ops[0];
+  return FLUID_OK;
+}
+
+int fluid_plan_bind_constant(fluid_plan_t* p, int t, const void* dev_ptr) {
+  if (!p || t < 0 || t >= (int)p->graph.tensors.size() || p->graph.tensors[t].kind != FLUID_CONST) {
+    set_error("bind_constant: not a constant tensor");
+    return FLUID_EINVAL;
+  }
+  if (!dev_ptr || (reinterpret_cast<uintptr_t>(dev_ptr) & 15)) {
+    set_error("bind_constant: pointer must be non-null and 16-byte aligned");
+    return FLUID_EALIGN;
+  }
+  std::lock_guard<std::mutex> lk(p->mu);
+  p->const_ptr[t] = dev_ptr;
+  p->maps_valid = false;
+  return FLUID_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,172 @@
+"""Host-side tests of the C-ABI library (no GPU): exports, error paths, and bit-exact agreement of
+the planner (Algorithms 1-4) with the oracle's step-by-step versions."""
+import ctypes
+
+import numpy as np
+import pytest
+
+from oracle import arena as OA
+from oracle import planner as OP
+from paper_2411_09242_b200 import fluid, synth
+from tests.helpers import ensure_lib, header_symbols, plan_records, random_dag, table_eval
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    return ensure_lib()
+
+
+def test_library_exports_every_declared_symbol():
+    L = fluid.lib()
+    names = header_symbols()
+    assert len(names) >= 24 and "fluid_plan" in names and "fluid_run" in names
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(names) == set(fluid._SIGNATURES)
+
+
+def test_graph_error_paths():
+    g = fluid.fluid_graph_create()
+    with pytest.raises(fluid.FluidError) as e:
+        fluid.fluid_graph_add_tensor(g, 7, [4, 4], synth.ACT)
+    assert e.value.code == fluid.FLUID_EINVAL
+    with pytest.raises(fluid.FluidError):
+        fluid.fluid_graph_add_tensor(g, synth.F32, [4, 0], synth.ACT)
+    a = fluid.fluid_graph_add_tensor(g, synth.F32, [4, 8], synth.INPUT)
+    w = fluid.fluid_graph_add_tensor(g, synth.F32, [7, 3], synth.CONST)
+    y = fluid.fluid_graph_add_tensor(g, synth.F32, [4, 3], synth.OUTPUT)
+    with pytest.raises(fluid.FluidError):                   # K mismatch
+        fluid.fluid_graph_add_op(g, synth.LINEAR, [a, w], [y], {"contract": 1})
+    with pytest.raises(fluid.FluidError):                   # bad tensor id
+        fluid.fluid_graph_add_op(g, synth.GELU, [99], [y])
+    with pytest.raises(fluid.FluidError):                   # writing an input
+        fluid.fluid_graph_add_op(g, synth.GELU, [y], [a])
+    with pytest.raises(fluid.FluidError):                   # empty graph
+        fluid.fluid_plan(g)
+    fluid.fluid_graph_destroy(g)
+
+
+def test_bad_candidates_are_rejected():
+    d = random_dag(0, 3)
+    g = fluid.graph_from_desc(d)
+    c = synth.canonical_candidates(d)
+    c[1] = [(1, 0)]                                          # first candidate must be the identity
+    with pytest.raises(fluid.FluidError):
+        fluid.fluid_plan(g, c)
+    c[1] = [(0, 1), (1, 1)]                                  # not a permutation
+    with pytest.raises(fluid.FluidError):
+        fluid.fluid_plan(g, c)
+    fluid.fluid_graph_destroy(g)
+
+
+def _oracle_inputs(d, cands):
+    ops = [{"ins": o["ins"], "outs": o["outs"]} for o in d.ops]
+    ncand = {}
+    for t, td in enumerate(d.tensors):
+        pinned = td["kind"] in (synth.INPUT, synth.OUTPUT)
+        ncand[t] = 1 if pinned else len(cands[t])
+    consts = {t for t, td in enumerate(d.tensors) if td["kind"] == synth.CONST}
+    return ops, ncand, consts
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_sequences_and_layouts_match_the_oracle_bit_for_bit(seed):
+    d = random_dag(seed, n_ops=6 + seed % 7)
+    cands = synth.default_candidates(d)
+    ops, ncand, consts = _oracle_inputs(d, cands)
+    ev = table_eval(seed)
+
+    def c_eval(user, node, n, tids, lidx):
+        return ev(node, {tids[i]: lidx[i] for i in range(n)})
+
+    plan = fluid.Plan(d, cands, eval=fluid.EVAL_FN(c_eval))
+    want, cost, seqs = OP.plan_layouts(ops, ncand, ev, consts)
+    assert plan.sequences() == seqs
+    got = {t: plan.tensor_info(t).layout_index for t in range(len(d.tensors))}
+    assert got == want
+    assert plan.cost == cost
+    assert plan.canonical_cost == OP.total_cost(ops, {t: 0 for t in ncand}, ev)
+    plan.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "bert_base", "gpt2_small", "llama"])
+def test_model_graph_sequences_match_oracle(name):
+    m = synth.build_model(synth.scaled(synth.CONFIGS[name], L=2), materialize=False)
+    d = m.graph
+    plan = fluid.Plan(d, synth.canonical_candidates(d), fusion=0)
+    ops, _, consts = _oracle_inputs(d, synth.canonical_candidates(d))
+    seqs = OP.split(OP.Flow(ops, consts))
+    assert plan.sequences() == seqs
+    assert sorted(o for s in seqs for o in s) == list(range(len(d.ops)))
+    plan.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "bert_base", "gpt2_small", "llama"])
+@pytest.mark.parametrize("policy", [0, 1])
+def test_arena_matches_greedy_by_size_oracle(name, policy):
+    cfg = synth.CONFIGS[name]
+    m = synth.build_model(synth.scaled(cfg, L=min(cfg.L, 3)), materialize=False)
+    plan = fluid.Plan(m.graph, synth.default_candidates(m.graph), arena_policy=policy)
+    recs, offs = plan_records(plan)
+    assert len(recs) > 5
+    want, peak = OA.greedy_by_size(recs, policy="best" if policy else "first")
+    assert offs == want and plan.arena_bytes == peak
+    assert OA.check_arena(recs, offs, plan.arena_bytes) == []
+    assert plan.live_bound_bytes == OA.live_set_bound(recs)
+    assert plan.naive_bytes == OA.naive_sum(recs)
+    assert plan.live_bound_bytes <= plan.arena_bytes <= plan.naive_bytes
+    # lifetimes recomputed independently from the step list
+    steps = plan.steps()
+    for tid, _, first, last in recs:
+        group = [t for t in range(len(m.graph.tensors)) if plan.tensor_info(t).alias_of == tid]
+        touched = [i for i, s in enumerate(steps) if set(group) & set(s["ins"] + s["outs"])]
+        assert (first, last) == (min(touched), max(touched))
+    plan.close()
+
+
+def test_no_reuse_plan_is_the_naive_sum():
+    m = synth.build_model(synth.CONFIGS["tiny"], materialize=False)
+    plan = fluid.Plan(m.graph, None, no_reuse=1)
+    recs, offs = plan_records(plan)
+    assert plan.arena_bytes == plan.naive_bytes == OA.naive_sum(recs)
+    spans = sorted((offs[r[0]], offs[r[0]] + r[1]) for r in recs)
+    assert all(a[1] <= b[0] for a, b in zip(spans, spans[1:]))
+    plan.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "bert_base", "gpt2_small", "llama"])
+def test_planned_layouts_elide_every_transpose(name):
+    cfg = synth.CONFIGS[name]
+    m = synth.build_model(synth.scaled(cfg, L=2), materialize=False)
+    d = m.graph
+    cands = synth.default_candidates(d)
+    plan = fluid.Plan(d, cands)
+    canon = fluid.Plan(d, None)
+    assert plan.cost <= plan.canonical_cost == pytest.approx(canon.cost)
+    kinds = [s["kernel_name"] for s in plan.steps()]
+    assert "PERMUTE" not in kinds
+    assert [s["kernel_name"] for s in canon.steps()].count("PERMUTE") == 4 * 2 + (0 if name != "gpt2_small" else 1)
+    for t in range(len(d.tensors)):
+        info = plan.tensor_info(t)
+        assert info.perm in [tuple(c) for c in cands[t]]
+        if d.tensors[t]["kind"] in (synth.INPUT, synth.OUTPUT):
+            assert info.layout_index == 0
+    # every op of the graph is covered by exactly one step or is an elided transpose
+    covered = sorted(o for s in plan.steps() for o in s["ops"])
+    elided = [i for i, o in enumerate(d.ops) if o["kind"] == synth.TRANSPOSE]
+    assert sorted(covered + elided) == list(range(len(d.ops)))
+    assert plan.arena_bytes <= canon.arena_bytes
+    plan.close(); canon.close()
+
+
+def test_fusion_folds_epilogues():
+    m = synth.build_model(synth.scaled(synth.CONFIGS["bert_base"], L=1), materialize=False)
+    fused = fluid.Plan(m.graph, None)
+    plain = fluid.Plan(m.graph, None, fusion=0)
+    assert fluid.fluid_plan_num_steps(plain.handle) == len(m.graph.ops)
+    names = lambda p: [s["kernel_name"] for s in p.steps()]
+    assert names(plain).count("ELTWISE") == 3 and names(fused).count("ELTWISE") == 0
+    gelu_steps = [s for s in fused.steps() if len(s["ops"]) == 3]        # LINEAR + GELU? no: LINEAR+ADD pairs
+    assert all(len(s["ops"]) <= 3 for s in fused.steps())
+    assert fused.arena_bytes <= plain.arena_bytes
+    fused.close(); plain.close()
