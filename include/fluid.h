@@ -112,7 +112,11 @@ typedef struct fluid_plan_options {
   int32_t no_reuse;         /* 1: one private slice per activation (the naive plan) */
   int32_t force_canonical;  /* 1: skip the layout search, every tensor canonical */
   int32_t gemm_path;        /* 0: tensor cores where eligible, 1: SIMT kernel everywhere */
-  int32_t reserved[3];
+  int32_t narrow_stream;    /* bf16 graphs: 0 = activations that only feed normalisations and
+                               residual additions (the residual stream) are held in fp32 inside the
+                               arena, with a bf16 twin where a GEMM also reads them; 1 = every
+                               activation is held in its declared dtype */
+  int32_t reserved[2];
   fluid_eval_fn eval;       /* NULL: built-in analytic B200 cost table */
   void* eval_user;
 } fluid_plan_options;
@@ -172,6 +176,13 @@ FLUID_API double fluid_plan_canonical_cost(const fluid_plan_t* plan);
 FLUID_API int fluid_plan_tensor_info(const fluid_plan_t* plan, int tensor_id, int* layout_index, int* perm,
                            int64_t* offset, int64_t* bytes, int* first_step, int* last_step,
                            int* alias_of);
+/* Arena slices. A tensor held in fp32 with a bf16 twin owns two slices. record_id is unique
+ * (tensor id, or tensor id + number of tensors for a twin); storage_dtype is the fluid_dtype the
+ * slice holds. Any out pointer may be NULL. */
+FLUID_API int fluid_plan_num_records(const fluid_plan_t* plan);
+FLUID_API int fluid_plan_record_info(const fluid_plan_t* plan, int index, int* record_id, int* tensor_id,
+                           int* is_twin, int* storage_dtype, int64_t* offset, int64_t* bytes,
+                           int* first_step, int* last_step);
 FLUID_API int fluid_plan_num_steps(const fluid_plan_t* plan);
 FLUID_API int fluid_plan_step_info(const fluid_plan_t* plan, int step, fluid_step_info* info);
 /* The sequences of Algorithm 2, as node ids (= op ids when fusion is 0). */

@@ -33,6 +33,7 @@ int finalize_steps(fluid_plan_s* p) {
         e.S = (int)ty.dims[1];
         e.H = (int)ty.dims[2];
         e.V = (int)T[n.b].dims[0];
+        e.y_f32 = p->wide[n.out];
         s.embed = e;
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.pos; s.t_ptr[3] = n.out;
         s.bytes = es * ty.numel() * (n.pos >= 0 ? 3.0 : 2.0) + 4.0 * e.tokens;
@@ -48,6 +49,9 @@ int finalize_steps(fluid_plan_s* p) {
         if (s.kernel == FLUID_K_GEMM_TC)
           s.variant = (s.tc.cfg.a_mn_major ? 1 : 0) | (s.tc.cfg.b_mn_major ? 2 : 0) | (s.tc.cfg.bn << 8);
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.out; s.t_ptr[3] = n.bias; s.t_ptr[4] = n.res;
+        s.t_narrow[0] = s.t_narrow[1] = 1;
+        s.gemm.c_f32 = p->wide[n.out];
+        s.gemm.r_f32 = n.res >= 0 ? p->wide[n.res] : 0;
         double fl = 2.0 * double(g.batch) * g.M * double(g.N) * g.K;
         double a = double(g.batch) * g.M * double(g.K), b = double(g.batch) * g.K * double(g.N),
                c = double(g.batch) * g.M * double(g.N);
@@ -69,8 +73,11 @@ int finalize_steps(fluid_plan_s* p) {
         q.rows = int(ty.numel() / q.width);
         q.eps = (float)n.eps;
         q.rms = n.rms;
+        q.x_f32 = p->wide[n.a];
+        q.res_f32 = n.res >= 0 ? p->wide[n.res] : 0;
         s.norm = q;
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.res; s.t_ptr[2] = n.gamma; s.t_ptr[3] = n.beta; s.t_ptr[4] = n.out;
+        s.t_ptr[5] = n.out; s.t_narrow[5] = 1;  // bf16 copy of an fp32-held output, if one is planned
         s.bytes = es * ty.numel() * (n.res >= 0 ? 3.0 : 2.0);
         break;
       }
@@ -84,7 +91,7 @@ int finalize_steps(fluid_plan_s* p) {
         q.scale = (float)n.scale;
         q.causal = n.sm_causal;
         s.softmax = q;
-        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out; s.t_narrow[0] = 1;
         double frac = 1.0;
         if (q.causal) frac = 0.5 * (1.0 + 1.0 / q.n);
         s.bytes = es * ty.numel() * 2.0 * frac;
@@ -104,7 +111,7 @@ int finalize_steps(fluid_plan_s* p) {
         q.base = (float)n.rope_base;
         q.interleaved = n.rope_interleaved;
         s.rope = q;
-        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out; s.t_narrow[0] = 1;
         s.bytes = es * ty.numel() * 2.0;
         break;
       }
@@ -114,6 +121,13 @@ int finalize_steps(fluid_plan_s* p) {
         q.dtype = ty.dtype;
         q.n = ty.numel();
         q.op = n.elt;
+        if (n.elt == ELT_ADD) {  // a residual addition reads and writes the fp32 copies
+          q.a_f32 = p->wide[n.a];
+          q.b_f32 = n.b >= 0 ? p->wide[n.b] : 0;
+        } else {
+          s.t_narrow[0] = s.t_narrow[1] = 1;
+        }
+        q.y_f32 = p->wide[n.out];
         s.elt = q;
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.out;
         s.bytes = es * ty.numel() * (n.b >= 0 ? 3.0 : 2.0);
@@ -136,7 +150,7 @@ int finalize_steps(fluid_plan_s* p) {
           if (j < ty.rank && q.dims[j] > 1 && q.ys[j] == 1) q.y_inner = j;
         }
         s.permute = q;
-        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out; s.t_narrow[0] = 1;
         s.bytes = es * ty.numel() * 2.0;
         break;
       }
@@ -168,9 +182,18 @@ struct Resolver {
   const void* const* inputs;
   void* const* outputs;
   bool ok = true;
-  const void* operator()(int t) {
+  const void* operator()(int t, int narrow = 0) {
     if (t < 0) return nullptr;
     const int r = p->alias_root[t];
+    if (narrow && p->wide[r]) {
+      const int rec = p->twin_record_of[r];
+      if (rec < 0) {
+        set_error("tensor %d has no bf16 copy", r);
+        ok = false;
+        return nullptr;
+      }
+      return arena + p->records[rec].offset;
+    }
     const TensorDesc& td = p->graph.tensors[r];
     switch (td.kind) {
       case FLUID_INPUT: return inputs[p->input_slot[r]];
@@ -228,8 +251,8 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
   if (!p->maps_valid || key != p->bound_key) {
     for (Step& s : p->steps) {
       if (s.kernel != FLUID_K_GEMM_TC) continue;
-      const void* a = R(s.t_ptr[0]);
-      const void* b = R(s.t_ptr[1]);
+      const void* a = R(s.t_ptr[0], 1);
+      const void* b = R(s.t_ptr[1], 1);
       if (!R.ok) return FLUID_EINVAL;
       if (encode_tensor_map(&s.tc.map_a, a, s.tc.a) != 0 || encode_tensor_map(&s.tc.map_b, b, s.tc.b) != 0) {
         set_error("tensor map encoding failed for the step of op %d", p->nodes[s.node].ops[0]);
@@ -267,7 +290,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       case FLUID_K_GEMM_SIMT:
       case FLUID_K_GEMM_TC: {
         GemmParams q = s.gemm;
-        q.A = R(s.t_ptr[0]); q.B = R(s.t_ptr[1]); q.C = const_cast<void*>(R(s.t_ptr[2]));
+        q.A = R(s.t_ptr[0], 1); q.B = R(s.t_ptr[1], 1); q.C = const_cast<void*>(R(s.t_ptr[2]));
         q.bias = R(s.t_ptr[3]); q.R = R(s.t_ptr[4]);
         if (R.ok) err = s.kernel == FLUID_K_GEMM_TC ? launch_gemm_tc(q, s.tc, status, stream) : launch_gemm_simt(q, stream);
         break;
@@ -275,32 +298,44 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       case FLUID_K_NORM: {
         NormParams q = s.norm;
         q.x = R(s.t_ptr[0]); q.res = R(s.t_ptr[1]); q.gamma = R(s.t_ptr[2]); q.beta = R(s.t_ptr[3]);
-        q.y = const_cast<void*>(R(s.t_ptr[4]));
+        {
+          const int out = s.t_ptr[4], root = p->alias_root[out];
+          if (p->wide[root]) {
+            q.y_hi = static_cast<float*>(const_cast<void*>(R(out)));
+            q.y_lo = p->twin_record_of[root] >= 0 ? const_cast<void*>(R(out, 1)) : nullptr;
+          } else if (p->graph.tensors[out].dtype == FLUID_F32) {
+            q.y_hi = nullptr;
+            q.y_lo = const_cast<void*>(R(out));
+          } else {
+            q.y_hi = nullptr;
+            q.y_lo = const_cast<void*>(R(out));
+          }
+        }
         if (R.ok) err = launch_norm(q, stream);
         break;
       }
       case FLUID_K_SOFTMAX: {
         SoftmaxParams q = s.softmax;
-        q.x = R(s.t_ptr[0]); q.y = const_cast<void*>(R(s.t_ptr[1]));
+        q.x = R(s.t_ptr[0], 1); q.y = const_cast<void*>(R(s.t_ptr[1]));
         if (R.ok) err = launch_softmax(q, stream);
         break;
       }
       case FLUID_K_ROPE: {
         RopeParams q = s.rope;
-        q.x = R(s.t_ptr[0]); q.y = const_cast<void*>(R(s.t_ptr[1]));
+        q.x = R(s.t_ptr[0], 1); q.y = const_cast<void*>(R(s.t_ptr[1]));
         if (R.ok) err = launch_rope(q, stream);
         break;
       }
       case FLUID_K_ELTWISE: {
         EltParams q = s.elt;
-        q.a = R(s.t_ptr[0]); q.b = R(s.t_ptr[1]); q.y = const_cast<void*>(R(s.t_ptr[2]));
+        q.a = R(s.t_ptr[0], s.t_narrow[0]); q.b = R(s.t_ptr[1], s.t_narrow[1]); q.y = const_cast<void*>(R(s.t_ptr[2]));
         if (R.ok) err = launch_eltwise(q, stream);
         break;
       }
       case FLUID_K_PERMUTE:
       case FLUID_K_SELECT_LAST: {
         PermuteParams q = s.permute;
-        q.x = R(s.t_ptr[0]); q.y = const_cast<void*>(R(s.t_ptr[1]));
+        q.x = R(s.t_ptr[0], 1); q.y = const_cast<void*>(R(s.t_ptr[1]));
         if (R.ok) err = launch_permute(q, stream);
         break;
       }

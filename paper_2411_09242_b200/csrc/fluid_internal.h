@@ -83,6 +83,7 @@ struct Step {
   EmbedParams embed{};
   // tensor ids whose device addresses fill the payload's pointer slots
   int t_ptr[8] = {-1, -1, -1, -1, -1, -1, -1, -1};
+  int t_narrow[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // 1: bind the bf16 twin of an fp32-held tensor
 };
 
 struct ArenaRecord {
@@ -90,6 +91,8 @@ struct ArenaRecord {
   int64_t bytes = 0;
   int first = 0, last = 0;
   int64_t offset = -1;
+  int id = -1;    // root, or root + number of tensors for a twin
+  int twin = 0;   // 1: the bf16 copy of a tensor whose primary storage is fp32
 };
 
 }  // namespace fluid
@@ -112,6 +115,8 @@ struct fluid_plan_s {
   std::vector<fluid::Step> steps;
   std::vector<fluid::ArenaRecord> records;
   std::vector<int> record_of;                   // per tensor (root): index in records or -1
+  std::vector<int> twin_record_of;              // per tensor: index of its bf16 twin slice or -1
+  std::vector<char> wide;                       // per tensor: 1 = held in fp32 although declared bf16
   std::vector<int> first_step, last_step;       // per tensor
   std::vector<const void*> const_ptr;           // per tensor
   std::vector<int> input_slot, output_slot;     // per tensor: index in inputs/outputs or -1

@@ -65,7 +65,11 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmParams p, int a_k_fa
     __syncthreads();
   }
   T* C = static_cast<T*>(p.C) + cb;
-  const T* R = p.has_res ? static_cast<const T*>(p.R) + split_off(bz, p.B0, p.r_s[0], p.r_s[1]) : nullptr;
+  float* Cf = static_cast<float*>(p.C) + cb;
+  const int64_t rb = p.has_res ? split_off(bz, p.B0, p.r_s[0], p.r_s[1]) : 0;
+  const T* R = p.has_res ? static_cast<const T*>(p.R) + rb : nullptr;
+  const float* Rf = static_cast<const float*>(p.R) + rb;
+  const bool c_wide = p.c_f32 && sizeof(T) == 2, r_wide = p.r_f32 && sizeof(T) == 2;
   const T* bias = static_cast<const T*>(p.bias);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -81,8 +85,13 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmParams p, int a_k_fa
       if (p.has_bias) v += to_f(bias[n]);
       if (p.act == ACT_GELU_ERF) v = gelu_erf(v);
       else if (p.act == ACT_GELU_TANH) v = gelu_tanh(v);
-      if (R) v += to_f(R[rm + split_off(n, p.N0, p.r_s[4], p.r_s[5])]);
-      C[cm + split_off(n, p.N0, p.c_s[4], p.c_s[5])] = from_f<T>(v);
+      if (R) {
+        const int64_t ro = rm + split_off(n, p.N0, p.r_s[4], p.r_s[5]);
+        v += r_wide ? Rf[ro] : to_f(R[ro]);
+      }
+      const int64_t co = cm + split_off(n, p.N0, p.c_s[4], p.c_s[5]);
+      if (c_wide) Cf[co] = v;
+      else C[co] = from_f<T>(v);
     }
   }
 }

@@ -30,6 +30,7 @@ struct GemmParams {
   int64_t b_s[6];      // strides for b1, b0, k1, k0, n1, n0
   int64_t c_s[6];      // strides for b1, b0, m1, m0, n1, n0
   int64_t r_s[6];
+  int c_f32, r_f32;    // bf16 models only: C / R are held in fp32 (residual-stream tensors)
   float scale;
   int act;
   int causal;  // CAUSAL_SKIP_UPPER: tiles with n > m everywhere are not computed;
@@ -73,8 +74,10 @@ struct NormParams {
   const void* res;    // optional second addend (x + res is normalised)
   const void* gamma;
   const void* beta;   // null for RMSNorm
-  void* y;
+  void* y_lo;         // output in the model dtype (may be null when only y_hi is wanted)
+  float* y_hi;        // bf16 models: optional fp32 copy of the output (residual stream)
   int dtype;
+  int x_f32, res_f32; // bf16 models: x / res are held in fp32
   int rows, width;
   float eps;
   int rms;
@@ -107,6 +110,7 @@ struct EltParams {
   const void* b;
   void* y;
   int dtype;
+  int a_f32, b_f32, y_f32;  // bf16 models: operand held in fp32 (residual-stream tensors)
   int64_t n;
   int op;
 };
@@ -130,6 +134,7 @@ struct EmbedParams {
   const void* pos;    // optional [S, H]
   void* y;
   int dtype;
+  int y_f32;          // bf16 models: y is held in fp32
   int tokens, S, H, V;
 };
 

@@ -12,7 +12,7 @@ namespace fluid {
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 // ---- EMBED: y[t, :] = tok[ids[t], :] (+ pos[t % S, :]) -------------------------------------------
-template <typename T, int VEC>
+template <typename T, bool VECTOR>
 __global__ void embed_kernel(EmbedParams p) {
   const int t = blockIdx.x;
   int id = p.ids[t];
@@ -20,7 +20,9 @@ __global__ void embed_kernel(EmbedParams p) {
   const T* tok = static_cast<const T*>(p.tok) + (size_t)id * p.H;
   const T* pos = p.pos ? static_cast<const T*>(p.pos) + (size_t)(t % p.S) * p.H : nullptr;
   T* y = static_cast<T*>(p.y) + (size_t)t * p.H;
-  if (VEC > 1) {
+  float* yf = static_cast<float*>(p.y) + (size_t)t * p.H;
+  const bool wide = p.y_f32 && sizeof(T) == 2;
+  if (VECTOR) {
     constexpr int V = VecOf<T>::N;
     for (int c = threadIdx.x * V; c < p.H; c += blockDim.x * V) {
       float a[V];
@@ -31,13 +33,20 @@ __global__ void embed_kernel(EmbedParams p) {
 #pragma unroll
         for (int i = 0; i < V; ++i) a[i] += b[i];
       }
-      store16(y + c, a);
+      if (wide) {
+#pragma unroll
+        for (int i = 0; i < V; i += 4)
+          *reinterpret_cast<float4*>(yf + c + i) = make_float4(a[i], a[i + 1], a[i + 2], a[i + 3]);
+      } else {
+        store16(y + c, a);
+      }
     }
   } else {
     for (int c = threadIdx.x; c < p.H; c += blockDim.x) {
       float a = to_f(tok[c]);
       if (pos) a += to_f(pos[c]);
-      y[c] = from_f<T>(a);
+      if (wide) yf[c] = a;
+      else y[c] = from_f<T>(a);
     }
   }
 }
@@ -47,8 +56,8 @@ static cudaError_t embed_t(const EmbedParams& p, cudaStream_t st) {
   constexpr int V = VecOf<T>::N;
   const bool vec = p.H % V == 0 && aligned16(p.tok) && aligned16(p.y) && (!p.pos || aligned16(p.pos));
   const int threads = std::min(256, std::max(32, ((p.H / (vec ? V : 1)) + 31) / 32 * 32));
-  if (vec) embed_kernel<T, 2><<<p.tokens, threads, 0, st>>>(p);
-  else embed_kernel<T, 1><<<p.tokens, threads, 0, st>>>(p);
+  if (vec) embed_kernel<T, true><<<p.tokens, threads, 0, st>>>(p);
+  else embed_kernel<T, false><<<p.tokens, threads, 0, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -57,16 +66,34 @@ cudaError_t launch_embed(const EmbedParams& p, cudaStream_t st) {
 }
 
 // ---- NORM: one row per CTA, row cached in registers, two block reductions ------------------------
+// In bf16 models the input, the residual addend and one copy of the output may be fp32: the
+// residual stream is carried in fp32 so that rounding does not pile up layer after layer.
 constexpr int NORM_MAXC = 4;
+
+template <typename T, int V>
+__device__ __forceinline__ void norm_load(const void* base, bool f32, size_t row_off, int c, float (&a)[V]) {
+  if (V == 1) {
+    a[0] = f32 ? static_cast<const float*>(base)[row_off + c] : to_f(static_cast<const T*>(base)[row_off + c]);
+  } else if (f32 || sizeof(T) == 4) {
+    const float* q = static_cast<const float*>(base) + row_off + (size_t)c * V;
+#pragma unroll
+    for (int i = 0; i < V; i += 4) {
+      const float4 f = *reinterpret_cast<const float4*>(q + i);
+      a[i] = f.x; a[i + 1] = f.y; a[i + 2] = f.z; a[i + 3] = f.w;
+    }
+  } else {
+    float t8[VecOf<T>::N];
+    load16(static_cast<const T*>(base) + row_off + (size_t)c * V, t8);
+#pragma unroll
+    for (int i = 0; i < V; ++i) a[i] = t8[i];
+  }
+}
 
 template <typename T, bool VECTOR>
 __global__ void norm_kernel(NormParams p) {
   constexpr int V = VECTOR ? VecOf<T>::N : 1;
   __shared__ float red[32];
-  const size_t row = blockIdx.x;
-  const T* x = static_cast<const T*>(p.x) + row * p.width;
-  const T* r = p.res ? static_cast<const T*>(p.res) + row * p.width : nullptr;
-  T* y = static_cast<T*>(p.y) + row * p.width;
+  const size_t roff = (size_t)blockIdx.x * p.width;
   const T* gamma = static_cast<const T*>(p.gamma);
   const T* beta = static_cast<const T*>(p.beta);
   const int nch = p.width / V;
@@ -76,19 +103,12 @@ __global__ void norm_kernel(NormParams p) {
   for (int j = 0; j < NORM_MAXC; ++j) {
     const int c = threadIdx.x + j * blockDim.x;
     if (c < nch) {
-      if (VECTOR) {
-        float a[VecOf<T>::N];
-        load16(x + c * VecOf<T>::N, a);
-        if (r) {
-          float b[VecOf<T>::N];
-          load16(r + c * VecOf<T>::N, b);
+      norm_load<T, V>(p.x, p.x_f32, roff, c, v[j]);
+      if (p.res) {
+        float b[V];
+        norm_load<T, V>(p.res, p.res_f32, roff, c, b);
 #pragma unroll
-          for (int i = 0; i < V; ++i) a[i] += b[i];
-        }
-#pragma unroll
-        for (int i = 0; i < V; ++i) v[j][i] = a[i];
-      } else {
-        v[j][0] = to_f(x[c]) + (r ? to_f(r[c]) : 0.f);
+        for (int i = 0; i < V; ++i) v[j][i] += b[i];
       }
 #pragma unroll
       for (int i = 0; i < V; ++i) s += p.rms ? v[j][i] * v[j][i] : v[j][i];
@@ -112,19 +132,31 @@ __global__ void norm_kernel(NormParams p) {
     q = block_sum(q, red);
     rstd = rsqrtf(q / p.width + p.eps);
   }
+  T* y_lo = static_cast<T*>(p.y_lo);
 #pragma unroll
   for (int j = 0; j < NORM_MAXC; ++j) {
     const int c = threadIdx.x + j * blockDim.x;
     if (c < nch) {
-      if (VECTOR) {
-        float g[VecOf<T>::N], b[VecOf<T>::N], o[VecOf<T>::N];
-        load16(gamma + c * VecOf<T>::N, g);
-        if (beta) load16(beta + c * VecOf<T>::N, b);
+      float g[V], b[V], o[V];
+      norm_load<T, V>(gamma, false, 0, c, g);
+      if (beta) norm_load<T, V>(beta, false, 0, c, b);
 #pragma unroll
-        for (int i = 0; i < V; ++i) o[i] = (v[j][i] - mean) * rstd * g[i] + (beta ? b[i] : 0.f);
-        store16(y + c * VecOf<T>::N, o);
+      for (int i = 0; i < V; ++i) o[i] = (v[j][i] - mean) * rstd * g[i] + (beta ? b[i] : 0.f);
+      if (VECTOR) {
+        if (y_lo) {
+          float t8[VecOf<T>::N];
+#pragma unroll
+          for (int i = 0; i < V; ++i) t8[i] = o[i];
+          store16(y_lo + roff + (size_t)c * V, t8);
+        }
+        if (p.y_hi) {
+#pragma unroll
+          for (int i = 0; i < V; i += 4)
+            *reinterpret_cast<float4*>(p.y_hi + roff + (size_t)c * V + i) = make_float4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+        }
       } else {
-        y[c] = from_f<T>((v[j][0] - mean) * rstd * to_f(gamma[c]) + (beta ? to_f(beta[c]) : 0.f));
+        if (y_lo) y_lo[roff + c] = from_f<T>(o[0]);
+        if (p.y_hi) p.y_hi[roff + c] = o[0];
       }
     }
   }
@@ -133,8 +165,8 @@ __global__ void norm_kernel(NormParams p) {
 template <typename T>
 static cudaError_t norm_t(const NormParams& p, cudaStream_t st) {
   constexpr int V = VecOf<T>::N;
-  const bool vec = p.width % V == 0 && aligned16(p.x) && aligned16(p.y) && aligned16(p.gamma) &&
-                   (!p.beta || aligned16(p.beta)) && (!p.res || aligned16(p.res));
+  const bool vec = p.width % V == 0 && aligned16(p.x) && (!p.y_lo || aligned16(p.y_lo)) && (!p.y_hi || aligned16(p.y_hi)) &&
+                   aligned16(p.gamma) && (!p.beta || aligned16(p.beta)) && (!p.res || aligned16(p.res));
   const int nch = p.width / (vec ? V : 1);
   int threads = (nch + 31) / 32 * 32;
   threads = std::min(1024, std::max(32, threads));
@@ -310,20 +342,30 @@ __device__ __forceinline__ float elt_apply(int op, float a, float b) {
 template <typename T, bool VECTOR>
 __global__ void eltwise_kernel(EltParams p) {
   constexpr int V = VECTOR ? VecOf<T>::N : 1;
-  const T* a = static_cast<const T*>(p.a);
-  const T* b = static_cast<const T*>(p.b);
   T* y = static_cast<T*>(p.y);
+  float* yf = static_cast<float*>(p.y);
+  const bool y_wide = p.y_f32 && sizeof(T) == 2;
   const int64_t nch = p.n / V;
   for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < nch; c += (int64_t)gridDim.x * blockDim.x) {
-    if (VECTOR) {
-      float va[VecOf<T>::N], vb[VecOf<T>::N];
-      load16(a + c * VecOf<T>::N, va);
-      if (b) load16(b + c * VecOf<T>::N, vb);
+    float va[V], vb[V];
+    norm_load<T, V>(p.a, p.a_f32, (size_t)c * V, 0, va);
+    if (p.b) norm_load<T, V>(p.b, p.b_f32, (size_t)c * V, 0, vb);
 #pragma unroll
-      for (int i = 0; i < V; ++i) va[i] = elt_apply(p.op, va[i], b ? vb[i] : 0.f);
-      store16(y + c * VecOf<T>::N, va);
+    for (int i = 0; i < V; ++i) va[i] = elt_apply(p.op, va[i], p.b ? vb[i] : 0.f);
+    if (VECTOR) {
+      if (y_wide || sizeof(T) == 4) {
+#pragma unroll
+        for (int i = 0; i < V; i += 4)
+          *reinterpret_cast<float4*>(yf + c * V + i) = make_float4(va[i], va[i + 1], va[i + 2], va[i + 3]);
+      } else {
+        float t8[VecOf<T>::N];
+#pragma unroll
+        for (int i = 0; i < V; ++i) t8[i] = va[i];
+        store16(y + c * V, t8);
+      }
     } else {
-      y[c] = from_f<T>(elt_apply(p.op, to_f(a[c]), b ? to_f(b[c]) : 0.f));
+      if (y_wide) yf[c] = va[0];
+      else y[c] = from_f<T>(va[0]);
     }
   }
 }

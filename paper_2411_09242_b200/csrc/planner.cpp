@@ -783,7 +783,7 @@ static void greedy_by_size(std::vector<ArenaRecord>& recs, int policy, bool no_r
   std::sort(order.begin(), order.end(), [&](int x, int y) {
     if (recs[x].bytes != recs[y].bytes) return recs[x].bytes > recs[y].bytes;
     if (recs[x].first != recs[y].first) return recs[x].first < recs[y].first;
-    return recs[x].root < recs[y].root;
+    return recs[x].id < recs[y].id;
   });
   int64_t arena = FLUID_ARENA_HEADER;
   std::vector<int> placed;
@@ -857,17 +857,57 @@ static int lower_and_place(fluid_plan_s* p) {
     p->first_step[t] = gfirst[p->alias_root[t]];
     p->last_step[t] = glast[p->alias_root[t]];
   }
+  // Residual-stream tensors of a bf16 graph are held in fp32: a tensor that feeds a
+  // normalisation or a residual addition and is written by a kernel that can emit fp32. If a GEMM
+  // also reads it as an operand, the producing norm writes a bf16 twin as well.
+  p->wide.assign(nt, 0);
+  std::vector<char> need_twin(nt, 0);
+  if (!p->opts.narrow_stream) {
+    std::vector<int> producer(nt, -1), group(nt, 0), stream_use(nt, 0), operand_use(nt, 0);
+    for (int t = 0; t < nt; ++t) group[p->alias_root[t]]++;
+    for (const Step& s : p->steps) {
+      const Node& n = p->nodes[s.node];
+      producer[n.out] = (n.kind == N_ELTWISE && n.elt != ELT_ADD) ? -2 : n.kind;
+      for (int t : n.ins) {
+        const bool stream = (n.kind == N_NORM && (t == n.a || t == n.res)) || (n.kind == N_GEMM && t == n.res) ||
+                            (n.kind == N_ELTWISE && n.elt == ELT_ADD);
+        const bool also_operand = n.kind == N_GEMM && (t == n.a || t == n.b);
+        if (stream) stream_use[t]++;
+        if (!stream || also_operand) operand_use[t]++;
+      }
+    }
+    for (int t = 0; t < nt; ++t) {
+      if (T[t].dtype != FLUID_BF16 || T[t].kind != FLUID_ACT || p->folded[t] || group[t] != 1 || p->alias_root[t] != t)
+        continue;
+      const int pk = producer[t];
+      const bool can = pk == N_NORM || pk == N_EMBED || pk == N_GEMM || pk == N_ELTWISE;
+      if (!can || stream_use[t] == 0) continue;
+      if (operand_use[t] > 0 && pk != N_NORM) continue;
+      p->wide[t] = 1;
+      need_twin[t] = operand_use[t] > 0;
+    }
+  }
   p->records.clear();
   p->record_of.assign(nt, -1);
+  p->twin_record_of.assign(nt, -1);
   for (int t = 0; t < nt; ++t) {
     if (p->alias_root[t] != t || T[t].kind != FLUID_ACT || p->folded[t] || gfirst[t] < 0) continue;
     ArenaRecord r;
     r.root = t;
-    r.bytes = round_up(T[t].numel() * T[t].esize(), FLUID_SLOT_ALIGN);
+    r.id = t;
+    r.bytes = round_up(T[t].numel() * (p->wide[t] ? 4 : T[t].esize()), FLUID_SLOT_ALIGN);
     r.first = gfirst[t];
     r.last = glast[t];
     p->record_of[t] = (int)p->records.size();
     p->records.push_back(r);
+    if (need_twin[t]) {
+      ArenaRecord w = r;
+      w.id = t + nt;
+      w.twin = 1;
+      w.bytes = round_up(T[t].numel() * T[t].esize(), FLUID_SLOT_ALIGN);
+      p->twin_record_of[t] = (int)p->records.size();
+      p->records.push_back(w);
+    }
   }
   greedy_by_size(p->records, p->opts.arena_policy, p->opts.no_reuse != 0, &p->arena_bytes);
   // reference figures: one slice per tensor, and the largest live set
@@ -1007,6 +1047,26 @@ int fluid_plan_tensor_info(const fluid_plan_t* p, int t, int* layout_index, int*
   if (first_step) *first_step = p->first_step[t];
   if (last_step) *last_step = p->last_step[t];
   if (alias_of) *alias_of = root;
+  return FLUID_OK;
+}
+
+int fluid_plan_num_records(const fluid_plan_t* p) { return p ? (int)p->records.size() : 0; }
+
+int fluid_plan_record_info(const fluid_plan_t* p, int index, int* record_id, int* tensor_id, int* is_twin,
+                           int* storage_dtype, int64_t* offset, int64_t* bytes, int* first_step, int* last_step) {
+  if (!p || index < 0 || index >= (int)p->records.size()) {
+    set_error("bad plan or record index");
+    return FLUID_EINVAL;
+  }
+  const ArenaRecord& r = p->records[index];
+  if (record_id) *record_id = r.id;
+  if (tensor_id) *tensor_id = r.root;
+  if (is_twin) *is_twin = r.twin;
+  if (storage_dtype) *storage_dtype = (p->wide[r.root] && !r.twin) ? FLUID_F32 : p->graph.tensors[r.root].dtype;
+  if (offset) *offset = r.offset;
+  if (bytes) *bytes = r.bytes;
+  if (first_step) *first_step = r.first;
+  if (last_step) *last_step = r.last;
   return FLUID_OK;
 }
 

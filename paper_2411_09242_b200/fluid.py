@@ -48,7 +48,8 @@ EVAL_FN = C.CFUNCTYPE(C.c_double, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.
 
 class PlanOptions(C.Structure):
     _fields_ = [("fusion", C.c_int32), ("arena_policy", C.c_int32), ("no_reuse", C.c_int32),
-                ("force_canonical", C.c_int32), ("gemm_path", C.c_int32), ("reserved", C.c_int32 * 3),
+                ("force_canonical", C.c_int32), ("gemm_path", C.c_int32), ("narrow_stream", C.c_int32),
+                ("reserved", C.c_int32 * 2),
                 ("eval", EVAL_FN), ("eval_user", C.c_void_p)]
 
 
@@ -76,6 +77,9 @@ _SIGNATURES = {
     "fluid_plan_canonical_cost": (C.c_double, [C.c_void_p]),
     "fluid_plan_tensor_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int64),
                                           C.POINTER(C.c_int64), C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int)]),
+    "fluid_plan_num_records": (C.c_int, [C.c_void_p]),
+    "fluid_plan_record_info": (C.c_int, [C.c_void_p, C.c_int] + [C.POINTER(C.c_int)] * 4 + [C.POINTER(C.c_int64)] * 2 +
+                               [C.POINTER(C.c_int)] * 2),
     "fluid_plan_num_steps": (C.c_int, [C.c_void_p]),
     "fluid_plan_step_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(StepInfo)]),
     "fluid_plan_num_sequences": (C.c_int, [C.c_void_p]),
@@ -222,6 +226,19 @@ def fluid_plan_tensor_info(p, tid, rank) -> TensorInfo:
     return TensorInfo(li.value, tuple(perm[:rank]), off.value, by.value, fs.value, ls.value, al.value)
 
 
+def fluid_plan_num_records(p):
+    return lib().fluid_plan_num_records(p)
+
+
+def fluid_plan_record_info(p, index) -> dict:
+    rid, tid, tw, dt, fs, ls = (C.c_int() for _ in range(6))
+    off, by = C.c_int64(), C.c_int64()
+    _check(lib().fluid_plan_record_info(p, index, C.byref(rid), C.byref(tid), C.byref(tw), C.byref(dt),
+                                        C.byref(off), C.byref(by), C.byref(fs), C.byref(ls)))
+    return {"id": rid.value, "tensor": tid.value, "twin": tw.value, "dtype": dt.value, "offset": off.value,
+            "bytes": by.value, "first": fs.value, "last": ls.value}
+
+
 def fluid_plan_num_steps(p):
     return lib().fluid_plan_num_steps(p)
 
@@ -353,6 +370,9 @@ class Plan:
     def tensor_info(self, tid) -> TensorInfo:
         return fluid_plan_tensor_info(self.handle, tid, len(self.desc.tensors[tid]["dims"]))
 
+    def records(self):
+        return [fluid_plan_record_info(self.handle, i) for i in range(fluid_plan_num_records(self.handle))]
+
     def steps(self):
         return [fluid_plan_step_info(self.handle, i) for i in range(fluid_plan_num_steps(self.handle))]
 
@@ -452,9 +472,10 @@ class Runner:
             return self.outputs[desc.outputs.index(tid)].float().cpu().numpy().astype(np.float64)
         if info.offset < 0:
             raise ValueError(f"tensor {tid} is not arena-resident")
+        rec = next(r for r in self.plan.records() if r["tensor"] == info.alias_of and not r["twin"])
         n = int(np.prod(t["dims"]))
-        es = synth.DTYPE_BYTES[t["dtype"]]
+        es = synth.DTYPE_BYTES[rec["dtype"]]
         raw = self.arena[info.offset: info.offset + n * es]
-        flat = raw.view(_TORCH_DTYPE[t["dtype"]]).float().cpu().numpy().astype(np.float64)
+        flat = raw.view(_TORCH_DTYPE[rec["dtype"]]).float().cpu().numpy().astype(np.float64)
         pd = [t["dims"][p] for p in info.perm]
         return np.ascontiguousarray(np.transpose(flat.reshape(pd), np.argsort(info.perm)))

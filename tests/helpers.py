@@ -41,11 +41,9 @@ def random_dag(seed, n_ops=10, dims=(4, 8)):
 def plan_records(plan):
     """(id, bytes, first, last) per arena-resident root tensor, and {id: offset}."""
     recs, offs = [], {}
-    for tid, t in enumerate(plan.desc.tensors):
-        info = plan.tensor_info(tid)
-        if info.offset >= 0 and info.alias_of == tid:
-            recs.append((tid, info.bytes, info.first_step, info.last_step))
-            offs[tid] = info.offset
+    for r in plan.records():
+        recs.append((r["id"], r["bytes"], r["first"], r["last"]))
+        offs[r["id"]] = r["offset"]
     return recs, offs
 
 
@@ -54,3 +52,52 @@ def table_eval(seed, hi=20):
         key = (seed, op) + tuple(sorted(lay.items()))
         return float(np.random.default_rng(abs(hash(key)) % (2 ** 32)).integers(1, hi))
     return ev
+
+
+# ---- GPU-side helpers (imported lazily by the gpu tests) ---------------------------------------
+def run_gpu(desc, feeds, candidates=None, poison=True, **opts):
+    """Plan + run a graph on the GPU through the C-ABI; returns ({output tid: fp64 array}, plan, runner)."""
+    ensure_lib()
+    plan = fluid.Plan(desc, candidates, **opts)
+    consts = {t: a for t, a in feeds.items() if desc.tensors[t]["kind"] == synth.CONST}
+    runner = fluid.Runner(plan, consts, poison=poison)
+    runner.set_inputs([feeds[t] for t in desc.inputs])
+    runner.run()
+    outs = runner.outputs_host()
+    assert runner.status() == 0
+    return dict(zip(desc.outputs, outs)), plan, runner
+
+
+def run_oracle(desc, feeds, keep_all=False):
+    from oracle import graph_exec
+    return graph_exec.run_graph(desc.tensors, desc.ops, feeds, keep_all=keep_all)
+
+
+def tol_for(dtype):
+    """max|err| <= tol * max|ref|: 1e-2 on bf16 paths, 1e-4 on fp32 paths."""
+    return 1e-2 if dtype == synth.BF16 else 1e-4
+
+
+def assert_close(got, ref, dtype, what="", tol=None):
+    tol = tol_for(dtype) if tol is None else tol
+    scale = float(np.max(np.abs(ref))) or 1.0
+    err = float(np.max(np.abs(got - ref)))
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output"
+    assert err <= tol * scale, f"{what}: max|err| {err:.3e} > {tol:g} * max|ref| {scale:.3e}"
+
+
+def single_op_graph(kind, in_shapes, out_shape, dtype, attrs=None, in_kinds=None):
+    g = synth.GraphDesc()
+    ins = []
+    for i, shp in enumerate(in_shapes):
+        k = (in_kinds or {}).get(i, synth.INPUT)
+        dt = synth.I32 if k == "ids" else dtype
+        ins.append(g.tensor(f"in{i}", dt, shp, synth.INPUT if k == "ids" else k))
+    out = g.tensor("out", dtype, out_shape, synth.OUTPUT)
+    g.op(kind, ins, [out], **(attrs or {}))
+    return g
+
+
+def rand_feed(shape, dtype, seed, lo=-1.0, hi=1.0):
+    a = synth.uniform(seed, 0, shape, lo, hi)
+    return synth.round_bf16(a) if dtype == synth.BF16 else a

@@ -1,0 +1,257 @@
+"""Parity of the CUDA path (through the C-ABI) against the fp64 oracle, element by element."""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2411_09242_b200 import fluid, synth
+from tests.helpers import assert_close, rand_feed, run_gpu, run_oracle, single_op_graph, tol_for
+
+pytestmark = pytest.mark.gpu
+
+DT = [synth.F32, synth.BF16]
+
+
+def model_feeds(m):
+    feeds = dict(m.consts)
+    feeds[m.graph.inputs[0]] = m.ids
+    return feeds
+
+
+SMALL = {
+    "encoder": synth.scaled(synth.CONFIGS["bert_base"], L=2, H=256, nh=4, F=512, S=160, B=2, V=1000),
+    "gpt": synth.scaled(synth.CONFIGS["gpt2_small"], L=2, H=256, nh=4, F=512, S=192, B=2, V=1003),
+    "llama": synth.scaled(synth.CONFIGS["llama"], L=2, H=512, nh=4, F=1408, S=256, B=1, V=2000),
+}
+
+
+def test_tiny_fp32_config_end_to_end():
+    m = synth.build_model(synth.CONFIGS["tiny"])
+    ref = run_oracle(m.graph, model_feeds(m))
+    for cands in (None, synth.default_candidates(m.graph)):
+        got, plan, _ = run_gpu(m.graph, model_feeds(m), cands)
+        for t in m.graph.outputs:
+            assert_close(got[t], ref[t], synth.F32, "tiny")
+        plan.close()
+
+
+@pytest.mark.parametrize("family", ["encoder", "gpt", "llama"])
+@pytest.mark.parametrize("dtype", DT)
+def test_small_models_planned_and_canonical(family, dtype):
+    cfg = synth.scaled(SMALL[family], dtype=dtype)
+    m = synth.build_model(cfg)
+    feeds = model_feeds(m)
+    ref = run_oracle(m.graph, feeds)
+    results = {}
+    for label, cands, opts in [("planned", synth.default_candidates(m.graph), {}),
+                               ("canonical", None, {}),
+                               ("unfused", synth.default_candidates(m.graph), {"fusion": 0}),
+                               ("simt", synth.default_candidates(m.graph), {"gemm_path": 1}),
+                               ("no_reuse", synth.default_candidates(m.graph), {"no_reuse": 1})]:
+        got, plan, _ = run_gpu(m.graph, feeds, cands, **opts)
+        for t in m.graph.outputs:
+            assert_close(got[t], ref[t], dtype, f"{family}/{label}")
+        results[label] = got
+        plan.close()
+    # same kernels, different arena offsets: bit-identical outputs
+    for t in m.graph.outputs:
+        assert np.array_equal(results["planned"][t], results["no_reuse"][t])
+
+
+@pytest.mark.parametrize("family", ["gpt", "llama"])
+def test_per_step_parity_localises_drift(family):
+    """Each step's output vs the oracle op applied to the GPU's own inputs of that step."""
+    cfg = synth.scaled(SMALL[family], dtype=synth.BF16, L=1)
+    m = synth.build_model(cfg)
+    feeds = model_feeds(m)
+    got, plan, runner = run_gpu(m.graph, feeds, synth.default_candidates(m.graph), fusion=0, no_reuse=1)
+    from oracle import graph_exec
+    d = m.graph
+    const_derived = run_oracle(d, feeds, keep_all=True)
+    for s in plan.steps():
+        op = d.ops[s["ops"][0]]
+        ins = []
+        for t in op["ins"]:
+            k = d.tensors[t]["kind"]
+            root_kind = d.tensors[plan.tensor_info(t).alias_of]["kind"]
+            if k in (synth.CONST, synth.INPUT):
+                ins.append(feeds[t])
+            elif root_kind == synth.CONST:          # a zero-copy view of a constant
+                ins.append(const_derived[t])
+            else:
+                ins.append(runner.read_tensor(t))
+        want = graph_exec.run_op(op["kind"], [np.asarray(a) if np.asarray(a).dtype.kind in "iu" else np.asarray(a, np.float64) for a in ins], op["attrs"])[0]
+        have = runner.read_tensor(op["outs"][0])
+        if op["kind"] == synth.BMM_QK:          # strictly-upper entries are never read downstream
+            S = want.shape[-1]
+            mask = np.tril(np.ones((S, S), bool))
+            want, have = want * mask, np.where(mask, have, 0.0)
+        assert_close(have, want, synth.BF16, f"{family} step {s['kernel_name']} op {s['ops'][0]}", tol=2 ** -7)
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("M,N,K", [(64, 64, 64), (130, 70, 50), (1, 33, 200), (257, 129, 72), (128, 256, 1024)])
+def test_linear_shapes_with_ragged_tails(dtype, M, N, K):
+    g = single_op_graph(synth.LINEAR, [[M, K], [K, N], [N]], [M, N], dtype, {"contract": 1},
+                        in_kinds={1: synth.CONST, 2: synth.CONST})
+    feeds = {0: rand_feed([M, K], dtype, 1), 1: rand_feed([K, N], dtype, 2), 2: rand_feed([N], dtype, 3)}
+    ref = run_oracle(g, feeds)
+    for cands in (None, synth.default_candidates(g)):
+        got, plan, _ = run_gpu(g, feeds, cands)
+        assert_close(got[3], ref[3], dtype, f"linear {M}x{N}x{K}")
+        plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("a_major", ["row", "col"])
+@pytest.mark.parametrize("b_major", ["row", "col"])
+@pytest.mark.parametrize("n", [96, 256])
+def test_gemm_operand_majors(dtype, a_major, b_major, n):
+    g, arrs = synth.gemm_case(n, n + 64, n + 128, a_major, b_major, dtype=dtype)
+    ref = run_oracle(g, arrs)
+    got, plan, _ = run_gpu(g, arrs, synth.default_candidates(g))
+    assert "PERMUTE" not in [s["kernel_name"] for s in plan.steps()]     # operands read in place
+    assert_close(got[g.outputs[0]], ref[g.outputs[0]], dtype, f"gemm {a_major}/{b_major}")
+    got_c, plan_c, _ = run_gpu(g, arrs, None)                            # canonical: real transposes
+    assert_close(got_c[g.outputs[0]], ref[g.outputs[0]], dtype, "gemm canonical")
+    plan.close(); plan_c.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("causal", [0, 1])
+@pytest.mark.parametrize("n", [1, 7, 128, 200, 1024, 2048, 4100])
+def test_softmax_rows(dtype, causal, n):
+    rows = 3 if not causal else n
+    if causal and n > 1024:
+        pytest.skip("square causal case kept small")
+    shape = [2, rows, n]
+    g = single_op_graph(synth.SOFTMAX, [shape], shape, dtype, {"causal": causal, "scale": 0.5})
+    feeds = {0: rand_feed(shape, dtype, 4, -8.0, 8.0)}
+    ref = run_oracle(g, feeds)[1]
+    got, plan, _ = run_gpu(g, feeds)
+    assert_close(got[1], ref, dtype, f"softmax n={n}")
+    np.testing.assert_allclose(got[1].sum(-1), 1.0, atol=2e-2 if dtype == synth.BF16 else 1e-5)
+    if causal:
+        iu = np.triu_indices(n, 1)
+        assert np.all(got[1][:, iu[0], iu[1]] == 0.0)
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("rows,width", [(5, 128), (33, 768), (4, 4096), (3, 100), (2, 8192)])
+@pytest.mark.parametrize("rms", [0, 1])
+def test_norm_rows(dtype, rows, width, rms):
+    kind = synth.RMSNORM if rms else synth.LAYERNORM
+    shapes = [[1, rows, width], [width]] + ([] if rms else [[width]])
+    g = single_op_graph(kind, shapes, [1, rows, width], dtype, {"eps": 1e-5},
+                        in_kinds={1: synth.CONST, 2: synth.CONST})
+    feeds = {0: rand_feed([1, rows, width], dtype, 5, -3.0, 5.0), 1: rand_feed([width], dtype, 6, 0.5, 1.5)}
+    if not rms:
+        feeds[2] = rand_feed([width], dtype, 7)
+    out = len(shapes)
+    ref = run_oracle(g, feeds)[out]
+    got, plan, _ = run_gpu(g, feeds)
+    assert_close(got[out], ref, dtype, "norm")
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("kind,attrs,nin", [(synth.ADD, {}, 2), (synth.MUL, {}, 2), (synth.GELU, {"gelu_tanh": 0}, 1),
+                                            (synth.GELU, {"gelu_tanh": 1}, 1), (synth.SILU, {}, 1)])
+@pytest.mark.parametrize("shape", [[3, 5, 7], [2, 64, 256]])
+def test_elementwise(dtype, kind, attrs, nin, shape):
+    g = single_op_graph(kind, [shape] * nin, shape, dtype, attrs)
+    feeds = {i: rand_feed(shape, dtype, 8 + i, -4.0, 4.0) for i in range(nin)}
+    ref = run_oracle(g, feeds)[nin]
+    got, plan, _ = run_gpu(g, feeds)
+    assert_close(got[nin], ref, dtype, "eltwise")
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("interleaved", [0, 1])
+def test_rope_in_every_head_layout(dtype, interleaved):
+    B, S, nh, D = 2, 70, 3, 64
+    d = synth.GraphDesc()
+    x = d.tensor("x", dtype, [B, S, nh, D], synth.INPUT)
+    for perm in [(0, 1, 2, 3), (0, 2, 1, 3), (0, 2, 3, 1)]:
+        # force the layout: transpose into it, rope there, transpose back
+        d = synth.GraphDesc()
+        x = d.tensor("x", dtype, [B, S, nh, D], synth.INPUT)
+        a = d.tensor("a", dtype, [B, S, nh, D], synth.ACT)
+        d.op(synth.GELU, [x], [a])          # a producer whose output layout is free
+        r = d.tensor("r", dtype, [B, S, nh, D], synth.ACT)
+        d.op(synth.ROPE, [a], [r], rope_base=10000.0, rope_interleaved=interleaved)
+        y = d.tensor("y", dtype, [B, S, nh, D], synth.OUTPUT)
+        d.op(synth.ADD, [r, r], [y])
+        feeds = {x: rand_feed([B, S, nh, D], dtype, 9)}
+        ref = run_oracle(d, feeds)[y]
+        cands = synth.canonical_candidates(d)
+        got, plan, _ = run_gpu(d, feeds, cands)
+        assert_close(got[y], ref, dtype, "rope canonical")
+        plan.close()
+    # rope directly on tensors held in non-canonical layouts, via a planned attention block
+    cfg = synth.scaled(SMALL["llama"], dtype=dtype, L=1, S=64)
+    m = synth.build_model(cfg)
+    got, plan, _ = run_gpu(m.graph, model_feeds(m), synth.default_candidates(m.graph))
+    ref = run_oracle(m.graph, model_feeds(m))
+    for t in m.graph.outputs:
+        assert_close(got[t], ref[t], dtype, "rope in planned model")
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("case", [dict(B=1, S=128, nh=12, D=64), dict(B=2, S=100, nh=3, D=40), dict(B=3, S=257, nh=2, D=128)])
+@pytest.mark.parametrize("target", ["BHSD", "BHDS"])
+def test_layout_transforms_bit_exact(dtype, case, target):
+    g, a = synth.permute_case(target=target, dtype=dtype, **case)
+    got, plan, _ = run_gpu(g, {0: a})
+    ref = run_oracle(g, {0: a})[1]
+    assert np.array_equal(got[1], ref)            # pure data movement: bit exact
+    assert [s["kernel_name"] for s in plan.steps()] == ["PERMUTE"]
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
+def test_embed_and_select_last(dtype):
+    g = synth.GraphDesc()
+    ids = g.tensor("ids", synth.I32, [3, 17], synth.INPUT)
+    tok = g.tensor("tok", dtype, [50, 96], synth.CONST)
+    pos = g.tensor("pos", dtype, [17, 96], synth.CONST)
+    x = g.tensor("x", dtype, [3, 17, 96], synth.OUTPUT)
+    g.op(synth.EMBED, [ids, tok, pos], [x])
+    last = g.tensor("last", dtype, [3, 96], synth.OUTPUT)
+    g.op(synth.SELECT_LAST_TOKEN, [x], [last])
+    feeds = {ids: synth.token_ids(3, 0, [3, 17], 50), tok: rand_feed([50, 96], dtype, 10), pos: rand_feed([17, 96], dtype, 11)}
+    ref = run_oracle(g, feeds)
+    got, plan, _ = run_gpu(g, feeds)
+    assert_close(got[x], ref[x], dtype, "embed")
+    assert np.array_equal(got[last], got[x][:, -1, :])
+    plan.close()
+
+
+def test_run_allocates_nothing_and_rejects_bad_pointers():
+    import torch
+    m = synth.build_model(synth.CONFIGS["tiny"])
+    plan = fluid.Plan(m.graph, synth.default_candidates(m.graph))
+    r = fluid.Runner(plan, m.consts)
+    r.set_inputs([m.ids])
+    r.run(); torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    before = fluid.fluid_launch_count()
+    for _ in range(5):
+        r.run()
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0                                   # no device allocation inside fluid_run
+    assert fluid.fluid_launch_count() - before == 5 * len(plan.steps())
+    with pytest.raises(fluid.FluidError) as e:              # misaligned arena
+        fluid.fluid_run(plan.handle, r.arena.data_ptr() + 8, [b.data_ptr() for b in r.inputs],
+                        [b.data_ptr() for b in r.outputs])
+    assert e.value.code == fluid.FLUID_EALIGN
+    plan2 = fluid.Plan(m.graph, None)                       # constants not bound
+    with pytest.raises(fluid.FluidError):
+        fluid.fluid_run(plan2.handle, r.arena.data_ptr(), [b.data_ptr() for b in r.inputs],
+                        [b.data_ptr() for b in r.outputs])
+    plan.close(); plan2.close()

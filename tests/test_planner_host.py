@@ -117,8 +117,10 @@ def test_arena_matches_greedy_by_size_oracle(name, policy):
     assert plan.live_bound_bytes <= plan.arena_bytes <= plan.naive_bytes
     # lifetimes recomputed independently from the step list
     steps = plan.steps()
-    for tid, _, first, last in recs:
-        group = [t for t in range(len(m.graph.tensors)) if plan.tensor_info(t).alias_of == tid]
+    nt = len(m.graph.tensors)
+    for rid, _, first, last in recs:
+        tid = rid % nt
+        group = [t for t in range(nt) if plan.tensor_info(t).alias_of == tid]
         touched = [i for i, s in enumerate(steps) if set(group) & set(s["ins"] + s["outs"])]
         assert (first, last) == (min(touched), max(touched))
     plan.close()
