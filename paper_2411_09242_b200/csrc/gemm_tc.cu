@@ -1,18 +1,525 @@
-// Tensor-core GEMM (tcgen05 / TMEM / TMA). Placeholder until the kernel lands: reports itself
-// unavailable so that the planner routes every GEMM to the SIMT kernel.
+// Tensor-core GEMM for sm_100a: TMA-fed shared-memory ring, tcgen05.mma with fp32 accumulators in
+// tensor memory, warp-specialised persistent CTAs (one per SM).
+//
+//   warp 0      TMA producer: one elected thread issues cp.async.bulk.tensor loads of the A and B
+//               tiles of each k-step into a ring of shared-memory stages (mbarrier complete_tx)
+//   warp 1      allocates tensor memory; one elected thread issues tcgen05.mma (128 x BN x 16 per
+//               instruction, four per stage) and commits stage-release / accumulator-ready barriers
+//   warps 2-9   epilogue: tcgen05.ld the accumulator (one row per thread), apply
+//               scale / bias / GELU / residual in fp32, store in whatever layout the plan chose
+//
+// Two accumulators (2 x BN tensor-memory columns) let the epilogue of tile i overlap the MMAs of
+// tile i+1. Operands may be K-major or MN-major in global memory (row-/column-/head-major
+// tensors): the TMA box and the shared-memory matrix descriptor follow the operand's major, so
+// no transpose kernel ever runs. No cluster multicast is used anywhere.
+//
+// Every wait is bounded: a wait that does not complete within about a second records a code in
+// the arena header and the CTA drains and exits; the host reads the code with fluid_status().
+#include <cuda.h>
+
+#include <algorithm>
+#include <cstdio>
+
+#include "device_utils.cuh"
 #include "fluid.h"
 #include "kernels.h"
 
 namespace fluid {
 
-bool tc_kernel_available() { return false; }
+namespace {
 
-int encode_tensor_map(TensorMapStorage*, const void*, const TmaOperand&) { return -1; }
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr uint32_t kATileBytes = BM * BK * 2;
+constexpr long long kWaitCycles = 3000000000LL;  // ~1.5 s at 2 GHz
 
-cudaError_t launch_gemm_tc(const GemmParams&, const GemmTcHost&, uint32_t*, cudaStream_t) {
-  return cudaErrorNotSupported;
+struct TcParams {
+  GemmParams g;
+  GemmTcCfg cfg;
+  int tiles_m, tiles_n;
+  int num_tiles;
+  int tiles_per_batch;
+  uint32_t* status;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete in time (the caller records it and drains).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255) == 0 && clock64() - t0 > kWaitCycles) return false;
+  }
+  return true;
 }
 
-int sm_count() { return 148; }
+// Every tensor map is padded to rank 5 (unit dims), so one instruction form serves all operands.
+__device__ __forceinline__ void tma_load(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                         int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle. K-major: rows of 128 bytes, 8-row groups
+// 1024 bytes apart. MN-major: 64-element chunks of the row index 8192 bytes apart (one chunk =
+// 64 k-rows of 128 bytes), 8-k groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
+  const uint64_t lbo = mn_major ? (8192 >> 4) : 1;
+  const uint64_t sbo = 1024 >> 4;
+  return uint64_t((saddr & 0x3FFFF) >> 4) | (lbo << 16) | (sbo << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
+}
+
+__device__ __forceinline__ uint32_t make_idesc(int bn, int a_mn, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(a_mn) << 15) | (uint32_t(b_mn) << 16) |
+         (uint32_t(bn >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+}
+
+// Tile index -> (batch, m tile, n tile); m runs fastest so that CTAs running together share the
+// B tile. With CAUSAL_SKIP_UPPER only tiles that touch the lower triangle are enumerated.
+__device__ __forceinline__ void decode_tile(const TcParams& p, int tile, int& bz, int& mt, int& nt) {
+  bz = tile / p.tiles_per_batch;
+  int r = tile - bz * p.tiles_per_batch;
+  if (p.g.causal == CAUSAL_SKIP_UPPER) {
+    for (int m = 0; m < p.tiles_m; ++m) {
+      const int nv = min(p.tiles_n, (m * BM + BM - 1) / p.cfg.bn + 1);
+      if (r < nv) { mt = m; nt = r; return; }
+      r -= nv;
+    }
+    mt = 0; nt = 0;
+    return;
+  }
+  nt = r / p.tiles_m;
+  mt = r - nt * p.tiles_m;
+}
+
+__device__ __forceinline__ int k_steps_of(const TcParams& p, int mt) {
+  int kend = p.g.K;
+  if (p.g.causal == CAUSAL_CLIP_K) kend = min(kend, mt * BM + BM);
+  return (kend + BK - 1) / BK;
+}
+
+__device__ __forceinline__ void fill_coords(const int* sel, int rank, int k0, int k1, int r0, int r1, int b0, int b1, int* c) {
+#pragma unroll
+  for (int d = 0; d < 5; ++d) {
+    const int q = sel[d];
+    c[d] = q == 0 ? k0 : q == 1 ? k1 : q == 2 ? r0 : q == 3 ? r1 : q == 4 ? b0 : q == 5 ? b1 : 0;
+  }
+}
+
+__device__ __forceinline__ int64_t split_off(int i, int x0, int64_t s1, int64_t s0) {
+  return (int64_t)(i / x0) * s1 + (int64_t)(i % x0) * s0;
+}
+
+__device__ __forceinline__ float act_apply(int act, float v) {
+  if (act == ACT_GELU_ERF) return gelu_erf(v);
+  if (act == ACT_GELU_TANH) return gelu_tanh(v);
+  return v;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte-swizzle atoms want 1024-byte alignment
+  const int bn = p.cfg.bn, stages = p.cfg.stages;
+  const uint32_t b_tile_bytes = uint32_t(bn) * BK * 2;
+  const uint32_t stage_bytes = kATileBytes + b_tile_bytes;
+  const uint32_t bars = base + uint32_t(stages) * stage_bytes;  // 8-byte barriers after the tiles
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (stages + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * stages + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * stages + 2 + a); };
+  const uint32_t tmem_slot = bars + 8u * (2 * stages + 4);
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
+  volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tmem_cols = uint32_t(2 * bn);  // 128, 256 or 512: a power of two >= 32
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kEpiWarps); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int s = 0, issued = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      const int a_boxes = p.cfg.a_mn_major ? BM / 64 : 1, b_boxes = p.cfg.b_mn_major ? bn / 64 : 1;
+      // which coordinate slots carry the running k split (the rest stay fixed over a tile)
+      int a_kd0 = 0, a_kd1 = -1, b_kd0 = 0, b_kd1 = -1;
+#pragma unroll
+      for (int d = 0; d < 5; ++d) {
+        if (p.cfg.a_sel[d] == 0) a_kd0 = d;
+        if (p.cfg.a_sel[d] == 1) a_kd1 = d;
+        if (p.cfg.b_sel[d] == 0) b_kd0 = d;
+        if (p.cfg.b_sel[d] == 1) b_kd1 = d;
+      }
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+        int bz, mt, nt;
+        decode_tile(p, tile, bz, mt, nt);
+        const int ksteps = k_steps_of(p, mt);
+        int ca[2][5], cb[4][5];  // fully unrolled below: these stay in registers
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          const int m = mt * BM + ch * 64;
+          fill_coords(p.cfg.a_sel, 5, 0, 0, m % p.cfg.a_r0, m / p.cfg.a_r0, bz % p.cfg.a_b0, bz / p.cfg.a_b0, ca[ch]);
+        }
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const int n = nt * bn + ch * 64;
+          fill_coords(p.cfg.b_sel, 5, 0, 0, n % p.cfg.b_r0, n / p.cfg.b_r0, bz % p.cfg.b_b0, bz / p.cfg.b_b0, cb[ch]);
+        }
+        int ak0 = 0, ak1 = 0, bk0 = 0, bk1 = 0;  // running split of the k index for each operand
+        for (int ks = 0; ks < ksteps; ++ks) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u)) { ok = false; break; }
+          const uint32_t fb = full_bar(s);
+          mbar_expect_tx(fb, stage_bytes);
+          const uint32_t sa = base + uint32_t(s) * stage_bytes, sb = sa + kATileBytes;
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) {
+            if (ch < a_boxes) {
+              int c[5];
+#pragma unroll
+              for (int d = 0; d < 5; ++d) c[d] = ca[ch][d] + (d == a_kd0 ? ak0 : 0) + (d == a_kd1 ? ak1 : 0);
+              tma_load(sa + ch * 8192u, &map_a, fb, c[0], c[1], c[2], c[3], c[4]);
+            }
+          }
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            if (ch < b_boxes) {
+              int c[5];
+#pragma unroll
+              for (int d = 0; d < 5; ++d) c[d] = cb[ch][d] + (d == b_kd0 ? bk0 : 0) + (d == b_kd1 ? bk1 : 0);
+              tma_load(sb + ch * 8192u, &map_b, fb, c[0], c[1], c[2], c[3], c[4]);
+            }
+          }
+          ++issued;
+          ak0 += BK; if (ak0 >= p.cfg.a_k0) { ak0 = 0; ++ak1; }
+          bk0 += BK; if (bk0 >= p.cfg.b_k0) { bk0 = 0; ++bk1; }
+          if (++s == stages) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {
+        if (!*abort_flag) atomicOr(p.status, 0x1u);
+        *abort_flag = 1;
+        // let the loads already issued land before this CTA's shared memory is given up
+        const int back = issued < stages ? issued : stages;
+        for (int j = 0; j < back; ++j) {
+          if (--s < 0) { s = stages - 1; ph ^= 1u; }
+          mbar_wait(full_bar(s), ph);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(bn, p.cfg.a_mn_major, p.cfg.b_mn_major);
+      const uint32_t a_step = p.cfg.a_mn_major ? 2048u : 32u, b_step = p.cfg.b_mn_major ? 2048u : 32u;
+      int s = 0, acc = 0;
+      uint32_t ph = 0, acc_ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+        int bz, mt, nt;
+        decode_tile(p, tile, bz, mt, nt);
+        const int ksteps = k_steps_of(p, mt);
+        if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_c = tmem_base + uint32_t(acc * bn);
+        for (int ks = 0; ks < ksteps; ++ks) {
+          if (!mbar_wait(full_bar(s), ph)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + uint32_t(s) * stage_bytes, sb = sa + kATileBytes;
+          const uint64_t ad0 = make_desc(sa, p.cfg.a_mn_major), bd0 = make_desc(sb, p.cfg.b_mn_major);
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk)
+            umma_bf16(tmem_c, ad0 + uint64_t((kk * a_step) >> 4), bd0 + uint64_t((kk * b_step) >> 4), idesc,
+                      (ks > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
+          if (++s == stages) { s = 0; ph ^= 1u; }
+        }
+        if (ok) umma_commit(tfull_bar(acc));  // accumulator complete
+        if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+      }
+      if (!ok) {
+        if (!*abort_flag) atomicOr(p.status, 0x2u);
+        *abort_flag = 1;
+      }
+    }
+  } else {
+    // ---------------- epilogue (warps 2..9) ----------------
+    // Warp w reads tensor-memory lanes 32*(w%4)..+31 (one accumulator row per thread); the two
+    // warps that share a lane quarter split the tile's columns between them.
+    const GemmParams& g = p.g;
+    const int lane_base = (warp & 3) * 32;
+    const int half = (warp - 2) >> 2;
+    const int col_begin = half * (bn / 2), col_end = col_begin + bn / 2;
+    const bool c_wide = g.c_f32 != 0, r_wide = g.r_f32 != 0;
+    const bool n_contig = g.c_s[5] == 1 && (!g.has_res || g.r_s[5] == 1);
+    const bool groups_ok = (g.N0 & 7) == 0;  // an aligned 8-column group never straddles an n split
+    int acc = 0;
+    uint32_t acc_ph = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+      int bz, mt, nt;
+      decode_tile(p, tile, bz, mt, nt);
+      if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
+      tc_fence_after();
+      const int m = mt * BM + lane_base + lane;
+      const bool row_ok = m < g.M;
+      const int64_t cb = split_off(bz, g.B0, g.c_s[0], g.c_s[1]) + (row_ok ? split_off(m, g.M0, g.c_s[2], g.c_s[3]) : 0);
+      const int64_t rb = g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) + (row_ok ? split_off(m, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
+      const int n_tile0 = nt * bn;
+      for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+        if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
+        uint32_t r[32];
+        tmem_ld32(tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn + c0), r);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+        // split of the first column of this chunk; advanced by 8 per group below
+        int n1 = (n_tile0 + c0) / g.N0, n0i = (n_tile0 + c0) - n1 * g.N0;
+#pragma unroll
+        for (int j0 = 0; j0 < 32; j0 += 8) {
+          const int n = n_tile0 + c0 + j0;
+          if (n >= g.N) break;
+          float v[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[j0 + j]) * g.scale;
+          const bool full8 = n + 8 <= g.N && groups_ok;
+          if (g.has_bias) {
+            const __nv_bfloat16* bias = static_cast<const __nv_bfloat16*>(g.bias) + n;
+            if (n + 8 <= g.N && (n & 7) == 0) {
+              float b8[8];
+              load16(bias, b8);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) v[j] += b8[j];
+            } else {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                if (n + j < g.N) v[j] += to_f(bias[j]);
+            }
+          }
+          if (g.act != ACT_NONE) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = act_apply(g.act, v[j]);
+          }
+          if (full8) {
+            const int64_t co = cb + (int64_t)n1 * g.c_s[4] + (int64_t)n0i * g.c_s[5];
+            const int64_t ro = g.has_res ? rb + (int64_t)n1 * g.r_s[4] + (int64_t)n0i * g.r_s[5] : 0;
+            if (n_contig && (co & 7) == 0 && (ro & 7) == 0) {
+              if (g.has_res) {
+                float q[8];
+                if (r_wide) {
+                  const float4 x0 = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + ro);
+                  const float4 x1 = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + ro + 4);
+                  q[0] = x0.x; q[1] = x0.y; q[2] = x0.z; q[3] = x0.w; q[4] = x1.x; q[5] = x1.y; q[6] = x1.z; q[7] = x1.w;
+                } else {
+                  load16(static_cast<const __nv_bfloat16*>(g.R) + ro, q);
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] += q[j];
+              }
+              if (c_wide) {
+                float* C = static_cast<float*>(g.C) + co;
+                *reinterpret_cast<float4*>(C) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4*>(C + 4) = make_float4(v[4], v[5], v[6], v[7]);
+              } else {
+                store16(static_cast<__nv_bfloat16*>(g.C) + co, v);
+              }
+            } else {
+              // same n split for all eight: constant element stride (e.g. row index contiguous)
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                float o = v[j];
+                if (g.has_res) {
+                  const int64_t rj = ro + j * g.r_s[5];
+                  o += r_wide ? static_cast<const float*>(g.R)[rj] : to_f(static_cast<const __nv_bfloat16*>(g.R)[rj]);
+                }
+                const int64_t cj = co + j * g.c_s[5];
+                if (c_wide) static_cast<float*>(g.C)[cj] = o;
+                else static_cast<__nv_bfloat16*>(g.C)[cj] = __float2bfloat16_rn(o);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              if (n + j >= g.N) break;
+              const int64_t cj = cb + split_off(n + j, g.N0, g.c_s[4], g.c_s[5]);
+              float o = v[j];
+              if (g.has_res) {
+                const int64_t rj = rb + split_off(n + j, g.N0, g.r_s[4], g.r_s[5]);
+                o += r_wide ? static_cast<const float*>(g.R)[rj] : to_f(static_cast<const __nv_bfloat16*>(g.R)[rj]);
+              }
+              if (c_wide) static_cast<float*>(g.C)[cj] = o;
+              else static_cast<__nv_bfloat16*>(g.C)[cj] = __float2bfloat16_rn(o);
+            }
+          }
+          n0i += 8;
+          if (n0i >= g.N0) { n0i -= g.N0; ++n1; }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+    }
+    if (!ok && lane == 0) {
+      if (!*abort_flag) atomicOr(p.status, 0x4u);
+      *abort_flag = 1;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+}  // namespace
+
+bool tc_kernel_available() { return true; }
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+int encode_tensor_map(TensorMapStorage* out, const void* base, const TmaOperand& op) {
+  static_assert(sizeof(CUtensorMap) == sizeof(TensorMapStorage), "tensor map size");
+  EncodeTiledFn enc = get_encode();
+  if (!enc || !base || (reinterpret_cast<uintptr_t>(base) & 15)) return -1;
+  cuuint64_t dims[5], strides[4];
+  cuuint32_t box[5], estr[5];
+  for (int d = 0; d < 5; ++d) {  // unit dims pad every map to rank 5
+    const bool real = d < op.rank;
+    dims[d] = real ? op.dims[d] : 1;
+    box[d] = real ? op.box[d] : 1;
+    estr[d] = 1;
+    if (d > 0) strides[d - 1] = (real ? op.strides[d] : 8) * 2;  // bytes
+  }
+  CUresult rc = enc(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5,
+                    const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? 0 : -2;
+}
+
+cudaError_t launch_gemm_tc(const GemmParams& g, const GemmTcHost& tc, uint32_t* status, cudaStream_t stream) {
+  TcParams p;
+  p.g = g;
+  p.cfg = tc.cfg;
+  p.tiles_m = (g.M + BM - 1) / BM;
+  p.tiles_n = (g.N + tc.cfg.bn - 1) / tc.cfg.bn;
+  long long per_batch = (long long)p.tiles_m * p.tiles_n;
+  if (g.causal == CAUSAL_SKIP_UPPER) {
+    per_batch = 0;
+    for (int m = 0; m < p.tiles_m; ++m) per_batch += std::min(p.tiles_n, (m * BM + BM - 1) / tc.cfg.bn + 1);
+  }
+  if (per_batch * g.batch > 0x7fffffffLL) return cudaErrorInvalidValue;
+  p.tiles_per_batch = (int)per_batch;
+  p.num_tiles = (int)(per_batch * g.batch);
+  p.status = status;
+  const size_t smem = size_t(tc.cfg.stages) * (kATileBytes + size_t(tc.cfg.bn) * BK * 2) + 1024 + 8 * (2 * tc.cfg.stages + 4) + 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int grid = std::min(p.num_tiles, sm_count());
+  if (grid <= 0) return cudaSuccess;
+  const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(&tc.map_a);
+  const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(&tc.map_b);
+  gemm_tc_kernel<<<grid, kThreads, smem, stream>>>(*ma, *mb, p);
+  return cudaGetLastError();
+}
 
 }  // namespace fluid

@@ -200,6 +200,7 @@ static bool build_tma_operand(int64_t R, int R0, const int64_t* rs, int64_t K, i
   }
   if (d > 5) return false;
   t.rank = d;
+  for (int q = d; q < 5; ++q) { t.dims[q] = 1; t.strides[q] = 8; t.box[q] = 1; t.sel[q] = 6; }
   // contiguity of the fastest level
   if (t.dims[0] > 1 && t.strides[0] != 1) return false;
   *o = t;
