@@ -145,9 +145,11 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
-def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=None):
+def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=None, overrides=None):
     """Plan, bind and time one model workload; returns a dict of measurements."""
     cfg = synth.CONFIGS[name]
+    if overrides:
+        cfg = synth.scaled(cfg, **overrides)
     m = synth.build_model(cfg)
     cands = synth.default_candidates(m.graph)
     t0 = time.perf_counter()
@@ -253,6 +255,9 @@ def main():
     ap.add_argument("--workload", default="bert_base", choices=list(synth.CONFIGS))
     ap.add_argument("--others", default="tiny,gpt2_small,llama", help="comma list of extra workloads to summarise")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="reduced copy of the workload (profiling captures only)")
+    ap.add_argument("--seq", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0)
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -286,7 +291,9 @@ def main():
 
     barrier()
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    main_res = time_workload(args.workload, args.steps, args.warmup, torch, fluid, peaks, full=True, sampler=sampler)
+    overrides = {k: v for k, v in (("L", args.layers), ("S", args.seq), ("B", args.batch)) if v}
+    main_res = time_workload(args.workload, args.steps, args.warmup, torch, fluid, peaks, full=True, sampler=sampler,
+                             overrides=overrides)
     barrier()
     lat = torch.tensor([main_res["latency_ms"], main_res["e2e_ms"]], device="cuda", dtype=torch.float64)
     if dist:
@@ -297,6 +304,8 @@ def main():
             dist.destroy_process_group()
         return
     cfg = synth.CONFIGS[args.workload]
+    if overrides:
+        cfg = synth.scaled(cfg, **overrides)
     kernels = main_res["kernels"]
     dom_name = max(kernels, key=lambda k: kernels[k]["ms"])
     dom = kernels[dom_name]
@@ -315,7 +324,7 @@ def main():
     if not args.no_cpu_baseline:
         scfg, sample = oracle_sample_config(cfg)
         m = main_res["_model"]
-        if scfg is cfg:
+        if scfg is cfg and not overrides:
             ref, dt = oracle_forward(m)
             outs = main_res["_runner"].outputs_host()
             errs = []

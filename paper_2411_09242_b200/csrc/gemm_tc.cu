@@ -160,12 +160,158 @@ __device__ __forceinline__ int64_t split_off(int i, int x0, int64_t s1, int64_t 
   return (int64_t)(i / x0) * s1 + (int64_t)(i % x0) * s0;
 }
 
-__device__ __forceinline__ float act_apply(int act, float v) {
-  if (act == ACT_GELU_ERF) return gelu_erf(v);
-  if (act == ACT_GELU_TANH) return gelu_tanh(v);
+
+// GELU (erf form) with erf from Abramowitz & Stegun 7.1.26 (|error| < 1.5e-7 before fp32
+// rounding): far below bf16 resolution and a third of the instructions of erff().
+__device__ __forceinline__ float gelu_erf_fast(float x) {
+  const float z = fabsf(x) * 0.70710678118654752f;
+  const float t = __frcp_rn(fmaf(0.3275911f, z, 1.f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float e = poly * t * __expf(-z * z);   // 1 - erf(z)
+  const float half_x = 0.5f * x;
+  return x >= 0.f ? fmaf(-half_x, e, x) : half_x * e;  // x/2 (1 + sign * (1 - e))
+}
+
+template <int ACT>
+__device__ __forceinline__ float act_t(float v) {
+  if (ACT == ACT_GELU_ERF) return gelu_erf_fast(v);
+  if (ACT == ACT_GELU_TANH) return gelu_tanh(v);
   return v;
 }
 
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+
+// Vector epilogue for one 32-column chunk of one accumulator row. Preconditions (checked on the
+// host): the n index is contiguous in C (and R), every 8-column group is 16-byte aligned and
+// never straddles an n split, N is a multiple of 8.
+template <int ACT, bool HAS_RES, bool C_WIDE, bool R_WIDE>
+__device__ __forceinline__ void epilogue_chunk_vec(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb,
+                                                   int64_t rb, int n) {
+  uint32_t r[32];
+  tmem_ld32(taddr, r);
+  // group offsets (an 8-column group shares one n split)
+  int64_t co[4], ro[4];
+  int n1 = n / g.N0, n0i = n - n1 * g.N0;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    co[q] = cb + (int64_t)n1 * g.c_s[4] + n0i;
+    ro[q] = HAS_RES ? rb + (int64_t)n1 * g.r_s[4] + n0i : 0;
+    n0i += 8;
+    if (n0i >= g.N0) { n0i -= g.N0; ++n1; }
+  }
+  // operands that do not depend on the accumulator are fetched while the tensor-memory load flies
+  uint4 bq[4];
+  uint4 rq[HAS_RES ? (R_WIDE ? 8 : 4) : 1];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const bool live = n + 8 * q < g.N;
+    if (g.has_bias) bq[q] = live ? *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(g.bias) + n + 8 * q) : make_uint4(0, 0, 0, 0);
+    if (HAS_RES && row_ok && live) {
+      if (R_WIDE) {
+        rq[2 * q] = *reinterpret_cast<const uint4*>(static_cast<const float*>(g.R) + ro[q]);
+        rq[2 * q + 1] = *reinterpret_cast<const uint4*>(static_cast<const float*>(g.R) + ro[q] + 4);
+      } else {
+        rq[q] = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(g.R) + ro[q]);
+      }
+    }
+  }
+  tmem_ld_wait();
+  if (!row_ok) return;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (n + 8 * q >= g.N) break;
+    float v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[8 * q + j]) * g.scale;
+    if (g.has_bias) {
+      const uint32_t w[4] = {bq[q].x, bq[q].y, bq[q].z, bq[q].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        v[2 * j] += __uint_as_float(w[j] << 16);
+        v[2 * j + 1] += __uint_as_float(w[j] & 0xffff0000u);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = act_t<ACT>(v[j]);
+    if (HAS_RES) {
+      if (R_WIDE) {
+        const uint4 a = rq[2 * q], b = rq[2 * q + 1];
+        v[0] += __uint_as_float(a.x); v[1] += __uint_as_float(a.y); v[2] += __uint_as_float(a.z); v[3] += __uint_as_float(a.w);
+        v[4] += __uint_as_float(b.x); v[5] += __uint_as_float(b.y); v[6] += __uint_as_float(b.z); v[7] += __uint_as_float(b.w);
+      } else {
+        const uint32_t w[4] = {rq[q].x, rq[q].y, rq[q].z, rq[q].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          v[2 * j] += __uint_as_float(w[j] << 16);
+          v[2 * j + 1] += __uint_as_float(w[j] & 0xffff0000u);
+        }
+      }
+    }
+    if (C_WIDE) {
+      float* C = static_cast<float*>(g.C) + co[q];
+      *reinterpret_cast<float4*>(C) = make_float4(v[0], v[1], v[2], v[3]);
+      *reinterpret_cast<float4*>(C + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    } else {
+      store16(static_cast<__nv_bfloat16*>(g.C) + co[q], v);
+    }
+  }
+}
+
+// General epilogue for one 8-column group: any strides, any tails, any storage width.
+__device__ __noinline__ void epilogue_group_any(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb, int64_t rb,
+                                                int n) {
+  uint32_t r[8];
+  tmem_ld8(taddr, r);
+  tmem_ld_wait();
+  if (!row_ok) return;
+  const bool c_wide = g.c_f32 != 0, r_wide = g.r_f32 != 0;
+#pragma unroll 1
+  for (int j = 0; j < 8; ++j) {
+    if (n + j >= g.N) break;
+    float v = __uint_as_float(r[0]) * g.scale;
+#pragma unroll
+    for (int q = 1; q < 8; ++q) v = j == q ? __uint_as_float(r[q]) * g.scale : v;
+    if (g.has_bias) v += to_f(static_cast<const __nv_bfloat16*>(g.bias)[n + j]);
+    v = g.act == ACT_GELU_ERF ? gelu_erf_fast(v) : (g.act == ACT_GELU_TANH ? gelu_tanh(v) : v);
+    if (g.has_res) {
+      const int64_t rj = rb + split_off(n + j, g.N0, g.r_s[4], g.r_s[5]);
+      v += r_wide ? static_cast<const float*>(g.R)[rj] : to_f(static_cast<const __nv_bfloat16*>(g.R)[rj]);
+    }
+    const int64_t cj = cb + split_off(n + j, g.N0, g.c_s[4], g.c_s[5]);
+    if (c_wide) static_cast<float*>(g.C)[cj] = v;
+    else static_cast<__nv_bfloat16*>(g.C)[cj] = __float2bfloat16_rn(v);
+  }
+}
+
+// Epilogue variants (template parameter of the kernel)
+enum EpiKind { EPI_ANY = 0, EPI_PLAIN = 1, EPI_PLAIN_WIDE = 2, EPI_RES = 3, EPI_RES_WIDE = 4, EPI_GELU_ERF = 5, EPI_GELU_TANH = 6 };
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb, int64_t rb, int n) {
+  if (EPI == EPI_PLAIN) epilogue_chunk_vec<ACT_NONE, false, false, false>(g, taddr, row_ok, cb, rb, n);
+  else if (EPI == EPI_PLAIN_WIDE) epilogue_chunk_vec<ACT_NONE, false, true, false>(g, taddr, row_ok, cb, rb, n);
+  else if (EPI == EPI_RES) epilogue_chunk_vec<ACT_NONE, true, false, false>(g, taddr, row_ok, cb, rb, n);
+  else if (EPI == EPI_RES_WIDE) epilogue_chunk_vec<ACT_NONE, true, true, true>(g, taddr, row_ok, cb, rb, n);
+  else if (EPI == EPI_GELU_ERF) epilogue_chunk_vec<ACT_GELU_ERF, false, false, false>(g, taddr, row_ok, cb, rb, n);
+  else if (EPI == EPI_GELU_TANH) epilogue_chunk_vec<ACT_GELU_TANH, false, false, false>(g, taddr, row_ok, cb, rb, n);
+  else {
+#pragma unroll 1
+    for (int q = 0; q < 4; ++q) {
+      if (n + 8 * q >= g.N) break;
+      epilogue_group_any(g, taddr + 8 * q, row_ok, cb, rb, n + 8 * q);
+    }
+  }
+}
+
+template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ TcParams p) {
@@ -319,109 +465,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int lane_base = (warp & 3) * 32;
     const int half = (warp - 2) >> 2;
     const int col_begin = half * (bn / 2), col_end = col_begin + bn / 2;
-    const bool c_wide = g.c_f32 != 0, r_wide = g.r_f32 != 0;
-    const bool n_contig = g.c_s[5] == 1 && (!g.has_res || g.r_s[5] == 1);
-    const bool groups_ok = (g.N0 & 7) == 0;  // an aligned 8-column group never straddles an n split
     int acc = 0;
     uint32_t acc_ph = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
       int bz, mt, nt;
       decode_tile(p, tile, bz, mt, nt);
-      if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
-      tc_fence_after();
       const int m = mt * BM + lane_base + lane;
       const bool row_ok = m < g.M;
       const int64_t cb = split_off(bz, g.B0, g.c_s[0], g.c_s[1]) + (row_ok ? split_off(m, g.M0, g.c_s[2], g.c_s[3]) : 0);
       const int64_t rb = g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) + (row_ok ? split_off(m, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
       const int n_tile0 = nt * bn;
+      if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn);
+#pragma unroll 1
       for (int c0 = col_begin; c0 < col_end; c0 += 32) {
         if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
-        uint32_t r[32];
-        tmem_ld32(tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn + c0), r);
-        tmem_ld_wait();
-        if (!row_ok) continue;
-        // split of the first column of this chunk; advanced by 8 per group below
-        int n1 = (n_tile0 + c0) / g.N0, n0i = (n_tile0 + c0) - n1 * g.N0;
-#pragma unroll
-        for (int j0 = 0; j0 < 32; j0 += 8) {
-          const int n = n_tile0 + c0 + j0;
-          if (n >= g.N) break;
-          float v[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[j0 + j]) * g.scale;
-          const bool full8 = n + 8 <= g.N && groups_ok;
-          if (g.has_bias) {
-            const __nv_bfloat16* bias = static_cast<const __nv_bfloat16*>(g.bias) + n;
-            if (n + 8 <= g.N && (n & 7) == 0) {
-              float b8[8];
-              load16(bias, b8);
-#pragma unroll
-              for (int j = 0; j < 8; ++j) v[j] += b8[j];
-            } else {
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                if (n + j < g.N) v[j] += to_f(bias[j]);
-            }
-          }
-          if (g.act != ACT_NONE) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = act_apply(g.act, v[j]);
-          }
-          if (full8) {
-            const int64_t co = cb + (int64_t)n1 * g.c_s[4] + (int64_t)n0i * g.c_s[5];
-            const int64_t ro = g.has_res ? rb + (int64_t)n1 * g.r_s[4] + (int64_t)n0i * g.r_s[5] : 0;
-            if (n_contig && (co & 7) == 0 && (ro & 7) == 0) {
-              if (g.has_res) {
-                float q[8];
-                if (r_wide) {
-                  const float4 x0 = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + ro);
-                  const float4 x1 = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + ro + 4);
-                  q[0] = x0.x; q[1] = x0.y; q[2] = x0.z; q[3] = x0.w; q[4] = x1.x; q[5] = x1.y; q[6] = x1.z; q[7] = x1.w;
-                } else {
-                  load16(static_cast<const __nv_bfloat16*>(g.R) + ro, q);
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] += q[j];
-              }
-              if (c_wide) {
-                float* C = static_cast<float*>(g.C) + co;
-                *reinterpret_cast<float4*>(C) = make_float4(v[0], v[1], v[2], v[3]);
-                *reinterpret_cast<float4*>(C + 4) = make_float4(v[4], v[5], v[6], v[7]);
-              } else {
-                store16(static_cast<__nv_bfloat16*>(g.C) + co, v);
-              }
-            } else {
-              // same n split for all eight: constant element stride (e.g. row index contiguous)
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                float o = v[j];
-                if (g.has_res) {
-                  const int64_t rj = ro + j * g.r_s[5];
-                  o += r_wide ? static_cast<const float*>(g.R)[rj] : to_f(static_cast<const __nv_bfloat16*>(g.R)[rj]);
-                }
-                const int64_t cj = co + j * g.c_s[5];
-                if (c_wide) static_cast<float*>(g.C)[cj] = o;
-                else static_cast<__nv_bfloat16*>(g.C)[cj] = __float2bfloat16_rn(o);
-              }
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              if (n + j >= g.N) break;
-              const int64_t cj = cb + split_off(n + j, g.N0, g.c_s[4], g.c_s[5]);
-              float o = v[j];
-              if (g.has_res) {
-                const int64_t rj = rb + split_off(n + j, g.N0, g.r_s[4], g.r_s[5]);
-                o += r_wide ? static_cast<const float*>(g.R)[rj] : to_f(static_cast<const __nv_bfloat16*>(g.R)[rj]);
-              }
-              if (c_wide) static_cast<float*>(g.C)[cj] = o;
-              else static_cast<__nv_bfloat16*>(g.C)[cj] = __float2bfloat16_rn(o);
-            }
-          }
-          n0i += 8;
-          if (n0i >= g.N0) { n0i -= g.N0; ++n1; }
-        }
+        epilogue_chunk<EPI>(g, trow + uint32_t(c0), row_ok, cb, rb, n_tile0 + c0);
       }
       tc_fence_before();
       __syncwarp();
@@ -508,17 +569,49 @@ cudaError_t launch_gemm_tc(const GemmParams& g, const GemmTcHost& tc, uint32_t* 
   p.num_tiles = (int)(per_batch * g.batch);
   p.status = status;
   const size_t smem = size_t(tc.cfg.stages) * (kATileBytes + size_t(tc.cfg.bn) * BK * 2) + 1024 + 8 * (2 * tc.cfg.stages + 4) + 16;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
   const int grid = std::min(p.num_tiles, sm_count());
   if (grid <= 0) return cudaSuccess;
   const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(&tc.map_a);
   const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(&tc.map_b);
-  gemm_tc_kernel<<<grid, kThreads, smem, stream>>>(*ma, *mb, p);
+  // The vector epilogues need: n contiguous in C (and R), 8-column groups aligned to 16 bytes and
+  // inside one n split, N a multiple of 8. Everything else takes the general epilogue.
+  auto mult8 = [](int64_t v) { return (v & 7) == 0; };
+  bool vec = g.c_s[5] == 1 && (g.N & 7) == 0 && (g.N0 & 7) == 0 && mult8(g.c_s[0]) && mult8(g.c_s[1]) && mult8(g.c_s[2]) &&
+             mult8(g.c_s[3]) && mult8(g.c_s[4]) && (reinterpret_cast<uintptr_t>(g.C) & 15) == 0 &&
+             (!g.has_bias || (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0);
+  if (g.has_res)
+    vec = vec && g.r_s[5] == 1 && mult8(g.r_s[0]) && mult8(g.r_s[1]) && mult8(g.r_s[2]) && mult8(g.r_s[3]) &&
+          mult8(g.r_s[4]) && (reinterpret_cast<uintptr_t>(g.R) & 15) == 0;
+  int epi = EPI_ANY;
+  if (vec) {
+    if (g.act == ACT_NONE && !g.has_res) epi = g.c_f32 ? EPI_PLAIN_WIDE : EPI_PLAIN;
+    else if (g.act == ACT_NONE && g.has_res && !g.c_f32 && !g.r_f32) epi = EPI_RES;
+    else if (g.act == ACT_NONE && g.has_res && g.c_f32 && g.r_f32) epi = EPI_RES_WIDE;
+    else if (g.act == ACT_GELU_ERF && !g.has_res && !g.c_f32) epi = EPI_GELU_ERF;
+    else if (g.act == ACT_GELU_TANH && !g.has_res && !g.c_f32) epi = EPI_GELU_TANH;
+  }
+  static bool attr_set[7] = {false, false, false, false, false, false, false};
+#define FLUID_TC_LAUNCH(E)                                                                                           \
+  case E: {                                                                                                          \
+    if (!attr_set[E]) {                                                                                              \
+      cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); \
+      if (e != cudaSuccess) return e;                                                                                \
+      attr_set[E] = true;                                                                                            \
+    }                                                                                                                \
+    gemm_tc_kernel<E><<<grid, kThreads, smem, stream>>>(*ma, *mb, p);                                                \
+    break;                                                                                                           \
+  }
+  switch (epi) {
+    FLUID_TC_LAUNCH(EPI_PLAIN)
+    FLUID_TC_LAUNCH(EPI_PLAIN_WIDE)
+    FLUID_TC_LAUNCH(EPI_RES)
+    FLUID_TC_LAUNCH(EPI_RES_WIDE)
+    FLUID_TC_LAUNCH(EPI_GELU_ERF)
+    FLUID_TC_LAUNCH(EPI_GELU_TANH)
+    default:
+      FLUID_TC_LAUNCH(EPI_ANY)
+  }
+#undef FLUID_TC_LAUNCH
   return cudaGetLastError();
 }
 

@@ -283,8 +283,9 @@ double node_cost(const fluid_plan_s* p, const Node& n, const int* lo) {
       const double fl = gemm_flops(g), by = gemm_bytes(g);
       if (gemm_tc_eligible(p, g, &tc)) {
         const double skew = 1.0 + 0.02 * (tc.cfg.a_mn_major + tc.cfg.b_mn_major);
-        const bool c_fast = g.c_s[5] == 1 || g.c_s[3] == 1;
-        return kLaunch + std::max(fl / kTcPeak, by / kBw) * skew * (c_fast ? 1.0 : 1.5);
+        // the vector epilogue wants the n index contiguous in C; anything else stores element-wise
+        const double c_pen = g.c_s[5] == 1 ? 1.0 : (g.c_s[3] == 1 ? 1.3 : 1.6);
+        return kLaunch + std::max(fl / kTcPeak, by / kBw) * skew * c_pen;
       }
       const bool a_fast = g.a_s[5] == 1 || g.a_s[3] == 1, b_fast = g.b_s[5] == 1 || g.b_s[3] == 1,
                  c_fast = g.c_s[5] == 1 || g.c_s[3] == 1;
