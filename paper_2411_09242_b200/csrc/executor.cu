@@ -63,6 +63,20 @@ int finalize_steps(fluid_plan_s* p) {
         }
         s.flops = fl;
         s.bytes = es * (a + b + c * (g.has_res ? 2.0 : 1.0) + (g.has_bias ? g.N : 0));
+        // grouped siblings: same A, own B / C / bias
+        for (size_t gi = 1; gi < s.nodes.size(); ++gi) {
+          const Node& m = p->nodes[s.nodes[gi]];
+          GemmParams& gx = s.gemm_x[gi - 1];
+          if (!lower_gemm(p, m, lo, &gx) || !gemm_tc_eligible(p, gx, &s.tc_x[gi - 1]) || s.kernel != FLUID_K_GEMM_TC) {
+            set_error("step for op %d: sibling GEMM cannot share a launch", m.ops[0]);
+            return FLUID_EUNSUPPORTED;
+          }
+          gx.c_f32 = p->wide[m.out];
+          s.x_ptr[gi - 1][0] = m.b; s.x_ptr[gi - 1][1] = m.out; s.x_ptr[gi - 1][2] = m.bias;
+          s.flops += fl;
+          s.bytes += es * (b + c + (g.has_bias ? g.N : 0));
+        }
+        if (s.nodes.size() > 1) s.variant |= int(s.nodes.size()) << 20;
         break;
       }
       case N_NORM: {
@@ -254,7 +268,13 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       const void* a = R(s.t_ptr[0], 1);
       const void* b = R(s.t_ptr[1], 1);
       if (!R.ok) return FLUID_EINVAL;
-      if (encode_tensor_map(&s.tc.map_a, a, s.tc.a) != 0 || encode_tensor_map(&s.tc.map_b, b, s.tc.b) != 0) {
+      bool enc_ok = encode_tensor_map(&s.tc.map_a, a, s.tc.a) == 0 && encode_tensor_map(&s.tc.map_b, b, s.tc.b) == 0;
+      for (size_t gi = 1; enc_ok && gi < s.nodes.size(); ++gi) {
+        const void* bx = R(s.x_ptr[gi - 1][0], 1);
+        if (!R.ok) return FLUID_EINVAL;
+        enc_ok = encode_tensor_map(&s.tc_x[gi - 1].map_b, bx, s.tc_x[gi - 1].b) == 0;
+      }
+      if (!enc_ok) {
         set_error("tensor map encoding failed for the step of op %d", p->nodes[s.node].ops[0]);
         return FLUID_ECUDA;
       }
@@ -292,7 +312,21 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
         GemmParams q = s.gemm;
         q.A = R(s.t_ptr[0], 1); q.B = R(s.t_ptr[1], 1); q.C = const_cast<void*>(R(s.t_ptr[2]));
         q.bias = R(s.t_ptr[3]); q.R = R(s.t_ptr[4]);
-        if (R.ok) err = s.kernel == FLUID_K_GEMM_TC ? launch_gemm_tc(q, s.tc, status, stream) : launch_gemm_simt(q, stream);
+        if (s.kernel == FLUID_K_GEMM_TC) {
+          GemmParams gs[3] = {q, s.gemm_x[0], s.gemm_x[1]};
+          GemmTcHost ts[3] = {s.tc, s.tc_x[0], s.tc_x[1]};
+          const int ng = (int)s.nodes.size();
+          for (int gi = 1; gi < ng; ++gi) {
+            gs[gi].A = q.A;
+            gs[gi].B = R(s.x_ptr[gi - 1][0], 1);
+            gs[gi].C = const_cast<void*>(R(s.x_ptr[gi - 1][1]));
+            gs[gi].bias = R(s.x_ptr[gi - 1][2]);
+            gs[gi].R = nullptr;
+          }
+          if (R.ok) err = launch_gemm_tc(gs, ts, ng, status, stream);
+        } else if (R.ok) {
+          err = launch_gemm_simt(q, stream);
+        }
         break;
       }
       case FLUID_K_NORM: {

@@ -70,11 +70,15 @@ struct Node {
 struct Step {
   int kernel = 0;
   int variant = 0;
-  int node = -1;
+  int node = -1;            // first (or only) planning node of this step
+  std::vector<int> nodes;   // all nodes run by this step (grouped sibling GEMMs: up to 3)
   double cost = 0, flops = 0, bytes = 0;
   // launch payloads (one of these is used, by kernel id)
   GemmParams gemm{};
   GemmTcHost tc{};
+  GemmParams gemm_x[2]{};   // groups 1 and 2 of a grouped GEMM step
+  GemmTcHost tc_x[2]{};
+  int x_ptr[2][3] = {{-1, -1, -1}, {-1, -1, -1}};  // tensor ids of B, C, bias for groups 1 and 2
   NormParams norm{};
   SoftmaxParams softmax{};
   RopeParams rope{};

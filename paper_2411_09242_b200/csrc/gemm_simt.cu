@@ -9,12 +9,17 @@ namespace fluid {
 
 constexpr int BM = 64, BN = 64, BK = 16;
 
+// offset of index i split as (i / x0, i % x0); no division in the common merged case (x0 > i)
 __device__ __forceinline__ int64_t split_off(int i, int x0, int64_t s1, int64_t s0) {
-  return (int64_t)(i / x0) * s1 + (int64_t)(i % x0) * s0;
+  if (i < x0) return (int64_t)i * s0;
+  const int hi = i / x0;
+  return (int64_t)hi * s1 + (int64_t)(i - hi * x0) * s0;
 }
 
 template <typename T>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmParams p, int a_k_fast, int b_n_fast) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float As[BK][BM + 4];
   __shared__ float Bs[BK][BN + 4];
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN, bz = blockIdx.z;
@@ -28,28 +33,42 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmParams p, int a_k_fa
   const T* B = static_cast<const T*>(p.B) + bb;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   float acc[4][4] = {};
+  // the row / column part of each thread's four A and four B elements does not change over k
+  int ar[4], akk[4], bc[4], bkk[4];
+  int64_t a_row[4], b_col[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int e = tid + 256 * j;
+    ar[j] = a_k_fast ? e / BK : e % BM;
+    akk[j] = a_k_fast ? e % BK : e / BM;
+    bc[j] = b_n_fast ? e % BN : e / BK;
+    bkk[j] = b_n_fast ? e / BN : e % BK;
+    a_row[j] = m0 + ar[j] < p.M ? split_off(m0 + ar[j], p.M0, p.a_s[2], p.a_s[3]) : -1;
+    b_col[j] = n0 + bc[j] < p.N ? split_off(n0 + bc[j], p.N0, p.b_s[4], p.b_s[5]) : -1;
+  }
+  // global -> registers -> shared, with the next k-slab's loads in flight during the FFMA loop
+  float va[4], vb[4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int k = k0 + akk[j];
+      va[j] = (a_row[j] >= 0 && k < kend) ? to_f(__ldg(A + a_row[j] + split_off(k, p.K0, p.a_s[4], p.a_s[5]))) : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int k = k0 + bkk[j];
+      vb[j] = (b_col[j] >= 0 && k < kend) ? to_f(__ldg(B + split_off(k, p.K0, p.b_s[2], p.b_s[3]) + b_col[j])) : 0.f;
+    }
+  };
+  fetch(0);
   for (int k0 = 0; k0 < kend; k0 += BK) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int e = tid + 256 * j;
-      const int r = a_k_fast ? e / BK : e % BM, kk = a_k_fast ? e % BK : e / BM;
-      const int m = m0 + r, k = k0 + kk;
-      float v = 0.f;
-      if (m < p.M && k < kend)
-        v = to_f(A[split_off(m, p.M0, p.a_s[2], p.a_s[3]) + split_off(k, p.K0, p.a_s[4], p.a_s[5])]);
-      As[kk][r] = v;
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int e = tid + 256 * j;
-      const int c = b_n_fast ? e % BN : e / BK, kk = b_n_fast ? e / BN : e % BK;
-      const int n = n0 + c, k = k0 + kk;
-      float v = 0.f;
-      if (n < p.N && k < kend)
-        v = to_f(B[split_off(k, p.K0, p.b_s[2], p.b_s[3]) + split_off(n, p.N0, p.b_s[4], p.b_s[5])]);
-      Bs[kk][c] = v;
+      As[akk[j]][ar[j]] = va[j];
+      Bs[bkk[j]][bc[j]] = vb[j];
     }
     __syncthreads();
+    if (k0 + BK < kend) fetch(k0 + BK);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
       float a[4], b[4];
@@ -100,9 +119,8 @@ cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t st) {
   dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, p.batch);
   const int a_k_fast = p.a_s[5] == 1 || p.a_s[3] != 1;
   const int b_n_fast = p.b_s[5] == 1 || p.b_s[3] != 1;
-  if (p.dtype == FLUID_BF16) gemm_simt_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(p, a_k_fast, b_n_fast);
-  else gemm_simt_kernel<float><<<grid, 256, 0, st>>>(p, a_k_fast, b_n_fast);
-  return cudaGetLastError();
+  return p.dtype == FLUID_BF16 ? launch_k(gemm_simt_kernel<__nv_bfloat16>, grid, 256, 0, st, p, a_k_fast, b_n_fast)
+                               : launch_k(gemm_simt_kernel<float>, grid, 256, 0, st, p, a_k_fast, b_n_fast);
 }
 
 }  // namespace fluid

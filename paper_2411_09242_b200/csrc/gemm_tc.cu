@@ -36,7 +36,10 @@ constexpr uint32_t kATileBytes = BM * BK * 2;
 constexpr long long kWaitCycles = 3000000000LL;  // ~1.5 s at 2 GHz
 
 struct TcParams {
-  GemmParams g;
+  GemmParams g;      // group 0 (shapes, A strides, flags are common to all groups)
+  GemmParams gx[2];  // groups 1, 2: own B, C, bias and C strides
+  int n_group;
+  int tiles_per_group;
   GemmTcCfg cfg;
   int tiles_m, tiles_n;
   int num_tiles;
@@ -124,11 +127,18 @@ __device__ __forceinline__ uint32_t make_idesc(int bn, int a_mn, int b_mn) {
          (uint32_t(bn >> 3) << 17) | (uint32_t(BM >> 4) << 24);
 }
 
+// i -> (i / x0, i % x0) without a division in the common merged case (x0 > i)
+__device__ __forceinline__ void split2(int i, int x0, int& hi, int& lo) {
+  if (i < x0) { hi = 0; lo = i; }
+  else { hi = i / x0; lo = i - hi * x0; }
+}
+
 // Tile index -> (batch, m tile, n tile); m runs fastest so that CTAs running together share the
 // B tile. With CAUSAL_SKIP_UPPER only tiles that touch the lower triangle are enumerated.
-__device__ __forceinline__ void decode_tile(const TcParams& p, int tile, int& bz, int& mt, int& nt) {
-  bz = tile / p.tiles_per_batch;
-  int r = tile - bz * p.tiles_per_batch;
+__device__ __forceinline__ void decode_tile(const TcParams& p, int tile, int& grp, int& bz, int& mt, int& nt) {
+  int r;
+  split2(tile, p.tiles_per_group, grp, r);
+  split2(r, p.tiles_per_batch, bz, r);
   if (p.g.causal == CAUSAL_SKIP_UPPER) {
     for (int m = 0; m < p.tiles_m; ++m) {
       const int nv = min(p.tiles_n, (m * BM + BM - 1) / p.cfg.bn + 1);
@@ -138,8 +148,7 @@ __device__ __forceinline__ void decode_tile(const TcParams& p, int tile, int& bz
     mt = 0; nt = 0;
     return;
   }
-  nt = r / p.tiles_m;
-  mt = r - nt * p.tiles_m;
+  split2(r, p.tiles_m, nt, mt);
 }
 
 __device__ __forceinline__ int k_steps_of(const TcParams& p, int mt) {
@@ -157,7 +166,9 @@ __device__ __forceinline__ void fill_coords(const int* sel, int rank, int k0, in
 }
 
 __device__ __forceinline__ int64_t split_off(int i, int x0, int64_t s1, int64_t s0) {
-  return (int64_t)(i / x0) * s1 + (int64_t)(i % x0) * s0;
+  int hi, lo;
+  split2(i, x0, hi, lo);
+  return (int64_t)hi * s1 + (int64_t)lo * s0;
 }
 
 
@@ -199,7 +210,8 @@ __device__ __forceinline__ void epilogue_chunk_vec(const GemmParams& g, uint32_t
   tmem_ld32(taddr, r);
   // group offsets (an 8-column group shares one n split)
   int64_t co[4], ro[4];
-  int n1 = n / g.N0, n0i = n - n1 * g.N0;
+  int n1, n0i;
+  split2(n, g.N0, n1, n0i);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     co[q] = cb + (int64_t)n1 * g.c_s[4] + n0i;
@@ -314,6 +326,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& g, uint32_t tad
 template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
                const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -330,6 +343,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
   volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
 
+  pdl_launch_dependents();  // the next step may start its prologue now
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tmem_cols = uint32_t(2 * bn);  // 128, 256 or 512: a power of two >= 32
 
@@ -357,6 +371,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t ph = 0;
       bool ok = true;
       const int a_boxes = p.cfg.a_mn_major ? BM / 64 : 1, b_boxes = p.cfg.b_mn_major ? bn / 64 : 1;
+      pdl_wait();  // the previous step's outputs are this step's operands
       // which coordinate slots carry the running k split (the rest stay fixed over a tile)
       int a_kd0 = 0, a_kd1 = -1, b_kd0 = 0, b_kd1 = -1;
 #pragma unroll
@@ -367,20 +382,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (p.cfg.b_sel[d] == 1) b_kd1 = d;
       }
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
-        int bz, mt, nt;
-        decode_tile(p, tile, bz, mt, nt);
+        int grp, bz, mt, nt;
+        decode_tile(p, tile, grp, bz, mt, nt);
         const int ksteps = k_steps_of(p, mt);
         int ca[2][5], cb[4][5];  // fully unrolled below: these stay in registers
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
-          const int m = mt * BM + ch * 64;
-          fill_coords(p.cfg.a_sel, 5, 0, 0, m % p.cfg.a_r0, m / p.cfg.a_r0, bz % p.cfg.a_b0, bz / p.cfg.a_b0, ca[ch]);
+          int r1, r0, b1, b0;
+          split2(mt * BM + ch * 64, p.cfg.a_r0, r1, r0);
+          split2(bz, p.cfg.a_b0, b1, b0);
+          fill_coords(p.cfg.a_sel, 5, 0, 0, r0, r1, b0, b1, ca[ch]);
         }
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
-          const int n = nt * bn + ch * 64;
-          fill_coords(p.cfg.b_sel, 5, 0, 0, n % p.cfg.b_r0, n / p.cfg.b_r0, bz % p.cfg.b_b0, bz / p.cfg.b_b0, cb[ch]);
+          int r1, r0, b1, b0;
+          split2(nt * bn + ch * 64, p.cfg.b_r0, r1, r0);
+          split2(bz, p.cfg.b_b0, b1, b0);
+          fill_coords(p.cfg.b_sel, 5, 0, 0, r0, r1, b0, b1, cb[ch]);
         }
+        const CUtensorMap* mapb = grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2);
         int ak0 = 0, ak1 = 0, bk0 = 0, bk1 = 0;  // running split of the k index for each operand
         for (int ks = 0; ks < ksteps; ++ks) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u)) { ok = false; break; }
@@ -402,7 +422,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               int c[5];
 #pragma unroll
               for (int d = 0; d < 5; ++d) c[d] = cb[ch][d] + (d == b_kd0 ? bk0 : 0) + (d == b_kd1 ? bk1 : 0);
-              tma_load(sb + ch * 8192u, &map_b, fb, c[0], c[1], c[2], c[3], c[4]);
+              tma_load(sb + ch * 8192u, mapb, fb, c[0], c[1], c[2], c[3], c[4]);
             }
           }
           ++issued;
@@ -431,8 +451,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
-        int bz, mt, nt;
-        decode_tile(p, tile, bz, mt, nt);
+        int grp, bz, mt, nt;
+        decode_tile(p, tile, grp, bz, mt, nt);
         const int ksteps = k_steps_of(p, mt);
         if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u)) { ok = false; break; }
         tc_fence_after();
@@ -461,16 +481,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ---------------- epilogue (warps 2..9) ----------------
     // Warp w reads tensor-memory lanes 32*(w%4)..+31 (one accumulator row per thread); the two
     // warps that share a lane quarter split the tile's columns between them.
-    const GemmParams& g = p.g;
     const int lane_base = (warp & 3) * 32;
     const int half = (warp - 2) >> 2;
     const int col_begin = half * (bn / 2), col_end = col_begin + bn / 2;
     int acc = 0;
     uint32_t acc_ph = 0;
     bool ok = true;
+    pdl_wait();  // before any global read (bias, residual) or write (C)
     for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
-      int bz, mt, nt;
-      decode_tile(p, tile, bz, mt, nt);
+      int grp, bz, mt, nt;
+      decode_tile(p, tile, grp, bz, mt, nt);
+      const GemmParams& g = grp == 0 ? p.g : p.gx[grp - 1];
       const int m = mt * BM + lane_base + lane;
       const bool row_ok = m < g.M;
       const int64_t cb = split_off(bz, g.B0, g.c_s[0], g.c_s[1]) + (row_ok ? split_off(m, g.M0, g.c_s[2], g.c_s[3]) : 0);
@@ -553,9 +574,14 @@ int encode_tensor_map(TensorMapStorage* out, const void* base, const TmaOperand&
   return rc == CUDA_SUCCESS ? 0 : -2;
 }
 
-cudaError_t launch_gemm_tc(const GemmParams& g, const GemmTcHost& tc, uint32_t* status, cudaStream_t stream) {
+cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_group, uint32_t* status,
+                           cudaStream_t stream) {
+  const GemmParams& g = gs[0];
+  const GemmTcHost& tc = tcs[0];
   TcParams p;
   p.g = g;
+  p.n_group = n_group;
+  for (int i = 1; i < 3; ++i) p.gx[i - 1] = gs[i < n_group ? i : 0];
   p.cfg = tc.cfg;
   p.tiles_m = (g.M + BM - 1) / BM;
   p.tiles_n = (g.N + tc.cfg.bn - 1) / tc.cfg.bn;
@@ -565,20 +591,28 @@ cudaError_t launch_gemm_tc(const GemmParams& g, const GemmTcHost& tc, uint32_t* 
     for (int m = 0; m < p.tiles_m; ++m) per_batch += std::min(p.tiles_n, (m * BM + BM - 1) / tc.cfg.bn + 1);
   }
   if (per_batch * g.batch > 0x7fffffffLL) return cudaErrorInvalidValue;
+  if (per_batch * g.batch * n_group > 0x7fffffffLL) return cudaErrorInvalidValue;
   p.tiles_per_batch = (int)per_batch;
-  p.num_tiles = (int)(per_batch * g.batch);
+  p.tiles_per_group = (int)(per_batch * g.batch);
+  p.num_tiles = p.tiles_per_group * n_group;
   p.status = status;
   const size_t smem = size_t(tc.cfg.stages) * (kATileBytes + size_t(tc.cfg.bn) * BK * 2) + 1024 + 8 * (2 * tc.cfg.stages + 4) + 16;
   const int grid = std::min(p.num_tiles, sm_count());
   if (grid <= 0) return cudaSuccess;
   const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(&tc.map_a);
   const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(&tc.map_b);
+  const CUtensorMap* mb1 = reinterpret_cast<const CUtensorMap*>(&tcs[n_group > 1 ? 1 : 0].map_b);
+  const CUtensorMap* mb2 = reinterpret_cast<const CUtensorMap*>(&tcs[n_group > 2 ? 2 : 0].map_b);
   // The vector epilogues need: n contiguous in C (and R), 8-column groups aligned to 16 bytes and
   // inside one n split, N a multiple of 8. Everything else takes the general epilogue.
   auto mult8 = [](int64_t v) { return (v & 7) == 0; };
-  bool vec = g.c_s[5] == 1 && (g.N & 7) == 0 && (g.N0 & 7) == 0 && mult8(g.c_s[0]) && mult8(g.c_s[1]) && mult8(g.c_s[2]) &&
-             mult8(g.c_s[3]) && mult8(g.c_s[4]) && (reinterpret_cast<uintptr_t>(g.C) & 15) == 0 &&
-             (!g.has_bias || (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0);
+  bool vec = true;
+  for (int i = 0; i < n_group; ++i) {
+    const GemmParams& q = gs[i];
+    vec = vec && q.c_s[5] == 1 && (q.N & 7) == 0 && (q.N0 & 7) == 0 && mult8(q.c_s[0]) && mult8(q.c_s[1]) && mult8(q.c_s[2]) &&
+          mult8(q.c_s[3]) && mult8(q.c_s[4]) && (reinterpret_cast<uintptr_t>(q.C) & 15) == 0 &&
+          (!q.has_bias || (reinterpret_cast<uintptr_t>(q.bias) & 15) == 0) && q.c_f32 == g.c_f32;
+  }
   if (g.has_res)
     vec = vec && g.r_s[5] == 1 && mult8(g.r_s[0]) && mult8(g.r_s[1]) && mult8(g.r_s[2]) && mult8(g.r_s[3]) &&
           mult8(g.r_s[4]) && (reinterpret_cast<uintptr_t>(g.R) & 15) == 0;
@@ -598,8 +632,7 @@ cudaError_t launch_gemm_tc(const GemmParams& g, const GemmTcHost& tc, uint32_t* 
       if (e != cudaSuccess) return e;                                                                                \
       attr_set[E] = true;                                                                                            \
     }                                                                                                                \
-    gemm_tc_kernel<E><<<grid, kThreads, smem, stream>>>(*ma, *mb, p);                                                \
-    break;                                                                                                           \
+    return launch_k(gemm_tc_kernel<E>, grid, kThreads, smem, stream, *ma, *mb, *mb1, *mb2, p);                                   \
   }
   switch (epi) {
     FLUID_TC_LAUNCH(EPI_PLAIN)
@@ -612,7 +645,7 @@ cudaError_t launch_gemm_tc(const GemmParams& g, const GemmTcHost& tc, uint32_t* 
       FLUID_TC_LAUNCH(EPI_ANY)
   }
 #undef FLUID_TC_LAUNCH
-  return cudaGetLastError();
+  return cudaSuccess;
 }
 
 }  // namespace fluid

@@ -140,7 +140,9 @@ struct EmbedParams {
 
 // Launchers: enqueue on `stream`, return the CUDA error of the launch.
 cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
-cudaError_t launch_gemm_tc(const GemmParams& p, const GemmTcHost& tc, uint32_t* status,
+// n_group (1..3) GEMMs that share the A operand, the shapes and the tile configuration run as one
+// launch (sibling projections such as Q/K/V or gate/up); group i uses g[i] and tc[i].map_b.
+cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, uint32_t* status,
                            cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);
 cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t stream);

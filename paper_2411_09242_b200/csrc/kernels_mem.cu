@@ -14,6 +14,8 @@ static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t
 // ---- EMBED: y[t, :] = tok[ids[t], :] (+ pos[t % S, :]) -------------------------------------------
 template <typename T, bool VECTOR>
 __global__ void embed_kernel(EmbedParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int t = blockIdx.x;
   int id = p.ids[t];
   id = min(max(id, 0), p.V - 1);
@@ -56,9 +58,7 @@ static cudaError_t embed_t(const EmbedParams& p, cudaStream_t st) {
   constexpr int V = VecOf<T>::N;
   const bool vec = p.H % V == 0 && aligned16(p.tok) && aligned16(p.y) && (!p.pos || aligned16(p.pos));
   const int threads = std::min(256, std::max(32, ((p.H / (vec ? V : 1)) + 31) / 32 * 32));
-  if (vec) embed_kernel<T, true><<<p.tokens, threads, 0, st>>>(p);
-  else embed_kernel<T, false><<<p.tokens, threads, 0, st>>>(p);
-  return cudaGetLastError();
+  return vec ? launch_k(embed_kernel<T, true>, p.tokens, threads, 0, st, p) : launch_k(embed_kernel<T, false>, p.tokens, threads, 0, st, p);
 }
 
 cudaError_t launch_embed(const EmbedParams& p, cudaStream_t st) {
@@ -91,6 +91,8 @@ __device__ __forceinline__ void norm_load(const void* base, bool f32, size_t row
 
 template <typename T, bool VECTOR>
 __global__ void norm_kernel(NormParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int V = VECTOR ? VecOf<T>::N : 1;
   __shared__ float red[32];
   const size_t roff = (size_t)blockIdx.x * p.width;
@@ -171,9 +173,7 @@ static cudaError_t norm_t(const NormParams& p, cudaStream_t st) {
   int threads = (nch + 31) / 32 * 32;
   threads = std::min(1024, std::max(32, threads));
   if ((int64_t)threads * NORM_MAXC < nch) return cudaErrorInvalidValue;  // rejected at plan time
-  if (vec) norm_kernel<T, true><<<p.rows, threads, 0, st>>>(p);
-  else norm_kernel<T, false><<<p.rows, threads, 0, st>>>(p);
-  return cudaGetLastError();
+  return vec ? launch_k(norm_kernel<T, true>, p.rows, threads, 0, st, p) : launch_k(norm_kernel<T, false>, p.rows, threads, 0, st, p);
 }
 
 cudaError_t launch_norm(const NormParams& p, cudaStream_t st) {
@@ -188,6 +188,8 @@ __device__ __forceinline__ float sm_exp(float x) {
 
 template <typename T, int NCH, bool VECTOR>
 __global__ void softmax_warp_kernel(SoftmaxParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int V = VECTOR ? VecOf<T>::N : 1;
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -247,6 +249,8 @@ __global__ void softmax_warp_kernel(SoftmaxParams p) {
 // Fallback for rows too long for the register-resident kernel: one CTA per row, three sweeps.
 template <typename T>
 __global__ void softmax_block_kernel(SoftmaxParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float red[32];
   const int64_t row = blockIdx.x;
   const T* x = static_cast<const T*>(p.x) + row * p.n;
@@ -274,16 +278,15 @@ static cudaError_t softmax_t(const SoftmaxParams& p, cudaStream_t st) {
   const int per_lane = (p.n + 32 * (vec ? V : 1) - 1) / (32 * (vec ? V : 1));
   const int warps = 4;
   const unsigned grid = (unsigned)((p.rows + warps - 1) / warps);
-#define SM_LAUNCH(NCH, VEC) softmax_warp_kernel<T, NCH, VEC><<<grid, warps * 32, 0, st>>>(p)
+#define SM_LAUNCH(NCH, VEC) return launch_k(softmax_warp_kernel<T, NCH, VEC>, grid, warps * 32, 0, st, p)
   if (vec && per_lane <= 1) SM_LAUNCH(1, true);
   else if (vec && per_lane <= 2) SM_LAUNCH(2, true);
   else if (vec && per_lane <= 4) SM_LAUNCH(4, true);
   else if (vec && per_lane <= 8) SM_LAUNCH(8, true);
   else if (vec && per_lane <= 16 && sizeof(T) == 4) SM_LAUNCH(16, true);
   else if (!vec && per_lane <= 8) SM_LAUNCH(8, false);
-  else softmax_block_kernel<T><<<(unsigned)p.rows, 256, 0, st>>>(p);
+  else return launch_k(softmax_block_kernel<T>, (unsigned)p.rows, 256, 0, st, p);
 #undef SM_LAUNCH
-  return cudaGetLastError();
 }
 
 cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t st) {
@@ -293,6 +296,8 @@ cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t st) {
 // ---- ROPE: one thread per rotated pair, threads ordered as the tensor lies in memory --------------
 template <typename T>
 __global__ void rope_kernel(RopeParams p, int64_t total) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int half = p.dims[3] / 2;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     int idx[4];
@@ -322,9 +327,8 @@ cudaError_t launch_rope(const RopeParams& p, cudaStream_t st) {
   const int64_t total = (int64_t)p.dims[0] * p.dims[1] * p.dims[2] * (p.dims[3] / 2);
   const int threads = 256;
   const unsigned grid = (unsigned)std::min<int64_t>((total + threads - 1) / threads, 148 * 32);
-  if (p.dtype == FLUID_BF16) rope_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>(p, total);
-  else rope_kernel<float><<<grid, threads, 0, st>>>(p, total);
-  return cudaGetLastError();
+  return p.dtype == FLUID_BF16 ? launch_k(rope_kernel<__nv_bfloat16>, grid, threads, 0, st, p, total)
+                               : launch_k(rope_kernel<float>, grid, threads, 0, st, p, total);
 }
 
 // ---- ELTWISE ---------------------------------------------------------------------------------------
@@ -341,6 +345,8 @@ __device__ __forceinline__ float elt_apply(int op, float a, float b) {
 
 template <typename T, bool VECTOR>
 __global__ void eltwise_kernel(EltParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int V = VECTOR ? VecOf<T>::N : 1;
   T* y = static_cast<T*>(p.y);
   float* yf = static_cast<float*>(p.y);
@@ -376,9 +382,7 @@ static cudaError_t eltwise_t(const EltParams& p, cudaStream_t st) {
   const bool vec = p.n % V == 0 && aligned16(p.a) && aligned16(p.y) && (!p.b || aligned16(p.b));
   const int64_t nch = p.n / (vec ? V : 1);
   const unsigned grid = (unsigned)std::min<int64_t>((nch + 255) / 256, 148 * 16);
-  if (vec) eltwise_kernel<T, true><<<grid, 256, 0, st>>>(p);
-  else eltwise_kernel<T, false><<<grid, 256, 0, st>>>(p);
-  return cudaGetLastError();
+  return vec ? launch_k(eltwise_kernel<T, true>, grid, 256, 0, st, p) : launch_k(eltwise_kernel<T, false>, grid, 256, 0, st, p);
 }
 
 cudaError_t launch_eltwise(const EltParams& p, cudaStream_t st) {
@@ -396,6 +400,8 @@ struct PermSorted {
 // Class A: the contiguous dim is the same on both sides -> move 16-byte (or element) rows.
 template <typename E>
 __global__ void permute_rows_kernel(const E* __restrict__ x, E* __restrict__ y, PermSorted s, int64_t total) {
+  pdl_launch_dependents();
+  pdl_wait();
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     int64_t rem = i, xo = 0, yo = 0;
 #pragma unroll
@@ -414,6 +420,8 @@ __global__ void permute_rows_kernel(const E* __restrict__ x, E* __restrict__ y, 
 template <typename E>
 __global__ void permute_tile_kernel(const E* __restrict__ x, E* __restrict__ y, PermSorted s, int di, int dn,
                                     int tiles_i, int tiles_o) {
+  pdl_launch_dependents();
+  pdl_wait();
   // s.dims[4] is the output-fast dim O (extent dn); s.dims[3] holds the input-fast dim I (extent di)
   __shared__ E tile[64][65];
   int64_t blk = blockIdx.x;
@@ -472,10 +480,10 @@ static void permute_dispatch(const PermuteParams& p, cudaStream_t st) {
       for (int k = 0; k < 4; ++k) { w.xs[k] /= W; w.ys[k] /= W; }
       const int64_t tw = total / W;
       const unsigned grid = (unsigned)std::min<int64_t>((tw + 255) / 256, 148 * 16);
-      permute_rows_kernel<uint4><<<grid, 256, 0, st>>>(reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(y), w, tw);
+      launch_k(permute_rows_kernel<uint4>, grid, 256, 0, st, reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(y), w, tw);
     } else {
       const unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 16);
-      permute_rows_kernel<E><<<grid, 256, 0, st>>>(x, y, s, total);
+      launch_k(permute_rows_kernel<E>, grid, 256, 0, st, x, y, s, total);
     }
     return;
   }
@@ -485,7 +493,7 @@ static void permute_dispatch(const PermuteParams& p, cudaStream_t st) {
     if (s.dims[k] > 1 && s.xs[k] == 1) xi = k;
   if (xi < 0) {
     const unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 16);
-    permute_rows_kernel<E><<<grid, 256, 0, st>>>(x, y, s, total);
+    launch_k(permute_rows_kernel<E>, grid, 256, 0, st, x, y, s, total);
     return;
   }
   PermSorted t = s;
@@ -495,7 +503,7 @@ static void permute_dispatch(const PermuteParams& p, cudaStream_t st) {
   t.dims[3] = dI; t.xs[3] = xI; t.ys[3] = yI;
   const int tiles_i = (t.dims[3] + 63) / 64, tiles_o = (t.dims[4] + 63) / 64;
   const int64_t blocks = (int64_t)tiles_i * tiles_o * t.dims[0] * t.dims[1] * t.dims[2];
-  permute_tile_kernel<E><<<(unsigned)blocks, 256, 0, st>>>(x, y, t, t.dims[3], t.dims[4], tiles_i, tiles_o);
+  launch_k(permute_tile_kernel<E>, (unsigned)blocks, 256, 0, st, x, y, t, t.dims[3], t.dims[4], tiles_i, tiles_o);
 }
 
 cudaError_t launch_permute(const PermuteParams& p, cudaStream_t st) {

@@ -217,7 +217,7 @@ bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& g, GemmTcHost* tc
   if (g.N <= 64) bn = 64;
   else {
     const int64_t tiles256 = int64_t((g.M + 127) / 128) * ((g.N + 255) / 256) * g.batch;
-    if (g.N >= 256 && tiles256 >= 120) bn = 256;
+    if (g.N >= 256 && tiles256 >= 74) bn = 256;
   }
   const int64_t a_rs[2] = {g.a_s[2], g.a_s[3]}, a_ks[2] = {g.a_s[4], g.a_s[5]}, a_bs[2] = {g.a_s[0], g.a_s[1]};
   const int64_t b_rs[2] = {g.b_s[4], g.b_s[5]}, b_ks[2] = {g.b_s[2], g.b_s[3]}, b_bs[2] = {g.b_s[0], g.b_s[1]};
@@ -825,7 +825,31 @@ static int lower_and_place(fluid_plan_s* p) {
   p->steps.clear();
   const int* lo = p->layout.data();
   Evaluator ev{p, std::vector<int>(nt, 0)};
+  std::vector<char> taken(p->nodes.size(), 0);
+  auto node_step_cost = [&](int ni) {
+    std::vector<int> tids = node_tensors(p->nodes[ni]), l;
+    for (int t : tids) l.push_back(lo[t]);
+    return ev(ni, tids, l);
+  };
+  // sibling projections (same input, same shapes, no residual) can share one launch
+  auto siblings_ok = [&](const Node& a, const Node& b) {
+    if (b.kind != N_GEMM || b.gemm_kind != G_LINEAR || b.a != a.a || b.res >= 0 || b.act != a.act ||
+        b.contract != a.contract || (a.bias >= 0) != (b.bias >= 0))
+      return false;
+    GemmParams ga, gb;
+    GemmTcHost ta, tb;
+    if (!lower_gemm(p, a, lo, &ga) || !lower_gemm(p, b, lo, &gb)) return false;
+    if (!gemm_tc_eligible(p, ga, &ta) || !gemm_tc_eligible(p, gb, &tb)) return false;
+    if (ga.M != gb.M || ga.N != gb.N || ga.K != gb.K || ga.N0 != gb.N0 || ga.M0 != gb.M0 || ga.K0 != gb.K0) return false;
+    if (std::memcmp(&ta.cfg, &tb.cfg, sizeof(GemmTcCfg)) != 0) return false;
+    for (int i = 0; i < 6; ++i)
+      if (ga.a_s[i] != gb.a_s[i]) return false;
+    for (int d = 0; d < 5; ++d)
+      if (ta.b.dims[d] != tb.b.dims[d] || ta.b.strides[d] != tb.b.strides[d] || ta.b.box[d] != tb.b.box[d]) return false;
+    return true;
+  };
   for (int ni = 0; ni < (int)p->nodes.size(); ++ni) {
+    if (taken[ni]) continue;
     const Node& n = p->nodes[ni];
     if (n.kind == N_TRANSPOSE && transpose_is_alias(p, n, lo)) {
       p->alias_root[n.out] = p->alias_root[n.a];
@@ -833,9 +857,19 @@ static int lower_and_place(fluid_plan_s* p) {
     }
     Step s;
     s.node = ni;
-    std::vector<int> tids = node_tensors(n), l;
-    for (int t : tids) l.push_back(lo[t]);
-    s.cost = ev(ni, tids, l);
+    s.nodes.push_back(ni);
+    s.cost = node_step_cost(ni);
+    if (p->opts.fusion && n.kind == N_GEMM && n.gemm_kind == G_LINEAR && n.res < 0) {
+      for (int nj = ni + 1; nj < (int)p->nodes.size() && s.nodes.size() < 3; ++nj) {
+        if (taken[nj]) continue;
+        const Node& m = p->nodes[nj];
+        if (m.kind == N_GEMM && m.gemm_kind == G_LINEAR && m.a == n.a && siblings_ok(n, m)) {
+          taken[nj] = 1;
+          s.nodes.push_back(nj);
+          s.cost += node_step_cost(nj) - kLaunch;
+        }
+      }
+    }
     p->steps.push_back(s);
   }
   // lifetimes in step indices, per alias group
@@ -843,16 +877,18 @@ static int lower_and_place(fluid_plan_s* p) {
   p->last_step.assign(nt, -1);
   std::vector<int> gfirst(nt, -1), glast(nt, -1);
   for (int si = 0; si < (int)p->steps.size(); ++si) {
-    const Node& n = p->nodes[p->steps[si].node];
-    for (int t : n.outs) {
-      int r = p->alias_root[t];
-      if (gfirst[r] < 0) gfirst[r] = si;
-      glast[r] = std::max(glast[r], si);
-    }
-    for (int t : n.ins) {
-      int r = p->alias_root[t];
-      if (gfirst[r] < 0) gfirst[r] = si;  // inputs and constants: alive from first use
-      glast[r] = std::max(glast[r], si);
+    for (int ni : p->steps[si].nodes) {
+      const Node& n = p->nodes[ni];
+      for (int t : n.outs) {
+        int r = p->alias_root[t];
+        if (gfirst[r] < 0) gfirst[r] = si;
+        glast[r] = std::max(glast[r], si);
+      }
+      for (int t : n.ins) {
+        int r = p->alias_root[t];
+        if (gfirst[r] < 0) gfirst[r] = si;  // inputs and constants: alive from first use
+        glast[r] = std::max(glast[r], si);
+      }
     }
   }
   for (int t = 0; t < nt; ++t) {
@@ -867,8 +903,9 @@ static int lower_and_place(fluid_plan_s* p) {
   if (!p->opts.narrow_stream) {
     std::vector<int> producer(nt, -1), group(nt, 0), stream_use(nt, 0), operand_use(nt, 0);
     for (int t = 0; t < nt; ++t) group[p->alias_root[t]]++;
-    for (const Step& s : p->steps) {
-      const Node& n = p->nodes[s.node];
+    for (const Step& s : p->steps)
+     for (int ni : s.nodes) {
+      const Node& n = p->nodes[ni];
       producer[n.out] = (n.kind == N_ELTWISE && n.elt != ELT_ADD) ? -2 : n.kind;
       for (int t : n.ins) {
         const bool stream = (n.kind == N_NORM && (t == n.a || t == n.res)) || (n.kind == N_GEMM && t == n.res) ||
@@ -1080,16 +1117,21 @@ int fluid_plan_step_info(const fluid_plan_t* p, int step, fluid_step_info* info)
     return FLUID_EINVAL;
   }
   const Step& s = p->steps[step];
-  const Node& n = p->nodes[s.node];
   std::memset(info, 0, sizeof(*info));
   info->kernel = s.kernel;
   info->variant = s.variant;
-  info->n_ops = (int)std::min<size_t>(n.ops.size(), 8);
-  for (int i = 0; i < info->n_ops; ++i) info->ops[i] = n.ops[i];
-  info->n_in = (int)std::min<size_t>(n.ins.size(), 8);
-  for (int i = 0; i < info->n_in; ++i) info->in_ids[i] = n.ins[i];
-  info->n_out = (int)std::min<size_t>(n.outs.size(), 4);
-  for (int i = 0; i < info->n_out; ++i) info->out_ids[i] = n.outs[i];
+  for (int ni : s.nodes) {
+    const Node& n = p->nodes[ni];
+    for (int o : n.ops)
+      if (info->n_ops < 8) info->ops[info->n_ops++] = o;
+    for (int t : n.ins) {
+      bool seen = false;
+      for (int i = 0; i < info->n_in; ++i) seen = seen || info->in_ids[i] == t;
+      if (!seen && info->n_in < 8) info->in_ids[info->n_in++] = t;
+    }
+    for (int t : n.outs)
+      if (info->n_out < 4) info->out_ids[info->n_out++] = t;
+  }
   info->cost = s.cost;
   info->flops = s.flops;
   info->bytes = s.bytes;
