@@ -104,6 +104,20 @@ int finalize_steps(fluid_plan_s* p) {
         q.rows_per_mat = ty.rank >= 2 ? (int)ty.dims[ty.rank - 2] : 1;
         q.scale = (float)n.scale;
         q.causal = n.sm_causal;
+        q.zero_block = 0;
+        if (q.causal) {  // zeros past the diagonal block are never read by k-clipped PV products
+          bool all_clipped = true, any = false;
+          for (const Step& s2 : p->steps)
+            for (int nj : s2.nodes) {
+              const Node& m = p->nodes[nj];
+              for (int t : m.ins)
+                if (p->alias_root[t] == p->alias_root[n.out]) {
+                  any = true;
+                  if (!(m.kind == N_GEMM && m.gemm_kind == G_PV && m.causal == CAUSAL_CLIP_K && m.a == t)) all_clipped = false;
+                }
+            }
+          if (any && all_clipped && T[n.out].kind == FLUID_ACT) q.zero_block = 128;
+        }
         s.softmax = q;
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.out; s.t_narrow[0] = 1;
         double frac = 1.0;

@@ -172,20 +172,6 @@ __device__ __forceinline__ int64_t split_off(int i, int x0, int64_t s1, int64_t 
 }
 
 
-// GELU (erf form) with erf from Abramowitz & Stegun 7.1.26 (|error| < 1.5e-7 before fp32
-// rounding): far below bf16 resolution and a third of the instructions of erff().
-__device__ __forceinline__ float gelu_erf_fast(float x) {
-  const float z = fabsf(x) * 0.70710678118654752f;
-  const float t = __frcp_rn(fmaf(0.3275911f, z, 1.f));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  const float e = poly * t * __expf(-z * z);   // 1 - erf(z)
-  const float half_x = 0.5f * x;
-  return x >= 0.f ? fmaf(-half_x, e, x) : half_x * e;  // x/2 (1 + sign * (1 - e))
-}
-
 template <int ACT>
 __device__ __forceinline__ float act_t(float v) {
   if (ACT == ACT_GELU_ERF) return gelu_erf_fast(v);

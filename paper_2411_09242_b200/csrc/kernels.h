@@ -92,6 +92,8 @@ struct SoftmaxParams {
   int rows_per_mat;   // causal: row index inside its matrix = row % rows_per_mat
   float scale;
   int causal;
+  int zero_block;     // causal: 0 = zeros are written to the end of the row; else only up to the next
+                      // multiple of zero_block past the diagonal (the consumer reads no further)
 };
 
 struct RopeParams {

@@ -164,12 +164,128 @@ __global__ void norm_kernel(NormParams p) {
   }
 }
 
+// Row handled by WPR warps (1, 2, 4 or 8) of a 256-thread CTA: each lane owns NCH 16-byte
+// chunks; sums go through shuffles and, for WPR > 1, a few words of shared memory.
+template <int WPR>
+__device__ __forceinline__ float row_sum(float v, float* red, int warp, int lane) {
+  v = warp_sum(v);
+  if (WPR == 1) return v;
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = 0.f;
+  const int g0 = warp / WPR * WPR;
+#pragma unroll
+  for (int i = 0; i < WPR; ++i) t += red[g0 + i];
+  return t;
+}
+
+template <typename T, int NCH, int WPR>
+__global__ void __launch_bounds__(256) norm_warp_kernel(NormParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  constexpr int V = VecOf<T>::N;
+  __shared__ float red[8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int row = blockIdx.x * (8 / WPR) + warp / WPR;
+  const bool live = row < p.rows;
+  const size_t roff = (size_t)(live ? row : 0) * p.width;
+  const int nch = live ? p.width / V : 0;
+  const int c_first = (warp % WPR) * 32 + lane;
+  float v[NCH][V];
+  float s = 0.f;
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const int c = c_first + 32 * WPR * j;
+    if (c < nch) norm_load<T, V>(p.x, p.x_f32, roff, c, v[j]);
+  }
+  if (p.res) {
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      const int c = c_first + 32 * WPR * j;
+      if (c < nch) {
+        float b[V];
+        norm_load<T, V>(p.res, p.res_f32, roff, c, b);
+#pragma unroll
+        for (int i = 0; i < V; ++i) v[j][i] += b[i];
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    if (c_first + 32 * WPR * j < nch) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) s += p.rms ? v[j][i] * v[j][i] : v[j][i];
+    }
+  }
+  s = row_sum<WPR>(s, red, warp, lane);
+  float mean = 0.f, rstd;
+  if (p.rms) {
+    rstd = rsqrtf(s / p.width + p.eps);
+  } else {
+    mean = s / p.width;
+    float q = 0.f;
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      if (c_first + 32 * WPR * j < nch) {
+#pragma unroll
+        for (int i = 0; i < V; ++i) q += (v[j][i] - mean) * (v[j][i] - mean);
+      }
+    }
+    q = row_sum<WPR>(q, red, warp, lane);
+    rstd = rsqrtf(q / p.width + p.eps);
+  }
+  T* y_lo = static_cast<T*>(p.y_lo);
+  const T* gamma = static_cast<const T*>(p.gamma);
+  const T* beta = static_cast<const T*>(p.beta);
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const int c = c_first + 32 * WPR * j;
+    if (c < nch) {
+      float g[V], b[V], o[V];
+      norm_load<T, V>(gamma, false, 0, c, g);
+      if (beta) norm_load<T, V>(beta, false, 0, c, b);
+#pragma unroll
+      for (int i = 0; i < V; ++i) o[i] = (v[j][i] - mean) * rstd * g[i] + (beta ? b[i] : 0.f);
+      if (y_lo) {
+        float t8[VecOf<T>::N];
+#pragma unroll
+        for (int i = 0; i < V; ++i) t8[i] = o[i];
+        store16(y_lo + roff + (size_t)c * V, t8);
+      }
+      if (p.y_hi) {
+#pragma unroll
+        for (int i = 0; i < V; i += 4)
+          *reinterpret_cast<float4*>(p.y_hi + roff + (size_t)c * V + i) = make_float4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+      }
+    }
+  }
+}
+
 template <typename T>
 static cudaError_t norm_t(const NormParams& p, cudaStream_t st) {
   constexpr int V = VecOf<T>::N;
   const bool vec = p.width % V == 0 && aligned16(p.x) && (!p.y_lo || aligned16(p.y_lo)) && (!p.y_hi || aligned16(p.y_hi)) &&
                    aligned16(p.gamma) && (!p.beta || aligned16(p.beta)) && (!p.res || aligned16(p.res));
   const int nch = p.width / (vec ? V : 1);
+  if (vec && nch <= 32 * 8 * 4) {
+    // warps per row so that a lane owns at most 4 chunks
+    const int wpr = nch <= 128 ? 1 : (nch <= 256 ? 2 : (nch <= 512 ? 4 : 8));
+    const int per_lane = (nch + 32 * wpr - 1) / (32 * wpr);
+    const unsigned grid = (unsigned)((p.rows + 8 / wpr - 1) / (8 / wpr));
+#define NW_LAUNCH(N, W) return launch_k(norm_warp_kernel<T, N, W>, grid, 256, 0, st, p)
+#define NW_PICK(W)              \
+  if (per_lane <= 1) NW_LAUNCH(1, W); \
+  if (per_lane <= 2) NW_LAUNCH(2, W); \
+  if (per_lane <= 3) NW_LAUNCH(3, W); \
+  NW_LAUNCH(4, W)
+    if (wpr == 1) { NW_PICK(1); }
+    if (wpr == 2) { NW_PICK(2); }
+    if (wpr == 4) { NW_PICK(4); }
+    NW_PICK(8);
+#undef NW_PICK
+#undef NW_LAUNCH
+  }
   int threads = (nch + 31) / 32 * 32;
   threads = std::min(1024, std::max(32, threads));
   if ((int64_t)threads * NORM_MAXC < nch) return cudaErrorInvalidValue;  // rejected at plan time
@@ -246,6 +362,78 @@ __global__ void softmax_warp_kernel(SoftmaxParams p) {
   }
 }
 
+// bf16 rows kept packed in registers (16 bytes per chunk): exp is evaluated twice (sum, then
+// output) so that twice as many rows are in flight per SM. CAUSAL adds the per-row bounds;
+// the dense instantiation carries no per-element predicates at all.
+template <int NCH, bool CAUSAL>
+__global__ void __launch_bounds__(256) softmax_bf16_kernel(SoftmaxParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= p.rows) return;
+  const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x) + row * p.n;
+  __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.y) + row * p.n;
+  const int valid = CAUSAL ? min(p.n, int(row % p.rows_per_mat) + 1) : p.n;
+  const int write_end = (CAUSAL && p.zero_block > 0) ? min(p.n, (valid + p.zero_block - 1) / p.zero_block * p.zero_block) : p.n;
+  const float k = p.scale * 1.4426950408889634f;  // exp(x) = exp2(x * log2 e)
+  // Columns past `valid` (and past the row's end) are set to -inf once, right after the load: they
+  // then drop out of max and sum and come out as exact zeros with no further predicates.
+  constexpr uint32_t NEG2 = 0xFF80FF80u;  // two bf16 -inf
+  uint4 raw[NCH];
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const int base = (lane + 32 * j) * 8;
+    raw[j] = base < valid ? *reinterpret_cast<const uint4*>(x + base) : make_uint4(NEG2, NEG2, NEG2, NEG2);
+  }
+  // (a separate loop: every load above is in flight before the first fix-up touches its data)
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const int base = (lane + 32 * j) * 8;
+    if (CAUSAL && base < valid && base + 8 > valid) {
+      uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (base + 2 * i >= valid) w[i] = NEG2;
+        else if (base + 2 * i + 1 >= valid) w[i] = (w[i] & 0xffffu) | 0xFF800000u;
+      }
+      raw[j] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+  float m = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      m = fmaxf(m, fmaxf(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u)));
+  }
+  m = warp_max(m) * k;  // k > 0: max commutes with the scaling
+  float s = 0.f;
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      s += exp2f(fmaf(__uint_as_float(w[i] << 16), k, -m)) + exp2f(fmaf(__uint_as_float(w[i] & 0xffff0000u), k, -m));
+  }
+  s = warp_sum(s);
+  const float inv = 1.f / s;
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const int base = (lane + 32 * j) * 8;
+    if (base < write_end) {
+      const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+      uint32_t q[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        q[i] = pack_bf16x2(exp2f(fmaf(__uint_as_float(w[i] << 16), k, -m)) * inv,
+                           exp2f(fmaf(__uint_as_float(w[i] & 0xffff0000u), k, -m)) * inv);
+      *reinterpret_cast<uint4*>(y + base) = make_uint4(q[0], q[1], q[2], q[3]);
+    }
+  }
+}
+
 // Fallback for rows too long for the register-resident kernel: one CTA per row, three sweeps.
 template <typename T>
 __global__ void softmax_block_kernel(SoftmaxParams p) {
@@ -276,6 +464,19 @@ static cudaError_t softmax_t(const SoftmaxParams& p, cudaStream_t st) {
   constexpr int V = VecOf<T>::N;
   const bool vec = p.n % V == 0 && aligned16(p.x) && aligned16(p.y);
   const int per_lane = (p.n + 32 * (vec ? V : 1) - 1) / (32 * (vec ? V : 1));
+  if (sizeof(T) == 2 && vec && per_lane <= 16 && p.scale > 0.f) {
+    const int w8 = 8;
+    const unsigned g8 = (unsigned)((p.rows + w8 - 1) / w8);
+#define SB_LAUNCH(N)                                                                           \
+  return p.causal ? launch_k(softmax_bf16_kernel<N, true>, g8, w8 * 32, 0, st, p)              \
+                  : launch_k(softmax_bf16_kernel<N, false>, g8, w8 * 32, 0, st, p)
+    if (per_lane <= 1) SB_LAUNCH(1);
+    if (per_lane <= 2) SB_LAUNCH(2);
+    if (per_lane <= 4) SB_LAUNCH(4);
+    if (per_lane <= 8) SB_LAUNCH(8);
+    SB_LAUNCH(16);
+#undef SB_LAUNCH
+  }
   const int warps = 4;
   const unsigned grid = (unsigned)((p.rows + warps - 1) / warps);
 #define SM_LAUNCH(NCH, VEC) return launch_k(softmax_warp_kernel<T, NCH, VEC>, grid, warps * 32, 0, st, p)
@@ -323,7 +524,53 @@ __global__ void rope_kernel(RopeParams p, int64_t total) {
   }
 }
 
+// Vector variant (D contiguous, rotate-half pairing, bf16): a thread owns 8 pairs of one token
+// and applies the same 8 (cos, sin) to a group of heads, moving 16 bytes per access.
+constexpr int ROPE_HG = 4;
+__global__ void __launch_bounds__(256) rope_vec_kernel(RopeParams p, int64_t total, int hgroups) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int D = p.dims[3], half = D / 2, cpr = half / 8;
+  const float lb = log2f(p.base);
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int64_t rem = i;
+    const int c = int(rem % cpr); rem /= cpr;
+    const int hg = int(rem % hgroups); rem /= hgroups;
+    const int s = int(rem % p.dims[1]);
+    const int b = int(rem / p.dims[1]);
+    float cs[8], sn[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float inv_freq = exp2f(-2.f * (c * 8 + j) / D * lb);
+      sincosf(s * inv_freq, &sn[j], &cs[j]);
+    }
+    const int h_end = min(p.dims[2], (hg + 1) * ROPE_HG);
+    for (int h = hg * ROPE_HG; h < h_end; ++h) {
+      const int64_t off = b * p.st[0] + s * p.st[1] + h * p.st[2] + c * 8;
+      const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x) + off;
+      __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.y) + off;
+      float a[8], bb[8], oa[8], ob[8];
+      load16(x, a);
+      load16(x + half, bb);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        oa[j] = a[j] * cs[j] - bb[j] * sn[j];
+        ob[j] = bb[j] * cs[j] + a[j] * sn[j];
+      }
+      store16(y, oa);
+      store16(y + half, ob);
+    }
+  }
+}
+
 cudaError_t launch_rope(const RopeParams& p, cudaStream_t st) {
+  if (p.dtype == FLUID_BF16 && !p.interleaved && p.st[3] == 1 && (p.dims[3] / 2) % 8 == 0 && p.st[0] % 8 == 0 &&
+      p.st[1] % 8 == 0 && p.st[2] % 8 == 0 && aligned16(p.x) && aligned16(p.y)) {
+    const int hgroups = (p.dims[2] + ROPE_HG - 1) / ROPE_HG;
+    const int64_t total = (int64_t)p.dims[0] * p.dims[1] * hgroups * (p.dims[3] / 16);
+    const unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8);
+    return launch_k(rope_vec_kernel, grid, 256, 0, st, p, total, hgroups);
+  }
   const int64_t total = (int64_t)p.dims[0] * p.dims[1] * p.dims[2] * (p.dims[3] / 2);
   const int threads = 256;
   const unsigned grid = (unsigned)std::min<int64_t>((total + threads - 1) / threads, 148 * 32);
@@ -332,47 +579,75 @@ cudaError_t launch_rope(const RopeParams& p, cudaStream_t st) {
 }
 
 // ---- ELTWISE ---------------------------------------------------------------------------------------
-__device__ __forceinline__ float elt_apply(int op, float a, float b) {
-  switch (op) {
-    case ELT_ADD: return a + b;
-    case ELT_MUL: return a * b;
-    case ELT_GELU_ERF: return gelu_erf(a);
-    case ELT_GELU_TANH: return gelu_tanh(a);
-    case ELT_SILU: return silu(a);
-    default: return silu(a) * b;
+template <int OP>
+__device__ __forceinline__ float elt_apply(float a, float b) {
+  if (OP == ELT_ADD) return a + b;
+  if (OP == ELT_MUL) return a * b;
+  if (OP == ELT_GELU_ERF) return gelu_erf_fast(a);
+  if (OP == ELT_GELU_TANH) return gelu_tanh(a);
+  if (OP == ELT_SILU) return silu(a);
+  return silu(a) * b;
+}
+
+// One 16-byte chunk per thread per operand, two chunks in flight; WIDE (bf16 graphs, ADD only)
+// lets operands / result be the fp32 copies of residual-stream tensors.
+template <typename T, bool VECTOR, int OP, bool WIDE>
+__global__ void __launch_bounds__(256) eltwise_kernel(EltParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  constexpr int V = VECTOR ? VecOf<T>::N : 1;
+  constexpr bool BINARY = OP == ELT_ADD || OP == ELT_MUL || OP == ELT_SILU_MUL;
+  T* y = static_cast<T*>(p.y);
+  float* yf = static_cast<float*>(p.y);
+  const bool a_f32 = WIDE && p.a_f32, b_f32 = WIDE && p.b_f32, y_wide = WIDE && p.y_f32;
+  const int64_t nch = p.n / V;
+  const int64_t c0 = ((int64_t)blockIdx.x * blockDim.x * 2) + threadIdx.x;
+  float va[2][V], vb[2][V];
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int64_t c = c0 + u * (int64_t)blockDim.x;
+    if (c < nch) {
+      norm_load<T, V>(p.a, a_f32, (size_t)c * V, 0, va[u]);
+      if (BINARY) norm_load<T, V>(p.b, b_f32, (size_t)c * V, 0, vb[u]);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int64_t c = c0 + u * (int64_t)blockDim.x;
+    if (c < nch) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) va[u][i] = elt_apply<OP>(va[u][i], BINARY ? vb[u][i] : 0.f);
+      if (VECTOR) {
+        if (y_wide || sizeof(T) == 4) {
+#pragma unroll
+          for (int i = 0; i < V; i += 4)
+            *reinterpret_cast<float4*>(yf + c * V + i) = make_float4(va[u][i], va[u][i + 1], va[u][i + 2], va[u][i + 3]);
+        } else {
+          float t8[VecOf<T>::N];
+#pragma unroll
+          for (int i = 0; i < V; ++i) t8[i] = va[u][i];
+          store16(y + c * V, t8);
+        }
+      } else {
+        if (y_wide) yf[c] = va[u][0];
+        else y[c] = from_f<T>(va[u][0]);
+      }
+    }
   }
 }
 
 template <typename T, bool VECTOR>
-__global__ void eltwise_kernel(EltParams p) {
-  pdl_launch_dependents();
-  pdl_wait();
-  constexpr int V = VECTOR ? VecOf<T>::N : 1;
-  T* y = static_cast<T*>(p.y);
-  float* yf = static_cast<float*>(p.y);
-  const bool y_wide = p.y_f32 && sizeof(T) == 2;
-  const int64_t nch = p.n / V;
-  for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < nch; c += (int64_t)gridDim.x * blockDim.x) {
-    float va[V], vb[V];
-    norm_load<T, V>(p.a, p.a_f32, (size_t)c * V, 0, va);
-    if (p.b) norm_load<T, V>(p.b, p.b_f32, (size_t)c * V, 0, vb);
-#pragma unroll
-    for (int i = 0; i < V; ++i) va[i] = elt_apply(p.op, va[i], p.b ? vb[i] : 0.f);
-    if (VECTOR) {
-      if (y_wide || sizeof(T) == 4) {
-#pragma unroll
-        for (int i = 0; i < V; i += 4)
-          *reinterpret_cast<float4*>(yf + c * V + i) = make_float4(va[i], va[i + 1], va[i + 2], va[i + 3]);
-      } else {
-        float t8[VecOf<T>::N];
-#pragma unroll
-        for (int i = 0; i < V; ++i) t8[i] = va[i];
-        store16(y + c * V, t8);
-      }
-    } else {
-      if (y_wide) yf[c] = va[0];
-      else y[c] = from_f<T>(va[0]);
-    }
+static cudaError_t eltwise_v(const EltParams& p, unsigned grid, cudaStream_t st) {
+  const bool wide = sizeof(T) == 2 && (p.a_f32 || p.b_f32 || p.y_f32);
+  switch (p.op) {
+    case ELT_ADD:
+      return wide ? launch_k(eltwise_kernel<T, VECTOR, ELT_ADD, true>, grid, 256, 0, st, p)
+                  : launch_k(eltwise_kernel<T, VECTOR, ELT_ADD, false>, grid, 256, 0, st, p);
+    case ELT_MUL: return launch_k(eltwise_kernel<T, VECTOR, ELT_MUL, false>, grid, 256, 0, st, p);
+    case ELT_GELU_ERF: return launch_k(eltwise_kernel<T, VECTOR, ELT_GELU_ERF, false>, grid, 256, 0, st, p);
+    case ELT_GELU_TANH: return launch_k(eltwise_kernel<T, VECTOR, ELT_GELU_TANH, false>, grid, 256, 0, st, p);
+    case ELT_SILU: return launch_k(eltwise_kernel<T, VECTOR, ELT_SILU, false>, grid, 256, 0, st, p);
+    default: return launch_k(eltwise_kernel<T, VECTOR, ELT_SILU_MUL, false>, grid, 256, 0, st, p);
   }
 }
 
@@ -381,8 +656,8 @@ static cudaError_t eltwise_t(const EltParams& p, cudaStream_t st) {
   constexpr int V = VecOf<T>::N;
   const bool vec = p.n % V == 0 && aligned16(p.a) && aligned16(p.y) && (!p.b || aligned16(p.b));
   const int64_t nch = p.n / (vec ? V : 1);
-  const unsigned grid = (unsigned)std::min<int64_t>((nch + 255) / 256, 148 * 16);
-  return vec ? launch_k(eltwise_kernel<T, true>, grid, 256, 0, st, p) : launch_k(eltwise_kernel<T, false>, grid, 256, 0, st, p);
+  const unsigned grid = (unsigned)((nch + 511) / 512);
+  return vec ? eltwise_v<T, true>(p, grid, st) : eltwise_v<T, false>(p, grid, st);
 }
 
 cudaError_t launch_eltwise(const EltParams& p, cudaStream_t st) {
