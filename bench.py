@@ -90,6 +90,15 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a short list of floats over all ranks (identity without a process group)."""
+    import torch
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
 def feeds_of(m):
     f = dict(m.consts)
     f[m.graph.inputs[0]] = m.ids
@@ -295,10 +304,7 @@ def main():
     main_res = time_workload(args.workload, args.steps, args.warmup, torch, fluid, peaks, full=True, sampler=sampler,
                              overrides=overrides)
     barrier()
-    lat = torch.tensor([main_res["latency_ms"], main_res["e2e_ms"]], device="cuda", dtype=torch.float64)
-    if dist:
-        dist.all_reduce(lat, op=dist.ReduceOp.MAX)     # max over ranks
-    latency_ms, e2e_ms = float(lat[0]), float(lat[1])
+    latency_ms, e2e_ms = max_over_ranks([main_res["latency_ms"], main_res["e2e_ms"]], dist, torch.device("cuda"))
     if rank != 0:
         if dist:
             dist.destroy_process_group()

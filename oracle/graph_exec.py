@@ -55,8 +55,14 @@ def run_op(kind, ins, attrs):
     raise ValueError(f"unknown op kind {kind}")
 
 
-def run_graph(tensors, op_list, feeds, keep_all=False):
+def run_graph(tensors, op_list, feeds, keep_all=False, store=None):
     """Execute the graph.
+
+    store: optional callable (tensor id, fp64 array) -> fp64 array applied to every op output
+    before it is handed on. The parity reference never uses it (no intermediate rounding). It is a
+    diagnostic mode: a test may pass a function that rounds each tensor the way a device plan
+    stores it (bf16, fp32, or not at all for tensors fused away), to tell storage rounding apart
+    from arithmetic errors.
 
     tensors : list of dicts with "dims" (and "kind"); op_list : list of dicts with "kind",
     "ins", "outs", "attrs"; feeds : {tensor id: array} for every graph input and constant.
@@ -74,7 +80,7 @@ def run_graph(tensors, op_list, feeds, keep_all=False):
         for tid, o in zip(op["outs"], outs):
             assert list(o.shape) == list(tensors[tid]["dims"]), (
                 tensors[tid].get("name"), o.shape, tensors[tid]["dims"])
-            vals[tid] = o
+            vals[tid] = o if store is None else np.asarray(store(tid, o), dtype=np.float64)
         consumed.update(op["ins"])
     if keep_all:
         return vals

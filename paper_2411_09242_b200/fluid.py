@@ -461,21 +461,26 @@ class Runner:
         torch.cuda.synchronize()
         return [o.float().cpu().numpy().astype(np.float64) for o in self.outputs]
 
-    def read_tensor(self, tid):
-        """Copy one arena-resident (or output) tensor back in canonical order, for per-op checks."""
+    def read_tensor(self, tid, index=None):
+        """Copy one arena-resident (or output) tensor back in canonical order, for per-op checks.
+        index: optional tuple of slices / index lists applied on the device before the copy."""
         torch = _torch()
         torch.cuda.synchronize()
         desc = self.plan.desc
         t = desc.tensors[tid]
         info = self.plan.tensor_info(tid)
         if t["kind"] == synth.OUTPUT:
-            return self.outputs[desc.outputs.index(tid)].float().cpu().numpy().astype(np.float64)
-        if info.offset < 0:
-            raise ValueError(f"tensor {tid} is not arena-resident")
-        rec = next(r for r in self.plan.records() if r["tensor"] == info.alias_of and not r["twin"])
-        n = int(np.prod(t["dims"]))
-        es = synth.DTYPE_BYTES[rec["dtype"]]
-        raw = self.arena[info.offset: info.offset + n * es]
-        flat = raw.view(_TORCH_DTYPE[rec["dtype"]]).float().cpu().numpy().astype(np.float64)
-        pd = [t["dims"][p] for p in info.perm]
-        return np.ascontiguousarray(np.transpose(flat.reshape(pd), np.argsort(info.perm)))
+            view = self.outputs[desc.outputs.index(tid)]
+        else:
+            if info.offset < 0:
+                raise ValueError(f"tensor {tid} is not arena-resident")
+            rec = next(r for r in self.plan.records() if r["tensor"] == info.alias_of and not r["twin"])
+            n = int(np.prod(t["dims"]))
+            es = synth.DTYPE_BYTES[rec["dtype"]]
+            raw = self.arena[info.offset: info.offset + n * es]
+            pd = [t["dims"][p] for p in info.perm]
+            inv = [int(i) for i in np.argsort(info.perm)]
+            view = raw.view(_TORCH_DTYPE[rec["dtype"]]).view(pd).permute(inv)
+        if index is not None:
+            view = view[index]
+        return view.float().cpu().numpy().astype(np.float64)

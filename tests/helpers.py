@@ -68,9 +68,9 @@ def run_gpu(desc, feeds, candidates=None, poison=True, **opts):
     return dict(zip(desc.outputs, outs)), plan, runner
 
 
-def run_oracle(desc, feeds, keep_all=False):
+def run_oracle(desc, feeds, keep_all=False, store=None):
     from oracle import graph_exec
-    return graph_exec.run_graph(desc.tensors, desc.ops, feeds, keep_all=keep_all)
+    return graph_exec.run_graph(desc.tensors, desc.ops, feeds, keep_all=keep_all, store=store)
 
 
 def tol_for(dtype):
@@ -101,3 +101,109 @@ def single_op_graph(kind, in_shapes, out_shape, dtype, attrs=None, in_kinds=None
 def rand_feed(shape, dtype, seed, lo=-1.0, hi=1.0):
     a = synth.uniform(seed, 0, shape, lo, hi)
     return synth.round_bf16(a) if dtype == synth.BF16 else a
+
+
+# ---- sampled per-step parity at full size -----------------------------------------------------------
+ROWWISE = (synth.LINEAR, synth.ADD, synth.MUL, synth.GELU, synth.SILU, synth.LAYERNORM, synth.RMSNORM, synth.EMBED)
+
+
+def check_steps_sampled(desc, plan, runner, feeds, n_rows=48, tol=2 ** -7, seed=0):
+    """Per-step parity on samples: for every executed step, the oracle op(s) of that step are fed the GPU's
+    own inputs restricted to sampled rows (row-wise ops) or to one sampled (batch, head) slice (attention
+    products, softmax, RoPE), and the GPU's output is compared there. Localises any error to one kernel
+    launch and is affordable at full model sizes. The plan must keep every tensor alive (no_reuse=1).
+    Returns the number of outputs compared."""
+    from oracle import graph_exec
+    rng = np.random.default_rng(seed)
+    T = desc.tensors
+    consts = {}
+
+    def const_like(t):
+        return T[t]["kind"] in (synth.CONST, synth.INPUT) or T[plan.tensor_info(t).alias_of]["kind"] == synth.CONST
+
+    def const_value(t):
+        if t not in consts:
+            if t in feeds:
+                consts[t] = np.asarray(feeds[t])
+            else:                              # a zero-copy view of a constant: replay its producer
+                op = next(o for o in desc.ops if t in o["outs"])
+                consts[t] = graph_exec.run_op(op["kind"], [np.asarray(const_value(i), np.float64) for i in op["ins"]],
+                                              op["attrs"])[0]
+        return consts[t]
+
+    compared = 0
+    for s in plan.steps():
+        ops = [desc.ops[o] for o in s["ops"]]
+        first = ops[0]
+        od = T[first["outs"][0]]["dims"]
+        if first["kind"] in (synth.BMM_QK, synth.BMM_PV, synth.SOFTMAX) and len(od) == 4:
+            b, h = int(rng.integers(od[0])), int(rng.integers(od[1]))
+            index = (slice(b, b + 1), slice(h, h + 1))
+        elif first["kind"] == synth.ROPE:
+            h = int(rng.integers(od[2]))
+            index = (slice(None), slice(None), slice(h, h + 1))
+        elif first["kind"] in ROWWISE:
+            x_dims = T[first["ins"][0]]["dims"]
+            nlead = len(x_dims) - (first["attrs"].get("contract", 1) if first["kind"] == synth.LINEAR else 1)
+            if first["kind"] == synth.EMBED:
+                nlead = 2
+            lead = (T[first["ins"][0]]["dims"] if first["kind"] != synth.EMBED else od)[:nlead]
+            total = int(np.prod(lead))
+            rows = np.sort(rng.choice(total, size=min(n_rows, total), replace=False))
+            index = tuple(list(int(v) for v in ix) for ix in np.unravel_index(rows, lead))
+        else:
+            index = None                        # small tensors (SELECT_LAST_TOKEN): whole tensor
+        local = {}
+
+        def value(t, sampled=True):
+            if t in local:
+                return local[t]
+            if const_like(t):
+                v = np.asarray(const_value(t))
+                return v[index] if (sampled and index is not None and v.ndim == len(T[t]["dims"]) and T[t]["kind"] == synth.INPUT) else v
+            return runner.read_tensor(t, index if sampled else None)
+
+        for op in ops:
+            kind, out = op["kind"], op["outs"][0]
+            if kind == synth.EMBED:
+                ids = np.asarray(feeds[op["ins"][0]])[index]
+                want = np.asarray(const_value(op["ins"][1]), np.float64)[ids]
+                if len(op["ins"]) > 2:
+                    want = want + np.asarray(const_value(op["ins"][2]), np.float64)[np.asarray(index[1])]
+            elif kind == synth.LINEAR:
+                x = value(op["ins"][0])
+                w_t = op["ins"][1]
+                w = np.asarray(const_value(w_t), np.float64) if const_like(w_t) else runner.read_tensor(w_t)
+                c = op["attrs"].get("contract", 1)
+                K = int(np.prod(w.shape[:c]))
+                want = x.reshape(x.shape[0], K) @ w.reshape(K, -1)
+                if len(op["ins"]) > 2:
+                    want = want + np.asarray(const_value(op["ins"][2]), np.float64).reshape(1, -1)
+                want = want.reshape((x.shape[0],) + tuple(T[out]["dims"][len(index):]))
+            elif kind in (synth.LAYERNORM, synth.RMSNORM):
+                want = graph_exec.run_op(kind, [value(op["ins"][0])] + [np.asarray(const_value(t), np.float64) for t in op["ins"][1:]],
+                                         op["attrs"])[0]
+            elif kind == synth.SELECT_LAST_TOKEN:
+                want = runner.read_tensor(op["ins"][0])[:, -1, :]
+            else:
+                ins = [np.asarray(value(t), np.float64) for t in op["ins"]]
+                if kind == synth.BMM_PV:        # causal probabilities are zero above the diagonal by definition;
+                    prod = next((d for d in desc.ops if op["ins"][0] in d["outs"]), None)   # the device need not store them
+                    if prod is not None and prod["kind"] == synth.SOFTMAX and prod["attrs"].get("causal"):
+                        ins[0] = np.where(np.tril(np.ones(ins[0].shape[-2:], bool)), ins[0], 0.0)
+                want = graph_exec.run_op(kind, ins, op["attrs"])[0]
+            local[out] = want
+            if out not in s["outs"]:
+                continue                       # folded into the fused step: never stored
+            have = runner.read_tensor(out, index)
+            if kind in (synth.BMM_QK, synth.SOFTMAX):
+                causal = op["attrs"].get("causal") or any(
+                    d["kind"] == synth.SOFTMAX and d["attrs"].get("causal") and out in d["ins"] for d in desc.ops)
+                if causal:                      # entries above the diagonal are never read downstream
+                    S = want.shape[-1]
+                    mask = np.tril(np.ones((S, S), bool))
+                    want, have = np.where(mask, want, 0.0), np.where(mask, have, 0.0)
+            assert_close(have.reshape(want.shape), want, synth.BF16,
+                         f"step {s['kernel_name']} ops {s['ops']} -> {T[out]['name']}", tol=tol)
+            compared += 1
+    return compared

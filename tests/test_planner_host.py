@@ -172,3 +172,39 @@ def test_fusion_folds_epilogues():
     assert all(len(s["ops"]) <= 3 for s in fused.steps())
     assert fused.arena_bytes <= plain.arena_bytes
     fused.close(); plain.close()
+
+
+def test_sibling_projections_share_one_launch():
+    m = synth.build_model(synth.scaled(synth.CONFIGS["bert_base"], L=1), materialize=False)
+    plan = fluid.Plan(m.graph, synth.default_candidates(m.graph))
+    grouped = [s for s in plan.steps() if s["kernel_name"] == "GEMM_TC" and (s["variant"] >> 20) == 3]
+    assert len(grouped) == 1 and len(grouped[0]["outs"]) == 3 and len(grouped[0]["ops"]) == 3
+    names = {m.graph.tensors[t]["name"] for t in grouped[0]["outs"]}
+    assert names == {"l0.q", "l0.k", "l0.v"}
+    # the three outputs are alive from that step on and keep separate slices
+    offs = {plan.tensor_info(t).offset for t in grouped[0]["outs"]}
+    assert len(offs) == 3 and all(o >= fluid.ARENA_HEADER for o in offs)
+    ll = synth.build_model(synth.scaled(synth.CONFIGS["llama"], L=1), materialize=False)
+    lp = fluid.Plan(ll.graph, synth.default_candidates(ll.graph))
+    groups = sorted((s["variant"] >> 20) for s in lp.steps() if s["kernel_name"] == "GEMM_TC" and (s["variant"] >> 20))
+    assert groups == [2, 3]                      # gate/up and q/k/v
+    unfused = fluid.Plan(ll.graph, synth.default_candidates(ll.graph), fusion=0)
+    assert all((s["variant"] >> 20) == 0 for s in unfused.steps())
+    plan.close(); lp.close(); unfused.close()
+
+
+def test_residual_stream_is_held_in_fp32():
+    m = synth.build_model(synth.scaled(synth.CONFIGS["gpt2_small"], L=2), materialize=False)
+    d = m.graph
+    plan = fluid.Plan(d, synth.default_candidates(d))
+    by_name = {d.tensors[r["tensor"]]["name"]: r for r in plan.records() if not r["twin"]}
+    assert by_name["embed"]["dtype"] == synth.F32 and by_name["l0.res1"]["dtype"] == synth.F32
+    assert by_name["l0.ln1.out"]["dtype"] == synth.BF16          # feeds GEMMs only
+    assert not any(r["twin"] for r in plan.records())            # pre-LN: no tensor needs both
+    narrow = fluid.Plan(d, synth.default_candidates(d), narrow_stream=1)
+    assert all(r["dtype"] == synth.BF16 for r in narrow.records())
+    enc = synth.build_model(synth.scaled(synth.CONFIGS["bert_base"], L=1), materialize=False)
+    ep = fluid.Plan(enc.graph, synth.default_candidates(enc.graph))
+    twins = {enc.graph.tensors[r["tensor"]]["name"] for r in ep.records() if r["twin"]}
+    assert "emb_ln.out" in twins and "l0.ln1.out" in twins       # post-LN: stream value also feeds GEMMs
+    plan.close(); narrow.close(); ep.close()
