@@ -107,7 +107,9 @@ typedef double (*fluid_eval_fn)(void* user, int32_t node_id, int32_t n_tensors,
 
 typedef struct fluid_plan_options {
   int32_t fusion;           /* 1: fold bias/GELU/residual into GEMM epilogues, residual into norms,
-                               SiLU*up into one pass; 0: one step per graph op */
+                               SiLU*up into one pass, and BMM_QK -> SOFTMAX -> BMM_PV into one
+                               attention step whose score tensor never leaves the SM;
+                               0: one step per graph op */
   int32_t arena_policy;     /* 0: first fit (Algorithm 4 as printed), 1: best fit (its prose) */
   int32_t no_reuse;         /* 1: one private slice per activation (the naive plan) */
   int32_t force_canonical;  /* 1: skip the layout search, every tensor canonical */
@@ -116,7 +118,8 @@ typedef struct fluid_plan_options {
                                residual additions (the residual stream) are held in fp32 inside the
                                arena, with a bf16 twin where a GEMM also reads them; 1 = every
                                activation is held in its declared dtype */
-  int32_t reserved[2];
+  int32_t unfused_attention; /* 1: keep BMM_QK -> SOFTMAX -> BMM_PV as three steps even when fusion is on */
+  int32_t reserved[1];
   fluid_eval_fn eval;       /* NULL: built-in analytic B200 cost table */
   void* eval_user;
 } fluid_plan_options;
@@ -124,7 +127,7 @@ typedef struct fluid_plan_options {
 typedef enum {
   FLUID_K_EMBED = 0, FLUID_K_NORM = 1, FLUID_K_GEMM_SIMT = 2, FLUID_K_GEMM_TC = 3,
   FLUID_K_SOFTMAX = 4, FLUID_K_ROPE = 5, FLUID_K_ELTWISE = 6, FLUID_K_PERMUTE = 7,
-  FLUID_K_SELECT_LAST = 8, FLUID_K_COUNT = 9
+  FLUID_K_SELECT_LAST = 8, FLUID_K_ATTN = 9, FLUID_K_COUNT = 10
 } fluid_kernel_id;
 
 typedef struct fluid_step_info {

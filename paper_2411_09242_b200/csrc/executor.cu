@@ -182,6 +182,18 @@ int finalize_steps(fluid_plan_s* p) {
         s.bytes = es * ty.numel() * 2.0;
         break;
       }
+      case N_ATTN: {
+        s.kernel = FLUID_K_ATTN;
+        if (!lower_attn(p, n, lo, &s.attn, &s.attn_host)) {
+          set_error("step for op %d: attention cannot be lowered under the chosen layouts", n.ops[0]);
+          return FLUID_EUNSUPPORTED;
+        }
+        s.variant = s.attn.D | (s.attn.k_mn_major << 8) | (s.attn.v_k_major << 9) | (s.attn.causal << 10);
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.v; s.t_ptr[3] = n.out;
+        s.flops = 4.0 * s.attn.B * s.attn.NH * double(s.attn.S) * s.attn.S * s.attn.D * (s.attn.causal ? 0.5 * (1.0 + 1.0 / s.attn.S) : 1.0);
+        s.bytes = es * (double(T[n.a].numel()) + T[n.b].numel() + T[n.v].numel() + ty.numel());
+        break;
+      }
       case N_SELECT: {
         s.kernel = FLUID_K_SELECT_LAST;
         const TensorDesc& tx = T[n.a];
@@ -278,6 +290,18 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
   // tensor maps hold absolute addresses: (re-)encode when any base address changed
   if (!p->maps_valid || key != p->bound_key) {
     for (Step& s : p->steps) {
+      if (s.kernel == FLUID_K_ATTN) {
+        const void* q = R(s.t_ptr[0], 1);
+        const void* k = R(s.t_ptr[1], 1);
+        const void* v = R(s.t_ptr[2], 1);
+        if (!R.ok) return FLUID_EINVAL;
+        if (encode_tensor_map(&s.attn_host.map_q, q, s.attn_host.q) != 0 || encode_tensor_map(&s.attn_host.map_k, k, s.attn_host.k) != 0 ||
+            encode_tensor_map(&s.attn_host.map_v, v, s.attn_host.v) != 0) {
+          set_error("tensor map encoding failed for the attention step of op %d", p->nodes[s.node].ops[0]);
+          return FLUID_ECUDA;
+        }
+        continue;
+      }
       if (s.kernel != FLUID_K_GEMM_TC) continue;
       const void* a = R(s.t_ptr[0], 1);
       const void* b = R(s.t_ptr[1], 1);
@@ -341,6 +365,13 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
         } else if (R.ok) {
           err = launch_gemm_simt(q, stream);
         }
+        break;
+      }
+      case FLUID_K_ATTN: {
+        AttnParams q = s.attn;
+        q.O = const_cast<void*>(R(s.t_ptr[3]));
+        q.status = status;
+        if (R.ok) err = launch_attn_tc(q, s.attn_host, stream);
         break;
       }
       case FLUID_K_NORM: {

@@ -140,12 +140,33 @@ struct EmbedParams {
   int tokens, S, H, V;
 };
 
+// Fused attention: O[b,h,i,:] = softmax_j(scale * q[b,h,i,:].k[b,h,j,:]) v[b,h,j,:]
+struct AttnParams {
+  void* O;
+  uint32_t* status;
+  int B, NH, S, D;
+  int64_t o_s[3];       // element strides of b, h, s in O (d contiguous)
+  float scale_log2;     // scale * log2(e)
+  int causal;
+  int k_mn_major;       // K has the sequence index contiguous ([B,nh,D,S] family)
+  int v_k_major;        // V has the sequence index contiguous
+  int q_sel[5], k_sel[5], v_sel[5];   // tensor-map coordinate feeds: 0 contraction, 2 row, 4 / 5 batch split, 6 zero
+  int q_b0, k_b0, v_b0;               // inner extent of each operand's (batch * head) index split
+};
+
+struct AttnHost {
+  int eligible;
+  TmaOperand q, k, v;
+  TensorMapStorage map_q, map_k, map_v;
+};
+
 // Launchers: enqueue on `stream`, return the CUDA error of the launch.
 cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
 // n_group (1..3) GEMMs that share the A operand, the shapes and the tile configuration run as one
 // launch (sibling projections such as Q/K/V or gate/up); group i uses g[i] and tc[i].map_b.
 cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, uint32_t* status,
                            cudaStream_t stream);
+cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);
 cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t stream);
 cudaError_t launch_rope(const RopeParams& p, cudaStream_t stream);

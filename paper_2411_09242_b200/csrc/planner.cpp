@@ -247,6 +247,40 @@ bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& g, GemmTcHost* tc
   return true;
 }
 
+bool lower_attn(const fluid_plan_s* p, const Node& n, const int* lo, AttnParams* ap, AttnHost* host) {
+  const auto& T = p->graph.tensors;
+  const TensorDesc &tq = T[n.a], &tk = T[n.b], &tv = T[n.v], &to = T[n.out];
+  if (!tc_kernel_available() || p->opts.gemm_path == 1 || to.dtype != FLUID_BF16) return false;
+  const int64_t B = tq.dims[0], NH = tq.dims[1], S = tq.dims[2], D = tq.dims[3];
+  if (!(D == 64 || D == 128) || tk.dims[3] != S || tv.dims[2] != S || n.scale <= 0.0) return false;
+  int64_t sq[FLUID_MAX_RANK], sk[FLUID_MAX_RANK], sv[FLUID_MAX_RANK], so[FLUID_MAX_RANK];
+  strides_of(tq, perm_of(p, n.a, lo), sq);
+  strides_of(tk, perm_of(p, n.b, lo), sk);
+  strides_of(tv, perm_of(p, n.v, lo), sv);
+  strides_of(to, perm_of(p, n.out, lo), so);
+  if (so[3] != 1 || so[0] % 8 || so[1] % 8 || so[2] % 8) return false;
+  AttnHost h{};
+  const int64_t q_rs[2] = {0, sq[2]}, q_ks[2] = {0, sq[3]}, q_bs[2] = {sq[0], sq[1]};
+  const int64_t k_rs[2] = {0, sk[3]}, k_ks[2] = {0, sk[2]}, k_bs[2] = {sk[0], sk[1]};
+  const int64_t v_rs[2] = {0, sv[3]}, v_ks[2] = {0, sv[2]}, v_bs[2] = {sv[0], sv[1]};
+  if (!build_tma_operand(S, (int)S, q_rs, D, (int)D, q_ks, B * NH, (int)NH, q_bs, 64, &h.q) || h.q.mn_major) return false;
+  if (!build_tma_operand(S, (int)S, k_rs, D, (int)D, k_ks, B * NH, (int)NH, k_bs, 64, &h.k)) return false;
+  if (!build_tma_operand(D, (int)D, v_rs, S, (int)S, v_ks, B * NH, (int)NH, v_bs, 64, &h.v)) return false;
+  AttnParams a{};
+  a.B = (int)B; a.NH = (int)NH; a.S = (int)S; a.D = (int)D;
+  a.o_s[0] = so[0]; a.o_s[1] = so[1]; a.o_s[2] = so[2];
+  a.scale_log2 = float(n.scale * 1.4426950408889634);
+  a.causal = n.sm_causal;
+  a.k_mn_major = h.k.mn_major;
+  a.v_k_major = h.v.mn_major ? 0 : 1;
+  for (int d = 0; d < 5; ++d) { a.q_sel[d] = h.q.sel[d]; a.k_sel[d] = h.k.sel[d]; a.v_sel[d] = h.v.sel[d]; }
+  a.q_b0 = h.q.b0; a.k_b0 = h.k.b0; a.v_b0 = h.v.b0;
+  h.eligible = 1;
+  *ap = a;
+  *host = h;
+  return true;
+}
+
 static double gemm_flops(const GemmParams& g) {
   double f = 2.0 * double(g.batch) * g.M * double(g.N) * g.K;
   if (g.causal != CAUSAL_NONE) f *= 0.5 * (1.0 + 1.0 / std::max(1, g.M));
@@ -324,6 +358,16 @@ double node_cost(const fluid_plan_s* p, const Node& n, const int* lo) {
     case N_SELECT:
       if (!is_identity(p, n.a, lo) || !is_identity(p, n.out, lo)) return kInf;
       return kLaunch + 2.0 * tbytes(p, n.out) / kBw;
+    case N_ATTN: {
+      AttnParams ap;
+      AttnHost ah;
+      if (!lower_attn(p, n, lo, &ap, &ah)) return kInf;
+      double fl = 4.0 * ap.B * ap.NH * double(ap.S) * ap.S * ap.D;
+      if (ap.causal) fl *= 0.5;
+      const double by = tbytes(p, n.a) + tbytes(p, n.b) + tbytes(p, n.v) + tbytes(p, n.out);
+      // K or V with the sequence index contiguous cost a little more (transposed operand path)
+      return kLaunch + std::max(fl / (0.35 * kTcPeak), by / kBw) * (1.0 + 0.02 * (ap.k_mn_major + ap.v_k_major));
+    }
   }
   return kInf;
 }
@@ -448,6 +492,40 @@ static void build_nodes(fluid_plan_s* p, const std::vector<int>& order) {
             }
           }
         }
+        if (fuse && !p->opts.unfused_attention && op.kind == FLUID_OP_BMM_QK && g.tensors[n.out].dtype == FLUID_BF16 &&
+            tc_kernel_available() && p->opts.gemm_path != 1 &&
+            (g.tensors[n.a].dims[3] == 64 || g.tensors[n.a].dims[3] == 128)) {
+          const int c1 = sole_consumer(n.out);
+          if (c1 >= 0 && g.ops[c1].kind == FLUID_OP_SOFTMAX && (!g.ops[c1].attrs.causal ||
+                                                                g.tensors[n.out].dims[2] == g.tensors[n.out].dims[3])) {
+            const int sm_out = g.ops[c1].outs[0];
+            const int c2 = sole_consumer(sm_out);
+            if (c2 >= 0 && g.ops[c2].kind == FLUID_OP_BMM_PV && g.ops[c2].ins[0] == sm_out &&
+                g.ops[c2].ins[1] != sm_out && available_before(g.ops[c2].ins[1], oi) && op.attrs.scale * g.ops[c1].attrs.scale > 0) {
+              // only if the all-canonical layouts can be fed to the kernel (so that a plan always exists)
+              Node trial = n;
+              trial.kind = N_ATTN;
+              trial.v = g.ops[c2].ins[1];
+              trial.out = g.ops[c2].outs[0];
+              trial.scale = op.attrs.scale * g.ops[c1].attrs.scale;
+              trial.sm_causal = g.ops[c1].attrs.causal;
+              std::vector<int> canon(nt, 0);
+              AttnParams tap;
+              AttnHost tah;
+              if (!lower_attn(p, trial, canon.data(), &tap, &tah)) goto no_attention_fusion;
+              n.kind = N_ATTN;
+              n.v = g.ops[c2].ins[1];
+              n.scale = op.attrs.scale * g.ops[c1].attrs.scale;
+              n.sm_causal = g.ops[c1].attrs.causal;
+              absorbed[c1] = absorbed[c2] = 1;
+              n.ops.push_back(c1); n.ops.push_back(c2);
+              p->folded[n.out] = 1; p->folded[sm_out] = 1;
+              n.out = g.ops[c2].outs[0];
+              break;
+            }
+          }
+        }
+      no_attention_fusion:
         if (fuse && op.kind == FLUID_OP_BMM_QK) {
           int c = sole_consumer(n.out);
           if (c >= 0 && g.ops[c].kind == FLUID_OP_SOFTMAX && g.ops[c].attrs.causal &&
@@ -524,7 +602,7 @@ static void build_nodes(fluid_plan_s* p, const std::vector<int>& order) {
     if (n.ops.size() == 1) {
       for (int t : op.ins) add_in(t);
     } else {
-      add_in(n.a); add_in(n.b); add_in(n.bias); add_in(n.res); add_in(n.gamma); add_in(n.beta); add_in(n.pos);
+      add_in(n.a); add_in(n.b); add_in(n.v); add_in(n.bias); add_in(n.res); add_in(n.gamma); add_in(n.beta); add_in(n.pos);
     }
     n.outs.push_back(n.out);
     for (int o2 : n.ops) p->node_of_op[o2] = (int)p->nodes.size();

@@ -24,7 +24,7 @@ LIB_PATH = os.path.join(_HERE, "libfluid.so")
 FLUID_OK = 0
 FLUID_EINVAL, FLUID_EUNSUPPORTED, FLUID_EALIGN, FLUID_ECUDA, FLUID_ENOMEM, FLUID_ETIMEOUT = -1, -2, -3, -4, -5, -6
 ARENA_ALIGN, ARENA_HEADER, SLOT_ALIGN = 1024, 256, 256
-KERNEL_NAMES = ["EMBED", "NORM", "GEMM_SIMT", "GEMM_TC", "SOFTMAX", "ROPE", "ELTWISE", "PERMUTE", "SELECT_LAST"]
+KERNEL_NAMES = ["EMBED", "NORM", "GEMM_SIMT", "GEMM_TC", "SOFTMAX", "ROPE", "ELTWISE", "PERMUTE", "SELECT_LAST", "ATTN"]
 
 
 class FluidError(RuntimeError):
@@ -49,7 +49,7 @@ EVAL_FN = C.CFUNCTYPE(C.c_double, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.
 class PlanOptions(C.Structure):
     _fields_ = [("fusion", C.c_int32), ("arena_policy", C.c_int32), ("no_reuse", C.c_int32),
                 ("force_canonical", C.c_int32), ("gemm_path", C.c_int32), ("narrow_stream", C.c_int32),
-                ("reserved", C.c_int32 * 2),
+                ("unfused_attention", C.c_int32), ("reserved", C.c_int32 * 1),
                 ("eval", EVAL_FN), ("eval_user", C.c_void_p)]
 
 

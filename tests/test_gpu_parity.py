@@ -47,6 +47,7 @@ def test_small_models_planned_and_canonical(family, dtype):
                                ("canonical", None, {}),
                                ("unfused", synth.default_candidates(m.graph), {"fusion": 0}),
                                ("simt", synth.default_candidates(m.graph), {"gemm_path": 1}),
+                               ("unfused_attention", synth.default_candidates(m.graph), {"unfused_attention": 1}),
                                ("no_reuse", synth.default_candidates(m.graph), {"no_reuse": 1})]:
         got, plan, _ = run_gpu(m.graph, feeds, cands, **opts)
         for t in m.graph.outputs:
@@ -255,3 +256,42 @@ def test_run_allocates_nothing_and_rejects_bad_pointers():
         fluid.fluid_run(plan2.handle, r.arena.data_ptr(), [b.data_ptr() for b in r.inputs],
                         [b.data_ptr() for b in r.outputs])
     plan.close(); plan2.close()
+
+
+def _attention_graph(B, S, nh, D, causal, k_layout, v_layout, dtype=synth.BF16):
+    """q, k, v arrive as graph inputs in [B,S,nh,D]; k and v are first copied into a chosen physical
+    layout (a GELU-free pass-through would change values, so a TRANSPOSE pair pins the layout)."""
+    g = synth.GraphDesc()
+    q = g.tensor("q", dtype, [B, S, nh, D], synth.INPUT)
+    k = g.tensor("k", dtype, [B, S, nh, D], synth.INPUT)
+    v = g.tensor("v", dtype, [B, S, nh, D], synth.INPUT)
+    qh = g.tensor("qh", dtype, [B, nh, S, D]); g.op(synth.TRANSPOSE, [q], [qh], perm=[0, 2, 1, 3])
+    kT = g.tensor("kT", dtype, [B, nh, D, S]); g.op(synth.TRANSPOSE, [k], [kT], perm=[0, 2, 3, 1])
+    vh = g.tensor("vh", dtype, [B, nh, S, D]); g.op(synth.TRANSPOSE, [v], [vh], perm=[0, 2, 1, 3])
+    sc = g.tensor("sc", dtype, [B, nh, S, S]); g.op(synth.BMM_QK, [qh, kT], [sc], scale=1.0 / math.sqrt(D))
+    pr = g.tensor("pr", dtype, [B, nh, S, S]); g.op(synth.SOFTMAX, [sc], [pr], causal=int(causal), scale=1.0)
+    ch = g.tensor("ch", dtype, [B, nh, S, D]); g.op(synth.BMM_PV, [pr, vh], [ch])
+    out = g.tensor("out", dtype, [B, nh, S, D], synth.OUTPUT)
+    g.op(synth.ADD, [ch, ch], [out])
+    cands = synth.canonical_candidates(g)
+    cands[kT] = [(0, 1, 2, 3), k_layout] if k_layout != (0, 1, 2, 3) else [(0, 1, 2, 3)]
+    cands[vh] = [(0, 1, 2, 3), v_layout] if v_layout != (0, 1, 2, 3) else [(0, 1, 2, 3)]
+    return g, cands, (kT, vh)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("causal", [0, 1])
+@pytest.mark.parametrize("S", [8, 104, 128, 328])
+def test_fused_attention_shapes_and_operand_majors(D, causal, S):
+    """Ragged sequence lengths (one tile, partial tiles, several tiles) and both majors of K and V: the
+    canonical kT [B,nh,D,S] is sequence-contiguous, its aliasing layout is head-dim-contiguous."""
+    B, nh = 2, 3
+    for k_layout, v_layout in [((0, 1, 2, 3), (0, 1, 2, 3)), ((0, 3, 1, 2), (0, 2, 1, 3)), ((0, 1, 2, 3), (0, 1, 3, 2))]:
+        g, cands, _ = _attention_graph(B, S, nh, D, causal, k_layout, v_layout)
+        feeds = {t: rand_feed([B, S, nh, D], synth.BF16, 20 + t, -2.0, 2.0) for t in g.inputs}
+        ref = run_oracle(g, feeds)[g.outputs[0]]
+        opts = {"force_canonical": 1} if k_layout == (0, 1, 2, 3) and v_layout == (0, 1, 2, 3) else {}
+        got, plan, _ = run_gpu(g, feeds, cands, **opts)
+        assert "ATTN" in [s["kernel_name"] for s in plan.steps()]
+        assert_close(got[g.outputs[0]], ref, synth.BF16, f"attention D={D} S={S} causal={causal} k={k_layout} v={v_layout}")
+        plan.close()

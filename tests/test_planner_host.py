@@ -208,3 +208,28 @@ def test_residual_stream_is_held_in_fp32():
     twins = {enc.graph.tensors[r["tensor"]]["name"] for r in ep.records() if r["twin"]}
     assert "emb_ln.out" in twins and "l0.ln1.out" in twins       # post-LN: stream value also feeds GEMMs
     plan.close(); narrow.close(); ep.close()
+
+
+def test_attention_chain_becomes_one_step_and_frees_the_score_tensors():
+    for name, arena_cap_mb in [("gpt2_small", 60), ("llama", 200)]:
+        m = synth.build_model(synth.CONFIGS[name], materialize=False)
+        d = m.graph
+        fused = fluid.Plan(d, synth.default_candidates(d))
+        unfused = fluid.Plan(d, synth.default_candidates(d), unfused_attention=1)
+        attn = [s for s in fused.steps() if s["kernel_name"] == "ATTN"]
+        assert len(attn) == m.cfg.L and all(len(s["ops"]) == 3 for s in attn)
+        assert [d.ops[o]["kind"] for o in attn[0]["ops"]] == [synth.BMM_QK, synth.SOFTMAX, synth.BMM_PV]
+        assert "SOFTMAX" not in [s["kernel_name"] for s in fused.steps()]
+        assert "ATTN" not in [s["kernel_name"] for s in unfused.steps()]
+        # scores and probabilities no longer exist as arena slices
+        names = {d.tensors[r["tensor"]]["name"] for r in fused.records()}
+        assert not any(n.endswith("scores") or n.endswith("probs") for n in names)
+        assert fused.arena_bytes < arena_cap_mb * 2 ** 20 < unfused.arena_bytes
+        recs, offs = plan_records(fused)
+        assert OA.check_arena(recs, offs, fused.arena_bytes) == []
+        fused.close(); unfused.close()
+    # head dims the tensor-core attention kernel does not take stay unfused
+    t = synth.build_model(synth.scaled(synth.CONFIGS["bert_base"], L=1, H=96, nh=2), materialize=False)   # D = 48
+    p = fluid.Plan(t.graph, synth.default_candidates(t.graph))
+    assert "ATTN" not in [s["kernel_name"] for s in p.steps()] and "SOFTMAX" in [s["kernel_name"] for s in p.steps()]
+    p.close()
