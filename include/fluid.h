@@ -119,7 +119,9 @@ typedef struct fluid_plan_options {
                                arena, with a bf16 twin where a GEMM also reads them; 1 = every
                                activation is held in its declared dtype */
   int32_t unfused_attention; /* 1: keep BMM_QK -> SOFTMAX -> BMM_PV as three steps even when fusion is on */
-  int32_t reserved[1];
+  int32_t split_k;          /* 1: GEMM steps with few output tiles and a long k range cut it across CTAs;
+                               the fp32 partial tiles take a scratch slice of the arena for that step.
+                               0 (default): never, the arena holds activations only */
   fluid_eval_fn eval;       /* NULL: built-in analytic B200 cost table */
   void* eval_user;
 } fluid_plan_options;
@@ -132,7 +134,8 @@ typedef enum {
 
 typedef struct fluid_step_info {
   int32_t kernel;        /* fluid_kernel_id */
-  int32_t variant;       /* kernel-specific (GEMM: bit0 A MN-major, bit1 B MN-major, bits 8.. tile N) */
+  int32_t variant;       /* kernel-specific (GEMM: bit0 A MN-major, bit1 B MN-major, bits 8-19 tile N,
+                            bits 20-23 grouped siblings, bits 24-27 split-K factor) */
   int32_t n_ops;         /* graph ops folded into this step */
   int32_t ops[8];
   int32_t n_in, n_out;   /* tensors read / written (graph tensor ids) */
@@ -179,9 +182,10 @@ FLUID_API double fluid_plan_canonical_cost(const fluid_plan_t* plan);
 FLUID_API int fluid_plan_tensor_info(const fluid_plan_t* plan, int tensor_id, int* layout_index, int* perm,
                            int64_t* offset, int64_t* bytes, int* first_step, int* last_step,
                            int* alias_of);
-/* Arena slices. A tensor held in fp32 with a bf16 twin owns two slices. record_id is unique
- * (tensor id, or tensor id + number of tensors for a twin); storage_dtype is the fluid_dtype the
- * slice holds. Any out pointer may be NULL. */
+/* Arena slices. A tensor held in fp32 with a bf16 twin owns two slices; a GEMM step that splits its
+ * k range across CTAs owns a scratch slice alive during that step only (tensor_id -1). record_id is
+ * unique (tensor id; tensor id + number of tensors for a twin; 2 * number of tensors + step for
+ * scratch); storage_dtype is the fluid_dtype the slice holds. Any out pointer may be NULL. */
 FLUID_API int fluid_plan_num_records(const fluid_plan_t* plan);
 FLUID_API int fluid_plan_record_info(const fluid_plan_t* plan, int index, int* record_id, int* tensor_id,
                            int* is_twin, int* storage_dtype, int64_t* offset, int64_t* bytes,

@@ -77,6 +77,7 @@ int finalize_steps(fluid_plan_s* p) {
           s.bytes += es * (b + c + (g.has_bias ? g.N : 0));
         }
         if (s.nodes.size() > 1) s.variant |= int(s.nodes.size()) << 20;
+        if (s.split_k > 1) s.variant |= s.split_k << 24;
         break;
       }
       case N_NORM: {
@@ -361,7 +362,10 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
             gs[gi].bias = R(s.x_ptr[gi - 1][2]);
             gs[gi].R = nullptr;
           }
-          if (R.ok) err = launch_gemm_tc(gs, ts, ng, status, stream);
+          float* partial = s.scratch_record >= 0
+                               ? reinterpret_cast<float*>(static_cast<char*>(arena_ptr) + p->records[s.scratch_record].offset)
+                               : nullptr;
+          if (R.ok) err = launch_gemm_tc(gs, ts, ng, s.split_k, partial, status, stream);
         } else if (R.ok) {
           err = launch_gemm_simt(q, stream);
         }

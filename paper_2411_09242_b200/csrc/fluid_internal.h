@@ -79,6 +79,9 @@ struct Step {
   GemmParams gemm_x[2]{};   // groups 1 and 2 of a grouped GEMM step
   GemmTcHost tc_x[2]{};
   int x_ptr[2][3] = {{-1, -1, -1}, {-1, -1, -1}};  // tensor ids of B, C, bias for groups 1 and 2
+  int split_k = 1;          // GEMM steps with few tiles cut their k range across CTAs
+  int64_t scratch_bytes = 0;
+  int scratch_record = -1;  // arena slice holding the split-K partial tiles (alive during this step only)
   NormParams norm{};
   SoftmaxParams softmax{};
   RopeParams rope{};
@@ -99,6 +102,7 @@ struct ArenaRecord {
   int64_t offset = -1;
   int id = -1;    // root, or root + number of tensors for a twin
   int twin = 0;   // 1: the bf16 copy of a tensor whose primary storage is fp32
+  int step = -1;  // >= 0: per-step scratch (root is -1)
 };
 
 }  // namespace fluid

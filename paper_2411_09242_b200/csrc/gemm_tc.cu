@@ -42,9 +42,12 @@ struct TcParams {
   int tiles_per_group;
   GemmTcCfg cfg;
   int tiles_m, tiles_n;
-  int num_tiles;
+  int num_tiles;        // work items = output tiles x split_k
   int tiles_per_batch;
-  uint32_t* status;
+  int split_k;          // >1: each output tile's k range is cut in split_k pieces run by different CTAs
+  int ksteps_per_split;
+  float* partial;       // split-K scratch: [tile][split][bn/4][128 rows][4] fp32
+  uint32_t* status;     // word 0: device status; words 8..63: per-tile arrival counters for split-K
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -157,6 +160,16 @@ __device__ __forceinline__ int k_steps_of(const TcParams& p, int mt) {
   return (kend + BK - 1) / BK;
 }
 
+// work item -> output tile and its k-step range [k_begin, k_begin + count)
+__device__ __forceinline__ void decode_item(const TcParams& p, int item, int& tile, int& sp, int& k_begin, int& count, int mt_hint = -1) {
+  if (p.split_k <= 1) { tile = item; sp = 0; k_begin = 0; count = -1; return; }
+  tile = item / p.split_k;
+  sp = item - tile * p.split_k;
+  const int total = (p.g.K + BK - 1) / BK;
+  k_begin = sp * p.ksteps_per_split;
+  count = min(p.ksteps_per_split, total - k_begin);
+}
+
 __device__ __forceinline__ void fill_coords(const int* sel, int rank, int k0, int k1, int r0, int r1, int b0, int b1, int* c) {
 #pragma unroll
   for (int d = 0; d < 5; ++d) {
@@ -189,11 +202,14 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
 // Vector epilogue for one 32-column chunk of one accumulator row. Preconditions (checked on the
 // host): the n index is contiguous in C (and R), every 8-column group is 16-byte aligned and
 // never straddles an n split, N is a multiple of 8.
+// With `partial` set (the last-arriving CTA of a split-K tile) the accumulator chunk is the sum, in
+// split order, of the partial tiles in scratch memory instead of a tensor-memory load.
 template <int ACT, bool HAS_RES, bool C_WIDE, bool R_WIDE>
 __device__ __forceinline__ void epilogue_chunk_vec(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb,
-                                                   int64_t rb, int n) {
+                                                   int64_t rb, int n, const float* partial = nullptr, int split_k = 1,
+                                                   size_t split_stride = 0) {
   uint32_t r[32];
-  tmem_ld32(taddr, r);
+  if (!partial) tmem_ld32(taddr, r);
   // group offsets (an 8-column group shares one n split)
   int64_t co[4], ro[4];
   int n1, n0i;
@@ -221,7 +237,24 @@ __device__ __forceinline__ void epilogue_chunk_vec(const GemmParams& g, uint32_t
       }
     }
   }
-  tmem_ld_wait();
+  if (!partial) {
+    tmem_ld_wait();
+  } else {
+    // partial + (c4 * 128 + row) * 4 floats; `partial` already points at this row's first chunk
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = 0;
+    for (int sp = 0; sp < split_k; ++sp) {
+      const float* src = partial + sp * split_stride;
+#pragma unroll
+      for (int c4 = 0; c4 < 8; ++c4) {
+        const float4 f = __ldcg(reinterpret_cast<const float4*>(src + (size_t)c4 * 512));
+        r[4 * c4] = __float_as_uint(__uint_as_float(r[4 * c4]) + f.x);
+        r[4 * c4 + 1] = __float_as_uint(__uint_as_float(r[4 * c4 + 1]) + f.y);
+        r[4 * c4 + 2] = __float_as_uint(__uint_as_float(r[4 * c4 + 2]) + f.z);
+        r[4 * c4 + 3] = __float_as_uint(__uint_as_float(r[4 * c4 + 3]) + f.w);
+      }
+    }
+  }
   if (!row_ok) return;
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
@@ -293,13 +326,14 @@ __device__ __noinline__ void epilogue_group_any(const GemmParams& g, uint32_t ta
 enum EpiKind { EPI_ANY = 0, EPI_PLAIN = 1, EPI_PLAIN_WIDE = 2, EPI_RES = 3, EPI_RES_WIDE = 4, EPI_GELU_ERF = 5, EPI_GELU_TANH = 6 };
 
 template <int EPI>
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb, int64_t rb, int n) {
-  if (EPI == EPI_PLAIN) epilogue_chunk_vec<ACT_NONE, false, false, false>(g, taddr, row_ok, cb, rb, n);
-  else if (EPI == EPI_PLAIN_WIDE) epilogue_chunk_vec<ACT_NONE, false, true, false>(g, taddr, row_ok, cb, rb, n);
-  else if (EPI == EPI_RES) epilogue_chunk_vec<ACT_NONE, true, false, false>(g, taddr, row_ok, cb, rb, n);
-  else if (EPI == EPI_RES_WIDE) epilogue_chunk_vec<ACT_NONE, true, true, true>(g, taddr, row_ok, cb, rb, n);
-  else if (EPI == EPI_GELU_ERF) epilogue_chunk_vec<ACT_GELU_ERF, false, false, false>(g, taddr, row_ok, cb, rb, n);
-  else if (EPI == EPI_GELU_TANH) epilogue_chunk_vec<ACT_GELU_TANH, false, false, false>(g, taddr, row_ok, cb, rb, n);
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb, int64_t rb, int n,
+                                               const float* partial = nullptr, int sk = 1, size_t ss = 0) {
+  if (EPI == EPI_PLAIN) epilogue_chunk_vec<ACT_NONE, false, false, false>(g, taddr, row_ok, cb, rb, n, partial, sk, ss);
+  else if (EPI == EPI_PLAIN_WIDE) epilogue_chunk_vec<ACT_NONE, false, true, false>(g, taddr, row_ok, cb, rb, n, partial, sk, ss);
+  else if (EPI == EPI_RES) epilogue_chunk_vec<ACT_NONE, true, false, false>(g, taddr, row_ok, cb, rb, n, partial, sk, ss);
+  else if (EPI == EPI_RES_WIDE) epilogue_chunk_vec<ACT_NONE, true, true, true>(g, taddr, row_ok, cb, rb, n, partial, sk, ss);
+  else if (EPI == EPI_GELU_ERF) epilogue_chunk_vec<ACT_GELU_ERF, false, false, false>(g, taddr, row_ok, cb, rb, n, partial, sk, ss);
+  else if (EPI == EPI_GELU_TANH) epilogue_chunk_vec<ACT_GELU_TANH, false, false, false>(g, taddr, row_ok, cb, rb, n, partial, sk, ss);
   else {
 #pragma unroll 1
     for (int q = 0; q < 4; ++q) {
@@ -367,10 +401,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (p.cfg.b_sel[d] == 0) b_kd0 = d;
         if (p.cfg.b_sel[d] == 1) b_kd1 = d;
       }
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+      for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
+        int tile, sp, k_begin, k_count;
+        decode_item(p, item, tile, sp, k_begin, k_count);
         int grp, bz, mt, nt;
         decode_tile(p, tile, grp, bz, mt, nt);
-        const int ksteps = k_steps_of(p, mt);
+        const int ksteps = k_count >= 0 ? k_count : k_steps_of(p, mt);
         int ca[2][5], cb[4][5];  // fully unrolled below: these stay in registers
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
@@ -387,7 +423,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           fill_coords(p.cfg.b_sel, 5, 0, 0, r0, r1, b0, b1, cb[ch]);
         }
         const CUtensorMap* mapb = grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2);
-        int ak0 = 0, ak1 = 0, bk0 = 0, bk1 = 0;  // running split of the k index for each operand
+        int ak0, ak1, bk0, bk1;  // running split of the k index for each operand
+        split2(k_begin * BK, p.cfg.a_k0, ak1, ak0);
+        split2(k_begin * BK, p.cfg.b_k0, bk1, bk0);
         for (int ks = 0; ks < ksteps; ++ks) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u)) { ok = false; break; }
           const uint32_t fb = full_bar(s);
@@ -436,10 +474,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+      for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
+        int tile, sp, k_begin, k_count;
+        decode_item(p, item, tile, sp, k_begin, k_count);
         int grp, bz, mt, nt;
         decode_tile(p, tile, grp, bz, mt, nt);
-        const int ksteps = k_steps_of(p, mt);
+        const int ksteps = k_count >= 0 ? k_count : k_steps_of(p, mt);
         if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_c = tmem_base + uint32_t(acc * bn);
@@ -474,7 +514,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint32_t acc_ph = 0;
     bool ok = true;
     pdl_wait();  // before any global read (bias, residual) or write (C)
-    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+    for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
+      int tile, sp, k_begin, k_count;
+      decode_item(p, item, tile, sp, k_begin, k_count);
       int grp, bz, mt, nt;
       decode_tile(p, tile, grp, bz, mt, nt);
       const GemmParams& g = grp == 0 ? p.g : p.gx[grp - 1];
@@ -486,14 +528,53 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn);
+      if (p.split_k <= 1) {
 #pragma unroll 1
-      for (int c0 = col_begin; c0 < col_end; c0 += 32) {
-        if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
-        epilogue_chunk<EPI>(g, trow + uint32_t(c0), row_ok, cb, rb, n_tile0 + c0);
+        for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+          if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
+          epilogue_chunk<EPI>(g, trow + uint32_t(c0), row_ok, cb, rb, n_tile0 + c0);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+      } else {
+        // ---- split-K: park this CTA's partial tile, the last CTA to arrive adds them up ----
+        const size_t tile_floats = size_t(BM) * bn;
+        float* mine = p.partial + (size_t(tile) * p.split_k + sp) * tile_floats + size_t(lane_base + lane) * 4;
+#pragma unroll 1
+        for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(trow + uint32_t(c0), r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4)
+            __stcg(reinterpret_cast<float4*>(mine + size_t(c0 / 4 + c4) * 512),
+                   make_float4(__uint_as_float(r[4 * c4]), __uint_as_float(r[4 * c4 + 1]), __uint_as_float(r[4 * c4 + 2]),
+                               __uint_as_float(r[4 * c4 + 3])));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));   // the accumulator is free again
+        __threadfence();
+        asm volatile("bar.sync 1, 256;" ::: "memory");      // all eight epilogue warps have stored
+        if (warp == 2 && lane == 0) {
+          const uint32_t prev = atomicAdd(p.status + 8 + tile, 1u);
+          *reinterpret_cast<volatile uint32_t*>(abort_flag + 1) = prev;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        const bool last = *reinterpret_cast<volatile uint32_t*>(abort_flag + 1) == uint32_t(p.split_k - 1);
+        if (last) {
+          __threadfence();
+          const float* base_row = p.partial + size_t(tile) * p.split_k * tile_floats + size_t(lane_base + lane) * 4;
+#pragma unroll 1
+          for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+            if (n_tile0 + c0 >= g.N) break;
+            epilogue_chunk<EPI>(g, 0u, row_ok, cb, rb, n_tile0 + c0, base_row + size_t(c0 / 4) * 512, p.split_k, tile_floats);
+          }
+          if (warp == 2 && lane == 0) p.status[8 + tile] = 0;   // ready for the next launch
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");      // the exchange word is reused by the next item
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
     if (!ok && lane == 0) {
@@ -560,8 +641,46 @@ int encode_tensor_map(TensorMapStorage* out, const void* base, const TmaOperand&
   return rc == CUDA_SUCCESS ? 0 : -2;
 }
 
-cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_group, uint32_t* status,
-                           cudaStream_t stream) {
+static bool vec_epilogue_ok(const GemmParams* gs, int n_group, bool check_pointers) {
+  auto mult8 = [](int64_t v) { return (v & 7) == 0; };
+  const GemmParams& g = gs[0];
+  bool vec = true;
+  for (int i = 0; i < n_group; ++i) {
+    const GemmParams& q = gs[i];
+    vec = vec && q.c_s[5] == 1 && (q.N & 7) == 0 && (q.N0 & 7) == 0 && mult8(q.c_s[0]) && mult8(q.c_s[1]) && mult8(q.c_s[2]) &&
+          mult8(q.c_s[3]) && mult8(q.c_s[4]) && q.c_f32 == g.c_f32;
+    if (check_pointers)
+      vec = vec && (reinterpret_cast<uintptr_t>(q.C) & 15) == 0 && (!q.has_bias || (reinterpret_cast<uintptr_t>(q.bias) & 15) == 0);
+  }
+  if (g.has_res) {
+    vec = vec && g.r_s[5] == 1 && mult8(g.r_s[0]) && mult8(g.r_s[1]) && mult8(g.r_s[2]) && mult8(g.r_s[3]) && mult8(g.r_s[4]);
+    if (check_pointers) vec = vec && (reinterpret_cast<uintptr_t>(g.R) & 15) == 0;
+    vec = vec && g.act == ACT_NONE && g.c_f32 == g.r_f32;
+  } else if (g.act != ACT_NONE) {
+    vec = vec && !g.c_f32;
+  }
+  return vec;
+}
+
+int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t* scratch_bytes) {
+  *scratch_bytes = 0;
+  if (g.causal != CAUSAL_NONE) return 1;
+  GemmParams gs[3] = {g, g, g};
+  if (!vec_epilogue_ok(gs, 1, false)) return 1;
+  const int64_t tiles = int64_t((g.M + BM - 1) / BM) * ((g.N + tc.cfg.bn - 1) / tc.cfg.bn) * g.batch * n_group;
+  const int ksteps = (g.K + BK - 1) / BK;
+  if (tiles > 56 || tiles * 2 > sm_count() || ksteps < 16) return 1;
+  int sk = (int)std::min<int64_t>(std::min<int64_t>(8, sm_count() / tiles), ksteps / 4);
+  if (sk < 2) return 1;
+  const int per = (ksteps + sk - 1) / sk;
+  sk = (ksteps + per - 1) / per;   // no empty split
+  if (sk < 2) return 1;
+  *scratch_bytes = tiles * sk * int64_t(BM) * tc.cfg.bn * 4;
+  return sk;
+}
+
+cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_group, int split_k, float* partial,
+                           uint32_t* status, cudaStream_t stream) {
   const GemmParams& g = gs[0];
   const GemmTcHost& tc = tcs[0];
   TcParams p;
@@ -583,25 +702,26 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
   p.num_tiles = p.tiles_per_group * n_group;
   p.status = status;
   const size_t smem = size_t(tc.cfg.stages) * (kATileBytes + size_t(tc.cfg.bn) * BK * 2) + 1024 + 8 * (2 * tc.cfg.stages + 4) + 16;
-  const int grid = std::min(p.num_tiles, sm_count());
-  if (grid <= 0) return cudaSuccess;
   const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(&tc.map_a);
   const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(&tc.map_b);
   const CUtensorMap* mb1 = reinterpret_cast<const CUtensorMap*>(&tcs[n_group > 1 ? 1 : 0].map_b);
   const CUtensorMap* mb2 = reinterpret_cast<const CUtensorMap*>(&tcs[n_group > 2 ? 2 : 0].map_b);
   // The vector epilogues need: n contiguous in C (and R), 8-column groups aligned to 16 bytes and
   // inside one n split, N a multiple of 8. Everything else takes the general epilogue.
-  auto mult8 = [](int64_t v) { return (v & 7) == 0; };
-  bool vec = true;
-  for (int i = 0; i < n_group; ++i) {
-    const GemmParams& q = gs[i];
-    vec = vec && q.c_s[5] == 1 && (q.N & 7) == 0 && (q.N0 & 7) == 0 && mult8(q.c_s[0]) && mult8(q.c_s[1]) && mult8(q.c_s[2]) &&
-          mult8(q.c_s[3]) && mult8(q.c_s[4]) && (reinterpret_cast<uintptr_t>(q.C) & 15) == 0 &&
-          (!q.has_bias || (reinterpret_cast<uintptr_t>(q.bias) & 15) == 0) && q.c_f32 == g.c_f32;
+  const bool vec = vec_epilogue_ok(gs, n_group, true);
+  if (!vec || !partial) split_k = 1;   // the general epilogue does not take part in split-K
+  p.split_k = split_k;
+  p.partial = partial;
+  {
+    const int ksteps = (g.K + BK - 1) / BK;
+    p.ksteps_per_split = (ksteps + split_k - 1) / split_k;
+    if (split_k > 1) {
+      if (p.num_tiles > 56) return cudaErrorInvalidValue;
+      p.num_tiles *= split_k;
+    }
   }
-  if (g.has_res)
-    vec = vec && g.r_s[5] == 1 && mult8(g.r_s[0]) && mult8(g.r_s[1]) && mult8(g.r_s[2]) && mult8(g.r_s[3]) &&
-          mult8(g.r_s[4]) && (reinterpret_cast<uintptr_t>(g.R) & 15) == 0;
+  const int grid = std::min(p.num_tiles, sm_count());
+  if (grid <= 0) return cudaSuccess;
   int epi = EPI_ANY;
   if (vec) {
     if (g.act == ACT_NONE && !g.has_res) epi = g.c_f32 ? EPI_PLAIN_WIDE : EPI_PLAIN;

@@ -164,8 +164,13 @@ struct AttnHost {
 cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
 // n_group (1..3) GEMMs that share the A operand, the shapes and the tile configuration run as one
 // launch (sibling projections such as Q/K/V or gate/up); group i uses g[i] and tc[i].map_b.
-cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, uint32_t* status,
-                           cudaStream_t stream);
+// split_k > 1 cuts every output tile's k range into split_k pieces run by different CTAs; `partial`
+// then points at n_tiles * split_k * 128 * bn floats of scratch and status[8..63] hold the per-tile
+// arrival counters (zero before the launch, left zero after it).
+cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, int split_k, float* partial,
+                           uint32_t* status, cudaStream_t stream);
+// Split factor a GEMM step should use (1 = none) and the scratch it then needs.
+int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t* scratch_bytes);
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);
 cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t stream);

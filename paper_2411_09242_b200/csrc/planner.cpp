@@ -1026,6 +1026,32 @@ static int lower_and_place(fluid_plan_s* p) {
       p->records.push_back(w);
     }
   }
+  // per-step scratch: split-K partial tiles of GEMM steps with too few output tiles to fill the GPU
+  for (int si = 0; si < (int)p->steps.size(); ++si) {
+    Step& st = p->steps[si];
+    const Node& n0 = p->nodes[st.node];
+    if (n0.kind != N_GEMM || !p->opts.split_k) continue;
+    GemmParams g;
+    GemmTcHost tc;
+    if (!lower_gemm(p, n0, lo, &g) || !gemm_tc_eligible(p, g, &tc)) continue;
+    g.c_f32 = p->wide[n0.out];
+    g.r_f32 = n0.res >= 0 ? p->wide[n0.res] : 0;
+    bool same_width = true;
+    for (int nj : st.nodes) same_width = same_width && p->wide[p->nodes[nj].out] == p->wide[n0.out];
+    if (!same_width) continue;
+    int64_t bytes = 0;
+    st.split_k = gemm_split_k(g, tc, (int)st.nodes.size(), &bytes);
+    if (st.split_k <= 1) continue;
+    ArenaRecord r;
+    r.root = -1;
+    r.step = si;
+    r.id = 2 * nt + si;
+    r.bytes = round_up(bytes, FLUID_SLOT_ALIGN);
+    r.first = r.last = si;
+    st.scratch_bytes = r.bytes;
+    st.scratch_record = (int)p->records.size();
+    p->records.push_back(r);
+  }
   greedy_by_size(p->records, p->opts.arena_policy, p->opts.no_reuse != 0, &p->arena_bytes);
   // reference figures: one slice per tensor, and the largest live set
   int64_t naive = FLUID_ARENA_HEADER, live = 0;
@@ -1179,7 +1205,7 @@ int fluid_plan_record_info(const fluid_plan_t* p, int index, int* record_id, int
   if (record_id) *record_id = r.id;
   if (tensor_id) *tensor_id = r.root;
   if (is_twin) *is_twin = r.twin;
-  if (storage_dtype) *storage_dtype = (p->wide[r.root] && !r.twin) ? FLUID_F32 : p->graph.tensors[r.root].dtype;
+  if (storage_dtype) *storage_dtype = r.root < 0 ? FLUID_F32 : ((p->wide[r.root] && !r.twin) ? FLUID_F32 : p->graph.tensors[r.root].dtype);
   if (offset) *offset = r.offset;
   if (bytes) *bytes = r.bytes;
   if (first_step) *first_step = r.first;

@@ -49,7 +49,7 @@ EVAL_FN = C.CFUNCTYPE(C.c_double, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.
 class PlanOptions(C.Structure):
     _fields_ = [("fusion", C.c_int32), ("arena_policy", C.c_int32), ("no_reuse", C.c_int32),
                 ("force_canonical", C.c_int32), ("gemm_path", C.c_int32), ("narrow_stream", C.c_int32),
-                ("unfused_attention", C.c_int32), ("reserved", C.c_int32 * 1),
+                ("unfused_attention", C.c_int32), ("split_k", C.c_int32),
                 ("eval", EVAL_FN), ("eval_user", C.c_void_p)]
 
 

@@ -106,7 +106,7 @@ def test_model_graph_sequences_match_oracle(name):
 def test_arena_matches_greedy_by_size_oracle(name, policy):
     cfg = synth.CONFIGS[name]
     m = synth.build_model(synth.scaled(cfg, L=min(cfg.L, 3)), materialize=False)
-    plan = fluid.Plan(m.graph, synth.default_candidates(m.graph), arena_policy=policy)
+    plan = fluid.Plan(m.graph, synth.default_candidates(m.graph), arena_policy=policy, split_k=policy)
     recs, offs = plan_records(plan)
     assert len(recs) > 5
     want, peak = OA.greedy_by_size(recs, policy="best" if policy else "first")
@@ -119,6 +119,9 @@ def test_arena_matches_greedy_by_size_oracle(name, policy):
     steps = plan.steps()
     nt = len(m.graph.tensors)
     for rid, _, first, last in recs:
+        if rid >= 2 * nt:
+            assert first == last == rid - 2 * nt      # per-step scratch lives during its step only
+            continue
         tid = rid % nt
         group = [t for t in range(nt) if plan.tensor_info(t).alias_of == tid]
         touched = [i for i, s in enumerate(steps) if set(group) & set(s["ins"] + s["outs"])]
@@ -233,3 +236,19 @@ def test_attention_chain_becomes_one_step_and_frees_the_score_tensors():
     p = fluid.Plan(t.graph, synth.default_candidates(t.graph))
     assert "ATTN" not in [s["kernel_name"] for s in p.steps()] and "SOFTMAX" in [s["kernel_name"] for s in p.steps()]
     p.close()
+
+
+def test_split_k_takes_a_step_lifetime_scratch_slice():
+    m = synth.build_model(synth.scaled(synth.CONFIGS["bert_base"], L=1), materialize=False)
+    d = m.graph
+    off = fluid.Plan(d, synth.default_candidates(d))
+    on = fluid.Plan(d, synth.default_candidates(d), split_k=1)
+    assert not any(r["tensor"] < 0 for r in off.records())
+    scratch = [r for r in on.records() if r["tensor"] < 0]
+    split_steps = [i for i, s in enumerate(on.steps()) if s["kernel_name"] == "GEMM_TC" and (s["variant"] >> 24) > 1]
+    assert len(scratch) == len(split_steps) >= 1
+    assert sorted(r["first"] for r in scratch) == split_steps and all(r["first"] == r["last"] for r in scratch)
+    recs, offs = plan_records(on)
+    assert OA.check_arena(recs, offs, on.arena_bytes) == []
+    assert on.arena_bytes >= off.arena_bytes
+    off.close(); on.close()
