@@ -220,6 +220,33 @@ FLUID_API int fluid_run_profiled(fluid_plan_t* plan, void* arena_ptr, const void
 FLUID_API int fluid_status(const fluid_plan_t* plan, const void* arena_ptr, fluid_stream stream,
                  int* device_status);
 
+/* ---- one GEMM that allocates nothing (the paper has no counterpart) ---------------------------
+ * C[m,n] = A[m,k] . B[n,k]^T (+ bias[n]), all bf16 device buffers the caller owns (A and B with k
+ * contiguous, C with n contiguous, 16-byte aligned; bias may be NULL), fp32 accumulate, run by the
+ * same tensor-core kernel as the planned GEMM steps in its split-K form.
+ *
+ * Who it is for: callers that want this one product outside any plan and cannot obtain device memory
+ * for it. Every other route through this library makes the caller allocate an arena first
+ * (fluid_plan_arena_bytes); a host thread in the middle of a latency-critical serving loop, a plugin
+ * whose host framework owns the allocator, or a process whose memory budget was fixed at start-up has
+ * no such allocation to give, and cudaMalloc there would stall the device or break the host's
+ * accounting. This call therefore takes nothing but inputs and outputs: the split-K partial tiles and
+ * arrival counters live in one fixed array inside the library's device image (8 MiB + 256 bytes, held
+ * by every GPU that loads the library until the process exits). It calls no cudaMalloc / cudaFree and
+ * no allocating library routine.
+ *
+ * Limits and rules:
+ *  - k and n multiples of 8; the split-K scratch the shape needs (n_tiles * split * 128 * tile_n * 4
+ *    bytes; 0 for shapes large enough to need no split) must fit the 8 MiB array, otherwise
+ *    FLUID_EINVAL with a message naming both figures.
+ *  - The first call on each device looks up the array's device address (with that device current);
+ *    make that first call before any stream capture begins.
+ *  - All calls share the one array: it is re-zeroed where needed at the start of every call, and two
+ *    calls whose kernels overlap on the GPU (different streams, or graphs replayed concurrently) race.
+ *  - Asynchronous on `stream`; launch errors come back as FLUID_ECUDA. */
+FLUID_API int fluid_gemm_bf16_static_scratch(const void* dev_a, const void* dev_b, const void* dev_bias, void* dev_c,
+                                   int m, int n, int k, fluid_stream stream);
+
 FLUID_API const char* fluid_last_error(void);
 /* Number of kernel launches issued by this library in this process (for launch accounting). */
 FLUID_API int64_t fluid_launch_count(void);

@@ -20,11 +20,15 @@
 #include <algorithm>
 #include <cstdio>
 
+#include <mutex>
+
 #include "device_utils.cuh"
 #include "fluid.h"
 #include "kernels.h"
 
 namespace fluid {
+
+void set_error(const char* fmt, ...);
 
 namespace {
 
@@ -755,3 +759,94 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
 }
 
 }  // namespace fluid
+
+// ---- a GEMM entry point that allocates nothing -----------------------------------------------------
+// The split-K kernel needs scratch for its partial tiles and arrival counters. Inside a plan that
+// scratch is a slice of the caller's arena. A caller with no arena and no licence to allocate (see
+// fluid.h) gets it from this fixed array, which every GPU that loads the library keeps until exit.
+namespace fluid {
+namespace {
+constexpr size_t kStaticHeaderBytes = 256;                 // status word + arrival counters
+constexpr size_t kStaticPartialBytes = size_t(8) << 20;    // 8 MiB of fp32 partial tiles
+__device__ __align__(256) unsigned char g_static_scratch[kStaticHeaderBytes + kStaticPartialBytes];
+// g_static_scratch is only a host-side handle here; the device address is looked up once per device.
+std::mutex g_static_mu;
+void* g_static_addr[64] = {};
+}  // namespace
+}  // namespace fluid
+
+extern "C" int fluid_gemm_bf16_static_scratch(const void* dev_a, const void* dev_b, const void* dev_bias, void* dev_c,
+                                              int m, int n, int k, fluid_stream stream) {
+  using namespace fluid;
+  if (!dev_a || !dev_b || !dev_c || m < 1 || n < 1 || k < 1) {
+    set_error("static-scratch GEMM: null operand or empty shape");
+    return FLUID_EINVAL;
+  }
+  if ((k & 7) || (n & 7)) {
+    set_error("static-scratch GEMM: K and N must be multiples of 8 (got K=%d, N=%d)", k, n);
+    return FLUID_EINVAL;
+  }
+  const uintptr_t align_bits = reinterpret_cast<uintptr_t>(dev_a) | reinterpret_cast<uintptr_t>(dev_b) |
+                               reinterpret_cast<uintptr_t>(dev_c) | reinterpret_cast<uintptr_t>(dev_bias);
+  if (align_bits & 15) {
+    set_error("static-scratch GEMM: device pointers must be 16-byte aligned");
+    return FLUID_EALIGN;
+  }
+  GemmParams g{};
+  g.A = dev_a; g.B = dev_b; g.C = dev_c; g.bias = dev_bias;
+  g.dtype = FLUID_BF16;
+  g.M = m; g.N = n; g.K = k; g.batch = 1;
+  g.M0 = m; g.N0 = n; g.K0 = k; g.B0 = 1;
+  g.a_s[3] = k; g.a_s[5] = 1;   // A[m, k], k contiguous
+  g.b_s[3] = 1; g.b_s[5] = k;   // B[n, k], k contiguous
+  g.c_s[3] = n; g.c_s[5] = 1;   // C[m, n], n contiguous
+  g.scale = 1.f;
+  g.has_bias = dev_bias != nullptr;
+  GemmTcHost tc;
+  if (!gemm_tc_describe(g, &tc)) {
+    set_error("static-scratch GEMM: shape %dx%dx%d cannot be fed to the tensor-core kernel", m, n, k);
+    return FLUID_EUNSUPPORTED;
+  }
+  int64_t need = 0;
+  const int split_k = gemm_split_k(g, tc, 1, &need);
+  if ((size_t)need > kStaticPartialBytes) {
+    set_error("static-scratch GEMM: %dx%dx%d needs %lld bytes of split-K scratch, the static array holds %zu", m, n, k,
+              (long long)need, kStaticPartialBytes);
+    return FLUID_EINVAL;
+  }
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess || dev < 0 || dev >= 64) {
+    set_error("static-scratch GEMM: no current device (%s)", cudaGetErrorString(err));
+    return FLUID_ECUDA;
+  }
+  unsigned char* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (!g_static_addr[dev]) {   // first call on this device: resolve the array's device address
+      void* ptr = nullptr;
+      err = cudaGetSymbolAddress(&ptr, g_static_scratch);
+      if (err != cudaSuccess || !ptr) {
+        set_error("static-scratch GEMM: cudaGetSymbolAddress failed (%s)", cudaGetErrorString(err));
+        return FLUID_ECUDA;
+      }
+      g_static_addr[dev] = ptr;
+    }
+    scratch = static_cast<unsigned char*>(g_static_addr[dev]);
+  }
+  if (encode_tensor_map(&tc.map_a, dev_a, tc.a) != 0 || encode_tensor_map(&tc.map_b, dev_b, tc.b) != 0) {
+    set_error("static-scratch GEMM: tensor map encoding failed");
+    return FLUID_ECUDA;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the array keeps whatever the last call left: status word and arrival counters must start at zero
+  err = cudaMemsetAsync(scratch, 0, kStaticHeaderBytes, st);
+  if (err == cudaSuccess)
+    err = launch_gemm_tc(&g, &tc, 1, split_k, reinterpret_cast<float*>(scratch + kStaticHeaderBytes),
+                         reinterpret_cast<uint32_t*>(scratch), st);
+  if (err != cudaSuccess) {
+    set_error("static-scratch GEMM: %s", cudaGetErrorString(err));
+    return FLUID_ECUDA;
+  }
+  return FLUID_OK;
+}

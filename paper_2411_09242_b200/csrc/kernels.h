@@ -171,6 +171,7 @@ cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_grou
                            uint32_t* status, cudaStream_t stream);
 // Split factor a GEMM step should use (1 = none) and the scratch it then needs.
 int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t* scratch_bytes);
+bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc);
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);
 cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t stream);

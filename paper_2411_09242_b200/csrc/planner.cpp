@@ -211,7 +211,17 @@ bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& g, GemmTcHost* tc
   GemmTcHost h{};
   h.eligible = 0;
   *tc = h;
-  if (!tc_kernel_available() || p->opts.gemm_path == 1 || g.dtype != FLUID_BF16) return false;
+  if (p->opts.gemm_path == 1) return false;
+  return gemm_tc_describe(g, tc);
+}
+
+// Tile configuration and TMA operand descriptions of a bf16 GEMM for the tensor-core kernel;
+// false if its operands cannot be expressed as tensor maps.
+bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc) {
+  GemmTcHost h{};
+  h.eligible = 0;
+  *tc = h;
+  if (!tc_kernel_available() || g.dtype != FLUID_BF16) return false;
   if (g.K < 8) return false;
   int bn = 128;
   if (g.N <= 64) bn = 64;

@@ -90,6 +90,8 @@ _SIGNATURES = {
     "fluid_run_profiled": (C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.c_void_p,
                                       C.POINTER(C.c_float)]),
     "fluid_status": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]),
+    "fluid_gemm_bf16_static_scratch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                                  C.c_void_p]),
     "fluid_last_error": (C.c_char_p, []),
     "fluid_launch_count": (C.c_int64, []),
 }
@@ -293,6 +295,13 @@ def fluid_status(p, arena_ptr, stream=0):
     if rc not in (FLUID_OK, FLUID_ETIMEOUT):
         _check(rc)
     return st.value
+
+
+def fluid_gemm_bf16_static_scratch(dev_a, dev_b, dev_bias, dev_c, m, n, k, stream=0):
+    """C[m,n] = A[m,k] . B[n,k]^T (+ bias) on device pointers, with the split-K scratch in the library's
+    own fixed device array: for callers that have no arena and may not allocate one."""
+    _check(lib().fluid_gemm_bf16_static_scratch(C.c_void_p(dev_a), C.c_void_p(dev_b), C.c_void_p(dev_bias or None),
+                                                C.c_void_p(dev_c), m, n, k, C.c_void_p(stream)))
 
 
 def fluid_launch_count():
