@@ -154,6 +154,26 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu capture
+# summarised in the named file under profiles/ (null where no capture of that workload was taken)
+NCU_TRAFFIC = {}
+
+
+def roofline_of(kernels, peaks):
+    """Roofline entry for the kernel with the largest share of the step."""
+    name = max(kernels, key=lambda k: kernels[k]["ms"])
+    dom = kernels[name]
+    if dom["bound"] == "tensor":
+        roof = {"bound": "tensor", "achieved": dom["tflops"], "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": dom["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": None, "kernel": name,
+                 "launches_per_step": dom["launches"], "avg_launch_us": dom["ms"] / dom["launches"] * 1e3,
+                 "share_of_step": dom["share"], "peak_source": peaks["source"], "frac_of_nominal": dom["frac_nominal"],
+                 "algorithmic_per_launch": (dom["flops"] if dom["bound"] == "tensor" else dom["bytes"]) / dom["launches"]})
+    return roof
+
+
 def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=None, overrides=None):
     """Plan, bind and time one model workload; returns a dict of measurements."""
     cfg = synth.CONFIGS[name]
@@ -242,10 +262,11 @@ def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=N
         k["share"] = k["ms"] / total
         k["gbs"] = k["bytes"] / (k["ms"] * 1e-3) / 1e9 if k["ms"] > 0 else 0.0
         k["tflops"] = k["flops"] / (k["ms"] * 1e-3) / 1e12 if k["ms"] > 0 else 0.0
-        k["bound"] = "tensor" if (k["flops"] / max(k["bytes"], 1.0)) > ridge and name_k == "GEMM_TC" else "hbm"
+        k["bound"] = "tensor" if (k["flops"] / max(k["bytes"], 1.0)) > ridge and name_k in ("GEMM_TC", "ATTN") else "hbm"
         k["frac_measured"] = (k["tflops"] / peaks["bf16_tflops_sustained"]) if k["bound"] == "tensor" else (k["gbs"] / peaks["hbm_gbs"])
         k["frac_nominal"] = (k["tflops"] / NOMINAL["bf16_tflops"]) if k["bound"] == "tensor" else (k["gbs"] / NOMINAL["hbm_gbs"])
     res["kernels"] = kernels
+    res["roofline"] = roofline_of(kernels, peaks)
     res["profile_total_ms"] = float(total)
     if full:
         res["_model"], res["_runner"], res["_plan"] = m, runner, plan
@@ -313,17 +334,10 @@ def main():
     if overrides:
         cfg = synth.scaled(cfg, **overrides)
     kernels = main_res["kernels"]
-    dom_name = max(kernels, key=lambda k: kernels[k]["ms"])
-    dom = kernels[dom_name]
-    per_launch_ms = dom["ms"] / dom["launches"]
-    if dom["bound"] == "tensor":
-        roof = {"bound": "tensor", "achieved": dom["tflops"], "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
-    else:
-        roof = {"bound": "hbm", "achieved": dom["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": None, "kernel": dom_name,
-                 "launches_per_step": dom["launches"], "avg_launch_us": per_launch_ms * 1e3,
-                 "share_of_step": dom["share"], "peak_source": peaks["source"],
-                 "frac_of_nominal": dom["frac_nominal"]})
+    roof = roofline_of(kernels, peaks)
+    if args.workload in NCU_TRAFFIC and not overrides and roof["kernel"] == NCU_TRAFFIC[args.workload]["kernel"]:
+        roof["traffic"] = NCU_TRAFFIC[args.workload]["bytes_per_launch"]
+        roof["traffic_source"] = NCU_TRAFFIC[args.workload]["source"]
     # parity of the timed configuration against the oracle, and the oracle's own time
     cpu = None
     parity = None

@@ -117,7 +117,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, row = threadIdx.x & 127, half = threadIdx.x >> 7;
-  const int mt = blockIdx.x, bz = blockIdx.y;
+  // CTAs are issued heaviest first: with a causal mask the last query tiles see the most key tiles,
+  // so they start first and the short ones fill the gaps (longest-processing-time order)
+  const int n_bz = p.B * p.NH;
+  const int mt = (int(gridDim.x) / n_bz - 1) - int(blockIdx.x) / n_bz, bz = int(blockIdx.x) % n_bz;
   const int h = bz % p.NH, b = bz / p.NH;
   const int m0 = mt * TQ, qi = m0 + row;
   int n_kv = (p.S + TK - 1) / TK;
@@ -364,7 +367,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream) {
   const int D = p.D;
   const size_t smem = size_t(5) * TQ * D * 2 + size_t(TQ) * TK * 2 + 1024 + 64 + 1024;
-  const dim3 grid((p.S + TQ - 1) / TQ, p.B * p.NH);
+  const dim3 grid(((p.S + TQ - 1) / TQ) * p.B * p.NH);
   const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(&host.map_q);
   const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(&host.map_k);
   const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(&host.map_v);

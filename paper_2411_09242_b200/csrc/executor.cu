@@ -62,7 +62,7 @@ int finalize_steps(fluid_plan_s* p) {
           else a *= tri;
         }
         s.flops = fl;
-        s.bytes = es * (a + b + c * (g.has_res ? 2.0 : 1.0) + (g.has_bias ? g.N : 0));
+        s.bytes = es * (a + b + (g.has_bias ? g.N : 0)) + c * (s.gemm.c_f32 ? 4.0 : es) + (g.has_res ? c * (s.gemm.r_f32 ? 4.0 : es) : 0.0);
         // grouped siblings: same A, own B / C / bias
         for (size_t gi = 1; gi < s.nodes.size(); ++gi) {
           const Node& m = p->nodes[s.nodes[gi]];
@@ -93,7 +93,12 @@ int finalize_steps(fluid_plan_s* p) {
         s.norm = q;
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.res; s.t_ptr[2] = n.gamma; s.t_ptr[3] = n.beta; s.t_ptr[4] = n.out;
         s.t_ptr[5] = n.out; s.t_narrow[5] = 1;  // bf16 copy of an fp32-held output, if one is planned
-        s.bytes = es * ty.numel() * (n.res >= 0 ? 3.0 : 2.0);
+        {
+          const double ne = (double)ty.numel();
+          const bool twin = p->twin_record_of[p->alias_root[n.out]] >= 0;
+          s.bytes = ne * (q.x_f32 ? 4.0 : es) + (n.res >= 0 ? ne * (q.res_f32 ? 4.0 : es) : 0.0) +
+                    ne * (p->wide[n.out] ? 4.0 + (twin ? es : 0.0) : es);
+        }
         break;
       }
       case N_SOFTMAX: {
