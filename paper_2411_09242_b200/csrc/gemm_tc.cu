@@ -165,8 +165,9 @@ __device__ __forceinline__ int k_steps_of(const TcParams& p, int mt) {
 }
 
 // work item -> output tile and its k-step range [k_begin, k_begin + count)
-__device__ __forceinline__ void decode_item(const TcParams& p, int item, int& tile, int& sp, int& k_begin, int& count, int mt_hint = -1) {
-  if (p.split_k <= 1) { tile = item; sp = 0; k_begin = 0; count = -1; return; }
+template <bool SPLIT>
+__device__ __forceinline__ void decode_item(const TcParams& p, int item, int& tile, int& sp, int& k_begin, int& count) {
+  if (!SPLIT || p.split_k <= 1) { tile = item; sp = 0; k_begin = 0; count = -1; return; }
   tile = item / p.split_k;
   sp = item - tile * p.split_k;
   const int total = (p.g.K + BK - 1) / BK;
@@ -347,7 +348,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& g, uint32_t tad
   }
 }
 
-template <int EPI>
+template <int EPI, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
@@ -407,7 +408,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
         int tile, sp, k_begin, k_count;
-        decode_item(p, item, tile, sp, k_begin, k_count);
+        decode_item<SPLIT>(p, item, tile, sp, k_begin, k_count);
         int grp, bz, mt, nt;
         decode_tile(p, tile, grp, bz, mt, nt);
         const int ksteps = k_count >= 0 ? k_count : k_steps_of(p, mt);
@@ -480,7 +481,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool ok = true;
       for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
         int tile, sp, k_begin, k_count;
-        decode_item(p, item, tile, sp, k_begin, k_count);
+        decode_item<SPLIT>(p, item, tile, sp, k_begin, k_count);
         int grp, bz, mt, nt;
         decode_tile(p, tile, grp, bz, mt, nt);
         const int ksteps = k_count >= 0 ? k_count : k_steps_of(p, mt);
@@ -520,7 +521,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     pdl_wait();  // before any global read (bias, residual) or write (C)
     for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
       int tile, sp, k_begin, k_count;
-      decode_item(p, item, tile, sp, k_begin, k_count);
+      decode_item<SPLIT>(p, item, tile, sp, k_begin, k_count);
       int grp, bz, mt, nt;
       decode_tile(p, tile, grp, bz, mt, nt);
       const GemmParams& g = grp == 0 ? p.g : p.gx[grp - 1];
@@ -532,7 +533,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn);
-      if (p.split_k <= 1) {
+      if (!SPLIT || p.split_k <= 1) {
 #pragma unroll 1
         for (int c0 = col_begin; c0 < col_end; c0 += 32) {
           if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
@@ -738,11 +739,14 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
 #define FLUID_TC_LAUNCH(E)                                                                                           \
   case E: {                                                                                                          \
     if (!attr_set[E]) {                                                                                              \
-      cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); \
+      cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<E, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); \
+      if (e == cudaSuccess)                                                                                          \
+        e = cudaFuncSetAttribute(gemm_tc_kernel<E, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);  \
       if (e != cudaSuccess) return e;                                                                                \
       attr_set[E] = true;                                                                                            \
     }                                                                                                                \
-    return launch_k(gemm_tc_kernel<E>, grid, kThreads, smem, stream, *ma, *mb, *mb1, *mb2, p);                                   \
+    return split_k > 1 ? launch_k(gemm_tc_kernel<E, true>, grid, kThreads, smem, stream, *ma, *mb, *mb1, *mb2, p)    \
+                       : launch_k(gemm_tc_kernel<E, false>, grid, kThreads, smem, stream, *ma, *mb, *mb1, *mb2, p);                                   \
   }
   switch (epi) {
     FLUID_TC_LAUNCH(EPI_PLAIN)
