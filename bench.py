@@ -174,7 +174,7 @@ def roofline_of(kernels, peaks):
     return roof
 
 
-def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=None, overrides=None):
+def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=None, overrides=None, plan_opts=None):
     """Plan, bind and time one model workload; returns a dict of measurements."""
     cfg = synth.CONFIGS[name]
     if overrides:
@@ -182,7 +182,7 @@ def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=N
     m = synth.build_model(cfg)
     cands = synth.default_candidates(m.graph)
     t0 = time.perf_counter()
-    plan = fluid.Plan(m.graph, cands)
+    plan = fluid.Plan(m.graph, cands, **(plan_opts or {}))
     plan_ms = 1e3 * (time.perf_counter() - t0)
     canon = fluid.Plan(m.graph, None)
     runner = fluid.Runner(plan, m.consts)
@@ -285,6 +285,7 @@ def main():
     ap.add_argument("--workload", default="bert_base", choices=list(synth.CONFIGS))
     ap.add_argument("--others", default="tiny,gpt2_small,llama", help="comma list of extra workloads to summarise")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--split-k", type=int, default=0, help="allow split-K GEMM steps (costs arena scratch)")
     ap.add_argument("--layers", type=int, default=0, help="reduced copy of the workload (profiling captures only)")
     ap.add_argument("--seq", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0)
@@ -323,7 +324,7 @@ def main():
     sampler = ClockSampler(local_rank) if rank == 0 else None
     overrides = {k: v for k, v in (("L", args.layers), ("S", args.seq), ("B", args.batch)) if v}
     main_res = time_workload(args.workload, args.steps, args.warmup, torch, fluid, peaks, full=True, sampler=sampler,
-                             overrides=overrides)
+                             overrides=overrides, plan_opts={"split_k": args.split_k} if args.split_k else None)
     barrier()
     latency_ms, e2e_ms = max_over_ranks([main_res["latency_ms"], main_res["e2e_ms"]], dist, torch.device("cuda"))
     if rank != 0:

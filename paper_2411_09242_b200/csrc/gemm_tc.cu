@@ -301,6 +301,91 @@ __device__ __forceinline__ void epilogue_chunk_vec(const GemmParams& g, uint32_t
   }
 }
 
+
+// Coalesced vector epilogue for one 32-column chunk of a warp's 32 accumulator rows. Tensor memory
+// hands each thread one row; writing rows straight out would touch 32 rows x 16 bytes per store
+// instruction. The chunk is therefore turned through a per-warp 4 KB shared-memory tile (16-byte
+// units XOR-swizzled by row, conflict-free both ways): afterwards 8 consecutive lanes hold one
+// row's 32 columns, so every global access covers 4 rows x 128 (fp32) or 64 (bf16) contiguous bytes.
+// Lane l stores rows (l >> 3) + 4 i, i = 0..7, columns 4 (l & 7) .. +3; cbs / rbs are those rows' offsets.
+template <int ACT, bool HAS_RES, bool C_WIDE, bool R_WIDE>
+__device__ __forceinline__ void epilogue_chunk_coal(const GemmParams& g, uint32_t taddr, const int64_t (&cbs)[8],
+                                                    const int64_t (&rbs)[8], uint32_t ok_mask, int n, float* stage, int lane,
+                                                    const float* partial, int split_k, size_t split_stride) {
+  uint32_t r[32];
+  if (!partial) tmem_ld32(taddr, r);
+  const int unit = lane & 7, rsub = lane >> 3;
+  const int nc = n + unit * 4;
+  const bool col_ok = nc < g.N;
+  int n1, n0i;
+  split2(nc, g.N0, n1, n0i);
+  const int64_t c_col = (int64_t)n1 * g.c_s[4] + n0i;
+  const int64_t r_col = HAS_RES ? (int64_t)n1 * g.r_s[4] + n0i : 0;
+  // operands that do not depend on the accumulator are fetched while the tensor-memory load flies
+  float bias4[4] = {0.f, 0.f, 0.f, 0.f};
+  if (g.has_bias && col_ok) {
+    const uint2 b2 = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.bias) + nc);
+    bias4[0] = __uint_as_float(b2.x << 16); bias4[1] = __uint_as_float(b2.x & 0xffff0000u);
+    bias4[2] = __uint_as_float(b2.y << 16); bias4[3] = __uint_as_float(b2.y & 0xffff0000u);
+  }
+  float4 res[HAS_RES ? 8 : 1];
+  if (HAS_RES) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      res[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (col_ok && ((ok_mask >> i) & 1u)) {
+        if (R_WIDE) {
+          res[i] = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + rbs[i] + r_col);
+        } else {
+          const uint2 q = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.R) + rbs[i] + r_col);
+          res[i] = make_float4(__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xffff0000u), __uint_as_float(q.y << 16),
+                               __uint_as_float(q.y & 0xffff0000u));
+        }
+      }
+    }
+  }
+  if (!partial) {
+    tmem_ld_wait();
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = 0;
+    for (int sp = 0; sp < split_k; ++sp) {
+      const float* src = partial + sp * split_stride;
+#pragma unroll
+      for (int c4 = 0; c4 < 8; ++c4) {
+        const float4 f = __ldcg(reinterpret_cast<const float4*>(src + (size_t)c4 * 512));
+        r[4 * c4] = __float_as_uint(__uint_as_float(r[4 * c4]) + f.x);
+        r[4 * c4 + 1] = __float_as_uint(__uint_as_float(r[4 * c4 + 1]) + f.y);
+        r[4 * c4 + 2] = __float_as_uint(__uint_as_float(r[4 * c4 + 2]) + f.z);
+        r[4 * c4 + 3] = __float_as_uint(__uint_as_float(r[4 * c4 + 3]) + f.w);
+      }
+    }
+  }
+  // row `lane` -> shared memory (unit u of row r lives at unit u ^ (r & 7))
+#pragma unroll
+  for (int u = 0; u < 8; ++u)
+    *reinterpret_cast<float4*>(stage + lane * 32 + ((u ^ (lane & 7)) << 2)) =
+        make_float4(__uint_as_float(r[4 * u]) * g.scale, __uint_as_float(r[4 * u + 1]) * g.scale,
+                    __uint_as_float(r[4 * u + 2]) * g.scale, __uint_as_float(r[4 * u + 3]) * g.scale);
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = rsub + 4 * i;
+    float4 v = *reinterpret_cast<const float4*>(stage + row * 32 + ((unit ^ (row & 7)) << 2));
+    if (!col_ok || !((ok_mask >> i) & 1u)) continue;
+    v.x = act_t<ACT>(v.x + bias4[0]); v.y = act_t<ACT>(v.y + bias4[1]);
+    v.z = act_t<ACT>(v.z + bias4[2]); v.w = act_t<ACT>(v.w + bias4[3]);
+    if (HAS_RES) { v.x += res[i].x; v.y += res[i].y; v.z += res[i].z; v.w += res[i].w; }
+    if (C_WIDE) {
+      *reinterpret_cast<float4*>(static_cast<float*>(g.C) + cbs[i] + c_col) = v;
+    } else {
+      *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.C) + cbs[i] + c_col) =
+          make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+    }
+  }
+  __syncwarp();   // the tile is reused by the next chunk
+}
+
 // General epilogue for one 8-column group: any strides, any tails, any storage width.
 __device__ __noinline__ void epilogue_group_any(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb, int64_t rb,
                                                 int n) {
@@ -329,6 +414,18 @@ __device__ __noinline__ void epilogue_group_any(const GemmParams& g, uint32_t ta
 
 // Epilogue variants (template parameter of the kernel)
 enum EpiKind { EPI_ANY = 0, EPI_PLAIN = 1, EPI_PLAIN_WIDE = 2, EPI_RES = 3, EPI_RES_WIDE = 4, EPI_GELU_ERF = 5, EPI_GELU_TANH = 6 };
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk_c(const GemmParams& g, uint32_t taddr, const int64_t (&cbs)[8], const int64_t (&rbs)[8],
+                                                 uint32_t ok_mask, int n, float* stage, int lane, const float* partial = nullptr,
+                                                 int sk = 1, size_t ss = 0) {
+  if (EPI == EPI_PLAIN) epilogue_chunk_coal<ACT_NONE, false, false, false>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
+  else if (EPI == EPI_PLAIN_WIDE) epilogue_chunk_coal<ACT_NONE, false, true, false>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
+  else if (EPI == EPI_RES) epilogue_chunk_coal<ACT_NONE, true, false, false>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
+  else if (EPI == EPI_RES_WIDE) epilogue_chunk_coal<ACT_NONE, true, true, true>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
+  else if (EPI == EPI_GELU_ERF) epilogue_chunk_coal<ACT_GELU_ERF, false, false, false>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
+  else if (EPI == EPI_GELU_TANH) epilogue_chunk_coal<ACT_GELU_TANH, false, false, false>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
+}
 
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb, int64_t rb, int n,
@@ -367,6 +464,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t tmem_slot = bars + 8u * (2 * stages + 4);
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
   volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
+  const uint32_t stage_base = (tmem_slot + 16u + 15u) & ~15u;   // 8 warps x 4 KB epilogue staging tiles
 
   pdl_launch_dependents();  // the next step may start its prologue now
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -514,6 +612,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // warps that share a lane quarter split the tile's columns between them.
     const int lane_base = (warp & 3) * 32;
     const int half = (warp - 2) >> 2;
+    float* stage = reinterpret_cast<float*>(smem_raw + (stage_base - raw)) + (warp - 2) * 1024;
     const int col_begin = half * (bn / 2), col_end = col_begin + bn / 2;
     int acc = 0;
     uint32_t acc_ph = 0;
@@ -530,6 +629,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int64_t cb = split_off(bz, g.B0, g.c_s[0], g.c_s[1]) + (row_ok ? split_off(m, g.M0, g.c_s[2], g.c_s[3]) : 0);
       const int64_t rb = g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) + (row_ok ? split_off(m, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
       const int n_tile0 = nt * bn;
+      // vector variants: offsets of the 8 rows this lane stores after the shared-memory turn
+      int64_t cbs[8], rbs[8];
+      uint32_t ok_mask = 0;
+      if (EPI != EPI_ANY) {
+        const int64_t cbz = split_off(bz, g.B0, g.c_s[0], g.c_s[1]);
+        const int64_t rbz = g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) : 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int mi = mt * BM + lane_base + (lane >> 3) + 4 * i;
+          const bool live = mi < g.M;
+          ok_mask |= live ? (1u << i) : 0u;
+          cbs[i] = cbz + (live ? split_off(mi, g.M0, g.c_s[2], g.c_s[3]) : 0);
+          rbs[i] = g.has_res ? rbz + (live ? split_off(mi, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
+        }
+      }
       if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn);
@@ -537,7 +651,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll 1
         for (int c0 = col_begin; c0 < col_end; c0 += 32) {
           if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
-          epilogue_chunk<EPI>(g, trow + uint32_t(c0), row_ok, cb, rb, n_tile0 + c0);
+          if (EPI == EPI_ANY) epilogue_chunk<EPI>(g, trow + uint32_t(c0), row_ok, cb, rb, n_tile0 + c0);
+          else epilogue_chunk_c<EPI>(g, trow + uint32_t(c0), cbs, rbs, ok_mask, n_tile0 + c0, stage, lane);
         }
         tc_fence_before();
         __syncwarp();
@@ -574,7 +689,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll 1
           for (int c0 = col_begin; c0 < col_end; c0 += 32) {
             if (n_tile0 + c0 >= g.N) break;
-            epilogue_chunk<EPI>(g, 0u, row_ok, cb, rb, n_tile0 + c0, base_row + size_t(c0 / 4) * 512, p.split_k, tile_floats);
+            epilogue_chunk_c<EPI>(g, 0u, cbs, rbs, ok_mask, n_tile0 + c0, stage, lane, base_row + size_t(c0 / 4) * 512, p.split_k, tile_floats);
           }
           if (warp == 2 && lane == 0) p.status[8 + tile] = 0;   // ready for the next launch
         }
@@ -706,7 +821,8 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
   p.tiles_per_group = (int)(per_batch * g.batch);
   p.num_tiles = p.tiles_per_group * n_group;
   p.status = status;
-  const size_t smem = size_t(tc.cfg.stages) * (kATileBytes + size_t(tc.cfg.bn) * BK * 2) + 1024 + 8 * (2 * tc.cfg.stages + 4) + 16;
+  const size_t smem = size_t(tc.cfg.stages) * (kATileBytes + size_t(tc.cfg.bn) * BK * 2) + 1024 + 8 * (2 * tc.cfg.stages + 4) + 16 +
+                      16 + size_t(kEpiWarps) * 4096;
   const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(&tc.map_a);
   const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(&tc.map_b);
   const CUtensorMap* mb1 = reinterpret_cast<const CUtensorMap*>(&tcs[n_group > 1 ? 1 : 0].map_b);
