@@ -156,7 +156,10 @@ def run_reference(args, rank):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu capture
 # summarised in the named file under profiles/ (null where no capture of that workload was taken)
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    "bert_base": {"kernel": "GEMM_TC", "bytes_per_launch": 4145717,
+                  "source": "profiles/dram_traffic_bert_base.md (48 launches of one inference, dram read + write)"},
+}
 
 
 def roofline_of(kernels, peaks):
@@ -228,6 +231,7 @@ def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=N
         res["eager_launches_counted"] = int(fluid.fluid_launch_count() - launches0)
         res["latency_ms"] = float(np.mean(t_graph))
         res["latency_min_ms"] = float(np.min(t_graph))
+        res["latency_median_ms"] = float(np.median(t_graph))
         res["latency_eager_ms"] = float(np.mean(t_eager))
         # end to end through the public API with host buffers: H2D ids, run, D2H outputs
         ids_host = torch.from_numpy(m.ids).pin_memory()
@@ -375,6 +379,7 @@ def main():
         "arena_live_bound_mb": main_res["arena_live_bound_mb"], "weights_mb": main_res["weights_mb"],
         "tokens_per_s": world * main_res["tokens"] / (latency_ms * 1e-3),
         "latency_eager_ms": main_res["latency_eager_ms"], "latency_min_ms": main_res["latency_min_ms"],
+        "latency_median_ms": main_res["latency_median_ms"],
         "e2e": {"value": e2e_ms, "unit": "ms", "h2d_bytes_per_step": main_res["h2d_bytes"],
                 "d2h_bytes_per_step": main_res["d2h_bytes"]},
         "gpu_launches": main_res["kernel_steps"] * args.steps * 3,
