@@ -103,6 +103,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_c, uint64_t adesc, uint6
       "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
       ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Same, with each descriptor given as its two 32-bit halves: only the low word (the 16-byte-unit
+// address field) moves from MMA to MMA, so the issuing thread does 32-bit arithmetic only.
+__device__ __forceinline__ void umma_bf16_lohi(uint32_t tmem_c, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n .reg .b64 da, db;\n mov.b64 da, {%1, %2};\n mov.b64 db, {%3, %4};\n setp.ne.b32 p, %6, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}"
+      ::"r"(tmem_c), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -504,6 +513,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (p.cfg.b_sel[d] == 0) b_kd0 = d;
         if (p.cfg.b_sel[d] == 1) b_kd1 = d;
       }
+      // k in one dim per operand: dim 0 for a K-major operand, dim 1 or 2 for an MN-major one
+      const bool k_simple = a_kd1 < 0 && b_kd1 < 0 && a_kd0 < 3 && b_kd0 < 3;
+      const int a_i0 = a_kd0 == 0 ? BK : 0, a_i1 = a_kd0 == 1 ? BK : 0, a_i2 = a_kd0 == 2 ? BK : 0;
+      const int b_i0 = b_kd0 == 0 ? BK : 0, b_i1 = b_kd0 == 1 ? BK : 0, b_i2 = b_kd0 == 2 ? BK : 0;
+      uint32_t sa = base, fb = full_bar(0), eb = empty_bar(0);   // the running stage
       for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
         int tile, sp, k_begin, k_count;
         decode_item<SPLIT>(p, item, tile, sp, k_begin, k_count);
@@ -526,14 +540,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           fill_coords(p.cfg.b_sel, 5, 0, 0, r0, r1, b0, b1, cb[ch]);
         }
         const CUtensorMap* mapb = grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2);
+        if (k_simple) {
+          // k lives in one tensor-map dim per operand (no two-level split): the coordinates of every
+          // box advance by BK in that dim per k-step. This loop is what one thread issues per k-step,
+          // so it holds no selects, no divisions and no address arithmetic beyond running sums.
+          const int kc = k_begin * BK;
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) { ca[ch][0] += a_i0 ? kc : 0; ca[ch][1] += a_i1 ? kc : 0; ca[ch][2] += a_i2 ? kc : 0; }
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) { cb[ch][0] += b_i0 ? kc : 0; cb[ch][1] += b_i1 ? kc : 0; cb[ch][2] += b_i2 ? kc : 0; }
+          for (int ks = 0; ks < ksteps; ++ks) {
+            if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
+            mbar_expect_tx(fb, stage_bytes);
+            tma_load(sa, &map_a, fb, ca[0][0], ca[0][1], ca[0][2], ca[0][3], ca[0][4]);
+            ca[0][0] += a_i0; ca[0][1] += a_i1; ca[0][2] += a_i2;
+            if (a_boxes > 1) {
+              tma_load(sa + 8192u, &map_a, fb, ca[1][0], ca[1][1], ca[1][2], ca[1][3], ca[1][4]);
+              ca[1][0] += a_i0; ca[1][1] += a_i1; ca[1][2] += a_i2;
+            }
+            tma_load(sa + kATileBytes, mapb, fb, cb[0][0], cb[0][1], cb[0][2], cb[0][3], cb[0][4]);
+            cb[0][0] += b_i0; cb[0][1] += b_i1; cb[0][2] += b_i2;
+            if (b_boxes > 1) {
+#pragma unroll
+              for (int ch = 1; ch < 4; ++ch) {
+                if (ch < b_boxes) {
+                  tma_load(sa + kATileBytes + ch * 8192u, mapb, fb, cb[ch][0], cb[ch][1], cb[ch][2], cb[ch][3], cb[ch][4]);
+                  cb[ch][0] += b_i0; cb[ch][1] += b_i1; cb[ch][2] += b_i2;
+                }
+              }
+            }
+            ++issued;
+            sa += stage_bytes; fb += 8u; eb += 8u;
+            if (++s == stages) { s = 0; ph ^= 1u; sa = base; fb = full_bar(0); eb = empty_bar(0); }
+          }
+          continue;
+        }
         int ak0, ak1, bk0, bk1;  // running split of the k index for each operand
         split2(k_begin * BK, p.cfg.a_k0, ak1, ak0);
         split2(k_begin * BK, p.cfg.b_k0, bk1, bk0);
         for (int ks = 0; ks < ksteps; ++ks) {
-          if (!mbar_wait(empty_bar(s), ph ^ 1u)) { ok = false; break; }
-          const uint32_t fb = full_bar(s);
+          if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
           mbar_expect_tx(fb, stage_bytes);
-          const uint32_t sa = base + uint32_t(s) * stage_bytes, sb = sa + kATileBytes;
 #pragma unroll
           for (int ch = 0; ch < 2; ++ch) {
             if (ch < a_boxes) {
@@ -549,13 +596,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               int c[5];
 #pragma unroll
               for (int d = 0; d < 5; ++d) c[d] = cb[ch][d] + (d == b_kd0 ? bk0 : 0) + (d == b_kd1 ? bk1 : 0);
-              tma_load(sb + ch * 8192u, mapb, fb, c[0], c[1], c[2], c[3], c[4]);
+              tma_load(sa + kATileBytes + ch * 8192u, mapb, fb, c[0], c[1], c[2], c[3], c[4]);
             }
           }
           ++issued;
           ak0 += BK; if (ak0 >= p.cfg.a_k0) { ak0 = 0; ++ak1; }
           bk0 += BK; if (bk0 >= p.cfg.b_k0) { bk0 = 0; ++bk1; }
-          if (++s == stages) { s = 0; ph ^= 1u; }
+          sa += stage_bytes; fb += 8u; eb += 8u;
+          if (++s == stages) { s = 0; ph ^= 1u; sa = base; fb = full_bar(0); eb = empty_bar(0); }
         }
       }
       if (!ok) {
@@ -573,7 +621,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       const uint32_t idesc = make_idesc(bn, p.cfg.a_mn_major, p.cfg.b_mn_major);
-      const uint32_t a_step = p.cfg.a_mn_major ? 2048u : 32u, b_step = p.cfg.b_mn_major ? 2048u : 32u;
+      // 16-byte units between the four 16-deep k slices of a stage: 32 bytes along a K-major row,
+      // 2048 bytes (16 k-rows of 128 bytes) in an MN-major tile
+      const uint32_t a_step = p.cfg.a_mn_major ? 128u : 2u, b_step = p.cfg.b_mn_major ? 128u : 2u;
+      const uint64_t ad_first = make_desc(base, p.cfg.a_mn_major), bd_first = make_desc(base + kATileBytes, p.cfg.b_mn_major);
+      const uint32_t a_hi = uint32_t(ad_first >> 32), b_hi = uint32_t(bd_first >> 32);
+      const uint32_t a_lo0 = uint32_t(ad_first), b_lo0 = uint32_t(bd_first), stage16 = stage_bytes >> 4;
+      // the running stage: descriptor low words (the address field never carries out of its 14 bits,
+      // shared memory being smaller than 256 KB) and barrier addresses
+      uint32_t a_lo = a_lo0, b_lo = b_lo0, fb = full_bar(0), eb = empty_bar(0);
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
@@ -586,17 +642,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_c = tmem_base + uint32_t(acc * bn);
+        uint32_t accum = 0u;
         for (int ks = 0; ks < ksteps; ++ks) {
-          if (!mbar_wait(full_bar(s), ph)) { ok = false; break; }
+          if (!mbar_wait(fb, ph)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + uint32_t(s) * stage_bytes, sb = sa + kATileBytes;
-          const uint64_t ad0 = make_desc(sa, p.cfg.a_mn_major), bd0 = make_desc(sb, p.cfg.b_mn_major);
-#pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk)
-            umma_bf16(tmem_c, ad0 + uint64_t((kk * a_step) >> 4), bd0 + uint64_t((kk * b_step) >> 4), idesc,
-                      (ks > 0 || kk > 0) ? 1u : 0u);
-          umma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
-          if (++s == stages) { s = 0; ph ^= 1u; }
+          umma_bf16_lohi(tmem_c, a_lo, a_hi, b_lo, b_hi, idesc, accum);
+          umma_bf16_lohi(tmem_c, a_lo + a_step, a_hi, b_lo + b_step, b_hi, idesc, 1u);
+          umma_bf16_lohi(tmem_c, a_lo + 2u * a_step, a_hi, b_lo + 2u * b_step, b_hi, idesc, 1u);
+          umma_bf16_lohi(tmem_c, a_lo + 3u * a_step, a_hi, b_lo + 3u * b_step, b_hi, idesc, 1u);
+          umma_commit(eb);  // the stage is free once these MMAs have read it
+          accum = 1u;
+          a_lo += stage16; b_lo += stage16; fb += 8u; eb += 8u;
+          if (++s == stages) { s = 0; ph ^= 1u; a_lo = a_lo0; b_lo = b_lo0; fb = full_bar(0); eb = empty_bar(0); }
         }
         if (ok) umma_commit(tfull_bar(acc));  // accumulator complete
         if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
