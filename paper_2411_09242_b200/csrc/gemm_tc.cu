@@ -98,13 +98,8 @@ __device__ __forceinline__ void tma_load(uint32_t dst, const CUtensorMap* map, u
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// Same, with each descriptor given as its two 32-bit halves: only the low word (the 16-byte-unit
-// address field) moves from MMA to MMA, so the issuing thread does 32-bit arithmetic only.
+// Each descriptor is given as its two 32-bit halves: only the low word (the 16-byte-unit address
+// field) moves from MMA to MMA, so the issuing thread does 32-bit arithmetic only.
 __device__ __forceinline__ void umma_bf16_lohi(uint32_t tmem_c, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
                                                uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -498,123 +493,86 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-    if (lane == 0) {
-      int s = 0, issued = 0;
+    // One lane per 64-wide box of a stage: lanes 0-1 the A boxes, lanes 2-5 the B boxes (a K-major
+    // operand is one box, an MN-major one is a box per 64 rows). The lanes run in lockstep on the
+    // same barriers, so the per-tile coordinate set-up (divisions, selects) costs one box's worth
+    // and the per-k-step loop is a wait, one TMA and three adds. A single thread issuing every
+    // box was the slowest part of a short tile (about 600 cycles per k-step, 3000 per tile).
+    const bool is_a = lane < 2;
+    const int ch = is_a ? lane : lane - 2;
+    const int n_box = is_a ? (p.cfg.a_mn_major ? BM / 64 : 1) : (p.cfg.b_mn_major ? bn / 64 : 1);
+    if (lane < 6 && ch < n_box) {
+      int s = 0;
       uint32_t ph = 0;
-      bool ok = true;
-      const int a_boxes = p.cfg.a_mn_major ? BM / 64 : 1, b_boxes = p.cfg.b_mn_major ? bn / 64 : 1;
-      pdl_wait();  // the previous step's outputs are this step's operands
+      bool ok = true, in_flight = false;
+      const uint32_t box_off = (is_a ? 0u : kATileBytes) + uint32_t(ch) * 8192u;
+      const int x_r0 = is_a ? p.cfg.a_r0 : p.cfg.b_r0, x_b0 = is_a ? p.cfg.a_b0 : p.cfg.b_b0;
+      const int x_k0 = is_a ? p.cfg.a_k0 : p.cfg.b_k0;
+      int sel[5];
+#pragma unroll
+      for (int d = 0; d < 5; ++d) sel[d] = is_a ? p.cfg.a_sel[d] : p.cfg.b_sel[d];
       // which coordinate slots carry the running k split (the rest stay fixed over a tile)
-      int a_kd0 = 0, a_kd1 = -1, b_kd0 = 0, b_kd1 = -1;
+      int kd0 = 0, kd1 = -1;
 #pragma unroll
       for (int d = 0; d < 5; ++d) {
-        if (p.cfg.a_sel[d] == 0) a_kd0 = d;
-        if (p.cfg.a_sel[d] == 1) a_kd1 = d;
-        if (p.cfg.b_sel[d] == 0) b_kd0 = d;
-        if (p.cfg.b_sel[d] == 1) b_kd1 = d;
+        if (sel[d] == 0) kd0 = d;
+        if (sel[d] == 1) kd1 = d;
       }
-      // k in one dim per operand: dim 0 for a K-major operand, dim 1 or 2 for an MN-major one
-      const bool k_simple = a_kd1 < 0 && b_kd1 < 0 && a_kd0 < 3 && b_kd0 < 3;
-      const int a_i0 = a_kd0 == 0 ? BK : 0, a_i1 = a_kd0 == 1 ? BK : 0, a_i2 = a_kd0 == 2 ? BK : 0;
-      const int b_i0 = b_kd0 == 0 ? BK : 0, b_i1 = b_kd0 == 1 ? BK : 0, b_i2 = b_kd0 == 2 ? BK : 0;
-      uint32_t sa = base, fb = full_bar(0), eb = empty_bar(0);   // the running stage
+      // k in one tensor-map dim (0 for a K-major operand, 1 or 2 for an MN-major one): running sums only
+      const bool k_simple = kd1 < 0 && kd0 < 3;
+      const int i0 = kd0 == 0 ? BK : 0, i1 = kd0 == 1 ? BK : 0, i2 = kd0 == 2 ? BK : 0;
+      uint32_t dst = base + box_off, fb = full_bar(0), eb = empty_bar(0);   // the running stage
+      pdl_wait();  // the previous step's outputs are this step's operands
       for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
         int tile, sp, k_begin, k_count;
         decode_item<SPLIT>(p, item, tile, sp, k_begin, k_count);
         int grp, bz, mt, nt;
         decode_tile(p, tile, grp, bz, mt, nt);
         const int ksteps = k_count >= 0 ? k_count : k_steps_of(p, mt);
-        int ca[2][5], cb[4][5];  // fully unrolled below: these stay in registers
-#pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
+        int c[5];
+        {
           int r1, r0, b1, b0;
-          split2(mt * BM + ch * 64, p.cfg.a_r0, r1, r0);
-          split2(bz, p.cfg.a_b0, b1, b0);
-          fill_coords(p.cfg.a_sel, 5, 0, 0, r0, r1, b0, b1, ca[ch]);
+          split2((is_a ? mt * BM : nt * bn) + ch * 64, x_r0, r1, r0);
+          split2(bz, x_b0, b1, b0);
+          fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
         }
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          int r1, r0, b1, b0;
-          split2(nt * bn + ch * 64, p.cfg.b_r0, r1, r0);
-          split2(bz, p.cfg.b_b0, b1, b0);
-          fill_coords(p.cfg.b_sel, 5, 0, 0, r0, r1, b0, b1, cb[ch]);
-        }
-        const CUtensorMap* mapb = grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2);
+        const CUtensorMap* map = is_a ? &map_a : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2));
         if (k_simple) {
-          // k lives in one tensor-map dim per operand (no two-level split): the coordinates of every
-          // box advance by BK in that dim per k-step. This loop is what one thread issues per k-step,
-          // so it holds no selects, no divisions and no address arithmetic beyond running sums.
           const int kc = k_begin * BK;
-#pragma unroll
-          for (int ch = 0; ch < 2; ++ch) { ca[ch][0] += a_i0 ? kc : 0; ca[ch][1] += a_i1 ? kc : 0; ca[ch][2] += a_i2 ? kc : 0; }
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch) { cb[ch][0] += b_i0 ? kc : 0; cb[ch][1] += b_i1 ? kc : 0; cb[ch][2] += b_i2 ? kc : 0; }
+          c[0] += i0 ? kc : 0; c[1] += i1 ? kc : 0; c[2] += i2 ? kc : 0;
           for (int ks = 0; ks < ksteps; ++ks) {
             if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
-            mbar_expect_tx(fb, stage_bytes);
-            tma_load(sa, &map_a, fb, ca[0][0], ca[0][1], ca[0][2], ca[0][3], ca[0][4]);
-            ca[0][0] += a_i0; ca[0][1] += a_i1; ca[0][2] += a_i2;
-            if (a_boxes > 1) {
-              tma_load(sa + 8192u, &map_a, fb, ca[1][0], ca[1][1], ca[1][2], ca[1][3], ca[1][4]);
-              ca[1][0] += a_i0; ca[1][1] += a_i1; ca[1][2] += a_i2;
-            }
-            tma_load(sa + kATileBytes, mapb, fb, cb[0][0], cb[0][1], cb[0][2], cb[0][3], cb[0][4]);
-            cb[0][0] += b_i0; cb[0][1] += b_i1; cb[0][2] += b_i2;
-            if (b_boxes > 1) {
-#pragma unroll
-              for (int ch = 1; ch < 4; ++ch) {
-                if (ch < b_boxes) {
-                  tma_load(sa + kATileBytes + ch * 8192u, mapb, fb, cb[ch][0], cb[ch][1], cb[ch][2], cb[ch][3], cb[ch][4]);
-                  cb[ch][0] += b_i0; cb[ch][1] += b_i1; cb[ch][2] += b_i2;
-                }
-              }
-            }
-            ++issued;
-            sa += stage_bytes; fb += 8u; eb += 8u;
-            if (++s == stages) { s = 0; ph ^= 1u; sa = base; fb = full_bar(0); eb = empty_bar(0); }
+            if (lane == 0) mbar_expect_tx(fb, stage_bytes);
+            tma_load(dst, map, fb, c[0], c[1], c[2], c[3], c[4]);
+            in_flight = true;
+            c[0] += i0; c[1] += i1; c[2] += i2;
+            dst += stage_bytes; fb += 8u; eb += 8u;
+            if (++s == stages) { s = 0; ph ^= 1u; dst = base + box_off; fb = full_bar(0); eb = empty_bar(0); }
           }
           continue;
         }
-        int ak0, ak1, bk0, bk1;  // running split of the k index for each operand
-        split2(k_begin * BK, p.cfg.a_k0, ak1, ak0);
-        split2(k_begin * BK, p.cfg.b_k0, bk1, bk0);
+        int k0, k1;  // running two-level split of the k index
+        split2(k_begin * BK, x_k0, k1, k0);
         for (int ks = 0; ks < ksteps; ++ks) {
           if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
-          mbar_expect_tx(fb, stage_bytes);
+          if (lane == 0) mbar_expect_tx(fb, stage_bytes);
+          int q[5];
 #pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
-            if (ch < a_boxes) {
-              int c[5];
-#pragma unroll
-              for (int d = 0; d < 5; ++d) c[d] = ca[ch][d] + (d == a_kd0 ? ak0 : 0) + (d == a_kd1 ? ak1 : 0);
-              tma_load(sa + ch * 8192u, &map_a, fb, c[0], c[1], c[2], c[3], c[4]);
-            }
-          }
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            if (ch < b_boxes) {
-              int c[5];
-#pragma unroll
-              for (int d = 0; d < 5; ++d) c[d] = cb[ch][d] + (d == b_kd0 ? bk0 : 0) + (d == b_kd1 ? bk1 : 0);
-              tma_load(sa + kATileBytes + ch * 8192u, mapb, fb, c[0], c[1], c[2], c[3], c[4]);
-            }
-          }
-          ++issued;
-          ak0 += BK; if (ak0 >= p.cfg.a_k0) { ak0 = 0; ++ak1; }
-          bk0 += BK; if (bk0 >= p.cfg.b_k0) { bk0 = 0; ++bk1; }
-          sa += stage_bytes; fb += 8u; eb += 8u;
-          if (++s == stages) { s = 0; ph ^= 1u; sa = base; fb = full_bar(0); eb = empty_bar(0); }
+          for (int d = 0; d < 5; ++d) q[d] = c[d] + (d == kd0 ? k0 : 0) + (d == kd1 ? k1 : 0);
+          tma_load(dst, map, fb, q[0], q[1], q[2], q[3], q[4]);
+          in_flight = true;
+          k0 += BK; if (k0 >= x_k0) { k0 = 0; ++k1; }
+          dst += stage_bytes; fb += 8u; eb += 8u;
+          if (++s == stages) { s = 0; ph ^= 1u; dst = base + box_off; fb = full_bar(0); eb = empty_bar(0); }
         }
       }
       if (!ok) {
         if (!*abort_flag) atomicOr(p.status, 0x1u);
         *abort_flag = 1;
-        // let the loads already issued land before this CTA's shared memory is given up
-        const int back = issued < stages ? issued : stages;
-        for (int j = 0; j < back; ++j) {
-          if (--s < 0) { s = stages - 1; ph ^= 1u; }
-          mbar_wait(full_bar(s), ph);
-        }
+        // let the loads already issued land before this CTA's shared memory is given up: the most
+        // recent fill of every stage this lane wrote (stages before s are in phase ph, the rest in ph ^ 1)
+        if (in_flight)
+          for (int j = 0; j < stages; ++j) mbar_wait(full_bar(j), j < s ? ph : ph ^ 1u);
       }
     }
   } else if (warp == 1) {
