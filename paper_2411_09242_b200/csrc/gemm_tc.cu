@@ -171,7 +171,7 @@ __device__ __forceinline__ int k_steps_of(const TcParams& p, int mt) {
 // work item -> output tile and its k-step range [k_begin, k_begin + count)
 template <bool SPLIT>
 __device__ __forceinline__ void decode_item(const TcParams& p, int item, int& tile, int& sp, int& k_begin, int& count) {
-  if (!SPLIT || p.split_k <= 1) { tile = item; sp = 0; k_begin = 0; count = -1; return; }
+  if (!SPLIT) { tile = item; sp = 0; k_begin = 0; count = -1; return; }
   tile = item / p.split_k;
   sp = item - tile * p.split_k;
   const int total = (p.g.K + BK - 1) / BK;
@@ -390,6 +390,98 @@ __device__ __forceinline__ void epilogue_chunk_coal(const GemmParams& g, uint32_
   __syncwarp();   // the tile is reused by the next chunk
 }
 
+// The same epilogue for a warp's whole column range [col_begin, col_end) of a tile, software-pipelined
+// over its 32-column chunks: the tensor-memory load and the bias of chunk i+1 are in
+// flight while chunk i is turned through shared memory and stored (the residual follows as soon as
+// chunk i has used its registers), so those latencies overlap the stores instead of preceding them.
+template <int ACT, bool HAS_RES, bool C_WIDE, bool R_WIDE>
+__device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
+                                                   const int64_t (&cbs)[8], const int64_t (&rbs)[8], uint32_t ok_mask,
+                                                   float* stage, int lane) {
+  const int unit = lane & 7, rsub = lane >> 3;
+  int n_chunks = (min(col_end, g.N - n_tile0) - col_begin + 31) >> 5;   // uniform across the warp
+  if (n_chunks <= 0) return;
+  uint32_t r[32];
+  float bias_cur[4], bias_nxt[4] = {0.f, 0.f, 0.f, 0.f};
+  float4 res[HAS_RES ? 8 : 1];
+  int64_t c_col = 0, c_col_nxt = 0, r_col = 0;
+  bool col_ok = false, col_ok_nxt = false;
+  // column offsets and bias of the chunk starting at tile column c0
+  auto fetch = [&](int c0, float (&bias4)[4], int64_t& ccol, int64_t& rcol, bool& cok) {
+    const int nc = n_tile0 + c0 + unit * 4;
+    cok = nc < g.N;
+    int n1, n0i;
+    split2(nc, g.N0, n1, n0i);
+    ccol = (int64_t)n1 * g.c_s[4] + n0i;
+    if (HAS_RES) rcol = (int64_t)n1 * g.r_s[4] + n0i;
+    bias4[0] = bias4[1] = bias4[2] = bias4[3] = 0.f;
+    if (g.has_bias && cok) {
+      const uint2 b2 = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.bias) + nc);
+      bias4[0] = __uint_as_float(b2.x << 16); bias4[1] = __uint_as_float(b2.x & 0xffff0000u);
+      bias4[2] = __uint_as_float(b2.y << 16); bias4[3] = __uint_as_float(b2.y & 0xffff0000u);
+    }
+  };
+  // residual of the current chunk (one buffer: the next chunk's loads are issued once this one is consumed)
+  auto fetch_res = [&](int64_t rcol, bool cok) {
+#pragma unroll
+    for (int i = 0; i < (HAS_RES ? 8 : 0); ++i) {
+      res[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (cok && ((ok_mask >> i) & 1u)) {
+        if (R_WIDE) {
+          res[i] = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + rbs[i] + rcol);
+        } else {
+          const uint2 q = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.R) + rbs[i] + rcol);
+          res[i] = make_float4(__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xffff0000u), __uint_as_float(q.y << 16),
+                               __uint_as_float(q.y & 0xffff0000u));
+        }
+      }
+    }
+  };
+  tmem_ld32(trow + uint32_t(col_begin), r);
+  fetch(col_begin, bias_cur, c_col, r_col, col_ok);
+  fetch_res(r_col, col_ok);
+#pragma unroll 1
+  for (int ci = 0; ci < n_chunks; ++ci) {
+    tmem_ld_wait();
+    // row `lane` -> shared memory (unit u of row r lives at unit u ^ (r & 7))
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      *reinterpret_cast<float4*>(stage + lane * 32 + ((u ^ (lane & 7)) << 2)) =
+          make_float4(__uint_as_float(r[4 * u]) * g.scale, __uint_as_float(r[4 * u + 1]) * g.scale,
+                      __uint_as_float(r[4 * u + 2]) * g.scale, __uint_as_float(r[4 * u + 3]) * g.scale);
+    __syncwarp();
+    const bool more = ci + 1 < n_chunks;
+    int64_t r_col_nxt = 0;
+    if (more) {
+      const int c0n = col_begin + 32 * (ci + 1);
+      tmem_ld32(trow + uint32_t(c0n), r);
+      fetch(c0n, bias_nxt, c_col_nxt, r_col_nxt, col_ok_nxt);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = rsub + 4 * i;
+      float4 v = *reinterpret_cast<const float4*>(stage + row * 32 + ((unit ^ (row & 7)) << 2));
+      if (!col_ok || !((ok_mask >> i) & 1u)) continue;
+      v.x = act_t<ACT>(v.x + bias_cur[0]); v.y = act_t<ACT>(v.y + bias_cur[1]);
+      v.z = act_t<ACT>(v.z + bias_cur[2]); v.w = act_t<ACT>(v.w + bias_cur[3]);
+      if (HAS_RES) { v.x += res[i].x; v.y += res[i].y; v.z += res[i].z; v.w += res[i].w; }
+      if (C_WIDE) {
+        *reinterpret_cast<float4*>(static_cast<float*>(g.C) + cbs[i] + c_col) = v;
+      } else {
+        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.C) + cbs[i] + c_col) =
+            make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+      }
+    }
+    __syncwarp();   // the staging tile is rewritten by the next chunk
+    if (more) {
+      if (HAS_RES) fetch_res(r_col_nxt, col_ok_nxt);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) bias_cur[q] = bias_nxt[q];
+      c_col = c_col_nxt; col_ok = col_ok_nxt;
+    }
+  }
+}
+
 // General epilogue for one 8-column group: any strides, any tails, any storage width.
 __device__ __noinline__ void epilogue_group_any(const GemmParams& g, uint32_t taddr, bool row_ok, int64_t cb, int64_t rb,
                                                 int n) {
@@ -429,6 +521,18 @@ __device__ __forceinline__ void epilogue_chunk_c(const GemmParams& g, uint32_t t
   else if (EPI == EPI_RES_WIDE) epilogue_chunk_coal<ACT_NONE, true, true, true>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
   else if (EPI == EPI_GELU_ERF) epilogue_chunk_coal<ACT_GELU_ERF, false, false, false>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
   else if (EPI == EPI_GELU_TANH) epilogue_chunk_coal<ACT_GELU_TANH, false, false, false>(g, taddr, cbs, rbs, ok_mask, n, stage, lane, partial, sk, ss);
+}
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_tile_c(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
+                                                const int64_t (&cbs)[8], const int64_t (&rbs)[8], uint32_t ok_mask, float* stage,
+                                                int lane) {
+  if (EPI == EPI_PLAIN) epilogue_tile_coal<ACT_NONE, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+  else if (EPI == EPI_PLAIN_WIDE) epilogue_tile_coal<ACT_NONE, false, true, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+  else if (EPI == EPI_RES) epilogue_tile_coal<ACT_NONE, true, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+  else if (EPI == EPI_RES_WIDE) epilogue_tile_coal<ACT_NONE, true, true, true>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+  else if (EPI == EPI_GELU_ERF) epilogue_tile_coal<ACT_GELU_ERF, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+  else if (EPI == EPI_GELU_TANH) epilogue_tile_coal<ACT_GELU_TANH, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
 }
 
 template <int EPI>
@@ -662,12 +766,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn);
-      if (!SPLIT || p.split_k <= 1) {
+      if (!SPLIT) {
+        if (EPI == EPI_ANY) {
 #pragma unroll 1
-        for (int c0 = col_begin; c0 < col_end; c0 += 32) {
-          if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
-          if (EPI == EPI_ANY) epilogue_chunk<EPI>(g, trow + uint32_t(c0), row_ok, cb, rb, n_tile0 + c0);
-          else epilogue_chunk_c<EPI>(g, trow + uint32_t(c0), cbs, rbs, ok_mask, n_tile0 + c0, stage, lane);
+          for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+            if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
+            epilogue_chunk<EPI>(g, trow + uint32_t(c0), row_ok, cb, rb, n_tile0 + c0);
+          }
+        } else {
+          epilogue_tile_c<EPI>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
         }
         tc_fence_before();
         __syncwarp();
