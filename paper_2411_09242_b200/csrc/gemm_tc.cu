@@ -124,6 +124,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ void sts128(uint32_t addr, float a, float b, float c, float d) {
+  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle. K-major: rows of 128 bytes, 8-row groups
 // 1024 bytes apart. MN-major: 64-element chunks of the row index 8192 bytes apart (one chunk =
 // 64 k-rows of 128 bytes), 8-k groups 1024 bytes apart.
@@ -399,6 +408,10 @@ __device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t
                                                    const int64_t (&cbs)[8], const int64_t (&rbs)[8], uint32_t ok_mask,
                                                    float* stage, int lane) {
   const int unit = lane & 7, rsub = lane >> 3;
+  const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
+  const float scale = g.scale;
+  float* const c_f32 = static_cast<float*>(g.C);
+  __nv_bfloat16* const c_b16 = static_cast<__nv_bfloat16*>(g.C);
   int n_chunks = (min(col_end, g.N - n_tile0) - col_begin + 31) >> 5;   // uniform across the warp
   if (n_chunks <= 0) return;
   uint32_t r[32];
@@ -446,9 +459,8 @@ __device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t
     // row `lane` -> shared memory (unit u of row r lives at unit u ^ (r & 7))
 #pragma unroll
     for (int u = 0; u < 8; ++u)
-      *reinterpret_cast<float4*>(stage + lane * 32 + ((u ^ (lane & 7)) << 2)) =
-          make_float4(__uint_as_float(r[4 * u]) * g.scale, __uint_as_float(r[4 * u + 1]) * g.scale,
-                      __uint_as_float(r[4 * u + 2]) * g.scale, __uint_as_float(r[4 * u + 3]) * g.scale);
+      sts128(st_row + (uint32_t(u ^ (lane & 7)) << 4), __uint_as_float(r[4 * u]) * scale, __uint_as_float(r[4 * u + 1]) * scale,
+             __uint_as_float(r[4 * u + 2]) * scale, __uint_as_float(r[4 * u + 3]) * scale);
     __syncwarp();
     const bool more = ci + 1 < n_chunks;
     int64_t r_col_nxt = 0;
@@ -457,19 +469,32 @@ __device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t
       tmem_ld32(trow + uint32_t(c0n), r);
       fetch(c0n, bias_nxt, c_col_nxt, r_col_nxt, col_ok_nxt);
     }
+    // all eight shared-memory reads first (independent), then the eight stores
+    float4 v8[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int row = rsub + 4 * i;
-      float4 v = *reinterpret_cast<const float4*>(stage + row * 32 + ((unit ^ (row & 7)) << 2));
-      if (!col_ok || !((ok_mask >> i) & 1u)) continue;
+      v8[i] = lds128(st_base + uint32_t(row * 128) + (uint32_t(unit ^ (row & 7)) << 4));
+    }
+    // straight-line arithmetic on all eight rows (rows past M and columns past N compute on whatever
+    // the accumulator holds and are not stored), then eight predicated stores
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float4& v = v8[i];
       v.x = act_t<ACT>(v.x + bias_cur[0]); v.y = act_t<ACT>(v.y + bias_cur[1]);
       v.z = act_t<ACT>(v.z + bias_cur[2]); v.w = act_t<ACT>(v.w + bias_cur[3]);
       if (HAS_RES) { v.x += res[i].x; v.y += res[i].y; v.z += res[i].z; v.w += res[i].w; }
+    }
+    const uint32_t live = col_ok ? ok_mask : 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
       if (C_WIDE) {
-        *reinterpret_cast<float4*>(static_cast<float*>(g.C) + cbs[i] + c_col) = v;
+        float4* dst = reinterpret_cast<float4*>(c_f32 + cbs[i] + c_col);
+        if ((live >> i) & 1u) *dst = v8[i];
       } else {
-        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.C) + cbs[i] + c_col) =
-            make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+        uint2* dst = reinterpret_cast<uint2*>(c_b16 + cbs[i] + c_col);
+        const uint2 q = make_uint2(pack_bf16x2(v8[i].x, v8[i].y), pack_bf16x2(v8[i].z, v8[i].w));
+        if ((live >> i) & 1u) *dst = q;
       }
     }
     __syncwarp();   // the staging tile is rewritten by the next chunk
