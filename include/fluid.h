@@ -119,9 +119,13 @@ typedef struct fluid_plan_options {
                                arena, with a bf16 twin where a GEMM also reads them; 1 = every
                                activation is held in its declared dtype */
   int32_t unfused_attention; /* 1: keep BMM_QK -> SOFTMAX -> BMM_PV as three steps even when fusion is on */
-  int32_t split_k;          /* 1: GEMM steps with few output tiles and a long k range cut it across CTAs;
-                               the fp32 partial tiles take a scratch slice of the arena for that step.
-                               0 (default): never, the arena holds activations only */
+  int32_t split_k;          /* GEMM steps with few output tiles cut their k range across CTAs.
+                               0 (default): where one thread-block cluster per output tile fits the GPU in one
+                               wave, the cut runs inside the cluster and the partial sums meet in distributed
+                               shared memory (no scratch; the arena holds activations only).
+                               1: in addition, steps with a long k range may park fp32 partial tiles in a scratch
+                               slice of the arena that lives for that step.
+                               -1: never split */
   fluid_eval_fn eval;       /* NULL: built-in analytic B200 cost table */
   void* eval_user;
 } fluid_plan_options;
@@ -135,7 +139,8 @@ typedef enum {
 typedef struct fluid_step_info {
   int32_t kernel;        /* fluid_kernel_id */
   int32_t variant;       /* kernel-specific (GEMM: bit0 A MN-major, bit1 B MN-major, bits 8-19 tile N,
-                            bits 20-23 grouped siblings, bits 24-27 split-K factor) */
+                            bits 20-23 grouped siblings, bits 24-27 split-K factor, bit 28: the split
+                            runs as one thread-block cluster per output tile) */
   int32_t n_ops;         /* graph ops folded into this step */
   int32_t ops[8];
   int32_t n_in, n_out;   /* tensors read / written (graph tensor ids) */

@@ -77,7 +77,13 @@ int finalize_steps(fluid_plan_s* p) {
           s.bytes += es * (b + c + (g.has_bias ? g.N : 0));
         }
         if (s.nodes.size() > 1) s.variant |= int(s.nodes.size()) << 20;
-        if (s.split_k > 1) s.variant |= s.split_k << 24;
+        if (s.split_k > 1) {
+          s.variant |= s.split_k << 24;
+        } else if (s.kernel == FLUID_K_GEMM_TC && p->opts.split_k >= 0) {
+          GemmParams gs[3] = {s.gemm, s.nodes.size() > 1 ? s.gemm_x[0] : s.gemm, s.nodes.size() > 2 ? s.gemm_x[1] : s.gemm};
+          s.cluster_k = gemm_cluster_split(gs, s.tc, int(s.nodes.size()));
+          if (s.cluster_k > 1) s.variant |= (s.cluster_k << 24) | (1 << 28);
+        }
         break;
       }
       case N_NORM: {
@@ -370,7 +376,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
           float* partial = s.scratch_record >= 0
                                ? reinterpret_cast<float*>(static_cast<char*>(arena_ptr) + p->records[s.scratch_record].offset)
                                : nullptr;
-          if (R.ok) err = launch_gemm_tc(gs, ts, ng, s.split_k, partial, status, stream);
+          if (R.ok) err = launch_gemm_tc(gs, ts, ng, s.split_k, s.cluster_k, partial, status, stream);
         } else if (R.ok) {
           err = launch_gemm_simt(q, stream);
         }

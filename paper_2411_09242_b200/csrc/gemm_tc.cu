@@ -18,6 +18,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstdio>
 
 #include <mutex>
@@ -857,6 +858,263 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
+// ---- cluster split-K: short-and-wide GEMMs (few output tiles, e.g. 128 tokens) -----------------------
+// With one row of output tiles a launch of the persistent kernel occupies a handful of SMs, and every
+// one of them walks the whole K range at the tensor core's fixed ~128 cycles per 128 x N x 16
+// instruction. Here a thread-block cluster of `split_k` CTAs shares one output tile: CTA r runs the
+// k-steps [r * kps, (r + 1) * kps) into its own tensor-memory accumulator, then the cluster
+// reduce-scatters the fp32 partials through distributed shared memory: CTA r receives rows
+// [r * 128 / split_k, ...) of every peer's partial, sums the split_k slices in rank order
+// (deterministic) and runs the epilogue for those rows. No global scratch, no atomics.
+// Warp roles as in the persistent kernel. Every thread of the cluster passes both cluster barriers
+// on every path (the bounded mbarrier waits only skip work), so a failed wait cannot leave a peer
+// waiting.
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+__device__ __forceinline__ void st_cluster128(uint32_t local_addr, uint32_t rank, float a, float b, float c, float d) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+template <int ACT, bool HAS_RES, bool C_WIDE, bool R_WIDE>
+__device__ __forceinline__ void final_store4(const GemmParams& g, float4 v, int64_t cb, int64_t rb, int nc) {
+  int n1, n0i;
+  split2(nc, g.N0, n1, n0i);
+  if (g.has_bias) {
+    const uint2 b2 = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.bias) + nc);
+    v.x += __uint_as_float(b2.x << 16); v.y += __uint_as_float(b2.x & 0xffff0000u);
+    v.z += __uint_as_float(b2.y << 16); v.w += __uint_as_float(b2.y & 0xffff0000u);
+  }
+  v.x = act_t<ACT>(v.x); v.y = act_t<ACT>(v.y); v.z = act_t<ACT>(v.z); v.w = act_t<ACT>(v.w);
+  if (HAS_RES) {
+    const int64_t ro = rb + (int64_t)n1 * g.r_s[4] + n0i;
+    if (R_WIDE) {
+      const float4 q = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + ro);
+      v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+    } else {
+      const uint2 q = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.R) + ro);
+      v.x += __uint_as_float(q.x << 16); v.y += __uint_as_float(q.x & 0xffff0000u);
+      v.z += __uint_as_float(q.y << 16); v.w += __uint_as_float(q.y & 0xffff0000u);
+    }
+  }
+  const int64_t co = cb + (int64_t)n1 * g.c_s[4] + n0i;
+  if (C_WIDE) *reinterpret_cast<float4*>(static_cast<float*>(g.C) + co) = v;
+  else *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.C) + co) = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+}
+
+template <int EPI>
+__device__ __forceinline__ void final_store4_c(const GemmParams& g, float4 v, int64_t cb, int64_t rb, int nc) {
+  if (EPI == EPI_PLAIN) final_store4<ACT_NONE, false, false, false>(g, v, cb, rb, nc);
+  else if (EPI == EPI_PLAIN_WIDE) final_store4<ACT_NONE, false, true, false>(g, v, cb, rb, nc);
+  else if (EPI == EPI_RES) final_store4<ACT_NONE, true, false, false>(g, v, cb, rb, nc);
+  else if (EPI == EPI_RES_WIDE) final_store4<ACT_NONE, true, true, true>(g, v, cb, rb, nc);
+  else if (EPI == EPI_GELU_ERF) final_store4<ACT_GELU_ERF, false, false, false>(g, v, cb, rb, nc);
+  else final_store4<ACT_GELU_TANH, false, false, false>(g, v, cb, rb, nc);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                       const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
+                       const __grid_constant__ TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const int bn = p.cfg.bn, stages = p.cfg.stages, sk = p.split_k;
+  const uint32_t stage_bytes = kATileBytes + uint32_t(bn) * BK * 2;
+  const uint32_t recv = base + uint32_t(stages) * stage_bytes;       // [split][128 / sk rows][bn] fp32, 16-byte units swizzled by row
+  const uint32_t bars = recv + uint32_t(BM) * uint32_t(bn) * 4u;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (stages + s); };
+  const uint32_t tfull = bars + 8u * (2 * stages);
+  const uint32_t tmem_slot = tfull + 8u;
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
+  volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
+
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tmem_cols = uint32_t(bn < 32 ? 32 : bn);
+  const int sp = (int)cluster_rank();
+  const int tile = int(blockIdx.x) / sk;
+  const int total_ksteps = (p.g.K + BK - 1) / BK;
+  const int k_begin = sp * p.ksteps_per_split;
+  const int ksteps = min(p.ksteps_per_split, total_ksteps - k_begin);   // >= 1 by the host's choice of sk
+  int grp, bz, mt, nt;
+  decode_tile(p, tile, grp, bz, mt, nt);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(tfull, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  cluster_arrive();   // "this CTA runs": peers may write into its receive buffer after the matching wait
+
+  if (warp == 0) {
+    // ---------------- TMA producer: one lane per 64-wide box, as in the persistent kernel ----------------
+    const bool is_a = lane < 2;
+    const int ch = is_a ? lane : lane - 2;
+    const int n_box = is_a ? (p.cfg.a_mn_major ? BM / 64 : 1) : (p.cfg.b_mn_major ? bn / 64 : 1);
+    if (lane < 6 && ch < n_box) {
+      const uint32_t box_off = (is_a ? 0u : kATileBytes) + uint32_t(ch) * 8192u;
+      const int x_r0 = is_a ? p.cfg.a_r0 : p.cfg.b_r0, x_b0 = is_a ? p.cfg.a_b0 : p.cfg.b_b0;
+      const int x_k0 = is_a ? p.cfg.a_k0 : p.cfg.b_k0;
+      int sel[5];
+#pragma unroll
+      for (int d = 0; d < 5; ++d) sel[d] = is_a ? p.cfg.a_sel[d] : p.cfg.b_sel[d];
+      int kd0 = 0, kd1 = -1;
+#pragma unroll
+      for (int d = 0; d < 5; ++d) {
+        if (sel[d] == 0) kd0 = d;
+        if (sel[d] == 1) kd1 = d;
+      }
+      int c[5];
+      {
+        int r1, r0, b1, b0;
+        split2((is_a ? mt * BM : nt * bn) + ch * 64, x_r0, r1, r0);
+        split2(bz, x_b0, b1, b0);
+        fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
+      }
+      const CUtensorMap* map = is_a ? &map_a : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2));
+      int k0, k1;
+      split2(k_begin * BK, x_k0, k1, k0);
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      pdl_wait();  // the previous step's outputs are this step's operands
+      for (int ks = 0; ks < ksteps; ++ks) {
+        if (!mbar_wait(empty_bar(s), ph ^ 1u)) { ok = false; break; }
+        if (lane == 0) mbar_expect_tx(full_bar(s), stage_bytes);
+        int q[5];
+#pragma unroll
+        for (int d = 0; d < 5; ++d) q[d] = c[d] + (d == kd0 ? k0 : 0) + (d == kd1 ? k1 : 0);
+        tma_load(base + uint32_t(s) * stage_bytes + box_off, map, full_bar(s), q[0], q[1], q[2], q[3], q[4]);
+        k0 += BK; if (k0 >= x_k0) { k0 = 0; ++k1; }
+        if (++s == stages) { s = 0; ph ^= 1u; }
+      }
+      if (!ok) {
+        if (!*abort_flag) atomicOr(p.status, 0x1u);
+        *abort_flag = 1;
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(bn, p.cfg.a_mn_major, p.cfg.b_mn_major);
+      const uint32_t a_step = p.cfg.a_mn_major ? 128u : 2u, b_step = p.cfg.b_mn_major ? 128u : 2u;
+      const uint64_t ad_first = make_desc(base, p.cfg.a_mn_major), bd_first = make_desc(base + kATileBytes, p.cfg.b_mn_major);
+      const uint32_t a_hi = uint32_t(ad_first >> 32), b_hi = uint32_t(bd_first >> 32), stage16 = stage_bytes >> 4;
+      uint32_t a_lo = uint32_t(ad_first), b_lo = uint32_t(bd_first);
+      int s = 0;
+      uint32_t ph = 0, accum = 0u;
+      bool ok = true;
+      for (int ks = 0; ks < ksteps; ++ks) {
+        if (!mbar_wait(full_bar(s), ph)) { ok = false; break; }
+        tc_fence_after();
+        umma_bf16_lohi(tmem_base, a_lo, a_hi, b_lo, b_hi, idesc, accum);
+        umma_bf16_lohi(tmem_base, a_lo + a_step, a_hi, b_lo + b_step, b_hi, idesc, 1u);
+        umma_bf16_lohi(tmem_base, a_lo + 2u * a_step, a_hi, b_lo + 2u * b_step, b_hi, idesc, 1u);
+        umma_bf16_lohi(tmem_base, a_lo + 3u * a_step, a_hi, b_lo + 3u * b_step, b_hi, idesc, 1u);
+        umma_commit(empty_bar(s));
+        accum = 1u;
+        a_lo += stage16; b_lo += stage16;
+        if (++s == stages) { s = 0; ph ^= 1u; a_lo = uint32_t(ad_first); b_lo = uint32_t(bd_first); }
+      }
+      if (ok) umma_commit(tfull);
+      if (!ok) {
+        if (!*abort_flag) atomicOr(p.status, 0x2u);
+        *abort_flag = 1;
+      }
+    }
+  }
+  const int rows_per = BM / sk;
+  bool have_acc = false;
+  if (warp >= 2) {
+    // ---------------- send: this CTA's partial rows to the CTAs that own them ----------------
+    have_acc = mbar_wait(tfull, 0u);
+    if (!have_acc && lane == 0) {
+      if (!*abort_flag) atomicOr(p.status, 0x4u);
+      *abort_flag = 1;
+    }
+    tc_fence_after();
+  }
+  __syncwarp();
+  cluster_wait();   // every CTA of the cluster has started: its shared memory may be written
+  if (warp >= 2 && have_acc) {
+    const int lane_base = (warp & 3) * 32, half = (warp - 2) >> 2;
+    const int m_loc = lane_base + lane;                 // this thread's accumulator row
+    const uint32_t dest = uint32_t(m_loc / rows_per);
+    const int lr = m_loc - int(dest) * rows_per;
+    const uint32_t row_addr = recv + uint32_t((sp * rows_per + lr) * bn) * 4u;
+    const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16);
+    const int col_begin = half * (bn / 2), col_end = col_begin + bn / 2;
+#pragma unroll 1
+    for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+      uint32_t r[32];
+      tmem_ld32(trow + uint32_t(c0), r);
+      tmem_ld_wait();
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c4 = (c0 >> 2) + u;
+        st_cluster128(row_addr + (uint32_t(c4 ^ (lr & 7)) << 4), dest, __uint_as_float(r[4 * u]), __uint_as_float(r[4 * u + 1]),
+                      __uint_as_float(r[4 * u + 2]), __uint_as_float(r[4 * u + 3]));
+      }
+    }
+    tc_fence_before();
+  }
+  __syncwarp();
+  cluster_arrive();   // release: this CTA's slices are written
+  cluster_wait();     // acquire: every peer's slices have arrived here
+  if (warp >= 2 && !*abort_flag) {
+    // ---------------- reduce the split_k slices of this CTA's rows, epilogue, store ----------------
+    const GemmParams& g = grp == 0 ? p.g : p.gx[grp - 1];
+    const int t = threadIdx.x - 64;
+    const int c4_per_row = bn >> 2;
+    const int items = rows_per * c4_per_row;
+    pdl_wait();  // before any global read (bias, residual) or write (C)
+    const int64_t cbz = split_off(bz, g.B0, g.c_s[0], g.c_s[1]);
+    const int64_t rbz = g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) : 0;
+#pragma unroll 1
+    for (int idx = t; idx < items; idx += kEpiWarps * 32) {
+      const int lr = idx / c4_per_row, c4 = idx - lr * c4_per_row;
+      const int m = mt * BM + sp * rows_per + lr, nc = nt * bn + c4 * 4;
+      const uint32_t a0 = recv + uint32_t(lr * bn) * 4u + (uint32_t(c4 ^ (lr & 7)) << 4);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int q = 0; q < sk; ++q) {
+        const float4 v = lds128(a0 + uint32_t(q * rows_per * bn) * 4u);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      if (m >= g.M || nc >= g.N) continue;
+      acc.x *= g.scale; acc.y *= g.scale; acc.z *= g.scale; acc.w *= g.scale;
+      const int64_t cb = cbz + split_off(m, g.M0, g.c_s[2], g.c_s[3]);
+      const int64_t rb = g.has_res ? rbz + split_off(m, g.M0, g.r_s[2], g.r_s[3]) : 0;
+      final_store4_c<EPI>(g, acc, cb, rb, nc);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -946,7 +1204,24 @@ int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t
   return sk;
 }
 
-cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_group, int split_k, float* partial,
+// Cluster size for the cluster split-K kernel, 0 if the step does not qualify: few output tiles (one
+// wave of CTAs even after the split), at least two k-steps per CTA, no empty split, vector epilogue.
+int gemm_cluster_split(const GemmParams* gs, const GemmTcHost& tc, int n_group) {
+  const GemmParams& g = gs[0];
+  if (g.causal != CAUSAL_NONE || tc.cfg.bn > 128) return 0;
+  if (!vec_epilogue_ok(gs, n_group, false)) return 0;
+  const int64_t tiles = int64_t((g.M + BM - 1) / BM) * ((g.N + tc.cfg.bn - 1) / tc.cfg.bn) * g.batch * n_group;
+  const int ksteps = (g.K + BK - 1) / BK;
+  for (int sk = 8; sk >= 2; sk >>= 1) {
+    if (tiles * sk > sm_count() || ksteps < 2 * sk) continue;
+    const int per = (ksteps + sk - 1) / sk;
+    if ((sk - 1) * per >= ksteps) continue;
+    return sk;
+  }
+  return 0;
+}
+
+cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_group, int split_k, int cluster_k, float* partial,
                            uint32_t* status, cudaStream_t stream) {
   const GemmParams& g = gs[0];
   const GemmTcHost& tc = tcs[0];
@@ -988,8 +1263,6 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
       p.num_tiles *= split_k;
     }
   }
-  const int grid = std::min(p.num_tiles, sm_count());
-  if (grid <= 0) return cudaSuccess;
   int epi = EPI_ANY;
   if (vec) {
     if (g.act == ACT_NONE && !g.has_res) epi = g.c_f32 ? EPI_PLAIN_WIDE : EPI_PLAIN;
@@ -998,6 +1271,50 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
     else if (g.act == ACT_GELU_ERF && !g.has_res && !g.c_f32) epi = EPI_GELU_ERF;
     else if (g.act == ACT_GELU_TANH && !g.has_res && !g.c_f32) epi = EPI_GELU_TANH;
   }
+  // ---- few tiles: one cluster of CTAs per tile, split along k, reduced through distributed shared memory ----
+  // (the caller chose cluster_k with gemm_cluster_split; it is re-derived here so that pointer alignment is checked too)
+  const int csk = (cluster_k > 1 && vec && split_k <= 1 && epi != EPI_ANY) ? gemm_cluster_split(gs, tc, n_group) : 0;
+  if (csk > 1 && p.num_tiles > 0) {
+    p.split_k = csk;
+    p.ksteps_per_split = ((g.K + BK - 1) / BK + csk - 1) / csk;
+    p.cfg.stages = std::min(tc.cfg.bn == 64 ? 6 : 4, p.ksteps_per_split);
+    const size_t csmem = size_t(p.cfg.stages) * (kATileBytes + size_t(tc.cfg.bn) * BK * 2) + size_t(BM) * tc.cfg.bn * 4 + 1024 +
+                         8 * (2 * p.cfg.stages + 1) + 16;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(p.num_tiles * csk));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = csmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = unsigned(csk); attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
+    static bool cattr_set[7] = {false, false, false, false, false, false, false};
+#define FLUID_TC_CLUSTER(E)                                                                                          \
+  case E: {                                                                                                          \
+    if (!cattr_set[E]) {                                                                                             \
+      cudaError_t e = cudaFuncSetAttribute(gemm_tc_cluster_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); \
+      if (e != cudaSuccess) return e;                                                                                \
+      cattr_set[E] = true;                                                                                           \
+    }                                                                                                                \
+    return cudaLaunchKernelEx(&cfg, gemm_tc_cluster_kernel<E>, *ma, *mb, *mb1, *mb2, p);                             \
+  }
+    switch (epi) {
+      FLUID_TC_CLUSTER(EPI_PLAIN)
+      FLUID_TC_CLUSTER(EPI_PLAIN_WIDE)
+      FLUID_TC_CLUSTER(EPI_RES)
+      FLUID_TC_CLUSTER(EPI_RES_WIDE)
+      FLUID_TC_CLUSTER(EPI_GELU_ERF)
+      FLUID_TC_CLUSTER(EPI_GELU_TANH)
+      default: break;
+    }
+#undef FLUID_TC_CLUSTER
+  }
+  const int grid = std::min(p.num_tiles, sm_count());
+  if (grid <= 0) return cudaSuccess;
   static bool attr_set[7] = {false, false, false, false, false, false, false};
 #define FLUID_TC_LAUNCH(E)                                                                                           \
   case E: {                                                                                                          \
@@ -1109,7 +1426,7 @@ extern "C" int fluid_gemm_bf16_static_scratch(const void* dev_a, const void* dev
   // the array keeps whatever the last call left: status word and arrival counters must start at zero
   err = cudaMemsetAsync(scratch, 0, kStaticHeaderBytes, st);
   if (err == cudaSuccess)
-    err = launch_gemm_tc(&g, &tc, 1, split_k, reinterpret_cast<float*>(scratch + kStaticHeaderBytes),
+    err = launch_gemm_tc(&g, &tc, 1, split_k, 0, reinterpret_cast<float*>(scratch + kStaticHeaderBytes),
                          reinterpret_cast<uint32_t*>(scratch), st);
   if (err != cudaSuccess) {
     set_error("static-scratch GEMM: %s", cudaGetErrorString(err));

@@ -167,10 +167,13 @@ cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
 // split_k > 1 cuts every output tile's k range into split_k pieces run by different CTAs; `partial`
 // then points at n_tiles * split_k * 128 * bn floats of scratch and status[8..63] hold the per-tile
 // arrival counters (zero before the launch, left zero after it).
-cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, int split_k, float* partial,
+cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, int split_k, int cluster_k, float* partial,
                            uint32_t* status, cudaStream_t stream);
 // Split factor a GEMM step should use (1 = none) and the scratch it then needs.
 int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t* scratch_bytes);
+// Cluster size of the cluster split-K form (CTAs of one cluster share an output tile, reduced through
+// distributed shared memory; no scratch); 0 if the step runs the persistent kernel.
+int gemm_cluster_split(const GemmParams* gs, const GemmTcHost& tc, int n_group);
 bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc);
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);

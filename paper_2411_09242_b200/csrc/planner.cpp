@@ -1040,7 +1040,7 @@ static int lower_and_place(fluid_plan_s* p) {
   for (int si = 0; si < (int)p->steps.size(); ++si) {
     Step& st = p->steps[si];
     const Node& n0 = p->nodes[st.node];
-    if (n0.kind != N_GEMM || !p->opts.split_k) continue;
+    if (n0.kind != N_GEMM || p->opts.split_k <= 0) continue;
     GemmParams g;
     GemmTcHost tc;
     if (!lower_gemm(p, n0, lo, &g) || !gemm_tc_eligible(p, g, &tc)) continue;

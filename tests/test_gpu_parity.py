@@ -308,10 +308,18 @@ def test_split_k_gemm_matches_oracle_and_unsplit(M, N, K):
     assert_close(split[3], ref, synth.BF16, "split-K")
     runner.run()                                   # counters are left at zero: a second run works the same
     assert np.array_equal(runner.outputs_host()[0], split[3])
-    whole, plan2, _ = run_gpu(g, feeds, synth.default_candidates(g))
+    whole, plan2, _ = run_gpu(g, feeds, synth.default_candidates(g), split_k=-1)
     assert (plan2.steps()[0]["variant"] >> 24) == 0
     assert_close(split[3], whole[3], synth.BF16, "split vs unsplit", tol=2 ** -7)
-    plan.close(); plan2.close()
+    # default options: the cut runs inside one thread-block cluster per output tile, no scratch record
+    clus, plan3, runner3 = run_gpu(g, feeds, synth.default_candidates(g))
+    v = plan3.steps()[0]["variant"]
+    assert (v >> 28) & 1 and ((v >> 24) & 15) in (2, 4, 8) and not any(r["tensor"] < 0 for r in plan3.records())
+    assert_close(clus[3], ref, synth.BF16, "cluster split-K")
+    assert_close(clus[3], whole[3], synth.BF16, "cluster split vs unsplit", tol=2 ** -7)
+    runner3.run()                                  # the summation order is fixed: bit-identical reruns
+    assert np.array_equal(runner3.outputs_host()[0], clus[3])
+    plan.close(); plan2.close(); plan3.close()
 
 
 def test_split_k_inside_a_model():

@@ -180,7 +180,7 @@ def test_fusion_folds_epilogues():
 def test_sibling_projections_share_one_launch():
     m = synth.build_model(synth.scaled(synth.CONFIGS["bert_base"], L=1), materialize=False)
     plan = fluid.Plan(m.graph, synth.default_candidates(m.graph))
-    grouped = [s for s in plan.steps() if s["kernel_name"] == "GEMM_TC" and (s["variant"] >> 20) == 3]
+    grouped = [s for s in plan.steps() if s["kernel_name"] == "GEMM_TC" and ((s["variant"] >> 20) & 15) == 3]
     assert len(grouped) == 1 and len(grouped[0]["outs"]) == 3 and len(grouped[0]["ops"]) == 3
     names = {m.graph.tensors[t]["name"] for t in grouped[0]["outs"]}
     assert names == {"l0.q", "l0.k", "l0.v"}
@@ -189,10 +189,10 @@ def test_sibling_projections_share_one_launch():
     assert len(offs) == 3 and all(o >= fluid.ARENA_HEADER for o in offs)
     ll = synth.build_model(synth.scaled(synth.CONFIGS["llama"], L=1), materialize=False)
     lp = fluid.Plan(ll.graph, synth.default_candidates(ll.graph))
-    groups = sorted((s["variant"] >> 20) for s in lp.steps() if s["kernel_name"] == "GEMM_TC" and (s["variant"] >> 20))
+    groups = sorted(((s["variant"] >> 20) & 15) for s in lp.steps() if s["kernel_name"] == "GEMM_TC" and ((s["variant"] >> 20) & 15))
     assert groups == [2, 3]                      # gate/up and q/k/v
     unfused = fluid.Plan(ll.graph, synth.default_candidates(ll.graph), fusion=0)
-    assert all((s["variant"] >> 20) == 0 for s in unfused.steps())
+    assert all(((s["variant"] >> 20) & 15) == 0 for s in unfused.steps())
     plan.close(); lp.close(); unfused.close()
 
 
@@ -245,8 +245,14 @@ def test_split_k_takes_a_step_lifetime_scratch_slice():
     on = fluid.Plan(d, synth.default_candidates(d), split_k=1)
     assert not any(r["tensor"] < 0 for r in off.records())
     scratch = [r for r in on.records() if r["tensor"] < 0]
-    split_steps = [i for i, s in enumerate(on.steps()) if s["kernel_name"] == "GEMM_TC" and (s["variant"] >> 24) > 1]
+    # bit 28 marks a cut that runs inside a thread-block cluster: it needs no scratch
+    split_steps = [i for i, s in enumerate(on.steps())
+                   if s["kernel_name"] == "GEMM_TC" and ((s["variant"] >> 24) & 15) > 1 and not (s["variant"] >> 28) & 1]
     assert len(scratch) == len(split_steps) >= 1
+    assert any((s["variant"] >> 28) & 1 for s in off.steps())
+    never = fluid.Plan(d, synth.default_candidates(d), split_k=-1)
+    assert all((s["variant"] >> 24) == 0 for s in never.steps() if s["kernel_name"] == "GEMM_TC")
+    never.close()
     assert sorted(r["first"] for r in scratch) == split_steps and all(r["first"] == r["last"] for r in scratch)
     recs, offs = plan_records(on)
     assert OA.check_arena(recs, offs, on.arena_bytes) == []
