@@ -128,6 +128,13 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 __device__ __forceinline__ void sts128(uint32_t addr, float a, float b, float c, float d) {
   asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
+// The same without the compiler-level memory clobber, for reads that follow a barrier wait (itself a
+// volatile statement with a clobber) and must not force every cached parameter to be re-read.
+__device__ __forceinline__ float4 lds128_relaxed(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ float4 lds128(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
@@ -863,12 +870,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // one of them walks the whole K range at the tensor core's fixed ~128 cycles per 128 x N x 16
 // instruction. Here a thread-block cluster of `split_k` CTAs shares one output tile: CTA r runs the
 // k-steps [r * kps, (r + 1) * kps) into its own tensor-memory accumulator, then the cluster
-// reduce-scatters the fp32 partials through distributed shared memory: CTA r receives rows
-// [r * 128 / split_k, ...) of every peer's partial, sums the split_k slices in rank order
-// (deterministic) and runs the epilogue for those rows. No global scratch, no atomics.
-// Warp roles as in the persistent kernel. Every thread of the cluster passes both cluster barriers
-// on every path (the bounded mbarrier waits only skip work), so a failed wait cannot leave a peer
-// waiting.
+// reduce-scatters the fp32 partials through distributed shared memory: every CTA lays its partial
+// tile out in its own shared memory (over the drained pipeline stages) and sends rows
+// [d * 128 / split_k, ...) to CTA d with one bulk copy that completes on d's receive barrier; CTA d
+// sums the split_k slices in rank order (deterministic) and runs the epilogue for its rows.
+// No global scratch, no atomics. Warp roles as in the persistent kernel. Every thread of the cluster
+// passes both cluster barriers on every path (the bounded mbarrier waits only skip work), so a
+// failed wait cannot leave a peer waiting; the second barrier also keeps a CTA's shared memory alive
+// until its outgoing copies have landed.
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -876,10 +885,15 @@ __device__ __forceinline__ uint32_t cluster_rank() {
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
-__device__ __forceinline__ void st_cluster128(uint32_t local_addr, uint32_t rank, float a, float b, float c, float d) {
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+  return remote;
+}
+// shared memory of this CTA -> shared memory of a CTA of the cluster, completing on that CTA's mbarrier
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t bar_cluster) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(bar_cluster) : "memory");
 }
 
 template <int ACT, bool HAS_RES, bool C_WIDE, bool R_WIDE>
@@ -933,7 +947,8 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (stages + s); };
   const uint32_t tfull = bars + 8u * (2 * stages);
-  const uint32_t tmem_slot = tfull + 8u;
+  const uint32_t recv_bar = tfull + 8u;
+  const uint32_t tmem_slot = recv_bar + 8u;
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
   volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
 
@@ -951,6 +966,7 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(tfull, 1);
+    mbar_init(recv_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
@@ -964,6 +980,7 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
+  if (threadIdx.x == 0) mbar_expect_tx(recv_bar, uint32_t(BM) * uint32_t(bn) * 4u);   // split_k slices of 128 / split_k rows
   cluster_arrive();   // "this CTA runs": peers may write into its receive buffer after the matching wait
 
   if (warp == 0) {
@@ -998,15 +1015,29 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       uint32_t ph = 0;
       bool ok = true;
       pdl_wait();  // the previous step's outputs are this step's operands
-      for (int ks = 0; ks < ksteps; ++ks) {
-        if (!mbar_wait(empty_bar(s), ph ^ 1u)) { ok = false; break; }
-        if (lane == 0) mbar_expect_tx(full_bar(s), stage_bytes);
-        int q[5];
+      if (kd1 < 0 && kd0 < 3) {
+        const int i0 = kd0 == 0 ? BK : 0, i1 = kd0 == 1 ? BK : 0, i2 = kd0 == 2 ? BK : 0;
+        c[0] += i0 ? k0 : 0; c[1] += i1 ? k0 : 0; c[2] += i2 ? k0 : 0;
+        uint32_t dst = base + box_off, fb = full_bar(0), eb = empty_bar(0);
+        for (int ks = 0; ks < ksteps; ++ks) {
+          if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
+          if (lane == 0) mbar_expect_tx(fb, stage_bytes);
+          tma_load(dst, map, fb, c[0], c[1], c[2], c[3], c[4]);
+          c[0] += i0; c[1] += i1; c[2] += i2;
+          dst += stage_bytes; fb += 8u; eb += 8u;
+          if (++s == stages) { s = 0; ph ^= 1u; dst = base + box_off; fb = full_bar(0); eb = empty_bar(0); }
+        }
+      } else {
+        for (int ks = 0; ks < ksteps; ++ks) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u)) { ok = false; break; }
+          if (lane == 0) mbar_expect_tx(full_bar(s), stage_bytes);
+          int q[5];
 #pragma unroll
-        for (int d = 0; d < 5; ++d) q[d] = c[d] + (d == kd0 ? k0 : 0) + (d == kd1 ? k1 : 0);
-        tma_load(base + uint32_t(s) * stage_bytes + box_off, map, full_bar(s), q[0], q[1], q[2], q[3], q[4]);
-        k0 += BK; if (k0 >= x_k0) { k0 = 0; ++k1; }
-        if (++s == stages) { s = 0; ph ^= 1u; }
+          for (int d = 0; d < 5; ++d) q[d] = c[d] + (d == kd0 ? k0 : 0) + (d == kd1 ? k1 : 0);
+          tma_load(base + uint32_t(s) * stage_bytes + box_off, map, full_bar(s), q[0], q[1], q[2], q[3], q[4]);
+          k0 += BK; if (k0 >= x_k0) { k0 = 0; ++k1; }
+          if (++s == stages) { s = 0; ph ^= 1u; }
+        }
       }
       if (!ok) {
         if (!*abort_flag) atomicOr(p.status, 0x1u);
@@ -1044,69 +1075,89 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     }
   }
   const int rows_per = BM / sk;
+  const uint32_t slice_bytes = uint32_t(rows_per) * uint32_t(bn) * 4u;
   bool have_acc = false;
   if (warp >= 2) {
-    // ---------------- send: this CTA's partial rows to the CTAs that own them ----------------
+    // ---------------- this CTA's partial tile -> shared memory, [128 rows][bn] fp32 over the drained stages ----------------
     have_acc = mbar_wait(tfull, 0u);
     if (!have_acc && lane == 0) {
       if (!*abort_flag) atomicOr(p.status, 0x4u);
       *abort_flag = 1;
     }
     tc_fence_after();
-  }
-  __syncwarp();
-  cluster_wait();   // every CTA of the cluster has started: its shared memory may be written
-  if (warp >= 2 && have_acc) {
-    const int lane_base = (warp & 3) * 32, half = (warp - 2) >> 2;
-    const int m_loc = lane_base + lane;                 // this thread's accumulator row
-    const uint32_t dest = uint32_t(m_loc / rows_per);
-    const int lr = m_loc - int(dest) * rows_per;
-    const uint32_t row_addr = recv + uint32_t((sp * rows_per + lr) * bn) * 4u;
-    const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16);
-    const int col_begin = half * (bn / 2), col_end = col_begin + bn / 2;
-#pragma unroll 1
-    for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+    if (have_acc) {
+      const int lane_base = (warp & 3) * 32, half = (warp - 2) >> 2;
+      const int m_loc = lane_base + lane;                 // this thread's accumulator row
+      const uint32_t row_addr = base + uint32_t(m_loc * bn) * 4u;
+      const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16);
+      const int col_begin = half * (bn / 2), col_end = col_begin + bn / 2;
       uint32_t r[32];
-      tmem_ld32(trow + uint32_t(c0), r);
-      tmem_ld_wait();
+      tmem_ld32(trow + uint32_t(col_begin), r);
+#pragma unroll 1
+      for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+        tmem_ld_wait();
+        float v[32];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int c4 = (c0 >> 2) + u;
-        st_cluster128(row_addr + (uint32_t(c4 ^ (lr & 7)) << 4), dest, __uint_as_float(r[4 * u]), __uint_as_float(r[4 * u + 1]),
-                      __uint_as_float(r[4 * u + 2]), __uint_as_float(r[4 * u + 3]));
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+        if (c0 + 32 < col_end) tmem_ld32(trow + uint32_t(c0 + 32), r);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)   // 16-byte unit c4 of row m lives at unit c4 ^ (m & 7)
+          sts128(row_addr + (uint32_t(((c0 >> 2) + u) ^ (m_loc & 7)) << 4), v[4 * u], v[4 * u + 1], v[4 * u + 2], v[4 * u + 3]);
       }
+      tc_fence_before();
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copies below read these writes
     }
-    tc_fence_before();
   }
   __syncwarp();
-  cluster_arrive();   // release: this CTA's slices are written
-  cluster_wait();     // acquire: every peer's slices have arrived here
-  if (warp >= 2 && !*abort_flag) {
+  cluster_wait();   // every CTA of the cluster has started: its shared memory and barriers may be written
+  if (warp >= 2) {
+    asm volatile("bar.sync 1, 256;" ::: "memory");   // the whole partial tile is in shared memory
+    // rows [d * rows_per, ...) go to CTA d, into the slice that belongs to this CTA's rank; CTA r starts
+    // with d = r and goes round, so that at any moment every CTA receives from one peer only
+    if (warp == 2 && lane < sk && !*abort_flag) {
+      const uint32_t d = uint32_t(sp + lane) & uint32_t(sk - 1);
+      bulk_copy_to_cta(map_to_rank(recv + uint32_t(sp) * slice_bytes, d), base + d * slice_bytes, slice_bytes, map_to_rank(recv_bar, d));
+    }
     // ---------------- reduce the split_k slices of this CTA's rows, epilogue, store ----------------
     const GemmParams& g = grp == 0 ? p.g : p.gx[grp - 1];
     const int t = threadIdx.x - 64;
-    const int c4_per_row = bn >> 2;
-    const int items = rows_per * c4_per_row;
+    const int lg = bn == 64 ? 4 : 5;              // 16-byte units per row = bn / 4
+    const int items = rows_per << lg;
     pdl_wait();  // before any global read (bias, residual) or write (C)
     const int64_t cbz = split_off(bz, g.B0, g.c_s[0], g.c_s[1]);
     const int64_t rbz = g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) : 0;
+    const float scale = g.scale;
+    const int gM = g.M, gN = g.N, gM0 = g.M0;
+    const int64_t cs2 = g.c_s[2], cs3 = g.c_s[3], rs2 = g.r_s[2], rs3 = g.r_s[3];
+    const bool has_res = g.has_res != 0;
+    bool got = mbar_wait(recv_bar, 0u);           // every peer's slice has landed (or a peer gave up)
+    if (!got && lane == 0) {
+      if (!*abort_flag) atomicOr(p.status, 0x8u);
+      *abort_flag = 1;
+    }
+    if (got) {
 #pragma unroll 1
-    for (int idx = t; idx < items; idx += kEpiWarps * 32) {
-      const int lr = idx / c4_per_row, c4 = idx - lr * c4_per_row;
-      const int m = mt * BM + sp * rows_per + lr, nc = nt * bn + c4 * 4;
-      const uint32_t a0 = recv + uint32_t(lr * bn) * 4u + (uint32_t(c4 ^ (lr & 7)) << 4);
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int q = 0; q < sk; ++q) {
-        const float4 v = lds128(a0 + uint32_t(q * rows_per * bn) * 4u);
-        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      for (int idx = t; idx < items; idx += kEpiWarps * 32) {
+        const int lr = idx >> lg, c4 = idx & ((1 << lg) - 1);
+        const int m = mt * BM + sp * rows_per + lr, nc = nt * bn + c4 * 4;
+        const uint32_t a0 = recv + uint32_t(lr * bn) * 4u + (uint32_t(c4 ^ (lr & 7)) << 4);
+        float4 part[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) part[q] = q < sk ? lds128_relaxed(a0 + uint32_t(q) * slice_bytes) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 acc = part[0];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) { acc.x += part[q].x; acc.y += part[q].y; acc.z += part[q].z; acc.w += part[q].w; }
+        if (m >= gM || nc >= gN) continue;
+        acc.x *= scale; acc.y *= scale; acc.z *= scale; acc.w *= scale;
+        const int64_t cb = cbz + split_off(m, gM0, cs2, cs3);
+        const int64_t rb = has_res ? rbz + split_off(m, gM0, rs2, rs3) : 0;
+        final_store4_c<EPI>(g, acc, cb, rb, nc);
       }
-      if (m >= g.M || nc >= g.N) continue;
-      acc.x *= g.scale; acc.y *= g.scale; acc.z *= g.scale; acc.w *= g.scale;
-      const int64_t cb = cbz + split_off(m, g.M0, g.c_s[2], g.c_s[3]);
-      const int64_t rb = g.has_res ? rbz + split_off(m, g.M0, g.r_s[2], g.r_s[3]) : 0;
-      final_store4_c<EPI>(g, acc, cb, rb, nc);
     }
   }
+  __syncwarp();
+  cluster_arrive();   // this CTA has received every slice, so every copy sent to it has completed
+  cluster_wait();     // ... and so have the copies it sent: its shared memory may go
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
