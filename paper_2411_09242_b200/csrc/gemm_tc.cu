@@ -896,40 +896,52 @@ __device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster, uint32_t 
                ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(bar_cluster) : "memory");
 }
 
+// What the last phase needs of a GemmParams, read into registers once (before the wait for the peers'
+// slices, so that the parameter reads overlap it).
+struct FinalCtx {
+  void* C;
+  const void* R;
+  const __nv_bfloat16* bias;
+  int64_t cs4, rs4;
+  int N0;
+  float scale;
+};
+
 template <int ACT, bool HAS_RES, bool C_WIDE, bool R_WIDE>
-__device__ __forceinline__ void final_store4(const GemmParams& g, float4 v, int64_t cb, int64_t rb, int nc) {
+__device__ __forceinline__ void final_store4(const FinalCtx& f, float4 v, int64_t cb, int64_t rb, int nc) {
   int n1, n0i;
-  split2(nc, g.N0, n1, n0i);
-  if (g.has_bias) {
-    const uint2 b2 = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.bias) + nc);
+  split2(nc, f.N0, n1, n0i);
+  v.x *= f.scale; v.y *= f.scale; v.z *= f.scale; v.w *= f.scale;
+  if (f.bias) {
+    const uint2 b2 = *reinterpret_cast<const uint2*>(f.bias + nc);
     v.x += __uint_as_float(b2.x << 16); v.y += __uint_as_float(b2.x & 0xffff0000u);
     v.z += __uint_as_float(b2.y << 16); v.w += __uint_as_float(b2.y & 0xffff0000u);
   }
   v.x = act_t<ACT>(v.x); v.y = act_t<ACT>(v.y); v.z = act_t<ACT>(v.z); v.w = act_t<ACT>(v.w);
   if (HAS_RES) {
-    const int64_t ro = rb + (int64_t)n1 * g.r_s[4] + n0i;
+    const int64_t ro = rb + (int64_t)n1 * f.rs4 + n0i;
     if (R_WIDE) {
-      const float4 q = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + ro);
+      const float4 q = *reinterpret_cast<const float4*>(static_cast<const float*>(f.R) + ro);
       v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
     } else {
-      const uint2 q = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.R) + ro);
+      const uint2 q = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(f.R) + ro);
       v.x += __uint_as_float(q.x << 16); v.y += __uint_as_float(q.x & 0xffff0000u);
       v.z += __uint_as_float(q.y << 16); v.w += __uint_as_float(q.y & 0xffff0000u);
     }
   }
-  const int64_t co = cb + (int64_t)n1 * g.c_s[4] + n0i;
-  if (C_WIDE) *reinterpret_cast<float4*>(static_cast<float*>(g.C) + co) = v;
-  else *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.C) + co) = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+  const int64_t co = cb + (int64_t)n1 * f.cs4 + n0i;
+  if (C_WIDE) *reinterpret_cast<float4*>(static_cast<float*>(f.C) + co) = v;
+  else *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(f.C) + co) = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
 }
 
 template <int EPI>
-__device__ __forceinline__ void final_store4_c(const GemmParams& g, float4 v, int64_t cb, int64_t rb, int nc) {
-  if (EPI == EPI_PLAIN) final_store4<ACT_NONE, false, false, false>(g, v, cb, rb, nc);
-  else if (EPI == EPI_PLAIN_WIDE) final_store4<ACT_NONE, false, true, false>(g, v, cb, rb, nc);
-  else if (EPI == EPI_RES) final_store4<ACT_NONE, true, false, false>(g, v, cb, rb, nc);
-  else if (EPI == EPI_RES_WIDE) final_store4<ACT_NONE, true, true, true>(g, v, cb, rb, nc);
-  else if (EPI == EPI_GELU_ERF) final_store4<ACT_GELU_ERF, false, false, false>(g, v, cb, rb, nc);
-  else final_store4<ACT_GELU_TANH, false, false, false>(g, v, cb, rb, nc);
+__device__ __forceinline__ void final_store4_c(const FinalCtx& f, float4 v, int64_t cb, int64_t rb, int nc) {
+  if (EPI == EPI_PLAIN) final_store4<ACT_NONE, false, false, false>(f, v, cb, rb, nc);
+  else if (EPI == EPI_PLAIN_WIDE) final_store4<ACT_NONE, false, true, false>(f, v, cb, rb, nc);
+  else if (EPI == EPI_RES) final_store4<ACT_NONE, true, false, false>(f, v, cb, rb, nc);
+  else if (EPI == EPI_RES_WIDE) final_store4<ACT_NONE, true, true, true>(f, v, cb, rb, nc);
+  else if (EPI == EPI_GELU_ERF) final_store4<ACT_GELU_ERF, false, false, false>(f, v, cb, rb, nc);
+  else final_store4<ACT_GELU_TANH, false, false, false>(f, v, cb, rb, nc);
 }
 
 template <int EPI>
@@ -1126,32 +1138,45 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     pdl_wait();  // before any global read (bias, residual) or write (C)
     const int64_t cbz = split_off(bz, g.B0, g.c_s[0], g.c_s[1]);
     const int64_t rbz = g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) : 0;
-    const float scale = g.scale;
     const int gM = g.M, gN = g.N, gM0 = g.M0;
     const int64_t cs2 = g.c_s[2], cs3 = g.c_s[3], rs2 = g.r_s[2], rs3 = g.r_s[3];
     const bool has_res = g.has_res != 0;
+    FinalCtx f;
+    f.C = g.C; f.R = g.R; f.bias = g.has_bias ? static_cast<const __nv_bfloat16*>(g.bias) : nullptr;
+    f.cs4 = g.c_s[4]; f.rs4 = g.r_s[4]; f.N0 = g.N0; f.scale = g.scale;
     bool got = mbar_wait(recv_bar, 0u);           // every peer's slice has landed (or a peer gave up)
     if (!got && lane == 0) {
       if (!*abort_flag) atomicOr(p.status, 0x8u);
       *abort_flag = 1;
     }
     if (got) {
+      // two items per pass: their shared-memory reads and address arithmetic overlap
 #pragma unroll 1
-      for (int idx = t; idx < items; idx += kEpiWarps * 32) {
-        const int lr = idx >> lg, c4 = idx & ((1 << lg) - 1);
-        const int m = mt * BM + sp * rows_per + lr, nc = nt * bn + c4 * 4;
-        const uint32_t a0 = recv + uint32_t(lr * bn) * 4u + (uint32_t(c4 ^ (lr & 7)) << 4);
-        float4 part[8];
+      for (int idx = t; idx < items; idx += 2 * kEpiWarps * 32) {
+        float4 acc[2];
+        int mm[2], nn[2];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) part[q] = q < sk ? lds128_relaxed(a0 + uint32_t(q) * slice_bytes) : make_float4(0.f, 0.f, 0.f, 0.f);
-        float4 acc = part[0];
+        for (int j = 0; j < 2; ++j) {
+          const int id = idx + j * kEpiWarps * 32;
+          const int lr = id >> lg, c4 = id & ((1 << lg) - 1);
+          mm[j] = id < items ? mt * BM + sp * rows_per + lr : gM;
+          nn[j] = nt * bn + c4 * 4;
+          const uint32_t a0 = recv + uint32_t(lr * bn) * 4u + (uint32_t(c4 ^ (lr & 7)) << 4);
+          float4 part[8];
 #pragma unroll
-        for (int q = 1; q < 8; ++q) { acc.x += part[q].x; acc.y += part[q].y; acc.z += part[q].z; acc.w += part[q].w; }
-        if (m >= gM || nc >= gN) continue;
-        acc.x *= scale; acc.y *= scale; acc.z *= scale; acc.w *= scale;
-        const int64_t cb = cbz + split_off(m, gM0, cs2, cs3);
-        const int64_t rb = has_res ? rbz + split_off(m, gM0, rs2, rs3) : 0;
-        final_store4_c<EPI>(g, acc, cb, rb, nc);
+          for (int q = 0; q < 8; ++q)
+            part[q] = (q < sk && id < items) ? lds128_relaxed(a0 + uint32_t(q) * slice_bytes) : make_float4(0.f, 0.f, 0.f, 0.f);
+          acc[j] = part[0];
+#pragma unroll
+          for (int q = 1; q < 8; ++q) { acc[j].x += part[q].x; acc[j].y += part[q].y; acc[j].z += part[q].z; acc[j].w += part[q].w; }
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          if (mm[j] >= gM || nn[j] >= gN) continue;
+          const int64_t cb = cbz + split_off(mm[j], gM0, cs2, cs3);
+          const int64_t rb = has_res ? rbz + split_off(mm[j], gM0, rs2, rs3) : 0;
+          final_store4_c<EPI>(f, acc[j], cb, rb, nn[j]);
+        }
       }
     }
   }

@@ -227,7 +227,12 @@ bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc) {
   if (g.N <= 64) bn = 64;
   else {
     const int64_t tiles256 = int64_t((g.M + 127) / 128) * ((g.N + 255) / 256) * g.batch;
+    const int64_t tiles64 = int64_t((g.M + 127) / 128) * ((g.N + 63) / 64) * g.batch;
     if (g.N >= 256 && tiles256 >= 74) bn = 256;
+    // few tiles and a k range worth cutting: the step will run as clusters that split k (the tensor core
+    // spends the same time on a 128 x 64 x 16 instruction as on a 128 x 128 x 16 one, and the narrower
+    // tile halves what the cluster has to exchange), if four CTAs per tile still fit one wave
+    else if (g.causal == CAUSAL_NONE && g.K >= 256 && tiles64 * 4 <= 148) bn = 64;
   }
   const int64_t a_rs[2] = {g.a_s[2], g.a_s[3]}, a_ks[2] = {g.a_s[4], g.a_s[5]}, a_bs[2] = {g.a_s[0], g.a_s[1]};
   const int64_t b_rs[2] = {g.b_s[4], g.b_s[5]}, b_ks[2] = {g.b_s[2], g.b_s[3]}, b_bs[2] = {g.b_s[0], g.b_s[1]};

@@ -14,10 +14,10 @@ from tests.helpers import assert_close, ensure_lib, rand_feed, run_gpu, single_o
 
 def test_sizes_beyond_the_static_array_are_rejected():
     ensure_lib()
-    # 128 x 2304 x 4096: 18 tiles of 128x128, split 8 ways, 64 KiB each = 9.4 MB > 8 MiB: refused before any
+    # 128 x 2432 x 4096: 19 tiles of 128x128, split 7 ways, 64 KiB each = 8.7 MB > 8 MiB: refused before any
     # device work is attempted
     with pytest.raises(fluid.FluidError) as e:
-        fluid.fluid_gemm_bf16_static_scratch(0x1000, 0x2000, 0, 0x3000, 128, 2304, 4096)
+        fluid.fluid_gemm_bf16_static_scratch(0x1000, 0x2000, 0, 0x3000, 128, 2432, 4096)
     assert e.value.code == fluid.FLUID_EINVAL and "static array holds" in str(e.value)
     with pytest.raises(fluid.FluidError) as e:          # K not a multiple of 8
         fluid.fluid_gemm_bf16_static_scratch(0x1000, 0x2000, 0, 0x3000, 128, 768, 100)
