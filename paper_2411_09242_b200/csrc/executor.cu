@@ -52,6 +52,7 @@ int finalize_steps(fluid_plan_s* p) {
         s.t_narrow[0] = s.t_narrow[1] = 1;
         s.gemm.c_f32 = p->wide[n.out];
         s.gemm.r_f32 = n.res >= 0 ? p->wide[n.res] : 0;
+        s.gemm.b_const = p->graph.tensors[n.b].kind == FLUID_CONST ? 1 : 0;
         double fl = 2.0 * double(g.batch) * g.M * double(g.N) * g.K;
         double a = double(g.batch) * g.M * double(g.K), b = double(g.batch) * g.K * double(g.N),
                c = double(g.batch) * g.M * double(g.N);
@@ -72,6 +73,7 @@ int finalize_steps(fluid_plan_s* p) {
             return FLUID_EUNSUPPORTED;
           }
           gx.c_f32 = p->wide[m.out];
+          gx.b_const = p->graph.tensors[m.b].kind == FLUID_CONST ? 1 : 0;
           s.x_ptr[gi - 1][0] = m.b; s.x_ptr[gi - 1][1] = m.out; s.x_ptr[gi - 1][2] = m.bias;
           s.flops += fl;
           s.bytes += es * (b + c + (g.has_bias ? g.N : 0));

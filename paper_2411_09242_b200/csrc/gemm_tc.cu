@@ -659,7 +659,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const bool k_simple = kd1 < 0 && kd0 < 3;
       const int i0 = kd0 == 0 ? BK : 0, i1 = kd0 == 1 ? BK : 0, i2 = kd0 == 2 ? BK : 0;
       uint32_t dst = base + box_off, fb = full_bar(0), eb = empty_bar(0);   // the running stage
-      pdl_wait();  // the previous step's outputs are this step's operands
+      // The previous step's outputs are this step's operands, except for weights: a constant B is loaded
+      // while the previous step is still finishing (its bytes may land before lane 0 posts the expected
+      // count; the barrier's pending arrival keeps the phase open until then).
+      const bool b_free = p.g.b_const && (p.n_group < 2 || p.gx[0].b_const) && (p.n_group < 3 || p.gx[1].b_const);
+      if (is_a || !b_free) pdl_wait();
       for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
         int tile, sp, k_begin, k_count;
         decode_item<SPLIT>(p, item, tile, sp, k_begin, k_count);
@@ -1026,7 +1030,9 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      pdl_wait();  // the previous step's outputs are this step's operands
+      // weights do not wait for the previous step (see the persistent kernel's producer)
+      const bool b_free = p.g.b_const && (p.n_group < 2 || p.gx[0].b_const) && (p.n_group < 3 || p.gx[1].b_const);
+      if (is_a || !b_free) pdl_wait();
       if (kd1 < 0 && kd0 < 3) {
         const int i0 = kd0 == 0 ? BK : 0, i1 = kd0 == 1 ? BK : 0, i2 = kd0 == 2 ? BK : 0;
         c[0] += i0 ? k0 : 0; c[1] += i1 ? k0 : 0; c[2] += i2 ? k0 : 0;

@@ -36,6 +36,7 @@ struct GemmParams {
   int causal;  // CAUSAL_SKIP_UPPER: tiles with n > m everywhere are not computed;
                // CAUSAL_CLIP_K: the k loop stops after the tile holding k = m_max
   int has_bias, has_res;
+  int b_const;  // B is a constant of the plan (a weight): its loads need not wait for the previous step
 };
 
 // Host-side description of the two TMA tensor maps of a tensor-core GEMM step.

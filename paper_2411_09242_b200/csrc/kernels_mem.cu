@@ -183,7 +183,6 @@ __device__ __forceinline__ float row_sum(float v, float* red, int warp, int lane
 template <typename T, int NCH, int WPR>
 __global__ void __launch_bounds__(256) norm_warp_kernel(NormParams p) {
   pdl_launch_dependents();
-  pdl_wait();
   constexpr int V = VecOf<T>::N;
   __shared__ float red[8];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -192,6 +191,22 @@ __global__ void __launch_bounds__(256) norm_warp_kernel(NormParams p) {
   const size_t roff = (size_t)(live ? row : 0) * p.width;
   const int nch = live ? p.width / V : 0;
   const int c_first = (warp % WPR) * 32 + lane;
+  // gain and bias are constants of the plan, not outputs of the previous step: they are fetched while
+  // that step is still finishing
+  const T* gamma = static_cast<const T*>(p.gamma);
+  const T* beta = static_cast<const T*>(p.beta);
+  float gv[NCH][V], bv[NCH][V];
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const int c = c_first + 32 * WPR * j;
+#pragma unroll
+    for (int i = 0; i < V; ++i) bv[j][i] = 0.f;
+    if (c < nch) {
+      norm_load<T, V>(gamma, false, 0, c, gv[j]);
+      if (beta) norm_load<T, V>(beta, false, 0, c, bv[j]);
+    }
+  }
+  pdl_wait();
   float v[NCH][V];
   float s = 0.f;
 #pragma unroll
@@ -236,17 +251,13 @@ __global__ void __launch_bounds__(256) norm_warp_kernel(NormParams p) {
     rstd = rsqrtf(q / p.width + p.eps);
   }
   T* y_lo = static_cast<T*>(p.y_lo);
-  const T* gamma = static_cast<const T*>(p.gamma);
-  const T* beta = static_cast<const T*>(p.beta);
 #pragma unroll
   for (int j = 0; j < NCH; ++j) {
     const int c = c_first + 32 * WPR * j;
     if (c < nch) {
-      float g[V], b[V], o[V];
-      norm_load<T, V>(gamma, false, 0, c, g);
-      if (beta) norm_load<T, V>(beta, false, 0, c, b);
+      float o[V];
 #pragma unroll
-      for (int i = 0; i < V; ++i) o[i] = (v[j][i] - mean) * rstd * g[i] + (beta ? b[i] : 0.f);
+      for (int i = 0; i < V; ++i) o[i] = (v[j][i] - mean) * rstd * gv[j][i] + bv[j][i];
       if (y_lo) {
         float t8[VecOf<T>::N];
 #pragma unroll
