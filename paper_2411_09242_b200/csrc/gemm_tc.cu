@@ -53,6 +53,7 @@ struct TcParams {
   int ksteps_per_split;
   float* partial;       // split-K scratch: [tile][split][bn/4][128 rows][4] fp32
   uint32_t* status;     // word 0: device status; words 8..63: per-tile arrival counters for split-K
+  int scalar_turn;      // general epilogue: n is contiguous and unsplit in C (and R), so the shared-memory turn applies
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -541,6 +542,52 @@ __device__ __noinline__ void epilogue_group_any(const GemmParams& g, uint32_t ta
   }
 }
 
+// General epilogue for outputs whose rows are not 16-byte aligned (an odd N, e.g. a vocabulary size)
+// but whose n index is contiguous and unsplit: the same shared-memory turn as the vector variants, then
+// scalar loads and stores, so that the lanes of a warp still cover runs of consecutive columns instead
+// of one row each. Flags are read at run time (this is the rare path).
+__device__ __noinline__ void epilogue_tile_scalar(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
+                                                  int64_t cbz, int64_t rbz, int m_base, float* stage, int lane) {
+  const int unit = lane & 7, rsub = lane >> 3;
+  const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
+  const bool c_wide = g.c_f32 != 0, r_wide = g.r_f32 != 0;
+  const float scale = g.scale;
+#pragma unroll 1
+  for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+    if (n_tile0 + c0 >= g.N) break;   // uniform across the warp
+    uint32_t r[32];
+    tmem_ld32(trow + uint32_t(c0), r);
+    tmem_ld_wait();
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      sts128(st_row + (uint32_t(u ^ (lane & 7)) << 4), __uint_as_float(r[4 * u]) * scale, __uint_as_float(r[4 * u + 1]) * scale,
+             __uint_as_float(r[4 * u + 2]) * scale, __uint_as_float(r[4 * u + 3]) * scale);
+    __syncwarp();
+    const int nc = n_tile0 + c0 + unit * 4;
+#pragma unroll 1
+    for (int i = 0; i < 8; ++i) {
+      const int row = rsub + 4 * i, m = m_base + row;
+      if (m >= g.M) break;            // rows only grow with i
+      const float4 q = lds128(st_base + uint32_t(row * 128) + (uint32_t(unit ^ (row & 7)) << 4));
+      const float v4[4] = {q.x, q.y, q.z, q.w};
+      const int64_t cb = cbz + split_off(m, g.M0, g.c_s[2], g.c_s[3]);
+      const int64_t rb = g.has_res ? rbz + split_off(m, g.M0, g.r_s[2], g.r_s[3]) : 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int n = nc + e;
+        if (n >= g.N) break;
+        float v = v4[e];
+        if (g.has_bias) v += to_f(static_cast<const __nv_bfloat16*>(g.bias)[n]);
+        v = g.act == ACT_GELU_ERF ? gelu_erf_fast(v) : (g.act == ACT_GELU_TANH ? gelu_tanh(v) : v);
+        if (g.has_res) v += r_wide ? static_cast<const float*>(g.R)[rb + n] : to_f(static_cast<const __nv_bfloat16*>(g.R)[rb + n]);
+        if (c_wide) static_cast<float*>(g.C)[cb + n] = v;
+        else static_cast<__nv_bfloat16*>(g.C)[cb + n] = __float2bfloat16_rn(v);
+      }
+    }
+    __syncwarp();   // the staging tile is rewritten by the next chunk
+  }
+}
+
 // Epilogue variants (template parameter of the kernel)
 enum EpiKind { EPI_ANY = 0, EPI_PLAIN = 1, EPI_PLAIN_WIDE = 2, EPI_RES = 3, EPI_RES_WIDE = 4, EPI_GELU_ERF = 5, EPI_GELU_TANH = 6 };
 
@@ -804,7 +851,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn);
       if (!SPLIT) {
-        if (EPI == EPI_ANY) {
+        if (EPI == EPI_ANY && p.scalar_turn) {
+          epilogue_tile_scalar(g, trow, col_begin, col_end, n_tile0, split_off(bz, g.B0, g.c_s[0], g.c_s[1]),
+                               g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) : 0, mt * BM + lane_base, stage, lane);
+        } else if (EPI == EPI_ANY) {
 #pragma unroll 1
           for (int c0 = col_begin; c0 < col_end; c0 += 32) {
             if (n_tile0 + c0 >= g.N) break;  // whole chunk out of range (uniform across the warp)
@@ -1334,6 +1384,9 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
   // The vector epilogues need: n contiguous in C (and R), 8-column groups aligned to 16 bytes and
   // inside one n split, N a multiple of 8. Everything else takes the general epilogue.
   const bool vec = vec_epilogue_ok(gs, n_group, true);
+  p.scalar_turn = 1;
+  for (int i = 0; i < n_group; ++i)
+    if (gs[i].c_s[5] != 1 || gs[i].N0 != gs[i].N || (gs[i].has_res && gs[i].r_s[5] != 1)) p.scalar_turn = 0;
   if (!vec || !partial) split_k = 1;   // the general epilogue does not take part in split-K
   p.split_k = split_k;
   p.partial = partial;
