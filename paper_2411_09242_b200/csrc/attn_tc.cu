@@ -62,6 +62,14 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_c, uint64_t adesc, uint6
   asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
+// Descriptors given as 32-bit halves: only the low word (the address field) differs between the MMAs of a tile.
+__device__ __forceinline__ void umma_bf16_lohi(uint32_t tmem_c, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n .reg .b64 da, db;\n mov.b64 da, {%1, %2};\n mov.b64 db, {%3, %4};\n setp.ne.b32 p, %6, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}"
+      ::"r"(tmem_c), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -99,257 +107,367 @@ __device__ __forceinline__ void coords(const int* sel, int k, int r, int bz, int
   }
 }
 
+__device__ __forceinline__ float ex2_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&q)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3]), "r"(q[4]), "r"(q[5]), "r"(q[6]),
+      "r"(q[7]), "r"(q[8]), "r"(q[9]), "r"(q[10]), "r"(q[11]), "r"(q[12]), "r"(q[13]), "r"(q[14]), "r"(q[15]),
+      "r"(q[16]), "r"(q[17]), "r"(q[18]), "r"(q[19]), "r"(q[20]), "r"(q[21]), "r"(q[22]), "r"(q[23]), "r"(q[24]),
+      "r"(q[25]), "r"(q[26]), "r"(q[27]), "r"(q[28]), "r"(q[29]), "r"(q[30]), "r"(q[31])
+      : "memory");
+}
+
+constexpr int kSoftmaxThreads = 256;
+constexpr int kAttnThreads = kSoftmaxThreads + 64;   // warps 0-7 softmax (two threads per query row), warp 8 MMAs, warp 9 loads
+
+// Warps 0-7: softmax. Warp 8, one thread: every tcgen05.mma. Warp 9: TMA loads. They meet only at mbarriers:
+//   s_full[i]  S tile i (of two, in tensor memory) holds Q.K_j^T          MMA commit -> softmax
+//   p_full[i]  P tile i (of two, in shared memory) is written and S tile i is read    256 softmax threads -> MMA
+//   o_done[i]  P_j.V_j has been accumulated into O (j odd / even)         MMA commit -> softmax (rescale, P reuse, end)
+//   k_full[i], v_full[i]  K / V stage i has landed                        TMA -> MMA
+// (the loader reuses a K stage when s_full says its Q.K^T has run, a V stage when o_done says its P.V has)
+// so the tensor core works on Q.K_{j+2}^T and P_j.V_j while the softmax warps are on tile j+1.
 template <int D>
-__global__ void __launch_bounds__(256, D == 64 ? 2 : 1)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const __grid_constant__ AttnParams p) {
   constexpr int DC = D / 64;                       // 64-wide chunks of the head dim
   constexpr uint32_t kTile = TQ * D * 2;           // bytes of one Q / K / V tile
   constexpr uint32_t kPBytes = TQ * TK * 2;
-  extern __shared__ uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;
-  const uint32_t sQ = base, sK = sQ + kTile, sV = sK + 2 * kTile, sP = sV + 2 * kTile, bars = sP + kPBytes;
-  const uint32_t bar_q = bars, bar_kv0 = bars + 8, bar_s = bars + 24, bar_o = bars + 32, tmem_slot = bars + 40;
-  float* xch = reinterpret_cast<float*>(smem_raw + (bars + 64 - raw));   // [2][128] row-max / row-sum exchange
+  const uint32_t base = raw;                       // 1024-byte aligned (checked below): the tiles leave no slack for rounding
+  const uint32_t sQ = base, sK = sQ + kTile, sV = sK + 2 * kTile, sP = sV + 2 * kTile, bars = sP + 2 * kPBytes;
+  const uint32_t bar_q = bars, k_full = bars + 8, v_full = bars + 24, s_full = bars + 40, p_full = bars + 56, o_done = bars + 72;
+  const uint32_t tmem_slot = bars + 88;
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
+  volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
+  float* xch = reinterpret_cast<float*>(smem_raw + (bars + 128 - raw));   // [2 tiles][2 halves][128 rows]
   uint8_t* p_smem = smem_raw + (sP - raw);
 
   pdl_launch_dependents();
-  const int warp = threadIdx.x >> 5, row = threadIdx.x & 127, half = threadIdx.x >> 7;
+  const int warp = threadIdx.x >> 5;
   // CTAs are issued heaviest first: with a causal mask the last query tiles see the most key tiles,
   // so they start first and the short ones fill the gaps (longest-processing-time order)
   const int n_bz = p.B * p.NH;
   const int mt = (int(gridDim.x) / n_bz - 1) - int(blockIdx.x) / n_bz, bz = int(blockIdx.x) % n_bz;
   const int h = bz % p.NH, b = bz / p.NH;
-  const int m0 = mt * TQ, qi = m0 + row;
+  const int m0 = mt * TQ;
   int n_kv = (p.S + TK - 1) / TK;
   if (p.causal) n_kv = min(n_kv, (m0 + TQ - 1) / TK + 1);
+  if (raw & 1023u) {   // cannot happen with the launch this file does; refuse rather than run misaligned tiles
+    if (threadIdx.x == 0) atomicOr(p.status, 0x100u | 0x08u);
+    return;
+  }
 
   if (threadIdx.x == 0) {
-    mbar_init(bar_q, 1); mbar_init(bar_kv0, 1); mbar_init(bar_kv0 + 8, 1); mbar_init(bar_s, 1); mbar_init(bar_o, 1);
+    mbar_init(bar_q, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(k_full + 8 * i, 1); mbar_init(v_full + 8 * i, 1); mbar_init(s_full + 8 * i, 1);
+      mbar_init(p_full + 8 * i, kSoftmaxThreads); mbar_init(o_done + 8 * i, 1);
+    }
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(256u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
-  const uint32_t tS = tmem_base, tO = tmem_base + TK;     // score columns, then PV columns
-  const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;   // warps w and w+4 share a lane quarter
+  const uint32_t tS = tmem_base, tO = tmem_base + 2 * TK;     // two score tiles, then the output accumulator
 
-  pdl_wait();  // Q, K, V come from the previous steps
+  if (warp == 9) {
+    // ======================= loads =======================
+    // Lane 0 does every wait. The TMA boxes of a K or V tile (four for D = 128, two for D = 64) each
+    // belong to one lane, which keeps that box's coordinates in registers and advances them by one key
+    // tile per load: the divisions and selects behind a coordinate are done once.
+    const int lane = threadIdx.x & 31;
+    const bool lead = lane == 0;
+    constexpr int NB = 2 * DC;               // boxes per tile
+    const bool k_lane = lane < NB, v_lane = lane >= NB && lane < 2 * NB;
+    const int bx = k_lane ? lane : lane - NB;
+    int cur[5] = {0, 0, 0, 0, 0}, inc[5] = {0, 0, 0, 0, 0};
+    uint32_t box_dst = 0;
+    if (k_lane) {
+      if (!p.k_mn_major) {          // [d chunk][128 keys][64 d]: box (dc, rh)
+        const int dc = bx >> 1, rh = bx & 1;
+        coords(p.k_sel, dc * 64, rh * 64, bz, p.k_b0, cur);
+        box_dst = sK + dc * 16384u + rh * 8192u;
+      } else {                      // [key chunk][D d-rows][64 keys]: box (sc, dc)
+        const int sc = bx / DC, dc = bx % DC;
+        coords(p.k_sel, dc * 64, sc * 64, bz, p.k_b0, cur);
+        box_dst = sK + sc * (D * 128u) + dc * 8192u;
+      }
+#pragma unroll
+      for (int d = 0; d < 5; ++d) inc[d] = p.k_sel[d] == 2 ? TK : 0;   // the key index is K's row index
+    } else if (v_lane) {
+      if (!p.v_k_major) {           // [d chunk][128 keys][64 d]  (MN-major B of P.V): box (dc, kc)
+        const int dc = bx >> 1, kc = bx & 1;
+        coords(p.v_sel, kc * 64, dc * 64, bz, p.v_b0, cur);
+        box_dst = sV + dc * 16384u + kc * 8192u;
+      } else {                      // [key chunk][D d-rows][64 keys]  (K-major B of P.V): box (kc, dh)
+        const int kc = bx / DC, dh = bx % DC;
+        coords(p.v_sel, kc * 64, dh * 64, bz, p.v_b0, cur);
+        box_dst = sV + kc * (D * 128u) + dh * 8192u;
+      }
+#pragma unroll
+      for (int d = 0; d < 5; ++d) inc[d] = p.v_sel[d] == 0 ? TK : 0;   // the key index is V's contraction index
+    }
+    uint32_t fail = 0;
+    int k_issued = 0, v_issued = 0;   // tiles whose loads have been issued (uniform across the warp)
+    auto load_k = [&](int j) {        // called by the whole warp
+      const uint32_t bar = k_full + 8u * (j & 1);
+      if (lead) mbar_expect_tx(bar, kTile);
+      if (k_lane) {
+        tma_load5(box_dst + uint32_t(j & 1) * kTile, &map_k, bar, cur);
+#pragma unroll
+        for (int d = 0; d < 5; ++d) cur[d] += inc[d];
+      }
+      k_issued = j + 1;
+    };
+    auto load_v = [&](int j) {
+      const uint32_t bar = v_full + 8u * (j & 1);
+      if (lead) mbar_expect_tx(bar, kTile);
+      if (v_lane) {
+        tma_load5(box_dst + uint32_t(j & 1) * kTile, &map_v, bar, cur);
+#pragma unroll
+        for (int d = 0; d < 5; ++d) cur[d] += inc[d];
+      }
+      v_issued = j + 1;
+    };
+    auto all_ok = [&](bool mine) { return __shfl_sync(0xffffffffu, mine ? 1 : 0, 0) != 0; };   // lane 0 decides; also re-converges the warp
 
-  // ---- loads (thread 0) ----
-  bool pending[2] = {false, false};   // thread 0: loads issued into a stage and not yet waited for
-  auto load_kv = [&](int j, int st) {
-    pending[st] = true;
-    const uint32_t bar = bar_kv0 + 8u * st;
-    mbar_expect_tx(bar, 2 * kTile);
-    const int kv0 = j * TK;
-    int c[5];
-    const uint32_t k_dst = sK + st * kTile, v_dst = sV + st * kTile;
-    if (!p.k_mn_major) {          // [d chunk][128 keys][64 d]
+    pdl_wait();  // Q, K, V come from the previous steps
+    if (lead) {
+      mbar_expect_tx(bar_q, kTile);
+      int c[5];
       for (int dc = 0; dc < DC; ++dc)
         for (int rh = 0; rh < 2; ++rh) {
-          coords(p.k_sel, dc * 64, kv0 + rh * 64, bz, p.k_b0, c);
-          tma_load5(k_dst + dc * 16384u + rh * 8192u, &map_k, bar, c);
-        }
-    } else {                      // [key chunk][D d-rows][64 keys]
-      for (int sc = 0; sc < 2; ++sc)
-        for (int dc = 0; dc < DC; ++dc) {
-          coords(p.k_sel, dc * 64, kv0 + sc * 64, bz, p.k_b0, c);
-          tma_load5(k_dst + sc * (D * 128u) + dc * 8192u, &map_k, bar, c);
+          coords(p.q_sel, dc * 64, m0 + rh * 64, bz, p.q_b0, c);
+          tma_load5(sQ + dc * 16384u + rh * 8192u, &map_q, bar_q, c);
         }
     }
-    if (!p.v_k_major) {           // [d chunk][128 keys][64 d]  (MN-major B of P.V)
-      for (int dc = 0; dc < DC; ++dc)
-        for (int kc = 0; kc < 2; ++kc) {
-          coords(p.v_sel, kv0 + kc * 64, dc * 64, bz, p.v_b0, c);
-          tma_load5(v_dst + dc * 16384u + kc * 8192u, &map_v, bar, c);
-        }
-    } else {                      // [key chunk][D d-rows][64 keys]  (K-major B of P.V)
-      for (int kc = 0; kc < 2; ++kc)
-        for (int dh = 0; dh < DC; ++dh) {
-          coords(p.v_sel, kv0 + kc * 64, dh * 64, bz, p.v_b0, c);
-          tma_load5(v_dst + kc * (D * 128u) + dh * 8192u, &map_v, bar, c);
-        }
+    load_k(0);
+    if (n_kv > 1) load_k(1);
+    load_v(0);
+    if (n_kv > 1) load_v(1);
+    bool ok = true;
+    for (int j = 0; ok && j + 2 < n_kv; ++j) {
+      const int st = j & 1;
+      const uint32_t ph = uint32_t(j >> 1) & 1u;
+      // K stage st is free once Q.K_j^T has run
+      if (lead && !mbar_wait(s_full + 8u * st, ph)) { fail |= 0x40u; ok = false; }
+      ok = all_ok(ok);
+      if (!ok) break;
+      load_k(j + 2);
+      // V stage st is free once P_j.V_j has run
+      if (lead && !mbar_wait(o_done + 8u * st, ph)) { fail |= 0x80u; ok = false; }
+      ok = all_ok(ok && !*abort_flag);
+      if (!ok) break;
+      load_v(j + 2);
     }
-  };
-  if (threadIdx.x == 0) {
-    mbar_expect_tx(bar_q, kTile);
-    int c[5];
-    for (int dc = 0; dc < DC; ++dc)
-      for (int rh = 0; rh < 2; ++rh) {
-        coords(p.q_sel, dc * 64, m0 + rh * 64, bz, p.q_b0, c);
-        tma_load5(sQ + dc * 16384u + rh * 8192u, &map_q, bar_q, c);
-      }
-    load_kv(0, 0);
-    if (n_kv > 1) load_kv(1, 1);
-  }
-
-  const uint32_t idesc_s = make_idesc(TK, 0, p.k_mn_major);
-  const uint32_t idesc_o = make_idesc(D, 0, p.v_k_major ? 0 : 1);
-  // m_used is the (possibly stale) row maximum the exponentials are taken against; O (in tensor
-  // memory) and l are rescaled only when the true maximum has moved by more than 2^8, so most
-  // key tiles accumulate P.V straight into tensor memory with no traffic on O at all.
-  float m_used = -INFINITY, l_run = 0.f;
-  bool ok = true;
-  uint32_t fail = 0;
-
-  auto issue_qk = [&](int j) {   // thread 0: S = Q.K_j^T
-    const int st = j & 1;
-    if (!mbar_wait(bar_kv0 + 8u * st, uint32_t(j >> 1) & 1u)) { fail |= 0x20u; return; }
-    pending[st] = false;
-    tc_fence_after();
-    const uint32_t kb = sK + st * kTile;
+    if (!ok && lead) {
+      *abort_flag = 1;
+      if (fail) atomicOr(p.status, 0x100u | fail);
+    }
+    if (lead && *abort_flag) {
+      // let loads still in flight land before the shared memory is given up (each wait is bounded)
+      for (int j = max(0, k_issued - 2); j < k_issued; ++j) mbar_wait(k_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
+      for (int j = max(0, v_issued - 2); j < v_issued; ++j) mbar_wait(v_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
+    }
+  } else if (warp == 8) {
+    // ======================= MMAs (one thread) =======================
+    if (threadIdx.x == kSoftmaxThreads) {
+      uint32_t fail = 0;
+      const uint32_t idesc_s = make_idesc(TK, 0, p.k_mn_major);
+      const uint32_t idesc_o = make_idesc(D, 0, p.v_k_major ? 0 : 1);
+      // descriptor halves: the high word is fixed per operand kind, the low word is base + a per-slice
+      // offset (16-byte units) + the stage offset
+      const uint64_t dq = make_desc(sQ, 16, 1024);
+      const uint64_t dk = p.k_mn_major ? make_desc(sK, D * 128u, 1024) : make_desc(sK, 16, 1024);
+      const uint64_t dp = make_desc(sP, 16, 1024);
+      const uint64_t dv = p.v_k_major ? make_desc(sV, 16, 1024) : make_desc(sV, 16384, 1024);
+      const uint32_t q_hi = uint32_t(dq >> 32), k_hi = uint32_t(dk >> 32), p_hi = uint32_t(dp >> 32), v_hi = uint32_t(dv >> 32);
+      const uint32_t q_lo = uint32_t(dq), k_lo = uint32_t(dk), p_lo = uint32_t(dp), v_lo = uint32_t(dv);
+      auto km_off = [](int kk) { return uint32_t(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4); };   // K-major operand, 64-wide chunks
+      auto issue_qk = [&](int j) -> bool {   // S[j & 1] = Q.K_j^T
+        const int st = j & 1;
+        if (!mbar_wait(k_full + 8u * st, uint32_t(j >> 1) & 1u)) { fail |= 0x20u; return false; }
+        tc_fence_after();
+        const uint32_t kb = k_lo + uint32_t(st) * (kTile >> 4);
 #pragma unroll
-    for (int kk = 0; kk < D / 16; ++kk) {
-      const uint64_t ad = make_desc(sQ + (kk >> 2) * 16384u + (kk & 3) * 32u, 16, 1024);
-      const uint64_t bd = p.k_mn_major ? make_desc(kb + kk * 2048u, D * 128u, 1024)
-                                       : make_desc(kb + (kk >> 2) * 16384u + (kk & 3) * 32u, 16, 1024);
-      umma_bf16(tS, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
+        for (int kk = 0; kk < D / 16; ++kk)
+          umma_bf16_lohi(tS + uint32_t(st * TK), q_lo + km_off(kk), q_hi, kb + (p.k_mn_major ? uint32_t(kk * 128) : km_off(kk)), k_hi,
+                         idesc_s, kk > 0 ? 1u : 0u);
+        umma_commit(s_full + 8u * st);
+        return true;
+      };
+      bool ok = mbar_wait(bar_q, 0);
+      if (!ok) fail |= 0x10u;
+      ok = ok && issue_qk(0);
+      if (ok && n_kv > 1) ok = issue_qk(1);
+      for (int j = 0; ok && j < n_kv; ++j) {
+        const int st = j & 1;
+        const uint32_t ph = uint32_t(j >> 1) & 1u;
+        // P_j is in shared memory and S tile st has been read
+        if (!mbar_wait(p_full + 8u * st, ph)) { fail |= 0x200u; ok = false; break; }
+        if (!mbar_wait(v_full + 8u * st, ph)) { fail |= 0x20u; ok = false; break; }
+        tc_fence_after();
+        const uint32_t vb = v_lo + uint32_t(st) * (kTile >> 4), pb = p_lo + uint32_t(st) * (kPBytes >> 4);
+#pragma unroll
+        for (int kk = 0; kk < TK / 16; ++kk)   // O accumulates across key tiles
+          umma_bf16_lohi(tO, pb + km_off(kk), p_hi,
+                         vb + (p.v_k_major ? uint32_t(((kk >> 2) * (D * 128) + (kk & 3) * 32) >> 4) : uint32_t(kk * 128)), v_hi, idesc_o,
+                         (j > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(o_done + 8u * st);
+        if (j + 2 < n_kv && !issue_qk(j + 2)) { ok = false; break; }   // into the S tile that was just read
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicOr(p.status, 0x100u | fail);
+      }
     }
-    umma_commit(bar_s);
-  };
-
-  if (!mbar_wait(bar_q, 0)) { ok = false; fail = 0x10u; }
-  ok = __syncthreads_and(ok);
-  if (ok && threadIdx.x == 0) issue_qk(0);
-  for (int j = 0; ok && j < n_kv; ++j) {
-    const int st = j & 1;
-    const uint32_t ph = uint32_t(j) & 1u;
-    const int kv0 = j * TK;
-    if (!mbar_wait(bar_s, ph)) { ok = false; fail |= 0x40u; }
-    ok = __syncthreads_and(ok);   // leave the loop together
-    if (!ok) break;
-    tc_fence_after();
-    // ---- this thread owns half (64 columns) of query row qi: read its scores once ----
+  } else {
+    // ======================= softmax (256 threads, two per query row) =======================
+    const int row = threadIdx.x & 127, half = threadIdx.x >> 7;
+    const int qi = m0 + row;
+    const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;   // warps w and w+4 share a lane quarter
     constexpr int HC = TK / 2;
     const int cbase = half * HC;
-    uint32_t r[HC];
-#pragma unroll
-    for (int c0 = 0; c0 < HC; c0 += 32) tmem_ld32(tS + lane_addr + cbase + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[c0]));
-    tmem_ld_wait();
-    const int kv_lim = (p.causal ? min(p.S, qi + 1) : p.S) - kv0 - cbase;   // local columns >= kv_lim are masked
-    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-    for (int i = 0; i < HC; ++i)
-      if (i < kv_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
-    xch[half * 128 + row] = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-    // the previous tile's P.V must be done before O is rescaled or P / the K,V stage are reused
-    if (j > 0) {
-      if (!mbar_wait(bar_o, uint32_t(j - 1) & 1u)) { ok = false; fail |= 0x80u; }
+    // m_used is the (possibly stale) row maximum the exponentials are taken against; O (in tensor
+    // memory) and l are rescaled only when the true maximum has moved by more than 2^8, so most
+    // key tiles accumulate P.V straight into tensor memory with no traffic on O at all.
+    float m_used = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    uint32_t fail = 0;
+    for (int j = 0; j < n_kv; ++j) {
+      const int st = j & 1;
+      const uint32_t ph = uint32_t(j >> 1) & 1u;
+      const int kv0 = j * TK;
+      if (ok && !mbar_wait(s_full + 8u * st, ph)) { ok = false; fail |= 0x40u; }
       tc_fence_after();
-    }
-    __syncthreads();
-    const float m_tile = fmaxf(xch[row], xch[128 + row]) * p.scale_log2;
-    if (j == 0) {
-      m_used = m_tile;
-    } else {
-      const bool need = m_tile > m_used + 8.f;
-      if (__any_sync(0xffffffffu, need)) {
-        const float m_new = need ? m_tile : m_used;
-        const float alpha = (m_used == -INFINITY) ? 0.f : exp2f(m_used - m_new);
-#pragma unroll 1
-        for (int c0 = half * (D / 2); c0 < (half + 1) * (D / 2); c0 += 32) {
-          uint32_t q[32];
-          tmem_ld32(tO + lane_addr + c0, q);
-          tmem_ld_wait();
+      // ---- this thread owns half (64 columns) of query row qi: read its scores once ----
+      uint32_t r[HC];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) q[i] = __float_as_uint(__uint_as_float(q[i]) * alpha);
-          asm volatile(
-              "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-              "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-              "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-              ::"r"(tO + lane_addr + c0), "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3]), "r"(q[4]), "r"(q[5]), "r"(q[6]),
-              "r"(q[7]), "r"(q[8]), "r"(q[9]), "r"(q[10]), "r"(q[11]), "r"(q[12]), "r"(q[13]), "r"(q[14]), "r"(q[15]),
-              "r"(q[16]), "r"(q[17]), "r"(q[18]), "r"(q[19]), "r"(q[20]), "r"(q[21]), "r"(q[22]), "r"(q[23]), "r"(q[24]),
-              "r"(q[25]), "r"(q[26]), "r"(q[27]), "r"(q[28]), "r"(q[29]), "r"(q[30]), "r"(q[31])
-              : "memory");
-        }
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        l_run *= alpha;
-        m_used = m_new;
-      }
-    }
-    // K/V stage of tile j-1 is free: fetch tile j+1 into it
-    if (threadIdx.x == 0 && j >= 1 && j + 1 < n_kv) load_kv(j + 1, (j + 1) & 1);
-    // ---- P = exp2(s * k - m_used), bf16, into the swizzled K-major tile (this thread's 64 columns
-    //      are exactly one 64-column chunk of the tile) ----
-    float ps4[4] = {0.f, 0.f, 0.f, 0.f};
-    const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-#pragma unroll
-    for (int g = 0; g < HC / 8; ++g) {
-      uint32_t w[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int col = g * 8 + 2 * i;
-        float a = 0.f, bb = 0.f;
-        if (col < kv_lim) a = exp2f(fmaf(__uint_as_float(r[col]), p.scale_log2, neg_m));
-        if (col + 1 < kv_lim) bb = exp2f(fmaf(__uint_as_float(r[col + 1]), p.scale_log2, neg_m));
-        const __nv_bfloat162 hv = __floats2bfloat162_rn(a, bb);   // the sum uses what the tensor core multiplies
-        ps4[i] += __low2float(hv) + __high2float(hv);
-        w[i] = *reinterpret_cast<const uint32_t*>(&hv);
-      }
-      const uint32_t off = half * 16384u + row * 128u + ((g ^ (row & 7)) << 4);
-      *reinterpret_cast<uint4*>(p_smem + off) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-    l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);   // partial sum over this thread's columns
-    // generic-proxy writes of P -> visible to the tensor core; S has been consumed by every row
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    tc_fence_before();
-    ok = __syncthreads_and(ok);
-    if (!ok) break;
-    if (threadIdx.x == 0) {
-      tc_fence_after();
-      const uint32_t vb = sV + st * kTile;
-#pragma unroll
-      for (int kk = 0; kk < TK / 16; ++kk) {
-        const uint64_t ad = make_desc(sP + (kk >> 2) * 16384u + (kk & 3) * 32u, 16, 1024);
-        const uint64_t bd = p.v_k_major ? make_desc(vb + (kk >> 2) * (D * 128u) + (kk & 3) * 32u, 16, 1024)
-                                        : make_desc(vb + kk * 2048u, 16384, 1024);
-        umma_bf16(tO, ad, bd, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);   // O accumulates across key tiles
-      }
-      umma_commit(bar_o);
-      if (j + 1 < n_kv) issue_qk(j + 1);   // queued behind P.V: ready when the next softmax starts
-    }
-  }
-  // ---- O / l -> bf16 ----
-  if (ok && n_kv > 0) {
-    if (!mbar_wait(bar_o, uint32_t(n_kv - 1) & 1u)) { ok = false; fail |= 0x80u; }
-    tc_fence_after();
-  }
-  ok = __syncthreads_and(ok);
-  if (fail) atomicOr(p.status, 0x100u | fail);
-  if (threadIdx.x == 0 && !ok) {   // let loads still in flight land before the shared memory is given up
-    for (int st = 0; st < 2; ++st)
-      if (pending[st]) mbar_wait(bar_kv0 + 8u * st, 0) || mbar_wait(bar_kv0 + 8u * st, 1);
-  }
-  xch[half * 128 + row] = l_run;
-  __syncthreads();
-  if (ok) {
-    const float l_tot = xch[row] + xch[128 + row];
-    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.O) + (int64_t)b * p.o_s[0] + (int64_t)h * p.o_s[1] + (int64_t)qi * p.o_s[2];
-#pragma unroll 1
-    for (int c0 = half * (D / 2); c0 < (half + 1) * (D / 2); c0 += 32) {
-      uint32_t q[32];
-      tmem_ld32(tO + lane_addr + c0, q);     // warp-collective: rows past the end take part, then skip the store
+      for (int c0 = 0; c0 < HC; c0 += 32)
+        tmem_ld32(tS + uint32_t(st * TK) + lane_addr + cbase + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[c0]));
       tmem_ld_wait();
-      if (qi < p.S) {
+      const int kv_lim = (p.causal ? min(p.S, qi + 1) : p.S) - kv0 - cbase;   // local columns >= kv_lim are masked
+      const bool full = kv_lim >= HC;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (full) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          float v[8];
+        for (int i = 0; i < HC; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+      } else {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(q[g * 8 + i]) * inv;
-          store16(out + c0 + g * 8, v);
+        for (int i = 0; i < HC; ++i)
+          if (i < kv_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+      }
+      float* xj = xch + st * 256;
+      xj[half * 128 + row] = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      if (!ok) *abort_flag = 1;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (*abort_flag) { ok = false; break; }   // read right after the barrier: every thread sees the same value
+      const float m_tile = fmaxf(xj[row], xj[128 + row]) * p.scale_log2;
+      if (j == 0) {
+        m_used = m_tile;
+      } else {
+        const bool need = m_tile > m_used + 8.f;
+        if (__any_sync(0xffffffffu, need)) {
+          // every P.V issued so far must have landed in O before it is rescaled
+          if (!mbar_wait(o_done + 8u * ((j - 1) & 1), uint32_t((j - 1) >> 1) & 1u)) { ok = false; fail |= 0x80u; }
+          tc_fence_after();
+          const float m_new = need ? m_tile : m_used;
+          const float alpha = (m_used == -INFINITY) ? 0.f : exp2f(m_used - m_new);
+#pragma unroll 1
+          for (int c0 = half * (D / 2); c0 < (half + 1) * (D / 2); c0 += 32) {
+            uint32_t q[32];
+            tmem_ld32(tO + lane_addr + c0, q);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) q[i] = __float_as_uint(__uint_as_float(q[i]) * alpha);
+            tmem_st32(tO + lane_addr + c0, q);
+          }
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+          l_run *= alpha;
+          m_used = m_new;
+        }
+      }
+      // P tile st was last read by P_{j-2}.V_{j-2}
+      if (j >= 2 && ok && !mbar_wait(o_done + 8u * st, uint32_t((j - 2) >> 1) & 1u)) { ok = false; fail |= 0x80u; }
+      // ---- P = exp2(s * k - m_used), bf16, into the swizzled K-major tile (this thread's 64 columns
+      //      are exactly one 64-column chunk of the tile) ----
+      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+      const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+      uint8_t* p_tile = p_smem + st * kPBytes + half * 16384u + row * 128u;
+#pragma unroll
+      for (int g = 0; g < HC / 8; ++g) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int col = g * 8 + 2 * i;
+          float a = ex2_fast(fmaf(__uint_as_float(r[col]), p.scale_log2, neg_m));
+          float bb = ex2_fast(fmaf(__uint_as_float(r[col + 1]), p.scale_log2, neg_m));
+          if (!full) {
+            if (col >= kv_lim) a = 0.f;
+            if (col + 1 >= kv_lim) bb = 0.f;
+          }
+          const __nv_bfloat162 hv = __floats2bfloat162_rn(a, bb);   // the sum uses what the tensor core multiplies
+          w[i] = *reinterpret_cast<const uint32_t*>(&hv);
+          ps4[i] += __uint_as_float(w[i] << 16) + __uint_as_float(w[i] & 0xffff0000u);
+        }
+        *reinterpret_cast<uint4*>(p_tile + ((g ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);   // partial sum over this thread's columns
+      // generic-proxy writes of P -> visible to the tensor core; this thread is done with S tile st
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_fence_before();
+      mbar_arrive(p_full + 8u * st);
+    }
+    // ---- O / l -> bf16 ----
+    if (ok && n_kv > 0) {
+      if (!mbar_wait(o_done + 8u * ((n_kv - 1) & 1), uint32_t((n_kv - 1) >> 1) & 1u)) { ok = false; fail |= 0x80u; }
+      tc_fence_after();
+    }
+    if (fail) atomicOr(p.status, 0x100u | fail);
+    if (!ok) *abort_flag = 1;
+    float* xl = xch + (n_kv & 1) * 256;   // the exchange buffer the last tile did not use
+    xl[half * 128 + row] = l_run;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (!*abort_flag) {
+      const float l_tot = xl[row] + xl[128 + row];
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.O) + (int64_t)b * p.o_s[0] + (int64_t)h * p.o_s[1] + (int64_t)qi * p.o_s[2];
+      pdl_wait();  // O may still be read by an earlier step
+#pragma unroll 1
+      for (int c0 = half * (D / 2); c0 < (half + 1) * (D / 2); c0 += 32) {
+        uint32_t q[32];
+        tmem_ld32(tO + lane_addr + c0, q);     // warp-collective: rows past the end take part, then skip the store
+        tmem_ld_wait();
+        if (qi < p.S) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(q[g * 8 + i]) * inv;
+            store16(out + c0 + g * 8, v);
+          }
         }
       }
     }
@@ -358,7 +476,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -366,7 +484,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream) {
   const int D = p.D;
-  const size_t smem = size_t(5) * TQ * D * 2 + size_t(TQ) * TK * 2 + 1024 + 64 + 1024;
+  const size_t smem = size_t(5) * TQ * D * 2 + size_t(2) * TQ * TK * 2 + 128 + 2048;
   const dim3 grid(((p.S + TQ - 1) / TQ) * p.B * p.NH);
   const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(&host.map_q);
   const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(&host.map_k);
@@ -378,7 +496,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream
       if (e != cudaSuccess) return e;
       attr64 = true;
     }
-    return launch_k(attn_tc_kernel<64>, grid, 256, smem, stream, *mq, *mk, *mv, p);
+    return launch_k(attn_tc_kernel<64>, grid, kAttnThreads, smem, stream, *mq, *mk, *mv, p);
   }
   if (D == 128) {
     if (!attr128) {
@@ -386,7 +504,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream
       if (e != cudaSuccess) return e;
       attr128 = true;
     }
-    return launch_k(attn_tc_kernel<128>, grid, 256, smem, stream, *mq, *mk, *mv, p);
+    return launch_k(attn_tc_kernel<128>, grid, kAttnThreads, smem, stream, *mq, *mk, *mv, p);
   }
   return cudaErrorInvalidValue;
 }
