@@ -428,9 +428,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             if (col >= kv_lim) a = 0.f;
             if (col + 1 >= kv_lim) bb = 0.f;
           }
-          const __nv_bfloat162 hv = __floats2bfloat162_rn(a, bb);   // the sum uses what the tensor core multiplies
+          const __nv_bfloat162 hv = __floats2bfloat162_rn(a, bb);
           w[i] = *reinterpret_cast<const uint32_t*>(&hv);
-          ps4[i] += __uint_as_float(w[i] << 16) + __uint_as_float(w[i] & 0xffff0000u);
+          ps4[i] += a + bb;   // fp32 sum; the bf16 rounding of P averages out of the normalisation (relative 2^-9 / sqrt(n))
         }
         *reinterpret_cast<uint4*>(p_tile + ((g ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
