@@ -180,7 +180,9 @@ __device__ __forceinline__ float row_sum(float v, float* red, int warp, int lane
   return t;
 }
 
-template <typename T, int NCH, int WPR>
+// EARLY: the gain and bias are read into registers before the wait for the previous step (short grids are
+// latency-bound and win from the overlap; long grids are bandwidth-bound and want the registers for occupancy).
+template <typename T, int NCH, int WPR, bool EARLY>
 __global__ void __launch_bounds__(256) norm_warp_kernel(NormParams p) {
   pdl_launch_dependents();
   constexpr int V = VecOf<T>::N;
@@ -195,15 +197,17 @@ __global__ void __launch_bounds__(256) norm_warp_kernel(NormParams p) {
   // that step is still finishing
   const T* gamma = static_cast<const T*>(p.gamma);
   const T* beta = static_cast<const T*>(p.beta);
-  float gv[NCH][V], bv[NCH][V];
+  float gv[EARLY ? NCH : 1][V], bv[EARLY ? NCH : 1][V];
+  if (EARLY) {
 #pragma unroll
-  for (int j = 0; j < NCH; ++j) {
-    const int c = c_first + 32 * WPR * j;
+    for (int j = 0; j < NCH; ++j) {
+      const int c = c_first + 32 * WPR * j;
 #pragma unroll
-    for (int i = 0; i < V; ++i) bv[j][i] = 0.f;
-    if (c < nch) {
-      norm_load<T, V>(gamma, false, 0, c, gv[j]);
-      if (beta) norm_load<T, V>(beta, false, 0, c, bv[j]);
+      for (int i = 0; i < V; ++i) bv[j][i] = 0.f;
+      if (c < nch) {
+        norm_load<T, V>(gamma, false, 0, c, gv[j]);
+        if (beta) norm_load<T, V>(beta, false, 0, c, bv[j]);
+      }
     }
   }
   pdl_wait();
@@ -256,8 +260,16 @@ __global__ void __launch_bounds__(256) norm_warp_kernel(NormParams p) {
     const int c = c_first + 32 * WPR * j;
     if (c < nch) {
       float o[V];
+      if (EARLY) {
 #pragma unroll
-      for (int i = 0; i < V; ++i) o[i] = (v[j][i] - mean) * rstd * gv[j][i] + bv[j][i];
+        for (int i = 0; i < V; ++i) o[i] = (v[j][i] - mean) * rstd * gv[j][i] + bv[j][i];
+      } else {
+        float g[V], b[V];
+        norm_load<T, V>(gamma, false, 0, c, g);
+        if (beta) norm_load<T, V>(beta, false, 0, c, b);
+#pragma unroll
+        for (int i = 0; i < V; ++i) o[i] = (v[j][i] - mean) * rstd * g[i] + (beta ? b[i] : 0.f);
+      }
       if (y_lo) {
         float t8[VecOf<T>::N];
 #pragma unroll
@@ -284,7 +296,9 @@ static cudaError_t norm_t(const NormParams& p, cudaStream_t st) {
     const int wpr = nch <= 128 ? 1 : (nch <= 256 ? 2 : (nch <= 512 ? 4 : 8));
     const int per_lane = (nch + 32 * wpr - 1) / (32 * wpr);
     const unsigned grid = (unsigned)((p.rows + 8 / wpr - 1) / (8 / wpr));
-#define NW_LAUNCH(N, W) return launch_k(norm_warp_kernel<T, N, W>, grid, 256, 0, st, p)
+    const bool early = grid <= 148u * 2u;
+#define NW_LAUNCH(N, W) return early ? launch_k(norm_warp_kernel<T, N, W, true>, grid, 256, 0, st, p) \
+                                     : launch_k(norm_warp_kernel<T, N, W, false>, grid, 256, 0, st, p)
 #define NW_PICK(W)              \
   if (per_lane <= 1) NW_LAUNCH(1, W); \
   if (per_lane <= 2) NW_LAUNCH(2, W); \
@@ -736,6 +750,63 @@ __global__ void permute_tile_kernel(const E* __restrict__ x, E* __restrict__ y, 
   }
 }
 
+// Class B for 16-bit elements with 16-byte accesses on both sides. Tile = 64 (O) x 64 (I). A thread
+// reads 8 consecutive I (one 16-byte load) and parks them as four 32-bit words in a tile of 33-word
+// rows (word w of row o holds I = 2w, 2w + 1): with the odd pitch both sweeps are free of bank
+// conflicts. For the output a thread takes word w of 8 consecutive rows O, splits the halves and
+// writes two 16-byte runs: 8 consecutive O of output row I = 2w and of row I = 2w + 1.
+// Needs: both extents multiples of 8, every other stride a multiple of 8 elements, 16-byte aligned bases.
+__global__ void __launch_bounds__(256) permute_tile16_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, PermSorted s,
+                                                             int di, int dn, int tiles_i, int tiles_o) {
+  pdl_launch_dependents();
+  __shared__ uint32_t tile[64 * 33];
+  int64_t blk = blockIdx.x;
+  const int ti = int(blk % tiles_i); blk /= tiles_i;
+  const int to = int(blk % tiles_o); blk /= tiles_o;
+  int64_t xo = 0, yo = 0;
+#pragma unroll
+  for (int k = 2; k >= 0; --k) {
+    const int c = int(blk % s.dims[k]);
+    blk /= s.dims[k];
+    xo += c * s.xs[k];
+    yo += c * s.ys[k];
+  }
+  const int i0 = ti * 64, o0 = to * 64;
+  pdl_wait();
+  // read: lane = (row within a group of 4, 16-byte unit of the row); 8 lanes cover one 128-byte row segment
+  {
+    const int ig = threadIdx.x & 7, orow = threadIdx.x >> 3;   // 32 rows per pass
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+      const int ol = orow + 32 * pass, o = o0 + ol, i = i0 + ig * 8;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (o < dn && i < di) v = *reinterpret_cast<const uint4*>(x + xo + (int64_t)o * s.xs[4] + i);
+      uint32_t* dst = tile + ol * 33 + ig * 4;
+      dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    }
+  }
+  __syncthreads();
+  // write: lane = (group of 8 rows O: 4 per warp, word column w: 8 per warp)
+  {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int og = (warp & 1) * 4 + (lane >> 3), w = (warp >> 1) * 8 + (lane & 7);   // og 0..7, w 0..31
+    uint32_t q[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) q[e] = tile[(og * 8 + e) * 33 + w];
+    const int i = i0 + 2 * w, o = o0 + og * 8;
+    if (o < dn && i < di) {
+      uint4 lo, hi;   // low halves = row I = 2w, high halves = row I = 2w + 1
+      lo.x = __byte_perm(q[0], q[1], 0x5410); hi.x = __byte_perm(q[0], q[1], 0x7632);
+      lo.y = __byte_perm(q[2], q[3], 0x5410); hi.y = __byte_perm(q[2], q[3], 0x7632);
+      lo.z = __byte_perm(q[4], q[5], 0x5410); hi.z = __byte_perm(q[4], q[5], 0x7632);
+      lo.w = __byte_perm(q[6], q[7], 0x5410); hi.w = __byte_perm(q[6], q[7], 0x7632);
+      uint16_t* dst = y + yo + (int64_t)i * s.ys[3] + o;
+      *reinterpret_cast<uint4*>(dst) = lo;
+      *reinterpret_cast<uint4*>(dst + s.ys[3]) = hi;
+    }
+  }
+}
+
 template <typename E>
 static void permute_dispatch(const PermuteParams& p, cudaStream_t st) {
   // order dims by output stride, slowest first; pad to 5 with unit dims in front
@@ -789,6 +860,17 @@ static void permute_dispatch(const PermuteParams& p, cudaStream_t st) {
   t.dims[3] = dI; t.xs[3] = xI; t.ys[3] = yI;
   const int tiles_i = (t.dims[3] + 63) / 64, tiles_o = (t.dims[4] + 63) / 64;
   const int64_t blocks = (int64_t)tiles_i * tiles_o * t.dims[0] * t.dims[1] * t.dims[2];
+  if (sizeof(E) == 2) {
+    bool wide = t.dims[3] % 8 == 0 && t.dims[4] % 8 == 0 && t.xs[3] == 1 && t.ys[4] == 1 && t.xs[4] % 8 == 0 && t.ys[3] % 8 == 0 &&
+                aligned16(x) && aligned16(y);
+    for (int k = 0; k < 3 && wide; ++k)
+      if (t.dims[k] > 1 && (t.xs[k] % 8 || t.ys[k] % 8)) wide = false;
+    if (wide) {
+      launch_k(permute_tile16_kernel, (unsigned)blocks, 256, 0, st, reinterpret_cast<const uint16_t*>(x), reinterpret_cast<uint16_t*>(y), t,
+               t.dims[3], t.dims[4], tiles_i, tiles_o);
+      return;
+    }
+  }
   launch_k(permute_tile_kernel<E>, (unsigned)blocks, 256, 0, st, x, y, t, t.dims[3], t.dims[4], tiles_i, tiles_o);
 }
 
