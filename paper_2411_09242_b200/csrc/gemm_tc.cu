@@ -684,12 +684,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // box was the slowest part of a short tile (about 600 cycles per k-step, 3000 per tile).
     const bool is_a = lane < 2;
     const int ch = is_a ? lane : lane - 2;
-    const int n_box = is_a ? (p.cfg.a_mn_major ? BM / 64 : 1) : (p.cfg.b_mn_major ? bn / 64 : 1);
+    // boxes per tile and rows per box: an MN-major operand comes in boxes of 64 rows, a K-major A in one box, a
+    // K-major B in boxes of b_box_rows rows (one, or two when the tensor map was cut for a CTA pair)
+    const int box_rows = (is_a ? p.cfg.a_mn_major : p.cfg.b_mn_major) ? 64 : (is_a ? BM : p.cfg.b_box_rows);
+    const int n_box = (is_a ? BM : bn) / box_rows;
     if (lane < 6 && ch < n_box) {
       int s = 0;
       uint32_t ph = 0;
       bool ok = true, in_flight = false;
-      const uint32_t box_off = (is_a ? 0u : kATileBytes) + uint32_t(ch) * 8192u;
+      const uint32_t box_off = (is_a ? 0u : kATileBytes) + uint32_t(ch) * uint32_t(box_rows) * 128u;
       const int x_r0 = is_a ? p.cfg.a_r0 : p.cfg.b_r0, x_b0 = is_a ? p.cfg.a_b0 : p.cfg.b_b0;
       const int x_k0 = is_a ? p.cfg.a_k0 : p.cfg.b_k0;
       int sel[5];
@@ -720,7 +723,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int c[5];
         {
           int r1, r0, b1, b0;
-          split2((is_a ? mt * BM : nt * bn) + ch * 64, x_r0, r1, r0);
+          split2((is_a ? mt * BM : nt * bn) + ch * box_rows, x_r0, r1, r0);
           split2(bz, x_b0, b1, b0);
           fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
         }
@@ -1053,9 +1056,12 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     // ---------------- TMA producer: one lane per 64-wide box, as in the persistent kernel ----------------
     const bool is_a = lane < 2;
     const int ch = is_a ? lane : lane - 2;
-    const int n_box = is_a ? (p.cfg.a_mn_major ? BM / 64 : 1) : (p.cfg.b_mn_major ? bn / 64 : 1);
+    // boxes per tile and rows per box: an MN-major operand comes in boxes of 64 rows, a K-major A in one box, a
+    // K-major B in boxes of b_box_rows rows (one, or two when the tensor map was cut for a CTA pair)
+    const int box_rows = (is_a ? p.cfg.a_mn_major : p.cfg.b_mn_major) ? 64 : (is_a ? BM : p.cfg.b_box_rows);
+    const int n_box = (is_a ? BM : bn) / box_rows;
     if (lane < 6 && ch < n_box) {
-      const uint32_t box_off = (is_a ? 0u : kATileBytes) + uint32_t(ch) * 8192u;
+      const uint32_t box_off = (is_a ? 0u : kATileBytes) + uint32_t(ch) * uint32_t(box_rows) * 128u;
       const int x_r0 = is_a ? p.cfg.a_r0 : p.cfg.b_r0, x_b0 = is_a ? p.cfg.a_b0 : p.cfg.b_b0;
       const int x_k0 = is_a ? p.cfg.a_k0 : p.cfg.b_k0;
       int sel[5];
@@ -1070,7 +1076,7 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       int c[5];
       {
         int r1, r0, b1, b0;
-        split2((is_a ? mt * BM : nt * bn) + ch * 64, x_r0, r1, r0);
+        split2((is_a ? mt * BM : nt * bn) + ch * box_rows, x_r0, r1, r0);
         split2(bz, x_b0, b1, b0);
         fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
       }

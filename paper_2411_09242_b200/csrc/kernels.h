@@ -57,6 +57,8 @@ struct GemmTcCfg {
   int a_sel[5], b_sel[5];
   int a_k0, a_r0, a_b0, b_k0, b_r0, b_b0;
   int a_rank, b_rank;
+  int b_box_rows;       // rows of one TMA box of a K-major B tile (bn, or 128 when a CTA pair shares a 256-wide tile)
+  int pair;             // 1: the step qualifies for the CTA-pair kernel (two CTAs, one 256 x 256 tile, tcgen05 cta_group::2)
 };
 
 struct alignas(64) TensorMapStorage {

@@ -238,11 +238,17 @@ bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc) {
   const int64_t b_rs[2] = {g.b_s[4], g.b_s[5]}, b_ks[2] = {g.b_s[2], g.b_s[3]}, b_bs[2] = {g.b_s[0], g.b_s[1]};
   if (!build_tma_operand(g.M, g.M0, a_rs, g.K, g.K0, a_ks, g.batch, g.B0, a_bs, 128, &h.a)) return false;
   // an unmerged n level narrower than the tile would be straddled: shrink the tile first
+  // A 256-wide tile over an even number of 128-row tiles can be shared by a pair of CTAs (each loads half
+  // of the B tile: its TMA box is then 128 rows, which the single-CTA kernel fetches as two boxes).
+  int b_box = bn;
   while (true) {
-    if (build_tma_operand(g.N, g.N0, b_rs, g.K, g.K0, b_ks, g.batch, g.B0, b_bs, bn, &h.b)) break;
+    b_box = (bn == 256 && g.causal == CAUSAL_NONE && g.M % 256 == 0) ? 128 : bn;
+    if (build_tma_operand(g.N, g.N0, b_rs, g.K, g.K0, b_ks, g.batch, g.B0, b_bs, b_box, &h.b)) break;
     if (bn == 64) return false;
     bn /= 2;
   }
+  h.cfg.b_box_rows = b_box;
+  h.cfg.pair = (bn == 256 && b_box == 128) ? 1 : 0;
   // output / residual vector accesses assume 8-element alignment of every outer stride when the
   // n index is contiguous; otherwise the epilogue falls back to scalar stores (always legal)
   h.cfg.bn = bn;
