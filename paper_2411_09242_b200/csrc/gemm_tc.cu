@@ -1253,6 +1253,245 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   }
 }
 
+// ---- CTA pair: two CTAs, one 256 x 256 output tile (tcgen05 cta_group::2) -------------------------------
+// The single-CTA kernel pulls 48 KB from L2 per k-step of a 128 x 256 tile; with all SMs doing so the L2
+// cannot keep the tensor cores fed. Here the two CTAs of a cluster share a 256 x 256 tile: each loads its
+// own 128 rows of A and its own 128 columns of B (32 KB per k-step, six stages), and CTA 0 issues one
+// 256 x 256 x 16 MMA that reads both CTAs' shared memory and writes rows 0-127 of the accumulator into its
+// own tensor memory and rows 128-255 into its peer's. Barrier traffic across the pair:
+//   full[s]    lives in CTA 0; the TMA loads of both CTAs complete on it (cta_group::2 loads)
+//   empty[s]   in both CTAs; CTA 0's commit after a stage's MMAs arrives on both
+//   tfull[a]   in both CTAs; CTA 0's commit after a tile's last MMA arrives on both
+//   tempty[a]  lives in CTA 0; the epilogue warps of both CTAs arrive on it
+// Every thread of both CTAs passes the cluster barriers at the start (barriers initialised) and at the end
+// (tensor memory may be released) on every path; all mbarrier waits are bounded.
+__device__ __forceinline__ void tma_load_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int c0, int c1, int c2,
+                                              int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void umma_pair_bf16_lohi(uint32_t tmem_c, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                    uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n .reg .b64 da, db;\n mov.b64 da, {%1, %2};\n mov.b64 db, {%3, %4};\n setp.ne.b32 p, %6, 0;\n"
+      " tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n}"
+      ::"r"(tmem_c), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives (once the MMAs issued so far have completed) on the barrier at this shared-memory offset in both CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
+                    const __grid_constant__ TcParams p) {
+  constexpr int PN = 256;                          // tile width of the pair (columns of the accumulator)
+  constexpr uint32_t kBHalfBytes = 128 * BK * 2;   // this CTA's 128 columns of the B tile
+  constexpr uint32_t stage_bytes = kATileBytes + kBHalfBytes;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const int stages = p.cfg.stages;
+  const uint32_t bars = base + uint32_t(stages) * stage_bytes;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (stages + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * stages + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * stages + 2 + a); };
+  const uint32_t tmem_slot = bars + 8u * (2 * stages + 4);
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
+  volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
+  const uint32_t stage_base = (tmem_slot + 16u + 15u) & ~15u;   // 8 warps x 4 KB epilogue staging tiles
+
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();            // 0: issues the MMAs; 1: its peer
+  const int n_pairs = int(gridDim.x) >> 1, pair_id = int(blockIdx.x) >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * kEpiWarps); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+  }
+  if (warp == 1) {   // the same warp of both CTAs: the allocation is made in both tensor memories at once
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();     // both CTAs' barriers are initialised before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  if (warp == 0) {
+    // ---------------- TMA producer: one lane per box of this CTA's A rows / B columns ----------------
+    const bool is_a = lane < 2;
+    const int ch = is_a ? lane : lane - 2;
+    const int box_rows = (is_a ? p.cfg.a_mn_major : p.cfg.b_mn_major) ? 64 : 128;
+    const int n_box = 128 / box_rows;
+    if (lane < 6 && ch < n_box) {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      const uint32_t box_off = (is_a ? 0u : kATileBytes) + uint32_t(ch) * uint32_t(box_rows) * 128u;
+      const int x_r0 = is_a ? p.cfg.a_r0 : p.cfg.b_r0, x_b0 = is_a ? p.cfg.a_b0 : p.cfg.b_b0;
+      const int x_k0 = is_a ? p.cfg.a_k0 : p.cfg.b_k0;
+      int sel[5];
+#pragma unroll
+      for (int d = 0; d < 5; ++d) sel[d] = is_a ? p.cfg.a_sel[d] : p.cfg.b_sel[d];
+      int kd0 = 0, kd1 = -1;
+#pragma unroll
+      for (int d = 0; d < 5; ++d) {
+        if (sel[d] == 0) kd0 = d;
+        if (sel[d] == 1) kd1 = d;
+      }
+      const bool k_simple = kd1 < 0 && kd0 < 3;
+      const int i0 = kd0 == 0 ? BK : 0, i1 = kd0 == 1 ? BK : 0, i2 = kd0 == 2 ? BK : 0;
+      uint32_t dst = base + box_off, eb = empty_bar(0);
+      uint32_t fb = map_to_rank(full_bar(0), 0u);       // the full barriers of CTA 0 collect both CTAs' bytes
+      const uint32_t fb0 = fb;
+      const bool b_free = p.g.b_const && (p.n_group < 2 || p.gx[0].b_const) && (p.n_group < 3 || p.gx[1].b_const);
+      if (is_a || !b_free) pdl_wait();   // weights do not wait for the previous step
+      for (int item = pair_id; ok && item < p.num_tiles; item += n_pairs) {
+        int grp, bz, pm, nt;
+        decode_tile(p, item, grp, bz, pm, nt);        // p.tiles_m counts pairs of row tiles here
+        const int mt = 2 * pm + int(rank);
+        const int ksteps = k_steps_of(p, mt);
+        int c[5];
+        {
+          int r1, r0, b1, b0;
+          split2((is_a ? mt * BM : nt * PN + int(rank) * 128) + ch * box_rows, x_r0, r1, r0);
+          split2(bz, x_b0, b1, b0);
+          fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
+        }
+        const CUtensorMap* map = is_a ? &map_a : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2));
+        int k0 = 0, k1 = 0;
+        for (int ks = 0; ks < ksteps; ++ks) {
+          if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
+          if (lane == 0 && rank == 0) mbar_expect_tx(full_bar(s), 2u * stage_bytes);
+          if (k_simple) {
+            tma_load_pair(dst, map, fb, c[0], c[1], c[2], c[3], c[4]);
+            c[0] += i0; c[1] += i1; c[2] += i2;
+          } else {
+            int q[5];
+#pragma unroll
+            for (int d = 0; d < 5; ++d) q[d] = c[d] + (d == kd0 ? k0 : 0) + (d == kd1 ? k1 : 0);
+            tma_load_pair(dst, map, fb, q[0], q[1], q[2], q[3], q[4]);
+            k0 += BK; if (k0 >= x_k0) { k0 = 0; ++k1; }
+          }
+          dst += stage_bytes; fb += 8u; eb += 8u;
+          if (++s == stages) { s = 0; ph ^= 1u; dst = base + box_off; fb = fb0; eb = empty_bar(0); }
+        }
+      }
+      if (!ok) {
+        if (!*abort_flag) atomicOr(p.status, 0x1u);
+        *abort_flag = 1;
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (CTA 0 only) ----------------
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(p.cfg.a_mn_major) << 15) |
+                             (uint32_t(p.cfg.b_mn_major) << 16) | (uint32_t(PN >> 3) << 17) | (uint32_t(256 >> 4) << 24);
+      const uint32_t a_step = p.cfg.a_mn_major ? 128u : 2u, b_step = p.cfg.b_mn_major ? 128u : 2u;
+      const uint64_t ad_first = make_desc(base, p.cfg.a_mn_major), bd_first = make_desc(base + kATileBytes, p.cfg.b_mn_major);
+      const uint32_t a_hi = uint32_t(ad_first >> 32), b_hi = uint32_t(bd_first >> 32);
+      const uint32_t a_lo0 = uint32_t(ad_first), b_lo0 = uint32_t(bd_first), stage16 = stage_bytes >> 4;
+      uint32_t a_lo = a_lo0, b_lo = b_lo0, fb = full_bar(0), eb = empty_bar(0);
+      int s = 0, acc = 0;
+      uint32_t ph = 0, acc_ph = 0;
+      bool ok = true;
+      for (int item = pair_id; ok && item < p.num_tiles; item += n_pairs) {
+        int grp, bz, pm, nt;
+        decode_tile(p, item, grp, bz, pm, nt);
+        const int ksteps = k_steps_of(p, 2 * pm);
+        if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_c = tmem_base + uint32_t(acc * PN);
+        uint32_t accum = 0u;
+        for (int ks = 0; ks < ksteps; ++ks) {
+          if (!mbar_wait(fb, ph)) { ok = false; break; }
+          tc_fence_after();
+          umma_pair_bf16_lohi(tmem_c, a_lo, a_hi, b_lo, b_hi, idesc, accum);
+          umma_pair_bf16_lohi(tmem_c, a_lo + a_step, a_hi, b_lo + b_step, b_hi, idesc, 1u);
+          umma_pair_bf16_lohi(tmem_c, a_lo + 2u * a_step, a_hi, b_lo + 2u * b_step, b_hi, idesc, 1u);
+          umma_pair_bf16_lohi(tmem_c, a_lo + 3u * a_step, a_hi, b_lo + 3u * b_step, b_hi, idesc, 1u);
+          umma_commit_pair(eb);  // the stage is free in both CTAs once these MMAs have read it
+          accum = 1u;
+          a_lo += stage16; b_lo += stage16; fb += 8u; eb += 8u;
+          if (++s == stages) { s = 0; ph ^= 1u; a_lo = a_lo0; b_lo = b_lo0; fb = full_bar(0); eb = empty_bar(0); }
+        }
+        if (ok) umma_commit_pair(tfull_bar(acc));  // accumulator complete, in both CTAs
+        if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+      }
+      if (!ok) {
+        if (!*abort_flag) atomicOr(p.status, 0x2u);
+        *abort_flag = 1;
+      }
+    }
+  } else {
+    // ---------------- epilogue (warps 2..9): this CTA's 128 rows of the tile ----------------
+    const int lane_base = (warp & 3) * 32;
+    const int half = (warp - 2) >> 2;
+    float* stage = reinterpret_cast<float*>(smem_raw + (stage_base - raw)) + (warp - 2) * 1024;
+    const int col_begin = half * (PN / 2), col_end = col_begin + PN / 2;
+    int acc = 0;
+    uint32_t acc_ph = 0;
+    bool ok = true;
+    pdl_wait();  // before any global read (bias, residual) or write (C)
+    for (int item = pair_id; ok && item < p.num_tiles; item += n_pairs) {
+      int grp, bz, pm, nt;
+      decode_tile(p, item, grp, bz, pm, nt);
+      const int mt = 2 * pm + int(rank);
+      const GemmParams& g = grp == 0 ? p.g : p.gx[grp - 1];
+      const int n_tile0 = nt * PN;
+      int64_t cbs[8], rbs[8];
+      uint32_t ok_mask = 0;
+      const int64_t cbz = split_off(bz, g.B0, g.c_s[0], g.c_s[1]);
+      const int64_t rbz = g.has_res ? split_off(bz, g.B0, g.r_s[0], g.r_s[1]) : 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int mi = mt * BM + lane_base + (lane >> 3) + 4 * i;
+        const bool live = mi < g.M;
+        ok_mask |= live ? (1u << i) : 0u;
+        cbs[i] = cbz + (live ? split_off(mi, g.M0, g.c_s[2], g.c_s[3]) : 0);
+        rbs[i] = g.has_res ? rbz + (live ? split_off(mi, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
+      }
+      if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * PN);
+      epilogue_tile_c<EPI>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0u));   // CTA 0 counts both CTAs' epilogue warps
+      if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+    }
+    if (!ok && lane == 0) {
+      if (!*abort_flag) atomicOr(p.status, 0x4u);
+      *abort_flag = 1;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();     // neither CTA releases tensor memory or leaves while its peer may still use it
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -1302,6 +1541,16 @@ int encode_tensor_map(TensorMapStorage* out, const void* base, const TmaOperand&
                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? 0 : -2;
+}
+
+// FLUID_PAIR=0 in the environment keeps every step on the single-CTA kernel.
+static bool pair_enabled() {
+  static int on = -1;
+  if (on < 0) {
+    const char* e = std::getenv("FLUID_PAIR");
+    on = (e && e[0] == '0') ? 0 : 1;
+  }
+  return on == 1;
 }
 
 static bool vec_epilogue_ok(const GemmParams* gs, int n_group, bool check_pointers) {
@@ -1453,6 +1702,52 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
       default: break;
     }
 #undef FLUID_TC_CLUSTER
+  }
+  // ---- many 256-wide tiles over an even number of row tiles: pairs of CTAs share 256 x 256 tiles ----
+  if (tc.cfg.pair && pair_enabled() && vec && epi != EPI_ANY && split_k <= 1 && g.causal == CAUSAL_NONE && (p.tiles_m & 1) == 0 &&
+      p.num_tiles > 0) {
+    TcParams q = p;
+    q.tiles_m = p.tiles_m / 2;                       // pairs of row tiles
+    q.tiles_per_batch = q.tiles_m * p.tiles_n;
+    q.tiles_per_group = q.tiles_per_batch * g.batch;
+    q.num_tiles = q.tiles_per_group * n_group;
+    q.cfg.stages = 6;
+    q.split_k = 1;
+    const size_t psmem = size_t(q.cfg.stages) * (kATileBytes + size_t(128) * BK * 2) + 1024 + 8 * (2 * q.cfg.stages + 4) + 16 + 16 +
+                         size_t(kEpiWarps) * 4096;
+    const int n_pairs = std::min(q.num_tiles, sm_count() / 2);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(2 * n_pairs));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = psmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
+    static bool pattr_set[7] = {false, false, false, false, false, false, false};
+#define FLUID_TC_PAIR(E)                                                                                             \
+  case E: {                                                                                                          \
+    if (!pattr_set[E]) {                                                                                             \
+      cudaError_t e = cudaFuncSetAttribute(gemm_tc_pair_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); \
+      if (e != cudaSuccess) return e;                                                                                \
+      pattr_set[E] = true;                                                                                           \
+    }                                                                                                                \
+    return cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel<E>, *ma, *mb, *mb1, *mb2, q);                                \
+  }
+    switch (epi) {
+      FLUID_TC_PAIR(EPI_PLAIN)
+      FLUID_TC_PAIR(EPI_PLAIN_WIDE)
+      FLUID_TC_PAIR(EPI_RES)
+      FLUID_TC_PAIR(EPI_RES_WIDE)
+      FLUID_TC_PAIR(EPI_GELU_ERF)
+      FLUID_TC_PAIR(EPI_GELU_TANH)
+      default: break;
+    }
+#undef FLUID_TC_PAIR
   }
   const int grid = std::min(p.num_tiles, sm_count());
   if (grid <= 0) return cudaSuccess;
