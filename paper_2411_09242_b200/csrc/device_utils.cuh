@@ -107,18 +107,24 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 __device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
-// GELU (erf form) with erf from Abramowitz & Stegun 7.1.26 (|error| < 1.5e-7 before fp32 rounding):
-// far below bf16 resolution and about a third of the instructions of erff().
+// GELU (erf form) on the fused-multiply-add pipe only: erf(z) = z * P(z^2) with a 9-term least-squares fit on
+// |z| <= 2.9 (|error| < 1.3e-5; beyond, z is clamped and erf stays within 3e-5 of +-1), so the absolute error of
+// the result is below 2.2e-5 for |x| <= 4.1 and below 1.7e-5 |x| after that: far under bf16 resolution of the
+// outputs it is used for. No reciprocal and no exponential: a GEMM epilogue that applies this to every element
+// of a 128 x 256 tile would otherwise spend 4000 cycles in the special-function unit alone.
 __device__ __forceinline__ float gelu_erf_fast(float x) {
-  const float z = fabsf(x) * 0.70710678118654752f;
-  const float t = __frcp_rn(fmaf(0.3275911f, z, 1.f));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  const float e = poly * t * __expf(-z * z);  // 1 - erf(z)
+  const float z = fminf(fmaxf(x * 0.70710678118654752f, -2.9f), 2.9f);
+  const float u = z * z;
+  float q = fmaf(4.85526996385488e-08f, u, -2.210898173871101e-06f);
+  q = fmaf(q, u, 4.476702451938763e-05f);
+  q = fmaf(q, u, -0.0005382060771808028f);
+  q = fmaf(q, u, 0.004347700159996748f);
+  q = fmaf(q, u, -0.02536272630095482f);
+  q = fmaf(q, u, 0.11139318346977234f);
+  q = fmaf(q, u, -0.375481516122818f);
+  q = fmaf(q, u, 1.128293514251709f);
   const float half_x = 0.5f * x;
-  return x >= 0.f ? fmaf(-half_x, e, x) : half_x * e;
+  return fmaf(half_x, q * z, half_x);
 }
 __device__ __forceinline__ float gelu_tanh(float x) {
   const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);

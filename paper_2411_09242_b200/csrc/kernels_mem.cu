@@ -567,7 +567,14 @@ __global__ void __launch_bounds__(256) rope_vec_kernel(RopeParams p, int64_t tot
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const float inv_freq = exp2f(-2.f * (c * 8 + j) / D * lb);
-      sincosf(s * inv_freq, &sn[j], &cs[j]);
+      // two-step reduction of the angle to [-pi, pi] (exact product k * 2pi_hi in the fused multiply-add), then the
+      // hardware sine / cosine, whose absolute error there is about 2^-21
+      const float ang = s * inv_freq;
+      const float k = rintf(ang * 0.15915494309189535f);
+      float r = fmaf(-k, 6.2831854820251465f, ang);
+      r = fmaf(-k, -1.7484555e-7f, r);
+      sn[j] = __sinf(r);
+      cs[j] = __cosf(r);
     }
     const int h_end = min(p.dims[2], (hg + 1) * ROPE_HG);
     for (int h = hg * ROPE_HG; h < h_end; ++h) {
@@ -715,6 +722,37 @@ __global__ void permute_rows_kernel(const E* __restrict__ x, E* __restrict__ y, 
   }
 }
 
+// The same for a dense output of fewer than 2^31 units (the usual case): the output offset of unit i is i
+// itself, the input offset comes from 32-bit divisions, and a thread moves four units that are a quarter
+// of the tensor apart (four loads in flight before the first store).
+template <typename E>
+__global__ void __launch_bounds__(256) permute_rows32_kernel(const E* __restrict__ x, E* __restrict__ y, PermSorted s, uint32_t total) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const uint32_t quarter = (total + 3u) / 4u;
+  const uint32_t d4 = uint32_t(s.dims[4]), d3 = uint32_t(s.dims[3]), d2 = uint32_t(s.dims[2]), d1 = uint32_t(s.dims[1]);
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < quarter; i += gridDim.x * blockDim.x) {
+    E v[4];
+    uint32_t idx[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      idx[u] = i + uint32_t(u) * quarter;
+      if (idx[u] < total) {
+        uint32_t rem = idx[u];
+        const uint32_t c4 = rem % d4; rem /= d4;
+        const uint32_t c3 = rem % d3; rem /= d3;
+        const uint32_t c2 = rem % d2; rem /= d2;
+        const uint32_t c1 = rem % d1; rem /= d1;
+        const int64_t xo = (int64_t)c4 * s.xs[4] + (int64_t)c3 * s.xs[3] + (int64_t)c2 * s.xs[2] + (int64_t)c1 * s.xs[1] + (int64_t)rem * s.xs[0];
+        v[u] = x[xo];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (idx[u] < total) y[idx[u]] = v[u];
+  }
+}
+
 // Class B: the contiguous dim changes -> shared-memory tile transpose. Tile = 64 (x-fast dim I)
 // by 64 (y-fast dim O); the odd row pitch keeps both sweeps free of bank conflicts.
 template <typename E>
@@ -836,6 +874,15 @@ static void permute_dispatch(const PermuteParams& p, cudaStream_t st) {
       w.dims[4] /= W;
       for (int k = 0; k < 4; ++k) { w.xs[k] /= W; w.ys[k] /= W; }
       const int64_t tw = total / W;
+      // dense output in sorted-stride order: unit i of y is at offset i
+      bool dense = w.ys[4] == 1 && tw < (int64_t(1) << 31);
+      for (int k = 3; k >= 0 && dense; --k) dense = w.ys[k] == w.ys[k + 1] * w.dims[k + 1];
+      if (dense) {
+        const unsigned grid32 = (unsigned)std::min<int64_t>((tw / 4 + 255) / 256, 148 * 16);
+        launch_k(permute_rows32_kernel<uint4>, std::max(1u, grid32), 256, 0, st, reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(y),
+                 w, (uint32_t)tw);
+        return;
+      }
       const unsigned grid = (unsigned)std::min<int64_t>((tw + 255) / 256, 148 * 16);
       launch_k(permute_rows_kernel<uint4>, grid, 256, 0, st, reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(y), w, tw);
     } else {
