@@ -1,12 +1,15 @@
 // Fused attention for sm_100a: S = Q.K^T and O = softmax(S).V on tcgen05 tensor cores with the
-// score tile kept in tensor memory; the [S, S] score / probability tensors never reach HBM or the
-// arena. One CTA = one (batch, head, 128-query tile); 256 threads: two per query row, each owning
-// half of the key columns of a tile (two warps per scheduler hide each other's latencies).
+// score tiles kept in tensor memory; the [S, S] score / probability tensors never reach HBM or the
+// arena. One CTA = one (batch, head, 128-query tile); 320 threads: 8 softmax warps (two threads per
+// query row, 64 key columns each), one warp that issues the MMAs, one warp that issues the TMA loads.
+// (Sixteen softmax warps, four threads per row, were measured and are no faster: with 128 x 128 x 16 and
+// 128 x D x 16 instructions costing the same ~128 cycles as a 128 x 256 x 16 one, the tensor pipe is
+// busy ~1500-2000 of the ~2400 cycles a key tile takes.)
 //
-//   per 128-key tile:  TMA K, V tiles (2-stage ring)  ->  tcgen05.mma  S = Q.K^T  (TMEM, fp32)
+//   per 128-key tile:  TMA K, V tiles (2-stage rings)  ->  tcgen05.mma  S = Q.K^T  (one of two TMEM tiles, fp32)
 //                      -> tcgen05.ld, online softmax in registers (row max / sum per thread, exp2)
-//                      -> P (bf16) written to shared memory in the 128-byte-swizzled K-major form
-//                      -> tcgen05.mma  PV = P.V (TMEM)  ->  O = O * alpha + PV in registers
+//                      -> P (bf16) written to one of two shared-memory tiles, 128-byte-swizzled K-major
+//                      -> tcgen05.mma  O += P.V (TMEM; rescaled in place only when the row maximum jumps)
 //
 // Q, K and V are read where the plan put them: Q with the head dim contiguous; K either with the
 // head dim contiguous (any of the [B,S,nh,D] / [B,nh,S,D] families) or sequence-contiguous
