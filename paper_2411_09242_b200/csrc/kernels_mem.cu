@@ -183,7 +183,7 @@ __device__ __forceinline__ float row_sum(float v, float* red, int warp, int lane
 // EARLY: the gain and bias are read into registers before the wait for the previous step (short grids are
 // latency-bound and win from the overlap; long grids are bandwidth-bound and want the registers for occupancy).
 template <typename T, int NCH, int WPR, bool EARLY>
-__global__ void __launch_bounds__(256) norm_warp_kernel(NormParams p) {
+__global__ void __launch_bounds__(256, (!EARLY && NCH <= 3) ? 5 : 1) norm_warp_kernel(NormParams p) {
   pdl_launch_dependents();
   constexpr int V = VecOf<T>::N;
   __shared__ float red[8];
@@ -753,6 +753,52 @@ __global__ void __launch_bounds__(256) permute_rows32_kernel(const E* __restrict
   }
 }
 
+// Class A where rows are short (<= 512 bytes) and the dim that follows them differs between input and output,
+// e.g. [B,S,nh,D] -> [B,nh,S,D]: moving one row at a time touches DRAM in isolated 128-256-byte pieces on
+// one side. Here a CTA moves a TP x TQ block of rows (16 x 8, or 8 x 8 for 512-byte rows) through shared memory: it reads TQ runs of TP rows that
+// are contiguous in the input and writes TP runs of TQ rows that are contiguous in the output (2-4 KB each).
+// Units are 16 bytes; U units per row; slot 3 of the sorted dims is the output-next dim Q, slot pk the
+// input-next dim P; the other two dims are spread over the grid.
+template <int U>
+__global__ void __launch_bounds__(256) permute_rows_tile_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, PermSorted s, int pk,
+                                                                int tiles_p, int tiles_q) {
+  constexpr int TP = U == 32 ? 8 : 16, TQ = 8, N = TP * TQ * U, PER = N / 256;   // at most 32 KB of shared memory
+  __shared__ uint4 tile[N];
+  pdl_launch_dependents();
+  int64_t blk = blockIdx.x;
+  const int tq = int(blk % tiles_q); blk /= tiles_q;
+  const int tp = int(blk % tiles_p); blk /= tiles_p;
+  int64_t xo = 0, yo = 0;
+#pragma unroll
+  for (int k = 2; k >= 0; --k) {
+    if (k == pk) continue;
+    const int c = int(blk % s.dims[k]);
+    blk /= s.dims[k];
+    xo += c * s.xs[k];
+    yo += c * s.ys[k];
+  }
+  const int p0 = tp * TP, q0 = tq * TQ, dp = s.dims[pk], dq = s.dims[3];
+  const int64_t xp = s.xs[pk], xq = s.xs[3], yp = s.ys[pk], yq = s.ys[3];
+  pdl_wait();
+  uint4 v[PER];
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {       // input order: u fastest, then p, then q
+    const int e = threadIdx.x + 256 * j;
+    const int u = e % U, pp = (e / U) % TP, qq = e / (U * TP);
+    v[j] = make_uint4(0u, 0u, 0u, 0u);
+    if (p0 + pp < dp && q0 + qq < dq) v[j] = x[xo + (p0 + pp) * xp + (q0 + qq) * xq + u];
+  }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) tile[threadIdx.x + 256 * j] = v[j];   // [q][p][u]
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {       // output order: u fastest, then q, then p
+    const int e = threadIdx.x + 256 * j;
+    const int u = e % U, qq = (e / U) % TQ, pp = e / (U * TQ);
+    if (p0 + pp < dp && q0 + qq < dq) y[yo + (p0 + pp) * yp + (q0 + qq) * yq + u] = tile[(qq * TP + pp) * U + u];
+  }
+}
+
 // Class B: the contiguous dim changes -> shared-memory tile transpose. Tile = 64 (x-fast dim I)
 // by 64 (y-fast dim O); the odd row pitch keeps both sweeps free of bank conflicts.
 template <typename E>
@@ -876,7 +922,29 @@ static void permute_dispatch(const PermuteParams& p, cudaStream_t st) {
       const int64_t tw = total / W;
       // dense output in sorted-stride order: unit i of y is at offset i
       bool dense = w.ys[4] == 1 && tw < (int64_t(1) << 31);
-      for (int k = 3; k >= 0 && dense; --k) dense = w.ys[k] == w.ys[k + 1] * w.dims[k + 1];
+      for (int k = 3; k >= 0 && dense; --k)
+        if (w.dims[k] > 1) dense = w.ys[k] == w.ys[k + 1] * w.dims[k + 1];   // (unit dims pad the front)
+      // short rows whose next dim differs between input and output: block-of-rows kernel
+      if (dense && (w.dims[4] == 8 || w.dims[4] == 16 || w.dims[4] == 32) && w.dims[3] > 1 && w.xs[3] != w.dims[4]) {
+        int pk = -1;
+        for (int k = 0; k < 3; ++k)
+          if (w.dims[k] > 1 && w.xs[k] == w.dims[4]) pk = k;
+        if (pk >= 0) {
+          const int tp_rows = w.dims[4] == 32 ? 8 : 16;
+          const int tiles_p = (w.dims[pk] + tp_rows - 1) / tp_rows, tiles_q = (w.dims[3] + 7) / 8;
+          int64_t blocks = (int64_t)tiles_p * tiles_q;
+          for (int k = 0; k < 3; ++k)
+            if (k != pk) blocks *= w.dims[k];
+          if (blocks < (int64_t(1) << 31)) {
+            const uint4* xv = reinterpret_cast<const uint4*>(x);
+            uint4* yv = reinterpret_cast<uint4*>(y);
+            if (w.dims[4] == 8) launch_k(permute_rows_tile_kernel<8>, (unsigned)blocks, 256, 0, st, xv, yv, w, pk, tiles_p, tiles_q);
+            else if (w.dims[4] == 16) launch_k(permute_rows_tile_kernel<16>, (unsigned)blocks, 256, 0, st, xv, yv, w, pk, tiles_p, tiles_q);
+            else launch_k(permute_rows_tile_kernel<32>, (unsigned)blocks, 256, 0, st, xv, yv, w, pk, tiles_p, tiles_q);
+            return;
+          }
+        }
+      }
       if (dense) {
         const unsigned grid32 = (unsigned)std::min<int64_t>((tw / 4 + 255) / 256, 148 * 16);
         launch_k(permute_rows32_kernel<uint4>, std::max(1u, grid32), 256, 0, st, reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(y),
