@@ -140,7 +140,8 @@ typedef struct fluid_step_info {
   int32_t kernel;        /* fluid_kernel_id */
   int32_t variant;       /* kernel-specific (GEMM: bit0 A MN-major, bit1 B MN-major, bits 8-19 tile N,
                             bits 20-23 grouped siblings, bits 24-27 split-K factor, bit 28: the split
-                            runs as one thread-block cluster per output tile) */
+                            runs as one thread-block cluster per output tile, bit 29: pairs of CTAs share
+                            256 x 256 tiles) */
   int32_t n_ops;         /* graph ops folded into this step */
   int32_t ops[8];
   int32_t n_in, n_out;   /* tensors read / written (graph tensor ids) */

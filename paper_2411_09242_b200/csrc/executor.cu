@@ -85,6 +85,7 @@ int finalize_steps(fluid_plan_s* p) {
           GemmParams gs[3] = {s.gemm, s.nodes.size() > 1 ? s.gemm_x[0] : s.gemm, s.nodes.size() > 2 ? s.gemm_x[1] : s.gemm};
           s.cluster_k = gemm_cluster_split(gs, s.tc, int(s.nodes.size()));
           if (s.cluster_k > 1) s.variant |= (s.cluster_k << 24) | (1 << 28);
+          else if (gemm_pair_eligible(gs, s.tc, int(s.nodes.size()))) s.variant |= 1 << 29;
         }
         break;
       }

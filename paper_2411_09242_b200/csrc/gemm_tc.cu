@@ -1608,6 +1608,14 @@ int gemm_cluster_split(const GemmParams* gs, const GemmTcHost& tc, int n_group) 
   return 0;
 }
 
+// True if the step runs as CTA pairs (two CTAs per 256 x 256 tile), judged on shapes and strides alone.
+bool gemm_pair_eligible(const GemmParams* gs, const GemmTcHost& tc, int n_group) {
+  const GemmParams& g = gs[0];
+  if (!tc.cfg.pair || !pair_enabled() || g.causal != CAUSAL_NONE || ((g.M + BM - 1) / BM) % 2 != 0) return false;
+  if (!vec_epilogue_ok(gs, n_group, false)) return false;
+  return (g.act == ACT_NONE) || (!g.has_res && !g.c_f32);   // one of the templated epilogues applies
+}
+
 cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_group, int split_k, int cluster_k, float* partial,
                            uint32_t* status, cudaStream_t stream) {
   const GemmParams& g = gs[0];

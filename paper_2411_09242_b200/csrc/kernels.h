@@ -177,6 +177,8 @@ int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t
 // Cluster size of the cluster split-K form (CTAs of one cluster share an output tile, reduced through
 // distributed shared memory; no scratch); 0 if the step runs the persistent kernel.
 int gemm_cluster_split(const GemmParams* gs, const GemmTcHost& tc, int n_group);
+// True if the step runs on the CTA-pair kernel (two CTAs of a cluster per 256 x 256 tile).
+bool gemm_pair_eligible(const GemmParams* gs, const GemmTcHost& tc, int n_group);
 bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc);
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);

@@ -203,7 +203,8 @@ def test_rope_in_every_head_layout(dtype, interleaved):
 
 
 @pytest.mark.parametrize("dtype", DT)
-@pytest.mark.parametrize("case", [dict(B=1, S=128, nh=12, D=64), dict(B=2, S=100, nh=3, D=40), dict(B=3, S=257, nh=2, D=128)])
+@pytest.mark.parametrize("case", [dict(B=1, S=128, nh=12, D=64), dict(B=2, S=100, nh=3, D=40), dict(B=3, S=257, nh=2, D=128),
+                                  dict(B=2, S=37, nh=5, D=64), dict(B=1, S=20, nh=33, D=256), dict(B=2, S=9, nh=17, D=128)])
 @pytest.mark.parametrize("target", ["BHSD", "BHDS"])
 def test_layout_transforms_bit_exact(dtype, case, target):
     g, a = synth.permute_case(target=target, dtype=dtype, **case)
@@ -295,6 +296,36 @@ def test_fused_attention_shapes_and_operand_majors(D, causal, S):
         assert "ATTN" in [s["kernel_name"] for s in plan.steps()]
         assert_close(got[g.outputs[0]], ref, synth.BF16, f"attention D={D} S={S} causal={causal} k={k_layout} v={v_layout}")
         plan.close()
+
+
+@pytest.mark.parametrize("M,N,K", [(1024, 2552, 136), (512, 5120, 72), (768, 4096, 200)])
+def test_cta_pair_gemm_ragged_shapes(M, N, K):
+    """Enough 256-wide tiles for the CTA-pair kernel (two CTAs per 256 x 256 tile), with a ragged last column
+    tile, a k range that is not a multiple of the stage depth and, in the last case, an odd number of row tiles
+    (which must fall back to the single-CTA kernel)."""
+    g = single_op_graph(synth.LINEAR, [[M, K], [K, N], [N]], [M, N], synth.BF16, {"contract": 1},
+                        in_kinds={1: synth.CONST, 2: synth.CONST})
+    feeds = {0: rand_feed([M, K], synth.BF16, 1), 1: rand_feed([K, N], synth.BF16, 2), 2: rand_feed([N], synth.BF16, 3)}
+    ref = run_oracle(g, feeds)[3]
+    got, plan, runner = run_gpu(g, feeds, synth.default_candidates(g))
+    v = plan.steps()[0]["variant"]
+    assert ((v >> 8) & 0xfff) == 256 and bool((v >> 29) & 1) == (M % 256 == 0)
+    assert_close(got[3], ref, synth.BF16, f"pair GEMM {M}x{N}x{K}")
+    runner.run()
+    assert np.array_equal(runner.outputs_host()[0], got[3])
+    plan.close()
+
+
+def test_gelu_erf_over_a_wide_range():
+    """The kernels evaluate erf as a clamped polynomial: check it element by element well beyond the clamp."""
+    shape = [4, 4096]
+    g = single_op_graph(synth.GELU, [shape], shape, synth.BF16, {"gelu_tanh": 0})
+    x = rand_feed(shape, synth.BF16, 77, -9.0, 9.0)
+    ref = run_oracle(g, {0: x})[1]
+    got, plan, _ = run_gpu(g, {0: x})
+    err = np.abs(got[1].astype(np.float64) - ref)
+    assert np.all(err <= 3e-4 + 2.0 ** -8 * np.abs(ref))      # polynomial error + bf16 rounding of the output
+    plan.close()
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 768, 3072), (100, 256, 2048), (64, 1536, 1024)])
