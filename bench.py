@@ -283,8 +283,8 @@ def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=N
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--workload", default="bert_base", choices=list(synth.CONFIGS))
     ap.add_argument("--others", default="tiny,gpt2_small,llama", help="comma list of extra workloads to summarise")

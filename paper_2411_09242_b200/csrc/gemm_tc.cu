@@ -1032,24 +1032,32 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   int grp, bz, mt, nt;
   decode_tile(p, tile, grp, bz, mt, nt);
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    mbar_init(tfull, 1);
-    mbar_init(recv_bar, 1);
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+  // The producer warp needs the barriers, not the tensor-memory address: it initialises them, arrives on a named
+  // barrier and goes on to its loads while warp 1 allocates tensor memory; everyone else waits for both.
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+      mbar_init(tfull, 1);
+      mbar_init(recv_bar, 1);
+      *abort_flag = 0;
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      mbar_expect_tx(recv_bar, uint32_t(BM) * uint32_t(bn) * 4u);   // split_k slices of 128 / split_k rows
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+    }
+    __syncwarp();
+    __threadfence_block();
+    asm volatile("bar.arrive 2, 320;" ::: "memory");
+  } else {
+    if (warp == 1) {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    asm volatile("bar.sync 2, 320;" ::: "memory");
+    tc_fence_after();
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(tmem_cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot_ptr;
-  if (threadIdx.x == 0) mbar_expect_tx(recv_bar, uint32_t(BM) * uint32_t(bn) * 4u);   // split_k slices of 128 / split_k rows
+  const uint32_t tmem_base = *tmem_slot_ptr;   // (not meaningful in warp 0, which does not use it)
   cluster_arrive();   // "this CTA runs": peers may write into its receive buffer after the matching wait
 
   if (warp == 0) {
@@ -1184,6 +1192,10 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   }
   __syncwarp();
   cluster_wait();   // every CTA of the cluster has started: its shared memory and barriers may be written
+  // Second cluster barrier, arrival: "every slice sent to this CTA has landed", which is what the senders need to
+  // know before their shared memory may go. Warps 0-1 have nothing to add and arrive now; the epilogue threads
+  // arrive once the receive barrier has completed; everybody waits at the very end, after the stores.
+  if (warp < 2) cluster_arrive();
   if (warp >= 2) {
     asm volatile("bar.sync 1, 256;" ::: "memory");   // the whole partial tile is in shared memory
     // rows [d * rows_per, ...) go to CTA d, into the slice that belongs to this CTA's rank; CTA r starts
@@ -1211,6 +1223,7 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       if (!*abort_flag) atomicOr(p.status, 0x8u);
       *abort_flag = 1;
     }
+    cluster_arrive();
     if (got) {
       // two items per pass: their shared-memory reads and address arithmetic overlap
 #pragma unroll 1
@@ -1243,8 +1256,7 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     }
   }
   __syncwarp();
-  cluster_arrive();   // this CTA has received every slice, so every copy sent to it has completed
-  cluster_wait();     // ... and so have the copies it sent: its shared memory may go
+  cluster_wait();     // every peer has received what this CTA sent: its shared memory may go
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
