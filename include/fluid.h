@@ -101,7 +101,10 @@ typedef struct fluid_layout_candidates {
 
 /* The paper's external cost function eval(node, layouts) (Algorithm 3): the time of one node
  * given a layout index for each of its tensors. Return +infinity for an unsupported
- * combination. node_id is the graph's op id (custom evaluation implies fusion = 0). */
+ * combination. node_id is the graph's op id (custom evaluation implies fusion = 0). If the function
+ * rates as finite a combination that no kernel can run and the plan ends up using it, fluid_plan
+ * still returns the plan (sequences, layouts and arena can be inspected) and fluid_run refuses it
+ * with FLUID_EUNSUPPORTED. */
 typedef double (*fluid_eval_fn)(void* user, int32_t node_id, int32_t n_tensors,
                                 const int32_t* tensor_ids, const int32_t* layout_index);
 

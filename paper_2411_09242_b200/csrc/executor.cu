@@ -2,6 +2,7 @@
 // arena_ptr + offset (or to a bound constant / caller buffer) and launches one kernel per step on
 // the caller's stream. No allocation, no synchronisation, no copies (the paper's "user only
 // needs to allocate a big block of buffer", Sec. "Evaluation", memory-allocation paragraph).
+#include <cmath>
 #include <atomic>
 #include <cstdio>
 #include <vector>
@@ -24,6 +25,21 @@ int finalize_steps(fluid_plan_s* p) {
     const Node& n = p->nodes[s.node];
     const TensorDesc& ty = T[n.out];
     const double es = (double)ty.esize();
+    // A caller's cost function may rate a combination of layouts the kernels cannot run (the built-in table
+    // never does): refuse it here, at plan time, rather than run a kernel on strides it does not understand.
+    // (Such a plan is kept: its sequences, layouts and arena can still be inspected. It refuses to run.)
+    bool feasible = true;
+    for (int ni : s.nodes) {
+      if (!std::isfinite(node_cost(p, p->nodes[ni], lo))) {
+        if (!p->opts.eval) {
+          set_error("step for op %d: no kernel runs this operator with the chosen layouts", p->nodes[ni].ops[0]);
+          return FLUID_EUNSUPPORTED;
+        }
+        if (p->not_runnable_op < 0) p->not_runnable_op = p->nodes[ni].ops[0];
+        feasible = false;
+      }
+    }
+    if (!feasible) continue;
     switch (n.kind) {
       case N_EMBED: {
         s.kernel = FLUID_K_EMBED;
@@ -281,6 +297,11 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
   if (reinterpret_cast<uintptr_t>(arena_ptr) % FLUID_ARENA_ALIGN) {
     set_error("arena_ptr must be %d-byte aligned", FLUID_ARENA_ALIGN);
     return FLUID_EALIGN;
+  }
+  if (p->not_runnable_op >= 0) {
+    set_error("the plan's cost function chose layouts for op %d that no kernel runs: the plan can be inspected, not run",
+              p->not_runnable_op);
+    return FLUID_EUNSUPPORTED;
   }
   const auto& T = p->graph.tensors;
   std::vector<const void*> key;

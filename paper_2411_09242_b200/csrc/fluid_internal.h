@@ -123,6 +123,7 @@ struct fluid_plan_s {
   std::vector<int> layout;                      // per tensor: candidate index
   std::vector<int> alias_root;                  // per tensor: root tensor id
   std::vector<int> folded;                      // per tensor: 1 if removed by fusion
+  int not_runnable_op = -1;                     // a caller's cost function chose layouts no kernel runs for this op: the plan is kept for inspection, fluid_run refuses it
   std::vector<fluid::Step> steps;
   std::vector<fluid::ArenaRecord> records;
   std::vector<int> record_of;                   // per tensor (root): index in records or -1
@@ -143,6 +144,7 @@ struct fluid_plan_s {
 namespace fluid {
 void set_error(const char* fmt, ...);
 int finalize_steps(fluid_plan_s* p);               // executor-side: derive launch payloads
+double node_cost(const fluid_plan_s* p, const Node& n, const int* lo);   // built-in table; +infinity = no kernel
 int pack_constant_launch(const fluid_plan_s* p, int tid, const void* src, void* dst, void* stream);
 double node_cost(const fluid_plan_s* p, const Node& n, const int* layout_of /*per tensor*/);
 bool transpose_is_alias(const fluid_plan_s* p, const Node& n, const int* layout_of);

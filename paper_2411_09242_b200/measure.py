@@ -1,0 +1,128 @@
+"""The paper's external cost function, measured: eval(node, layouts) = the time of that operator, alone,
+with its tensors in those layouts, on the GPU at hand (Algorithm 3's `eval`; Sec. "Implementation": the
+compiler tries a layout and the runtime times it).
+
+`MeasuredEval(graph, candidates)` is a callable for `fluid.Plan(..., eval=...)`. Every time the planner's
+dynamic programme asks for the cost of (operator, layout per tensor), the answer comes from a table keyed
+by the operator's signature (kind, attributes, tensor shapes and dtypes) and the layouts; a missing entry is
+measured on the spot: a two-operator graph (the operator, then a copy to the caller's buffer) is planned
+with a cost function that forces exactly those layouts, bound to random constants, run a few times with one
+CUDA event pair per step, and the operator's own step time is recorded. Combinations the kernels cannot
+run are recorded as +infinity. Operators repeat across layers, so a model needs a few hundred measurements.
+
+Only marshalling and bookkeeping live here; the planning and the timed kernels are the library's.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+from . import fluid, synth
+
+FORBIDDEN = 1e9   # cost of a layout combination other than the forced one, inside a measuring plan
+
+
+class MeasuredEval:
+    def __init__(self, desc: synth.GraphDesc, candidates: dict, reps: int = 5, warmup: int = 2, seed: int = 7):
+        import torch
+        self.torch = torch
+        self.desc, self.cands, self.reps, self.warmup, self.seed = desc, candidates, reps, warmup, seed
+        self.table = {}        # (signature, layouts) -> seconds
+        self.measured = 0      # GPU measurements taken (table misses)
+        self._c = fluid.EVAL_FN(self._call)
+
+    @property
+    def callback(self):
+        """The C function pointer for `fluid.Plan(..., eval=...)` (keep this object alive while planning)."""
+        return self._c
+
+    # ---- the planner's side ----
+    def _call(self, user, node, n, tids, lidx):
+        try:
+            return self.cost(int(node), {int(tids[i]): int(lidx[i]) for i in range(n)})
+        except Exception:   # never let an exception cross the C boundary: unknown means unusable
+            return math.inf
+
+    def cost(self, op_id: int, layout_index: dict) -> float:
+        op = self.desc.ops[op_id]
+        tids = list(op["ins"]) + list(op["outs"])
+        perms = tuple(tuple(self.cands.get(t, [synth.identity_perm(len(self.desc.dims(t)))])[layout_index.get(t, 0)])
+                      for t in tids)
+        attrs = tuple(sorted((k, tuple(v) if isinstance(v, (list, tuple)) else v) for k, v in op["attrs"].items()))
+        sig = (op["kind"], attrs,
+               tuple((self.desc.tensors[t]["dtype"], tuple(self.desc.dims(t))) for t in tids))
+        key = (sig, perms)
+        if key not in self.table:
+            self.table[key] = self._measure(op, tids, perms)
+            self.measured += 1
+        return self.table[key]
+
+    # ---- one measurement ----
+    def _measure(self, op, tids, perms) -> float:
+        torch = self.torch
+        d = self.desc
+        g = synth.GraphDesc()
+        local, cands, consts, int_inputs = {}, {}, {}, []
+        for t, perm in zip(op["ins"], perms):
+            src = d.tensors[t]
+            if src["dtype"] == synth.I32:
+                lt = g.tensor(f"in{t}", synth.I32, src["dims"], synth.INPUT)
+                int_inputs.append(lt)
+            else:
+                # a constant may sit in any candidate layout and is packed outside the timed path
+                lt = g.tensor(f"in{t}", src["dtype"], src["dims"], synth.CONST)
+                a = synth.uniform(self.seed, lt, src["dims"], -1.0, 1.0)
+                consts[lt] = synth.round_bf16(a) if src["dtype"] == synth.BF16 else a
+            local[t] = lt
+            ident = synth.identity_perm(len(src["dims"]))
+            cands[lt] = [ident] if tuple(perm) == ident else [ident, tuple(perm)]
+        (t_out,), perm_out = op["outs"], perms[len(op["ins"])]
+        src = d.tensors[t_out]
+        y = g.tensor("y", src["dtype"], src["dims"], synth.ACT)
+        z = g.tensor("z", src["dtype"], src["dims"], synth.OUTPUT)
+        ident = synth.identity_perm(len(src["dims"]))
+        cands[y] = [ident] if tuple(perm_out) == ident else [ident, tuple(perm_out)]
+        cands[z] = [ident]
+        g.op(op["kind"], [local[t] for t in op["ins"]], [y], **op["attrs"])
+        g.op(synth.TRANSPOSE, [y], [z], perm=list(ident))
+        want = {lt: len(c) - 1 for lt, c in cands.items()}   # index of the forced layout of each local tensor
+
+        def forcing(user, node, n, ltids, lidx):
+            if node != 0:
+                return 0.0
+            return 0.0 if all(lidx[i] == want[ltids[i]] for i in range(n)) else FORBIDDEN
+
+        cb = fluid.EVAL_FN(forcing)
+        try:
+            plan = fluid.Plan(g, cands, eval=cb)
+        except fluid.FluidError:
+            return math.inf
+        try:
+            got = {lt: plan.tensor_info(lt).layout_index for lt in want}
+            if got != want:
+                return math.inf   # the planner could not honour the combination (its guard fell back to canonical)
+            runner = fluid.Runner(plan, consts)
+            if int_inputs:
+                # ids index the first dim of the table they look up
+                hi = d.dims(op["ins"][1])[0] if op["kind"] == synth.EMBED else 2
+                ids_shape = d.dims(op["ins"][0])
+                runner.set_inputs([np.asarray(synth.token_ids(self.seed, 0, ids_shape, hi), dtype=np.int32)])
+            steps = plan.steps()
+            mine = [i for i, s in enumerate(steps) if 0 in s["ops"]]
+            if len(mine) != 1:
+                return math.inf
+            stream = torch.cuda.current_stream().cuda_stream
+            args = (plan.handle, runner.arena.data_ptr(), [b.data_ptr() for b in runner.inputs],
+                    [b.data_ptr() for b in runner.outputs], stream)
+            for _ in range(self.warmup):
+                fluid.fluid_run(*args)
+            ms = [fluid.fluid_run_profiled(*args)[mine[0]] for _ in range(self.reps)]
+            torch.cuda.synchronize()
+            if runner.status() != 0:
+                return math.inf
+            return float(np.median(ms)) * 1e-3
+        except fluid.FluidError:
+            return math.inf
+        finally:
+            plan.close()

@@ -362,3 +362,29 @@ def test_split_k_inside_a_model():
     for t in m.graph.outputs:
         assert_close(got[t], ref[t], synth.BF16, "encoder with split-K")
     plan.close()
+
+
+@pytest.mark.parametrize("family,dtype", [("encoder", synth.F32), ("gpt", synth.BF16), ("llama", synth.BF16)])
+def test_plan_from_measured_costs(family, dtype):
+    """The paper's eval: every (operator, layouts) cost the dynamic programme asks for is measured on the GPU
+    (one operator alone, its tensors forced into those layouts). The plan that comes out is a valid plan:
+    same results as the oracle, a cost that is the sum of measured times, not above the all-canonical cost."""
+    from paper_2411_09242_b200.measure import MeasuredEval
+    cfg = synth.scaled(SMALL[family], dtype=dtype, L=1)
+    m = synth.build_model(cfg)
+    cands = synth.default_candidates(m.graph)
+    ev = MeasuredEval(m.graph, cands, reps=3, warmup=1)
+    plan = fluid.Plan(m.graph, cands, eval=ev.callback)
+    assert ev.measured > len({o["kind"] for o in m.graph.ops}) and 0 < plan.cost <= plan.canonical_cost < 1.0
+    ref = run_oracle(m.graph, model_feeds(m))
+    runner = fluid.Runner(plan, m.consts)
+    runner.set_inputs([m.ids])
+    runner.run()
+    assert runner.status() == 0
+    for tid, got in zip(m.graph.outputs, runner.outputs_host()):
+        assert_close(got, ref[tid], dtype, f"measured-cost plan {family} output {tid}")
+    # asking again costs nothing: the table answers
+    before = ev.measured
+    plan2 = fluid.Plan(m.graph, cands, eval=ev.callback)
+    assert ev.measured == before and plan2.cost == plan.cost
+    plan.close(); plan2.close()

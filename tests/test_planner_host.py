@@ -258,3 +258,35 @@ def test_split_k_takes_a_step_lifetime_scratch_slice():
     assert OA.check_arena(recs, offs, on.arena_bytes) == []
     assert on.arena_bytes >= off.arena_bytes
     off.close(); on.close()
+
+
+def test_a_cost_function_that_picks_unrunnable_layouts_gives_a_plan_that_refuses_to_run():
+    """The caller's eval may rate as cheap a combination no kernel can run (here: a softmax whose input and
+    output sit in different, non-row-contiguous layouts). The plan is still returned, for inspection, and
+    fluid_run refuses it before any device work."""
+    ensure_lib()
+    g = synth.GraphDesc()
+    BF = synth.BF16
+    x = g.tensor("x", BF, [2, 3, 16, 16], synth.INPUT)
+    a = g.tensor("a", BF, [2, 3, 16, 16])
+    b = g.tensor("b", BF, [2, 3, 16, 16])
+    y = g.tensor("y", BF, [2, 3, 16, 16], synth.OUTPUT)
+    g.op(synth.TRANSPOSE, [x], [a], perm=[0, 1, 2, 3])
+    sm = g.op(synth.SOFTMAX, [a], [b], causal=0, scale=1.0)
+    g.op(synth.TRANSPOSE, [b], [y], perm=[0, 1, 2, 3])
+    cands = synth.default_candidates(g)
+    assert len(cands[a]) == 6
+
+    def ev(user, node, n, tids, lidx):
+        if node != sm:
+            return 1.0
+        want = {a: 5, b: 2}
+        return 0.0 if all(lidx[i] == want[tids[i]] for i in range(n)) else 100.0
+
+    plan = fluid.Plan(g, cands, eval=fluid.EVAL_FN(ev))
+    assert plan.tensor_info(a).layout_index == 5 and plan.tensor_info(b).layout_index == 2
+    assert len(plan.steps()) >= 1 and plan.arena_bytes > 0
+    with pytest.raises(fluid.FluidError) as e:
+        fluid.fluid_run(plan.handle, 0x10000, [0x20000], [0x30000])
+    assert e.value.code == fluid.FLUID_EUNSUPPORTED and "no kernel runs" in str(e.value)
+    plan.close()
