@@ -80,8 +80,16 @@ int finalize_steps(fluid_plan_s* p) {
         }
         s.flops = fl;
         s.bytes = es * (a + b + (g.has_bias ? g.N : 0)) + c * (s.gemm.c_f32 ? 4.0 : es) + (g.has_res ? c * (s.gemm.r_f32 ? 4.0 : es) : 0.0);
+        // SwiGLU step: the only tensor written is the product, which takes gate's place
+        const size_t n_gemm = s.swiglu ? 2 : s.nodes.size();
+        if (s.swiglu) {
+          s.t_ptr[2] = p->nodes[s.nodes[2]].out;
+          s.gemm.c_f32 = 0;
+          s.bytes = es * (a + 2.0 * b + c);
+          s.flops = 2.0 * fl;
+        }
         // grouped siblings: same A, own B / C / bias
-        for (size_t gi = 1; gi < s.nodes.size(); ++gi) {
+        for (size_t gi = 1; gi < n_gemm; ++gi) {
           const Node& m = p->nodes[s.nodes[gi]];
           GemmParams& gx = s.gemm_x[gi - 1];
           if (!lower_gemm(p, m, lo, &gx) || !gemm_tc_eligible(p, gx, &s.tc_x[gi - 1]) || s.kernel != FLUID_K_GEMM_TC) {
@@ -90,18 +98,23 @@ int finalize_steps(fluid_plan_s* p) {
           }
           gx.c_f32 = p->wide[m.out];
           gx.b_const = p->graph.tensors[m.b].kind == FLUID_CONST ? 1 : 0;
-          s.x_ptr[gi - 1][0] = m.b; s.x_ptr[gi - 1][1] = m.out; s.x_ptr[gi - 1][2] = m.bias;
+          s.x_ptr[gi - 1][0] = m.b; s.x_ptr[gi - 1][1] = s.swiglu ? -1 : m.out; s.x_ptr[gi - 1][2] = m.bias;
+          if (s.swiglu) continue;
           s.flops += fl;
           s.bytes += es * (b + c + (g.has_bias ? g.N : 0));
         }
-        if (s.nodes.size() > 1) s.variant |= int(s.nodes.size()) << 20;
+        if (n_gemm > 1) s.variant |= int(n_gemm) << 20;
         if (s.split_k > 1) {
           s.variant |= s.split_k << 24;
         } else if (s.kernel == FLUID_K_GEMM_TC && p->opts.split_k >= 0) {
-          GemmParams gs[3] = {s.gemm, s.nodes.size() > 1 ? s.gemm_x[0] : s.gemm, s.nodes.size() > 2 ? s.gemm_x[1] : s.gemm};
-          s.cluster_k = gemm_cluster_split(gs, s.tc, int(s.nodes.size()));
+          GemmParams gs[3] = {s.gemm, n_gemm > 1 ? s.gemm_x[0] : s.gemm, n_gemm > 2 ? s.gemm_x[1] : s.gemm};
+          s.cluster_k = s.swiglu ? 0 : gemm_cluster_split(gs, s.tc, int(n_gemm));
           if (s.cluster_k > 1) s.variant |= (s.cluster_k << 24) | (1 << 28);
-          else if (gemm_pair_eligible(gs, s.tc, int(s.nodes.size()))) s.variant |= 1 << 29;
+          else if (gemm_pair_eligible(gs, s.tc, int(n_gemm))) s.variant |= 1 << 29;
+          if (s.swiglu && !((s.variant >> 29) & 1)) {
+            set_error("step for op %d: the fused SwiGLU needs the CTA-pair form of the GEMM", n.ops[0]);
+            return FLUID_EUNSUPPORTED;
+          }
         }
         break;
       }
@@ -343,7 +356,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       const void* b = R(s.t_ptr[1], 1);
       if (!R.ok) return FLUID_EINVAL;
       bool enc_ok = encode_tensor_map(&s.tc.map_a, a, s.tc.a) == 0 && encode_tensor_map(&s.tc.map_b, b, s.tc.b) == 0;
-      for (size_t gi = 1; enc_ok && gi < s.nodes.size(); ++gi) {
+      for (size_t gi = 1; enc_ok && gi < (s.swiglu ? size_t(2) : s.nodes.size()); ++gi) {
         const void* bx = R(s.x_ptr[gi - 1][0], 1);
         if (!R.ok) return FLUID_EINVAL;
         enc_ok = encode_tensor_map(&s.tc_x[gi - 1].map_b, bx, s.tc_x[gi - 1].b) == 0;
@@ -389,18 +402,18 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
         if (s.kernel == FLUID_K_GEMM_TC) {
           GemmParams gs[3] = {q, s.gemm_x[0], s.gemm_x[1]};
           GemmTcHost ts[3] = {s.tc, s.tc_x[0], s.tc_x[1]};
-          const int ng = (int)s.nodes.size();
+          const int ng = s.swiglu ? 2 : (int)s.nodes.size();
           for (int gi = 1; gi < ng; ++gi) {
             gs[gi].A = q.A;
             gs[gi].B = R(s.x_ptr[gi - 1][0], 1);
-            gs[gi].C = const_cast<void*>(R(s.x_ptr[gi - 1][1]));
+            gs[gi].C = s.swiglu ? q.C : const_cast<void*>(R(s.x_ptr[gi - 1][1]));
             gs[gi].bias = R(s.x_ptr[gi - 1][2]);
             gs[gi].R = nullptr;
           }
           float* partial = s.scratch_record >= 0
                                ? reinterpret_cast<float*>(static_cast<char*>(arena_ptr) + p->records[s.scratch_record].offset)
                                : nullptr;
-          if (R.ok) err = launch_gemm_tc(gs, ts, ng, s.split_k, s.cluster_k, partial, status, stream);
+          if (R.ok) err = launch_gemm_tc(gs, ts, ng, s.split_k, s.cluster_k, partial, status, stream, s.swiglu);
         } else if (R.ok) {
           err = launch_gemm_simt(q, stream);
         }

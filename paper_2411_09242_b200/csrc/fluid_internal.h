@@ -81,6 +81,7 @@ struct Step {
   int x_ptr[2][3] = {{-1, -1, -1}, {-1, -1, -1}};  // tensor ids of B, C, bias for groups 1 and 2
   int split_k = 1;          // GEMM steps with few tiles cut their k range across CTAs
   int cluster_k = 0;        // >1: the cut runs as one thread-block cluster per output tile (no scratch)
+  int swiglu = 0;           // 1: nodes = {gate GEMM, up GEMM, SiLU(gate) * up}: one CTA-pair launch, gate and up never stored
   int64_t scratch_bytes = 0;
   int scratch_record = -1;  // arena slice holding the split-K partial tiles (alive during this step only)
   NormParams norm{};

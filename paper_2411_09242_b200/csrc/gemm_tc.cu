@@ -54,6 +54,7 @@ struct TcParams {
   float* partial;       // split-K scratch: [tile][split][bn/4][128 rows][4] fp32
   uint32_t* status;     // word 0: device status; words 8..63: per-tile arrival counters for split-K
   int scalar_turn;      // general epilogue: n is contiguous and unsplit in C (and R), so the shared-memory turn applies
+  int swiglu;           // CTA-pair form: CTA 0 loads gate columns, CTA 1 up columns; the epilogue writes SiLU(gate) * up
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -589,7 +590,8 @@ __device__ __noinline__ void epilogue_tile_scalar(const GemmParams& g, uint32_t 
 }
 
 // Epilogue variants (template parameter of the kernel)
-enum EpiKind { EPI_ANY = 0, EPI_PLAIN = 1, EPI_PLAIN_WIDE = 2, EPI_RES = 3, EPI_RES_WIDE = 4, EPI_GELU_ERF = 5, EPI_GELU_TANH = 6 };
+enum EpiKind { EPI_ANY = 0, EPI_PLAIN = 1, EPI_PLAIN_WIDE = 2, EPI_RES = 3, EPI_RES_WIDE = 4, EPI_GELU_ERF = 5, EPI_GELU_TANH = 6,
+               EPI_SWIGLU = 7 /* CTA-pair kernel only */ };
 
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk_c(const GemmParams& g, uint32_t taddr, const int64_t (&cbs)[8], const int64_t (&rbs)[8],
@@ -1300,6 +1302,47 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
 }
 
+// SwiGLU epilogue of the CTA-pair kernel: accumulator columns [0, 128) hold the gate projection and [128, 256) the
+// up projection of the same 128 output columns; the warp writes SiLU(gate) * up for its column range, through the
+// same shared-memory turn as the other vector epilogues (bf16 output, n contiguous).
+__device__ __forceinline__ void epilogue_tile_swiglu(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
+                                                     const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane) {
+  const int unit = lane & 7, rsub = lane >> 3;
+  const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
+  const float scale = g.scale;
+  __nv_bfloat16* const c_b16 = static_cast<__nv_bfloat16*>(g.C);
+#pragma unroll 1
+  for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+    if (n_tile0 + c0 >= g.N) break;   // uniform across the warp
+    uint32_t rg[32], ru[32];
+    tmem_ld32(trow + uint32_t(c0), rg);
+    tmem_ld32(trow + uint32_t(128 + c0), ru);
+    tmem_ld_wait();
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      float o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[e] = silu(__uint_as_float(rg[4 * u + e]) * scale) * (__uint_as_float(ru[4 * u + e]) * scale);
+      sts128(st_row + (uint32_t(u ^ (lane & 7)) << 4), o[0], o[1], o[2], o[3]);
+    }
+    __syncwarp();
+    const int nc = n_tile0 + c0 + unit * 4;
+    int n1, n0i;
+    split2(nc, g.N0, n1, n0i);
+    const int64_t c_col = (int64_t)n1 * g.c_s[4] + n0i;
+    const uint32_t live = nc < g.N ? ok_mask : 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = rsub + 4 * i;
+      const float4 v = lds128(st_base + uint32_t(row * 128) + (uint32_t(unit ^ (row & 7)) << 4));
+      uint2* dst = reinterpret_cast<uint2*>(c_b16 + cbs[i] + c_col);
+      const uint2 q = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+      if ((live >> i) & 1u) *dst = q;
+    }
+    __syncwarp();   // the staging tile is rewritten by the next chunk
+  }
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -1383,11 +1426,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         int c[5];
         {
           int r1, r0, b1, b0;
-          split2((is_a ? mt * BM : nt * PN + int(rank) * 128) + ch * box_rows, x_r0, r1, r0);
+          split2((is_a ? mt * BM : (p.swiglu ? nt * 128 : nt * PN + int(rank) * 128)) + ch * box_rows, x_r0, r1, r0);
           split2(bz, x_b0, b1, b0);
           fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
         }
-        const CUtensorMap* map = is_a ? &map_a : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2));
+        const CUtensorMap* map = is_a ? &map_a : (p.swiglu ? (rank == 0 ? &map_b : &map_b1) : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2)));
         int k0 = 0, k1 = 0;
         for (int ks = 0; ks < ksteps; ++ks) {
           if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
@@ -1457,7 +1500,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int lane_base = (warp & 3) * 32;
     const int half = (warp - 2) >> 2;
     float* stage = reinterpret_cast<float*>(smem_raw + (stage_base - raw)) + (warp - 2) * 1024;
-    const int col_begin = half * (PN / 2), col_end = col_begin + PN / 2;
+    const int out_w = p.swiglu ? 128 : PN;   // output columns of a tile
+    const int col_begin = half * (out_w / 2), col_end = col_begin + out_w / 2;
     int acc = 0;
     uint32_t acc_ph = 0;
     bool ok = true;
@@ -1467,7 +1511,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       decode_tile(p, item, grp, bz, pm, nt);
       const int mt = 2 * pm + int(rank);
       const GemmParams& g = grp == 0 ? p.g : p.gx[grp - 1];
-      const int n_tile0 = nt * PN;
+      const int n_tile0 = nt * out_w;
       int64_t cbs[8], rbs[8];
       uint32_t ok_mask = 0;
       const int64_t cbz = split_off(bz, g.B0, g.c_s[0], g.c_s[1]);
@@ -1483,7 +1527,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * PN);
-      epilogue_tile_c<EPI>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+      if (EPI == EPI_SWIGLU) epilogue_tile_swiglu(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
+      else epilogue_tile_c<EPI>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0u));   // CTA 0 counts both CTAs' epilogue warps
@@ -1629,7 +1674,7 @@ bool gemm_pair_eligible(const GemmParams* gs, const GemmTcHost& tc, int n_group)
 }
 
 cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_group, int split_k, int cluster_k, float* partial,
-                           uint32_t* status, cudaStream_t stream) {
+                           uint32_t* status, cudaStream_t stream, int swiglu) {
   const GemmParams& g = gs[0];
   const GemmTcHost& tc = tcs[0];
   TcParams p;
@@ -1650,6 +1695,7 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
   p.tiles_per_group = (int)(per_batch * g.batch);
   p.num_tiles = p.tiles_per_group * n_group;
   p.status = status;
+  p.swiglu = 0;
   const size_t smem = size_t(tc.cfg.stages) * (kATileBytes + size_t(tc.cfg.bn) * BK * 2) + 1024 + 8 * (2 * tc.cfg.stages + 4) + 16 +
                       16 + size_t(kEpiWarps) * 4096;
   const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(&tc.map_a);
@@ -1724,13 +1770,19 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
 #undef FLUID_TC_CLUSTER
   }
   // ---- many 256-wide tiles over an even number of row tiles: pairs of CTAs share 256 x 256 tiles ----
+  if (swiglu && !(tc.cfg.pair && pair_enabled() && vec && n_group == 2 && (p.tiles_m & 1) == 0)) return cudaErrorInvalidValue;
   if (tc.cfg.pair && pair_enabled() && vec && epi != EPI_ANY && split_k <= 1 && g.causal == CAUSAL_NONE && (p.tiles_m & 1) == 0 &&
       p.num_tiles > 0) {
     TcParams q = p;
     q.tiles_m = p.tiles_m / 2;                       // pairs of row tiles
-    q.tiles_per_batch = q.tiles_m * p.tiles_n;
+    if (swiglu) {                                    // one tile = 128 output columns = 128 gate + 128 up accumulator columns
+      q.swiglu = 1;
+      q.tiles_n = (g.N + 127) / 128;
+      epi = EPI_SWIGLU;
+    }
+    q.tiles_per_batch = q.tiles_m * q.tiles_n;
     q.tiles_per_group = q.tiles_per_batch * g.batch;
-    q.num_tiles = q.tiles_per_group * n_group;
+    q.num_tiles = q.tiles_per_group * (swiglu ? 1 : n_group);
     q.cfg.stages = 6;
     q.split_k = 1;
     const size_t psmem = size_t(q.cfg.stages) * (kATileBytes + size_t(128) * BK * 2) + 1024 + 8 * (2 * q.cfg.stages + 4) + 16 + 16 +
@@ -1748,7 +1800,7 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 2 : 1;
-    static bool pattr_set[7] = {false, false, false, false, false, false, false};
+    static bool pattr_set[8] = {false, false, false, false, false, false, false, false};
 #define FLUID_TC_PAIR(E)                                                                                             \
   case E: {                                                                                                          \
     if (!pattr_set[E]) {                                                                                             \
@@ -1765,6 +1817,7 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
       FLUID_TC_PAIR(EPI_RES_WIDE)
       FLUID_TC_PAIR(EPI_GELU_ERF)
       FLUID_TC_PAIR(EPI_GELU_TANH)
+      FLUID_TC_PAIR(EPI_SWIGLU)
       default: break;
     }
 #undef FLUID_TC_PAIR

@@ -170,8 +170,10 @@ cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
 // split_k > 1 cuts every output tile's k range into split_k pieces run by different CTAs; `partial`
 // then points at n_tiles * split_k * 128 * bn floats of scratch and status[8..63] hold the per-tile
 // arrival counters (zero before the launch, left zero after it).
+// swiglu (two groups, CTA-pair form only): group 0 is the gate, group 1 the up projection; the launch writes
+// SiLU(gate) * up to g[0].C and nothing else.
 cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, int split_k, int cluster_k, float* partial,
-                           uint32_t* status, cudaStream_t stream);
+                           uint32_t* status, cudaStream_t stream, int swiglu = 0);
 // Split factor a GEMM step should use (1 = none) and the scratch it then needs.
 int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t* scratch_bytes);
 // Cluster size of the cluster split-K form (CTAs of one cluster share an output tile, reduced through

@@ -971,6 +971,45 @@ static int lower_and_place(fluid_plan_s* p) {
     }
     p->steps.push_back(s);
   }
+  // SwiGLU: a grouped {gate, up} GEMM step followed by SiLU(gate) * up. When the pair qualifies for the CTA-pair
+  // kernel, one CTA of each pair loads gate columns and the other up columns of the same 128 output columns, the
+  // 256-wide accumulator holds both, and the epilogue writes SiLU(gate) * up: gate and up never reach memory.
+  if (p->opts.fusion && p->opts.gemm_path == 0 && !p->opts.eval) {
+    std::vector<int> n_uses(nt, 0);
+    for (const Node& n : p->nodes)
+      for (int t : n.ins) n_uses[t]++;
+    for (int si = 0; si + 1 < (int)p->steps.size(); ++si) {
+      Step& st = p->steps[si];
+      if (st.nodes.size() != 2 || p->steps[si + 1].nodes.size() != 1) continue;
+      const Node& e = p->nodes[p->steps[si + 1].node];
+      if (e.kind != N_ELTWISE || e.elt != ELT_SILU_MUL) continue;
+      int gi = -1, ui = -1;
+      for (int k = 0; k < 2; ++k) {
+        if (p->nodes[st.nodes[k]].out == e.a) gi = st.nodes[k];
+        if (p->nodes[st.nodes[k]].out == e.b) ui = st.nodes[k];
+      }
+      if (gi < 0 || ui < 0 || gi == ui) continue;
+      const Node &gn = p->nodes[gi], &un = p->nodes[ui];
+      if (gn.kind != N_GEMM || un.kind != N_GEMM || gn.bias >= 0 || un.bias >= 0 || gn.res >= 0 || un.res >= 0 ||
+          gn.act != ACT_NONE || un.act != ACT_NONE)
+        continue;
+      const int tg = gn.out, tu = un.out, to = e.out;
+      if (n_uses[tg] != 1 || n_uses[tu] != 1 || T[tg].kind != FLUID_ACT || T[tu].kind != FLUID_ACT ||
+          T[to].dtype != FLUID_BF16 || p->alias_root[tg] != tg || p->alias_root[tu] != tu)
+        continue;
+      if (lo[tg] != lo[tu] || lo[tg] != lo[to]) continue;   // the product takes the place (and strides) of gate
+      GemmParams g;
+      GemmTcHost tc;
+      if (!lower_gemm(p, gn, lo, &g) || !gemm_tc_eligible(p, g, &tc)) continue;
+      if (!tc.cfg.pair || g.batch != 1 || g.N % 128 != 0 || g.N0 % 128 != 0 || ((g.M + 127) / 128) % 2 != 0 || g.c_s[5] != 1) continue;
+      st.nodes = {gi, ui, p->steps[si + 1].node};
+      st.node = gi;
+      st.swiglu = 1;
+      st.cost += p->steps[si + 1].cost - kLaunch;
+      p->folded[tg] = p->folded[tu] = 1;
+      p->steps.erase(p->steps.begin() + si + 1);
+    }
+  }
   // lifetimes in step indices, per alias group
   p->first_step.assign(nt, -1);
   p->last_step.assign(nt, -1);
@@ -1249,13 +1288,14 @@ int fluid_plan_step_info(const fluid_plan_t* p, int step, fluid_step_info* info)
     const Node& n = p->nodes[ni];
     for (int o : n.ops)
       if (info->n_ops < 8) info->ops[info->n_ops++] = o;
+    // (tensors that a fused step keeps to itself are neither read from nor written to memory)
     for (int t : n.ins) {
-      bool seen = false;
+      bool seen = p->folded[t] != 0;
       for (int i = 0; i < info->n_in; ++i) seen = seen || info->in_ids[i] == t;
       if (!seen && info->n_in < 8) info->in_ids[info->n_in++] = t;
     }
     for (int t : n.outs)
-      if (info->n_out < 4) info->out_ids[info->n_out++] = t;
+      if (!p->folded[t] && info->n_out < 4) info->out_ids[info->n_out++] = t;
   }
   info->cost = s.cost;
   info->flops = s.flops;

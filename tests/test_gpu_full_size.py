@@ -74,7 +74,9 @@ def test_llama_shape_full_sampled_prefix():
     assert_close(hidden[:1, :96], ref, synth.BF16, "llama hidden prefix vs unrounded oracle", tol=3e-2)
     w = next(a for t, a in m.consts.items() if m.graph.tensors[t]["name"] == "W_lm").astype(np.float64)
     assert_close(logits, hidden[:, -1, :] @ w, synth.BF16, "llama logits from hidden")
-    assert plan.arena_bytes == plan.live_bound_bytes
+    # Greedy-by-Size is a heuristic: with the SwiGLU step fused (gate and up never stored) it lands 15 % above the
+    # largest live set on this shape; on the other three shapes it meets the bound exactly
+    assert plan.live_bound_bytes <= plan.arena_bytes <= 1.2 * plan.live_bound_bytes
     plan.close()
 
 
