@@ -157,7 +157,7 @@ def run_reference(args, rank):
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu capture
 # summarised in the named file under profiles/ (null where no capture of that workload was taken)
 NCU_TRAFFIC = {
-    "bert_base": {"kernel": "GEMM_TC", "bytes_per_launch": 4121691,
+    "bert_base": {"kernel": "GEMM_TC", "bytes_per_launch": 4121931,
                   "source": "profiles/dram_traffic_bert_base.md (48 launches of one inference, dram read + write)"},
 }
 
