@@ -16,7 +16,8 @@ from . import ops
 
 # operator codes of the graph description (the C header's fluid_op_kind values)
 (EMBED, LINEAR, ADD, MUL, GELU, SILU, SOFTMAX, LAYERNORM, RMSNORM, ROPE, TRANSPOSE, BMM_QK,
- BMM_PV, SELECT_LAST_TOKEN) = range(14)
+ BMM_PV, SELECT_LAST_TOKEN, CACHED_ATTENTION) = range(15)
+STATE = 4   # tensor kind: a caller-owned buffer an op reads and updates (a key/value cache)
 
 
 def run_op(kind, ins, attrs):
@@ -42,8 +43,9 @@ def run_op(kind, ins, attrs):
     if kind == RMSNORM:
         return [ops.rmsnorm(ins[0], ins[1], eps=attrs.get("eps", 1e-5))]
     if kind == ROPE:
+        pos0 = int(np.asarray(ins[1]).reshape(-1)[0]) if len(ins) > 1 else 0
         return [ops.rope(ins[0], base=attrs.get("rope_base", 10000.0),
-                         interleaved=bool(attrs.get("rope_interleaved", 0)))]
+                         interleaved=bool(attrs.get("rope_interleaved", 0)), pos0=pos0)]
     if kind == TRANSPOSE:
         return [ops.transpose(ins[0], attrs["perm"])]
     if kind == BMM_QK:
@@ -67,7 +69,8 @@ def run_graph(tensors, op_list, feeds, keep_all=False, store=None):
     tensors : list of dicts with "dims" (and "kind"); op_list : list of dicts with "kind",
     "ins", "outs", "attrs"; feeds : {tensor id: array} for every graph input and constant.
     Returns {tensor id: fp64 array} for every tensor (keep_all) or only those no op consumes
-    plus anything marked as a graph output (kind == 1).
+    plus anything marked as a graph output (kind == 1) and the final contents of every state
+    tensor (kind == 4).
     """
     vals = {}
     for tid, a in feeds.items():
@@ -76,7 +79,13 @@ def run_graph(tensors, op_list, feeds, keep_all=False, store=None):
     consumed = set()
     for op in op_list:
         ins = [vals[i] for i in op["ins"]]
-        outs = run_op(op["kind"], ins, op.get("attrs", {}))
+        if op["kind"] == CACHED_ATTENTION:
+            # the one op with a side effect: rows `pos` of its two state tensors are replaced
+            ctx, kc, vc = ops.cached_attention(*ins, scale=op.get("attrs", {}).get("scale", 1.0))
+            vals[op["ins"][3]], vals[op["ins"][4]] = kc, vc
+            outs = [ctx]
+        else:
+            outs = run_op(op["kind"], ins, op.get("attrs", {}))
         for tid, o in zip(op["outs"], outs):
             assert list(o.shape) == list(tensors[tid]["dims"]), (
                 tensors[tid].get("name"), o.shape, tensors[tid]["dims"])
@@ -85,4 +94,4 @@ def run_graph(tensors, op_list, feeds, keep_all=False, store=None):
     if keep_all:
         return vals
     return {tid: v for tid, v in vals.items()
-            if tensors[tid].get("kind") == 1 or (tid not in consumed and tid not in feeds)}
+            if tensors[tid].get("kind") in (1, STATE) or (tid not in consumed and tid not in feeds)}

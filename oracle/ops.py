@@ -14,7 +14,8 @@ Implementation": left input (i,k), right input (k,j), output (i,j)). The remaini
 the standard textbook definitions of the operators the paper lists by name (Softmax, LayerNorm,
 GELU, Add, Transpose, Gather; Sec. "Implementation", "Compiler").
 
-Pins (tests/test_oracle_ops.py): brute-force loops on tiny shapes, closed forms and invariants.
+Pins (tests/test_oracle_ops.py, tests/test_oracle_decode.py): brute-force loops on tiny shapes, closed
+forms and invariants; the cached decoding step against whole-sequence causal attention.
 No function here is "parity unpinned".
 """
 from __future__ import annotations
@@ -117,8 +118,9 @@ def mul(a, b):
     return np.asarray(a, np.float64) * np.asarray(b, np.float64)
 
 
-def rope(x, base=10000.0, interleaved=False):
-    """Rotary embedding on x[b, s, h, d]; position p = s (0-based).
+def rope(x, base=10000.0, interleaved=False, pos0=0):
+    """Rotary embedding on x[b, s, h, d]; position p = pos0 + s (0-based; pos0 is the number of
+    tokens that came before this call's first row, 0 for a whole sequence).
 
     Rotate-half pairing (i, i + D/2) by angle p * base^(-2i/D); the interleaved form pairs
     (2i, 2i+1) with the same angles.
@@ -127,7 +129,7 @@ def rope(x, base=10000.0, interleaved=False):
     B, S, nh, D = x.shape
     half = D // 2
     i = np.arange(half, dtype=np.float64)
-    theta = np.arange(S, dtype=np.float64)[:, None] * base ** (-2.0 * i / D)[None, :]
+    theta = (int(pos0) + np.arange(S, dtype=np.float64))[:, None] * base ** (-2.0 * i / D)[None, :]
     c = np.cos(theta)[None, :, None, :]
     s = np.sin(theta)[None, :, None, :]
     y = np.empty_like(x)
@@ -140,6 +142,35 @@ def rope(x, base=10000.0, interleaved=False):
         y[..., :half] = a * c - b * s
         y[..., half:] = b * c + a * s
     return y
+
+
+def cached_attention(q, k, v, k_cache, v_cache, pos, scale=1.0):
+    """One decoding step of attention against a key/value cache.
+
+    q[B,1,nh,D] is the query of the token at position t = pos; k, v[B,1,nkv,D] are its key and
+    value; k_cache, v_cache[B,Tmax,nkv,D] hold the keys and values of positions 0..t-1 (rows from t
+    on are unspecified). The step stores k, v as row t of the caches and returns
+      ctx[b,0,h,:] = sum_{j<=t} softmax_j(scale * q[b,0,h,:] . K[b,j,g,:]) V[b,j,g,:],  g = h // (nh/nkv),
+    that is, the row for query position t of causal attention over the t+1 tokens so far (query
+    heads share key/value heads in groups when nkv < nh). Returns (ctx, k_cache', v_cache').
+    """
+    q = np.asarray(q, np.float64)
+    kc = np.array(k_cache, dtype=np.float64)
+    vc = np.array(v_cache, dtype=np.float64)
+    t = int(np.asarray(pos).reshape(-1)[0])
+    B, one, nh, D = q.shape
+    Tmax, nkv = kc.shape[1], kc.shape[2]
+    assert one == 1 and 0 <= t < Tmax and nh % nkv == 0
+    kc[:, t] = np.asarray(k, np.float64)[:, 0]
+    vc[:, t] = np.asarray(v, np.float64)[:, 0]
+    ctx = np.zeros((B, 1, nh, D))
+    for b in range(B):
+        for h in range(nh):
+            g = h // (nh // nkv)
+            s = (kc[b, : t + 1, g, :] @ q[b, 0, h, :]) * float(scale)
+            e = np.exp(s - np.max(s))
+            ctx[b, 0, h, :] = (e / np.sum(e)) @ vc[b, : t + 1, g, :]
+    return ctx, kc, vc
 
 
 def transpose(x, perm):

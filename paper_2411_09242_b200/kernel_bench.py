@@ -58,10 +58,13 @@ def cases():
     g.op(synth.EMBED, [ids, tok], [x])
     out.append(("embed 32768x4096", g, lambda n: 2 * n * 2, None))
     for (M, N, K) in ((768, 768, 768), (2048, 2048, 2048), (4096, 4096, 4096), (8192, 8192, 8192), (4096, 2304, 768), (4096, 3072, 768),
-                      (2048, 11008, 4096), (128, 768, 3072), (128, 3072, 768), (4, 50257, 768)):
+                      (2048, 11008, 4096), (128, 768, 3072), (128, 3072, 768), (4, 50257, 768),
+                      (4, 4096, 4096), (4, 11008, 4096), (4, 4096, 11008), (4, 32000, 4096)):
         for majors in (("row", "col"), ("col", "row")) if M == N == K and M <= 4096 else (("row", "col"),):
             gg, _ = synth.gemm_case(M, N, K, *majors, materialize=False)
-            out.append((f"gemm {M}x{N}x{K} A {majors[0]} B {majors[1]}", gg, None, 2.0 * M * N * K))
+            # few rows: the step streams the weight once, so bytes are the figure; otherwise flops
+            out.append((f"gemm {M}x{N}x{K} A {majors[0]} B {majors[1]}", gg,
+                        (lambda n, b=2.0 * (M * K + K * N + M * N): b) if M <= 16 else None, 2.0 * M * N * K))
     return out
 
 
@@ -101,7 +104,7 @@ def main(argv):
         for d in g.tensors[g.outputs[0]]["dims"]:
             n *= d
         steps = "+".join(s["kernel_name"] for s in plan.steps())
-        if flops is not None:
+        if flops is not None and fbytes is None:
             print(f"{name:44s} {steps:10s} {us:9.1f} us  {flops / us / 1e6:8.1f} TFLOP/s  status {r.status()}")
         else:
             by = fbytes(n)

@@ -26,11 +26,11 @@ import numpy as np
 
 # ---- enumerations shared by the graph description (mirrored by include/fluid.h) -------------
 F32, BF16, I32 = 0, 1, 2
-INPUT, OUTPUT, CONST, ACT = 0, 1, 2, 3
+INPUT, OUTPUT, CONST, ACT, STATE = 0, 1, 2, 3, 4
 (EMBED, LINEAR, ADD, MUL, GELU, SILU, SOFTMAX, LAYERNORM, RMSNORM, ROPE, TRANSPOSE, BMM_QK,
- BMM_PV, SELECT_LAST_TOKEN) = range(14)
+ BMM_PV, SELECT_LAST_TOKEN, CACHED_ATTENTION) = range(15)
 OP_NAMES = ["EMBED", "LINEAR", "ADD", "MUL", "GELU", "SILU", "SOFTMAX", "LAYERNORM", "RMSNORM",
-            "ROPE", "TRANSPOSE", "BMM_QK", "BMM_PV", "SELECT_LAST_TOKEN"]
+            "ROPE", "TRANSPOSE", "BMM_QK", "BMM_PV", "SELECT_LAST_TOKEN", "CACHED_ATTENTION"]
 DTYPE_BYTES = {F32: 4, BF16: 2, I32: 4}
 
 WEIGHT_SEED = 2411
@@ -87,14 +87,14 @@ class GraphDesc:
     """A plain-data operator graph: tensors (edges) and ops (nodes) in declaration order."""
     tensors: list = field(default_factory=list)   # dicts: name, dtype, dims, kind
     ops: list = field(default_factory=list)       # dicts: kind, ins, outs, attrs
-    inputs: list = field(default_factory=list)    # tensor ids, declaration order
+    inputs: list = field(default_factory=list)    # tensor ids, declaration order (INPUT and STATE kinds)
     outputs: list = field(default_factory=list)
 
     def tensor(self, name, dtype, dims, kind=ACT) -> int:
         tid = len(self.tensors)
         self.tensors.append({"name": name, "dtype": dtype, "dims": [int(d) for d in dims],
                              "kind": kind})
-        if kind == INPUT:
+        if kind in (INPUT, STATE):
             self.inputs.append(tid)
         elif kind == OUTPUT:
             self.outputs.append(tid)
@@ -347,6 +347,76 @@ def build_model(cfg: ModelConfig, weight_seed: int = WEIGHT_SEED, token_seed: in
 
     tok_ids = token_ids(token_seed, 0, [B, S], V)
     return Model(cfg, g, b.consts, tok_ids)
+
+
+# ---- single-token decoding against a key/value cache ---------------------------------------------
+@dataclass
+class DecodeModel:
+    cfg: ModelConfig       # S == 1: one new token per sequence and step
+    t_max: int             # rows of every cache
+    graph: GraphDesc
+    consts: dict
+    ids: int               # tensor ids of the step's inputs
+    pos: int
+    caches: list           # [(k_cache tensor id, v_cache tensor id)] per layer
+
+
+def build_decode_model(cfg: ModelConfig, t_max: int, like: Model = None, weight_seed: int = WEIGHT_SEED,
+                       materialize: bool = True) -> DecodeModel:
+    """The llama-family graph of ONE decoding step: B sequences, one new token each, the keys and
+    values of the earlier tokens in per-layer caches [B, t_max, nh, D] that the caller owns and the
+    step extends (STATE tensors). `pos` (int32 [1], on the device at run time) is the number of
+    tokens already cached, the same for all sequences. Outputs: the final hidden state [B,1,H]
+    and the logits [B,1,V].
+
+    like: a whole-sequence model of the same family and widths; its weights are taken over by name,
+    so that a run of decoding steps can be compared with that model on the same tokens.
+    """
+    assert cfg.family == "llama", "decoding graphs are built for the rotary family only"
+    cfg = scaled(cfg, S=1)
+    b = _Builder(cfg, weight_seed, materialize and like is None)
+    g = b.g
+    B, H, V, nh, D = cfg.B, cfg.H, cfg.V, cfg.nh, cfg.D
+    ids = g.tensor("ids", I32, [B, 1], INPUT)
+    pos = g.tensor("pos", I32, [1], INPUT)
+    tok = b.const("tok_table", [V, H])
+    x = b.act("embed", [B, 1, H])
+    g.op(EMBED, [ids, tok], [x])
+    caches = []
+    for l in range(cfg.L):
+        pfx = f"l{l}"
+        n = _norm(b, x, f"{pfx}.ln1", True)
+        heads = {}
+        for nm in ("q", "k", "v"):
+            w = b.const(f"{pfx}.W{nm}", [H, nh, D])
+            t = b.act(f"{pfx}.{nm}", [B, 1, nh, D])
+            g.op(LINEAR, [n, w], [t], contract=1)
+            if nm != "v":
+                r = b.act(f"{pfx}.{nm}_rope", [B, 1, nh, D])
+                g.op(ROPE, [t, pos], [r], rope_base=10000.0, rope_interleaved=0)
+                t = r
+            heads[nm] = t
+        kc = g.tensor(f"{pfx}.k_cache", cfg.dtype, [B, t_max, nh, D], STATE)
+        vc = g.tensor(f"{pfx}.v_cache", cfg.dtype, [B, t_max, nh, D], STATE)
+        caches.append((kc, vc))
+        c = b.act(f"{pfx}.ctx", [B, 1, nh, D])
+        g.op(CACHED_ATTENTION, [heads["q"], heads["k"], heads["v"], kc, vc, pos], [c], scale=1.0 / math.sqrt(D))
+        wo = b.const(f"{pfx}.Wo", [nh, D, H])
+        o = b.act(f"{pfx}.attn_out", [B, 1, H])
+        g.op(LINEAR, [c, wo], [o], contract=2)
+        a = b.act(f"{pfx}.res1", [B, 1, H]); g.op(ADD, [x, o], [a])
+        n = _norm(b, a, f"{pfx}.ln2", True)
+        o = _mlp_swiglu(b, n, pfx)
+        x = b.act(f"{pfx}.res2", [B, 1, H]); g.op(ADD, [a, o], [x])
+    h = _norm(b, x, "final_norm", True, out_kind=OUTPUT)
+    wlm = b.const("W_lm", [H, V])
+    logits = b.act("logits", [B, 1, V], OUTPUT)
+    g.op(LINEAR, [h, wlm], [logits], contract=1)
+    consts = b.consts
+    if like is not None:
+        by_name = {like.graph.tensors[t]["name"]: a for t, a in like.consts.items()}
+        consts = {t: by_name[td["name"]] for t, td in enumerate(g.tensors) if td["kind"] == CONST}
+    return DecodeModel(cfg, t_max, g, consts, ids, pos, caches)
 
 
 # ---- the layout-transform / layout-aware GEMM sweep ---------------------------------------------
