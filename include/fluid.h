@@ -54,7 +54,10 @@ typedef enum {
 } fluid_status_t;
 
 typedef enum { FLUID_F32 = 0, FLUID_BF16 = 1, FLUID_I32 = 2 } fluid_dtype;
-typedef enum { FLUID_INPUT = 0, FLUID_OUTPUT = 1, FLUID_CONST = 2, FLUID_ACT = 3 } fluid_tensor_kind;
+/* FLUID_STATE: a caller-owned device buffer that a step both reads and updates and that lives on between runs (a
+ * key/value cache). It is passed to fluid_run among `inputs`, in declaration order with the FLUID_INPUT tensors,
+ * stays canonical and never sits in the arena. */
+typedef enum { FLUID_INPUT = 0, FLUID_OUTPUT = 1, FLUID_CONST = 2, FLUID_ACT = 3, FLUID_STATE = 4 } fluid_tensor_kind;
 
 /* Primitive operators ("nodes"). Shapes are logical, independent of layout.
  *  EMBED   (ids[B,S] i32, tok[V,H] [, pos[S,H]]) -> x[B,S,H] = tok[ids] (+ pos)
@@ -65,17 +68,24 @@ typedef enum { FLUID_INPUT = 0, FLUID_OUTPUT = 1, FLUID_CONST = 2, FLUID_ACT = 3
  *  SOFTMAX (s[..., n]) -> over the last dim, after multiplying by `scale`; causal: column j of
  *          row i (the last two dims) takes part only if j <= i, other outputs are exactly 0
  *  LAYERNORM (x, gamma, beta) / RMSNORM (x, gamma) -> over the last dim, population variance
- *  ROPE    (x[B,S,nh,D]) -> rotary embedding with position = index along dim 1
+ *  ROPE    (x[B,S,nh,D] [, pos i32[1]]) -> rotary embedding with position = index along dim 1 (+ pos[0], read on
+ *          the device at run time: the number of tokens that came before this call's first row)
  *  TRANSPOSE (x) -> y with y dim j = x dim perm[j]
  *  BMM_QK  (q[B,nh,S,D], kt[B,nh,D,S]) -> scale * q.kt  [B,nh,S,S]
  *  BMM_PV  (p[B,nh,S,S], v[B,nh,S,D]) -> p.v  [B,nh,S,D]
  *  SELECT_LAST_TOKEN (x[B,S,H]) -> x[:, S-1, :]  [B,H]
+ *  CACHED_ATTENTION (q[B,1,nh,D], k[B,1,nkv,D], v[B,1,nkv,D], k_cache STATE[B,Tmax,nkv,D], v_cache STATE[B,Tmax,nkv,D],
+ *          pos i32[1]) -> ctx[B,1,nh,D]: one decoding step. With t = pos[0] (read on the device at run time,
+ *          0 <= t < Tmax; the same for every sequence) the step stores k, v as row t of the caches and returns
+ *          ctx[b,0,h,:] = sum_{j<=t} softmax_j(scale * q[b,0,h,:] . k_cache[b,j,g,:]) v_cache[b,j,g,:], g = h / (nh/nkv):
+ *          the row for position t of causal attention over the t+1 tokens so far. Cache rows beyond t are neither
+ *          read nor written. t outside [0, Tmax) leaves caches and ctx untouched and sets bit 0x10 of fluid_status.
  */
 typedef enum {
   FLUID_OP_EMBED = 0, FLUID_OP_LINEAR = 1, FLUID_OP_ADD = 2, FLUID_OP_MUL = 3, FLUID_OP_GELU = 4,
   FLUID_OP_SILU = 5, FLUID_OP_SOFTMAX = 6, FLUID_OP_LAYERNORM = 7, FLUID_OP_RMSNORM = 8,
   FLUID_OP_ROPE = 9, FLUID_OP_TRANSPOSE = 10, FLUID_OP_BMM_QK = 11, FLUID_OP_BMM_PV = 12,
-  FLUID_OP_SELECT_LAST_TOKEN = 13, FLUID_OP_COUNT = 14
+  FLUID_OP_SELECT_LAST_TOKEN = 13, FLUID_OP_CACHED_ATTENTION = 14, FLUID_OP_COUNT = 15
 } fluid_op_kind;
 
 /* One attribute block serves every operator; unused fields are ignored. */
@@ -85,7 +95,7 @@ typedef struct fluid_op_attrs {
   int32_t gelu_tanh;         /* GELU: 0 = erf form, 1 = tanh approximation */
   int32_t rope_interleaved;  /* ROPE: 0 = pairs (i, i+D/2), 1 = pairs (2i, 2i+1) */
   int32_t perm[8];           /* TRANSPOSE */
-  double scale;              /* BMM_QK, SOFTMAX (0 is read as 1) */
+  double scale;              /* BMM_QK, SOFTMAX, CACHED_ATTENTION (0 is read as 1) */
   double eps;                /* LAYERNORM, RMSNORM */
   double rope_base;          /* ROPE */
 } fluid_op_attrs;
@@ -136,7 +146,7 @@ typedef struct fluid_plan_options {
 typedef enum {
   FLUID_K_EMBED = 0, FLUID_K_NORM = 1, FLUID_K_GEMM_SIMT = 2, FLUID_K_GEMM_TC = 3,
   FLUID_K_SOFTMAX = 4, FLUID_K_ROPE = 5, FLUID_K_ELTWISE = 6, FLUID_K_PERMUTE = 7,
-  FLUID_K_SELECT_LAST = 8, FLUID_K_ATTN = 9, FLUID_K_COUNT = 10
+  FLUID_K_SELECT_LAST = 8, FLUID_K_ATTN = 9, FLUID_K_ATTN_DECODE = 10, FLUID_K_COUNT = 11
 } fluid_kernel_id;
 
 typedef struct fluid_step_info {
@@ -225,7 +235,8 @@ FLUID_API int fluid_run(fluid_plan_t* plan, void* arena_ptr, const void* const* 
 FLUID_API int fluid_run_profiled(fluid_plan_t* plan, void* arena_ptr, const void* const* inputs,
                        void* const* outputs, fluid_stream stream, float* step_ms);
 /* Synchronises `stream`, reads the arena header and reports in *device_status 0 or the code a
- * kernel left when one of its bounded waits expired (returns FLUID_ETIMEOUT in that case). */
+ * kernel left: when one of its bounded waits expired (returns FLUID_ETIMEOUT), or, bit 0x10, when a
+ * CACHED_ATTENTION step read a position outside its cache (returns FLUID_EINVAL). */
 FLUID_API int fluid_status(const fluid_plan_t* plan, const void* arena_ptr, fluid_stream stream,
                  int* device_status);
 

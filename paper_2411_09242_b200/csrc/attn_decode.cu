@@ -1,0 +1,277 @@
+// Attention of one decoding step against a key/value cache (single new token per sequence).
+//
+// The step is bound by reading the cache once: per (sequence, head) t+1 rows of D keys and D values, one
+// multiply-add per byte pair. No tensor cores: rows stream through registers with 16-byte loads.
+//
+// Work split: one thread-block cluster of 8 CTAs per (sequence, query head); CTA r of the cluster takes a
+// contiguous eighth of the rows 0..t. Inside a CTA a row is owned by LPR = D / (16 bytes of elements)
+// adjacent lanes (a warp covers 32 / LPR rows per load instruction); every such lane group keeps a running
+// (max, sum, output) triple in the base-2 online-softmax form and has U rows of keys and of values in
+// flight at a time. Triples are merged lane group -> warp (shuffles) -> CTA (shared memory) -> cluster (each
+// CTA stores its triple into CTA 0's shared memory; one cluster barrier), and CTA 0 writes the D outputs.
+// The row of the new token comes from the step's own k and v operands, and the CTA that meets it stores it
+// as row t of the caches: no row is read from the cache in the launch that writes it.
+//
+// Nothing here spins: the only waits are __syncthreads and the hardware cluster barrier.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "device_utils.cuh"
+#include "fluid.h"
+#include "kernels.h"
+
+namespace fluid {
+
+namespace {
+
+constexpr int kSplits = 8;    // CTAs per cluster = row ranges per (sequence, head)
+constexpr int kWarps = 8;
+constexpr int kInFlight = 4;  // rows of K and of V a lane group holds before it consumes them
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+template <typename T>
+__device__ __forceinline__ void unpack16(const uint4& q, float (&v)[VecOf<T>::N]);
+template <>
+__device__ __forceinline__ void unpack16<float>(const uint4& q, float (&v)[4]) {
+  v[0] = __uint_as_float(q.x); v[1] = __uint_as_float(q.y); v[2] = __uint_as_float(q.z); v[3] = __uint_as_float(q.w);
+}
+template <>
+__device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4& q, float (&v)[8]) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+// weight of a partial with maximum m inside a merge whose maximum is M (an empty partial has m = -inf)
+__device__ __forceinline__ float merge_weight(float m, float M) { return m == -INFINITY ? 0.f : exp2f(m - M); }
+
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodeParams p) {
+  constexpr int V = VecOf<T>::N;
+  constexpr int D = LPR * V;
+  constexpr int GPW = 32 / LPR;          // rows per warp and load instruction
+  constexpr int RPI = GPW * kWarps;      // rows per CTA and load instruction
+  __shared__ float part[kWarps][D + 2];  // per warp: D outputs, max, sum
+  __shared__ float cl[kSplits][D + 2];   // per CTA of the cluster (filled in CTA 0 only)
+  pdl_launch_dependents();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int grp = lane / LPR, li = lane % LPR;
+  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.NH / p.NKV);
+  const int t = *p.pos;   // a graph input: nothing in this run writes it
+  pdl_wait();
+  if (t < 0 || t >= p.Tmax) {   // the same in every CTA: nobody reaches the cluster barrier
+    if (threadIdx.x == 0 && split == 0 && h == 0 && b == 0) atomicOr(p.status, 0x10u);
+    return;
+  }
+  const int n = t + 1;
+  const int chunk = ((n + kSplits - 1) / kSplits + RPI - 1) / RPI * RPI;
+  const int r0 = split * chunk, r1 = min(n, r0 + chunk);
+
+  float qv[V];
+  {
+    const uint4 raw = *reinterpret_cast<const uint4*>(static_cast<const T*>(p.q) + b * p.q_sb + h * p.q_sh + li * V);
+    unpack16<T>(raw, qv);
+#pragma unroll
+    for (int i = 0; i < V; ++i) qv[i] *= p.scale_log2;
+  }
+  const T* k_new = static_cast<const T*>(p.k) + b * p.k_sb + g * p.k_sh + li * V;
+  const T* v_new = static_cast<const T*>(p.v) + b * p.v_sb + g * p.v_sh + li * V;
+  const int64_t row_stride = (int64_t)p.NKV * D;
+  T* kc = static_cast<T*>(p.kc) + ((int64_t)b * p.Tmax * p.NKV + g) * D + li * V;
+  T* vc = static_cast<T*>(p.vc) + ((int64_t)b * p.Tmax * p.NKV + g) * D + li * V;
+
+  float m = -INFINITY, l = 0.f, o[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) o[i] = 0.f;
+
+  // the loop bound is the warp's, not the lane group's: every lane takes part in the shuffles of every pass, a
+  // group whose rows are all past the end carries -inf scores through it
+#pragma unroll 1
+  for (int wbase = r0 + warp * GPW; wbase < r1; wbase += RPI * kInFlight) {
+    const int base = wbase + grp;
+    uint4 kr[kInFlight], vr[kInFlight];
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) {
+      const int j = base + u * RPI;
+      if (j < r1) {
+        const bool fresh = j == t;
+        kr[u] = *reinterpret_cast<const uint4*>(fresh ? k_new : kc + j * row_stride);
+        vr[u] = *reinterpret_cast<const uint4*>(fresh ? v_new : vc + j * row_stride);
+      }
+    }
+    float s[kInFlight], mb = -INFINITY;
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) {
+      const int j = base + u * RPI;
+      s[u] = -INFINITY;
+      if (j < r1) {
+        float kf[V];
+        unpack16<T>(kr[u], kf);
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < V; ++i) acc = fmaf(qv[i], kf[i], acc);
+        s[u] = acc;
+        if (j == t) {   // the new token's key and value take their row of the caches
+          *reinterpret_cast<uint4*>(kc + j * row_stride) = kr[u];
+          *reinterpret_cast<uint4*>(vc + j * row_stride) = vr[u];
+        }
+      }
+    }
+    // the lanes of a group hold partial dot products of the same rows; j < r1 is uniform inside a group, and the
+    // exchange stays inside it (LPR is a power of two, groups are aligned)
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) {
+#pragma unroll
+      for (int off = LPR / 2; off > 0; off >>= 1) s[u] += __shfl_xor_sync(0xffffffffu, s[u], off);
+      mb = fmaxf(mb, s[u]);
+    }
+    const float m_new = fmaxf(m, mb);
+    const float corr = merge_weight(m, m_new);
+    l *= corr;
+#pragma unroll
+    for (int i = 0; i < V; ++i) o[i] *= corr;
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) {
+      if (base + u * RPI < r1) {
+        const float e = exp2f(s[u] - m_new);   // the row exists, so m_new is finite
+        float vf[V];
+        unpack16<T>(vr[u], vf);
+        l += e;
+#pragma unroll
+        for (int i = 0; i < V; ++i) o[i] = fmaf(e, vf[i], o[i]);
+      }
+    }
+    m = m_new;
+  }
+
+  // lane groups of a warp -> one triple per warp
+#pragma unroll
+  for (int off = LPR; off < 32; off <<= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+    const float l2 = __shfl_xor_sync(0xffffffffu, l, off);
+    const float M = fmaxf(m, m2);
+    const float a = merge_weight(m, M), a2 = merge_weight(m2, M);
+    l = l * a + l2 * a2;
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      const float o2 = __shfl_xor_sync(0xffffffffu, o[i], off);
+      o[i] = o[i] * a + o2 * a2;
+    }
+    m = M;
+  }
+  if (grp == 0) {
+#pragma unroll
+    for (int i = 0; i < V; ++i) part[warp][li * V + i] = o[i];
+    if (li == 0) {
+      part[warp][D] = m;
+      part[warp][D + 1] = l;
+    }
+  }
+  __syncthreads();
+  // warps -> one triple per CTA, stored into CTA 0's table
+  if (threadIdx.x < D + 2) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, part[w][D]);
+    float val;
+    if (threadIdx.x == D) {
+      val = M;
+    } else {
+      const int col = threadIdx.x < D ? threadIdx.x : D + 1;
+      val = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) val = fmaf(merge_weight(part[w][D], M), part[w][col], val);
+    }
+    st_cluster_f32(map_to_cta(smem_addr(&cl[split][threadIdx.x]), 0u), val);
+  }
+  cluster_sync_all();
+  if (split != 0) return;
+  if (threadIdx.x < D) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int r = 0; r < kSplits; ++r) M = fmaxf(M, cl[r][D]);
+    float acc = 0.f, L = 0.f;
+#pragma unroll
+    for (int r = 0; r < kSplits; ++r) {
+      const float a = merge_weight(cl[r][D], M);
+      acc = fmaf(a, cl[r][threadIdx.x], acc);
+      L = fmaf(a, cl[r][D + 1], L);
+    }
+    static_cast<T*>(p.out)[b * p.o_sb + h * p.o_sh + threadIdx.x] = from_f<T>(acc / L);
+  }
+}
+
+template <typename T, int LPR>
+cudaError_t launch_one(const AttnDecodeParams& p, cudaStream_t st) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(kSplits, (unsigned)p.NH, (unsigned)p.B);
+  cfg.blockDim = dim3(kWarps * 32);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kSplits;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, attn_decode_kernel<T, LPR>, p);
+}
+
+template <typename T>
+cudaError_t launch_t(const AttnDecodeParams& p, cudaStream_t st) {
+  switch (p.D / VecOf<T>::N) {
+    case 1: return launch_one<T, 1>(p, st);
+    case 2: return launch_one<T, 2>(p, st);
+    case 4: return launch_one<T, 4>(p, st);
+    case 8: return launch_one<T, 8>(p, st);
+    case 16: return launch_one<T, 16>(p, st);
+    case 32:
+      if constexpr (sizeof(T) == 4) return launch_one<T, 32>(p, st);
+      break;
+  }
+  return cudaErrorInvalidValue;
+}
+
+inline bool al16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; }
+
+}  // namespace
+
+bool attn_decode_supported(int dtype, int D) {
+  if (dtype != FLUID_BF16 && dtype != FLUID_F32) return false;
+  const int v = dtype == FLUID_BF16 ? 8 : 4;
+  if (D % v) return false;
+  const int lpr = D / v;
+  return D <= 128 && lpr >= 1 && lpr <= 32 && (lpr & (lpr - 1)) == 0;   // the merge steps use one thread per output column
+}
+
+cudaError_t launch_attn_decode(const AttnDecodeParams& p, cudaStream_t st) {
+  if (!attn_decode_supported(p.dtype, p.D) || p.NKV < 1 || p.NH % p.NKV || p.B < 1 || p.B > 65535 || p.NH > 65535)
+    return cudaErrorInvalidValue;
+  const int v = p.dtype == FLUID_BF16 ? 8 : 4;
+  const int64_t strides[8] = {p.q_sb, p.q_sh, p.k_sb, p.k_sh, p.v_sb, p.v_sh, p.o_sb, p.o_sh};
+  for (int i = 0; i < 6; ++i)
+    if (strides[i] % v) return cudaErrorInvalidValue;
+  if (!al16(p.q) || !al16(p.k) || !al16(p.v) || !al16(p.kc) || !al16(p.vc)) return cudaErrorInvalidValue;
+  return p.dtype == FLUID_BF16 ? launch_t<__nv_bfloat16>(p, st) : launch_t<float>(p, st);
+}
+
+}  // namespace fluid

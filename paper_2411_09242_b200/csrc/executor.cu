@@ -183,7 +183,7 @@ int finalize_steps(fluid_plan_s* p) {
         q.base = (float)n.rope_base;
         q.interleaved = n.rope_interleaved;
         s.rope = q;
-        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out; s.t_narrow[0] = 1;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.out; s.t_ptr[2] = n.pos; s.t_narrow[0] = 1;
         s.bytes = es * ty.numel() * 2.0;
         break;
       }
@@ -238,6 +238,27 @@ int finalize_steps(fluid_plan_s* p) {
         s.bytes = es * (double(T[n.a].numel()) + T[n.b].numel() + T[n.v].numel() + ty.numel());
         break;
       }
+      case N_ATTN_DECODE: {
+        s.kernel = FLUID_K_ATTN_DECODE;
+        AttnDecodeParams q{};
+        const TensorDesc &tq = T[n.a], &tk = T[n.b], &tc = T[n.kc];
+        q.dtype = ty.dtype;
+        q.B = (int)tq.dims[0]; q.NH = (int)tq.dims[2]; q.NKV = (int)tk.dims[2]; q.D = (int)tq.dims[3]; q.Tmax = (int)tc.dims[1];
+        q.scale_log2 = (float)(n.scale * 1.4426950408889634);
+        int64_t st[FLUID_MAX_RANK];
+        perm_strides(p, n.a, st);   q.q_sb = st[0]; q.q_sh = st[2];
+        perm_strides(p, n.b, st);   q.k_sb = st[0]; q.k_sh = st[2];
+        perm_strides(p, n.v, st);   q.v_sb = st[0]; q.v_sh = st[2];
+        perm_strides(p, n.out, st); q.o_sb = st[0]; q.o_sh = st[2];
+        s.attn_dec = q;
+        s.variant = q.D | (q.NH / q.NKV) << 8;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.v; s.t_ptr[3] = n.kc; s.t_ptr[4] = n.vc; s.t_ptr[5] = n.pos;
+        s.t_ptr[6] = n.out;
+        // figures for a full cache; a run reads pos + 1 of its Tmax rows
+        s.flops = 4.0 * q.B * q.NH * double(q.Tmax) * q.D;
+        s.bytes = es * (double(T[n.kc].numel()) + T[n.vc].numel() + 2.0 * tq.numel() + 2.0 * tk.numel());
+        break;
+      }
       case N_SELECT: {
         s.kernel = FLUID_K_SELECT_LAST;
         const TensorDesc& tx = T[n.a];
@@ -280,7 +301,8 @@ struct Resolver {
     }
     const TensorDesc& td = p->graph.tensors[r];
     switch (td.kind) {
-      case FLUID_INPUT: return inputs[p->input_slot[r]];
+      case FLUID_INPUT:
+      case FLUID_STATE: return inputs[p->input_slot[r]];
       case FLUID_OUTPUT: return outputs[p->output_slot[r]];
       case FLUID_CONST:
         if (!p->const_ptr[r]) {
@@ -321,7 +343,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
   key.push_back(arena_ptr);
   for (int t = 0; t < (int)T.size(); ++t) {
     const void* q = nullptr;
-    if (T[t].kind == FLUID_INPUT) {
+    if (T[t].kind == FLUID_INPUT || T[t].kind == FLUID_STATE) {
       if (!inputs || !(q = inputs[p->input_slot[t]])) { set_error("input %d is null", p->input_slot[t]); return FLUID_EINVAL; }
     } else if (T[t].kind == FLUID_OUTPUT) {
       if (!outputs || !(q = outputs[p->output_slot[t]])) { set_error("output %d is null", p->output_slot[t]); return FLUID_EINVAL; }
@@ -454,7 +476,18 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       case FLUID_K_ROPE: {
         RopeParams q = s.rope;
         q.x = R(s.t_ptr[0], 1); q.y = const_cast<void*>(R(s.t_ptr[1]));
+        q.pos = static_cast<const int*>(R(s.t_ptr[2]));
         if (R.ok) err = launch_rope(q, stream);
+        break;
+      }
+      case FLUID_K_ATTN_DECODE: {
+        AttnDecodeParams q = s.attn_dec;
+        q.q = R(s.t_ptr[0], 1); q.k = R(s.t_ptr[1], 1); q.v = R(s.t_ptr[2], 1);
+        q.kc = const_cast<void*>(R(s.t_ptr[3])); q.vc = const_cast<void*>(R(s.t_ptr[4]));
+        q.pos = static_cast<const int*>(R(s.t_ptr[5]));
+        q.out = const_cast<void*>(R(s.t_ptr[6]));
+        q.status = status;
+        if (R.ok) err = launch_attn_decode(q, stream);
         break;
       }
       case FLUID_K_ELTWISE: {
@@ -565,6 +598,10 @@ int fluid_status(const fluid_plan_t* plan, const void* arena_ptr, fluid_stream s
     return FLUID_ECUDA;
   }
   *device_status = (int)word;
+  if (word & 0x10u) {
+    set_error("CACHED_ATTENTION: the position read on the device lies outside the cache (status 0x%x)", word);
+    return FLUID_EINVAL;
+  }
   if (word != 0) {
     set_error("a device-side wait expired (code 0x%x)", word);
     return FLUID_ETIMEOUT;

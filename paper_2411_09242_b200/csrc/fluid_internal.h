@@ -50,7 +50,7 @@ inline void strides_of(const TensorDesc& t, const Perm& perm, int64_t* st) {
 }
 
 // A planning node: one graph op, or several folded into one kernel step.
-enum NodeKind { N_EMBED, N_GEMM, N_NORM, N_SOFTMAX, N_ROPE, N_ELTWISE, N_TRANSPOSE, N_SELECT, N_ATTN };
+enum NodeKind { N_EMBED, N_GEMM, N_NORM, N_SOFTMAX, N_ROPE, N_ELTWISE, N_TRANSPOSE, N_SELECT, N_ATTN, N_ATTN_DECODE };
 enum GemmKind { G_LINEAR, G_QK, G_PV };
 
 struct Node {
@@ -58,7 +58,7 @@ struct Node {
   std::vector<int> ops;        // graph op ids folded into this node, first = anchor
   std::vector<int> ins, outs;  // distinct external tensors, inputs in role order
   // role-tagged tensor ids (-1 = absent)
-  int a = -1, b = -1, bias = -1, res = -1, out = -1, gamma = -1, beta = -1, pos = -1, v = -1;
+  int a = -1, b = -1, bias = -1, res = -1, out = -1, gamma = -1, beta = -1, pos = -1, v = -1, kc = -1, vc = -1;
   int gemm_kind = G_LINEAR, contract = 1, act = ACT_NONE, causal = CAUSAL_NONE;
   double scale = 1.0, eps = 1e-5, rope_base = 10000.0;
   int elt = ELT_ADD, rms = 0, rope_interleaved = 0, sm_causal = 0;
@@ -92,6 +92,7 @@ struct Step {
   EmbedParams embed{};
   AttnParams attn{};
   AttnHost attn_host{};
+  AttnDecodeParams attn_dec{};
   // tensor ids whose device addresses fill the payload's pointer slots
   int t_ptr[8] = {-1, -1, -1, -1, -1, -1, -1, -1};
   int t_narrow[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // 1: bind the bf16 twin of an fp32-held tensor

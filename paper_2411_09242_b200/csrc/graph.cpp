@@ -34,6 +34,11 @@ static int check_op(const fluid_graph_s* g, const OpDesc& op) {
   const TensorDesc& y = T(op.outs[0]);
   if (!need(y.kind == FLUID_ACT || y.kind == FLUID_OUTPUT, "an op may only write ACT or OUTPUT tensors"))
     return FLUID_EINVAL;
+  for (int i = 0; i < ni; ++i)
+    if (T(op.ins[i]).kind == FLUID_STATE && !(op.kind == FLUID_OP_CACHED_ATTENTION && (i == 3 || i == 4))) {
+      need(false, "a STATE tensor is read only as the cache of a CACHED_ATTENTION op");
+      return FLUID_EINVAL;
+    }
   switch (op.kind) {
     case FLUID_OP_EMBED: {
       if (!need(ni == 2 || ni == 3, "EMBED takes ids, table [, positions]")) return FLUID_EINVAL;
@@ -96,11 +101,36 @@ static int check_op(const fluid_graph_s* g, const OpDesc& op) {
       break;
     }
     case FLUID_OP_ROPE:
-      if (!need(ni == 1 && y.rank == 4 && same_dims(T(op.ins[0]), y) && T(op.ins[0]).dtype == y.dtype &&
+      if (!need((ni == 1 || ni == 2) && y.rank == 4 && same_dims(T(op.ins[0]), y) && T(op.ins[0]).dtype == y.dtype &&
                     y.dims[3] % 2 == 0 && y.dtype != FLUID_I32,
                 "ROPE wants x[B,S,nh,D] with even D"))
         return FLUID_EINVAL;
+      if (ni == 2 && !need(T(op.ins[1]).dtype == FLUID_I32 && T(op.ins[1]).rank == 1 && T(op.ins[1]).dims[0] == 1 &&
+                               T(op.ins[1]).kind == FLUID_INPUT,
+                           "ROPE's position offset is an int32 [1] graph input"))
+        return FLUID_EINVAL;
       break;
+    case FLUID_OP_CACHED_ATTENTION: {
+      bool ok = ni == 6;
+      if (ok) {
+        const TensorDesc &q = T(op.ins[0]), &k = T(op.ins[1]), &v = T(op.ins[2]), &kc = T(op.ins[3]), &vc = T(op.ins[4]),
+                         &pos = T(op.ins[5]);
+        ok = q.rank == 4 && same_dims(q, y) && q.dims[1] == 1 && k.rank == 4 && same_dims(k, v) && k.dims[0] == q.dims[0] &&
+             k.dims[1] == 1 && k.dims[3] == q.dims[3] && q.dims[2] % k.dims[2] == 0 && kc.rank == 4 && same_dims(kc, vc) &&
+             kc.dims[0] == q.dims[0] && kc.dims[2] == k.dims[2] && kc.dims[3] == q.dims[3] && kc.kind == FLUID_STATE &&
+             vc.kind == FLUID_STATE && op.ins[3] != op.ins[4] && pos.dtype == FLUID_I32 && pos.rank == 1 && pos.dims[0] == 1 &&
+             pos.kind == FLUID_INPUT && y.dtype != FLUID_I32 && q.dtype == y.dtype && k.dtype == y.dtype &&
+             v.dtype == y.dtype && kc.dtype == y.dtype && vc.dtype == y.dtype;
+      }
+      if (!need(ok, "CACHED_ATTENTION wants q[B,1,nh,D], k, v[B,1,nkv,D], two STATE caches [B,Tmax,nkv,D], pos i32[1]"))
+        return FLUID_EINVAL;
+      for (const OpDesc& o : g->ops)
+        if (o.kind == FLUID_OP_CACHED_ATTENTION)
+          for (int s = 3; s <= 4; ++s)
+            if (!need(o.ins[3] != op.ins[s] && o.ins[4] != op.ins[s], "a cache belongs to one CACHED_ATTENTION op"))
+              return FLUID_EINVAL;
+      break;
+    }
     case FLUID_OP_TRANSPOSE: {
       const TensorDesc& x = T(op.ins.empty() ? op.outs[0] : op.ins[0]);
       bool ok = ni == 1 && x.rank == y.rank && x.dtype == y.dtype;
@@ -176,7 +206,7 @@ int fluid_graph_add_tensor(fluid_graph_t* g, int dtype, int rank, const int64_t*
     set_error("null argument");
     return FLUID_EINVAL;
   }
-  if (dtype < FLUID_F32 || dtype > FLUID_I32 || kind < FLUID_INPUT || kind > FLUID_ACT || rank < 1 ||
+  if (dtype < FLUID_F32 || dtype > FLUID_I32 || kind < FLUID_INPUT || kind > FLUID_STATE || rank < 1 ||
       rank > FLUID_MAX_RANK) {
     set_error("bad dtype/kind/rank (%d/%d/%d)", dtype, kind, rank);
     return FLUID_EINVAL;
@@ -209,7 +239,7 @@ int fluid_graph_add_op(fluid_graph_t* g, int op_kind, int n_in, const int* in_id
     set_error("null argument");
     return FLUID_EINVAL;
   }
-  if (op_kind < 0 || op_kind >= FLUID_OP_COUNT || n_in < 1 || n_in > 4 || n_out != 1) {
+  if (op_kind < 0 || op_kind >= FLUID_OP_COUNT || n_in < 1 || n_in > 6 || n_out != 1) {
     set_error("bad op kind or arity (%d, %d in, %d out)", op_kind, n_in, n_out);
     return FLUID_EINVAL;
   }

@@ -108,6 +108,7 @@ struct RopeParams {
   int order[4];       // logical dims, slowest to fastest, in memory
   float base;
   int interleaved;
+  const int* pos;     // device: position of row 0 (null = 0)
 };
 
 struct EltParams {
@@ -156,6 +157,22 @@ struct AttnParams {
   int q_sel[5], k_sel[5], v_sel[5];   // tensor-map coordinate feeds: 0 contraction, 2 row, 4 / 5 batch split, 6 zero
   int q_b0, k_b0, v_b0;               // inner extent of each operand's (batch * head) index split
 };
+
+// One decoding step against a key/value cache [B, Tmax, NKV, D] (canonical, caller-owned): the new key and
+// value become row t = *pos of the caches, the query attends over rows 0..t.
+struct AttnDecodeParams {
+  int dtype;
+  const void *q, *k, *v;  // [B,1,NH,D], [B,1,NKV,D] x 2: d contiguous, strides below
+  void *kc, *vc;
+  const int* pos;         // device
+  void* out;              // [B,1,NH,D]
+  uint32_t* status;
+  int B, NH, NKV, D, Tmax;
+  float scale_log2;       // scale * log2(e)
+  int64_t q_sb, q_sh, k_sb, k_sh, v_sb, v_sh, o_sb, o_sh;   // element strides of batch and head
+};
+cudaError_t launch_attn_decode(const AttnDecodeParams& p, cudaStream_t stream);
+bool attn_decode_supported(int dtype, int D);
 
 struct AttnHost {
   int eligible;

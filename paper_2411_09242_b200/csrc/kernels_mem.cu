@@ -525,6 +525,7 @@ __global__ void rope_kernel(RopeParams p, int64_t total) {
   pdl_launch_dependents();
   pdl_wait();
   const int half = p.dims[3] / 2;
+  const int pos0 = p.pos ? *p.pos : 0;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     int idx[4];
     int64_t rem = i;
@@ -540,7 +541,7 @@ __global__ void rope_kernel(RopeParams p, int64_t total) {
     const int64_t base = idx[0] * p.st[0] + idx[1] * p.st[1] + idx[2] * p.st[2];
     const float inv_freq = exp2f(-2.f * pr / p.dims[3] * log2f(p.base));
     float sn, cs;
-    sincosf(idx[1] * inv_freq, &sn, &cs);
+    sincosf((idx[1] + pos0) * inv_freq, &sn, &cs);
     const T* x = static_cast<const T*>(p.x);
     T* y = static_cast<T*>(p.y);
     const float a = to_f(x[base + d0 * p.st[3]]), b = to_f(x[base + d1 * p.st[3]]);
@@ -557,6 +558,7 @@ __global__ void __launch_bounds__(256) rope_vec_kernel(RopeParams p, int64_t tot
   pdl_wait();
   const int D = p.dims[3], half = D / 2, cpr = half / 8;
   const float lb = log2f(p.base);
+  const int pos0 = p.pos ? *p.pos : 0;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     int64_t rem = i;
     const int c = int(rem % cpr); rem /= cpr;
@@ -569,7 +571,7 @@ __global__ void __launch_bounds__(256) rope_vec_kernel(RopeParams p, int64_t tot
       const float inv_freq = exp2f(-2.f * (c * 8 + j) / D * lb);
       // two-step reduction of the angle to [-pi, pi] (exact product k * 2pi_hi in the fused multiply-add), then the
       // hardware sine / cosine, whose absolute error there is about 2^-21
-      const float ang = s * inv_freq;
+      const float ang = (s + pos0) * inv_freq;
       const float k = rintf(ang * 0.15915494309189535f);
       float r = fmaf(-k, 6.2831854820251465f, ang);
       r = fmaf(-k, -1.7484555e-7f, r);

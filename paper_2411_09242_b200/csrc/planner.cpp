@@ -379,6 +379,13 @@ double node_cost(const fluid_plan_s* p, const Node& n, const int* lo) {
     case N_SELECT:
       if (!is_identity(p, n.a, lo) || !is_identity(p, n.out, lo)) return kInf;
       return kLaunch + 2.0 * tbytes(p, n.out) / kBw;
+    case N_ATTN_DECODE: {
+      // q, k, v and the result are [B,1,heads,D] rows: any order of the leading dims, D contiguous
+      for (int t : {n.a, n.b, n.v, n.out})
+        if (perm_of(p, t, lo)[3] != 3) return kInf;
+      if (!attn_decode_supported(T[n.out].dtype, (int)T[n.out].dims[3])) return kInf;
+      return kLaunch + (tbytes(p, n.kc) + tbytes(p, n.vc)) / kBw;   // the whole cache: the row count is a run-time value
+    }
     case N_ATTN: {
       AttnParams ap;
       AttnHost ah;
@@ -607,6 +614,11 @@ static void build_nodes(fluid_plan_s* p, const std::vector<int>& order) {
         break;
       case FLUID_OP_ROPE:
         n.kind = N_ROPE; n.rope_base = op.attrs.rope_base; n.rope_interleaved = op.attrs.rope_interleaved;
+        n.pos = op.ins.size() > 1 ? op.ins[1] : -1;
+        break;
+      case FLUID_OP_CACHED_ATTENTION:
+        n.kind = N_ATTN_DECODE; n.b = op.ins[1]; n.v = op.ins[2]; n.kc = op.ins[3]; n.vc = op.ins[4]; n.pos = op.ins[5];
+        n.scale = op.attrs.scale;
         break;
       case FLUID_OP_TRANSPOSE:
         n.kind = N_TRANSPOSE;
@@ -1194,7 +1206,7 @@ int fluid_plan(const fluid_graph_t* g, const fluid_layout_candidates* cands, con
         return FLUID_EINVAL;
       }
       // the caller's buffers stay canonical whatever the list says
-      if ((td.kind == FLUID_INPUT || td.kind == FLUID_OUTPUT) && c > 0) continue;
+      if ((td.kind == FLUID_INPUT || td.kind == FLUID_OUTPUT || td.kind == FLUID_STATE) && c > 0) continue;
       p->cands[t].push_back(pm);
     }
     if (p->cands[t].empty()) p->cands[t].push_back(identity_perm());
@@ -1205,7 +1217,7 @@ int fluid_plan(const fluid_graph_t* g, const fluid_layout_candidates* cands, con
   p->const_ptr.assign(nt, nullptr);
   int ni = 0, no = 0;
   for (int t = 0; t < nt; ++t) {
-    if (g->tensors[t].kind == FLUID_INPUT) p->input_slot[t] = ni++;
+    if (g->tensors[t].kind == FLUID_INPUT || g->tensors[t].kind == FLUID_STATE) p->input_slot[t] = ni++;
     if (g->tensors[t].kind == FLUID_OUTPUT) p->output_slot[t] = no++;
   }
   std::vector<int> order;

@@ -1,0 +1,136 @@
+"""Parity of the decoding path (key/value cache) on the GPU against the CPU oracle, through the C-ABI."""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2411_09242_b200 import fluid, synth
+from tests import helpers
+
+pytestmark = pytest.mark.gpu
+
+
+def _cached_graph(B, nh, nkv, D, Tmax, dtype):
+    g = synth.GraphDesc()
+    q = g.tensor("q", dtype, [B, 1, nh, D], synth.INPUT)
+    k = g.tensor("k", dtype, [B, 1, nkv, D], synth.INPUT)
+    v = g.tensor("v", dtype, [B, 1, nkv, D], synth.INPUT)
+    kc = g.tensor("kc", dtype, [B, Tmax, nkv, D], synth.STATE)
+    vc = g.tensor("vc", dtype, [B, Tmax, nkv, D], synth.STATE)
+    pos = g.tensor("pos", synth.I32, [1], synth.INPUT)
+    out = g.tensor("ctx", dtype, [B, 1, nh, D], synth.OUTPUT)
+    g.op(synth.CACHED_ATTENTION, [q, k, v, kc, vc, pos], [out], scale=1.0 / math.sqrt(D))
+    return g, (q, k, v, kc, vc, pos, out)
+
+
+@pytest.mark.parametrize("B,nh,nkv,D,Tmax,dtype,ts", [
+    (2, 8, 8, 128, 700, synth.BF16, (0, 1, 5, 127, 128, 255, 256, 699)),
+    (3, 8, 2, 128, 300, synth.BF16, (0, 17, 299)),
+    (2, 12, 12, 64, 1100, synth.BF16, (0, 63, 64, 1023, 1099)),
+    (1, 6, 3, 32, 90, synth.F32, (0, 7, 89)),
+    (2, 4, 4, 8, 40, synth.F32, (0, 3, 39)),
+    (1, 2, 1, 128, 50, synth.F32, (0, 33, 49)),
+])
+def test_cached_attention_step(B, nh, nkv, D, Tmax, dtype, ts):
+    g, (q, k, v, kc, vc, pos, out) = _cached_graph(B, nh, nkv, D, Tmax, dtype)
+    helpers.ensure_lib()
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    assert [s["kernel_name"] for s in plan.steps()] == ["ATTN_DECODE"]
+    runner = fluid.Runner(plan, {}, poison=True)
+    for t in ts:
+        feeds = {q: helpers.rand_feed([B, 1, nh, D], dtype, 10 + t, -2, 2), k: helpers.rand_feed([B, 1, nkv, D], dtype, 20 + t, -2, 2),
+                 v: helpers.rand_feed([B, 1, nkv, D], dtype, 30 + t), kc: helpers.rand_feed([B, Tmax, nkv, D], dtype, 40 + t, -2, 2),
+                 vc: helpers.rand_feed([B, Tmax, nkv, D], dtype, 50 + t), pos: np.array([t], dtype=np.int32)}
+        # rows past t are unspecified: huge values there would wreck the result if they were read
+        dev = {x: a.copy() for x, a in feeds.items()}
+        dev[kc][:, t + 1:] = 32768.0
+        dev[vc][:, t + 1:] = -32768.0
+        runner.set_inputs([dev[x] for x in g.inputs])
+        runner.run()
+        got = runner.outputs_host()[0]
+        assert runner.status() == 0
+        ref = helpers.run_oracle(g, feeds)
+        helpers.assert_close(got, ref[out], dtype, f"ctx t={t}")
+        # caches: row t is the new key / value bit for bit, every other row is untouched
+        kc_dev = runner.inputs[g.inputs.index(kc)].float().cpu().numpy()
+        vc_dev = runner.inputs[g.inputs.index(vc)].float().cpu().numpy()
+        assert np.array_equal(kc_dev[:, t], feeds[k][:, 0]) and np.array_equal(vc_dev[:, t], feeds[v][:, 0])
+        keep = np.ones(Tmax, bool)
+        keep[t] = False
+        assert np.array_equal(kc_dev[:, keep], dev[kc][:, keep]) and np.array_equal(vc_dev[:, keep], dev[vc][:, keep])
+    plan.close()
+
+
+def test_position_outside_the_cache_is_reported_and_nothing_is_written():
+    g, (q, k, v, kc, vc, pos, out) = _cached_graph(1, 4, 4, 64, 32, synth.BF16)
+    helpers.ensure_lib()
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    runner = fluid.Runner(plan, {})
+    for bad in (-1, 32, 1000):
+        feeds = [np.zeros(g.dims(t), np.float32) for t in g.inputs]
+        feeds[g.inputs.index(pos)] = np.array([bad], dtype=np.int32)
+        feeds[g.inputs.index(kc)] += 1.0
+        runner.set_inputs(feeds)
+        runner.run()
+        with pytest.raises(fluid.FluidError):
+            runner.status()
+        assert float(runner.inputs[g.inputs.index(kc)].float().min()) == 1.0
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype,D", [(synth.BF16, 128), (synth.BF16, 64), (synth.F32, 16)])
+def test_rope_with_a_position_read_on_the_device(dtype, D):
+    g = synth.GraphDesc()
+    x = g.tensor("x", dtype, [2, 3, 4, D], synth.INPUT)
+    pos = g.tensor("pos", synth.I32, [1], synth.INPUT)
+    y = g.tensor("y", dtype, [2, 3, 4, D], synth.OUTPUT)
+    g.op(synth.ROPE, [x, pos], [y], rope_base=10000.0, rope_interleaved=0)
+    for p0 in (0, 5, 2047):
+        feeds = {x: helpers.rand_feed([2, 3, 4, D], dtype, 3), pos: np.array([p0], dtype=np.int32)}
+        got, plan, _ = helpers.run_gpu(g, feeds)
+        helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], dtype, f"rope pos {p0}")
+        plan.close()
+
+
+@pytest.mark.parametrize("dtype,kw", [
+    (synth.F32, dict(L=2, H=64, nh=4, F=96, B=2, V=100)),
+    (synth.BF16, dict(L=2, H=256, nh=4, F=384, B=3, V=500)),
+    (synth.BF16, dict(L=1, H=512, nh=4, F=1024, B=1, V=1000)),
+])
+def test_decoding_steps_of_a_small_model(dtype, kw):
+    """Several decoding steps in a row on one plan: the caches the device carries forward are its own; every
+    step's logits are compared with the oracle run on the oracle's own caches."""
+    cfg = synth.scaled(synth.CONFIGS["llama"], dtype=dtype, S=1, **kw)
+    t_max = 24
+    dec = synth.build_decode_model(cfg, t_max)
+    g = dec.graph
+    helpers.ensure_lib()
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    names = [s["kernel_name"] for s in plan.steps()]
+    assert names.count("ATTN_DECODE") == cfg.L
+    runner = fluid.Runner(plan, dec.consts, poison=True)
+    rng = np.random.default_rng(1)
+    state_ids = [t for pair in dec.caches for t in pair]
+    oracle_state = {t: np.zeros(g.dims(t)) for t in state_ids}
+    for t in state_ids:   # the device's unwritten rows hold NaN patterns
+        runner.inputs[g.inputs.index(t)].fill_(float("nan"))
+    for step in range(7):
+        ids = rng.integers(0, cfg.V, size=(cfg.B, 1)).astype(np.int32)
+        feeds = dict(dec.consts)
+        feeds[dec.ids] = ids
+        feeds[dec.pos] = np.array([step], dtype=np.int32)
+        feeds.update(oracle_state)
+        ref = helpers.run_oracle(g, feeds)
+        for t in state_ids:
+            oracle_state[t] = ref[t]
+        runner.inputs[g.inputs.index(dec.ids)].copy_(fluid.to_device(ids, synth.I32, "cuda"))
+        runner.inputs[g.inputs.index(dec.pos)].copy_(fluid.to_device(feeds[dec.pos], synth.I32, "cuda"))
+        runner.run()
+        outs = runner.outputs_host()
+        assert runner.status() == 0
+        for tid, got in zip(g.outputs, outs):
+            helpers.assert_close(got, ref[tid], dtype, f"step {step} {g.tensors[tid]['name']}", tol=2e-2 if dtype == synth.BF16 else None)
+        for t in state_ids:
+            dev = runner.inputs[g.inputs.index(t)].float().cpu().numpy()[:, :step + 1]
+            helpers.assert_close(dev, oracle_state[t][:, :step + 1], dtype, f"step {step} cache")
+    plan.close()
