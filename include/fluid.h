@@ -146,7 +146,7 @@ typedef struct fluid_plan_options {
 typedef enum {
   FLUID_K_EMBED = 0, FLUID_K_NORM = 1, FLUID_K_GEMM_SIMT = 2, FLUID_K_GEMM_TC = 3,
   FLUID_K_SOFTMAX = 4, FLUID_K_ROPE = 5, FLUID_K_ELTWISE = 6, FLUID_K_PERMUTE = 7,
-  FLUID_K_SELECT_LAST = 8, FLUID_K_ATTN = 9, FLUID_K_ATTN_DECODE = 10, FLUID_K_COUNT = 11
+  FLUID_K_SELECT_LAST = 8, FLUID_K_ATTN = 9, FLUID_K_ATTN_DECODE = 10, FLUID_K_GEMM_ROWS = 11, FLUID_K_COUNT = 12
 } fluid_kernel_id;
 
 typedef struct fluid_step_info {

@@ -24,9 +24,8 @@ namespace fluid {
 
 namespace {
 
-constexpr int kSplits = 8;    // CTAs per cluster = row ranges per (sequence, head)
+constexpr int kSplits = 8;    // most CTAs per cluster = row ranges per (sequence, head); a launch uses 1, 2, 4 or 8
 constexpr int kWarps = 8;
-constexpr int kInFlight = 4;  // rows of K and of V a lane group holds before it consumes them
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
@@ -60,7 +59,37 @@ __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4& q, float (&
 // weight of a partial with maximum m inside a merge whose maximum is M (an empty partial has m = -inf)
 __device__ __forceinline__ float merge_weight(float m, float M) { return m == -INFINITY ? 0.f : exp2f(m - M); }
 
-template <typename T, int LPR>
+template <typename T>
+__device__ __forceinline__ uint4 pack16(const float (&v)[VecOf<T>::N]);
+template <>
+__device__ __forceinline__ uint4 pack16<float>(const float (&v)[4]) {
+  return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+}
+template <>
+__device__ __forceinline__ uint4 pack16<__nv_bfloat16>(const float (&v)[8]) {
+  return make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+}
+
+// Rotary embedding (pairs (d, d + D/2)) of one row of D = LPR * V elements spread over LPR adjacent lanes, lane li
+// holding elements li*V .. li*V + V-1, at position pos. Every lane of the warp must call it.
+template <int V, int LPR>
+__device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, float log2_base) {
+  constexpr int D = LPR * V, half = D / 2;
+  float partner[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) partner[i] = LPR > 1 ? __shfl_xor_sync(0xffffffffu, x[i], LPR / 2) : x[(i + V / 2) % V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    const int d = li * V + i;
+    const int dd = d < half ? d : d - half;
+    const float inv_freq = exp2f(-2.f * dd / D * log2_base);
+    float sn, cs;
+    sincosf(pos * inv_freq, &sn, &cs);
+    x[i] = d < half ? x[i] * cs - partner[i] * sn : x[i] * cs + partner[i] * sn;
+  }
+}
+
+template <typename T, int LPR, int kInFlight>
 __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodeParams p) {
   constexpr int V = VecOf<T>::N;
   constexpr int D = LPR * V;
@@ -71,7 +100,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
   pdl_launch_dependents();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = lane / LPR, li = lane % LPR;
-  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int split = blockIdx.x, n_split = gridDim.x, h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.NH / p.NKV);
   const int t = *p.pos;   // a graph input: nothing in this run writes it
   pdl_wait();
@@ -80,18 +109,26 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
     return;
   }
   const int n = t + 1;
-  const int chunk = ((n + kSplits - 1) / kSplits + RPI - 1) / RPI * RPI;
+  const int chunk = ((n + n_split - 1) / n_split + RPI - 1) / RPI * RPI;
   const int r0 = split * chunk, r1 = min(n, r0 + chunk);
 
   float qv[V];
   {
     const uint4 raw = *reinterpret_cast<const uint4*>(static_cast<const T*>(p.q) + b * p.q_sb + h * p.q_sh + li * V);
     unpack16<T>(raw, qv);
+    if (p.rope) rotate_row<V, LPR>(qv, li, t, p.rope_log2_base);
 #pragma unroll
     for (int i = 0; i < V; ++i) qv[i] *= p.scale_log2;
   }
-  const T* k_new = static_cast<const T*>(p.k) + b * p.k_sb + g * p.k_sh + li * V;
-  const T* v_new = static_cast<const T*>(p.v) + b * p.v_sb + g * p.v_sh + li * V;
+  // the new token's key (rotated here when the step carries the rotary embedding) and value
+  uint4 k_fresh = *reinterpret_cast<const uint4*>(static_cast<const T*>(p.k) + b * p.k_sb + g * p.k_sh + li * V);
+  const uint4 v_fresh = *reinterpret_cast<const uint4*>(static_cast<const T*>(p.v) + b * p.v_sb + g * p.v_sh + li * V);
+  if (p.rope) {
+    float kf[V];
+    unpack16<T>(k_fresh, kf);
+    rotate_row<V, LPR>(kf, li, t, p.rope_log2_base);
+    k_fresh = pack16<T>(kf);   // rounded as the cache will hold it: later steps read exactly what this one used
+  }
   const int64_t row_stride = (int64_t)p.NKV * D;
   T* kc = static_cast<T*>(p.kc) + ((int64_t)b * p.Tmax * p.NKV + g) * D + li * V;
   T* vc = static_cast<T*>(p.vc) + ((int64_t)b * p.Tmax * p.NKV + g) * D + li * V;
@@ -100,40 +137,35 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
 #pragma unroll
   for (int i = 0; i < V; ++i) o[i] = 0.f;
 
-  // the loop bound is the warp's, not the lane group's: every lane takes part in the shuffles of every pass, a
-  // group whose rows are all past the end carries -inf scores through it
+  // rows before t come from the caches. The loop bound is the warp's, not the lane group's: every lane takes part in
+  // the shuffles of every pass, a group whose rows are all past the end carries -inf scores through it
+  const int r1c = min(r1, t);
 #pragma unroll 1
-  for (int wbase = r0 + warp * GPW; wbase < r1; wbase += RPI * kInFlight) {
+  for (int wbase = r0 + warp * GPW; wbase < r1c; wbase += RPI * kInFlight) {
     const int base = wbase + grp;
     uint4 kr[kInFlight], vr[kInFlight];
 #pragma unroll
     for (int u = 0; u < kInFlight; ++u) {
       const int j = base + u * RPI;
-      if (j < r1) {
-        const bool fresh = j == t;
-        kr[u] = *reinterpret_cast<const uint4*>(fresh ? k_new : kc + j * row_stride);
-        vr[u] = *reinterpret_cast<const uint4*>(fresh ? v_new : vc + j * row_stride);
+      if (j < r1c) {
+        kr[u] = *reinterpret_cast<const uint4*>(kc + j * row_stride);
+        vr[u] = *reinterpret_cast<const uint4*>(vc + j * row_stride);
       }
     }
     float s[kInFlight], mb = -INFINITY;
 #pragma unroll
     for (int u = 0; u < kInFlight; ++u) {
-      const int j = base + u * RPI;
       s[u] = -INFINITY;
-      if (j < r1) {
+      if (base + u * RPI < r1c) {
         float kf[V];
         unpack16<T>(kr[u], kf);
         float acc = 0.f;
 #pragma unroll
         for (int i = 0; i < V; ++i) acc = fmaf(qv[i], kf[i], acc);
         s[u] = acc;
-        if (j == t) {   // the new token's key and value take their row of the caches
-          *reinterpret_cast<uint4*>(kc + j * row_stride) = kr[u];
-          *reinterpret_cast<uint4*>(vc + j * row_stride) = vr[u];
-        }
       }
     }
-    // the lanes of a group hold partial dot products of the same rows; j < r1 is uniform inside a group, and the
+    // the lanes of a group hold partial dot products of the same rows; j < r1c is uniform inside a group, and the
     // exchange stays inside it (LPR is a power of two, groups are aligned)
 #pragma unroll
     for (int u = 0; u < kInFlight; ++u) {
@@ -148,7 +180,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
     for (int i = 0; i < V; ++i) o[i] *= corr;
 #pragma unroll
     for (int u = 0; u < kInFlight; ++u) {
-      if (base + u * RPI < r1) {
+      if (base + u * RPI < r1c) {
         const float e = exp2f(s[u] - m_new);   // the row exists, so m_new is finite
         float vf[V];
         unpack16<T>(vr[u], vf);
@@ -158,6 +190,28 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
       }
     }
     m = m_new;
+  }
+  // row t, the new token: from the step's own operands, in the first warp of the CTA whose range holds it; that
+  // warp's first lane group counts it and stores it as row t of the caches
+  if (t >= r0 && t < r1 && warp == 0) {
+    float kf[V], vf[V];
+    unpack16<T>(k_fresh, kf);
+    unpack16<T>(v_fresh, vf);
+    float sc = 0.f;
+#pragma unroll
+    for (int i = 0; i < V; ++i) sc = fmaf(qv[i], kf[i], sc);
+#pragma unroll
+    for (int off = LPR / 2; off > 0; off >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, off);
+    if (grp == 0) {
+      const float m_new = fmaxf(m, sc);
+      const float corr = merge_weight(m, m_new), e = exp2f(sc - m_new);
+      l = l * corr + e;
+#pragma unroll
+      for (int i = 0; i < V; ++i) o[i] = fmaf(e, vf[i], o[i] * corr);
+      m = m_new;
+      *reinterpret_cast<uint4*>(kc + t * row_stride) = k_fresh;
+      *reinterpret_cast<uint4*>(vc + t * row_stride) = v_fresh;
+    }
   }
 
   // lane groups of a warp -> one triple per warp
@@ -205,10 +259,9 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
   if (threadIdx.x < D) {
     float M = -INFINITY;
 #pragma unroll
-    for (int r = 0; r < kSplits; ++r) M = fmaxf(M, cl[r][D]);
+    for (int r = 0; r < n_split; ++r) M = fmaxf(M, cl[r][D]);
     float acc = 0.f, L = 0.f;
-#pragma unroll
-    for (int r = 0; r < kSplits; ++r) {
+    for (int r = 0; r < n_split; ++r) {
       const float a = merge_weight(cl[r][D], M);
       acc = fmaf(a, cl[r][threadIdx.x], acc);
       L = fmaf(a, cl[r][D + 1], L);
@@ -217,23 +270,30 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
   }
 }
 
-template <typename T, int LPR>
-cudaError_t launch_one(const AttnDecodeParams& p, cudaStream_t st) {
+template <typename T, int LPR, int U>
+cudaError_t launch_u(const AttnDecodeParams& p, int splits, cudaStream_t st) {
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(kSplits, (unsigned)p.NH, (unsigned)p.B);
+  cfg.gridDim = dim3((unsigned)splits, (unsigned)p.NH, (unsigned)p.B);
   cfg.blockDim = dim3(kWarps * 32);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = kSplits;
+  attr[0].val.clusterDim.x = (unsigned)splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, attn_decode_kernel<T, LPR>, p);
+  return cudaLaunchKernelEx(&cfg, attn_decode_kernel<T, LPR, U>, p);
+}
+
+template <typename T, int LPR>
+cudaError_t launch_one(const AttnDecodeParams& p, cudaStream_t st) {
+  static const int env_s = [] { const char* e = std::getenv("FLUID_AD_SPLITS"); return e ? atoi(e) : 8; }();
+  static const int env_u = [] { const char* e = std::getenv("FLUID_AD_U"); return e ? atoi(e) : 4; }();
+  return env_u == 8 ? launch_u<T, LPR, 8>(p, env_s, st) : launch_u<T, LPR, 4>(p, env_s, st);
 }
 
 template <typename T>

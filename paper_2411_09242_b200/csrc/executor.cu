@@ -104,6 +104,16 @@ int finalize_steps(fluid_plan_s* p) {
           s.bytes += es * (b + c + (g.has_bias ? g.N : 0));
         }
         if (n_gemm > 1) s.variant |= int(n_gemm) << 20;
+        // a handful of rows: the weight-streaming kernel, when every GEMM of the step has k contiguous on both sides
+        if (p->opts.gemm_path == 0 && s.split_k <= 1 && g.dtype == FLUID_BF16) {
+          bool rows = gemm_rows_eligible(s.gemm);
+          for (size_t gi = 1; gi < n_gemm; ++gi) rows = rows && gemm_rows_eligible(s.gemm_x[gi - 1]);
+          if (rows) {
+            s.kernel = FLUID_K_GEMM_ROWS;
+            s.variant = (n_gemm > 1 ? int(n_gemm) << 20 : 0) | (s.swiglu ? 1 << 29 : 0);
+            break;
+          }
+        }
         if (s.split_k > 1) {
           s.variant |= s.split_k << 24;
         } else if (s.kernel == FLUID_K_GEMM_TC && p->opts.split_k >= 0) {
@@ -245,13 +255,15 @@ int finalize_steps(fluid_plan_s* p) {
         q.dtype = ty.dtype;
         q.B = (int)tq.dims[0]; q.NH = (int)tq.dims[2]; q.NKV = (int)tk.dims[2]; q.D = (int)tq.dims[3]; q.Tmax = (int)tc.dims[1];
         q.scale_log2 = (float)(n.scale * 1.4426950408889634);
+        q.rope = n.rope_fused;
+        q.rope_log2_base = (float)std::log2(n.rope_base);
         int64_t st[FLUID_MAX_RANK];
         perm_strides(p, n.a, st);   q.q_sb = st[0]; q.q_sh = st[2];
         perm_strides(p, n.b, st);   q.k_sb = st[0]; q.k_sh = st[2];
         perm_strides(p, n.v, st);   q.v_sb = st[0]; q.v_sh = st[2];
         perm_strides(p, n.out, st); q.o_sb = st[0]; q.o_sh = st[2];
         s.attn_dec = q;
-        s.variant = q.D | (q.NH / q.NKV) << 8;
+        s.variant = q.D | (q.NH / q.NKV) << 8 | q.rope << 16;
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.v; s.t_ptr[3] = n.kc; s.t_ptr[4] = n.vc; s.t_ptr[5] = n.pos;
         s.t_ptr[6] = n.out;
         // figures for a full cache; a run reads pos + 1 of its Tmax rows
@@ -439,6 +451,21 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
         } else if (R.ok) {
           err = launch_gemm_simt(q, stream);
         }
+        break;
+      }
+      case FLUID_K_GEMM_ROWS: {
+        GemmParams gs[3] = {s.gemm, s.gemm_x[0], s.gemm_x[1]};
+        const int ng = s.swiglu ? 2 : (int)s.nodes.size();
+        gs[0].A = R(s.t_ptr[0], 1); gs[0].B = R(s.t_ptr[1], 1); gs[0].C = const_cast<void*>(R(s.t_ptr[2]));
+        gs[0].bias = R(s.t_ptr[3]); gs[0].R = R(s.t_ptr[4]);
+        for (int gi = 1; gi < ng; ++gi) {
+          gs[gi].A = gs[0].A;
+          gs[gi].B = R(s.x_ptr[gi - 1][0], 1);
+          gs[gi].C = s.swiglu ? gs[0].C : const_cast<void*>(R(s.x_ptr[gi - 1][1]));
+          gs[gi].bias = R(s.x_ptr[gi - 1][2]);
+          gs[gi].R = nullptr;
+        }
+        if (R.ok) err = launch_gemm_rows(gs, ng, stream, s.swiglu);
         break;
       }
       case FLUID_K_ATTN: {

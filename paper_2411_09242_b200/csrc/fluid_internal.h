@@ -61,7 +61,7 @@ struct Node {
   int a = -1, b = -1, bias = -1, res = -1, out = -1, gamma = -1, beta = -1, pos = -1, v = -1, kc = -1, vc = -1;
   int gemm_kind = G_LINEAR, contract = 1, act = ACT_NONE, causal = CAUSAL_NONE;
   double scale = 1.0, eps = 1e-5, rope_base = 10000.0;
-  int elt = ELT_ADD, rms = 0, rope_interleaved = 0, sm_causal = 0;
+  int elt = ELT_ADD, rms = 0, rope_interleaved = 0, sm_causal = 0, rope_fused = 0;
   int perm[8] = {0, 1, 2, 3, 4, 5, 6, 7};
 };
 

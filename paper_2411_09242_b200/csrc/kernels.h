@@ -169,8 +169,15 @@ struct AttnDecodeParams {
   uint32_t* status;
   int B, NH, NKV, D, Tmax;
   float scale_log2;       // scale * log2(e)
+  int rope;               // 1: q and k arrive unrotated; the step applies the rotary embedding (pairs (d, d + D/2)) at position *pos
+  float rope_log2_base;
   int64_t q_sb, q_sh, k_sb, k_sh, v_sb, v_sh, o_sb, o_sh;   // element strides of batch and head
 };
+// GEMM with at most 8 rows and both operands k-contiguous (bf16): the weights stream through registers once.
+// n_group (1..3) sibling GEMMs that share A and the shapes run as one launch. swiglu (two groups: gate, up): the launch
+// writes SiLU(gate) * up to g[0].C and nothing else.
+bool gemm_rows_eligible(const GemmParams& g);
+cudaError_t launch_gemm_rows(const GemmParams* g, int n_group, cudaStream_t stream, int swiglu = 0);
 cudaError_t launch_attn_decode(const AttnDecodeParams& p, cudaStream_t stream);
 bool attn_decode_supported(int dtype, int D);
 

@@ -336,6 +336,8 @@ double node_cost(const fluid_plan_s* p, const Node& n, const int* lo) {
       }
       GemmTcHost tc;
       const double fl = gemm_flops(g), by = gemm_bytes(g);
+      // a handful of rows with k contiguous on both sides: the weight streams through registers once
+      if (p->opts.gemm_path == 0 && gemm_rows_eligible(g)) return kLaunch + 0.95 * by / kBw;
       if (gemm_tc_eligible(p, g, &tc)) {
         const double skew = 1.0 + 0.02 * (tc.cfg.a_mn_major + tc.cfg.b_mn_major);
         // the vector epilogue wants the n index contiguous in C; anything else stores element-wise
@@ -484,6 +486,22 @@ static void build_nodes(fluid_plan_s* p, const std::vector<int>& order) {
     return absorbed[c] ? -1 : c;
   };
   auto available_before = [&](int t, int at_pos) { return producer[t] < 0 || pos[producer[t]] < at_pos; };
+  // the ROPE op producing tensor t, if it can run inside the CACHED_ATTENTION op `att` that consumes t as its query or
+  // key: rotate-half pairing, position taken from the attention's own pos input, no other reader
+  auto rope_into_decode = [&](int t, int att) -> int {
+    const int r = producer[t];
+    if (r < 0 || g.ops[r].kind != FLUID_OP_ROPE || g.tensors[t].kind != FLUID_ACT || consumers[t].size() != 1) return -1;
+    const OpDesc& ro = g.ops[r];
+    if (ro.attrs.rope_interleaved || ro.ins.size() != 2 || ro.ins[1] != g.ops[att].ins[5]) return -1;
+    return r;
+  };
+  // ROPE ops that a later CACHED_ATTENTION takes over produce no node of their own
+  if (fuse)
+    for (int o = 0; o < nops; ++o) {
+      if (g.ops[o].kind != FLUID_OP_CACHED_ATTENTION) continue;
+      const int rq = rope_into_decode(g.ops[o].ins[0], o), rk = rope_into_decode(g.ops[o].ins[1], o);
+      if (rq >= 0 && rk >= 0 && g.ops[rq].attrs.rope_base == g.ops[rk].attrs.rope_base) absorbed[rq] = absorbed[rk] = 1;
+    }
   for (int oi = 0; oi < nops; ++oi) {
     const int o = order[oi];
     if (absorbed[o]) continue;
@@ -616,10 +634,24 @@ static void build_nodes(fluid_plan_s* p, const std::vector<int>& order) {
         n.kind = N_ROPE; n.rope_base = op.attrs.rope_base; n.rope_interleaved = op.attrs.rope_interleaved;
         n.pos = op.ins.size() > 1 ? op.ins[1] : -1;
         break;
-      case FLUID_OP_CACHED_ATTENTION:
+      case FLUID_OP_CACHED_ATTENTION: {
         n.kind = N_ATTN_DECODE; n.b = op.ins[1]; n.v = op.ins[2]; n.kc = op.ins[3]; n.vc = op.ins[4]; n.pos = op.ins[5];
         n.scale = op.attrs.scale;
+        // the rotary embedding of the query and the key at the same position, when both feed nothing else, runs
+        // inside the attention step (the rotated tensors never exist)
+        if (fuse) {
+          const int rq = rope_into_decode(n.a, o), rk = rope_into_decode(n.b, o);
+          if (rq >= 0 && rk >= 0 && g.ops[rq].attrs.rope_base == g.ops[rk].attrs.rope_base) {
+            n.rope_fused = 1;
+            n.rope_base = g.ops[rq].attrs.rope_base;
+            p->folded[n.a] = p->folded[n.b] = 1;
+            n.a = g.ops[rq].ins[0];
+            n.b = g.ops[rk].ins[0];
+            n.ops.push_back(rq); n.ops.push_back(rk);
+          }
+        }
         break;
+      }
       case FLUID_OP_TRANSPOSE:
         n.kind = N_TRANSPOSE;
         for (int i = 0; i < 8; ++i) n.perm[i] = op.attrs.perm[i];
@@ -635,7 +667,7 @@ static void build_nodes(fluid_plan_s* p, const std::vector<int>& order) {
     if (n.ops.size() == 1) {
       for (int t : op.ins) add_in(t);
     } else {
-      add_in(n.a); add_in(n.b); add_in(n.v); add_in(n.bias); add_in(n.res); add_in(n.gamma); add_in(n.beta); add_in(n.pos);
+      add_in(n.a); add_in(n.b); add_in(n.v); add_in(n.bias); add_in(n.res); add_in(n.gamma); add_in(n.beta); add_in(n.kc); add_in(n.vc); add_in(n.pos);
     }
     n.outs.push_back(n.out);
     for (int o2 : n.ops) p->node_of_op[o2] = (int)p->nodes.size();
@@ -1013,7 +1045,11 @@ static int lower_and_place(fluid_plan_s* p) {
       GemmParams g;
       GemmTcHost tc;
       if (!lower_gemm(p, gn, lo, &g) || !gemm_tc_eligible(p, g, &tc)) continue;
-      if (!tc.cfg.pair || g.batch != 1 || g.N % 128 != 0 || g.N0 % 128 != 0 || ((g.M + 127) / 128) % 2 != 0 || g.c_s[5] != 1) continue;
+      GemmParams gu;
+      // a handful of rows: the weight-streaming kernel keeps the same tiles of gate and up in one CTA
+      const bool rows = gemm_rows_eligible(g) && lower_gemm(p, un, lo, &gu) && gemm_rows_eligible(gu);
+      if (!rows && (!tc.cfg.pair || g.batch != 1 || g.N % 128 != 0 || g.N0 % 128 != 0 || ((g.M + 127) / 128) % 2 != 0 || g.c_s[5] != 1))
+        continue;
       st.nodes = {gi, ui, p->steps[si + 1].node};
       st.node = gi;
       st.swiglu = 1;

@@ -24,7 +24,7 @@ LIB_PATH = os.path.join(_HERE, "libfluid.so")
 FLUID_OK = 0
 FLUID_EINVAL, FLUID_EUNSUPPORTED, FLUID_EALIGN, FLUID_ECUDA, FLUID_ENOMEM, FLUID_ETIMEOUT = -1, -2, -3, -4, -5, -6
 ARENA_ALIGN, ARENA_HEADER, SLOT_ALIGN = 1024, 256, 256
-KERNEL_NAMES = ["EMBED", "NORM", "GEMM_SIMT", "GEMM_TC", "SOFTMAX", "ROPE", "ELTWISE", "PERMUTE", "SELECT_LAST", "ATTN", "ATTN_DECODE"]
+KERNEL_NAMES = ["EMBED", "NORM", "GEMM_SIMT", "GEMM_TC", "SOFTMAX", "ROPE", "ELTWISE", "PERMUTE", "SELECT_LAST", "ATTN", "ATTN_DECODE", "GEMM_ROWS"]
 
 
 class FluidError(RuntimeError):

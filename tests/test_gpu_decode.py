@@ -134,3 +134,42 @@ def test_decoding_steps_of_a_small_model(dtype, kw):
             dev = runner.inputs[g.inputs.index(t)].float().cpu().numpy()[:, :step + 1]
             helpers.assert_close(dev, oracle_state[t][:, :step + 1], dtype, f"step {step} cache")
     plan.close()
+
+
+@pytest.mark.parametrize("M,N,K,bias,act,res", [
+    (1, 4096, 4096, False, False, False),
+    (4, 1000, 136, True, True, True),
+    (8, 50, 8, True, False, True),
+    (3, 2304, 768, True, False, False),
+    (5, 97, 1032, False, True, False),
+    (8, 11008, 4096, False, False, True),
+])
+def test_few_row_linear_streams_its_weight(M, N, K, bias, act, res):
+    """LINEAR with at most 8 rows: the weight-streaming kernel, with the fused bias / GELU / residual epilogue."""
+    g = synth.GraphDesc()
+    x = g.tensor("x", synth.BF16, [M, K], synth.INPUT)
+    w = g.tensor("w", synth.BF16, [K, N], synth.CONST)
+    ins = [x, w]
+    feeds = {x: helpers.rand_feed([M, K], synth.BF16, 1), w: synth.round_bf16(synth.normal(7, 1, [K, N], 0.05))}
+    if bias:
+        b = g.tensor("b", synth.BF16, [N], synth.CONST)
+        ins.append(b)
+        feeds[b] = helpers.rand_feed([N], synth.BF16, 2)
+    last = not (act or res)
+    y = g.tensor("y", synth.BF16, [M, N], synth.OUTPUT if last else synth.ACT)
+    g.op(synth.LINEAR, ins, [y], contract=1)
+    if act:
+        a = g.tensor("a", synth.BF16, [M, N], synth.ACT if res else synth.OUTPUT)
+        g.op(synth.GELU, [y], [a], gelu_tanh=0)
+        y = a
+    if res:
+        r = g.tensor("r", synth.BF16, [M, N], synth.INPUT)
+        feeds[r] = helpers.rand_feed([M, N], synth.BF16, 3)
+        o = g.tensor("o", synth.BF16, [M, N], synth.OUTPUT)
+        g.op(synth.ADD, [y, r], [o])
+        y = o
+    got, plan, _ = helpers.run_gpu(g, feeds, synth.default_candidates(g))
+    names = [s["kernel_name"] for s in plan.steps()]
+    assert names[0] == "GEMM_ROWS", names
+    helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], synth.BF16, f"{M}x{N}x{K}")
+    plan.close()
