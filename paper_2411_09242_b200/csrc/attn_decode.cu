@@ -3,11 +3,11 @@
 // The step is bound by reading the cache once: per (sequence, head) t+1 rows of D keys and D values, one
 // multiply-add per byte pair. No tensor cores: rows stream through registers with 16-byte loads.
 //
-// Work split: one thread-block cluster of 8 CTAs per (sequence, query head); CTA r of the cluster takes a
-// contiguous eighth of the rows 0..t. Inside a CTA a row is owned by LPR = D / (16 bytes of elements)
+// Work split: one thread-block cluster of up to 8 CTAs per (sequence, query head); CTA r of the cluster takes a
+// contiguous share of the rows 0..t. Inside a CTA a row is owned by LPR = D / (16 bytes of elements)
 // adjacent lanes (a warp covers 32 / LPR rows per load instruction); every such lane group keeps a running
-// (max, sum, output) triple in the base-2 online-softmax form and has U rows of keys and of values in
-// flight at a time. Triples are merged lane group -> warp (shuffles) -> CTA (shared memory) -> cluster (each
+// (max, sum, output) triple in the base-2 online-softmax form; its rows of keys and values arrive through a
+// per-lane ring of asynchronous copies in shared memory, several rows deep. Triples are merged lane group -> warp (shuffles) -> CTA (shared memory) -> cluster (each
 // CTA stores its triple into CTA 0's shared memory; one cluster barrier), and CTA 0 writes the D outputs.
 // The row of the new token comes from the step's own k and v operands, and the CTA that meets it stores it
 // as row t of the caches: no row is read from the cache in the launch that writes it.
@@ -56,6 +56,21 @@ __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4& q, float (&
   }
 }
 
+constexpr int kStages = 8;    // ring depth: rows of K and of V a lane group has in flight, plus the one being consumed
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool ok) {
+  const int bytes = ok ? 16 : 0;   // 0: the 16 bytes are zero-filled, nothing is read
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");   // past L1: read once
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+
 // weight of a partial with maximum m inside a merge whose maximum is M (an empty partial has m = -inf)
 __device__ __forceinline__ float merge_weight(float m, float M) { return m == -INFINITY ? 0.f : exp2f(m - M); }
 
@@ -83,13 +98,18 @@ __device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, float
     const int d = li * V + i;
     const int dd = d < half ? d : d - half;
     const float inv_freq = exp2f(-2.f * dd / D * log2_base);
-    float sn, cs;
-    sincosf(pos * inv_freq, &sn, &cs);
+    // two-step reduction of the angle to [-pi, pi] (exact product k * 2pi_hi in the fused multiply-add), then the
+    // hardware sine / cosine, whose absolute error there is about 2^-21
+    const float ang = pos * inv_freq;
+    const float kk = rintf(ang * 0.15915494309189535f);
+    float r = fmaf(-kk, 6.2831854820251465f, ang);
+    r = fmaf(-kk, -1.7484555e-7f, r);
+    const float sn = __sinf(r), cs = __cosf(r);
     x[i] = d < half ? x[i] * cs - partner[i] * sn : x[i] * cs + partner[i] * sn;
   }
 }
 
-template <typename T, int LPR, int kInFlight>
+template <typename T, int LPR>
 __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodeParams p) {
   constexpr int V = VecOf<T>::N;
   constexpr int D = LPR * V;
@@ -103,14 +123,40 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
   const int split = blockIdx.x, n_split = gridDim.x, h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.NH / p.NKV);
   const int t = *p.pos;   // a graph input: nothing in this run writes it
+  const bool t_ok = t >= 0 && t < p.Tmax;
+  const int n = t_ok ? t + 1 : 0;
+  const int chunk = ((n + n_split - 1) / n_split + RPI - 1) / RPI * RPI;
+  const int r0 = split * chunk, r1 = min(n, r0 + chunk);
+  const int r1c = min(r1, t);   // rows before t come from the caches
+  const int64_t row_stride = (int64_t)p.NKV * D;
+  T* kc = static_cast<T*>(p.kc) + ((int64_t)b * p.Tmax * p.NKV + g) * D + li * V;
+  T* vc = static_cast<T*>(p.vc) + ((int64_t)b * p.Tmax * p.NKV + g) * D + li * V;
+  // Each lane copies the 16 bytes of K and of V it will consume itself into a private ring in shared memory
+  // (asynchronous copies, kStages deep): it only ever reads back its own copies, so the ring needs no barrier, and the
+  // bytes in flight are set by the ring's depth. The cache rows were written by earlier runs, not by this run's
+  // earlier steps: the first copies are requested before the wait for the previous step.
+  extern __shared__ __align__(16) unsigned char ring_raw[];
+  const uint32_t my_ring = static_cast<uint32_t>(__cvta_generic_to_shared(ring_raw)) + uint32_t(warp) * (kStages * 2 * 32 * 16) + uint32_t(lane) * 16;
+  auto slot = [&](int i, int which) { return my_ring + uint32_t(i % kStages) * (2 * 32 * 16) + uint32_t(which) * (32 * 16); };
+  const int jbase = r0 + warp * GPW + grp;
+  const int n_slots = r0 + warp * GPW < r1c ? (r1c - (r0 + warp * GPW) + RPI - 1) / RPI : 0;
+  auto fill = [&](int i) {
+    const int j = jbase + i * RPI;
+    const bool ok = i < n_slots && j < r1c;
+    const int64_t off = ok ? j * row_stride : 0;   // a zero-filled copy reads nothing, its address stays inside the cache
+    cp_async16(slot(i, 0), kc + off, ok);
+    cp_async16(slot(i, 1), vc + off, ok);
+  };
+  for (int i = 0; i < kStages - 1; ++i) {
+    fill(i);
+    cp_async_commit();
+  }
   pdl_wait();
-  if (t < 0 || t >= p.Tmax) {   // the same in every CTA: nobody reaches the cluster barrier
+  if (!t_ok) {   // the same in every CTA: nobody reaches the cluster barrier
+    cp_async_wait<0>();
     if (threadIdx.x == 0 && split == 0 && h == 0 && b == 0) atomicOr(p.status, 0x10u);
     return;
   }
-  const int n = t + 1;
-  const int chunk = ((n + n_split - 1) / n_split + RPI - 1) / RPI * RPI;
-  const int r0 = split * chunk, r1 = min(n, r0 + chunk);
 
   float qv[V];
   {
@@ -129,68 +175,40 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
     rotate_row<V, LPR>(kf, li, t, p.rope_log2_base);
     k_fresh = pack16<T>(kf);   // rounded as the cache will hold it: later steps read exactly what this one used
   }
-  const int64_t row_stride = (int64_t)p.NKV * D;
-  T* kc = static_cast<T*>(p.kc) + ((int64_t)b * p.Tmax * p.NKV + g) * D + li * V;
-  T* vc = static_cast<T*>(p.vc) + ((int64_t)b * p.Tmax * p.NKV + g) * D + li * V;
 
   float m = -INFINITY, l = 0.f, o[V];
 #pragma unroll
   for (int i = 0; i < V; ++i) o[i] = 0.f;
 
-  // rows before t come from the caches. The loop bound is the warp's, not the lane group's: every lane takes part in
-  // the shuffles of every pass, a group whose rows are all past the end carries -inf scores through it
-  const int r1c = min(r1, t);
+  // rows before t come from the caches, through the ring. The loop bound is the warp's, not the lane group's: every
+  // lane takes part in the shuffles of every pass; a group whose row is past the end contributes nothing
 #pragma unroll 1
-  for (int wbase = r0 + warp * GPW; wbase < r1c; wbase += RPI * kInFlight) {
-    const int base = wbase + grp;
-    uint4 kr[kInFlight], vr[kInFlight];
+  for (int i = 0; i < n_slots; ++i) {
+    cp_async_wait<kStages - 2>();   // this lane's copies of slot i have landed
+    const uint4 kq = lds128(slot(i, 0)), vq = lds128(slot(i, 1));
+    fill(i + kStages - 1);          // refills the slot read one pass ago
+    cp_async_commit();
+    const bool live = jbase + i * RPI < r1c;
+    float kf[V], vf[V];
+    unpack16<T>(kq, kf);
+    unpack16<T>(vq, vf);
+    float sc = 0.f;
 #pragma unroll
-    for (int u = 0; u < kInFlight; ++u) {
-      const int j = base + u * RPI;
-      if (j < r1c) {
-        kr[u] = *reinterpret_cast<const uint4*>(kc + j * row_stride);
-        vr[u] = *reinterpret_cast<const uint4*>(vc + j * row_stride);
-      }
+    for (int e = 0; e < V; ++e) sc = fmaf(qv[e], kf[e], sc);
+    // the lanes of a group hold partial dot products of the same row; the exchange stays inside the group (LPR is a
+    // power of two, groups are aligned)
+#pragma unroll
+    for (int off = LPR / 2; off > 0; off >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, off);
+    if (live) {
+      const float m_new = fmaxf(m, sc);
+      const float corr = merge_weight(m, m_new), e = exp2f(sc - m_new);
+      l = fmaf(l, corr, e);
+#pragma unroll
+      for (int d = 0; d < V; ++d) o[d] = fmaf(e, vf[d], o[d] * corr);
+      m = m_new;
     }
-    float s[kInFlight], mb = -INFINITY;
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u) {
-      s[u] = -INFINITY;
-      if (base + u * RPI < r1c) {
-        float kf[V];
-        unpack16<T>(kr[u], kf);
-        float acc = 0.f;
-#pragma unroll
-        for (int i = 0; i < V; ++i) acc = fmaf(qv[i], kf[i], acc);
-        s[u] = acc;
-      }
-    }
-    // the lanes of a group hold partial dot products of the same rows; j < r1c is uniform inside a group, and the
-    // exchange stays inside it (LPR is a power of two, groups are aligned)
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u) {
-#pragma unroll
-      for (int off = LPR / 2; off > 0; off >>= 1) s[u] += __shfl_xor_sync(0xffffffffu, s[u], off);
-      mb = fmaxf(mb, s[u]);
-    }
-    const float m_new = fmaxf(m, mb);
-    const float corr = merge_weight(m, m_new);
-    l *= corr;
-#pragma unroll
-    for (int i = 0; i < V; ++i) o[i] *= corr;
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u) {
-      if (base + u * RPI < r1c) {
-        const float e = exp2f(s[u] - m_new);   // the row exists, so m_new is finite
-        float vf[V];
-        unpack16<T>(vr[u], vf);
-        l += e;
-#pragma unroll
-        for (int i = 0; i < V; ++i) o[i] = fmaf(e, vf[i], o[i]);
-      }
-    }
-    m = m_new;
   }
+  cp_async_wait<0>();
   // row t, the new token: from the step's own operands, in the first warp of the CTA whose range holds it; that
   // warp's first lane group counts it and stores it as row t of the caches
   if (t >= r0 && t < r1 && warp == 0) {
@@ -270,12 +288,20 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
   }
 }
 
-template <typename T, int LPR, int U>
-cudaError_t launch_u(const AttnDecodeParams& p, int splits, cudaStream_t st) {
+template <typename T, int LPR>
+cudaError_t launch_one(const AttnDecodeParams& p, cudaStream_t st) {
+  constexpr size_t smem = size_t(kWarps) * kStages * 2 * 32 * 16;
+  static const cudaError_t attr_rc = cudaFuncSetAttribute(attn_decode_kernel<T, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (attr_rc != cudaSuccess) return attr_rc;
+  // row ranges per (sequence, head): the fewest that still give every SM about three CTAs
+  int splits = 1;
+  while (splits < kSplits && (int64_t)p.B * p.NH * splits < 148 * 3) splits *= 2;
+  static const int env_s = [] { const char* e = std::getenv("FLUID_AD_SPLITS"); return e ? atoi(e) : 0; }();
+  if (env_s) splits = env_s;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)splits, (unsigned)p.NH, (unsigned)p.B);
   cfg.blockDim = dim3(kWarps * 32);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -286,14 +312,7 @@ cudaError_t launch_u(const AttnDecodeParams& p, int splits, cudaStream_t st) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, attn_decode_kernel<T, LPR, U>, p);
-}
-
-template <typename T, int LPR>
-cudaError_t launch_one(const AttnDecodeParams& p, cudaStream_t st) {
-  static const int env_s = [] { const char* e = std::getenv("FLUID_AD_SPLITS"); return e ? atoi(e) : 8; }();
-  static const int env_u = [] { const char* e = std::getenv("FLUID_AD_U"); return e ? atoi(e) : 4; }();
-  return env_u == 8 ? launch_u<T, LPR, 8>(p, env_s, st) : launch_u<T, LPR, 4>(p, env_s, st);
+  return cudaLaunchKernelEx(&cfg, attn_decode_kernel<T, LPR>, p);
 }
 
 template <typename T>

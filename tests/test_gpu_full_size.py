@@ -118,3 +118,31 @@ def test_sweep_layout_aware_gemm(n, a_major, b_major):
     rows = np.linspace(0, n - 1, 64).astype(int)           # sampled rows, computed exactly
     assert_close(got[g.outputs[0]][rows], A[rows] @ Bm, synth.BF16, f"gemm {n} {a_major}/{b_major}")
     plan.close()
+
+
+@pytest.mark.parametrize("t", [2047, 1000])
+def test_llama_decode_step_full_width(t):
+    """One decoding step at the llama-shaped widths (hidden 4096, 32 heads of 128, FFN 11008, vocabulary 32000), batch 4,
+    caches of 2048 rows filled with random keys and values up to row t (layer count cut to bound host memory)."""
+    cfg = synth.scaled(synth.CONFIGS["llama"], L=1, B=4)
+    dec = synth.build_decode_model(cfg, 2048)
+    g = dec.graph
+    feeds = dict(dec.consts)
+    feeds[dec.ids] = synth.token_ids(synth.TOKEN_SEED, 1, [4, 1], cfg.V)
+    feeds[dec.pos] = np.array([t], dtype=np.int32)
+    for i, (kc, vc) in enumerate(dec.caches):
+        feeds[kc] = synth.round_bf16(synth.uniform(11, 2 * i, g.dims(kc), -2.0, 2.0))
+        feeds[vc] = synth.round_bf16(synth.uniform(11, 2 * i + 1, g.dims(vc), -1.0, 1.0))
+    ref = run_oracle(g, feeds)
+    got, plan, runner = run_gpu(g, feeds, synth.default_candidates(g))
+    names = [s["kernel_name"] for s in plan.steps()]
+    assert names.count("ATTN_DECODE") == 1 and "ROPE" not in names and "GEMM_TC" not in names and names.count("GEMM_ROWS") == 5
+    for tid in g.outputs:
+        assert_close(got[tid], ref[tid], synth.BF16, g.tensors[tid]["name"])
+    for kc, vc in dec.caches:
+        for c in (kc, vc):
+            dev = runner.inputs[g.inputs.index(c)].float().cpu().numpy()
+            assert_close(dev[:, t], ref[c][:, t], synth.BF16, "new cache row")
+            keep = np.arange(2048) != t
+            assert np.array_equal(dev[:, keep], feeds[c][:, keep])
+    plan.close()
