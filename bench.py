@@ -130,6 +130,56 @@ def oracle_sample_config(cfg):
     return synth.scaled(cfg, S=128, L=2), "first 128 positions, 2 of 4 layers"
 
 
+def time_decode(steps, warmup, torch, fluid, peaks, batch=4, t_max=2048):
+    """The second workload: one decoding step of the llama-shaped model (one new token per sequence) against
+    key/value caches holding t_max - 1 earlier tokens (the longest, most expensive step). The step is bound by
+    reading every weight and every cached row once: bytes streamed / time is reported against the copy peak."""
+    cfg = synth.scaled(synth.CONFIGS["llama"], S=1, B=batch)
+    dec = synth.build_decode_model(cfg, t_max)
+    g = dec.graph
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    runner = fluid.Runner(plan, dec.consts)
+    for t in g.inputs:
+        buf = runner.inputs[g.inputs.index(t)]
+        if t == dec.pos:
+            buf.fill_(t_max - 1)
+        elif t == dec.ids:
+            buf.copy_(torch.from_numpy(synth.token_ids(synth.TOKEN_SEED, 1, [batch, 1], cfg.V)))
+        else:
+            buf.uniform_(-1, 1)      # cache contents: values only matter to the parity tests
+    stream = torch.cuda.Stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    with torch.cuda.stream(stream):
+        for _ in range(max(3, warmup)):
+            runner.run(stream)
+        stream.synchronize()
+        assert runner.status() == 0
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            runner.run(torch.cuda.current_stream())
+        ts = []
+        for _ in range(steps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); graph.replay(); b.record(stream)
+            b.synchronize()
+            ts.append(a.elapsed_time(b))
+    es = synth.DTYPE_BYTES[cfg.dtype]
+    # every constant but the embedding table (gathered: batch rows of it) is read once, and so are the cached rows
+    w_bytes = sum(a.size for t, a in dec.consts.items() if g.tensors[t]["name"] != "tok_table") * es + batch * cfg.H * es
+    c_bytes = 2 * cfg.L * batch * t_max * cfg.H * es
+    ms = float(np.mean(ts))
+    info = plan.steps()
+    res = {"workload": "llama_decode", "batch": batch, "cache_rows": t_max, "position": t_max - 1, "layers": cfg.L,
+           "latency_ms": ms, "latency_min_ms": float(np.min(ts)), "tokens_per_s": batch / (ms * 1e-3),
+           "kernel_steps": len(info), "kernels": sorted({s["kernel_name"] for s in info}),
+           "weight_mb": w_bytes / 2 ** 20, "cache_mb": c_bytes / 2 ** 20, "arena_mb": plan.arena_bytes / 2 ** 20,
+           "streamed_gbs": (w_bytes + c_bytes) / (ms * 1e-3) / 1e9,
+           "frac_measured_hbm": (w_bytes + c_bytes) / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    plan.close()
+    return res
+
+
 def run_reference(args, rank):
     """The reference arm: the CPU oracle as it stands, timed on this machine's host cores."""
     if rank != 0:
@@ -367,6 +417,12 @@ def main():
             others.append({k: v for k, v in r.items() if not k.startswith("_")})
         except Exception as e:  # a failed extra workload must not hide the headline number
             others.append({"workload": name, "error": repr(e)[:300]})
+        torch.cuda.empty_cache()
+    if "llama" in args.others.split(","):
+        try:
+            others.append(time_decode(max(5, args.steps // 3), args.warmup, torch, fluid, peaks))
+        except Exception as e:
+            others.append({"workload": "llama_decode", "error": repr(e)[:300]})
         torch.cuda.empty_cache()
     line = {
         "metric": METRIC, "value": latency_ms, "unit": "ms", "n_gpus": world, "steps": args.steps,

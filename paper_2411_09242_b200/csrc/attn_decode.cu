@@ -13,6 +13,8 @@
 // as row t of the caches: no row is read from the cache in the launch that writes it.
 //
 // Nothing here spins: the only waits are __syncthreads and the hardware cluster barrier.
+#include <algorithm>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -24,7 +26,7 @@ namespace fluid {
 
 namespace {
 
-constexpr int kSplits = 8;    // most CTAs per cluster = row ranges per (sequence, head); a launch uses 1, 2, 4 or 8
+constexpr int kSplits = 8;    // most CTAs per cluster = row ranges per (sequence, head); a launch uses 1 to 8
 constexpr int kWarps = 8;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -293,9 +295,10 @@ cudaError_t launch_one(const AttnDecodeParams& p, cudaStream_t st) {
   constexpr size_t smem = size_t(kWarps) * kStages * 2 * 32 * 16;
   static const cudaError_t attr_rc = cudaFuncSetAttribute(attn_decode_kernel<T, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (attr_rc != cudaSuccess) return attr_rc;
-  // row ranges per (sequence, head): the fewest that still give every SM about three CTAs
-  int splits = 1;
-  while (splits < kSplits && (int64_t)p.B * p.NH * splits < 148 * 3) splits *= 2;
+  // row ranges per (sequence, head): as many as still leave the whole launch resident at once (three CTAs fit an SM);
+  // a second, partial wave would run with few bytes in flight
+  const int64_t heads = (int64_t)p.B * p.NH;
+  int splits = (int)std::max<int64_t>(1, std::min<int64_t>(kSplits, (148 * 3) / heads));
   static const int env_s = [] { const char* e = std::getenv("FLUID_AD_SPLITS"); return e ? atoi(e) : 0; }();
   if (env_s) splits = env_s;
   cudaLaunchConfig_t cfg{};
