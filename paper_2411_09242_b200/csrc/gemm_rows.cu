@@ -28,7 +28,10 @@ namespace fluid {
 
 namespace {
 
-constexpr int kWarps = 8;
+// warps of a CTA: the KS warps of one tile (times two with SwiGLU: gate and up), at least two. Small CTAs spread the
+// tiles evenly over the SMs: with eight-warp CTAs a launch of 250 CTAs left a third of the SMs with half the work.
+__host__ __device__ constexpr int rows_warps(int ks, bool swiglu) { return ks * (swiglu ? 2 : 1) < 2 ? 2 : ks * (swiglu ? 2 : 1); }
+constexpr int kWarpsPerSm = 24;   // resident warps an SM's shared memory holds rings for
 
 struct RowsGroup {
   const __nv_bfloat16* W;
@@ -84,7 +87,8 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 // SWIGLU: groups 0 and 1 are the gate and up projections; a CTA holds the same tiles of both (their warps side by
 // side) and writes SiLU(gate) * up to group 0's C, so neither projection is ever stored.
 template <int KS, int LW, int ST, bool SWIGLU>
-__global__ void __launch_bounds__(kWarps * 32) gemm_rows_kernel(RowsParams p, int tiles) {
+__global__ void __launch_bounds__(rows_warps(KS, SWIGLU) * 32) gemm_rows_kernel(RowsParams p, int tiles) {
+  constexpr int kWarps = rows_warps(KS, SWIGLU);
   constexpr int kBlk = 32 * LW, kStages = ST;
   constexpr int kStageBytes = 3 * LW * 32 * 16;
   constexpr int NG = SWIGLU ? 2 : 1;               // groups inside a CTA
@@ -204,6 +208,7 @@ __global__ void __launch_bounds__(kWarps * 32) gemm_rows_kernel(RowsParams p, in
 
 template <int KS, int LW, int ST, bool SWIGLU>
 cudaError_t launch_rows(const RowsParams& p, int tiles, int n_group, cudaStream_t st) {
+  constexpr int kWarps = rows_warps(KS, SWIGLU);
   constexpr size_t smem = size_t(kWarps) * ST * 3 * LW * 32 * 16 + size_t(kWarps) * 16 * 9 * sizeof(float);
   static const cudaError_t attr =
       cudaFuncSetAttribute(gemm_rows_kernel<KS, LW, ST, SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -216,7 +221,8 @@ cudaError_t launch_rows(const RowsParams& p, int tiles, int n_group, cudaStream_
 template <int LW, int ST>
 cudaError_t launch_rows_ks(const RowsParams& p, int tiles, int n_group, int cps, bool swiglu, cudaStream_t st) {
   // as many warps per tile (k slices) as keep the whole launch resident at once
-  const int64_t items = (int64_t)tiles * n_group, cap = 148 * cps * kWarps;
+  const int64_t items = (int64_t)tiles * n_group, cap = 148 * kWarpsPerSm;
+  (void)cps;
   if (swiglu) {
     if (items * 4 <= cap) return launch_rows<4, LW, ST, true>(p, tiles, n_group, st);
     if (items * 2 <= cap) return launch_rows<2, LW, ST, true>(p, tiles, n_group, st);
