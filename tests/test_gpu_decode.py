@@ -173,3 +173,47 @@ def test_few_row_linear_streams_its_weight(M, N, K, bias, act, res):
     assert names[0] == "GEMM_ROWS", names
     helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], synth.BF16, f"{M}x{N}x{K}")
     plan.close()
+
+
+def test_one_captured_graph_serves_every_step_of_a_generation_loop():
+    """The position is read on the device, so a single CUDA-graph capture of fluid_run is replayed for every step while
+    the caller only rewrites the ids and the position buffers: results equal the step-by-step oracle."""
+    import torch
+    cfg = synth.scaled(synth.CONFIGS["llama"], dtype=synth.BF16, S=1, L=2, H=256, nh=4, F=512, B=2, V=300)
+    dec = synth.build_decode_model(cfg, 16)
+    g = dec.graph
+    helpers.ensure_lib()
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    runner = fluid.Runner(plan, dec.consts)
+    state_ids = [t for pair in dec.caches for t in pair]
+    for t in state_ids:
+        runner.inputs[g.inputs.index(t)].zero_()
+    oracle_state = {t: np.zeros(g.dims(t)) for t in state_ids}
+    ids_buf, pos_buf = runner.inputs[g.inputs.index(dec.ids)], runner.inputs[g.inputs.index(dec.pos)]
+    stream = torch.cuda.Stream()
+    rng = np.random.default_rng(5)
+    with torch.cuda.stream(stream):
+        ids_buf.zero_(); pos_buf.zero_()
+        runner.run(stream)                       # warm-up outside the capture (tensor maps, function attributes)
+        for t in state_ids:
+            runner.inputs[g.inputs.index(t)].zero_()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            runner.run(torch.cuda.current_stream())
+        for t in state_ids:                      # the capture itself ran nothing, but start clean all the same
+            runner.inputs[g.inputs.index(t)].zero_()
+        for step in range(10):
+            ids = rng.integers(0, cfg.V, size=(cfg.B, 1)).astype(np.int32)
+            ids_buf.copy_(torch.from_numpy(ids)); pos_buf.fill_(step)
+            graph.replay()
+            stream.synchronize()
+            feeds = dict(dec.consts)
+            feeds[dec.ids], feeds[dec.pos] = ids, np.array([step], dtype=np.int32)
+            feeds.update(oracle_state)
+            ref = helpers.run_oracle(g, feeds)
+            for t in state_ids:
+                oracle_state[t] = ref[t]
+            logits = runner.outputs[1].float().cpu().numpy()
+            helpers.assert_close(logits, ref[g.outputs[1]], synth.BF16, f"replayed step {step}", tol=2e-2)
+    assert runner.status() == 0
+    plan.close()

@@ -296,3 +296,68 @@ def test_a_cost_function_that_picks_unrunnable_layouts_gives_a_plan_that_refuses
         fluid.fluid_run(plan.handle, 0x10000, [0x20000], [0x30000])
     assert e.value.code == fluid.FLUID_EUNSUPPORTED and "no kernel runs" in str(e.value)
     plan.close()
+
+
+def test_decoding_graph_plans_without_a_gpu():
+    """Host logic of the decoding workload: state tensors stay outside the arena and among the inputs, the rotary ops
+    and SwiGLU fold into their consumers, every LINEAR of a few rows takes the weight-streaming kernel."""
+    cfg = synth.scaled(synth.CONFIGS["llama"], S=1, L=2, B=4)
+    dec = synth.build_decode_model(cfg, 2048, materialize=False)
+    g = dec.graph
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    names = [s["kernel_name"] for s in plan.steps()]
+    assert names == ["EMBED"] + ["NORM", "GEMM_ROWS", "ATTN_DECODE", "GEMM_ROWS", "NORM", "GEMM_ROWS", "GEMM_ROWS"] * 2 + ["NORM", "GEMM_ROWS"]
+    att = [s for s in plan.steps() if s["kernel_name"] == "ATTN_DECODE"]
+    assert all(len(s["ops"]) == 3 and (s["variant"] >> 16) & 1 for s in att)            # attention + two ROPE ops
+    fused = [s for s in plan.steps() if s["kernel_name"] == "GEMM_ROWS" and len(s["ops"]) == 4]
+    assert len(fused) == 2 and all(len(s["outs"]) == 1 for s in fused)                   # gate, up, SiLU, MUL
+    for kc, vc in dec.caches:
+        for t in (kc, vc):
+            info = plan.tensor_info(t)
+            assert info.offset < 0 and info.layout_index == 0
+    assert g.inputs == [dec.ids, dec.pos] + [t for pair in dec.caches for t in pair]
+    assert plan.arena_bytes < 2 ** 20                                                     # a few [B,1,.] rows
+    unfused = fluid.Plan(g, synth.default_candidates(g), fusion=0)
+    un = [s["kernel_name"] for s in unfused.steps()]
+    assert un.count("ROPE") == 4 and un.count("ATTN_DECODE") == 2
+    simt = fluid.Plan(g, synth.default_candidates(g), gemm_path=1)
+    assert "GEMM_ROWS" not in [s["kernel_name"] for s in simt.steps()]
+    for p in (plan, unfused, simt):
+        p.close()
+
+
+def test_state_tensors_and_cached_attention_are_checked():
+    def base():
+        g = synth.GraphDesc()
+        q = g.tensor("q", synth.BF16, [2, 1, 4, 64], synth.INPUT)
+        k = g.tensor("k", synth.BF16, [2, 1, 2, 64], synth.INPUT)
+        v = g.tensor("v", synth.BF16, [2, 1, 2, 64], synth.INPUT)
+        kc = g.tensor("kc", synth.BF16, [2, 16, 2, 64], synth.STATE)
+        vc = g.tensor("vc", synth.BF16, [2, 16, 2, 64], synth.STATE)
+        pos = g.tensor("pos", synth.I32, [1], synth.INPUT)
+        out = g.tensor("o", synth.BF16, [2, 1, 4, 64], synth.OUTPUT)
+        return g, [q, k, v, kc, vc, pos], out
+    g, ins, out = base()
+    g.op(synth.CACHED_ATTENTION, ins, [out], scale=0.125)
+    fluid.Plan(g, None).close()
+    # the same cache twice, a cache that is a plain input, a state tensor read by another op, a query of two rows
+    g, ins, out = base()
+    g.op(synth.CACHED_ATTENTION, ins[:4] + [ins[3], ins[5]], [out], scale=0.125)
+    with pytest.raises(fluid.FluidError):
+        fluid.Plan(g, None)
+    g, ins, out = base()
+    g.tensors[ins[3]]["kind"] = synth.INPUT
+    g.op(synth.CACHED_ATTENTION, ins, [out], scale=0.125)
+    with pytest.raises(fluid.FluidError):
+        fluid.Plan(g, None)
+    g, ins, out = base()
+    y = g.tensor("y", synth.BF16, [2, 16, 2, 64], synth.OUTPUT)
+    g.op(synth.GELU, [ins[3]], [y])
+    with pytest.raises(fluid.FluidError):
+        fluid.Plan(g, None)
+    g, ins, out = base()
+    g.tensors[ins[0]]["dims"] = [2, 2, 4, 64]
+    g.tensors[out]["dims"] = [2, 2, 4, 64]
+    g.op(synth.CACHED_ATTENTION, ins, [out], scale=0.125)
+    with pytest.raises(fluid.FluidError):
+        fluid.Plan(g, None)
