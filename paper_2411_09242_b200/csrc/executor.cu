@@ -81,7 +81,7 @@ int finalize_steps(fluid_plan_s* p) {
         s.flops = fl;
         s.bytes = es * (a + b + (g.has_bias ? g.N : 0)) + c * (s.gemm.c_f32 ? 4.0 : es) + (g.has_res ? c * (s.gemm.r_f32 ? 4.0 : es) : 0.0);
         // SwiGLU step: the only tensor written is the product, which takes gate's place
-        const size_t n_gemm = s.swiglu ? 2 : s.nodes.size();
+        const size_t n_gemm = s.swiglu ? 2 : s.nodes.size() - s.norm_fused;
         if (s.swiglu) {
           s.t_ptr[2] = p->nodes[s.nodes[2]].out;
           s.gemm.c_f32 = 0;
@@ -110,9 +110,19 @@ int finalize_steps(fluid_plan_s* p) {
           for (size_t gi = 1; gi < n_gemm; ++gi) rows = rows && gemm_rows_eligible(s.gemm_x[gi - 1]);
           if (rows) {
             s.kernel = FLUID_K_GEMM_ROWS;
-            s.variant = (n_gemm > 1 ? int(n_gemm) << 20 : 0) | (s.swiglu ? 1 << 29 : 0);
+            s.variant = (n_gemm > 1 ? int(n_gemm) << 20 : 0) | (s.swiglu ? 1 << 29 : 0) | (s.norm_fused ? 1 << 30 : 0);
+            if (s.norm_fused) {
+              const Node& nn = p->nodes[s.nodes.back()];
+              s.t_ptr[5] = nn.a; s.t_ptr[6] = nn.gamma;
+              s.norm_eps = (float)nn.eps;
+              s.norm_x_f32 = p->wide[nn.a];
+            }
             break;
           }
+        }
+        if (s.norm_fused) {
+          set_error("step for op %d: the fused normalisation needs the few-row GEMM kernel", n.ops[0]);
+          return FLUID_EUNSUPPORTED;
         }
         if (s.split_k > 1) {
           s.variant |= s.split_k << 24;
@@ -455,8 +465,12 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       }
       case FLUID_K_GEMM_ROWS: {
         GemmParams gs[3] = {s.gemm, s.gemm_x[0], s.gemm_x[1]};
-        const int ng = s.swiglu ? 2 : (int)s.nodes.size();
-        gs[0].A = R(s.t_ptr[0], 1); gs[0].B = R(s.t_ptr[1], 1); gs[0].C = const_cast<void*>(R(s.t_ptr[2]));
+        const int ng = s.swiglu ? 2 : (int)s.nodes.size() - s.norm_fused;
+        RowsNorm rn{};
+        if (s.norm_fused) {
+          rn.x = R(s.t_ptr[5]); rn.gamma = R(s.t_ptr[6]); rn.eps = s.norm_eps; rn.x_f32 = s.norm_x_f32;
+        }
+        gs[0].A = s.norm_fused ? rn.x : R(s.t_ptr[0], 1); gs[0].B = R(s.t_ptr[1], 1); gs[0].C = const_cast<void*>(R(s.t_ptr[2]));
         gs[0].bias = R(s.t_ptr[3]); gs[0].R = R(s.t_ptr[4]);
         for (int gi = 1; gi < ng; ++gi) {
           gs[gi].A = gs[0].A;
@@ -465,7 +479,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
           gs[gi].bias = R(s.x_ptr[gi - 1][2]);
           gs[gi].R = nullptr;
         }
-        if (R.ok) err = launch_gemm_rows(gs, ng, stream, s.swiglu);
+        if (R.ok) err = launch_gemm_rows(gs, ng, stream, s.swiglu, s.norm_fused ? &rn : nullptr);
         break;
       }
       case FLUID_K_ATTN: {

@@ -17,6 +17,8 @@
 // A warp owns 16 weight rows and a slice of the k range; the warps that share a tile add their partial sums
 // through shared memory and the CTA's threads apply bias / activation / residual and store.
 // Sibling projections that share X (Q/K/V, gate/up) run as one launch (blockIdx.y = group).
+#include <algorithm>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -28,10 +30,11 @@ namespace fluid {
 
 namespace {
 
-// warps of a CTA: the KS warps of one tile (times two with SwiGLU: gate and up), at least two. Small CTAs spread the
-// tiles evenly over the SMs: with eight-warp CTAs a launch of 250 CTAs left a third of the SMs with half the work.
-__host__ __device__ constexpr int rows_warps(int ks, bool swiglu) { return ks * (swiglu ? 2 : 1) < 2 ? 2 : ks * (swiglu ? 2 : 1); }
-constexpr int kWarpsPerSm = 24;   // resident warps an SM's shared memory holds rings for
+constexpr int kWarps = 16;         // one CTA per SM: 16 warps, each streaming its own weight rows
+constexpr int kBlk = 32;           // k per pass: 4 lanes x 8 elements per weight row
+constexpr int kXPad = 32;          // bf16 elements of padding per staged activation row (64 bytes: rows g and g + 1 then sit 16
+                                   // banks apart, so the eight lanes of a 16-byte shared load never collide)
+constexpr int kSmemBudget = 227 * 1024 - 1024;
 
 struct RowsGroup {
   const __nv_bfloat16* W;
@@ -44,11 +47,15 @@ struct RowsGroup {
 };
 
 struct RowsParams {
-  const __nv_bfloat16* X;
+  const void* X;           // bf16, or fp32 when x_f32
   int M, N, K, M0, N0;
   int64_t a_s2, a_s3;      // activation row strides of the two-level m index
+  const __nv_bfloat16* gamma;   // fused RMS normalisation: the gain (else null)
+  float eps;
+  int x_f32;
   float scale;
   int w_const;             // the weights are constants of the plan: their first loads need not wait
+  int tiles, units, upc, rounds;   // 16-row weight tiles per group; (group, tile) units in all; units per CTA and round; rounds
   RowsGroup g[3];
 };
 
@@ -64,11 +71,6 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// A warp's work item is (16-row weight tile, k slice): KS warps share a tile, a CTA holds 8 / KS tiles. The weights
-// of a slice go through a per-lane ring in shared memory filled by 16-byte asynchronous copies (a lane only ever
-// reads back what it copied itself, so the ring needs no barrier): the bytes in flight are set by the ring's
-// depth, not by registers.
-
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool ok) {
   const int bytes = ok ? 16 : 0;   // 0: the 16 bytes are zero-filled, nothing is read
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");   // past L1: read once
@@ -82,156 +84,217 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   return v;
 }
 
-// LW = 16-byte pieces a lane takes of each row per stage (a stage covers 32 * LW k: 4 lanes x 8 * LW contiguous
-// elements per row), ST = ring depth.
-// SWIGLU: groups 0 and 1 are the gate and up projections; a CTA holds the same tiles of both (their warps side by
-// side) and writes SiLU(gate) * up to group 0's C, so neither projection is ever stored.
-template <int KS, int LW, int ST, bool SWIGLU>
-__global__ void __launch_bounds__(rows_warps(KS, SWIGLU) * 32) gemm_rows_kernel(RowsParams p, int tiles) {
-  constexpr int kWarps = rows_warps(KS, SWIGLU);
-  constexpr int kBlk = 32 * LW, kStages = ST;
-  constexpr int kStageBytes = 3 * LW * 32 * 16;
+// One CTA per SM. The CTA first stages the activation rows in shared memory, once, as bf16 (with the RMS
+// normalisation's gain multiplied in and the rows' 1/rms computed when the step carries the normalisation): every
+// warp of the GPU reading the same few rows from L2 pass by pass was measured to cost more L2 traffic than the
+// weights themselves and to serialise on the lines everybody wants at once. Then every warp takes work items
+// (16-row weight tile, k slice): KS warps share a tile, the weights of a slice go through a per-lane ring in shared
+// memory filled by 16-byte asynchronous copies (a lane only ever reads back what it copied itself, so the ring needs
+// no barrier; the bytes in flight are set by the ring's depth, not by registers), the activation fragment comes from
+// the staged copy. ST = ring depth. SWIGLU: groups 0 and 1 are the gate and up projections; the same tiles of both
+// sit in neighbouring warps and the CTA writes SiLU(gate) * up to group 0's C, so neither projection is ever stored.
+template <int KS, int ST, bool SWIGLU>
+__global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p) {
   constexpr int NG = SWIGLU ? 2 : 1;               // groups inside a CTA
-  constexpr int TPC = kWarps / (KS * NG);          // tiles per CTA
+  constexpr int UMAX = kWarps / (KS * NG);         // most (group, tile) units per CTA and round
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // ring: [warp][stage][3 = weight row g, weight row g + 8, activation row g][lane] x 16 bytes
-  const uint32_t ring0 = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw));
-  float(*red)[16][9] = reinterpret_cast<float(*)[16][9]>(smem_raw + kWarps * kStages * kStageBytes);   // [warp][row][m]
+  const int pitch = p.K + kXPad;                   // staged activation row, bf16 elements
+  __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);
+  unsigned char* after_x = smem_raw + size_t(p.M) * pitch * 2;
+  const uint32_t ring0 = static_cast<uint32_t>(__cvta_generic_to_shared(after_x));
+  float(*red)[16][9] = reinterpret_cast<float(*)[16][9]>(after_x + kWarps * ST * 1024);   // [warp][row][m]
+  float* rstd = reinterpret_cast<float*>(after_x + kWarps * ST * 1024 + kWarps * 16 * 9 * sizeof(float));   // [8]
+  float* ssq_part = rstd + 8;                                                             // [warp][8]
   pdl_launch_dependents();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int tile = blockIdx.x * TPC + warp / (KS * NG), ks = warp % KS;
-  const RowsGroup& grp = p.g[SWIGLU ? (warp / KS) % 2 : blockIdx.y];
-  const bool tile_live = tile < tiles;
   const int nblk = (p.K + kBlk - 1) / kBlk;
   const int per = (nblk + KS - 1) / KS;
-  const int blk0 = ks * per, blk1 = tile_live ? min(nblk, blk0 + per) : blk0;
-  const int n_base = tile * 16;
-  // weight rows of this lane: g and g + 8 of the tile (rows past N read row N-1 and are dropped at the end)
-  const __nv_bfloat16* wrow[2];
-#pragma unroll
-  for (int hh = 0; hh < 2; ++hh) {
-    const int n = max(0, min(p.N - 1, n_base + hh * 8 + g));
-    wrow[hh] = grp.W + split2(n, p.N0, grp.b_s4, grp.b_s5) + t * 8 * LW;
-  }
+  const int ks = warp % KS;
+  const int blk0 = ks * per;
+  const uint32_t my_ring = ring0 + uint32_t(warp) * (ST * 1024) + uint32_t(lane) * 16;
+  auto slot = [&](int i, int piece) { return my_ring + uint32_t(i % ST) * 1024 + uint32_t(piece) * 512; };
+  const uint32_t xs_lane = static_cast<uint32_t>(__cvta_generic_to_shared(xs)) + uint32_t((g < p.M ? g : 0) * pitch + t * 8) * 2;
   const bool x_live = g < p.M;
-  const __nv_bfloat16* xrow = p.X + (x_live ? split2(g, p.M0, p.a_s2, p.a_s3) : 0) + t * 8 * LW;
-  const uint32_t my_ring = ring0 + uint32_t(warp) * (kStages * kStageBytes) + uint32_t(lane) * 16;
-  auto slot = [&](int blk, int which, int piece) {
-    return my_ring + uint32_t((blk - blk0) % kStages) * kStageBytes + uint32_t(which * LW + piece) * (32 * 16);
-  };
-  auto fill_w = [&](int blk) {
+
+  for (int round = 0; round < p.rounds; ++round) {
+    // units are dealt out evenly: a CTA takes p.upc <= UMAX of them per round, so that every SM streams
+    const int ul = warp / (KS * NG);
+    const int unit = (round * p.upc + ul) * gridDim.x + blockIdx.x;   // strided: CTA c takes units c, c + grid, ...
+    const bool live = ul < p.upc && unit < p.units;
+    const int tile = SWIGLU ? unit : unit % p.tiles;
+    const RowsGroup& grp = p.g[SWIGLU ? (warp / KS) % 2 : (live ? unit / p.tiles : 0)];
+    const int blk1 = live ? min(nblk, blk0 + per) : blk0;
+    const int nloc = max(0, blk1 - blk0);
+    const int n_base = tile * 16;
+    // weight rows of this lane: g and g + 8 of the tile (rows past N read row N-1 and are dropped at the end)
+    const __nv_bfloat16* wrow[2];
 #pragma unroll
-    for (int q = 0; q < LW; ++q) {
-      const int k = blk * kBlk + q * 8;
-      const bool ok = blk < blk1 && k + t * 8 * LW < p.K;   // K is a multiple of 8: a piece is all inside or all outside
+    for (int hh = 0; hh < 2; ++hh) {
+      const int n = max(0, min(p.N - 1, n_base + hh * 8 + g));
+      wrow[hh] = grp.W + split2(n, p.N0, grp.b_s4, grp.b_s5) + t * 8;
+    }
+    auto fill_w = [&](int i) {
+      const int k = (blk0 + i) * kBlk;
+      const bool ok = i < nloc && k + t * 8 < p.K;   // K is a multiple of 8: a piece is all inside or all outside
       const int kk = ok ? k : 0;
-      cp_async16(slot(blk, 0, q), wrow[0] + kk, ok);
-      cp_async16(slot(blk, 1, q), wrow[1] + kk, ok);
+      cp_async16(slot(i, 0), wrow[0] + kk, ok);
+      cp_async16(slot(i, 1), wrow[1] + kk, ok);
+    };
+    // constant weights do not depend on the previous step: the ring fills while the activations are staged
+    if (round > 0 || p.w_const) {
+      for (int i = 0; i < ST - 1; ++i) {
+        fill_w(i);
+        cp_async_commit();
+      }
     }
-  };
-  // the activations ride in the same ring (they come from L2 at best: the ring leaves little L1)
-  auto fill_x = [&](int blk) {
+    if (round == 0) {
+      pdl_wait();
+      if (!p.w_const) {
+        for (int i = 0; i < ST - 1; ++i) {
+          fill_w(i);
+          cp_async_commit();
+        }
+      }
+      // ---- stage the activations: thread -> 8 consecutive k of one row ----
+      const int chunks = p.K / 8;
+      float ssq[8];
 #pragma unroll
-    for (int q = 0; q < LW; ++q) {
-      const int k = blk * kBlk + q * 8;
-      const bool ok = x_live && blk < blk1 && k + t * 8 * LW < p.K;
-      cp_async16(slot(blk, 2, q), xrow + (ok ? k : 0), ok);
+      for (int m = 0; m < 8; ++m) {
+        ssq[m] = 0.f;
+        if (m >= p.M) continue;
+        const int64_t roff = split2(m, p.M0, p.a_s2, p.a_s3);
+        float acc = 0.f;
+        for (int c = threadIdx.x; c < chunks + kXPad / 8; c += kWarps * 32) {
+          uint4 out;
+          if (c >= chunks) {
+            out = make_uint4(0u, 0u, 0u, 0u);   // the padding is read (against zero weights) when K is not a multiple of 32
+          } else if (p.gamma || p.x_f32) {
+            float xf[8];
+            if (p.x_f32) {
+              const float4 lo = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + roff + c * 8);
+              const float4 hi = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + roff + c * 8 + 4);
+              xf[0] = lo.x; xf[1] = lo.y; xf[2] = lo.z; xf[3] = lo.w; xf[4] = hi.x; xf[5] = hi.y; xf[6] = hi.z; xf[7] = hi.w;
+            } else {
+              load16(static_cast<const __nv_bfloat16*>(p.X) + roff + c * 8, xf);
+            }
+            if (p.gamma) {
+              float gf[8];
+              load16(p.gamma + c * 8, gf);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                acc = fmaf(xf[i], xf[i], acc);
+                xf[i] *= gf[i];
+              }
+            }
+            out = make_uint4(pack_bf16x2(xf[0], xf[1]), pack_bf16x2(xf[2], xf[3]), pack_bf16x2(xf[4], xf[5]), pack_bf16x2(xf[6], xf[7]));
+          } else {
+            out = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.X) + roff + c * 8);
+          }
+          *reinterpret_cast<uint4*>(xs + size_t(m) * pitch + c * 8) = out;
+        }
+        ssq[m] = acc;
+      }
+      if (p.gamma) {
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          const float v = warp_sum(ssq[m]);
+          if (lane == 0) ssq_part[warp * 8 + m] = v;
+        }
+      }
+      __syncthreads();
+      if (threadIdx.x < 8) {
+        float q2 = 0.f;
+        for (int w = 0; w < kWarps; ++w) q2 += ssq_part[w * 8 + threadIdx.x];
+        rstd[threadIdx.x] = p.gamma ? rsqrtf(q2 / p.K + p.eps) : 1.f;
+      }
+      // (rstd is read after the __syncthreads that follows the main loop)
     }
-  };
-  // the weights do not depend on the previous step: their first stages are requested before the wait
-  if (p.w_const)
-    for (int i = 0; i < kStages - 1; ++i) fill_w(blk0 + i);
-  pdl_wait();
-  for (int i = 0; i < kStages - 1; ++i) {
-    if (!p.w_const) fill_w(blk0 + i);
-    fill_x(blk0 + i);
-    cp_async_commit();
-  }
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
-  for (int blk = blk0; blk < blk1; ++blk) {
-    cp_async_wait<kStages - 2>();   // this lane's copies of stage `blk` have landed
-    uint4 w0[LW], w1[LW], x[LW];
-#pragma unroll
-    for (int q = 0; q < LW; ++q) {
-      w0[q] = lds128(slot(blk, 0, q));
-      w1[q] = lds128(slot(blk, 1, q));
-      x[q] = lds128(slot(blk, 2, q));
+    for (int i = 0; i < nloc; ++i) {
+      cp_async_wait<ST - 2>();   // this lane's copies of pass i have landed
+      const uint4 w0 = lds128(slot(i, 0)), w1 = lds128(slot(i, 1));
+      const uint4 x = x_live ? lds128(xs_lane + uint32_t(blk0 + i) * (kBlk * 2)) : make_uint4(0u, 0u, 0u, 0u);
+      fill_w(i + ST - 1);        // refills the slot read one pass ago
+      cp_async_commit();
+      mma_bf16(acc, w0.x, w1.x, w0.y, w1.y, x.x, x.y);
+      mma_bf16(acc, w0.z, w1.z, w0.w, w1.w, x.z, x.w);
     }
-    // refill the slot read one pass ago
-    fill_w(blk + kStages - 1);
-    fill_x(blk + kStages - 1);
-    cp_async_commit();
+    cp_async_wait<0>();
+    // accumulator fragment: acc[0..1] = (weight row g; activation rows 2t, 2t+1), acc[2..3] = (weight row g + 8; same)
+    red[warp][g][2 * t] = acc[0];
+    red[warp][g][2 * t + 1] = acc[1];
+    red[warp][g + 8][2 * t] = acc[2];
+    red[warp][g + 8][2 * t + 1] = acc[3];
+    __syncthreads();
+    // thread -> (tile of the CTA, m, row of the tile) with the row fastest, so that stores to an n-contiguous C coalesce
+    for (int e = threadIdx.x; e < p.upc * 16 * 8; e += kWarps * 32) {
+      const int nl = e % 16, m = (e / 16) % 8, tl = e / 128;
+      const int u = (round * p.upc + tl) * gridDim.x + blockIdx.x;
+      if (u >= p.units) continue;
+      const int n = (SWIGLU ? u : u % p.tiles) * 16 + nl;
+      if (m >= p.M || n >= p.N) continue;
+      const float sc = p.scale * rstd[m];
+      float v = 0.f;
 #pragma unroll
-    for (int q = 0; q < LW; ++q) {
-      mma_bf16(acc, w0[q].x, w1[q].x, w0[q].y, w1[q].y, x[q].x, x[q].y);
-      mma_bf16(acc, w0[q].z, w1[q].z, w0[q].w, w1[q].w, x[q].z, x[q].w);
-    }
-  }
-  cp_async_wait<0>();
-  // accumulator fragment: acc[0..1] = (weight row g; activation rows 2t, 2t+1), acc[2..3] = (weight row g + 8; same)
-  red[warp][g][2 * t] = acc[0];
-  red[warp][g][2 * t + 1] = acc[1];
-  red[warp][g + 8][2 * t] = acc[2];
-  red[warp][g + 8][2 * t + 1] = acc[3];
-  __syncthreads();
-  // thread -> (tile of the CTA, m, row of the tile) with the row fastest, so that stores to an n-contiguous C coalesce
-  for (int e = threadIdx.x; e < TPC * 16 * 8; e += kWarps * 32) {
-    const int nl = e % 16, m = (e / 16) % 8, tl = e / 128;
-    const int n = (blockIdx.x * TPC + tl) * 16 + nl;
-    if (m >= p.M || n >= p.N) continue;
-    float v = 0.f;
+      for (int q = 0; q < KS; ++q) v += red[tl * NG * KS + q][nl][m];
+      v *= sc;
+      if (SWIGLU) {
+        float u = 0.f;
 #pragma unroll
-    for (int q = 0; q < KS; ++q) v += red[tl * NG * KS + q][nl][m];
-    v *= p.scale;
-    if (SWIGLU) {
-      float u = 0.f;
-#pragma unroll
-      for (int q = 0; q < KS; ++q) u += red[(tl * NG + 1) * KS + q][nl][m];
-      v = silu(v) * (u * p.scale);
+        for (int q = 0; q < KS; ++q) u += red[(tl * NG + 1) * KS + q][nl][m];
+        v = silu(v) * (u * sc);
+      }
+      const RowsGroup& og = p.g[SWIGLU ? 0 : u / p.tiles];
+      if (og.has_bias) v += __bfloat162float(og.bias[n]);
+      if (og.act == ACT_GELU_ERF) v = gelu_erf(v);
+      else if (og.act == ACT_GELU_TANH) v = gelu_tanh(v);
+      if (og.has_res) {
+        const int64_t ro = split2(m, p.M0, og.r_s[2], og.r_s[3]) + split2(n, p.N0, og.r_s[4], og.r_s[5]);
+        v += og.r_f32 ? static_cast<const float*>(og.R)[ro] : __bfloat162float(static_cast<const __nv_bfloat16*>(og.R)[ro]);
+      }
+      const int64_t co = split2(m, p.M0, og.c_s[2], og.c_s[3]) + split2(n, p.N0, og.c_s[4], og.c_s[5]);
+      if (og.c_f32) static_cast<float*>(og.C)[co] = v;
+      else static_cast<__nv_bfloat16*>(og.C)[co] = __float2bfloat16_rn(v);
     }
-    const RowsGroup& grp = p.g[SWIGLU ? 0 : blockIdx.y];
-    if (grp.has_bias) v += __bfloat162float(grp.bias[n]);
-    if (grp.act == ACT_GELU_ERF) v = gelu_erf(v);
-    else if (grp.act == ACT_GELU_TANH) v = gelu_tanh(v);
-    if (grp.has_res) {
-      const int64_t ro = split2(m, p.M0, grp.r_s[2], grp.r_s[3]) + split2(n, p.N0, grp.r_s[4], grp.r_s[5]);
-      v += grp.r_f32 ? static_cast<const float*>(grp.R)[ro] : __bfloat162float(static_cast<const __nv_bfloat16*>(grp.R)[ro]);
-    }
-    const int64_t co = split2(m, p.M0, grp.c_s[2], grp.c_s[3]) + split2(n, p.N0, grp.c_s[4], grp.c_s[5]);
-    if (grp.c_f32) static_cast<float*>(grp.C)[co] = v;
-    else static_cast<__nv_bfloat16*>(grp.C)[co] = __float2bfloat16_rn(v);
+    __syncthreads();   // the partial sums are overwritten by the next round
   }
 }
 
+inline size_t rows_fixed_smem(int M, int K) {
+  return size_t(M) * (K + kXPad) * 2 + size_t(kWarps) * 16 * 9 * sizeof(float) + (8 + kWarps * 8) * sizeof(float);
+}
 
-template <int KS, int LW, int ST, bool SWIGLU>
-cudaError_t launch_rows(const RowsParams& p, int tiles, int n_group, cudaStream_t st) {
-  constexpr int kWarps = rows_warps(KS, SWIGLU);
-  constexpr size_t smem = size_t(kWarps) * ST * 3 * LW * 32 * 16 + size_t(kWarps) * 16 * 9 * sizeof(float);
+template <int KS, int ST, bool SWIGLU>
+cudaError_t launch_rows(RowsParams& p, int n_group, cudaStream_t st) {
+  const size_t smem = rows_fixed_smem(p.M, p.K) + size_t(kWarps) * ST * 1024;
   static const cudaError_t attr =
-      cudaFuncSetAttribute(gemm_rows_kernel<KS, LW, ST, SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      cudaFuncSetAttribute(gemm_rows_kernel<KS, ST, SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
   if (attr != cudaSuccess) return attr;
-  constexpr int TPC = kWarps / (KS * (SWIGLU ? 2 : 1));
-  dim3 grid((unsigned)((tiles + TPC - 1) / TPC), (unsigned)(SWIGLU ? 1 : n_group));
-  return launch_k(gemm_rows_kernel<KS, LW, ST, SWIGLU>, grid, dim3(kWarps * 32), smem, st, p, tiles);
+  constexpr int UMAX = kWarps / (KS * (SWIGLU ? 2 : 1));
+  p.units = SWIGLU ? p.tiles : p.tiles * n_group;
+  const int grid = std::min(148, p.units);
+  p.upc = std::min(UMAX, (p.units + grid - 1) / grid);
+  p.rounds = (p.units + grid * p.upc - 1) / (grid * p.upc);
+  return launch_k(gemm_rows_kernel<KS, ST, SWIGLU>, dim3((unsigned)grid), dim3(kWarps * 32), smem, st, p);
 }
 
-template <int LW, int ST>
-cudaError_t launch_rows_ks(const RowsParams& p, int tiles, int n_group, int cps, bool swiglu, cudaStream_t st) {
-  // as many warps per tile (k slices) as keep the whole launch resident at once
-  const int64_t items = (int64_t)tiles * n_group, cap = 148 * kWarpsPerSm;
-  (void)cps;
+template <int ST>
+cudaError_t launch_rows_ks(RowsParams& p, int n_group, bool swiglu, cudaStream_t st) {
+  // as many warps per tile (k slices) as keep the whole launch in one round of the grid
+  const int64_t items = (int64_t)p.tiles * n_group, cap = 148 * kWarps;
   if (swiglu) {
-    if (items * 4 <= cap) return launch_rows<4, LW, ST, true>(p, tiles, n_group, st);
-    if (items * 2 <= cap) return launch_rows<2, LW, ST, true>(p, tiles, n_group, st);
-    return launch_rows<1, LW, ST, true>(p, tiles, n_group, st);
+    if (items * 8 <= cap) return launch_rows<8, ST, true>(p, n_group, st);
+    if (items * 4 <= cap) return launch_rows<4, ST, true>(p, n_group, st);
+    if (items * 2 <= cap) return launch_rows<2, ST, true>(p, n_group, st);
+    return launch_rows<1, ST, true>(p, n_group, st);
   }
-  if (items * 8 <= cap) return launch_rows<8, LW, ST, false>(p, tiles, n_group, st);
-  if (items * 4 <= cap) return launch_rows<4, LW, ST, false>(p, tiles, n_group, st);
-  if (items * 2 <= cap) return launch_rows<2, LW, ST, false>(p, tiles, n_group, st);
-  return launch_rows<1, LW, ST, false>(p, tiles, n_group, st);
+  if (items * 16 <= cap) return launch_rows<16, ST, false>(p, n_group, st);
+  if (items * 8 <= cap) return launch_rows<8, ST, false>(p, n_group, st);
+  if (items * 4 <= cap) return launch_rows<4, ST, false>(p, n_group, st);
+  if (items * 2 <= cap) return launch_rows<2, ST, false>(p, n_group, st);
+  return launch_rows<1, ST, false>(p, n_group, st);
 }
 
 inline bool flat(int X, int X0, int64_t s1, int64_t s0) { return X0 >= X || s1 == (int64_t)X0 * s0; }
@@ -242,6 +305,8 @@ inline bool al16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) =
 bool gemm_rows_eligible(const GemmParams& g) {
   if (g.dtype != FLUID_BF16 || g.batch != 1 || g.M < 1 || g.M > 8 || g.causal != CAUSAL_NONE) return false;
   if (g.K % 8 || g.K < 8) return false;
+  // the activation rows are staged in shared memory next to a ring of at least six stages per warp
+  if (rows_fixed_smem(g.M, g.K) + size_t(kWarps) * 6 * 1024 > size_t(kSmemBudget)) return false;
   // both operands with a flat, contiguous k index
   if (g.a_s[5] != 1 || !flat(g.K, g.K0, g.a_s[4], 1)) return false;
   if (g.b_s[3] != 1 || !flat(g.K, g.K0, g.b_s[2], 1)) return false;
@@ -252,16 +317,19 @@ bool gemm_rows_eligible(const GemmParams& g) {
   return true;
 }
 
-cudaError_t launch_gemm_rows(const GemmParams* gs, int n_group, cudaStream_t st, int swiglu) {
+cudaError_t launch_gemm_rows(const GemmParams* gs, int n_group, cudaStream_t st, int swiglu, const RowsNorm* norm) {
   if (n_group < 1 || n_group > 3 || (swiglu && n_group != 2)) return cudaErrorInvalidValue;
   const GemmParams& g0 = gs[0];
   RowsParams p{};
-  p.X = static_cast<const __nv_bfloat16*>(g0.A);
+  p.X = norm ? norm->x : g0.A;
+  p.x_f32 = norm ? norm->x_f32 : 0;
+  p.gamma = norm ? static_cast<const __nv_bfloat16*>(norm->gamma) : nullptr;
+  p.eps = norm ? norm->eps : 0.f;
   p.M = g0.M; p.N = g0.N; p.K = g0.K; p.M0 = g0.M0; p.N0 = g0.N0;
   p.a_s2 = g0.a_s[2]; p.a_s3 = g0.a_s[3];
   p.scale = g0.scale;
   p.w_const = 1;
-  if (!al16(g0.A)) return cudaErrorInvalidValue;
+  if (!al16(p.X) || (norm && !al16(norm->gamma))) return cudaErrorInvalidValue;
   for (int i = 0; i < n_group; ++i) {
     const GemmParams& g = gs[i];
     if (!gemm_rows_eligible(g) || g.M != g0.M || g.N != g0.N || g.K != g0.K || g.N0 != g0.N0 || g.M0 != g0.M0 || !al16(g.B))
@@ -276,10 +344,12 @@ cudaError_t launch_gemm_rows(const GemmParams* gs, int n_group, cudaStream_t st,
     q.c_f32 = g.c_f32; q.r_f32 = g.r_f32; q.has_bias = g.has_bias; q.has_res = g.has_res; q.act = g.act;
     p.w_const = p.w_const && g.b_const;
   }
-  const int tiles = (p.N + 15) / 16;
-  // one 16-byte piece per lane, row and stage (wider pieces measured three times slower: a copy instruction of the
-  // warp then touches every 32-byte sector half), ring five deep, which lets three CTAs share an SM
-  return launch_rows_ks<1, 5>(p, tiles, n_group, 3, swiglu != 0, st);
+  p.tiles = (p.N + 15) / 16;
+  // ring depth: what the staged activations leave (one 16-byte piece per lane, row and stage; wider pieces measured
+  // three times slower: a copy instruction of the warp then touches every 32-byte sector half)
+  const size_t left = size_t(kSmemBudget) - rows_fixed_smem(p.M, p.K);
+  if (left >= size_t(kWarps) * 10 * 1024) return launch_rows_ks<10>(p, n_group, swiglu != 0, st);
+  return launch_rows_ks<6>(p, n_group, swiglu != 0, st);
 }
 
 }  // namespace fluid

@@ -1058,6 +1058,38 @@ static int lower_and_place(fluid_plan_s* p) {
       p->steps.erase(p->steps.begin() + si + 1);
     }
   }
+  // RMSNorm in front of few-row GEMMs: when every reader of the normalised tensor is a GEMM of the next step and that
+  // step runs the weight-streaming kernel, the normalisation runs inside it (the gain on the way in, 1/rms in the
+  // epilogue) and the normalised tensor is never stored.
+  if (p->opts.fusion && p->opts.gemm_path == 0 && !p->opts.eval && p->opts.split_k <= 0) {
+    std::vector<int> n_uses(nt, 0);
+    for (const Node& n : p->nodes)
+      for (int t : n.ins) n_uses[t]++;
+    for (int si = 0; si + 1 < (int)p->steps.size(); ++si) {
+      const Step& sn = p->steps[si];
+      if (sn.nodes.size() != 1) continue;
+      const Node& nn = p->nodes[sn.node];
+      if (nn.kind != N_NORM || !nn.rms || nn.res >= 0 || T[nn.out].kind != FLUID_ACT || T[nn.out].dtype != FLUID_BF16 ||
+          p->alias_root[nn.out] != nn.out || T[nn.gamma].kind != FLUID_CONST || lo[nn.gamma] != 0)
+        continue;
+      Step& sg = p->steps[si + 1];
+      int readers = 0;
+      bool ok = true;
+      for (int ni : sg.nodes) {
+        const Node& m = p->nodes[ni];
+        if (m.kind != N_GEMM) continue;   // the SiLU * up node of a SwiGLU step
+        GemmParams g;
+        ok = ok && m.a == nn.out && m.gemm_kind == G_LINEAR && lower_gemm(p, m, lo, &g) && gemm_rows_eligible(g);
+        ++readers;
+      }
+      if (!ok || readers == 0 || n_uses[nn.out] != readers) continue;
+      sg.nodes.push_back(sn.node);
+      sg.norm_fused = 1;
+      sg.cost += sn.cost - kLaunch;
+      p->folded[nn.out] = 1;
+      p->steps.erase(p->steps.begin() + si);
+    }
+  }
   // lifetimes in step indices, per alias group
   p->first_step.assign(nt, -1);
   p->last_step.assign(nt, -1);

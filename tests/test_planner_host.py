@@ -306,11 +306,14 @@ def test_decoding_graph_plans_without_a_gpu():
     g = dec.graph
     plan = fluid.Plan(g, synth.default_candidates(g))
     names = [s["kernel_name"] for s in plan.steps()]
-    assert names == ["EMBED"] + ["NORM", "GEMM_ROWS", "ATTN_DECODE", "GEMM_ROWS", "NORM", "GEMM_ROWS", "GEMM_ROWS"] * 2 + ["NORM", "GEMM_ROWS"]
+    # per layer: RMSNorm + Q/K/V, attention (+ rotary), O + residual, RMSNorm + gate/up + SwiGLU, down + residual
+    assert names == ["EMBED"] + ["GEMM_ROWS", "ATTN_DECODE", "GEMM_ROWS", "GEMM_ROWS", "GEMM_ROWS"] * 2 + ["NORM", "GEMM_ROWS"]
+    normed = [s for s in plan.steps() if s["kernel_name"] == "GEMM_ROWS" and (s["variant"] >> 30) & 1]
+    assert len(normed) == 4 and all(synth.RMSNORM in [g.ops[o]["kind"] for o in s["ops"]] for s in normed)
     att = [s for s in plan.steps() if s["kernel_name"] == "ATTN_DECODE"]
     assert all(len(s["ops"]) == 3 and (s["variant"] >> 16) & 1 for s in att)            # attention + two ROPE ops
-    fused = [s for s in plan.steps() if s["kernel_name"] == "GEMM_ROWS" and len(s["ops"]) == 4]
-    assert len(fused) == 2 and all(len(s["outs"]) == 1 for s in fused)                   # gate, up, SiLU, MUL
+    fused = [s for s in plan.steps() if s["kernel_name"] == "GEMM_ROWS" and len(s["ops"]) == 5]
+    assert len(fused) == 2 and all(len(s["outs"]) == 1 for s in fused)                   # RMSNorm, gate, up, SiLU, MUL
     for kc, vc in dec.caches:
         for t in (kc, vc):
             info = plan.tensor_info(t)
