@@ -298,9 +298,7 @@ cudaError_t launch_one(const AttnDecodeParams& p, cudaStream_t st) {
   // row ranges per (sequence, head): as many as still leave the whole launch resident at once (three CTAs fit an SM);
   // a second, partial wave would run with few bytes in flight
   const int64_t heads = (int64_t)p.B * p.NH;
-  int splits = (int)std::max<int64_t>(1, std::min<int64_t>(kSplits, (148 * 3) / heads));
-  static const int env_s = [] { const char* e = std::getenv("FLUID_AD_SPLITS"); return e ? atoi(e) : 0; }();
-  if (env_s) splits = env_s;
+  const int splits = (int)std::max<int64_t>(1, std::min<int64_t>(kSplits, (148 * 3) / heads));
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)splits, (unsigned)p.NH, (unsigned)p.B);
   cfg.blockDim = dim3(kWarps * 32);

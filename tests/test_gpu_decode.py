@@ -61,6 +61,19 @@ def test_cached_attention_step(B, nh, nkv, D, Tmax, dtype, ts):
     plan.close()
 
 
+@pytest.mark.parametrize("B,nh", [(25, 8), (10, 12), (10, 10), (10, 8), (7, 10), (6, 10), (37, 16)])
+def test_cached_attention_every_cluster_size(B, nh):
+    """The number of CTAs that share a head's rows follows the head count (1 to 8, powers of two or not)."""
+    D, Tmax, t = 64, 131, 130
+    g, (q, k, v, kc, vc, pos, out) = _cached_graph(B, nh, nh, D, Tmax, synth.BF16)
+    feeds = {q: helpers.rand_feed([B, 1, nh, D], synth.BF16, 1, -2, 2), k: helpers.rand_feed([B, 1, nh, D], synth.BF16, 2, -2, 2),
+             v: helpers.rand_feed([B, 1, nh, D], synth.BF16, 3), kc: helpers.rand_feed([B, Tmax, nh, D], synth.BF16, 4, -2, 2),
+             vc: helpers.rand_feed([B, Tmax, nh, D], synth.BF16, 5), pos: np.array([t], dtype=np.int32)}
+    got, plan, _ = helpers.run_gpu(g, feeds, synth.default_candidates(g))
+    helpers.assert_close(got[out], helpers.run_oracle(g, feeds)[out], synth.BF16, f"{B}x{nh}")
+    plan.close()
+
+
 def test_position_outside_the_cache_is_reported_and_nothing_is_written():
     g, (q, k, v, kc, vc, pos, out) = _cached_graph(1, 4, 4, 64, 32, synth.BF16)
     helpers.ensure_lib()
