@@ -43,7 +43,7 @@ def run_op(kind, ins, attrs):
     if kind == RMSNORM:
         return [ops.rmsnorm(ins[0], ins[1], eps=attrs.get("eps", 1e-5))]
     if kind == ROPE:
-        pos0 = int(np.asarray(ins[1]).reshape(-1)[0]) if len(ins) > 1 else 0
+        pos0 = np.asarray(ins[1]).reshape(-1) if len(ins) > 1 else 0
         return [ops.rope(ins[0], base=attrs.get("rope_base", 10000.0),
                          interleaved=bool(attrs.get("rope_interleaved", 0)), pos0=pos0)]
     if kind == TRANSPOSE:

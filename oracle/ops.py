@@ -120,7 +120,8 @@ def mul(a, b):
 
 def rope(x, base=10000.0, interleaved=False, pos0=0):
     """Rotary embedding on x[b, s, h, d]; position p = pos0 + s (0-based; pos0 is the number of
-    tokens that came before this call's first row, 0 for a whole sequence).
+    tokens that came before this call's first row, 0 for a whole sequence; one number for the whole
+    batch or one per sequence).
 
     Rotate-half pairing (i, i + D/2) by angle p * base^(-2i/D); the interleaved form pairs
     (2i, 2i+1) with the same angles.
@@ -129,9 +130,12 @@ def rope(x, base=10000.0, interleaved=False, pos0=0):
     B, S, nh, D = x.shape
     half = D // 2
     i = np.arange(half, dtype=np.float64)
-    theta = (int(pos0) + np.arange(S, dtype=np.float64))[:, None] * base ** (-2.0 * i / D)[None, :]
-    c = np.cos(theta)[None, :, None, :]
-    s = np.sin(theta)[None, :, None, :]
+    p0 = np.asarray(pos0, dtype=np.float64).reshape(-1)
+    assert p0.size in (1, B)
+    p0 = np.broadcast_to(p0, (B,))
+    theta = (p0[:, None] + np.arange(S, dtype=np.float64)[None, :])[:, :, None] * base ** (-2.0 * i / D)[None, None, :]
+    c = np.cos(theta)[:, :, None, :]
+    s = np.sin(theta)[:, :, None, :]
     y = np.empty_like(x)
     if interleaved:
         a, b = x[..., 0::2], x[..., 1::2]
@@ -147,9 +151,10 @@ def rope(x, base=10000.0, interleaved=False, pos0=0):
 def cached_attention(q, k, v, k_cache, v_cache, pos, scale=1.0):
     """One decoding step of attention against a key/value cache.
 
-    q[B,1,nh,D] is the query of the token at position t = pos; k, v[B,1,nkv,D] are its key and
-    value; k_cache, v_cache[B,Tmax,nkv,D] hold the keys and values of positions 0..t-1 (rows from t
-    on are unspecified). The step stores k, v as row t of the caches and returns
+    q[B,1,nh,D] is the query of the token at position t = pos (one position for the whole batch, or
+    pos[b] per sequence); k, v[B,1,nkv,D] are its key and value; k_cache, v_cache[B,Tmax,nkv,D] hold
+    the keys and values of positions 0..t-1 (rows from t on are unspecified). The step stores k, v as
+    row t of the caches and returns
       ctx[b,0,h,:] = sum_{j<=t} softmax_j(scale * q[b,0,h,:] . K[b,j,g,:]) V[b,j,g,:],  g = h // (nh/nkv),
     that is, the row for query position t of causal attention over the t+1 tokens so far (query
     heads share key/value heads in groups when nkv < nh). Returns (ctx, k_cache', v_cache').
@@ -157,14 +162,17 @@ def cached_attention(q, k, v, k_cache, v_cache, pos, scale=1.0):
     q = np.asarray(q, np.float64)
     kc = np.array(k_cache, dtype=np.float64)
     vc = np.array(v_cache, dtype=np.float64)
-    t = int(np.asarray(pos).reshape(-1)[0])
     B, one, nh, D = q.shape
     Tmax, nkv = kc.shape[1], kc.shape[2]
-    assert one == 1 and 0 <= t < Tmax and nh % nkv == 0
-    kc[:, t] = np.asarray(k, np.float64)[:, 0]
-    vc[:, t] = np.asarray(v, np.float64)[:, 0]
+    ts = np.asarray(pos).reshape(-1)
+    assert ts.size in (1, B) and one == 1 and nh % nkv == 0
+    ts = [int(ts[b if ts.size == B else 0]) for b in range(B)]
     ctx = np.zeros((B, 1, nh, D))
     for b in range(B):
+        t = ts[b]
+        assert 0 <= t < Tmax
+        kc[b, t] = np.asarray(k, np.float64)[b, 0]
+        vc[b, t] = np.asarray(v, np.float64)[b, 0]
         for h in range(nh):
             g = h // (nh // nkv)
             s = (kc[b, : t + 1, g, :] @ q[b, 0, h, :]) * float(scale)

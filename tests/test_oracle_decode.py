@@ -118,3 +118,19 @@ def test_decoding_steps_reproduce_the_whole_sequence_model():
     for l, (kc, vc) in enumerate(dec.caches):
         np.testing.assert_allclose(state[kc][:, :cfg.S], by_name[f"l{l}.k_rope"], rtol=1e-9, atol=1e-12)
         np.testing.assert_allclose(state[vc][:, :cfg.S], by_name[f"l{l}.v"], rtol=1e-9, atol=1e-12)
+
+
+def test_positions_per_sequence_equal_each_sequence_alone():
+    rng = np.random.default_rng(9)
+    B, nh, D, Tmax = 3, 2, 8, 10
+    q = rng.standard_normal((B, 1, nh, D)); k = rng.standard_normal((B, 1, nh, D)); v = rng.standard_normal((B, 1, nh, D))
+    kc = rng.standard_normal((B, Tmax, nh, D)); vc = rng.standard_normal((B, Tmax, nh, D))
+    pos = np.array([0, 9, 4])
+    ctx, kc2, vc2 = ops.cached_attention(q, k, v, kc, vc, pos, scale=0.5)
+    for b in range(B):
+        one = ops.cached_attention(q[b:b + 1], k[b:b + 1], v[b:b + 1], kc[b:b + 1], vc[b:b + 1], [pos[b]], scale=0.5)
+        assert np.array_equal(ctx[b:b + 1], one[0]) and np.array_equal(kc2[b:b + 1], one[1]) and np.array_equal(vc2[b:b + 1], one[2])
+    x = rng.standard_normal((B, 2, nh, D))
+    r = ops.rope(x, base=100.0, pos0=pos)
+    for b in range(B):
+        np.testing.assert_allclose(r[b:b + 1], ops.rope(x[b:b + 1], base=100.0, pos0=int(pos[b])), rtol=1e-14, atol=1e-14)
