@@ -68,18 +68,20 @@ typedef enum { FLUID_INPUT = 0, FLUID_OUTPUT = 1, FLUID_CONST = 2, FLUID_ACT = 3
  *  SOFTMAX (s[..., n]) -> over the last dim, after multiplying by `scale`; causal: column j of
  *          row i (the last two dims) takes part only if j <= i, other outputs are exactly 0
  *  LAYERNORM (x, gamma, beta) / RMSNORM (x, gamma) -> over the last dim, population variance
- *  ROPE    (x[B,S,nh,D] [, pos i32[1]]) -> rotary embedding with position = index along dim 1 (+ pos[0], read on
- *          the device at run time: the number of tokens that came before this call's first row)
+ *  ROPE    (x[B,S,nh,D] [, pos i32[1] or i32[B]]) -> rotary embedding with position = index along dim 1 (+ pos[0], or
+ *          pos[b] per sequence, read on the device at run time: the number of tokens that came before this call's
+ *          first row)
  *  TRANSPOSE (x) -> y with y dim j = x dim perm[j]
  *  BMM_QK  (q[B,nh,S,D], kt[B,nh,D,S]) -> scale * q.kt  [B,nh,S,S]
  *  BMM_PV  (p[B,nh,S,S], v[B,nh,S,D]) -> p.v  [B,nh,S,D]
  *  SELECT_LAST_TOKEN (x[B,S,H]) -> x[:, S-1, :]  [B,H]
  *  CACHED_ATTENTION (q[B,1,nh,D], k[B,1,nkv,D], v[B,1,nkv,D], k_cache STATE[B,Tmax,nkv,D], v_cache STATE[B,Tmax,nkv,D],
- *          pos i32[1]) -> ctx[B,1,nh,D]: one decoding step. With t = pos[0] (read on the device at run time,
- *          0 <= t < Tmax; the same for every sequence) the step stores k, v as row t of the caches and returns
+ *          pos i32[1] or i32[B]) -> ctx[B,1,nh,D]: one decoding step. With t = pos[0] for every sequence, or pos[b]
+ *          for sequence b (read on the device at run time, 0 <= t < Tmax) the step stores k, v as row t of the caches and returns
  *          ctx[b,0,h,:] = sum_{j<=t} softmax_j(scale * q[b,0,h,:] . k_cache[b,j,g,:]) v_cache[b,j,g,:], g = h / (nh/nkv):
  *          the row for position t of causal attention over the t+1 tokens so far. Cache rows beyond t are neither
- *          read nor written. t outside [0, Tmax) leaves caches and ctx untouched and sets bit 0x10 of fluid_status.
+ *          read nor written. t outside [0, Tmax) leaves that sequence's caches and ctx untouched and sets bit 0x10 of
+ *          fluid_status.
  */
 typedef enum {
   FLUID_OP_EMBED = 0, FLUID_OP_LINEAR = 1, FLUID_OP_ADD = 2, FLUID_OP_MUL = 3, FLUID_OP_GELU = 4,

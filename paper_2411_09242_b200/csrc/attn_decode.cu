@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
   const int grp = lane / LPR, li = lane % LPR;
   const int split = blockIdx.x, n_split = gridDim.x, h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.NH / p.NKV);
-  const int t = *p.pos;   // a graph input: nothing in this run writes it
+  const int t = p.pos[b * p.pos_stride];   // a graph input: nothing in this run writes it
   const bool t_ok = t >= 0 && t < p.Tmax;
   const int n = t_ok ? t + 1 : 0;
   const int chunk = ((n + n_split - 1) / n_split + RPI - 1) / RPI * RPI;
@@ -154,9 +154,9 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
     cp_async_commit();
   }
   pdl_wait();
-  if (!t_ok) {   // the same in every CTA: nobody reaches the cluster barrier
+  if (!t_ok) {   // the same in every CTA of the cluster (one sequence, one head): nobody reaches the cluster barrier
     cp_async_wait<0>();
-    if (threadIdx.x == 0 && split == 0 && h == 0 && b == 0) atomicOr(p.status, 0x10u);
+    if (threadIdx.x == 0 && split == 0 && h == 0) atomicOr(p.status, 0x10u);
     return;
   }
 

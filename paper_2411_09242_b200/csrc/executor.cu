@@ -202,6 +202,7 @@ int finalize_steps(fluid_plan_s* p) {
         }
         q.base = (float)n.rope_base;
         q.interleaved = n.rope_interleaved;
+        q.pos_stride = (n.pos >= 0 && T[n.pos].dims[0] > 1) ? 1 : 0;
         s.rope = q;
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.out; s.t_ptr[2] = n.pos; s.t_narrow[0] = 1;
         s.bytes = es * ty.numel() * 2.0;
@@ -266,6 +267,7 @@ int finalize_steps(fluid_plan_s* p) {
         q.B = (int)tq.dims[0]; q.NH = (int)tq.dims[2]; q.NKV = (int)tk.dims[2]; q.D = (int)tq.dims[3]; q.Tmax = (int)tc.dims[1];
         q.scale_log2 = (float)(n.scale * 1.4426950408889634);
         q.rope = n.rope_fused;
+        q.pos_stride = T[n.pos].dims[0] > 1 ? 1 : 0;
         q.rope_log2_base = (float)std::log2(n.rope_base);
         int64_t st[FLUID_MAX_RANK];
         perm_strides(p, n.a, st);   q.q_sb = st[0]; q.q_sh = st[2];

@@ -105,9 +105,9 @@ static int check_op(const fluid_graph_s* g, const OpDesc& op) {
                     y.dims[3] % 2 == 0 && y.dtype != FLUID_I32,
                 "ROPE wants x[B,S,nh,D] with even D"))
         return FLUID_EINVAL;
-      if (ni == 2 && !need(T(op.ins[1]).dtype == FLUID_I32 && T(op.ins[1]).rank == 1 && T(op.ins[1]).dims[0] == 1 &&
-                               T(op.ins[1]).kind == FLUID_INPUT,
-                           "ROPE's position offset is an int32 [1] graph input"))
+      if (ni == 2 && !need(T(op.ins[1]).dtype == FLUID_I32 && T(op.ins[1]).rank == 1 &&
+                               (T(op.ins[1]).dims[0] == 1 || T(op.ins[1]).dims[0] == y.dims[0]) && T(op.ins[1]).kind == FLUID_INPUT,
+                           "ROPE's position offset is an int32 [1] or [B] graph input"))
         return FLUID_EINVAL;
       break;
     case FLUID_OP_CACHED_ATTENTION: {
@@ -118,11 +118,11 @@ static int check_op(const fluid_graph_s* g, const OpDesc& op) {
         ok = q.rank == 4 && same_dims(q, y) && q.dims[1] == 1 && k.rank == 4 && same_dims(k, v) && k.dims[0] == q.dims[0] &&
              k.dims[1] == 1 && k.dims[3] == q.dims[3] && q.dims[2] % k.dims[2] == 0 && kc.rank == 4 && same_dims(kc, vc) &&
              kc.dims[0] == q.dims[0] && kc.dims[2] == k.dims[2] && kc.dims[3] == q.dims[3] && kc.kind == FLUID_STATE &&
-             vc.kind == FLUID_STATE && op.ins[3] != op.ins[4] && pos.dtype == FLUID_I32 && pos.rank == 1 && pos.dims[0] == 1 &&
-             pos.kind == FLUID_INPUT && y.dtype != FLUID_I32 && q.dtype == y.dtype && k.dtype == y.dtype &&
+             vc.kind == FLUID_STATE && op.ins[3] != op.ins[4] && pos.dtype == FLUID_I32 && pos.rank == 1 &&
+             (pos.dims[0] == 1 || pos.dims[0] == q.dims[0]) && pos.kind == FLUID_INPUT && y.dtype != FLUID_I32 && q.dtype == y.dtype && k.dtype == y.dtype &&
              v.dtype == y.dtype && kc.dtype == y.dtype && vc.dtype == y.dtype;
       }
-      if (!need(ok, "CACHED_ATTENTION wants q[B,1,nh,D], k, v[B,1,nkv,D], two STATE caches [B,Tmax,nkv,D], pos i32[1]"))
+      if (!need(ok, "CACHED_ATTENTION wants q[B,1,nh,D], k, v[B,1,nkv,D], two STATE caches [B,Tmax,nkv,D], pos i32[1] or [B]"))
         return FLUID_EINVAL;
       for (const OpDesc& o : g->ops)
         if (o.kind == FLUID_OP_CACHED_ATTENTION)

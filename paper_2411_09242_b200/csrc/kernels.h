@@ -109,6 +109,7 @@ struct RopeParams {
   float base;
   int interleaved;
   const int* pos;     // device: position of row 0 (null = 0)
+  int pos_stride;     // 0: one position for the batch, 1: pos[b] per sequence
 };
 
 struct EltParams {
@@ -165,6 +166,7 @@ struct AttnDecodeParams {
   const void *q, *k, *v;  // [B,1,NH,D], [B,1,NKV,D] x 2: d contiguous, strides below
   void *kc, *vc;
   const int* pos;         // device
+  int pos_stride;         // 0: one position for the batch, 1: pos[b] per sequence
   void* out;              // [B,1,NH,D]
   uint32_t* status;
   int B, NH, NKV, D, Tmax;

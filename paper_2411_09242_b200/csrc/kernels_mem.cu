@@ -525,7 +525,6 @@ __global__ void rope_kernel(RopeParams p, int64_t total) {
   pdl_launch_dependents();
   pdl_wait();
   const int half = p.dims[3] / 2;
-  const int pos0 = p.pos ? *p.pos : 0;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     int idx[4];
     int64_t rem = i;
@@ -541,6 +540,7 @@ __global__ void rope_kernel(RopeParams p, int64_t total) {
     const int64_t base = idx[0] * p.st[0] + idx[1] * p.st[1] + idx[2] * p.st[2];
     const float inv_freq = exp2f(-2.f * pr / p.dims[3] * log2f(p.base));
     float sn, cs;
+    const int pos0 = p.pos ? p.pos[idx[0] * p.pos_stride] : 0;
     sincosf((idx[1] + pos0) * inv_freq, &sn, &cs);
     const T* x = static_cast<const T*>(p.x);
     T* y = static_cast<T*>(p.y);
@@ -558,13 +558,13 @@ __global__ void __launch_bounds__(256) rope_vec_kernel(RopeParams p, int64_t tot
   pdl_wait();
   const int D = p.dims[3], half = D / 2, cpr = half / 8;
   const float lb = log2f(p.base);
-  const int pos0 = p.pos ? *p.pos : 0;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     int64_t rem = i;
     const int c = int(rem % cpr); rem /= cpr;
     const int hg = int(rem % hgroups); rem /= hgroups;
     const int s = int(rem % p.dims[1]);
     const int b = int(rem / p.dims[1]);
+    const int pos0 = p.pos ? p.pos[b * p.pos_stride] : 0;
     float cs[8], sn[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {

@@ -362,11 +362,11 @@ class DecodeModel:
 
 
 def build_decode_model(cfg: ModelConfig, t_max: int, like: Model = None, weight_seed: int = WEIGHT_SEED,
-                       materialize: bool = True) -> DecodeModel:
+                       materialize: bool = True, per_sequence_pos: bool = False) -> DecodeModel:
     """The llama-family graph of ONE decoding step: B sequences, one new token each, the keys and
     values of the earlier tokens in per-layer caches [B, t_max, nh, D] that the caller owns and the
-    step extends (STATE tensors). `pos` (int32 [1], on the device at run time) is the number of
-    tokens already cached, the same for all sequences. Outputs: the final hidden state [B,1,H]
+    step extends (STATE tensors). `pos` (int32 [1], or [B] with per_sequence_pos; on the device at run
+    time) is the number of tokens already cached, for all sequences or per sequence. Outputs: the final hidden state [B,1,H]
     and the logits [B,1,V].
 
     like: a whole-sequence model of the same family and widths; its weights are taken over by name,
@@ -378,7 +378,7 @@ def build_decode_model(cfg: ModelConfig, t_max: int, like: Model = None, weight_
     g = b.g
     B, H, V, nh, D = cfg.B, cfg.H, cfg.V, cfg.nh, cfg.D
     ids = g.tensor("ids", I32, [B, 1], INPUT)
-    pos = g.tensor("pos", I32, [1], INPUT)
+    pos = g.tensor("pos", I32, [B if per_sequence_pos else 1], INPUT)
     tok = b.const("tok_table", [V, H])
     x = b.act("embed", [B, 1, H])
     g.op(EMBED, [ids, tok], [x])

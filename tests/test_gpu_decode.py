@@ -230,3 +230,86 @@ def test_one_captured_graph_serves_every_step_of_a_generation_loop():
             helpers.assert_close(logits, ref[g.outputs[1]], synth.BF16, f"replayed step {step}", tol=2e-2)
     assert runner.status() == 0
     plan.close()
+
+
+def test_positions_per_sequence():
+    """pos of shape [B]: every sequence appends at, and attends up to, its own position; a sequence whose position lies
+    outside the cache is left alone and reported, the others are served."""
+    B, nh, nkv, D, Tmax = 5, 8, 4, 128, 300
+    g = synth.GraphDesc()
+    q = g.tensor("q", synth.BF16, [B, 1, nh, D], synth.INPUT)
+    k = g.tensor("k", synth.BF16, [B, 1, nkv, D], synth.INPUT)
+    v = g.tensor("v", synth.BF16, [B, 1, nkv, D], synth.INPUT)
+    kc = g.tensor("kc", synth.BF16, [B, Tmax, nkv, D], synth.STATE)
+    vc = g.tensor("vc", synth.BF16, [B, Tmax, nkv, D], synth.STATE)
+    pos = g.tensor("pos", synth.I32, [B], synth.INPUT)
+    out = g.tensor("ctx", synth.BF16, [B, 1, nh, D], synth.OUTPUT)
+    g.op(synth.CACHED_ATTENTION, [q, k, v, kc, vc, pos], [out], scale=1.0 / math.sqrt(D))
+    helpers.ensure_lib()
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    runner = fluid.Runner(plan, {}, poison=True)
+    feeds = {q: helpers.rand_feed([B, 1, nh, D], synth.BF16, 1, -2, 2), k: helpers.rand_feed([B, 1, nkv, D], synth.BF16, 2, -2, 2),
+             v: helpers.rand_feed([B, 1, nkv, D], synth.BF16, 3), kc: helpers.rand_feed([B, Tmax, nkv, D], synth.BF16, 4, -2, 2),
+             vc: helpers.rand_feed([B, Tmax, nkv, D], synth.BF16, 5), pos: np.array([0, 299, 17, 128, 255], dtype=np.int32)}
+    runner.set_inputs([feeds[t] for t in g.inputs])
+    runner.run()
+    got = runner.outputs_host()[0]
+    assert runner.status() == 0
+    ref = helpers.run_oracle(g, feeds)
+    helpers.assert_close(got, ref[out], synth.BF16, "ragged positions")
+    kc_dev = runner.inputs[g.inputs.index(kc)].float().cpu().numpy()
+    assert np.array_equal(kc_dev, ref[kc])
+    # sequence 2 out of range: its context row and caches keep what they held, the others are computed
+    bad = dict(feeds)
+    bad[pos] = np.array([3, 4, 300, 5, 6], dtype=np.int32)
+    runner.set_inputs([bad[t] for t in g.inputs])
+    runner.outputs[0].fill_(7.0)
+    runner.run()
+    with pytest.raises(fluid.FluidError):
+        runner.status()
+    got = runner.outputs[0].float().cpu().numpy()
+    ok_rows = [0, 1, 3, 4]
+    good = {t: (a[ok_rows] if a.shape[0] == B else a) for t, a in bad.items()}
+    good[pos] = bad[pos][ok_rows]
+    g4 = synth.GraphDesc()
+    ids4 = [g4.tensor(g.tensors[t]["name"], g.tensors[t]["dtype"], [4] + g.dims(t)[1:] if t != pos else [4], g.tensors[t]["kind"]) for t in (q, k, v, kc, vc, pos)]
+    o4 = g4.tensor("ctx", synth.BF16, [4, 1, nh, D], synth.OUTPUT)
+    g4.op(synth.CACHED_ATTENTION, ids4, [o4], scale=1.0 / math.sqrt(D))
+    ref4 = helpers.run_oracle(g4, {i4: good[t] for i4, t in zip(ids4, (q, k, v, kc, vc, pos))})
+    helpers.assert_close(got[ok_rows], ref4[o4], synth.BF16, "served sequences")
+    assert np.all(got[2] == 7.0)
+    plan.close()
+
+
+def test_decoding_with_ragged_lengths():
+    """A batch whose sequences are at different lengths: positions per sequence through the whole model (rotary offset,
+    cache append and attention span all per sequence), several steps in a row."""
+    cfg = synth.scaled(synth.CONFIGS["llama"], dtype=synth.BF16, S=1, L=2, H=256, nh=4, F=384, B=3, V=400)
+    t_max = 40
+    dec = synth.build_decode_model(cfg, t_max, per_sequence_pos=True)
+    g = dec.graph
+    helpers.ensure_lib()
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    runner = fluid.Runner(plan, dec.consts)
+    rng = np.random.default_rng(2)
+    start = np.array([0, 11, 30], dtype=np.int32)
+    state_ids = [t for pair in dec.caches for t in pair]
+    oracle_state = {t: synth.round_bf16(synth.uniform(8, t, g.dims(t))).astype(np.float64) for t in state_ids}
+    for t in state_ids:
+        runner.inputs[g.inputs.index(t)].copy_(fluid.to_device(oracle_state[t].astype(np.float32), synth.BF16, "cuda"))
+    for step in range(6):
+        ids = rng.integers(0, cfg.V, size=(cfg.B, 1)).astype(np.int32)
+        feeds = dict(dec.consts)
+        feeds[dec.ids], feeds[dec.pos] = ids, start + step
+        feeds.update(oracle_state)
+        ref = helpers.run_oracle(g, feeds)
+        for t in state_ids:
+            oracle_state[t] = ref[t]
+        runner.inputs[g.inputs.index(dec.ids)].copy_(fluid.to_device(ids, synth.I32, "cuda"))
+        runner.inputs[g.inputs.index(dec.pos)].copy_(fluid.to_device(feeds[dec.pos], synth.I32, "cuda"))
+        runner.run()
+        outs = runner.outputs_host()
+        assert runner.status() == 0
+        for tid, got in zip(g.outputs, outs):
+            helpers.assert_close(got, ref[tid], synth.BF16, f"ragged step {step} {g.tensors[tid]['name']}", tol=2e-2)
+    plan.close()
