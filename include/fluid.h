@@ -60,7 +60,9 @@ typedef enum { FLUID_F32 = 0, FLUID_BF16 = 1, FLUID_I32 = 2 } fluid_dtype;
 typedef enum { FLUID_INPUT = 0, FLUID_OUTPUT = 1, FLUID_CONST = 2, FLUID_ACT = 3, FLUID_STATE = 4 } fluid_tensor_kind;
 
 /* Primitive operators ("nodes"). Shapes are logical, independent of layout.
- *  EMBED   (ids[B,S] i32, tok[V,H] [, pos[S,H]]) -> x[B,S,H] = tok[ids] (+ pos)
+ *  EMBED   (ids[B,S] i32, tok[V,H] [, pos[P,H] [, off i32[1] or i32[B]]]) -> x[b,s,:] = tok[ids[b,s]] (+ pos[s + off]);
+ *          off (read on the device at run time) is the number of tokens that came before, for the batch or per
+ *          sequence; ids are clamped to [0,V) and position rows to [0,P)
  *  LINEAR  (x[..m.., ..k..], w[..k.., ..n..] [, bias[..n..]]) -> y[..m.., ..n..]; contracts the
  *          last `contract` dims of x with the first `contract` dims of w (the paper's GEMM:
  *          left (i,k), right (k,j), out (i,j))

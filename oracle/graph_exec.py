@@ -23,7 +23,8 @@ STATE = 4   # tensor kind: a caller-owned buffer an op reads and updates (a key/
 def run_op(kind, ins, attrs):
     """Apply one node to canonical fp64 inputs; returns the list of outputs."""
     if kind == EMBED:
-        return [ops.embed(ins[0], ins[1], ins[2] if len(ins) > 2 else None)]
+        return [ops.embed(ins[0], ins[1], ins[2] if len(ins) > 2 else None,
+                          pos0=np.asarray(ins[3]).reshape(-1) if len(ins) > 3 else 0)]
     if kind == LINEAR:
         return [ops.linear(ins[0], ins[1], ins[2] if len(ins) > 2 else None,
                            contract=attrs.get("contract", 1))]

@@ -30,11 +30,17 @@ except Exception:  # pragma: no cover
     _erf = np.vectorize(math.erf, otypes=[np.float64])
 
 
-def embed(ids, tok, pos=None):
-    """x[b,s,:] = tok[ids[b,s],:] (+ pos[s,:]) — a gather plus an optional broadcast add."""
+def embed(ids, tok, pos=None, pos0=0):
+    """x[b,s,:] = tok[ids[b,s],:] (+ pos[pos0 + s,:]) — a gather plus an optional add of the position rows; pos0 is
+    the number of tokens that came before (0 for a whole sequence; one number for the batch or one per sequence)."""
     x = np.asarray(tok, dtype=np.float64)[np.asarray(ids, dtype=np.int64)]
     if pos is not None:
-        x = x + np.asarray(pos, dtype=np.float64)[None, : x.shape[1], :]
+        B, S = x.shape[0], x.shape[1]
+        p0 = np.asarray(pos0, dtype=np.int64).reshape(-1)
+        assert p0.size in (1, B)
+        rows = np.broadcast_to(p0, (B,))[:, None] + np.arange(S)[None, :]
+        assert rows.min() >= 0 and rows.max() < np.asarray(pos).shape[0]
+        x = x + np.asarray(pos, dtype=np.float64)[rows]
     return x
 
 

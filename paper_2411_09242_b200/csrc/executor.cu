@@ -50,8 +50,10 @@ int finalize_steps(fluid_plan_s* p) {
         e.H = (int)ty.dims[2];
         e.V = (int)T[n.b].dims[0];
         e.y_f32 = p->wide[n.out];
+        e.P = n.pos >= 0 ? (int)T[n.pos].dims[0] : 0;
+        e.pos_off_stride = (n.pos_off >= 0 && T[n.pos_off].dims[0] > 1) ? 1 : 0;
         s.embed = e;
-        s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.pos; s.t_ptr[3] = n.out;
+        s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.pos; s.t_ptr[3] = n.out; s.t_ptr[4] = n.pos_off;
         s.bytes = es * ty.numel() * (n.pos >= 0 ? 3.0 : 2.0) + 4.0 * e.tokens;
         break;
       }
@@ -437,6 +439,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
         EmbedParams q = s.embed;
         q.ids = static_cast<const int*>(R(s.t_ptr[0])); q.tok = R(s.t_ptr[1]); q.pos = R(s.t_ptr[2]);
         q.y = const_cast<void*>(R(s.t_ptr[3]));
+        q.pos_off = static_cast<const int*>(R(s.t_ptr[4]));
         if (R.ok) err = launch_embed(q, stream);
         break;
       }

@@ -58,7 +58,7 @@ struct Node {
   std::vector<int> ops;        // graph op ids folded into this node, first = anchor
   std::vector<int> ins, outs;  // distinct external tensors, inputs in role order
   // role-tagged tensor ids (-1 = absent)
-  int a = -1, b = -1, bias = -1, res = -1, out = -1, gamma = -1, beta = -1, pos = -1, v = -1, kc = -1, vc = -1;
+  int a = -1, b = -1, bias = -1, res = -1, out = -1, gamma = -1, beta = -1, pos = -1, v = -1, kc = -1, vc = -1, pos_off = -1;
   int gemm_kind = G_LINEAR, contract = 1, act = ACT_NONE, causal = CAUSAL_NONE;
   double scale = 1.0, eps = 1e-5, rope_base = 10000.0;
   int elt = ELT_ADD, rms = 0, rope_interleaved = 0, sm_causal = 0, rope_fused = 0;

@@ -41,14 +41,18 @@ static int check_op(const fluid_graph_s* g, const OpDesc& op) {
     }
   switch (op.kind) {
     case FLUID_OP_EMBED: {
-      if (!need(ni == 2 || ni == 3, "EMBED takes ids, table [, positions]")) return FLUID_EINVAL;
+      if (!need(ni >= 2 && ni <= 4, "EMBED takes ids, table [, positions [, offset]]")) return FLUID_EINVAL;
       const TensorDesc &ids = T(op.ins[0]), &tok = T(op.ins[1]);
       bool ok = ids.dtype == FLUID_I32 && ids.rank == 2 && tok.rank == 2 && y.rank == 3 &&
                 y.dims[0] == ids.dims[0] && y.dims[1] == ids.dims[1] && y.dims[2] == tok.dims[1] &&
                 tok.dtype == y.dtype;
-      if (ok && ni == 3) {
+      if (ok && ni >= 3) {
         const TensorDesc& pos = T(op.ins[2]);
         ok = pos.rank == 2 && pos.dims[0] >= ids.dims[1] && pos.dims[1] == tok.dims[1] && pos.dtype == y.dtype;
+      }
+      if (ok && ni == 4) {
+        const TensorDesc& off = T(op.ins[3]);
+        ok = off.dtype == FLUID_I32 && off.rank == 1 && (off.dims[0] == 1 || off.dims[0] == ids.dims[0]) && off.kind == FLUID_INPUT;
       }
       if (!need(ok, "EMBED shapes")) return FLUID_EINVAL;
       break;

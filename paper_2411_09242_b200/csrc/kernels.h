@@ -138,7 +138,10 @@ struct PermuteParams {
 struct EmbedParams {
   const int* ids;
   const void* tok;
-  const void* pos;    // optional [S, H]
+  const void* pos;    // optional [P, H]
+  const int* pos_off; // optional, device: index of the first position row, for the batch or per sequence
+  int pos_off_stride; // 0 or 1
+  int P;              // rows of pos
   void* y;
   int dtype;
   int y_f32;          // bf16 models: y is held in fp32

@@ -20,7 +20,9 @@ __global__ void embed_kernel(EmbedParams p) {
   int id = p.ids[t];
   id = min(max(id, 0), p.V - 1);
   const T* tok = static_cast<const T*>(p.tok) + (size_t)id * p.H;
-  const T* pos = p.pos ? static_cast<const T*>(p.pos) + (size_t)(t % p.S) * p.H : nullptr;
+  int prow = t % p.S;
+  if (p.pos_off) prow = min(max(prow + p.pos_off[(t / p.S) * p.pos_off_stride], 0), p.P - 1);
+  const T* pos = p.pos ? static_cast<const T*>(p.pos) + (size_t)prow * p.H : nullptr;
   T* y = static_cast<T*>(p.y) + (size_t)t * p.H;
   float* yf = static_cast<float*>(p.y) + (size_t)t * p.H;
   const bool wide = p.y_f32 && sizeof(T) == 2;

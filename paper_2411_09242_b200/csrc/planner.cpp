@@ -513,6 +513,7 @@ static void build_nodes(fluid_plan_s* p, const std::vector<int>& order) {
     switch (op.kind) {
       case FLUID_OP_EMBED:
         n.kind = N_EMBED; n.b = op.ins[1]; n.pos = op.ins.size() > 2 ? op.ins[2] : -1;
+        n.pos_off = op.ins.size() > 3 ? op.ins[3] : -1;
         break;
       case FLUID_OP_LINEAR:
       case FLUID_OP_BMM_QK:

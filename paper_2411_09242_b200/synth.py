@@ -363,16 +363,19 @@ class DecodeModel:
 
 def build_decode_model(cfg: ModelConfig, t_max: int, like: Model = None, weight_seed: int = WEIGHT_SEED,
                        materialize: bool = True, per_sequence_pos: bool = False) -> DecodeModel:
-    """The llama-family graph of ONE decoding step: B sequences, one new token each, the keys and
-    values of the earlier tokens in per-layer caches [B, t_max, nh, D] that the caller owns and the
-    step extends (STATE tensors). `pos` (int32 [1], or [B] with per_sequence_pos; on the device at run
-    time) is the number of tokens already cached, for all sequences or per sequence. Outputs: the final hidden state [B,1,H]
-    and the logits [B,1,V].
+    """The graph of ONE decoding step of a causal family ("llama": RMSNorm, rotary q/k, SwiGLU; "gpt": LayerNorm,
+    learned positions, biases, GELU, tied head): B sequences, one new token each, the keys and values of the
+    earlier tokens in per-layer caches [B, t_max, nh, D] that the caller owns and the step extends (STATE
+    tensors). `pos` (int32 [1], or [B] with per_sequence_pos; on the device at run time) is the number of tokens
+    already cached, for all sequences or per sequence. Outputs: the final hidden state [B,1,H] and the logits
+    [B,1,V].
 
-    like: a whole-sequence model of the same family and widths; its weights are taken over by name,
-    so that a run of decoding steps can be compared with that model on the same tokens.
+    like: a whole-sequence model of the same family and widths; its weights are taken over by name, so that a run
+    of decoding steps can be compared with that model on the same tokens.
     """
-    assert cfg.family == "llama", "decoding graphs are built for the rotary family only"
+    assert cfg.family in ("llama", "gpt"), "decoding graphs are built for the causal families"
+    rms = cfg.family == "llama"
+    pos_rows = like.cfg.S if like is not None else t_max    # rows of the learned position table (gpt)
     cfg = scaled(cfg, S=1)
     b = _Builder(cfg, weight_seed, materialize and like is None)
     g = b.g
@@ -381,17 +384,24 @@ def build_decode_model(cfg: ModelConfig, t_max: int, like: Model = None, weight_
     pos = g.tensor("pos", I32, [B if per_sequence_pos else 1], INPUT)
     tok = b.const("tok_table", [V, H])
     x = b.act("embed", [B, 1, H])
-    g.op(EMBED, [ids, tok], [x])
+    if rms:
+        g.op(EMBED, [ids, tok], [x])
+    else:
+        ptab = b.const("pos_table", [pos_rows, H])
+        g.op(EMBED, [ids, tok, ptab, pos], [x])
     caches = []
     for l in range(cfg.L):
         pfx = f"l{l}"
-        n = _norm(b, x, f"{pfx}.ln1", True)
+        n = _norm(b, x, f"{pfx}.ln1", rms)
         heads = {}
         for nm in ("q", "k", "v"):
             w = b.const(f"{pfx}.W{nm}", [H, nh, D])
+            ins = [n, w]
+            if not rms:
+                ins.append(b.const(f"{pfx}.b{nm}", [nh, D]))
             t = b.act(f"{pfx}.{nm}", [B, 1, nh, D])
-            g.op(LINEAR, [n, w], [t], contract=1)
-            if nm != "v":
+            g.op(LINEAR, ins, [t], contract=1)
+            if rms and nm != "v":
                 r = b.act(f"{pfx}.{nm}_rope", [B, 1, nh, D])
                 g.op(ROPE, [t, pos], [r], rope_base=10000.0, rope_interleaved=0)
                 t = r
@@ -402,14 +412,21 @@ def build_decode_model(cfg: ModelConfig, t_max: int, like: Model = None, weight_
         c = b.act(f"{pfx}.ctx", [B, 1, nh, D])
         g.op(CACHED_ATTENTION, [heads["q"], heads["k"], heads["v"], kc, vc, pos], [c], scale=1.0 / math.sqrt(D))
         wo = b.const(f"{pfx}.Wo", [nh, D, H])
+        ins = [c, wo]
+        if not rms:
+            ins.append(b.const(f"{pfx}.bo", [H]))
         o = b.act(f"{pfx}.attn_out", [B, 1, H])
-        g.op(LINEAR, [c, wo], [o], contract=2)
+        g.op(LINEAR, ins, [o], contract=2)
         a = b.act(f"{pfx}.res1", [B, 1, H]); g.op(ADD, [x, o], [a])
-        n = _norm(b, a, f"{pfx}.ln2", True)
-        o = _mlp_swiglu(b, n, pfx)
+        n = _norm(b, a, f"{pfx}.ln2", rms)
+        o = _mlp_swiglu(b, n, pfx) if rms else _mlp_gelu(b, n, pfx)
         x = b.act(f"{pfx}.res2", [B, 1, H]); g.op(ADD, [a, o], [x])
-    h = _norm(b, x, "final_norm", True, out_kind=OUTPUT)
-    wlm = b.const("W_lm", [H, V])
+    h = _norm(b, x, "final_norm", rms, out_kind=OUTPUT)
+    if rms:
+        wlm = b.const("W_lm", [H, V])
+    else:
+        wlm = b.act("tok_table_T", [H, V])
+        g.op(TRANSPOSE, [tok], [wlm], perm=[1, 0])
     logits = b.act("logits", [B, 1, V], OUTPUT)
     g.op(LINEAR, [h, wlm], [logits], contract=1)
     consts = b.consts

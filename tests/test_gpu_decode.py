@@ -105,15 +105,17 @@ def test_rope_with_a_position_read_on_the_device(dtype, D):
         plan.close()
 
 
-@pytest.mark.parametrize("dtype,kw", [
-    (synth.F32, dict(L=2, H=64, nh=4, F=96, B=2, V=100)),
-    (synth.BF16, dict(L=2, H=256, nh=4, F=384, B=3, V=500)),
-    (synth.BF16, dict(L=1, H=512, nh=4, F=1024, B=1, V=1000)),
+@pytest.mark.parametrize("family,dtype,kw", [
+    ("llama", synth.F32, dict(L=2, H=64, nh=4, F=96, B=2, V=100)),
+    ("llama", synth.BF16, dict(L=2, H=256, nh=4, F=384, B=3, V=500)),
+    ("llama", synth.BF16, dict(L=1, H=512, nh=4, F=1024, B=1, V=1000)),
+    ("gpt2_small", synth.F32, dict(L=2, H=64, nh=4, F=96, B=2, V=100)),
+    ("gpt2_small", synth.BF16, dict(L=2, H=256, nh=4, F=512, B=3, V=501)),
 ])
-def test_decoding_steps_of_a_small_model(dtype, kw):
+def test_decoding_steps_of_a_small_model(family, dtype, kw):
     """Several decoding steps in a row on one plan: the caches the device carries forward are its own; every
     step's logits are compared with the oracle run on the oracle's own caches."""
-    cfg = synth.scaled(synth.CONFIGS["llama"], dtype=dtype, S=1, **kw)
+    cfg = synth.scaled(synth.CONFIGS[family], dtype=dtype, S=1, **kw)
     t_max = 24
     dec = synth.build_decode_model(cfg, t_max)
     g = dec.graph
@@ -312,4 +314,20 @@ def test_decoding_with_ragged_lengths():
         assert runner.status() == 0
         for tid, got in zip(g.outputs, outs):
             helpers.assert_close(got, ref[tid], synth.BF16, f"ragged step {step} {g.tensors[tid]['name']}", tol=2e-2)
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", [synth.BF16, synth.F32])
+def test_embedding_with_a_position_read_on_the_device(dtype):
+    g = synth.GraphDesc()
+    ids = g.tensor("ids", synth.I32, [3, 2], synth.INPUT)
+    tok = g.tensor("tok", dtype, [50, 64], synth.CONST)
+    ptab = g.tensor("ptab", dtype, [40, 64], synth.CONST)
+    off = g.tensor("off", synth.I32, [3], synth.INPUT)
+    y = g.tensor("y", dtype, [3, 2, 64], synth.OUTPUT)
+    g.op(synth.EMBED, [ids, tok, ptab, off], [y])
+    feeds = {ids: synth.token_ids(1, 0, [3, 2], 50), tok: helpers.rand_feed([50, 64], dtype, 2), ptab: helpers.rand_feed([40, 64], dtype, 3),
+             off: np.array([0, 17, 38], dtype=np.int32)}
+    got, plan, _ = helpers.run_gpu(g, feeds)
+    helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], dtype, "embed with offsets")
     plan.close()

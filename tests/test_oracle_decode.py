@@ -89,10 +89,11 @@ def test_rope_with_an_offset_is_a_slice_of_the_whole_sequence():
             np.testing.assert_allclose(part, whole[:, p0:p0 + 3], rtol=1e-13, atol=1e-13)
 
 
-def test_decoding_steps_reproduce_the_whole_sequence_model():
+@pytest.mark.parametrize("family", ["llama", "gpt2_small"])
+def test_decoding_steps_reproduce_the_whole_sequence_model(family):
     """S decoding steps from empty caches give, at step t, the logits of the whole-sequence model run on the
-    first t+1 tokens; the caches end up holding the rotated keys and the values of the whole sequence."""
-    cfg = synth.scaled(synth.CONFIGS["llama"], dtype=synth.F32, L=2, H=32, nh=4, F=48, S=6, B=2, V=50)
+    first t+1 tokens; the caches end up holding the (rotated) keys and the values of the whole sequence."""
+    cfg = synth.scaled(synth.CONFIGS[family], dtype=synth.F32, L=2, H=32, nh=4, F=48, S=6, B=2, V=50)
     whole = synth.build_model(cfg)
     dec = synth.build_decode_model(cfg, t_max=8, like=whole)
     g = dec.graph
@@ -111,12 +112,12 @@ def test_decoding_steps_reproduce_the_whole_sequence_model():
         for tid in state:
             state[tid] = out[tid]
         logits = out[g.outputs[1]]
-        _, ref_logits = models.forward("llama", cfg.L, names, whole.ids[:, :t + 1])
+        _, ref_logits = models.forward(cfg.family, cfg.L, names, whole.ids[:, :t + 1])
         np.testing.assert_allclose(logits[:, 0], ref_logits, rtol=1e-9, atol=1e-12)
     vals = graph_exec.run_graph(whole.graph.tensors, whole.graph.ops, {**whole.consts, whole.graph.inputs[0]: whole.ids}, keep_all=True)
     by_name = {td["name"]: vals[t] for t, td in enumerate(whole.graph.tensors) if t in vals}
     for l, (kc, vc) in enumerate(dec.caches):
-        np.testing.assert_allclose(state[kc][:, :cfg.S], by_name[f"l{l}.k_rope"], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(state[kc][:, :cfg.S], by_name[f"l{l}.k_rope" if cfg.family == "llama" else f"l{l}.k"], rtol=1e-9, atol=1e-12)
         np.testing.assert_allclose(state[vc][:, :cfg.S], by_name[f"l{l}.v"], rtol=1e-9, atol=1e-12)
 
 
@@ -134,3 +135,14 @@ def test_positions_per_sequence_equal_each_sequence_alone():
     r = ops.rope(x, base=100.0, pos0=pos)
     for b in range(B):
         np.testing.assert_allclose(r[b:b + 1], ops.rope(x[b:b + 1], base=100.0, pos0=int(pos[b])), rtol=1e-14, atol=1e-14)
+
+
+def test_embedding_with_a_position_offset_is_a_slice_of_the_whole_sequence():
+    rng = np.random.default_rng(6)
+    tok, pos = rng.standard_normal((20, 8)), rng.standard_normal((12, 8))
+    ids = rng.integers(0, 20, size=(2, 12))
+    whole = ops.embed(ids, tok, pos)
+    for p0 in (0, 3, 9):
+        np.testing.assert_array_equal(ops.embed(ids[:, p0:p0 + 2], tok, pos, pos0=p0), whole[:, p0:p0 + 2])
+    both = ops.embed(np.stack([ids[0, 3:5], ids[1, 7:9]]), tok, pos, pos0=[3, 7])
+    np.testing.assert_array_equal(both, np.stack([whole[0, 3:5], whole[1, 7:9]]))
