@@ -58,7 +58,8 @@ def cases():
     x = g.tensor("x", BF, [16, 2048, 4096], synth.OUTPUT)
     g.op(synth.EMBED, [ids, tok], [x])
     out.append(("embed 32768x4096", g, lambda n: 2 * n * 2, None))
-    for (B_, nh, D, T) in ((4, 32, 128, 2048), (16, 32, 128, 4096), (4, 12, 64, 2048)):
+    # (128, 1, 128, 2048) moves the same bytes as (4, 32, 128, 2048) with every head's rows contiguous in memory
+    for (B_, nh, D, T) in ((4, 32, 128, 2048), (128, 1, 128, 2048), (16, 32, 128, 4096), (4, 12, 64, 2048)):
         g = synth.GraphDesc()
         q = g.tensor("q", BF, [B_, 1, nh, D], synth.INPUT)
         k = g.tensor("k", BF, [B_, 1, nh, D], synth.INPUT)
