@@ -287,6 +287,171 @@ __global__ void __launch_bounds__(256, (!EARLY && NCH <= 3) ? 5 : 1) norm_warp_k
   }
 }
 
+// Long inputs (many more rows than resident warps): persistent warps, each walking rows with the grid's stride. The
+// row's 16-byte pieces reach the lane that will use them through a lane-private ring of asynchronous copies in
+// shared memory (no barrier: a lane reads back only what it copied), so a warp has RING - 1 rows in flight while it
+// reduces and stores one, and the gain and bias are read once per warp instead of once per row.
+constexpr int NORM_RING = 4;
+__device__ __forceinline__ void norm_cp16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+// sum over the WPR warps that share a row (named barrier per row group; `red` alternates between two sets of slots
+// so that a fast warp's next sum cannot overwrite what a slow warp has not read yet)
+template <int WPR>
+__device__ __forceinline__ float ring_row_sum(float v, float* red, int slot, int warp, int lane) {
+  v = warp_sum(v);
+  if (WPR == 1) return v;
+  if (lane == 0) red[slot * 8 + warp] = v;
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + warp / WPR), "r"(WPR * 32) : "memory");
+  float t = 0.f;
+  const int g0 = warp / WPR * WPR;
+#pragma unroll
+  for (int i = 0; i < WPR; ++i) t += red[slot * 8 + g0 + i];
+  return t;
+}
+
+template <typename T, int NCH, int WPR, bool XF32>
+__global__ void __launch_bounds__(256, 2) norm_ring_kernel(NormParams p) {
+  __shared__ float red[4 * 8];
+  constexpr int V = VecOf<T>::N;                      // elements per chunk (a lane's unit of work)
+  constexpr int PCS = (XF32 && sizeof(T) == 2) ? 2 : 1;   // 16-byte pieces per chunk in the ring
+  constexpr int SLOT = NCH * PCS * 512;               // bytes per row and warp
+  extern __shared__ __align__(16) unsigned char norm_ring_raw[];
+  pdl_launch_dependents();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nch = p.width / V;
+  const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(norm_ring_raw)) + uint32_t(warp) * (NORM_RING * SLOT) + uint32_t(lane) * 16;
+  const T* gamma = static_cast<const T*>(p.gamma);
+  const T* beta = static_cast<const T*>(p.beta);
+  const int c_first = (warp % WPR) * 32 + lane;
+  float gv[NCH][V], bv[NCH][V];
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const int c = c_first + 32 * WPR * j;
+#pragma unroll
+    for (int i = 0; i < V; ++i) { gv[j][i] = 0.f; bv[j][i] = 0.f; }
+    if (c < nch) {
+      norm_load<T, V>(gamma, false, 0, c, gv[j]);
+      if (beta) norm_load<T, V>(beta, false, 0, c, bv[j]);
+    }
+  }
+  constexpr int RPB = 8 / WPR;   // rows per CTA and pass
+  const int64_t stride = (int64_t)gridDim.x * RPB;
+  const int64_t row0 = (int64_t)blockIdx.x * RPB + warp / WPR;
+  const int64_t n_mine = row0 < p.rows ? (p.rows - row0 + stride - 1) / stride : 0;
+  auto fill = [&](int64_t i) {
+    if (i >= n_mine) return;
+    const size_t roff = (size_t)(row0 + i * stride) * p.width;
+    const uint32_t dst = ring + uint32_t(i % NORM_RING) * SLOT;
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      const int c = c_first + 32 * WPR * j;
+      if (c < nch) {
+        if (PCS == 2) {
+          const float* src = static_cast<const float*>(p.x) + roff + (size_t)c * V;
+          norm_cp16(dst + (2 * j) * 512, src);
+          norm_cp16(dst + (2 * j + 1) * 512, src + 4);
+        } else {
+          norm_cp16(dst + j * 512, static_cast<const unsigned char*>(p.x) + (roff + (size_t)c * V) * (XF32 ? 4 : sizeof(T)));
+        }
+      }
+    }
+  };
+  pdl_wait();
+  for (int i = 0; i < NORM_RING - 1; ++i) {
+    fill(i);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  T* y_lo = static_cast<T*>(p.y_lo);
+#pragma unroll 1
+  for (int64_t i = 0; i < n_mine; ++i) {
+    asm volatile("cp.async.wait_group %0;" ::"n"(NORM_RING - 2) : "memory");
+    const uint32_t src = ring + uint32_t(i % NORM_RING) * SLOT;
+    float v[NCH][V];
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      const int c = c_first + 32 * WPR * j;
+#pragma unroll
+      for (int q = 0; q < V; ++q) v[j][q] = 0.f;
+      if (c < nch) {
+        if (XF32 || sizeof(T) == 4) {
+#pragma unroll
+          for (int h = 0; h < PCS; ++h) {
+            uint4 w;
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w) : "r"(src + (PCS * j + h) * 512) : "memory");
+            v[j][4 * h] = __uint_as_float(w.x); v[j][4 * h + 1] = __uint_as_float(w.y);
+            v[j][4 * h + 2] = __uint_as_float(w.z); v[j][4 * h + 3] = __uint_as_float(w.w);
+          }
+        } else {
+          uint4 w;
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w) : "r"(src + j * 512) : "memory");
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            v[j][2 * q] = __uint_as_float(ww[q] << 16);
+            v[j][2 * q + 1] = __uint_as_float(ww[q] & 0xffff0000u);
+          }
+        }
+#pragma unroll
+        for (int q = 0; q < V; ++q) s += p.rms ? v[j][q] * v[j][q] : v[j][q];
+      }
+    }
+    fill(i + NORM_RING - 1);   // refills the slot read one pass ago
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    const int par = int(i & 1) * 2;
+    s = ring_row_sum<WPR>(s, red, par, warp, lane);
+    float mean = 0.f, rstd;
+    if (p.rms) {
+      rstd = rsqrtf(s / p.width + p.eps);
+    } else {
+      mean = s / p.width;
+      float q2 = 0.f;
+#pragma unroll
+      for (int j = 0; j < NCH; ++j)
+        if (c_first + 32 * WPR * j < nch) {
+#pragma unroll
+          for (int q = 0; q < V; ++q) q2 += (v[j][q] - mean) * (v[j][q] - mean);
+        }
+      q2 = ring_row_sum<WPR>(q2, red, par + 1, warp, lane);
+      rstd = rsqrtf(q2 / p.width + p.eps);
+    }
+    const size_t roff = (size_t)(row0 + i * stride) * p.width;
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      const int c = c_first + 32 * WPR * j;
+      if (c < nch) {
+        float o[V];
+#pragma unroll
+        for (int q = 0; q < V; ++q) o[q] = (v[j][q] - mean) * rstd * gv[j][q] + bv[j][q];
+        if (y_lo) {
+          float t8[VecOf<T>::N];
+#pragma unroll
+          for (int q = 0; q < V; ++q) t8[q] = o[q];
+          store16(y_lo + roff + (size_t)c * V, t8);
+        }
+        if (p.y_hi) {
+#pragma unroll
+          for (int q = 0; q < V; q += 4)
+            *reinterpret_cast<float4*>(p.y_hi + roff + (size_t)c * V + q) = make_float4(o[q], o[q + 1], o[q + 2], o[q + 3]);
+        }
+      }
+    }
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+template <typename T, int NCH, int WPR, bool XF32>
+static cudaError_t norm_ring_launch(const NormParams& p, cudaStream_t st) {
+  constexpr int PCS = (XF32 && sizeof(T) == 2) ? 2 : 1;
+  constexpr int smem = 8 * NORM_RING * NCH * PCS * 512;
+  static const cudaError_t attr = cudaFuncSetAttribute(norm_ring_kernel<T, NCH, WPR, XF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (attr != cudaSuccess) return attr;
+  const int per_sm = std::max(1, std::min(2, (200 * 1024) / smem));   // two CTAs per SM by registers
+  return launch_k(norm_ring_kernel<T, NCH, WPR, XF32>, 148u * per_sm, 256, smem, st, p);
+}
+
 template <typename T>
 static cudaError_t norm_t(const NormParams& p, cudaStream_t st) {
   constexpr int V = VecOf<T>::N;
@@ -299,6 +464,23 @@ static cudaError_t norm_t(const NormParams& p, cudaStream_t st) {
     const int per_lane = (nch + 32 * wpr - 1) / (32 * wpr);
     const unsigned grid = (unsigned)((p.rows + 8 / wpr - 1) / (8 / wpr));
     const bool early = grid <= 148u * 2u;
+    // many more rows than resident warps, no second addend: the persistent ring kernel
+    // (with fewer rows per warp the ring never fills: measured slower on the 2048- and 4096-row norms of the model steps)
+    if (!p.res && (int64_t)p.rows * wpr >= 148 * 2 * 8 * 8 && (sizeof(T) == 2 || !p.x_f32)) {
+      const bool xf = p.x_f32 && sizeof(T) == 2;
+#define NR_LAUNCH(N, W) return xf ? norm_ring_launch<T, N, W, true>(p, st) : norm_ring_launch<T, N, W, false>(p, st)
+#define NR_PICK(W)                  \
+  if (per_lane <= 1) NR_LAUNCH(1, W); \
+  if (per_lane <= 2) NR_LAUNCH(2, W); \
+  if (per_lane <= 3) NR_LAUNCH(3, W); \
+  NR_LAUNCH(4, W)
+      if (wpr == 1) { NR_PICK(1); }
+      if (wpr == 2) { NR_PICK(2); }
+      if (wpr == 4) { NR_PICK(4); }
+      NR_PICK(8);
+#undef NR_PICK
+#undef NR_LAUNCH
+    }
 #define NW_LAUNCH(N, W) return early ? launch_k(norm_warp_kernel<T, N, W, true>, grid, 256, 0, st, p) \
                                      : launch_k(norm_warp_kernel<T, N, W, false>, grid, 256, 0, st, p)
 #define NW_PICK(W)              \

@@ -388,3 +388,48 @@ def test_plan_from_measured_costs(family, dtype):
     plan2 = fluid.Plan(m.graph, cands, eval=ev.callback)
     assert ev.measured == before and plan2.cost == plan.cost
     plan.close(); plan2.close()
+
+
+@pytest.mark.parametrize("kind,dtype,rows,width", [
+    (synth.LAYERNORM, synth.BF16, 20001, 768),
+    (synth.RMSNORM, synth.BF16, 19000, 1024),
+    (synth.LAYERNORM, synth.BF16, 19500, 200),
+    (synth.LAYERNORM, synth.F32, 19001, 256),
+    (synth.RMSNORM, synth.F32, 19000, 500),
+    (synth.RMSNORM, synth.BF16, 5001, 4096),      # a row shared by four warps
+    (synth.LAYERNORM, synth.BF16, 9999, 2048),    # by two
+    (synth.LAYERNORM, synth.F32, 5000, 2048),     # fp32: by four
+    (synth.RMSNORM, synth.BF16, 2501, 8192),      # by eight
+])
+def test_norm_over_many_rows(kind, dtype, rows, width):
+    """Inputs with many more rows than resident warps take the persistent kernel (rows walked with the grid's stride,
+    pieces prefetched through a per-lane ring); ragged row counts and widths that leave lanes idle included."""
+    shapes = [[1, rows, width], [width]] + ([[width]] if kind == synth.LAYERNORM else [])
+    g = single_op_graph(kind, shapes, [1, rows, width], dtype, {"eps": 1e-5})
+    feeds = {0: rand_feed(shapes[0], dtype, 1, -3, 3), 1: rand_feed([width], dtype, 2, 0.5, 1.5)}
+    if kind == synth.LAYERNORM:
+        feeds[2] = rand_feed([width], dtype, 3)
+    got, plan, _ = run_gpu(g, feeds)
+    out = g.outputs[0]
+    assert_close(got[out], run_oracle(g, feeds)[out], dtype, "norm, many rows")
+    plan.close()
+
+
+def test_norm_over_many_rows_reading_the_fp32_stream():
+    """EMBED -> LAYERNORM over 20480 tokens: the embedding is held in fp32 (it feeds a normalisation only), so the
+    persistent kernel reads 32-byte chunks through its ring."""
+    g = synth.GraphDesc()
+    ids = g.tensor("ids", synth.I32, [10, 2048], synth.INPUT)
+    tok = g.tensor("tok", synth.BF16, [1000, 768], synth.CONST)
+    x = g.tensor("x", synth.BF16, [10, 2048, 768], synth.ACT)
+    gam = g.tensor("gamma", synth.BF16, [768], synth.CONST)
+    bet = g.tensor("beta", synth.BF16, [768], synth.CONST)
+    y = g.tensor("y", synth.BF16, [10, 2048, 768], synth.OUTPUT)
+    g.op(synth.EMBED, [ids, tok], [x])
+    g.op(synth.LAYERNORM, [x, gam, bet], [y], eps=1e-5)
+    feeds = {ids: synth.token_ids(4, 0, [10, 2048], 1000), tok: rand_feed([1000, 768], synth.BF16, 5, -2, 2),
+             gam: rand_feed([768], synth.BF16, 6, 0.5, 1.5), bet: rand_feed([768], synth.BF16, 7)}
+    got, plan, _ = run_gpu(g, feeds)
+    assert plan.tensor_info(x).bytes >= 10 * 2048 * 768 * 4     # held in fp32
+    assert_close(got[y], run_oracle(g, feeds)[y], synth.BF16, "embed -> layernorm")
+    plan.close()
