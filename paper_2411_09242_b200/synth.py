@@ -214,7 +214,7 @@ class _Builder:
         return self.g.tensor(name, self.cfg.dtype, dims, kind)
 
 
-def _attention(b: _Builder, x, pfx, causal, bias, rope):
+def _attention(b: _Builder, x, pfx, causal, bias, rope, emit_kv=False):
     cfg, g = b.cfg, b.g
     B, S, H, nh, D = cfg.B, cfg.S, cfg.H, cfg.nh, cfg.D
     heads = {}
@@ -223,10 +223,13 @@ def _attention(b: _Builder, x, pfx, causal, bias, rope):
         ins = [x, w]
         if bias:
             ins.append(b.const(f"{pfx}.b{nm}", [nh, D]))
-        t = b.act(f"{pfx}.{nm}", [B, S, nh, D])
+        # emit_kv: the keys (after the rotary embedding, if any) and the values are graph outputs, in the layout of a
+        # key/value cache, so that decoding steps can continue from them
+        kv_out = emit_kv and nm in ("k", "v")
+        t = b.act(f"{pfx}.{nm}", [B, S, nh, D], OUTPUT if kv_out and not (rope and nm == "k") else ACT)
         g.op(LINEAR, ins, [t], contract=1)
         if rope and nm in ("q", "k"):
-            r = b.act(f"{pfx}.{nm}_rope", [B, S, nh, D])
+            r = b.act(f"{pfx}.{nm}_rope", [B, S, nh, D], OUTPUT if kv_out else ACT)
             g.op(ROPE, [t], [r], rope_base=10000.0, rope_interleaved=0)
             t = r
         heads[nm] = t
@@ -290,7 +293,7 @@ def _mlp_swiglu(b: _Builder, x, pfx):
 
 
 def build_model(cfg: ModelConfig, weight_seed: int = WEIGHT_SEED, token_seed: int = TOKEN_SEED,
-                materialize: bool = True) -> Model:
+                materialize: bool = True, emit_kv: bool = False) -> Model:
     """Graph + seeded weights + token ids for one configuration.
 
     Wiring (generic public architecture families):
@@ -298,6 +301,8 @@ def build_model(cfg: ModelConfig, weight_seed: int = WEIGHT_SEED, token_seed: in
       gpt    : x0 = embed; per layer x += attn(LN(x)); x += ffn(LN(x)); h = LN(x);
                outputs h and last-token logits against the tied token table.
       llama  : as gpt with RMSNorm, rotary q/k, bias-free linears, SwiGLU, separate LM head.
+    emit_kv (causal families): every layer's keys and values [B,S,nh,D] are extra graph outputs (declared before the
+    hidden state and the logits), the prompt's contribution to a key/value cache.
     Attention is written the way exported graphs spell it: per-head tensors are produced by
     explicit TRANSPOSE ops, which the planner may turn into zero-copy views.
     """
@@ -329,7 +334,7 @@ def build_model(cfg: ModelConfig, weight_seed: int = WEIGHT_SEED, token_seed: in
         for l in range(cfg.L):
             pfx = f"l{l}"
             n = _norm(b, x, f"{pfx}.ln1", rms)
-            o = _attention(b, n, pfx, causal=True, bias=not rms, rope=rms)
+            o = _attention(b, n, pfx, causal=True, bias=not rms, rope=rms, emit_kv=emit_kv)
             a = b.act(f"{pfx}.res1", [B, S, H]); g.op(ADD, [x, o], [a])
             n = _norm(b, a, f"{pfx}.ln2", rms)
             o = _mlp_swiglu(b, n, pfx) if rms else _mlp_gelu(b, n, pfx)

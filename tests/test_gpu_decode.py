@@ -331,3 +331,50 @@ def test_embedding_with_a_position_read_on_the_device(dtype):
     got, plan, _ = helpers.run_gpu(g, feeds)
     helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], dtype, "embed with offsets")
     plan.close()
+
+
+@pytest.mark.parametrize("family", ["llama", "gpt2_small"])
+def test_prefill_then_decode_continues_the_sequence(family):
+    """A prompt goes through the whole-sequence graph, whose keys and values are graph outputs; they are copied into the
+    caches and the next tokens are decoded one by one. Every step's logits are compared with the oracle's direct
+    whole-sequence formulas on the prefix so far."""
+    import torch
+    from oracle import models
+    S0, S1, t_max = 12, 16, 20
+    base = synth.scaled(synth.CONFIGS[family], dtype=synth.BF16, L=2, H=256, nh=4, F=512, B=2, V=300)
+    whole = synth.build_model(synth.scaled(base, S=S1))                  # weights and tokens of the full sequence
+    by_name = {whole.graph.tensors[t]["name"]: a for t, a in whole.consts.items()}
+    pre = synth.build_model(synth.scaled(base, S=S0), materialize=False, emit_kv=True)
+    pre_consts = {t: (by_name[td["name"]][:S0] if td["name"] == "pos_table" else by_name[td["name"]])
+                  for t, td in enumerate(pre.graph.tensors) if td["kind"] == synth.CONST}
+    helpers.ensure_lib()
+    pplan = fluid.Plan(pre.graph, synth.default_candidates(pre.graph))
+    prun = fluid.Runner(pplan, pre_consts, poison=True)
+    prun.set_inputs([whole.ids[:, :S0]])
+    prun.run()
+    assert prun.status() == 0
+    outs = dict(zip(pre.graph.outputs, prun.outputs))
+    names = {pre.graph.tensors[t]["name"]: t for t in pre.graph.outputs}
+    _, ref_logits = models.forward(base.family, base.L, by_name, whole.ids[:, :S0])
+    helpers.assert_close(outs[names["logits"]].float().cpu().numpy(), ref_logits, synth.BF16, "prompt logits", tol=2e-2)
+
+    dec = synth.build_decode_model(synth.scaled(base, S=S1), t_max, like=whole)
+    g = dec.graph
+    dplan = fluid.Plan(g, synth.default_candidates(g))
+    drun = fluid.Runner(dplan, dec.consts, poison=True)
+    for l, (kc, vc) in enumerate(dec.caches):
+        kname = f"l{l}.k_rope" if base.family == "llama" else f"l{l}.k"
+        for cache, name in ((kc, kname), (vc, f"l{l}.v")):
+            buf = drun.inputs[g.inputs.index(cache)]
+            buf.fill_(float("nan"))
+            buf[:, :S0].copy_(outs[names[name]])
+    for t in range(S0, S1):
+        drun.inputs[g.inputs.index(dec.ids)].copy_(torch.from_numpy(np.ascontiguousarray(whole.ids[:, t:t + 1])))
+        drun.inputs[g.inputs.index(dec.pos)].fill_(t)
+        drun.run()
+        logits = drun.outputs[1].float().cpu().numpy()
+        assert drun.status() == 0
+        _, ref_logits = models.forward(base.family, base.L, by_name, whole.ids[:, :t + 1])
+        helpers.assert_close(logits[:, 0], ref_logits, synth.BF16, f"decoded token {t}", tol=2e-2)
+    pplan.close()
+    dplan.close()
