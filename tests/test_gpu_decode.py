@@ -378,3 +378,82 @@ def test_prefill_then_decode_continues_the_sequence(family):
         helpers.assert_close(logits[:, 0], ref_logits, synth.BF16, f"decoded token {t}", tol=2e-2)
     pplan.close()
     dplan.close()
+
+
+def test_cached_attention_random_shapes():
+    """Seeded random sweep: head dims, grouped heads, batch sizes (hence cluster sizes), cache lengths, positions shared
+    or per sequence, both dtypes."""
+    rng = np.random.default_rng(20241125)
+    helpers.ensure_lib()
+    for it in range(24):
+        dtype = synth.BF16 if rng.random() < 0.7 else synth.F32
+        vec = 8 if dtype == synth.BF16 else 4
+        D = min(128, int(vec * rng.choice([1, 2, 4, 8, 16])))
+        nkv = int(rng.choice([1, 2, 3, 4, 8]))
+        nh = nkv * int(rng.choice([1, 2, 4]))
+        B, Tmax, per_seq = int(rng.integers(1, 40)), int(rng.integers(1, 700)), bool(rng.random() < 0.5)
+        g = synth.GraphDesc()
+        q = g.tensor("q", dtype, [B, 1, nh, D], synth.INPUT)
+        k = g.tensor("k", dtype, [B, 1, nkv, D], synth.INPUT)
+        v = g.tensor("v", dtype, [B, 1, nkv, D], synth.INPUT)
+        kc = g.tensor("kc", dtype, [B, Tmax, nkv, D], synth.STATE)
+        vc = g.tensor("vc", dtype, [B, Tmax, nkv, D], synth.STATE)
+        pos = g.tensor("pos", synth.I32, [B if per_seq else 1], synth.INPUT)
+        out = g.tensor("o", dtype, [B, 1, nh, D], synth.OUTPUT)
+        g.op(synth.CACHED_ATTENTION, [q, k, v, kc, vc, pos], [out], scale=1 / math.sqrt(D))
+        feeds = {q: helpers.rand_feed([B, 1, nh, D], dtype, it, -2, 2), k: helpers.rand_feed([B, 1, nkv, D], dtype, it + 1000, -2, 2),
+                 v: helpers.rand_feed([B, 1, nkv, D], dtype, it + 2000), kc: helpers.rand_feed([B, Tmax, nkv, D], dtype, it + 3000, -2, 2),
+                 vc: helpers.rand_feed([B, Tmax, nkv, D], dtype, it + 4000),
+                 pos: rng.integers(0, Tmax, size=(B if per_seq else 1)).astype(np.int32)}
+        got, plan, runner = helpers.run_gpu(g, feeds, synth.default_candidates(g))
+        ref = helpers.run_oracle(g, feeds)
+        what = f"case {it}: D {D} nh {nh} nkv {nkv} B {B} Tmax {Tmax} per_seq {per_seq}"
+        helpers.assert_close(got[out], ref[out], dtype, what)
+        assert np.array_equal(runner.inputs[g.inputs.index(kc)].float().cpu().numpy(), ref[kc]), what
+        assert np.array_equal(runner.inputs[g.inputs.index(vc)].float().cpu().numpy(), ref[vc]), what
+        plan.close()
+
+
+def test_few_row_linear_random_shapes():
+    """Seeded random sweep of LINEAR with 1 to 8 rows: ragged N and K, bias / GELU / residual epilogues, and the RMS
+    normalisation folded in."""
+    rng = np.random.default_rng(2411)
+    helpers.ensure_lib()
+    for it in range(24):
+        M, N, K = int(rng.integers(1, 9)), int(rng.integers(1, 5000)), 8 * int(rng.integers(1, 600))
+        bias, act, res, rms = (bool(rng.random() < p) for p in (0.5, 0.3, 0.5, 0.4))
+        g = synth.GraphDesc()
+        x = g.tensor("x", synth.BF16, [M, K], synth.INPUT)
+        feeds = {x: helpers.rand_feed([M, K], synth.BF16, it)}
+        a = x
+        if rms:
+            gam = g.tensor("gam", synth.BF16, [K], synth.CONST)
+            feeds[gam] = helpers.rand_feed([K], synth.BF16, it + 50, 0.5, 1.5)
+            a = g.tensor("n", synth.BF16, [M, K], synth.ACT)
+            g.op(synth.RMSNORM, [x, gam], [a], eps=1e-5)
+        w = g.tensor("w", synth.BF16, [K, N], synth.CONST)
+        feeds[w] = synth.round_bf16(synth.normal(7, it, [K, N], 0.05))
+        ins = [a, w]
+        if bias:
+            b = g.tensor("b", synth.BF16, [N], synth.CONST)
+            ins.append(b)
+            feeds[b] = helpers.rand_feed([N], synth.BF16, it + 100)
+        y = g.tensor("y", synth.BF16, [M, N], synth.ACT if (act or res) else synth.OUTPUT)
+        g.op(synth.LINEAR, ins, [y], contract=1)
+        if act:
+            a2 = g.tensor("a2", synth.BF16, [M, N], synth.ACT if res else synth.OUTPUT)
+            g.op(synth.GELU, [y], [a2], gelu_tanh=0)
+            y = a2
+        if res:
+            r = g.tensor("r", synth.BF16, [M, N], synth.INPUT)
+            feeds[r] = helpers.rand_feed([M, N], synth.BF16, it + 200)
+            o = g.tensor("o", synth.BF16, [M, N], synth.OUTPUT)
+            g.op(synth.ADD, [y, r], [o])
+            y = o
+        got, plan, _ = helpers.run_gpu(g, feeds, synth.default_candidates(g))
+        steps = plan.steps()
+        assert "GEMM_ROWS" in [s["kernel_name"] for s in steps]
+        if rms:
+            assert len(steps) == 1 and (steps[0]["variant"] >> 30) & 1      # one launch: norm, GEMM and epilogue
+        helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], synth.BF16, f"case {it}: {M}x{N}x{K} bias {bias} act {act} res {res} rms {rms}")
+        plan.close()
