@@ -115,7 +115,7 @@ int finalize_steps(fluid_plan_s* p) {
             s.variant = (n_gemm > 1 ? int(n_gemm) << 20 : 0) | (s.swiglu ? 1 << 29 : 0) | (s.norm_fused ? 1 << 30 : 0);
             if (s.norm_fused) {
               const Node& nn = p->nodes[s.nodes.back()];
-              s.t_ptr[5] = nn.a; s.t_ptr[6] = nn.gamma;
+              s.t_ptr[5] = nn.a; s.t_ptr[6] = nn.gamma; s.t_ptr[7] = nn.beta;
               s.norm_eps = (float)nn.eps;
               s.norm_x_f32 = p->wide[nn.a];
             }
@@ -473,7 +473,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
         const int ng = s.swiglu ? 2 : (int)s.nodes.size() - s.norm_fused;
         RowsNorm rn{};
         if (s.norm_fused) {
-          rn.x = R(s.t_ptr[5]); rn.gamma = R(s.t_ptr[6]); rn.eps = s.norm_eps; rn.x_f32 = s.norm_x_f32;
+          rn.x = R(s.t_ptr[5]); rn.gamma = R(s.t_ptr[6]); rn.beta = R(s.t_ptr[7]); rn.eps = s.norm_eps; rn.x_f32 = s.norm_x_f32;
         }
         gs[0].A = s.norm_fused ? rn.x : R(s.t_ptr[0], 1); gs[0].B = R(s.t_ptr[1], 1); gs[0].C = const_cast<void*>(R(s.t_ptr[2]));
         gs[0].bias = R(s.t_ptr[3]); gs[0].R = R(s.t_ptr[4]);

@@ -50,7 +50,8 @@ struct RowsParams {
   const void* X;           // bf16, or fp32 when x_f32
   int M, N, K, M0, N0;
   int64_t a_s2, a_s3;      // activation row strides of the two-level m index
-  const __nv_bfloat16* gamma;   // fused RMS normalisation: the gain (else null)
+  const __nv_bfloat16* gamma;   // fused normalisation: the gain (else null)
+  const __nv_bfloat16* beta;    // fused LayerNorm: the bias (null: RMS normalisation)
   float eps;
   int x_f32;
   float scale;
@@ -100,7 +101,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int pitch = p.K + kXPad;                   // staged activation row, bf16 elements
   __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);
-  unsigned char* after_x = smem_raw + size_t(p.M) * pitch * 2;
+  const int ln = p.beta ? 1 : 0;                   // LayerNorm: one more staged row (the bias), see below
+  unsigned char* after_x = smem_raw + size_t(p.M + ln) * pitch * 2;
   const uint32_t ring0 = static_cast<uint32_t>(__cvta_generic_to_shared(after_x));
   float(*red)[16][9] = reinterpret_cast<float(*)[16][9]>(after_x + kWarps * ST * 1024);   // [warp][row][m]
   float* rstd = reinterpret_cast<float*>(after_x + kWarps * ST * 1024 + kWarps * 16 * 9 * sizeof(float));   // [8]
@@ -114,8 +116,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
   const int blk0 = ks * per;
   const uint32_t my_ring = ring0 + uint32_t(warp) * (ST * 1024) + uint32_t(lane) * 16;
   auto slot = [&](int i, int piece) { return my_ring + uint32_t(i % ST) * 1024 + uint32_t(piece) * 512; };
-  const uint32_t xs_lane = static_cast<uint32_t>(__cvta_generic_to_shared(xs)) + uint32_t((g < p.M ? g : 0) * pitch + t * 8) * 2;
-  const bool x_live = g < p.M;
+  const uint32_t xs_lane = static_cast<uint32_t>(__cvta_generic_to_shared(xs)) + uint32_t((g < p.M + ln ? g : 0) * pitch + t * 8) * 2;
+  const bool x_live = g < p.M + ln;
 
   for (int round = 0; round < p.rounds; ++round) {
     // units are dealt out evenly: a CTA takes p.upc <= UMAX of them per round, so that every SM streams
@@ -158,6 +160,46 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
       }
       // ---- stage the activations: thread -> 8 consecutive k of one row ----
       const int chunks = p.K / 8;
+      // LayerNorm: ((x - mean) * rstd * gamma + beta) . W = rstd * (((x - mean) * gamma) . W) + beta . W. The rows are
+      // centred and multiplied by the gain here; the bias rides along as one more activation row (an MMA column that
+      // would otherwise be idle), so beta . W comes out of the same accumulators.
+      float mean[8];
+#pragma unroll
+      for (int m = 0; m < 8; ++m) mean[m] = 0.f;
+      if (ln) {
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          float sm = 0.f;
+          if (m < p.M) {
+            const int64_t roff = split2(m, p.M0, p.a_s2, p.a_s3);
+            for (int c = threadIdx.x; c < chunks; c += kWarps * 32) {
+              float xf[8];
+              if (p.x_f32) {
+                const float4 lo = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + roff + c * 8);
+                const float4 hi = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + roff + c * 8 + 4);
+                xf[0] = lo.x; xf[1] = lo.y; xf[2] = lo.z; xf[3] = lo.w; xf[4] = hi.x; xf[5] = hi.y; xf[6] = hi.z; xf[7] = hi.w;
+              } else {
+                load16(static_cast<const __nv_bfloat16*>(p.X) + roff + c * 8, xf);
+              }
+#pragma unroll
+              for (int i = 0; i < 8; ++i) sm += xf[i];
+            }
+          }
+          sm = warp_sum(sm);
+          if (lane == 0) ssq_part[warp * 8 + m] = sm;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          float tot = 0.f;
+          for (int w = 0; w < kWarps; ++w) tot += ssq_part[w * 8 + m];
+          mean[m] = tot / p.K;
+        }
+        __syncthreads();   // the slots are reused for the sums of squares
+        for (int c = threadIdx.x; c < chunks + kXPad / 8; c += kWarps * 32)
+          *reinterpret_cast<uint4*>(xs + size_t(p.M) * pitch + c * 8) =
+              c < chunks ? *reinterpret_cast<const uint4*>(p.beta + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+      }
       float ssq[8];
 #pragma unroll
       for (int m = 0; m < 8; ++m) {
@@ -183,6 +225,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
               load16(p.gamma + c * 8, gf);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
+                xf[i] -= mean[m];
                 acc = fmaf(xf[i], xf[i], acc);
                 xf[i] *= gf[i];
               }
@@ -246,6 +289,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
         for (int q = 0; q < KS; ++q) u += red[(tl * NG + 1) * KS + q][nl][m];
         v = silu(v) * (u * sc);
       }
+      if (ln) {   // + beta . W
+        float bw = 0.f;
+#pragma unroll
+        for (int q = 0; q < KS; ++q) bw += red[tl * NG * KS + q][nl][p.M];
+        v = fmaf(bw, p.scale, v);
+      }
       const RowsGroup& og = p.g[SWIGLU ? 0 : u / p.tiles];
       if (og.has_bias) v += __bfloat162float(og.bias[n]);
       if (og.act == ACT_GELU_ERF) v = gelu_erf(v);
@@ -268,7 +317,7 @@ inline size_t rows_fixed_smem(int M, int K) {
 
 template <int KS, int ST, bool SWIGLU>
 cudaError_t launch_rows(RowsParams& p, int n_group, cudaStream_t st) {
-  const size_t smem = rows_fixed_smem(p.M, p.K) + size_t(kWarps) * ST * 1024;
+  const size_t smem = rows_fixed_smem(p.M + (p.beta ? 1 : 0), p.K) + size_t(kWarps) * ST * 1024;
   static const cudaError_t attr =
       cudaFuncSetAttribute(gemm_rows_kernel<KS, ST, SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
   if (attr != cudaSuccess) return attr;
@@ -324,6 +373,8 @@ cudaError_t launch_gemm_rows(const GemmParams* gs, int n_group, cudaStream_t st,
   p.X = norm ? norm->x : g0.A;
   p.x_f32 = norm ? norm->x_f32 : 0;
   p.gamma = norm ? static_cast<const __nv_bfloat16*>(norm->gamma) : nullptr;
+  p.beta = norm ? static_cast<const __nv_bfloat16*>(norm->beta) : nullptr;
+  if (p.beta && (swiglu || g0.M > 7 || !al16(p.beta))) return cudaErrorInvalidValue;
   p.eps = norm ? norm->eps : 0.f;
   p.M = g0.M; p.N = g0.N; p.K = g0.K; p.M0 = g0.M0; p.N0 = g0.N0;
   p.a_s2 = g0.a_s[2]; p.a_s3 = g0.a_s[3];
@@ -347,7 +398,9 @@ cudaError_t launch_gemm_rows(const GemmParams* gs, int n_group, cudaStream_t st,
   p.tiles = (p.N + 15) / 16;
   // ring depth: what the staged activations leave (one 16-byte piece per lane, row and stage; wider pieces measured
   // three times slower: a copy instruction of the warp then touches every 32-byte sector half)
-  const size_t left = size_t(kSmemBudget) - rows_fixed_smem(p.M, p.K);
+  const size_t fixed = rows_fixed_smem(p.M + (p.beta ? 1 : 0), p.K);
+  if (fixed + size_t(kWarps) * 6 * 1024 > size_t(kSmemBudget)) return cudaErrorInvalidValue;
+  const size_t left = size_t(kSmemBudget) - fixed;
   if (left >= size_t(kWarps) * 10 * 1024) return launch_rows_ks<10>(p, n_group, swiglu != 0, st);
   return launch_rows_ks<6>(p, n_group, swiglu != 0, st);
 }

@@ -181,11 +181,12 @@ struct AttnDecodeParams {
 // GEMM with at most 8 rows and both operands k-contiguous (bf16): the weights stream through registers once.
 // n_group (1..3) sibling GEMMs that share A and the shapes run as one launch. swiglu (two groups: gate, up): the launch
 // writes SiLU(gate) * up to g[0].C and nothing else.
-// norm (optional): the RMS normalisation in front of the GEMMs runs inside the launch: A is then x (bf16, or fp32 when
+// norm (optional): the RMS normalisation or (M <= 7, no swiglu) LayerNorm in front of the GEMMs runs inside the launch: A is then x (bf16, or fp32 when
 // x_f32) with the strides of g[0]'s A operand, and the normalised tensor is never stored.
 struct RowsNorm {
   const void* x;
   const void* gamma;
+  const void* beta;   // LayerNorm's bias; null for an RMS normalisation
   float eps;
   int x_f32;
 };

@@ -1059,7 +1059,7 @@ static int lower_and_place(fluid_plan_s* p) {
       p->steps.erase(p->steps.begin() + si + 1);
     }
   }
-  // RMSNorm in front of few-row GEMMs: when every reader of the normalised tensor is a GEMM of the next step and that
+  // RMSNorm or LayerNorm in front of few-row GEMMs: when every reader of the normalised tensor is a GEMM of the next step and that
   // step runs the weight-streaming kernel, the normalisation runs inside it (the gain on the way in, 1/rms in the
   // epilogue) and the normalised tensor is never stored.
   if (p->opts.fusion && p->opts.gemm_path == 0 && !p->opts.eval && p->opts.split_k <= 0) {
@@ -1070,9 +1070,12 @@ static int lower_and_place(fluid_plan_s* p) {
       const Step& sn = p->steps[si];
       if (sn.nodes.size() != 1) continue;
       const Node& nn = p->nodes[sn.node];
-      if (nn.kind != N_NORM || !nn.rms || nn.res >= 0 || T[nn.out].kind != FLUID_ACT || T[nn.out].dtype != FLUID_BF16 ||
+      if (nn.kind != N_NORM || nn.res >= 0 || T[nn.out].kind != FLUID_ACT || T[nn.out].dtype != FLUID_BF16 ||
           p->alias_root[nn.out] != nn.out || T[nn.gamma].kind != FLUID_CONST || lo[nn.gamma] != 0)
         continue;
+      // LayerNorm: its bias rides along as one more activation row, so at most 7 rows, and not with SwiGLU
+      const bool layer = !nn.rms;
+      if (layer && (nn.beta < 0 || T[nn.beta].kind != FLUID_CONST || lo[nn.beta] != 0 || p->steps[si + 1].swiglu)) continue;
       Step& sg = p->steps[si + 1];
       int readers = 0;
       bool ok = true;
@@ -1081,6 +1084,11 @@ static int lower_and_place(fluid_plan_s* p) {
         if (m.kind != N_GEMM) continue;   // the SiLU * up node of a SwiGLU step
         GemmParams g;
         ok = ok && m.a == nn.out && m.gemm_kind == G_LINEAR && lower_gemm(p, m, lo, &g) && gemm_rows_eligible(g);
+        if (ok && layer) {   // room for the extra staged row
+          GemmParams g1 = g;
+          g1.M = g.M + 1;
+          ok = g.M <= 7 && gemm_rows_eligible(g1);
+        }
         ++readers;
       }
       if (!ok || readers == 0 || n_uses[nn.out] != readers) continue;

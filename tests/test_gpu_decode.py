@@ -421,16 +421,22 @@ def test_few_row_linear_random_shapes():
     helpers.ensure_lib()
     for it in range(24):
         M, N, K = int(rng.integers(1, 9)), int(rng.integers(1, 5000)), 8 * int(rng.integers(1, 600))
-        bias, act, res, rms = (bool(rng.random() < p) for p in (0.5, 0.3, 0.5, 0.4))
+        bias, act, res, rms = (bool(rng.random() < p) for p in (0.5, 0.3, 0.5, 0.6))
+        layer = rms and M <= 7 and bool(rng.random() < 0.5)      # LayerNorm instead of RMSNorm
         g = synth.GraphDesc()
         x = g.tensor("x", synth.BF16, [M, K], synth.INPUT)
-        feeds = {x: helpers.rand_feed([M, K], synth.BF16, it)}
+        feeds = {x: helpers.rand_feed([M, K], synth.BF16, it, -1.0, 3.0)}   # a mean well away from zero
         a = x
         if rms:
             gam = g.tensor("gam", synth.BF16, [K], synth.CONST)
             feeds[gam] = helpers.rand_feed([K], synth.BF16, it + 50, 0.5, 1.5)
             a = g.tensor("n", synth.BF16, [M, K], synth.ACT)
-            g.op(synth.RMSNORM, [x, gam], [a], eps=1e-5)
+            if layer:
+                bet = g.tensor("bet", synth.BF16, [K], synth.CONST)
+                feeds[bet] = helpers.rand_feed([K], synth.BF16, it + 60)
+                g.op(synth.LAYERNORM, [x, gam, bet], [a], eps=1e-5)
+            else:
+                g.op(synth.RMSNORM, [x, gam], [a], eps=1e-5)
         w = g.tensor("w", synth.BF16, [K, N], synth.CONST)
         feeds[w] = synth.round_bf16(synth.normal(7, it, [K, N], 0.05))
         ins = [a, w]
@@ -455,5 +461,5 @@ def test_few_row_linear_random_shapes():
         assert "GEMM_ROWS" in [s["kernel_name"] for s in steps]
         if rms:
             assert len(steps) == 1 and (steps[0]["variant"] >> 30) & 1      # one launch: norm, GEMM and epilogue
-        helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], synth.BF16, f"case {it}: {M}x{N}x{K} bias {bias} act {act} res {res} rms {rms}")
+        helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], synth.BF16, f"case {it}: {M}x{N}x{K} bias {bias} act {act} res {res} norm {rms} layer {layer}")
         plan.close()

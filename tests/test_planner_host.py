@@ -327,6 +327,14 @@ def test_decoding_graph_plans_without_a_gpu():
     assert "GEMM_ROWS" not in [s["kernel_name"] for s in simt.steps()]
     for p in (plan, unfused, simt):
         p.close()
+    # the GPT-family step: LayerNorm folds into the few-row GEMMs as well (its bias as one more activation row)
+    gcfg = synth.scaled(synth.CONFIGS["gpt2_small"], S=1, L=2, B=4)
+    gdec = synth.build_decode_model(gcfg, 1024, materialize=False)
+    gplan = fluid.Plan(gdec.graph, synth.default_candidates(gdec.graph))
+    gnames = [s["kernel_name"] for s in gplan.steps()]
+    assert gnames[0] == "EMBED" and gnames[1:11] == ["GEMM_ROWS", "ATTN_DECODE", "GEMM_ROWS", "GEMM_ROWS", "GEMM_ROWS"] * 2
+    assert sum((s["variant"] >> 30) & 1 for s in gplan.steps() if s["kernel_name"] == "GEMM_ROWS") == 4
+    gplan.close()
 
 
 def test_state_tensors_and_cached_attention_are_checked():
