@@ -63,12 +63,21 @@ class MeasuredEval:
         torch = self.torch
         d = self.desc
         g = synth.GraphDesc()
-        local, cands, consts, int_inputs = {}, {}, {}, []
-        for t, perm in zip(op["ins"], perms):
+        local, cands, consts, fed = {}, {}, {}, {}     # fed: local input / state tensor -> array handed to the runner
+        for slot, (t, perm) in enumerate(zip(op["ins"], perms)):
             src = d.tensors[t]
+            if t in local:                                 # the same tensor in two roles (the position of a decoding step)
+                continue
             if src["dtype"] == synth.I32:
                 lt = g.tensor(f"in{t}", synth.I32, src["dims"], synth.INPUT)
-                int_inputs.append(lt)
+                if op["kind"] == synth.EMBED and slot == 0:     # ids index the first dim of the table they look up
+                    fed[lt] = np.asarray(synth.token_ids(self.seed, 0, src["dims"], d.dims(op["ins"][1])[0]), dtype=np.int32)
+                else:                                           # a position: the start of the sequence
+                    fed[lt] = np.zeros(src["dims"], dtype=np.int32)
+            elif src["kind"] == synth.STATE:
+                # a caller-owned cache: canonical, read and updated in place by the timed step
+                lt = g.tensor(f"in{t}", src["dtype"], src["dims"], synth.STATE)
+                fed[lt] = np.zeros(src["dims"], dtype=np.float32)
             else:
                 # a constant may sit in any candidate layout and is packed outside the timed path
                 lt = g.tensor(f"in{t}", src["dtype"], src["dims"], synth.CONST)
@@ -103,11 +112,8 @@ class MeasuredEval:
             if got != want:
                 return math.inf   # the planner could not honour the combination (its guard fell back to canonical)
             runner = fluid.Runner(plan, consts)
-            if int_inputs:
-                # ids index the first dim of the table they look up
-                hi = d.dims(op["ins"][1])[0] if op["kind"] == synth.EMBED else 2
-                ids_shape = d.dims(op["ins"][0])
-                runner.set_inputs([np.asarray(synth.token_ids(self.seed, 0, ids_shape, hi), dtype=np.int32)])
+            if fed:
+                runner.set_inputs([fed[lt] for lt in g.inputs])
             steps = plan.steps()
             mine = [i for i, s in enumerate(steps) if 0 in s["ops"]]
             if len(mine) != 1:

@@ -463,3 +463,33 @@ def test_few_row_linear_random_shapes():
             assert len(steps) == 1 and (steps[0]["variant"] >> 30) & 1      # one launch: norm, GEMM and epilogue
         helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], synth.BF16, f"case {it}: {M}x{N}x{K} bias {bias} act {act} res {res} norm {rms} layer {layer}")
         plan.close()
+
+
+def test_plan_of_a_decoding_step_from_measured_costs():
+    """The measured cost function handles the decoding operators too (state tensors, device-side positions): the plan
+    built from measured per-operator times gives the oracle's results."""
+    from paper_2411_09242_b200.measure import MeasuredEval
+    cfg = synth.scaled(synth.CONFIGS["llama"], dtype=synth.BF16, S=1, L=1, H=256, nh=4, F=384, B=3, V=300)
+    dec = synth.build_decode_model(cfg, 24)
+    g = dec.graph
+    helpers.ensure_lib()
+    cands = synth.default_candidates(g)
+    ev = MeasuredEval(g, cands, reps=3, warmup=1)
+    plan = fluid.Plan(g, cands, eval=ev.callback)
+    assert ev.measured >= 8 and 0 < plan.cost <= plan.canonical_cost < 1.0
+    kinds = [s["kernel_name"] for s in plan.steps()]
+    assert "ATTN_DECODE" in kinds and "GEMM_ROWS" in kinds
+    feeds = dict(dec.consts)
+    feeds[dec.ids] = synth.token_ids(3, 0, [cfg.B, 1], cfg.V)
+    feeds[dec.pos] = np.array([9], dtype=np.int32)
+    for i, pair in enumerate(dec.caches):
+        for j, t in enumerate(pair):
+            feeds[t] = synth.round_bf16(synth.uniform(5, 2 * i + j, g.dims(t)))
+    runner = fluid.Runner(plan, dec.consts)
+    runner.set_inputs([feeds[t] for t in g.inputs])
+    runner.run()
+    assert runner.status() == 0
+    ref = helpers.run_oracle(g, feeds)
+    for tid, got in zip(g.outputs, runner.outputs_host()):
+        helpers.assert_close(got, ref[tid], synth.BF16, f"measured-cost decoding plan output {tid}", tol=2e-2)
+    plan.close()
