@@ -1665,7 +1665,7 @@ int gemm_cluster_split(const GemmParams* gs, const GemmTcHost& tc, int n_group) 
   return 0;
 }
 
-// True if the step runs as CTA pairs (two CTAs per 256 x 256 tile), judged on shapes and strides alone.
+// True if the step runs as CTA pairs (two CTAs per 256 x 256 tile), decided from shapes and strides alone.
 bool gemm_pair_eligible(const GemmParams* gs, const GemmTcHost& tc, int n_group) {
   const GemmParams& g = gs[0];
   if (!tc.cfg.pair || !pair_enabled() || g.causal != CAUSAL_NONE || ((g.M + BM - 1) / BM) % 2 != 0) return false;

@@ -1,4 +1,4 @@
-"""Parity at the benchmark's full sizes, in the configuration bench.py times (planned layouts, fused
+"""Parity at the full sizes of the benchmark configurations, in the configuration bench.py times (planned layouts, fused
 epilogues, tensor-core GEMMs). Where a full oracle pass is too slow, outputs are sampled in a way the
 oracle can compute exactly: a causal model's first rows depend only on the first tokens."""
 import numpy as np
