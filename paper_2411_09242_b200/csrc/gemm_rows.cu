@@ -1,4 +1,4 @@
-// GEMM with a handful of rows (M <= 8: the LINEAR steps of single-token decoding). The step reads every
+// GEMM with a handful of rows (M <= 16: the LINEAR steps of single-token decoding). The step reads every
 // weight once and does M multiply-adds per weight, so it is bound by streaming the weight matrix from HBM,
 // not by arithmetic: a 128-row tcgen05 tile would stage 16x more rows than exist through shared memory and
 // tensor memory and pay that pipeline's fill and drain per short k range. Here every lane copies the 16 bytes it
@@ -9,7 +9,8 @@
 // held k-contiguous ("column-major" in the paper's matmul figure).
 //
 // The multiply-adds use the warp-level m16n8k16 bf16 MMA with fp32 accumulation as the arithmetic unit, with the
-// roles swapped: 16 weight rows are the MMA's row operand, the (up to 8) activation rows its 8 columns. The
+// roles swapped: 16 weight rows are the MMA's row operand, the activation rows its 8 columns (two MMAs side by side
+// for 9 to 16 activation rows). The
 // contraction index may be fed in any order as long as both operands agree, so a lane takes 8 *consecutive* k of
 // one weight row (one 16-byte copy) and the same 8 k of one activation row, and two MMAs consume them: no
 // unpacking, no shuffles, no exchange between lanes.
@@ -94,19 +95,21 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 // no barrier; the bytes in flight are set by the ring's depth, not by registers), the activation fragment comes from
 // the staged copy. ST = ring depth. SWIGLU: groups 0 and 1 are the gate and up projections; the same tiles of both
 // sit in neighbouring warps and the CTA writes SiLU(gate) * up to group 0's C, so neither projection is ever stored.
-template <int KS, int ST, bool SWIGLU>
+// MT = 8-row groups of activation rows (1: M <= 8, 2: M <= 16; a second MMA column block).
+template <int KS, int ST, bool SWIGLU, int MT>
 __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p) {
+  constexpr int MC = 8 * MT;                       // activation rows the accumulators cover
   constexpr int NG = SWIGLU ? 2 : 1;               // groups inside a CTA
-  constexpr int UMAX = kWarps / (KS * NG);         // most (group, tile) units per CTA and round
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int pitch = p.K + kXPad;                   // staged activation row, bf16 elements
   __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);
   const int ln = p.beta ? 1 : 0;                   // LayerNorm: one more staged row (the bias), see below
   unsigned char* after_x = smem_raw + size_t(p.M + ln) * pitch * 2;
   const uint32_t ring0 = static_cast<uint32_t>(__cvta_generic_to_shared(after_x));
-  float(*red)[16][9] = reinterpret_cast<float(*)[16][9]>(after_x + kWarps * ST * 1024);   // [warp][row][m]
-  float* rstd = reinterpret_cast<float*>(after_x + kWarps * ST * 1024 + kWarps * 16 * 9 * sizeof(float));   // [8]
-  float* ssq_part = rstd + 8;                                                             // [warp][8]
+  // partial sums [row][m] of a warp: laid over the warp's own ring, which is drained by the time they are written
+  auto red = [&](int w) { return reinterpret_cast<float(*)[MC + 1]>(after_x + size_t(w) * (ST * 1024)); };
+  float* rstd = reinterpret_cast<float*>(after_x + kWarps * ST * 1024);   // [16]
+  float* part = rstd + 16;                                                // [16]: per-warp sums while staging
   pdl_launch_dependents();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -118,6 +121,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
   auto slot = [&](int i, int piece) { return my_ring + uint32_t(i % ST) * 1024 + uint32_t(piece) * 512; };
   const uint32_t xs_lane = static_cast<uint32_t>(__cvta_generic_to_shared(xs)) + uint32_t((g < p.M + ln ? g : 0) * pitch + t * 8) * 2;
   const bool x_live = g < p.M + ln;
+  const bool x_live2 = MT == 2 && g + 8 < p.M + ln;   // activation rows 8 .. 15
 
   for (int round = 0; round < p.rounds; ++round) {
     // units are dealt out evenly: a CTA takes p.upc <= UMAX of them per round, so that every SM streams
@@ -159,73 +163,63 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
         }
       }
       // ---- stage the activations: thread -> 8 consecutive k of one row ----
-      const int chunks = p.K / 8;
+      // The 16 warps are dealt to the rows (the LayerNorm bias counts as one): 16 / rows warps each, rounded down to a
+      // power of two; a row's statistics go through a few words of shared memory.
       // LayerNorm: ((x - mean) * rstd * gamma + beta) . W = rstd * (((x - mean) * gamma) . W) + beta . W. The rows are
       // centred and multiplied by the gain here; the bias rides along as one more activation row (an MMA column that
       // would otherwise be idle), so beta . W comes out of the same accumulators.
-      float mean[8];
-#pragma unroll
-      for (int m = 0; m < 8; ++m) mean[m] = 0.f;
+      const int chunks = p.K / 8;
+      const int n_rows = p.M + ln;
+      const int wpr = n_rows > 8 ? 1 : (n_rows > 4 ? 2 : (n_rows > 2 ? 4 : (n_rows > 1 ? 8 : 16)));
+      const int row = warp / wpr, c0 = (warp % wpr) * 32 + lane, cstep = 32 * wpr;
+      const bool is_x = row < p.M, is_beta = ln && row == p.M;
+      auto load_x8 = [&](int64_t off, float (&xf)[8]) {
+        if (p.x_f32) {
+          const float4 lo = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + off);
+          const float4 hi = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + off + 4);
+          xf[0] = lo.x; xf[1] = lo.y; xf[2] = lo.z; xf[3] = lo.w; xf[4] = hi.x; xf[5] = hi.y; xf[6] = hi.z; xf[7] = hi.w;
+        } else {
+          load16(static_cast<const __nv_bfloat16*>(p.X) + off, xf);
+        }
+      };
+      const int64_t roff = is_x ? split2(row, p.M0, p.a_s2, p.a_s3) : 0;
+      __nv_bfloat16* dst = xs + size_t(row < n_rows ? row : 0) * pitch;
+      float mean = 0.f;
       if (ln) {
-#pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          float sm = 0.f;
-          if (m < p.M) {
-            const int64_t roff = split2(m, p.M0, p.a_s2, p.a_s3);
-            for (int c = threadIdx.x; c < chunks; c += kWarps * 32) {
-              float xf[8];
-              if (p.x_f32) {
-                const float4 lo = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + roff + c * 8);
-                const float4 hi = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + roff + c * 8 + 4);
-                xf[0] = lo.x; xf[1] = lo.y; xf[2] = lo.z; xf[3] = lo.w; xf[4] = hi.x; xf[5] = hi.y; xf[6] = hi.z; xf[7] = hi.w;
-              } else {
-                load16(static_cast<const __nv_bfloat16*>(p.X) + roff + c * 8, xf);
-              }
-#pragma unroll
-              for (int i = 0; i < 8; ++i) sm += xf[i];
-            }
-          }
-          sm = warp_sum(sm);
-          if (lane == 0) ssq_part[warp * 8 + m] = sm;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          float tot = 0.f;
-          for (int w = 0; w < kWarps; ++w) tot += ssq_part[w * 8 + m];
-          mean[m] = tot / p.K;
-        }
-        __syncthreads();   // the slots are reused for the sums of squares
-        for (int c = threadIdx.x; c < chunks + kXPad / 8; c += kWarps * 32)
-          *reinterpret_cast<uint4*>(xs + size_t(p.M) * pitch + c * 8) =
-              c < chunks ? *reinterpret_cast<const uint4*>(p.beta + c * 8) : make_uint4(0u, 0u, 0u, 0u);
-      }
-      float ssq[8];
-#pragma unroll
-      for (int m = 0; m < 8; ++m) {
-        ssq[m] = 0.f;
-        if (m >= p.M) continue;
-        const int64_t roff = split2(m, p.M0, p.a_s2, p.a_s3);
-        float acc = 0.f;
-        for (int c = threadIdx.x; c < chunks + kXPad / 8; c += kWarps * 32) {
-          uint4 out;
-          if (c >= chunks) {
-            out = make_uint4(0u, 0u, 0u, 0u);   // the padding is read (against zero weights) when K is not a multiple of 32
-          } else if (p.gamma || p.x_f32) {
+        float sm = 0.f;
+        if (is_x) {
+#pragma unroll 4
+          for (int c = c0; c < chunks; c += cstep) {
             float xf[8];
-            if (p.x_f32) {
-              const float4 lo = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + roff + c * 8);
-              const float4 hi = *reinterpret_cast<const float4*>(static_cast<const float*>(p.X) + roff + c * 8 + 4);
-              xf[0] = lo.x; xf[1] = lo.y; xf[2] = lo.z; xf[3] = lo.w; xf[4] = hi.x; xf[5] = hi.y; xf[6] = hi.z; xf[7] = hi.w;
-            } else {
-              load16(static_cast<const __nv_bfloat16*>(p.X) + roff + c * 8, xf);
-            }
+            load_x8(roff + c * 8, xf);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sm += xf[i];
+          }
+        }
+        sm = warp_sum(sm);
+        if (lane == 0) part[warp] = sm;
+        __syncthreads();
+        if (is_x) {
+          float tot = 0.f;
+          for (int q = 0; q < wpr; ++q) tot += part[row * wpr + q];
+          mean = tot / p.K;
+        }
+        __syncthreads();   // the words are reused for the sums of squares
+      }
+      float acc = 0.f;
+      if (is_x) {
+#pragma unroll 4
+        for (int c = c0; c < chunks; c += cstep) {
+          uint4 out;
+          if (p.gamma || p.x_f32) {
+            float xf[8];
+            load_x8(roff + c * 8, xf);
             if (p.gamma) {
               float gf[8];
               load16(p.gamma + c * 8, gf);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                xf[i] -= mean[m];
+                xf[i] -= mean;
                 acc = fmaf(xf[i], xf[i], acc);
                 xf[i] *= gf[i];
               }
@@ -234,46 +228,57 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
           } else {
             out = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.X) + roff + c * 8);
           }
-          *reinterpret_cast<uint4*>(xs + size_t(m) * pitch + c * 8) = out;
+          *reinterpret_cast<uint4*>(dst + c * 8) = out;
         }
-        ssq[m] = acc;
+      } else if (is_beta) {
+        for (int c = c0; c < chunks; c += cstep) *reinterpret_cast<uint4*>(dst + c * 8) = *reinterpret_cast<const uint4*>(p.beta + c * 8);
       }
-      if (p.gamma) {
-#pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          const float v = warp_sum(ssq[m]);
-          if (lane == 0) ssq_part[warp * 8 + m] = v;
-        }
-      }
+      // the padding is read (against zero weights) when K is not a multiple of 32
+      if ((is_x || is_beta) && warp % wpr == 0 && lane < kXPad / 8) *reinterpret_cast<uint4*>(dst + (chunks + lane) * 8) = make_uint4(0u, 0u, 0u, 0u);
+      acc = warp_sum(acc);
+      if (lane == 0) part[warp] = acc;
       __syncthreads();
-      if (threadIdx.x < 8) {
+      if (threadIdx.x < p.M) {
         float q2 = 0.f;
-        for (int w = 0; w < kWarps; ++w) q2 += ssq_part[w * 8 + threadIdx.x];
+        for (int q = 0; q < wpr; ++q) q2 += part[threadIdx.x * wpr + q];
         rstd[threadIdx.x] = p.gamma ? rsqrtf(q2 / p.K + p.eps) : 1.f;
       }
       // (rstd is read after the __syncthreads that follows the main loop)
     }
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
     for (int i = 0; i < nloc; ++i) {
       cp_async_wait<ST - 2>();   // this lane's copies of pass i have landed
       const uint4 w0 = lds128(slot(i, 0)), w1 = lds128(slot(i, 1));
-      const uint4 x = x_live ? lds128(xs_lane + uint32_t(blk0 + i) * (kBlk * 2)) : make_uint4(0u, 0u, 0u, 0u);
+      const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+      const uint4 x = x_live ? lds128(xs_lane + uint32_t(blk0 + i) * (kBlk * 2)) : zero4;
+      uint4 x2 = zero4;
+      if (MT == 2 && x_live2) x2 = lds128(xs_lane + uint32_t(8 * pitch * 2) + uint32_t(blk0 + i) * (kBlk * 2));
       fill_w(i + ST - 1);        // refills the slot read one pass ago
       cp_async_commit();
       mma_bf16(acc, w0.x, w1.x, w0.y, w1.y, x.x, x.y);
       mma_bf16(acc, w0.z, w1.z, w0.w, w1.w, x.z, x.w);
+      if (MT == 2) {
+        mma_bf16(acc2, w0.x, w1.x, w0.y, w1.y, x2.x, x2.y);
+        mma_bf16(acc2, w0.z, w1.z, w0.w, w1.w, x2.z, x2.w);
+      }
     }
     cp_async_wait<0>();
     // accumulator fragment: acc[0..1] = (weight row g; activation rows 2t, 2t+1), acc[2..3] = (weight row g + 8; same)
-    red[warp][g][2 * t] = acc[0];
-    red[warp][g][2 * t + 1] = acc[1];
-    red[warp][g + 8][2 * t] = acc[2];
-    red[warp][g + 8][2 * t + 1] = acc[3];
+    red(warp)[g][2 * t] = acc[0];
+    red(warp)[g][2 * t + 1] = acc[1];
+    red(warp)[g + 8][2 * t] = acc[2];
+    red(warp)[g + 8][2 * t + 1] = acc[3];
+    if (MT == 2) {
+      red(warp)[g][8 + 2 * t] = acc2[0];
+      red(warp)[g][8 + 2 * t + 1] = acc2[1];
+      red(warp)[g + 8][8 + 2 * t] = acc2[2];
+      red(warp)[g + 8][8 + 2 * t + 1] = acc2[3];
+    }
     __syncthreads();
     // thread -> (tile of the CTA, m, row of the tile) with the row fastest, so that stores to an n-contiguous C coalesce
-    for (int e = threadIdx.x; e < p.upc * 16 * 8; e += kWarps * 32) {
-      const int nl = e % 16, m = (e / 16) % 8, tl = e / 128;
+    for (int e = threadIdx.x; e < p.upc * 16 * MC; e += kWarps * 32) {
+      const int nl = e % 16, m = (e / 16) % MC, tl = e / (16 * MC);
       const int u = (round * p.upc + tl) * gridDim.x + blockIdx.x;
       if (u >= p.units) continue;
       const int n = (SWIGLU ? u : u % p.tiles) * 16 + nl;
@@ -281,18 +286,18 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
       const float sc = p.scale * rstd[m];
       float v = 0.f;
 #pragma unroll
-      for (int q = 0; q < KS; ++q) v += red[tl * NG * KS + q][nl][m];
+      for (int q = 0; q < KS; ++q) v += red(tl * NG * KS + q)[nl][m];
       v *= sc;
       if (SWIGLU) {
         float u = 0.f;
 #pragma unroll
-        for (int q = 0; q < KS; ++q) u += red[(tl * NG + 1) * KS + q][nl][m];
+        for (int q = 0; q < KS; ++q) u += red((tl * NG + 1) * KS + q)[nl][m];
         v = silu(v) * (u * sc);
       }
       if (ln) {   // + beta . W
         float bw = 0.f;
 #pragma unroll
-        for (int q = 0; q < KS; ++q) bw += red[tl * NG * KS + q][nl][p.M];
+        for (int q = 0; q < KS; ++q) bw += red(tl * NG * KS + q)[nl][p.M];
         v = fmaf(bw, p.scale, v);
       }
       const RowsGroup& og = p.g[SWIGLU ? 0 : u / p.tiles];
@@ -311,22 +316,28 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_rows_kernel(RowsParams p)
   }
 }
 
-inline size_t rows_fixed_smem(int M, int K) {
-  return size_t(M) * (K + kXPad) * 2 + size_t(kWarps) * 16 * 9 * sizeof(float) + (8 + kWarps * 8) * sizeof(float);
-}
+// staged rows (the LayerNorm bias counts as a row) + 1/rms and the staging sums (the partial sums of the epilogue lie
+// over the rings)
+inline size_t rows_fixed_smem(int rows, int K) { return size_t(rows) * (K + kXPad) * 2 + 32 * sizeof(float); }
+constexpr int kRingMin = 5;   // fewest ring stages worth running with
 
-template <int KS, int ST, bool SWIGLU>
-cudaError_t launch_rows(RowsParams& p, int n_group, cudaStream_t st) {
+template <int KS, int ST, bool SWIGLU, int MT>
+cudaError_t launch_rows_mt(RowsParams& p, int n_group, cudaStream_t st) {
   const size_t smem = rows_fixed_smem(p.M + (p.beta ? 1 : 0), p.K) + size_t(kWarps) * ST * 1024;
   static const cudaError_t attr =
-      cudaFuncSetAttribute(gemm_rows_kernel<KS, ST, SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      cudaFuncSetAttribute(gemm_rows_kernel<KS, ST, SWIGLU, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
   if (attr != cudaSuccess) return attr;
   constexpr int UMAX = kWarps / (KS * (SWIGLU ? 2 : 1));
   p.units = SWIGLU ? p.tiles : p.tiles * n_group;
   const int grid = std::min(148, p.units);
   p.upc = std::min(UMAX, (p.units + grid - 1) / grid);
   p.rounds = (p.units + grid * p.upc - 1) / (grid * p.upc);
-  return launch_k(gemm_rows_kernel<KS, ST, SWIGLU>, dim3((unsigned)grid), dim3(kWarps * 32), smem, st, p);
+  return launch_k(gemm_rows_kernel<KS, ST, SWIGLU, MT>, dim3((unsigned)grid), dim3(kWarps * 32), smem, st, p);
+}
+
+template <int KS, int ST, bool SWIGLU>
+cudaError_t launch_rows(RowsParams& p, int n_group, cudaStream_t st) {
+  return p.M + (p.beta ? 1 : 0) > 8 ? launch_rows_mt<KS, ST, SWIGLU, 2>(p, n_group, st) : launch_rows_mt<KS, ST, SWIGLU, 1>(p, n_group, st);
 }
 
 template <int ST>
@@ -352,10 +363,11 @@ inline bool al16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) =
 }  // namespace
 
 bool gemm_rows_eligible(const GemmParams& g) {
-  if (g.dtype != FLUID_BF16 || g.batch != 1 || g.M < 1 || g.M > 8 || g.causal != CAUSAL_NONE) return false;
+  if (g.dtype != FLUID_BF16 || g.batch != 1 || g.M < 1 || g.M > 16 || g.causal != CAUSAL_NONE) return false;
   if (g.K % 8 || g.K < 8) return false;
-  // the activation rows are staged in shared memory next to a ring of at least six stages per warp
-  if (rows_fixed_smem(g.M, g.K) + size_t(kWarps) * 6 * 1024 > size_t(kSmemBudget)) return false;
+  // the activation rows are staged in shared memory next to a ring of at least five stages per warp
+  // (with more than 8 rows the tcgen05 path is no slower than this kernel on a five-stage ring: ask for seven)
+  if (rows_fixed_smem(g.M, g.K) + size_t(kWarps) * (g.M > 8 ? 7 : kRingMin) * 1024 > size_t(kSmemBudget)) return false;
   // both operands with a flat, contiguous k index
   if (g.a_s[5] != 1 || !flat(g.K, g.K0, g.a_s[4], 1)) return false;
   if (g.b_s[3] != 1 || !flat(g.K, g.K0, g.b_s[2], 1)) return false;
@@ -374,7 +386,7 @@ cudaError_t launch_gemm_rows(const GemmParams* gs, int n_group, cudaStream_t st,
   p.x_f32 = norm ? norm->x_f32 : 0;
   p.gamma = norm ? static_cast<const __nv_bfloat16*>(norm->gamma) : nullptr;
   p.beta = norm ? static_cast<const __nv_bfloat16*>(norm->beta) : nullptr;
-  if (p.beta && (swiglu || g0.M > 7 || !al16(p.beta))) return cudaErrorInvalidValue;
+  if (p.beta && (swiglu || g0.M > 15 || !al16(p.beta))) return cudaErrorInvalidValue;
   p.eps = norm ? norm->eps : 0.f;
   p.M = g0.M; p.N = g0.N; p.K = g0.K; p.M0 = g0.M0; p.N0 = g0.N0;
   p.a_s2 = g0.a_s[2]; p.a_s3 = g0.a_s[3];
@@ -399,10 +411,11 @@ cudaError_t launch_gemm_rows(const GemmParams* gs, int n_group, cudaStream_t st,
   // ring depth: what the staged activations leave (one 16-byte piece per lane, row and stage; wider pieces measured
   // three times slower: a copy instruction of the warp then touches every 32-byte sector half)
   const size_t fixed = rows_fixed_smem(p.M + (p.beta ? 1 : 0), p.K);
-  if (fixed + size_t(kWarps) * 6 * 1024 > size_t(kSmemBudget)) return cudaErrorInvalidValue;
+  if (fixed + size_t(kWarps) * kRingMin * 1024 > size_t(kSmemBudget)) return cudaErrorInvalidValue;
   const size_t left = size_t(kSmemBudget) - fixed;
   if (left >= size_t(kWarps) * 10 * 1024) return launch_rows_ks<10>(p, n_group, swiglu != 0, st);
-  return launch_rows_ks<6>(p, n_group, swiglu != 0, st);
+  if (left >= size_t(kWarps) * 7 * 1024) return launch_rows_ks<7>(p, n_group, swiglu != 0, st);
+  return launch_rows_ks<kRingMin>(p, n_group, swiglu != 0, st);
 }
 
 }  // namespace fluid

@@ -178,10 +178,10 @@ struct AttnDecodeParams {
   float rope_log2_base;
   int64_t q_sb, q_sh, k_sb, k_sh, v_sb, v_sh, o_sb, o_sh;   // element strides of batch and head
 };
-// GEMM with at most 8 rows and both operands k-contiguous (bf16): the weights stream through registers once.
+// GEMM with at most 16 rows and both operands k-contiguous (bf16): the weights stream through the SM once.
 // n_group (1..3) sibling GEMMs that share A and the shapes run as one launch. swiglu (two groups: gate, up): the launch
 // writes SiLU(gate) * up to g[0].C and nothing else.
-// norm (optional): the RMS normalisation or (M <= 7, no swiglu) LayerNorm in front of the GEMMs runs inside the launch: A is then x (bf16, or fp32 when
+// norm (optional): the RMS normalisation or (M <= 15, no swiglu) LayerNorm in front of the GEMMs runs inside the launch: A is then x (bf16, or fp32 when
 // x_f32) with the strides of g[0]'s A operand, and the normalised tensor is never stored.
 struct RowsNorm {
   const void* x;

@@ -1073,7 +1073,7 @@ static int lower_and_place(fluid_plan_s* p) {
       if (nn.kind != N_NORM || nn.res >= 0 || T[nn.out].kind != FLUID_ACT || T[nn.out].dtype != FLUID_BF16 ||
           p->alias_root[nn.out] != nn.out || T[nn.gamma].kind != FLUID_CONST || lo[nn.gamma] != 0)
         continue;
-      // LayerNorm: its bias rides along as one more activation row, so at most 7 rows, and not with SwiGLU
+      // LayerNorm: its bias rides along as one more activation row, so at most 15 rows, and not with SwiGLU
       const bool layer = !nn.rms;
       if (layer && (nn.beta < 0 || T[nn.beta].kind != FLUID_CONST || lo[nn.beta] != 0 || p->steps[si + 1].swiglu)) continue;
       Step& sg = p->steps[si + 1];
@@ -1087,7 +1087,7 @@ static int lower_and_place(fluid_plan_s* p) {
         if (ok && layer) {   // room for the extra staged row
           GemmParams g1 = g;
           g1.M = g.M + 1;
-          ok = g.M <= 7 && gemm_rows_eligible(g1);
+          ok = g.M <= 15 && gemm_rows_eligible(g1);
         }
         ++readers;
       }
