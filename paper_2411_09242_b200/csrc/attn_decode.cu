@@ -1,14 +1,15 @@
 // Attention of one decoding step against a key/value cache (single new token per sequence).
 //
 // The step is bound by reading the cache once: per (sequence, head) t+1 rows of D keys and D values, one
-// multiply-add per byte pair. No tensor cores: rows stream through registers with 16-byte loads.
+// multiply-add per byte pair. No tensor cores: rows stream through the SM in 16-byte pieces.
 //
 // Work split: one thread-block cluster of up to 8 CTAs per (sequence, query head); CTA r of the cluster takes a
 // contiguous share of the rows 0..t. Inside a CTA a row is owned by LPR = D / (16 bytes of elements)
 // adjacent lanes (a warp covers 32 / LPR rows per load instruction); every such lane group keeps a running
 // (max, sum, output) triple in the base-2 online-softmax form; its rows of keys and values arrive through a
-// per-lane ring of asynchronous copies in shared memory, several rows deep. Triples are merged lane group -> warp (shuffles) -> CTA (shared memory) -> cluster (each
-// CTA stores its triple into CTA 0's shared memory; one cluster barrier), and CTA 0 writes the D outputs.
+// per-lane ring of asynchronous copies in shared memory, several rows deep. Triples are merged lane group -> warp
+// (shuffles) -> CTA (shared memory) -> cluster (each CTA stores its triple into CTA 0's shared memory; one cluster
+// barrier), and CTA 0 writes the D outputs.
 // The row of the new token comes from the step's own k and v operands, and the CTA that meets it stores it
 // as row t of the caches: no row is read from the cache in the launch that writes it.
 //
