@@ -127,7 +127,8 @@ typedef struct fluid_plan_options {
                                SiLU*up into one pass, and BMM_QK -> SOFTMAX -> BMM_PV into one
                                attention step whose score tensor never leaves the SM;
                                0: one step per graph op */
-  int32_t arena_policy;     /* 0: first fit (Algorithm 4 as printed), 1: best fit (its prose) */
+  int32_t arena_policy;     /* 0: first fit (Algorithm 4 as printed), 1: best fit (its prose), 2 (not in the paper): the
+                               same placement over several record orders and both fits, the smallest arena kept */
   int32_t no_reuse;         /* 1: one private slice per activation (the naive plan) */
   int32_t force_canonical;  /* 1: skip the layout search, every tensor canonical */
   int32_t gemm_path;        /* 0: tensor cores where eligible, 1: SIMT kernel everywhere */

@@ -923,14 +923,9 @@ static int plan_layouts(fluid_plan_s* p) {
 // ---- Algorithm 4: Greedy-by-Size --------------------------------------------------------------------------
 static int64_t round_up(int64_t n, int64_t a) { return (n + a - 1) / a * a; }
 
-static void greedy_by_size(std::vector<ArenaRecord>& recs, int policy, bool no_reuse, size_t* arena_bytes) {
-  std::vector<int> order(recs.size());
-  for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
-  std::sort(order.begin(), order.end(), [&](int x, int y) {
-    if (recs[x].bytes != recs[y].bytes) return recs[x].bytes > recs[y].bytes;
-    if (recs[x].first != recs[y].first) return recs[x].first < recs[y].first;
-    return recs[x].id < recs[y].id;
-  });
+// Algorithm 4 (Greedy-by-Size): records in the given order, each into a gap among the lifetime-overlapping records placed
+// so far (first fit as printed, or the tightest gap as the prose has it), else at the tail.
+static int64_t place_in_order(std::vector<ArenaRecord>& recs, const std::vector<int>& order, bool best_fit, bool no_reuse) {
   int64_t arena = FLUID_ARENA_HEADER;
   std::vector<int> placed;
   for (int ri : order) {
@@ -945,7 +940,7 @@ static void greedy_by_size(std::vector<ArenaRecord>& recs, int policy, bool no_r
     for (auto& b : busy) {
       const int64_t gap = b.first - cursor;
       if (gap >= r.bytes) {
-        if (policy == 0) {
+        if (!best_fit) {
           if (best_off < 0) { best_off = cursor; best_gap = gap; }
         } else if (best_off < 0 || gap < best_gap) {
           best_off = cursor; best_gap = gap;
@@ -957,7 +952,60 @@ static void greedy_by_size(std::vector<ArenaRecord>& recs, int policy, bool no_r
     arena = std::max(arena, r.offset + r.bytes);
     placed.push_back(ri);
   }
-  *arena_bytes = (size_t)arena;
+  return arena;
+}
+
+// policy 0 / 1: the paper's order (size, descending) with first / best fit. policy 2 (not in the paper): the same
+// placement run over a handful of orders and both fits, keeping the smallest arena; the paper's order comes first, so
+// the result is never larger than policy 0's or 1's.
+static void greedy_by_size(std::vector<ArenaRecord>& recs, int policy, bool no_reuse, size_t* arena_bytes) {
+  std::vector<int> order(recs.size());
+  for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
+  auto by_size = [&](int x, int y) {
+    if (recs[x].bytes != recs[y].bytes) return recs[x].bytes > recs[y].bytes;
+    if (recs[x].first != recs[y].first) return recs[x].first < recs[y].first;
+    return recs[x].id < recs[y].id;
+  };
+  std::sort(order.begin(), order.end(), by_size);
+  if (policy != 2) {
+    *arena_bytes = (size_t)place_in_order(recs, order, policy == 1, no_reuse);
+    return;
+  }
+  auto span = [&](int x) { return int64_t(recs[x].last - recs[x].first + 1); };
+  std::vector<std::vector<int>> orders;
+  orders.push_back(order);
+  {  // long-lived records first, then size
+    std::vector<int> o = order;
+    std::stable_sort(o.begin(), o.end(), [&](int x, int y) { return span(x) > span(y); });
+    orders.push_back(o);
+  }
+  {  // bytes x steps alive
+    std::vector<int> o = order;
+    std::stable_sort(o.begin(), o.end(), [&](int x, int y) { return recs[x].bytes * span(x) > recs[y].bytes * span(y); });
+    orders.push_back(o);
+  }
+  {  // in order of first use
+    std::vector<int> o = order;
+    std::stable_sort(o.begin(), o.end(), [&](int x, int y) { return recs[x].first < recs[y].first; });
+    orders.push_back(o);
+  }
+  {  // in reverse order of last use
+    std::vector<int> o = order;
+    std::stable_sort(o.begin(), o.end(), [&](int x, int y) { return recs[x].last > recs[y].last; });
+    orders.push_back(o);
+  }
+  int64_t best = -1;
+  std::vector<int64_t> best_off(recs.size(), 0);
+  for (const auto& o : orders)
+    for (int fit = 0; fit < 2; ++fit) {
+      const int64_t a = place_in_order(recs, o, fit == 1, no_reuse);
+      if (best < 0 || a < best) {
+        best = a;
+        for (size_t i = 0; i < recs.size(); ++i) best_off[i] = recs[i].offset;
+      }
+    }
+  for (size_t i = 0; i < recs.size(); ++i) recs[i].offset = best_off[i];
+  *arena_bytes = (size_t)best;
 }
 
 // ---- lowering: nodes -> steps, aliases, lifetimes ----------------------------------------------------------

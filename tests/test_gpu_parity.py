@@ -48,7 +48,9 @@ def test_small_models_planned_and_canonical(family, dtype):
                                ("unfused", synth.default_candidates(m.graph), {"fusion": 0}),
                                ("simt", synth.default_candidates(m.graph), {"gemm_path": 1}),
                                ("unfused_attention", synth.default_candidates(m.graph), {"unfused_attention": 1}),
-                               ("no_reuse", synth.default_candidates(m.graph), {"no_reuse": 1})]:
+                               ("no_reuse", synth.default_candidates(m.graph), {"no_reuse": 1}),
+                               ("best_fit", synth.default_candidates(m.graph), {"arena_policy": 1}),
+                               ("several_orders", synth.default_candidates(m.graph), {"arena_policy": 2})]:
         got, plan, _ = run_gpu(m.graph, feeds, cands, **opts)
         for t in m.graph.outputs:
             assert_close(got[t], ref[t], dtype, f"{family}/{label}")
