@@ -340,6 +340,8 @@ def main():
     ap.add_argument("--others", default="tiny,gpt2_small,llama", help="comma list of extra workloads to summarise")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--split-k", type=int, default=0, help="allow split-K GEMM steps (costs arena scratch)")
+    ap.add_argument("--decode-batch", type=int, default=4, help="sequences of the decoding workload")
+    ap.add_argument("--decode-cache-rows", type=int, default=2048, help="rows of its key/value caches (the step times the last)")
     ap.add_argument("--layers", type=int, default=0, help="reduced copy of the workload (profiling captures only)")
     ap.add_argument("--seq", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0)
@@ -420,7 +422,8 @@ def main():
         torch.cuda.empty_cache()
     if "llama" in args.others.split(","):
         try:
-            others.append(time_decode(max(5, args.steps // 3), args.warmup, torch, fluid, peaks))
+            others.append(time_decode(max(5, args.steps // 3), args.warmup, torch, fluid, peaks, batch=args.decode_batch,
+                                      t_max=args.decode_cache_rows))
         except Exception as e:
             others.append({"workload": "llama_decode", "error": repr(e)[:300]})
         torch.cuda.empty_cache()
