@@ -122,12 +122,10 @@ def test_gemm_operand_majors(dtype, a_major, b_major, n):
 
 
 @pytest.mark.parametrize("dtype", DT)
-@pytest.mark.parametrize("causal", [0, 1])
-@pytest.mark.parametrize("n", [1, 7, 128, 200, 1024, 2048, 4100])
+@pytest.mark.parametrize("causal,n", [(0, n) for n in (1, 7, 128, 200, 1024, 2048, 4100)] +
+                         [(1, n) for n in (1, 7, 128, 200, 1024)])     # the square causal cases are kept small
 def test_softmax_rows(dtype, causal, n):
     rows = 3 if not causal else n
-    if causal and n > 1024:
-        pytest.skip("square causal case kept small")
     shape = [2, rows, n]
     g = single_op_graph(synth.SOFTMAX, [shape], shape, dtype, {"causal": causal, "scale": 0.5})
     feeds = {0: rand_feed(shape, dtype, 4, -8.0, 8.0)}
