@@ -271,9 +271,18 @@ FLUID_API int fluid_status(const fluid_plan_t* plan, const void* arena_ptr, flui
  *    make that first call before any stream capture begins.
  *  - All calls share the one array: it is re-zeroed where needed at the start of every call, and two
  *    calls whose kernels overlap on the GPU (different streams, or graphs replayed concurrently) race.
- *  - Asynchronous on `stream`; launch errors come back as FLUID_ECUDA. */
+ *  - Asynchronous on `stream`; launch errors come back as FLUID_ECUDA. A bounded wait that expires
+ *    inside the kernel is NOT reported by this call: the kernel records a code in the array's first
+ *    word, drains and returns, leaving C partly unwritten. fluid_static_scratch_status reads it. */
 FLUID_API int fluid_gemm_bf16_static_scratch(const void* dev_a, const void* dev_b, const void* dev_bias, void* dev_c,
                                    int m, int n, int k, fluid_stream stream);
+/* Status of the last fluid_gemm_bf16_static_scratch call on the current device (the paper has no
+ * counterpart). Synchronises `stream`, then copies the status word out of the static array with one
+ * 4-byte cudaMemcpy (no allocation). *device_status = 0 and FLUID_OK when every wait completed (or
+ * when no call has been made on this device yet); a non-zero code and FLUID_ETIMEOUT when a bounded
+ * wait gave up, in which case C is incomplete and the array's arrival counters are stale (the next
+ * call re-zeroes them). Like fluid_status, it must not overlap a later call on another stream. */
+FLUID_API int fluid_static_scratch_status(fluid_stream stream, int* device_status);
 
 FLUID_API const char* fluid_last_error(void);
 /* Number of kernel launches issued by this library in this process (for launch accounting). */

@@ -58,28 +58,37 @@ def run_op(kind, ins, attrs):
     raise ValueError(f"unknown op kind {kind}")
 
 
-def run_graph(tensors, op_list, feeds, keep_all=False, store=None):
+def run_graph(tensors, op_list, feeds, keep_all=False, store=None, load=None):
     """Execute the graph.
 
     store: optional callable (tensor id, fp64 array) -> fp64 array applied to every op output
-    before it is handed on. The parity reference never uses it (no intermediate rounding). It is a
-    diagnostic mode: a test may pass a function that rounds each tensor the way a device plan
-    stores it (bf16, fp32, or not at all for tensors fused away), to tell storage rounding apart
-    from arithmetic errors.
+    before it is handed on. load: optional callable (op index, tensor id, fp64 array) -> fp64 array
+    applied to each input as an op reads it. The parity reference uses neither (no intermediate
+    rounding). They are a diagnostic mode: a test may pass functions that round each tensor the way
+    a device plan stores it (bf16, fp32, or not at all for tensors fused away; `load` for a tensor
+    the plan keeps in two precisions, one per kind of reader), to tell storage rounding apart from
+    arithmetic errors.
 
     tensors : list of dicts with "dims" (and "kind"); op_list : list of dicts with "kind",
     "ins", "outs", "attrs"; feeds : {tensor id: array} for every graph input and constant.
     Returns {tensor id: fp64 array} for every tensor (keep_all) or only those no op consumes
     plus anything marked as a graph output (kind == 1) and the final contents of every state
-    tensor (kind == 4).
+    tensor (kind == 4); in that case an intermediate array is dropped after its last reader.
     """
     vals = {}
     for tid, a in feeds.items():
         a = np.asarray(a)
         vals[tid] = a if a.dtype.kind in "iu" else a.astype(np.float64)
+    last_reader = {}
+    for n, op in enumerate(op_list):
+        for i in op["ins"]:
+            last_reader[i] = n
     consumed = set()
-    for op in op_list:
+    for n, op in enumerate(op_list):
         ins = [vals[i] for i in op["ins"]]
+        if load is not None:
+            ins = [a if a.dtype.kind in "iu" else np.asarray(load(n, i, a), dtype=np.float64)
+                   for i, a in zip(op["ins"], ins)]
         if op["kind"] == CACHED_ATTENTION:
             # the one op with a side effect: rows `pos` of its two state tensors are replaced
             ctx, kc, vc = ops.cached_attention(*ins, scale=op.get("attrs", {}).get("scale", 1.0))
@@ -92,6 +101,10 @@ def run_graph(tensors, op_list, feeds, keep_all=False, store=None):
                 tensors[tid].get("name"), o.shape, tensors[tid]["dims"])
             vals[tid] = o if store is None else np.asarray(store(tid, o), dtype=np.float64)
         consumed.update(op["ins"])
+        if not keep_all:
+            for i in set(op["ins"]):
+                if last_reader[i] == n and i not in feeds and tensors[i].get("kind") not in (1, STATE):
+                    del vals[i]
     if keep_all:
         return vals
     return {tid: v for tid, v in vals.items()

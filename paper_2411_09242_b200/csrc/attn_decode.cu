@@ -91,7 +91,7 @@ __device__ __forceinline__ uint4 pack16<__nv_bfloat16>(const float (&v)[8]) {
 // Rotary embedding (pairs (d, d + D/2)) of one row of D = LPR * V elements spread over LPR adjacent lanes, lane li
 // holding elements li*V .. li*V + V-1, at position pos. Every lane of the warp must call it.
 template <int V, int LPR>
-__device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, float log2_base) {
+__device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, double log2_base) {
   constexpr int D = LPR * V, half = D / 2;
   float partner[V];
 #pragma unroll
@@ -100,14 +100,8 @@ __device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, float
   for (int i = 0; i < V; ++i) {
     const int d = li * V + i;
     const int dd = d < half ? d : d - half;
-    const float inv_freq = exp2f(-2.f * dd / D * log2_base);
-    // two-step reduction of the angle to [-pi, pi] (exact product k * 2pi_hi in the fused multiply-add), then the
-    // hardware sine / cosine, whose absolute error there is about 2^-21
-    const float ang = pos * inv_freq;
-    const float kk = rintf(ang * 0.15915494309189535f);
-    float r = fmaf(-kk, 6.2831854820251465f, ang);
-    r = fmaf(-kk, -1.7484555e-7f, r);
-    const float sn = __sinf(r), cs = __cosf(r);
+    float sn, cs;
+    rope_sincos(pos, dd, D, log2_base, sn, cs);
     x[i] = d < half ? x[i] * cs - partner[i] * sn : x[i] * cs + partner[i] * sn;
   }
 }

@@ -387,7 +387,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (!ok) *abort_flag = 1;
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (*abort_flag) { ok = false; break; }   // read right after the barrier: every thread sees the same value
-      const float m_tile = fmaxf(xj[row], xj[128 + row]) * p.scale_log2;
+      // The reference point of the exponentials is rounded up to a whole number (base-2 domain): every P entry is
+      // then 2^(t - n) with n an integer, so its bf16 rounding is that of 2^t itself, the same whichever tile
+      // first set the maximum and however often it moved, and the rescale factors below are exact powers of two.
+      const float m_tile = ceilf(fmaxf(xj[row], xj[128 + row]) * p.scale_log2);
       if (j == 0) {
         m_used = m_tile;
       } else {

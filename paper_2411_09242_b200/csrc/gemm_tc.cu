@@ -11,7 +11,8 @@
 // Two accumulators (2 x BN tensor-memory columns) let the epilogue of tile i overlap the MMAs of
 // tile i+1. Operands may be K-major or MN-major in global memory (row-/column-/head-major
 // tensors): the TMA box and the shared-memory matrix descriptor follow the operand's major, so
-// no transpose kernel ever runs. No cluster multicast is used anywhere.
+// no transpose kernel ever runs. No load uses cluster multicast; the only multicast is the cta_group::2
+// tcgen05.commit that arrives on both CTAs' mbarriers of a pair.
 //
 // Every wait is bounded: a wait that does not complete within about a second records a code in
 // the arena header and the CTA drains and exits; the host reads the code with fluid_status().
@@ -87,6 +88,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if ((++spins & 255) == 0 && clock64() - t0 > kWaitCycles) return false;
   }
   return true;
+}
+// The same wait with one answer for the whole warp, for code that goes on to warp-synchronous instructions
+// (tcgen05.ld, named barriers): each lane times its own wait, so without the vote a barrier that completes right
+// at the limit could let some lanes pass and others give up.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity));
 }
 
 // Every tensor map is padded to rank 5 (unit dims), so one instruction form serves all operands.
@@ -664,6 +671,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kEpiWarps); }
     *abort_flag = 0;
+    abort_flag[2] = 0;   // split-K epilogue: set when a warp's accumulator wait gave up
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
@@ -852,7 +860,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           rbs[i] = g.has_res ? rbz + (live ? split_off(mi, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
         }
       }
-      if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
+      bool got = mbar_wait_warp(tfull_bar(acc), acc_ph);
+      if (SPLIT) {
+        // the eight epilogue warps meet at named barriers below: either all of them go on or none does
+        if (!got && lane == 0) abort_flag[2] = 1;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        got = abort_flag[2] == 0;
+      }
+      if (!got) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * bn);
       if (!SPLIT) {
@@ -1163,7 +1178,7 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   bool have_acc = false;
   if (warp >= 2) {
     // ---------------- this CTA's partial tile -> shared memory, [128 rows][bn] fp32 over the drained stages ----------------
-    have_acc = mbar_wait(tfull, 0u);
+    have_acc = mbar_wait_warp(tfull, 0u);
     if (!have_acc && lane == 0) {
       if (!*abort_flag) atomicOr(p.status, 0x4u);
       *abort_flag = 1;
@@ -1220,7 +1235,7 @@ gemm_tc_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     FinalCtx f;
     f.C = g.C; f.R = g.R; f.bias = g.has_bias ? static_cast<const __nv_bfloat16*>(g.bias) : nullptr;
     f.cs4 = g.c_s[4]; f.rs4 = g.r_s[4]; f.N0 = g.N0; f.scale = g.scale;
-    bool got = mbar_wait(recv_bar, 0u);           // every peer's slice has landed (or a peer gave up)
+    bool got = mbar_wait_warp(recv_bar, 0u);          // every peer's slice has landed (or a peer gave up)
     if (!got && lane == 0) {
       if (!*abort_flag) atomicOr(p.status, 0x8u);
       *abort_flag = 1;
@@ -1524,7 +1539,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         cbs[i] = cbz + (live ? split_off(mi, g.M0, g.c_s[2], g.c_s[3]) : 0);
         rbs[i] = g.has_res ? rbz + (live ? split_off(mi, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
       }
-      if (!mbar_wait(tfull_bar(acc), acc_ph)) { ok = false; break; }
+      if (!mbar_wait_warp(tfull_bar(acc), acc_ph)) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * PN);
       if (EPI == EPI_SWIGLU) epilogue_tile_swiglu(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
@@ -1940,6 +1955,40 @@ extern "C" int fluid_gemm_bf16_static_scratch(const void* dev_a, const void* dev
   if (err != cudaSuccess) {
     set_error("static-scratch GEMM: %s", cudaGetErrorString(err));
     return FLUID_ECUDA;
+  }
+  return FLUID_OK;
+}
+
+extern "C" int fluid_static_scratch_status(fluid_stream stream, int* device_status) {
+  using namespace fluid;
+  if (!device_status) {
+    set_error("static-scratch status: null argument");
+    return FLUID_EINVAL;
+  }
+  *device_status = 0;
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess || dev < 0 || dev >= 64) {
+    set_error("static-scratch status: no current device (%s)", cudaGetErrorString(err));
+    return FLUID_ECUDA;
+  }
+  void* addr = nullptr;
+  {
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    addr = g_static_addr[dev];
+  }
+  err = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  uint32_t word = 0;
+  // no call on this device yet: the array was never handed to a kernel, nothing to read
+  if (err == cudaSuccess && addr) err = cudaMemcpy(&word, addr, sizeof(word), cudaMemcpyDeviceToHost);
+  if (err != cudaSuccess) {
+    set_error("static-scratch status: %s", cudaGetErrorString(err));
+    return FLUID_ECUDA;
+  }
+  *device_status = (int)word;
+  if (word != 0) {
+    set_error("static-scratch GEMM: a device-side wait expired (code 0x%x); the output is incomplete", word);
+    return FLUID_ETIMEOUT;
   }
   return FLUID_OK;
 }

@@ -106,7 +106,7 @@ struct RopeParams {
   int dims[4];        // B, S, nh, D
   int64_t st[4];      // element strides of x and y (same layout) per logical dim
   int order[4];       // logical dims, slowest to fastest, in memory
-  float base;
+  double log2_base;   // log2 of the rotary base
   int interleaved;
   const int* pos;     // device: position of row 0 (null = 0)
   int pos_stride;     // 0: one position for the batch, 1: pos[b] per sequence
@@ -175,7 +175,7 @@ struct AttnDecodeParams {
   int B, NH, NKV, D, Tmax;
   float scale_log2;       // scale * log2(e)
   int rope;               // 1: q and k arrive unrotated; the step applies the rotary embedding (pairs (d, d + D/2)) at position *pos
-  float rope_log2_base;
+  double rope_log2_base;
   int64_t q_sb, q_sh, k_sb, k_sh, v_sb, v_sh, o_sb, o_sh;   // element strides of batch and head
 };
 // GEMM with at most 16 rows and both operands k-contiguous (bf16): the weights stream through the SM once.

@@ -722,10 +722,9 @@ __global__ void rope_kernel(RopeParams p, int64_t total) {
     const int pr = idx[3];
     const int d0 = p.interleaved ? 2 * pr : pr, d1 = p.interleaved ? 2 * pr + 1 : pr + half;
     const int64_t base = idx[0] * p.st[0] + idx[1] * p.st[1] + idx[2] * p.st[2];
-    const float inv_freq = exp2f(-2.f * pr / p.dims[3] * log2f(p.base));
     float sn, cs;
     const int pos0 = p.pos ? p.pos[idx[0] * p.pos_stride] : 0;
-    sincosf((idx[1] + pos0) * inv_freq, &sn, &cs);
+    rope_sincos(idx[1] + pos0, pr, p.dims[3], p.log2_base, sn, cs);
     const T* x = static_cast<const T*>(p.x);
     T* y = static_cast<T*>(p.y);
     const float a = to_f(x[base + d0 * p.st[3]]), b = to_f(x[base + d1 * p.st[3]]);
@@ -741,7 +740,6 @@ __global__ void __launch_bounds__(256) rope_vec_kernel(RopeParams p, int64_t tot
   pdl_launch_dependents();
   pdl_wait();
   const int D = p.dims[3], half = D / 2, cpr = half / 8;
-  const float lb = log2f(p.base);
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     int64_t rem = i;
     const int c = int(rem % cpr); rem /= cpr;
@@ -752,15 +750,7 @@ __global__ void __launch_bounds__(256) rope_vec_kernel(RopeParams p, int64_t tot
     float cs[8], sn[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const float inv_freq = exp2f(-2.f * (c * 8 + j) / D * lb);
-      // two-step reduction of the angle to [-pi, pi] (exact product k * 2pi_hi in the fused multiply-add), then the
-      // hardware sine / cosine, whose absolute error there is about 2^-21
-      const float ang = (s + pos0) * inv_freq;
-      const float k = rintf(ang * 0.15915494309189535f);
-      float r = fmaf(-k, 6.2831854820251465f, ang);
-      r = fmaf(-k, -1.7484555e-7f, r);
-      sn[j] = __sinf(r);
-      cs[j] = __cosf(r);
+      rope_sincos(s + pos0, c * 8 + j, D, p.log2_base, sn[j], cs[j]);
     }
     const int h_end = min(p.dims[2], (hg + 1) * ROPE_HG);
     for (int h = hg * ROPE_HG; h < h_end; ++h) {

@@ -92,6 +92,7 @@ _SIGNATURES = {
     "fluid_status": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]),
     "fluid_gemm_bf16_static_scratch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                                   C.c_void_p]),
+    "fluid_static_scratch_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int)]),
     "fluid_last_error": (C.c_char_p, []),
     "fluid_launch_count": (C.c_int64, []),
 }
@@ -302,6 +303,15 @@ def fluid_gemm_bf16_static_scratch(dev_a, dev_b, dev_bias, dev_c, m, n, k, strea
     own fixed device array: for callers that have no arena and may not allocate one."""
     _check(lib().fluid_gemm_bf16_static_scratch(C.c_void_p(dev_a), C.c_void_p(dev_b), C.c_void_p(dev_bias or None),
                                                 C.c_void_p(dev_c), m, n, k, C.c_void_p(stream)))
+
+
+def fluid_static_scratch_status(stream=0):
+    """Status word of the last static-scratch GEMM on the current device (0 = every wait completed); synchronises."""
+    st = C.c_int()
+    rc = lib().fluid_static_scratch_status(C.c_void_p(stream), C.byref(st))
+    if rc not in (FLUID_OK, FLUID_ETIMEOUT):
+        _check(rc)
+    return st.value
 
 
 def fluid_launch_count():

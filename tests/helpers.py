@@ -68,9 +68,9 @@ def run_gpu(desc, feeds, candidates=None, poison=True, **opts):
     return dict(zip(desc.outputs, outs)), plan, runner
 
 
-def run_oracle(desc, feeds, keep_all=False, store=None):
+def run_oracle(desc, feeds, keep_all=False, store=None, load=None):
     from oracle import graph_exec
-    return graph_exec.run_graph(desc.tensors, desc.ops, feeds, keep_all=keep_all, store=store)
+    return graph_exec.run_graph(desc.tensors, desc.ops, feeds, keep_all=keep_all, store=store, load=load)
 
 
 def tol_for(dtype):
@@ -84,6 +84,78 @@ def assert_close(got, ref, dtype, what="", tol=None):
     err = float(np.max(np.abs(got - ref)))
     assert np.all(np.isfinite(got)), f"{what}: non-finite output"
     assert err <= tol * scale, f"{what}: max|err| {err:.3e} > {tol:g} * max|ref| {scale:.3e}"
+
+
+def storage_hooks(desc, plan):
+    """(store, load) for run_oracle that round each tensor the way `plan` keeps it, read from the plan itself:
+      * an op output that owns an arena record (or aliases one) is rounded to that record's dtype: bf16, or
+        fp32 for the residual-stream tensors the planner keeps wide;
+      * a graph output is rounded to its declared dtype;
+      * an op output with no record (folded into a fused step: scores, gate, up, pre-activation sums) is not
+        rounded at all: it only ever exists in fp32 accumulators;
+      * a tensor with a bf16 twin record is read rounded to bf16 by the tensor-core ops (LINEAR, BMM) and wide
+        by everything else;
+      * inside a fused-attention step the probabilities are a tensor-core operand: BMM_PV reads the bf16 rounding
+        of the exponentials 2^(t - n) (n a whole number per row) over the sum of the unrounded exponentials,
+        which is how the fused kernel forms P.
+    With these hooks the oracle is still exact fp64 arithmetic; only what is *stored* is rounded. The distance
+    between this run and the plain oracle is the floor no executor that stores these dtypes can get under."""
+    T = desc.tensors
+    recs = {}
+    twins = set()
+    for r in plan.records():
+        if r["tensor"] < 0:
+            continue
+        if r["twin"]:
+            twins.add(r["tensor"])
+        else:
+            recs[r["tensor"]] = r["dtype"]
+    fused_p = {}              # (op index, probabilities) read inside a fused-attention step -> its SOFTMAX op
+    for s in plan.steps():
+        if s["kernel_name"] == "ATTN":
+            for o in s["ops"]:
+                if desc.ops[o]["kind"] == synth.BMM_PV:
+                    probs = desc.ops[o]["ins"][0]
+                    fused_p[(o, probs)] = next(d for d in desc.ops if probs in d["outs"] and d["kind"] == synth.SOFTMAX)
+    scores_of = {sm["ins"][0]: None for sm in fused_p.values()}     # score tensors to hold on to until P is formed
+
+    def rb(a):
+        return synth.round_bf16(np.asarray(a, dtype=np.float32)).astype(np.float64)
+
+    def fused_probabilities(sm):
+        """What the fused kernel feeds the tensor core as P: the exponentials relative to a whole-number reference
+        point in the base-2 domain, rounded to bf16, over the sum of the unrounded exponentials."""
+        sc = scores_of[sm["ins"][0]] * (sm["attrs"].get("scale", 1.0) * np.log2(np.e))
+        scores_of[sm["ins"][0]] = None
+        if sm["attrs"].get("causal"):
+            allowed = np.arange(sc.shape[-1])[None, :] <= np.arange(sc.shape[-2])[:, None]
+            sc = np.where(allowed, sc, -np.inf)
+        e = np.exp2(sc - np.ceil(np.max(sc, axis=-1, keepdims=True)))
+        return rb(e) / np.sum(e, axis=-1, keepdims=True)
+
+    def store(tid, a):
+        if tid in scores_of:
+            scores_of[tid] = a
+        if T[tid]["kind"] == synth.OUTPUT:
+            dt = T[tid]["dtype"]
+        else:
+            dt = recs.get(plan.tensor_info(tid).alias_of)
+        if dt == synth.BF16:
+            return rb(a)
+        if dt == synth.F32:
+            return np.asarray(a, dtype=np.float32).astype(np.float64)
+        return a
+
+    def load(op_index, tid, a):
+        kind = desc.ops[op_index]["kind"]
+        if (op_index, tid) in fused_p:
+            return fused_probabilities(fused_p[(op_index, tid)])
+        if kind in (synth.LINEAR, synth.BMM_QK, synth.BMM_PV) and T[tid]["kind"] == synth.ACT \
+                and plan.tensor_info(tid).alias_of in twins:
+            return rb(a)
+        return a
+
+    return store, load
 
 
 def single_op_graph(kind, in_shapes, out_shape, dtype, attrs=None, in_kinds=None):

@@ -1,11 +1,11 @@
 """Parity at the full sizes of the benchmark configurations, in the configuration bench.py times (planned layouts, fused
-epilogues, tensor-core GEMMs). Where a full oracle pass is too slow, outputs are sampled in a way the
-oracle can compute exactly: a causal model's first rows depend only on the first tokens."""
+epilogues, tensor-core GEMMs): whole outputs against full passes of the fp64 oracle (minutes of host time for the two
+largest shapes), and every launch on its own against the oracle op on sampled rows."""
 import numpy as np
 import pytest
 
 from paper_2411_09242_b200 import fluid, synth
-from tests.helpers import assert_close, check_steps_sampled, run_gpu, run_oracle
+from tests.helpers import assert_close, check_steps_sampled, run_gpu, run_oracle, storage_hooks
 
 pytestmark = pytest.mark.gpu
 
@@ -32,51 +32,79 @@ def test_bert_base_shape_full():
     plan.close()
 
 
-def _prefix_reference(full, S_prefix, L=None):
-    """Oracle output for batch row 0, first S_prefix positions, using the full model's weights."""
-    cfg = synth.scaled(full.cfg, B=1, S=S_prefix, **({"L": L} if L else {}))
-    small = synth.build_model(cfg, materialize=False)
-    name_to_full = {full.graph.tensors[t]["name"]: a for t, a in full.consts.items()}
-    feeds = {}
-    for tid, td in enumerate(small.graph.tensors):
-        if td["kind"] == synth.CONST:
-            a = name_to_full[td["name"]]
-            feeds[tid] = a[:S_prefix] if td["name"] == "pos_table" else a
-    feeds[small.graph.inputs[0]] = full.ids[:1, :S_prefix]
-    out = run_oracle(small.graph, feeds)
-    return out[small.graph.outputs[0]]
-
-
-def test_gpt2_small_shape_full_sampled_prefix():
+def test_gpt2_small_shape_full():
+    """Every element of the hidden state [4, 1024, 768] and of the last-token logits [4, 50257] against one full
+    pass of the fp64 oracle, at the stated bf16 tolerance."""
     m = synth.build_model(synth.CONFIGS["gpt2_small"])
+    ref = run_oracle(m.graph, feeds_of(m))
     got, plan, _ = run_gpu(m.graph, feeds_of(m), synth.default_candidates(m.graph))
-    hidden, logits = (got[t] for t in m.graph.outputs)
-    ref = _prefix_reference(m, 192)
-    assert_close(hidden[:1, :192], ref, synth.BF16, "gpt2_small hidden prefix")
-    # every batch row went through the same kernels: rows with equal prefixes would agree; check
-    # finiteness and scale of the rest, and the tied-head logits against the GPU's own hidden state
-    assert np.all(np.isfinite(hidden)) and np.all(np.isfinite(logits))
-    tok = next(a for t, a in m.consts.items() if m.graph.tensors[t]["name"] == "tok_table").astype(np.float64)
-    assert_close(logits, hidden[:, -1, :] @ tok.T, synth.BF16, "gpt2_small logits from hidden")
+    for t in m.graph.outputs:
+        assert_close(got[t], ref[t], synth.BF16, f"gpt2_small {m.graph.tensors[t]['name']} (whole tensor)")
+    assert "PERMUTE" not in [s["kernel_name"] for s in plan.steps()]
     plan.close()
 
 
-def test_llama_shape_full_sampled_prefix():
+def test_llama_shape_full():
+    """The Llama-shaped config, whole outputs, against two full oracle passes.
+
+    With hidden 4096 / FFN 11008 and N(0, 0.02) weights this four-layer network amplifies a relative perturbation
+    of a stored activation several times over on its way to the output. (i) An fp64 run that does nothing but round
+    each tensor to the dtype the plan stores it in (read from the plan: bf16 GEMM operands, fp32 residual stream,
+    nothing for tensors fused away) already lands about 1.8 % of max|ref| from the unrounded oracle: the stated 1e-2
+    cannot be met by any executor that keeps bf16 activations for this shape. (ii) Against that storage-rounded
+    oracle the GPU differs only by arithmetic (fp32 accumulation order in the tensor core, ex2.approx) and by which
+    way borderline values round; those flips (0.3 % of the first projection's elements, see the cascade test below)
+    grow through the same amplification, so the two agree to about 1 %, not to a rounding unit: bounded at 1.5e-2.
+    (iii) The distance to the unrounded oracle is bounded at 2.5e-2 (measured 1.86 %, the floor itself being 1.82 %)."""
     m = synth.build_model(synth.CONFIGS["llama"])
-    got, plan, _ = run_gpu(m.graph, feeds_of(m), synth.default_candidates(m.graph))
-    hidden, logits = (got[t] for t in m.graph.outputs)
-    # With hidden 4096 / FFN 11008 and N(0,0.02) weights the residual stream grows to ~20 and rounding the
-    # GEMM operands to bf16 alone moves the final output by 2.3 % of max|ref|: an fp64 run that does nothing
-    # but round the tensors the plan stores in bf16 shows the same figure (0.1086 vs the GPU's 0.1085). The
-    # 1e-2 bar therefore cannot hold end to end against the unrounded oracle for this shape; the kernels are
-    # held to 2^-7 launch by launch at full size (test below) and the end-to-end gap is bounded at 3e-2.
-    ref = _prefix_reference(m, 96)
-    assert_close(hidden[:1, :96], ref, synth.BF16, "llama hidden prefix vs unrounded oracle", tol=3e-2)
-    w = next(a for t, a in m.consts.items() if m.graph.tensors[t]["name"] == "W_lm").astype(np.float64)
-    assert_close(logits, hidden[:, -1, :] @ w, synth.BF16, "llama logits from hidden")
+    g = m.graph
+    got, plan, _ = run_gpu(g, feeds_of(m), synth.default_candidates(g))
+    store, load = storage_hooks(g, plan)
+    ref = run_oracle(g, feeds_of(m))
+    ref_stored = run_oracle(g, feeds_of(m), store=store, load=load)
+    for t in g.outputs:
+        name = g.tensors[t]["name"]
+        scale = float(np.max(np.abs(ref[t])))
+        floor = float(np.max(np.abs(ref_stored[t] - ref[t]))) / scale
+        gap = float(np.max(np.abs(got[t] - ref[t]))) / scale
+        arith = float(np.max(np.abs(got[t] - ref_stored[t]))) / scale
+        print(f"llama {name}: storage floor {floor:.4%}, GPU vs plain oracle {gap:.4%}, GPU vs storage-rounded oracle {arith:.4%}")
+        if g.tensors[t]["dims"][-1] == m.cfg.H:
+            assert floor > 1e-2, "the storage floor moved under the stated tolerance: tighten this test to 1e-2"
+        assert_close(got[t], ref_stored[t], synth.BF16, f"llama {name} vs storage-rounded oracle", tol=1.5e-2)
+        assert_close(got[t], ref[t], synth.BF16, f"llama {name} vs plain oracle", tol=2.5e-2)
     # Greedy-by-Size is a heuristic: with the SwiGLU step fused (gate and up never stored) it lands 15 % above the
     # largest live set on this shape; on the other three shapes it meets the bound exactly
     assert plan.live_bound_bytes <= plan.arena_bytes <= 1.2 * plan.live_bound_bytes
+    plan.close()
+
+
+def test_llama_first_layer_rounding_cascade():
+    """Why the Llama shape agrees with the storage-rounded oracle to a per cent and not to a rounding unit. One layer
+    at full widths, every tensor kept (no arena reuse), each stored tensor compared with the storage-rounded oracle's:
+    the first projections differ in well under 1 % of their elements (a bf16 rounding that went the other way,
+    because the tensor core's fp32 accumulation and the oracle's fp64 differ by ~1e-5 relative) and by ~2e-4 rms;
+    after attention, whose output mixes thousands of such inputs, an order of magnitude more elements differ; by the
+    end of the layer the difference is a few times 1e-3 rms, and the next layer starts from there. Every stored
+    tensor of the layer still agrees within one bf16 unit of max|ref| (2^-7)."""
+    m = synth.build_model(synth.scaled(synth.CONFIGS["llama"], L=1))
+    g = m.graph
+    got, plan, runner = run_gpu(g, feeds_of(m), synth.default_candidates(g), no_reuse=1)
+    store, load = storage_hooks(g, plan)
+    stored = run_oracle(g, feeds_of(m), keep_all=True, store=store, load=load)
+    frac, rms = {}, {}
+    for s in plan.steps():
+        for t in s["outs"]:
+            have = got[t] if g.tensors[t]["kind"] == synth.OUTPUT else runner.read_tensor(t)
+            name = g.tensors[t]["name"]
+            d = np.abs(have - stored[t])
+            frac[name] = float(np.mean(d > 0))
+            rms[name] = float(np.sqrt(np.mean(d ** 2)) / np.sqrt(np.mean(stored[t] ** 2)))
+            print(f"{s['kernel_name']:10s} {name:16s} differing {frac[name]:.4f}  rms {rms[name]:.2e}  max {d.max() / np.abs(stored[t]).max():.2e}")
+            assert_close(have, stored[t], synth.BF16, f"one layer, {name} vs storage-rounded oracle", tol=2 ** -7)
+    assert frac["l0.q"] < 0.01 and rms["l0.q"] < 5e-4
+    assert frac["l0.ctx_h"] > 5 * frac["l0.q"]
+    assert rms["final_norm.out"] > 5 * rms["l0.q"]
     plan.close()
 
 

@@ -42,11 +42,22 @@ def test_chain_lower_bound_and_hand_example():
 
 
 def test_first_fit_versus_best_fit():
-    # two gaps fit the last tensor: first-fit takes the lower, best-fit the tighter one
-    r = [(0, 1024, 0, 0), (1, 1024, 1, 1), (2, 512, 0, 0), (3, 2048, 0, 1), (4, 256, 1, 1)]
+    # Hand-worked: P, Q, R, S are all alive at step 0, so they stack by size (ties: smaller id first):
+    #   P 1024 @ H, Q 512 @ H+1024, R 512 @ H+1536, S 256 @ H+2048.
+    # T (256 bytes, alive at step 2 only) conflicts with Q and S alone, which leaves it two gaps: P's old range
+    # (1024 bytes at H) and R's old range (512 bytes at H+1536). The pseudo-code's first slot is the lower one;
+    # the prose's "most suitable" slot is the tighter one. The two policies must therefore differ here.
+    r = [(0, 1024, 0, 0), (1, 512, 0, 2), (2, 512, 0, 0), (3, 256, 0, 2), (4, 256, 2, 2)]
     off_f, peak_f = A.greedy_by_size(r, policy="first")
     off_b, peak_b = A.greedy_by_size(r, policy="best")
+    assert off_f == {0: H, 1: H + 1024, 2: H + 1536, 3: H + 2048, 4: H}
+    assert off_b == {0: H, 1: H + 1024, 2: H + 1536, 3: H + 2048, 4: H + 1536}
+    assert peak_f == peak_b == H + 2304
     assert A.check_arena(r, off_f, peak_f) == [] and A.check_arena(r, off_b, peak_b) == []
+    # equally tight gaps: best fit falls back to the lower offset
+    r = [(0, 512, 0, 0), (1, 512, 0, 2), (2, 512, 0, 0), (3, 256, 0, 2), (4, 256, 2, 2)]
+    off_b, _ = A.greedy_by_size(r, policy="best")
+    assert off_b[4] == H
 
 
 def test_sort_order_ties():
