@@ -91,7 +91,7 @@ __device__ __forceinline__ uint4 pack16<__nv_bfloat16>(const float (&v)[8]) {
 // Rotary embedding (pairs (d, d + D/2)) of one row of D = LPR * V elements spread over LPR adjacent lanes, lane li
 // holding elements li*V .. li*V + V-1, at position pos. Every lane of the warp must call it.
 template <int V, int LPR>
-__device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, double log2_base) {
+__device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, const RopeFreq& freq) {
   constexpr int D = LPR * V, half = D / 2;
   float partner[V];
 #pragma unroll
@@ -101,7 +101,7 @@ __device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, doubl
     const int d = li * V + i;
     const int dd = d < half ? d : d - half;
     float sn, cs;
-    rope_sincos(pos, dd, D, log2_base, sn, cs);
+    rope_sincos(pos, rope_freq(freq, dd, D), sn, cs);
     x[i] = d < half ? x[i] * cs - partner[i] * sn : x[i] * cs + partner[i] * sn;
   }
 }
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
   {
     const uint4 raw = *reinterpret_cast<const uint4*>(static_cast<const T*>(p.q) + b * p.q_sb + h * p.q_sh + li * V);
     unpack16<T>(raw, qv);
-    if (p.rope) rotate_row<V, LPR>(qv, li, t, p.rope_log2_base);
+    if (p.rope) rotate_row<V, LPR>(qv, li, t, p.rope_freq);
 #pragma unroll
     for (int i = 0; i < V; ++i) qv[i] *= p.scale_log2;
   }
@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(AttnDecodePara
   if (p.rope) {
     float kf[V];
     unpack16<T>(k_fresh, kf);
-    rotate_row<V, LPR>(kf, li, t, p.rope_log2_base);
+    rotate_row<V, LPR>(kf, li, t, p.rope_freq);
     k_fresh = pack16<T>(kf);   // rounded as the cache will hold it: later steps read exactly what this one used
   }
 

@@ -6,8 +6,11 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cmath>
 #include <cstdlib>
 #include <utility>
+
+#include "kernels.h"
 
 namespace fluid {
 
@@ -130,15 +133,19 @@ __device__ __forceinline__ float gelu_tanh(float x) {
   const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
   return 0.5f * x * (1.f + tanhf(u));
 }
-// Rotary angle pos * base^(-2i/D) as (sin, cos). Frequency, product and reduction to [-pi, pi] in double: in fp32
+// Rotary angle pos * f as (sin, cos), f = base^(-2i/D) in double. Product and reduction to [-pi, pi] in double: in fp32
 // the frequency alone is off by ~1e-6 relative, which at position 2047 is 2e-3 rad, as much as the bf16 rounding of
 // the rotated value. The hardware sine / cosine on the reduced angle have an absolute error of about 2^-21.
-__device__ __forceinline__ void rope_sincos(int pos, int i, int D, double log2_base, float& sn, float& cs) {
-  const double ang = (double)pos * exp2(-2.0 * i / D * log2_base);
+__device__ __forceinline__ void rope_sincos(int pos, double inv_freq, float& sn, float& cs) {
+  const double ang = (double)pos * inv_freq;
   const double k = rint(ang * 0.15915494309189535);
   const float r = (float)fma(-k, 6.283185307179586, ang);
   sn = __sinf(r);
   cs = __cosf(r);
+}
+__device__ __forceinline__ double rope_inv_freq(int i, int D, double log2_base) { return exp2(-2.0 * i / D * log2_base); }
+__device__ __forceinline__ double rope_freq(const RopeFreq& t, int i, int D) {
+  return i < 64 ? t.f[i] : rope_inv_freq(i, D, t.log2_base);
 }
 __device__ __forceinline__ float silu(float x) { return x / (1.f + __expf(-x)); }
 

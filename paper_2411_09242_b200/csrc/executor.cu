@@ -202,7 +202,7 @@ int finalize_steps(fluid_plan_s* p) {
           q.st[i] = st[i];
           q.order[i] = p->cands[n.out][lo[n.out]][i];
         }
-        q.log2_base = std::log2(n.rope_base);
+        rope_freq_fill(q.freq, n.rope_base, (int)ty.dims[3]);
         q.interleaved = n.rope_interleaved;
         q.pos_stride = (n.pos >= 0 && T[n.pos].dims[0] > 1) ? 1 : 0;
         s.rope = q;
@@ -270,7 +270,7 @@ int finalize_steps(fluid_plan_s* p) {
         q.scale_log2 = (float)(n.scale * 1.4426950408889634);
         q.rope = n.rope_fused;
         q.pos_stride = T[n.pos].dims[0] > 1 ? 1 : 0;
-        q.rope_log2_base = std::log2(n.rope_base);
+        rope_freq_fill(q.rope_freq, n.rope_base, q.D);
         int64_t st[FLUID_MAX_RANK];
         perm_strides(p, n.a, st);   q.q_sb = st[0]; q.q_sh = st[2];
         perm_strides(p, n.b, st);   q.k_sb = st[0]; q.k_sh = st[2];

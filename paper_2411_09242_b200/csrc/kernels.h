@@ -3,6 +3,7 @@
 // bound constants and the caller's input/output pointers.
 #pragma once
 
+#include <cmath>
 #include <cstdint>
 
 #include <cuda_runtime.h>
@@ -99,6 +100,17 @@ struct SoftmaxParams {
                       // multiple of zero_block past the diagonal (the consumer reads no further)
 };
 
+// Rotary frequencies base^(-2i/D) of the first 64 pairs in double, computed once on the host (head dims up to 128);
+// pairs beyond that are computed on the device from log2_base.
+struct RopeFreq {
+  double log2_base;
+  double f[64];
+};
+inline void rope_freq_fill(RopeFreq& t, double base, int D) {
+  t.log2_base = std::log2(base);
+  for (int i = 0; i < 64; ++i) t.f[i] = std::exp2(-2.0 * i / D * t.log2_base);
+}
+
 struct RopeParams {
   const void* x;
   void* y;
@@ -106,7 +118,7 @@ struct RopeParams {
   int dims[4];        // B, S, nh, D
   int64_t st[4];      // element strides of x and y (same layout) per logical dim
   int order[4];       // logical dims, slowest to fastest, in memory
-  double log2_base;   // log2 of the rotary base
+  RopeFreq freq;      // base^(-2i/D), double
   int interleaved;
   const int* pos;     // device: position of row 0 (null = 0)
   int pos_stride;     // 0: one position for the batch, 1: pos[b] per sequence
@@ -175,7 +187,7 @@ struct AttnDecodeParams {
   int B, NH, NKV, D, Tmax;
   float scale_log2;       // scale * log2(e)
   int rope;               // 1: q and k arrive unrotated; the step applies the rotary embedding (pairs (d, d + D/2)) at position *pos
-  double rope_log2_base;
+  RopeFreq rope_freq;
   int64_t q_sb, q_sh, k_sb, k_sh, v_sb, v_sh, o_sb, o_sh;   // element strides of batch and head
 };
 // GEMM with at most 16 rows and both operands k-contiguous (bf16): the weights stream through the SM once.
