@@ -131,6 +131,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&q)[32
 }
 
 constexpr int kSoftmaxThreads = 256;
+#ifndef FLUID_ATTN_POLY_EVERY
+#define FLUID_ATTN_POLY_EVERY 0
+#endif
+// One pair of exponentials in this many goes to the fused-multiply-add pipe instead of the special-function unit (0: none).
+// Measured with a share of 1/4 and 1/2: slower (2 x 4096 x 32 x 128: 918 -> 807 -> 652 TFLOP/s): a softmax warp is bound by
+// the instructions it can issue alone on its scheduler, not by the special-function unit, and the polynomial costs 8.
+constexpr int kPolyEvery = FLUID_ATTN_POLY_EVERY;
 constexpr int kAttnThreads = kSoftmaxThreads + 64;   // warps 0-7 softmax (two threads per query row), warp 8 MMAs, warp 9 loads
 
 // Warps 0-7: softmax. Warp 8, one thread: every tcgen05.mma. Warp 9: TMA loads. They meet only at mbarriers:
@@ -486,33 +493,499 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
 }
 
+
+// ---- two query tiles per CTA, probabilities in tensor memory ------------------------------------------------------
+// One CTA = one (batch, head) and 256 consecutive queries, as two 128-row tiles that share every K / V tile the CTA
+// loads. Warps 0-3 are the softmax of query tile 0, warps 4-7 of tile 1 (one thread per query row: the row's maximum
+// and sum never leave the thread), warp 8 (one thread) issues every tcgen05.mma, warp 9 the TMA loads. Tensor memory:
+// S_0, S_1 (128 fp32 columns each), O_0, O_1 (D columns each). A softmax thread reads its row of S_t, writes the bf16
+// probabilities back over the same columns (two per 32-bit column, 64 columns), and P_t.V runs with the A operand
+// taken from tensor memory: P never passes through shared memory. Per query tile the chain S = Q.K_j^T -> softmax ->
+// O += P.V_j is serial; the two tiles run half a step apart, so the tensor core works for one tile while the other
+// tile's softmax runs.
+//   q_full        both Q tiles have landed                           TMA -> MMA
+//   k_full[s], v_full[s]   K / V stage s has landed                  TMA -> MMA
+//   k_free[s], v_free[s]   every MMA that reads stage s is complete  MMA commit -> loader
+//   s_full[t]     S_t holds Q_t.K_j^T                                MMA commit -> softmax t
+//   p_full[t]     P_t is written (and S_t read)                      128 softmax threads -> MMA
+//   o_done[t]     O_t holds P_t.V_j                                  MMA commit -> softmax t (rescale, end)
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_c, uint32_t tmem_a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                             uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n .reg .b64 db;\n mov.b64 db, {%2, %3};\n setp.ne.b32 p, %5, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}"
+      ::"r"(tmem_c), "r"(tmem_a), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+}
+// Forms for a role that the whole warp runs in lockstep: every lane executes the instruction, one lane's carries a true
+// issue predicate.
+__device__ __forceinline__ void umma_ss_elect(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc,
+                                              uint32_t leader) {
+  asm volatile(
+      "{\n .reg .pred p, q;\n setp.ne.b32 p, %4, 0;\n setp.ne.b32 q, %5, 0;\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void umma_ts_elect(uint32_t tmem_c, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc,
+                                              uint32_t leader) {
+  asm volatile(
+      "{\n .reg .pred p, q;\n setp.ne.b32 p, %4, 0;\n setp.ne.b32 q, %5, 0;\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(tmem_c), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void umma_commit_elect(uint32_t bar, uint32_t leader) {
+  asm volatile(
+      "{\n .reg .pred q;\n setp.ne.b32 q, %1, 0;\n"
+      " @q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}"
+      ::"r"(bar), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&q)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3]), "r"(q[4]), "r"(q[5]), "r"(q[6]), "r"(q[7]), "r"(q[8]),
+      "r"(q[9]), "r"(q[10]), "r"(q[11]), "r"(q[12]), "r"(q[13]), "r"(q[14]), "r"(q[15])
+      : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity));
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// two fp32 lanes in one 64-bit register: one issue slot for two fused multiply-adds / additions
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+  return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x for x <= 0 on the fused-multiply-add pipe (no special-function unit): nearest-integer split by the 1.5 * 2^23
+// trick, degree-4 polynomial for 2^f on [-0.5, 0.5] (relative error < 3e-6, far below the bf16 rounding of P), the
+// integer part added into the exponent field. A share of each tile's exponentials goes this way so that the
+// special-function unit (4 lanes per clock and scheduler) is not what a softmax warp waits for.
+__device__ __forceinline__ float ex2_poly(float x) {
+  x = fmaxf(x, -125.f);
+  const float z = x + 12582912.f;
+  const float f = x - (z - 12582912.f);
+  float q = fmaf(0.009582852944731712f, f, 0.055906426161527634f);
+  q = fmaf(q, f, 0.24024099111557007f);
+  q = fmaf(q, f, 0.6931241750717163f);
+  q = fmaf(q, f, 1.0f);
+  return __int_as_float(__float_as_int(q) + (__float_as_int(z) << 23));
+}
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, const __grid_constant__ AttnParams p) {
+  constexpr int DC = D / 64;                       // 64-wide chunks of the head dim
+  constexpr uint32_t kTile = TQ * D * 2;           // bytes of one Q / K / V tile
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t sQ = raw, sK = sQ + 2 * kTile, sV = sK + 2 * kTile, bars = sV + 2 * kTile;
+  const uint32_t q_full = bars, k_full = bars + 8, v_full = bars + 24, k_free = bars + 40, v_free = bars + 56,
+                 s_full = bars + 72, p_full = bars + 88, o_done = bars + 104;
+  const uint32_t tmem_slot = bars + 120;
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
+  volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
+
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // heaviest first: with a causal mask the last query tiles see the most key tiles
+  const int n_bz = p.B * p.NH;
+  const int mt = (int(gridDim.x) / n_bz - 1) - int(blockIdx.x) / n_bz, bz = int(blockIdx.x) % n_bz;
+  const int h = bz % p.NH, b = bz / p.NH;
+  const int m0 = mt * 2 * TQ;
+  // key tiles each query tile needs (0: the tile lies beyond the sequence)
+  int n_kv[2];
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int mq = m0 + t * TQ;
+    int n = mq < p.S ? (p.S + TK - 1) / TK : 0;
+    if (p.causal && n) n = min(n, (mq + TQ - 1) / TK + 1);
+    n_kv[t] = n;
+  }
+  const int n_max = max(n_kv[0], n_kv[1]);
+  if (raw & 1023u) {   // cannot happen with the launch this file does; refuse rather than run misaligned tiles
+    if (threadIdx.x == 0) atomicOr(p.status, 0x100u | 0x08u);
+    return;
+  }
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(k_full + 8 * i, 1); mbar_init(v_full + 8 * i, 1); mbar_init(k_free + 8 * i, 1); mbar_init(v_free + 8 * i, 1);
+      mbar_init(s_full + 8 * i, 1); mbar_init(p_full + 8 * i, 128); mbar_init(o_done + 8 * i, 1);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  // S_t at columns 128 t (P_t over its first 64), O_t at 256 + D t
+
+  if (warp == 9) {
+    // ======================= loads =======================
+    const bool lead = lane == 0;
+    constexpr int NB = 2 * DC;               // boxes per tile
+    const bool k_lane = lane < NB, v_lane = lane >= NB && lane < 2 * NB;
+    const int bx = k_lane ? lane : lane - NB;
+    int cur[5] = {0, 0, 0, 0, 0}, inc[5] = {0, 0, 0, 0, 0};
+    uint32_t box_dst = 0;
+    if (k_lane) {
+      if (!p.k_mn_major) {          // [d chunk][128 keys][64 d]: box (dc, rh)
+        const int dc = bx >> 1, rh = bx & 1;
+        coords(p.k_sel, dc * 64, rh * 64, bz, p.k_b0, cur);
+        box_dst = sK + dc * 16384u + rh * 8192u;
+      } else {                      // [key chunk][D d-rows][64 keys]: box (sc, dc)
+        const int sc = bx / DC, dc = bx % DC;
+        coords(p.k_sel, dc * 64, sc * 64, bz, p.k_b0, cur);
+        box_dst = sK + sc * (D * 128u) + dc * 8192u;
+      }
+#pragma unroll
+      for (int d = 0; d < 5; ++d) inc[d] = p.k_sel[d] == 2 ? TK : 0;
+    } else if (v_lane) {
+      if (!p.v_k_major) {           // [d chunk][128 keys][64 d]  (MN-major B of P.V): box (dc, kc)
+        const int dc = bx >> 1, kc = bx & 1;
+        coords(p.v_sel, kc * 64, dc * 64, bz, p.v_b0, cur);
+        box_dst = sV + dc * 16384u + kc * 8192u;
+      } else {                      // [key chunk][D d-rows][64 keys]  (K-major B of P.V): box (kc, dh)
+        const int kc = bx / DC, dh = bx % DC;
+        coords(p.v_sel, kc * 64, dh * 64, bz, p.v_b0, cur);
+        box_dst = sV + kc * (D * 128u) + dh * 8192u;
+      }
+#pragma unroll
+      for (int d = 0; d < 5; ++d) inc[d] = p.v_sel[d] == 0 ? TK : 0;
+    }
+    uint32_t fail = 0;
+    int k_issued = 0, v_issued = 0;
+    auto load_k = [&](int j) {
+      const uint32_t bar = k_full + 8u * (j & 1);
+      if (lead) mbar_expect_tx(bar, kTile);
+      if (k_lane) {
+        tma_load5(box_dst + uint32_t(j & 1) * kTile, &map_k, bar, cur);
+#pragma unroll
+        for (int d = 0; d < 5; ++d) cur[d] += inc[d];
+      }
+      k_issued = j + 1;
+    };
+    auto load_v = [&](int j) {
+      const uint32_t bar = v_full + 8u * (j & 1);
+      if (lead) mbar_expect_tx(bar, kTile);
+      if (v_lane) {
+        tma_load5(box_dst + uint32_t(j & 1) * kTile, &map_v, bar, cur);
+#pragma unroll
+        for (int d = 0; d < 5; ++d) cur[d] += inc[d];
+      }
+      v_issued = j + 1;
+    };
+    auto all_ok = [&](bool mine) { return __shfl_sync(0xffffffffu, mine ? 1 : 0, 0) != 0; };   // lane 0 decides
+
+    pdl_wait();  // Q, K, V come from the previous steps
+    if (lead) {
+      const int n_q = n_kv[1] ? 2 : 1;
+      mbar_expect_tx(q_full, uint32_t(n_q) * kTile);
+      int c[5];
+      for (int t = 0; t < n_q; ++t)
+        for (int dc = 0; dc < DC; ++dc)
+          for (int rh = 0; rh < 2; ++rh) {
+            coords(p.q_sel, dc * 64, m0 + t * TQ + rh * 64, bz, p.q_b0, c);
+            tma_load5(sQ + uint32_t(t) * kTile + dc * 16384u + rh * 8192u, &map_q, q_full, c);
+          }
+    }
+    if (n_max > 0) { load_k(0); load_v(0); }
+    if (n_max > 1) { load_k(1); load_v(1); }
+    bool ok = true;
+    for (int j = 0; ok && j + 2 < n_max; ++j) {
+      const int st = j & 1;
+      const uint32_t ph = uint32_t(j >> 1) & 1u;
+      if (lead && !mbar_wait(k_free + 8u * st, ph)) { fail |= 0x40u; ok = false; }
+      ok = all_ok(ok);
+      if (!ok) break;
+      load_k(j + 2);
+      if (lead && !mbar_wait(v_free + 8u * st, ph)) { fail |= 0x80u; ok = false; }
+      ok = all_ok(ok && !*abort_flag);
+      if (!ok) break;
+      load_v(j + 2);
+    }
+    if (!ok && lead) {
+      *abort_flag = 1;
+      if (fail) atomicOr(p.status, 0x100u | fail);
+    }
+    if (lead && *abort_flag) {
+      // let loads still in flight land before the shared memory is given up (each wait is bounded)
+      for (int j = max(0, k_issued - 2); j < k_issued; ++j) mbar_wait(k_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
+      for (int j = max(0, v_issued - 2); j < v_issued; ++j) mbar_wait(v_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
+    }
+  } else if (warp == 8) {
+    // ======================= MMAs =======================
+    // The whole warp runs this role in lockstep and one lane's instructions carry the issue predicate. Kept
+    // convergent, the descriptor arithmetic stays on the uniform datapath, where tcgen05.mma takes its operands
+    // from; with the role under a one-lane branch every operand went through per-instruction register moves and a
+    // 128 x 128 x 16 instruction cost ~107 cycles to issue against the 64 the tensor core needs to run it.
+    {
+      const uint32_t leader = lane == 0 ? 1u : 0u;
+      uint32_t fail = 0;
+      const uint32_t idesc_s = make_idesc(TK, 0, p.k_mn_major);
+      const uint32_t idesc_o = make_idesc(D, 0, p.v_k_major ? 0 : 1);
+      const uint64_t dq = make_desc(sQ, 16, 1024);
+      const uint64_t dk = p.k_mn_major ? make_desc(sK, D * 128u, 1024) : make_desc(sK, 16, 1024);
+      const uint64_t dv = p.v_k_major ? make_desc(sV, 16, 1024) : make_desc(sV, 16384, 1024);
+      auto km_off = [](int kk) { return uint64_t(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4); };   // K-major operand, 64-wide chunks
+      const int last_t = n_kv[1] ? 1 : 0;    // the tile whose MMA is the last reader of a K / V stage (n_kv[1] >= n_kv[0] when tile 1 exists)
+      const uint32_t tm = __shfl_sync(0xffffffffu, tmem_base, 0);
+      auto issue_qk = [&](int t, int j) -> bool {   // S_t = Q_t.K_j^T
+        const int st = j & 1;
+        if (!mbar_wait_warp(k_full + 8u * st, uint32_t(j >> 1) & 1u)) { fail |= 0x20u; return false; }
+        tc_fence_after();
+        const uint64_t kb = dk + uint64_t(st) * (kTile >> 4), qb = dq + uint64_t(t) * (kTile >> 4);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk)
+          umma_ss_elect(tm + uint32_t(t * TK), qb + km_off(kk), kb + (p.k_mn_major ? uint64_t(kk * 128) : km_off(kk)), idesc_s,
+                        kk > 0 ? 1u : 0u, leader);
+        umma_commit_elect(s_full + 8u * t, leader);
+        if (t == last_t || j >= n_kv[1]) umma_commit_elect(k_free + 8u * st, leader);
+        return true;
+      };
+      auto issue_pv = [&](int t, int j) -> bool {   // O_t += P_t.V_j
+        const int st = j & 1;
+        if (!mbar_wait_warp(p_full + 8u * t, uint32_t(j) & 1u)) { fail |= 0x200u; return false; }
+        if (!mbar_wait_warp(v_full + 8u * st, uint32_t(j >> 1) & 1u)) { fail |= 0x20u; return false; }
+        tc_fence_after();
+        const uint64_t vb = dv + uint64_t(st) * (kTile >> 4);
+        const uint32_t tP = tm + uint32_t(t * TK), tO = tm + 2 * TK + uint32_t(t * D);
+#pragma unroll
+        for (int kk = 0; kk < TK / 16; ++kk)   // 16 keys = 8 packed columns of P per instruction
+          umma_ts_elect(tO, tP + uint32_t(kk * 8),
+                        vb + (p.v_k_major ? uint64_t(((kk >> 2) * (D * 128) + (kk & 3) * 32) >> 4) : uint64_t(kk * 128)), idesc_o,
+                        (j > 0 || kk > 0) ? 1u : 0u, leader);
+        umma_commit_elect(o_done + 8u * t, leader);
+        if (t == last_t || j >= n_kv[1]) umma_commit_elect(v_free + 8u * st, leader);
+        return true;
+      };
+      bool ok = mbar_wait_warp(q_full, 0);
+      if (!ok) fail |= 0x10u;
+      for (int t = 0; ok && t < 2; ++t)
+        if (n_kv[t] > 0) ok = issue_qk(t, 0);
+      for (int j = 0; ok && j < n_max; ++j) {
+        for (int t = 0; ok && t < 2; ++t) {
+          if (j >= n_kv[t]) continue;
+          ok = issue_pv(t, j);
+          if (ok && j + 1 < n_kv[t]) ok = issue_qk(t, j + 1);   // into the S tile whose probabilities were just consumed
+        }
+      }
+      if (!ok && leader) {
+        *abort_flag = 1;
+        atomicOr(p.status, 0x100u | fail);
+      }
+    }
+  } else {
+    // ======================= softmax: warps 0-3 query tile 0, warps 4-7 query tile 1 =======================
+    const int t = warp >> 2, row = threadIdx.x & 127;
+    const int qi = m0 + t * TQ + row;
+    const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem_base + lane_addr + uint32_t(t * TK);
+    const uint32_t tO = tmem_base + lane_addr + 2 * TK + uint32_t(t * D);
+    const int n = n_kv[t];
+    float m_used = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    uint32_t fail = 0;
+    // (Making the two softmax groups take turns through a pair of named barriers, so that they never share the
+    // schedulers, was measured and is slower: 918 -> 876 TFLOP/s on 2 x 4096 x 32 x 128. A pass is bound by what one
+    // warp can issue alone, so two groups running together get more out of a scheduler than one at a time.)
+    for (int j = 0; j < n; ++j) {
+      if (!mbar_wait_warp(s_full + 8u * t, uint32_t(j) & 1u)) { ok = false; fail |= 0x40u; break; }
+      const int kv0 = j * TK;
+      tc_fence_after();
+      // Two passes over the row of S, 32 columns at a time, so that a thread holds 64 scores at most (with all 128 in
+      // registers the kernel spills at the 168 registers ten warps leave a thread). Pass 1: the row maximum.
+      const int kv_lim = (p.causal ? min(p.S, qi + 1) : p.S) - kv0;   // local columns >= kv_lim are masked
+      // one answer per warp: both branches of pass 2 issue warp-collective tensor-memory stores (on the diagonal
+      // tile the last row of a warp sees every column while the other rows do not)
+      const bool full = __all_sync(0xffffffffu, kv_lim >= TK);
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      {
+        uint32_t q[2][32];
+        tmem_ld32(tS, q[0]);
+#pragma unroll
+        for (int c = 0; c < TK / 32; ++c) {
+          tmem_ld_wait();
+          if (c + 1 < TK / 32) tmem_ld32(tS + (c + 1) * 32, q[(c + 1) & 1]);
+          if (full) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8)
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+                mx4[u] = max3(mx4[u], __uint_as_float(q[c & 1][i + 2 * u]), __uint_as_float(q[c & 1][i + 2 * u + 1]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i < kv_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(q[c & 1][i]));
+          }
+        }
+      }
+      // whole-number reference point (base-2 domain): P's bf16 rounding is then that of 2^t itself and the rescale
+      // factors are exact powers of two
+      const float m_tile = ceilf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2);
+      if (j == 0) {
+        m_used = m_tile;
+      } else {
+        const bool need = m_tile > m_used + 8.f;
+        if (__any_sync(0xffffffffu, need)) {
+          // P_{j-1}.V_{j-1} must have landed in O before it is rescaled
+          if (!mbar_wait_warp(o_done + 8u * t, uint32_t(j - 1) & 1u)) { ok = false; fail |= 0x80u; break; }
+          tc_fence_after();
+          const float m_new = need ? m_tile : m_used;
+          const float alpha = exp2f(m_used - m_new);
+#pragma unroll 1
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t q[32];
+            tmem_ld32(tO + c0, q);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) q[i] = __float_as_uint(__uint_as_float(q[i]) * alpha);
+            tmem_st32(tO + c0, q);
+          }
+          l_run *= alpha;
+          m_used = m_new;
+        }
+      }
+      // ---- P = exp2(s * k - m_used) as bf16 pairs, written over S's first 64 columns ----
+      // Pass 2: P = exp2(s * k - m_used) as bf16 pairs over S's first 64 columns. Chunk c (columns 32c..32c+31) is
+      // read before P chunk c (packed columns 16c..16c+15) is written, and the chunk read ahead lies above both.
+      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+      const float neg_m = -m_used;
+      {
+        const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(neg_m, neg_m);
+        uint64_t acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+        uint32_t q[2][32];
+        tmem_ld32(tS, q[0]);
+#pragma unroll
+        for (int c = 0; c < TK / 32; ++c) {
+          tmem_ld_wait();
+          if (c + 1 < TK / 32) tmem_ld32(tS + (c + 1) * 32, q[(c + 1) & 1]);
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(q[c & 1][2 * i]), __uint_as_float(q[c & 1][2 * i + 1])), sc2, nm2), x0, x1);
+            float a, bb;
+            if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) { a = ex2_poly(x0); bb = ex2_poly(x1); }
+            else { a = ex2_fast(x0); bb = ex2_fast(x1); }
+            if (!full) {
+              if (c * 32 + 2 * i >= kv_lim) a = 0.f;
+              if (c * 32 + 2 * i + 1 >= kv_lim) bb = 0.f;
+            }
+            w[i] = pack_bf16x2(a, bb);
+            acc[i & 1] = add2(acc[i & 1], pack2(a, bb));   // fp32 sum of the unrounded exponentials
+          }
+          tmem_st16(tS + c * 16, w);
+        }
+        unpack2(acc[0], ps4[0], ps4[1]);
+        unpack2(acc[1], ps4[2], ps4[3]);
+      }
+      l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      tc_fence_before();
+      mbar_arrive(p_full + 8u * t);
+    }
+    // ---- O / l -> bf16 ----
+    if (ok && n > 0) {
+      if (!mbar_wait_warp(o_done + 8u * t, uint32_t(n - 1) & 1u)) { ok = false; fail |= 0x80u; }
+      tc_fence_after();
+    }
+    if (fail && lane == 0) atomicOr(p.status, 0x100u | fail);
+    if (!ok) *abort_flag = 1;
+    if (ok && n > 0) {
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.O) + (int64_t)b * p.o_s[0] + (int64_t)h * p.o_s[1] + (int64_t)qi * p.o_s[2];
+      pdl_wait();  // O may still be read by an earlier step
+#pragma unroll 1
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t q[32];
+        tmem_ld32(tO + c0, q);     // warp-collective: rows past the end take part, then skip the store
+        tmem_ld_wait();
+        if (qi < p.S) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(q[g * 8 + i]) * inv;
+            store16(out + c0 + g * 8, v);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 }  // namespace
+
+// Which form runs: two query tiles per CTA (probabilities in tensor memory) when the sequence has more than one query
+// tile, else the one-tile form. FLUID_ATTN_FORM=1 / 2 in the environment forces one of them (A/B timing).
+static int attn_form(const AttnParams& p) {
+  static const int forced = [] {
+    const char* e = std::getenv("FLUID_ATTN_FORM");
+    return e ? std::atoi(e) : 0;
+  }();
+  if (forced == 1 || forced == 2) return forced;
+  return p.S > TQ ? 2 : 1;
+}
+
+template <typename K>
+static cudaError_t launch_attn_form(K kernel, bool* attr_done, size_t smem, dim3 grid, cudaStream_t stream, const CUtensorMap* mq,
+                                    const CUtensorMap* mk, const CUtensorMap* mv, const AttnParams& p) {
+  if (!*attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    *attr_done = true;
+  }
+  return launch_k(kernel, grid, kAttnThreads, smem, stream, *mq, *mk, *mv, p);
+}
 
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream) {
   const int D = p.D;
-  const size_t smem = size_t(5) * TQ * D * 2 + size_t(2) * TQ * TK * 2 + 128 + 2048;
-  const dim3 grid(((p.S + TQ - 1) / TQ) * p.B * p.NH);
   const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(&host.map_q);
   const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(&host.map_k);
   const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(&host.map_v);
-  static bool attr64 = false, attr128 = false;
-  if (D == 64) {
-    if (!attr64) {
-      cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-      attr64 = true;
-    }
-    return launch_k(attn_tc_kernel<64>, grid, kAttnThreads, smem, stream, *mq, *mk, *mv, p);
+  static bool attr[4] = {false, false, false, false};
+  if (D != 64 && D != 128) return cudaErrorInvalidValue;
+  if (attn_form(p) == 2) {
+    const size_t smem = size_t(6) * TQ * D * 2 + 256 + 1024;
+    const dim3 grid(((p.S + 2 * TQ - 1) / (2 * TQ)) * p.B * p.NH);
+    return D == 64 ? launch_attn_form(attn_tc2_kernel<64>, &attr[2], smem, grid, stream, mq, mk, mv, p)
+                   : launch_attn_form(attn_tc2_kernel<128>, &attr[3], smem, grid, stream, mq, mk, mv, p);
   }
-  if (D == 128) {
-    if (!attr128) {
-      cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-      attr128 = true;
-    }
-    return launch_k(attn_tc_kernel<128>, grid, kAttnThreads, smem, stream, *mq, *mk, *mv, p);
-  }
-  return cudaErrorInvalidValue;
+  const size_t smem = size_t(5) * TQ * D * 2 + size_t(2) * TQ * TK * 2 + 128 + 2048;
+  const dim3 grid(((p.S + TQ - 1) / TQ) * p.B * p.NH);
+  return D == 64 ? launch_attn_form(attn_tc_kernel<64>, &attr[0], smem, grid, stream, mq, mk, mv, p)
+                 : launch_attn_form(attn_tc_kernel<128>, &attr[1], smem, grid, stream, mq, mk, mv, p);
 }
 
 }  // namespace fluid
