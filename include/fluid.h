@@ -121,6 +121,8 @@ typedef struct fluid_layout_candidates {
  * with FLUID_EUNSUPPORTED. */
 typedef double (*fluid_eval_fn)(void* user, int32_t node_id, int32_t n_tensors,
                                 const int32_t* tensor_ids, const int32_t* layout_index);
+typedef double (*fluid_eval_variant_fn)(void* user, int32_t node_id, int32_t n_tensors,
+                                        const int32_t* tensor_ids, const int32_t* layout_index, int32_t variant);
 
 typedef struct fluid_plan_options {
   int32_t fusion;           /* 1: fold bias/GELU/residual into GEMM epilogues, residual into norms,
@@ -146,6 +148,20 @@ typedef struct fluid_plan_options {
                                -1: never split */
   fluid_eval_fn eval;       /* NULL: built-in analytic B200 cost table */
   void* eval_user;
+  /* Implementation variants (the paper's "Loop Reordering": the time T of a matrix-multiply-like node that the
+   * dynamic programme sees is the best over its implementation variants, and that variant is the one that runs).
+   * A tensor-core GEMM node has the variants listed by fluid_gemm_variants for its shape and layouts
+   * (code = form | tile_n << 4; form 1: one CTA per 128 x tile_n tile, 2: a CTA pair per 256 x 256 tile,
+   * 3: a thread-block cluster per tile that splits k). With the built-in table every variant is rated by an analytic
+   * model (waves of tiles, cycles per tensor-core instruction of that width, epilogue, bytes) and the cheapest is
+   * kept. eval_variant, when set, replaces eval: it is called once per variant of a node (variant 0 for nodes that
+   * have none), the minimum becomes the node's cost and the arg-min is recorded for the step. */
+  fluid_eval_variant_fn eval_variant;
+  /* Per graph op (the LINEAR / BMM op a GEMM step is built on): a variant code to run that step with instead of the
+   * rated best; 0 or an entry beyond n_op_variant leaves the choice to the planner; a code the step's shape cannot
+   * take is ignored. Copied by fluid_plan. */
+  const int32_t* op_variant;
+  int32_t n_op_variant;
 } fluid_plan_options;
 
 typedef enum {
@@ -156,7 +172,8 @@ typedef enum {
 
 typedef struct fluid_step_info {
   int32_t kernel;        /* fluid_kernel_id */
-  int32_t variant;       /* kernel-specific (GEMM: bit0 A MN-major, bit1 B MN-major, bits 8-19 tile N,
+  int32_t variant;       /* kernel-specific (GEMM: the implementation variant that runs, as chosen by the planner's
+                            rating or the caller's eval_variant / op_variant: bit0 A MN-major, bit1 B MN-major, bits 8-19 tile N,
                             bits 20-23 grouped siblings, bits 24-27 split-K factor, bit 28: the split
                             runs as one thread-block cluster per output tile, bit 29: pairs of CTAs share
                             256 x 256 tiles. GEMM_ROWS: bits 20-23 grouped siblings, bit 29: SiLU(gate) * up is
@@ -192,6 +209,11 @@ FLUID_API int fluid_plan(const fluid_graph_t* g, const fluid_layout_candidates* 
                       const fluid_plan_options* opts, fluid_plan_t** plan);
 FLUID_API void fluid_plan_destroy(fluid_plan_t* plan);
 FLUID_API void fluid_plan_default_options(fluid_plan_options* opts);
+
+/* The implementation variants the GEMM step built on graph op `op_id` can run with under the plan's layouts
+ * (codes as in fluid_plan_options), and the one the plan runs (*chosen). codes may be NULL to query the count.
+ * An op that is not the anchor of a tensor-core GEMM step has no variants (*n = 0, *chosen = 0). */
+FLUID_API int fluid_plan_gemm_variants(const fluid_plan_t* plan, int op_id, int* codes, int capacity, int* n, int* chosen);
 
 /* Peak bytes of the arena, header included; the caller allocates exactly this much. */
 FLUID_API size_t fluid_plan_arena_bytes(const fluid_plan_t* plan);

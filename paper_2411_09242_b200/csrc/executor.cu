@@ -31,7 +31,7 @@ int finalize_steps(fluid_plan_s* p) {
     bool feasible = true;
     for (int ni : s.nodes) {
       if (!std::isfinite(node_cost(p, p->nodes[ni], lo))) {
-        if (!p->opts.eval) {
+        if (!p->opts.eval && !p->opts.eval_variant) {
           set_error("step for op %d: no kernel runs this operator with the chosen layouts", p->nodes[ni].ops[0]);
           return FLUID_EUNSUPPORTED;
         }
@@ -63,7 +63,9 @@ int finalize_steps(fluid_plan_s* p) {
           return FLUID_EUNSUPPORTED;
         }
         const GemmParams& g = s.gemm;
-        s.kernel = gemm_tc_eligible(p, g, &s.tc) ? FLUID_K_GEMM_TC : FLUID_K_GEMM_SIMT;
+        // the variant the planner rated best for this node (or the caller asked for); the fused SwiGLU form exists for CTA pairs only
+        const int gv = s.swiglu ? gemm_variant_code(GV_PAIR, 256) : gemm_variant_of(p, n);
+        s.kernel = gemm_tc_eligible(p, g, &s.tc, gv) ? FLUID_K_GEMM_TC : FLUID_K_GEMM_SIMT;
         if (s.kernel == FLUID_K_GEMM_TC)
           s.variant = (s.tc.cfg.a_mn_major ? 1 : 0) | (s.tc.cfg.b_mn_major ? 2 : 0) | (s.tc.cfg.bn << 8);
         s.t_ptr[0] = n.a; s.t_ptr[1] = n.b; s.t_ptr[2] = n.out; s.t_ptr[3] = n.bias; s.t_ptr[4] = n.res;
@@ -94,7 +96,8 @@ int finalize_steps(fluid_plan_s* p) {
         for (size_t gi = 1; gi < n_gemm; ++gi) {
           const Node& m = p->nodes[s.nodes[gi]];
           GemmParams& gx = s.gemm_x[gi - 1];
-          if (!lower_gemm(p, m, lo, &gx) || !gemm_tc_eligible(p, gx, &s.tc_x[gi - 1]) || s.kernel != FLUID_K_GEMM_TC) {
+          if (!lower_gemm(p, m, lo, &gx) || !gemm_tc_eligible(p, gx, &s.tc_x[gi - 1], gv) || s.kernel != FLUID_K_GEMM_TC ||
+              s.tc_x[gi - 1].cfg.bn != s.tc.cfg.bn || s.tc_x[gi - 1].cfg.pair != s.tc.cfg.pair) {
             set_error("step for op %d: sibling GEMM cannot share a launch", m.ops[0]);
             return FLUID_EUNSUPPORTED;
           }

@@ -128,6 +128,8 @@ struct fluid_plan_s {
   std::vector<int> layout;                      // per tensor: candidate index
   std::vector<int> alias_root;                  // per tensor: root tensor id
   std::vector<int> folded;                      // per tensor: 1 if removed by fusion
+  std::vector<int> op_variant;                  // per graph op: the caller's variant request (copy of opts.op_variant)
+  std::vector<int> node_variant;                // per node: the variant rated best under the final layouts (0: none)
   int not_runnable_op = -1;                     // a caller's cost function chose layouts no kernel runs for this op: the plan is kept for inspection, fluid_run refuses it
   std::vector<fluid::Step> steps;
   std::vector<fluid::ArenaRecord> records;
@@ -155,7 +157,11 @@ double node_cost(const fluid_plan_s* p, const Node& n, const int* layout_of /*pe
 bool transpose_is_alias(const fluid_plan_s* p, const Node& n, const int* layout_of);
 // Lower a GEMM-like node under the given layouts; false if the node cannot be expressed.
 bool lower_gemm(const fluid_plan_s* p, const Node& n, const int* layout_of, GemmParams* gp);
-bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& gp, GemmTcHost* tc);
+bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& gp, GemmTcHost* tc, int variant = 0);
+// Implementation variants of a tensor-core GEMM node (codes of kernels.h), their analytic rating, and the choice.
+std::vector<int> gemm_tc_variants(const fluid_plan_s* p, const GemmParams& g, int n_group);
+double gemm_tc_variant_cost(const GemmParams& g, const GemmTcHost& tc, int n_group);
+int gemm_variant_of(const fluid_plan_s* p, const Node& n);   // requested or rated-best variant of a node, 0 if none
 // Lower a fused attention node; false if the layouts cannot be fed to the attention kernel.
 bool lower_attn(const fluid_plan_s* p, const Node& n, const int* layout_of, AttnParams* ap, AttnHost* host);
 }  // namespace fluid

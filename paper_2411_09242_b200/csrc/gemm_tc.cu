@@ -1667,7 +1667,7 @@ int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t
 // wave of CTAs even after the split), at least two k-steps per CTA, no empty split, vector epilogue.
 int gemm_cluster_split(const GemmParams* gs, const GemmTcHost& tc, int n_group) {
   const GemmParams& g = gs[0];
-  if (g.causal != CAUSAL_NONE || tc.cfg.bn > 128) return 0;
+  if (g.causal != CAUSAL_NONE || tc.cfg.bn > 128 || tc.cfg.no_cluster) return 0;
   if (!vec_epilogue_ok(gs, n_group, false)) return 0;
   const int64_t tiles = int64_t((g.M + BM - 1) / BM) * ((g.N + tc.cfg.bn - 1) / tc.cfg.bn) * g.batch * n_group;
   const int ksteps = (g.K + BK - 1) / BK;

@@ -60,7 +60,19 @@ struct GemmTcCfg {
   int a_rank, b_rank;
   int b_box_rows;       // rows of one TMA box of a K-major B tile (bn, or 128 when a CTA pair shares a 256-wide tile)
   int pair;             // 1: the step qualifies for the CTA-pair kernel (two CTAs, one 256 x 256 tile, tcgen05 cta_group::2)
+  int no_cluster;       // 1: the step was asked to run without the cluster split-K form
+  int want_cluster;     // 1: the step was asked to run as clusters that split k (refused at lowering if the shape does not qualify)
 };
+
+// Implementation variants of a tensor-core GEMM step (the counterpart of the paper's loop orders: same numbers, different
+// time). code = form | tile_n << 4; 0 = chosen by the built-in rules.
+//   form 1: one CTA per 128 x tile_n tile (persistent, tile_n 64 / 128 / 256)
+//   form 2: a pair of CTAs per 256 x 256 tile (tcgen05 cta_group::2; tile_n 256)
+//   form 3: a thread-block cluster per 128 x tile_n tile that splits k (tile_n 64 / 128; few-tile steps only)
+constexpr int GV_AUTO = 0, GV_SINGLE = 1, GV_PAIR = 2, GV_CLUSTER = 3;
+inline int gemm_variant_code(int form, int bn) { return form | (bn << 4); }
+inline int gemm_variant_form(int code) { return code & 15; }
+inline int gemm_variant_bn(int code) { return code >> 4; }
 
 struct alignas(64) TensorMapStorage {
   unsigned char bytes[128];
@@ -231,7 +243,7 @@ int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t
 int gemm_cluster_split(const GemmParams* gs, const GemmTcHost& tc, int n_group);
 // True if the step runs on the CTA-pair kernel (two CTAs of a cluster per 256 x 256 tile).
 bool gemm_pair_eligible(const GemmParams* gs, const GemmTcHost& tc, int n_group);
-bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc);
+bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc, int variant = 0);
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);
 cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t stream);

@@ -207,24 +207,33 @@ static bool build_tma_operand(int64_t R, int R0, const int64_t* rs, int64_t K, i
   return true;
 }
 
-bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& g, GemmTcHost* tc) {
+bool gemm_tc_eligible(const fluid_plan_s* p, const GemmParams& g, GemmTcHost* tc, int variant) {
   GemmTcHost h{};
   h.eligible = 0;
   *tc = h;
   if (p->opts.gemm_path == 1) return false;
-  return gemm_tc_describe(g, tc);
+  if (variant && gemm_tc_describe(g, tc, variant)) return true;   // a variant the shape cannot take falls back to the rules
+  return gemm_tc_describe(g, tc, 0);
 }
 
 // Tile configuration and TMA operand descriptions of a bf16 GEMM for the tensor-core kernel;
 // false if its operands cannot be expressed as tensor maps.
-bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc) {
+bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc, int variant) {
   GemmTcHost h{};
   h.eligible = 0;
   *tc = h;
   if (!tc_kernel_available() || g.dtype != FLUID_BF16) return false;
   if (g.K < 8) return false;
+  const int form = gemm_variant_form(variant), want_bn = gemm_variant_bn(variant);
+  if (variant) {
+    if (want_bn != 64 && want_bn != 128 && want_bn != 256) return false;
+    if (form == GV_PAIR && (want_bn != 256 || g.causal != CAUSAL_NONE || g.M % 256 != 0)) return false;
+    if (form == GV_CLUSTER && (want_bn > 128 || g.causal != CAUSAL_NONE)) return false;
+    if (form < GV_SINGLE || form > GV_CLUSTER) return false;
+  }
   int bn = 128;
-  if (g.N <= 64) bn = 64;
+  if (variant) bn = want_bn;
+  else if (g.N <= 64) bn = 64;
   else {
     const int64_t tiles256 = int64_t((g.M + 127) / 128) * ((g.N + 255) / 256) * g.batch;
     const int64_t tiles64 = int64_t((g.M + 127) / 128) * ((g.N + 63) / 64) * g.batch;
@@ -242,13 +251,16 @@ bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc) {
   // of the B tile: its TMA box is then 128 rows, which the single-CTA kernel fetches as two boxes).
   int b_box = bn;
   while (true) {
-    b_box = (bn == 256 && g.causal == CAUSAL_NONE && g.M % 256 == 0) ? 128 : bn;
+    b_box = (bn == 256 && g.causal == CAUSAL_NONE && g.M % 256 == 0 && form != GV_SINGLE) ? 128 : bn;
     if (build_tma_operand(g.N, g.N0, b_rs, g.K, g.K0, b_ks, g.batch, g.B0, b_bs, b_box, &h.b)) break;
-    if (bn == 64) return false;
+    if (bn == 64 || variant) return false;   // a requested tile width is not traded for a narrower one
     bn /= 2;
   }
   h.cfg.b_box_rows = b_box;
   h.cfg.pair = (bn == 256 && b_box == 128) ? 1 : 0;
+  if (form == GV_PAIR && !h.cfg.pair) return false;
+  h.cfg.no_cluster = (form == GV_SINGLE || form == GV_PAIR) ? 1 : 0;
+  h.cfg.want_cluster = form == GV_CLUSTER ? 1 : 0;
   // output / residual vector accesses assume 8-element alignment of every outer stride when the
   // n index is contiguous; otherwise the epilogue falls back to scalar stores (always legal)
   h.cfg.bn = bn;
@@ -266,6 +278,73 @@ bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc) {
   h.eligible = 1;
   *tc = h;
   return true;
+}
+
+// ---- implementation variants of a tensor-core GEMM step (the paper's "Loop Reordering") ----------------------
+// Every (form, tile width) the shape can run with; the order is the tie-break of the rating.
+std::vector<int> gemm_tc_variants(const fluid_plan_s* p, const GemmParams& g, int n_group) {
+  std::vector<int> out;
+  if (p->opts.gemm_path == 1) return out;
+  GemmParams gs[3] = {g, g, g};
+  for (int form : {GV_PAIR, GV_SINGLE, GV_CLUSTER})
+    for (int bn : {256, 128, 64}) {
+      GemmTcHost tc;
+      const int code = gemm_variant_code(form, bn);
+      if (bn > 64 && g.N <= bn / 2) continue;            // a tile more than twice as wide as the matrix
+      if (!gemm_tc_describe(g, &tc, code)) continue;
+      if (form == GV_PAIR && !gemm_pair_eligible(gs, tc, n_group)) continue;
+      if (form == GV_CLUSTER && (p->opts.split_k < 0 || gemm_cluster_split(gs, tc, n_group) < 2)) continue;
+      out.push_back(code);
+    }
+  return out;
+}
+
+// Analytic rating of one variant, seconds. Measured on B200 and used as constants here: a 128 x N x 16 tensor-core
+// instruction issued from shared-memory operands takes about 97 / 107 / 171 cycles for N = 64 / 128 / 256 (the A
+// tile's 4 KB are fetched per instruction: ~43 cycles on top of N / 2), a 256 x 256 x 16 instruction of a CTA pair 128
+// per CTA; the distributed-shared-memory exchange of a cluster moves ~21 bytes per clock into an SM; an SM stores
+// ~32 bytes per clock. Tiles run in waves over the SMs (or SM pairs); the epilogue of a tile overlaps the next
+// tile's main loop (two accumulators), so a wave costs the longer of the two and the last epilogue is exposed.
+double gemm_tc_variant_cost(const GemmParams& g, const GemmTcHost& tc, int n_group) {
+  const double clk = 1.8e9;
+  const int sms = 148, bn = tc.cfg.bn;
+  const int form = tc.cfg.want_cluster ? GV_CLUSTER : (tc.cfg.pair && tc.cfg.no_cluster ? GV_PAIR : GV_SINGLE);
+  const double ksteps = std::ceil(g.K / 64.0);
+  const double tiles_m = std::ceil(g.M / 128.0), tiles_n = std::ceil(double(g.N) / bn);
+  double tiles = tiles_m * tiles_n * g.batch * n_group;
+  if (g.causal != CAUSAL_NONE) tiles *= 0.5 * (1.0 + 1.0 / std::max(1.0, tiles_m));
+  const double out_bytes = (g.c_f32 ? 4.0 : 2.0) + (g.has_res ? (g.r_f32 ? 4.0 : 2.0) : 0.0);
+  const double act = g.act != ACT_NONE ? 1.6 : 1.0;     // an activation in the epilogue costs issue slots
+  const double fill = 1800.0;                           // first loads of a CTA: tensor-map fetch, pipeline ramp
+  double cycles;
+  if (form == GV_PAIR) {
+    const double units = sms / 2, pair_tiles = std::ceil(tiles_m / 2.0) * tiles_n * g.batch * n_group;
+    const double main = ksteps * 4.0 * 128.0, epi = (128.0 * 256.0 * out_bytes / 32.0 + 128.0 * 256.0 / 256.0 * 10.0) * act;
+    cycles = fill + std::ceil(pair_tiles / units) * std::max(main, epi) + epi;
+  } else if (form == GV_SINGLE) {
+    const double per = bn == 256 ? 171.0 : (bn == 128 ? 107.0 : 97.0);
+    const double main = ksteps * 4.0 * per, epi = (128.0 * bn * out_bytes / 32.0 + 128.0 * bn / 256.0 * 10.0) * act;
+    cycles = fill + std::ceil(tiles / sms) * std::max(main, epi) + epi;
+  } else {
+    GemmParams gs[3] = {g, g, g};
+    const int sk = std::max(2, gemm_cluster_split(gs, tc, n_group));
+    const double per = bn == 128 ? 107.0 : 97.0;
+    const double main = std::ceil(ksteps / sk) * 4.0 * per, exchange = 128.0 * bn * 4.0 * (sk - 1) / sk / 21.0;
+    const double epi = (128.0 * bn * out_bytes / 32.0 + 128.0 * bn / 256.0 * 10.0) * act / sk;
+    cycles = fill + main + exchange + epi + 600.0;     // two cluster barriers
+  }
+  return cycles / clk;
+}
+
+// The variant a GEMM node runs with: the caller's request for its anchor op if there is one, else the rated best
+// recorded when the layouts were final, else 0 (the shape rules).
+int gemm_variant_of(const fluid_plan_s* p, const Node& n) {
+  if (n.kind != N_GEMM || n.ops.empty()) return 0;
+  const int op = n.ops[0];
+  if (op >= 0 && op < (int)p->op_variant.size() && p->op_variant[op]) return p->op_variant[op];
+  const int ni = op < (int)p->node_of_op.size() ? p->node_of_op[op] : -1;
+  if (ni >= 0 && ni < (int)p->node_variant.size()) return p->node_variant[ni];
+  return 0;
 }
 
 bool lower_attn(const fluid_plan_s* p, const Node& n, const int* lo, AttnParams* ap, AttnHost* host) {
@@ -342,7 +421,16 @@ double node_cost(const fluid_plan_s* p, const Node& n, const int* lo) {
         const double skew = 1.0 + 0.02 * (tc.cfg.a_mn_major + tc.cfg.b_mn_major);
         // the vector epilogue wants the n index contiguous in C; anything else stores element-wise
         const double c_pen = g.c_s[5] == 1 ? 1.0 : (g.c_s[3] == 1 ? 1.3 : 1.6);
-        return kLaunch + std::max(fl / kTcPeak, by / kBw) * skew * c_pen;
+        // T of the node = the best over its implementation variants (tile width, CTA pair, cluster split-K)
+        double best = kInf;
+        // (a caller's op_variant request does not enter the rating: it swaps the variant of a step, not the plan)
+        for (int code : gemm_tc_variants(p, g, 1)) {
+          GemmTcHost tv;
+          if (!gemm_tc_describe(g, &tv, code)) continue;
+          best = std::min(best, gemm_tc_variant_cost(g, tv, 1));
+        }
+        if (best == kInf) best = fl / kTcPeak;
+        return kLaunch + std::max(std::max(best, fl / (1.25 * kTcPeak)), by / kBw) * skew * c_pen;
       }
       const bool a_fast = g.a_s[5] == 1 || g.a_s[3] == 1, b_fast = g.b_s[5] == 1 || g.b_s[3] == 1,
                  c_fast = g.c_s[5] == 1 || g.c_s[3] == 1;
@@ -408,11 +496,47 @@ struct Evaluator {
   std::vector<int> lo;  // scratch: layout index per tensor
   double operator()(int node, const std::vector<int>& tids, const std::vector<int>& lidx) {
     const Node& n = p->nodes[node];
+    if (p->opts.eval_variant) return best_variant(node, tids, lidx, nullptr);
     if (p->opts.eval) {
       return p->opts.eval(p->opts.eval_user, n.ops[0], (int)tids.size(), tids.data(), lidx.data());
     }
     for (size_t i = 0; i < tids.size(); ++i) lo[tids[i]] = lidx[i];
     return node_cost(p, n, lo.data());
+  }
+  // The caller's eval_variant over every variant of the node under these layouts: the minimum, and its arg-min.
+  double best_variant(int node, const std::vector<int>& tids, const std::vector<int>& lidx, int* chosen) {
+    const Node& n = p->nodes[node];
+    for (size_t i = 0; i < tids.size(); ++i) lo[tids[i]] = lidx[i];
+    std::vector<int> codes;
+    GemmParams g;
+    GemmTcHost tc;
+    if (n.kind == N_GEMM && lower_gemm(p, n, lo.data(), &g) && gemm_tc_eligible(p, g, &tc)) codes = gemm_tc_variants(p, g, 1);
+    if (codes.empty()) codes.push_back(0);
+    double best = kInf;
+    int arg = codes[0];
+    for (int code : codes) {
+      const double c = p->opts.eval_variant(p->opts.eval_user, n.ops[0], (int)tids.size(), tids.data(), lidx.data(), code);
+      if (c < best) { best = c; arg = code; }
+    }
+    if (chosen) *chosen = arg;
+    return best;
+  }
+  // Built-in table: the arg-min variant of a GEMM node under these layouts (0 if the node has none).
+  int rated_variant(int node, const std::vector<int>& tids, const std::vector<int>& lidx) {
+    const Node& n = p->nodes[node];
+    for (size_t i = 0; i < tids.size(); ++i) lo[tids[i]] = lidx[i];
+    GemmParams g;
+    GemmTcHost tc;
+    if (n.kind != N_GEMM || !lower_gemm(p, n, lo.data(), &g) || !gemm_tc_eligible(p, g, &tc)) return 0;
+    double best = kInf;
+    int arg = 0;
+    for (int code : gemm_tc_variants(p, g, 1)) {
+      GemmTcHost tv;
+      if (!gemm_tc_describe(g, &tv, code)) continue;
+      const double c = gemm_tc_variant_cost(g, tv, 1);
+      if (c < best) { best = c; arg = code; }
+    }
+    return arg;
   }
 };
 
@@ -917,6 +1041,17 @@ static int plan_layouts(fluid_plan_s* p) {
     p->layout = assign;
     p->cost = c;
   }
+  // the implementation variant each GEMM node was rated with under the final layouts is the one its step runs
+  p->node_variant.assign(p->nodes.size(), 0);
+  for (size_t i = 0; i < p->nodes.size(); ++i) {
+    if (p->nodes[i].kind != N_GEMM) continue;
+    std::vector<int> tids = node_tensors(p->nodes[i]), l;
+    for (int t : tids) l.push_back(p->layout[t]);
+    int code = 0;
+    if (p->opts.eval_variant) ev.best_variant((int)i, tids, l, &code);
+    else if (!p->opts.eval) code = ev.rated_variant((int)i, tids, l);
+    p->node_variant[i] = code;
+  }
   return FLUID_OK;
 }
 
@@ -1295,7 +1430,10 @@ int fluid_plan(const fluid_graph_t* g, const fluid_layout_candidates* cands, con
   p->graph = *g;
   if (opts) p->opts = *opts;
   else fluid_plan_default_options(&p->opts);
-  if (p->opts.eval) p->opts.fusion = 0;
+  if (p->opts.eval || p->opts.eval_variant) p->opts.fusion = 0;
+  if (p->opts.op_variant && p->opts.n_op_variant > 0) p->op_variant.assign(p->opts.op_variant, p->opts.op_variant + p->opts.n_op_variant);
+  p->opts.op_variant = nullptr;   // the caller's array is not kept
+  p->opts.n_op_variant = 0;
   const int nt = (int)g->tensors.size();
   // layout candidates
   p->cands.assign(nt, {});
@@ -1411,6 +1549,31 @@ int fluid_plan_record_info(const fluid_plan_t* p, int index, int* record_id, int
 }
 
 int fluid_plan_num_steps(const fluid_plan_t* p) { return p ? (int)p->steps.size() : 0; }
+
+int fluid_plan_gemm_variants(const fluid_plan_t* p, int op_id, int* codes, int capacity, int* n_out, int* chosen) {
+  if (!p || !n_out || op_id < 0 || op_id >= (int)p->node_of_op.size()) {
+    set_error("gemm variants: bad plan or op id");
+    return FLUID_EINVAL;
+  }
+  *n_out = 0;
+  if (chosen) *chosen = 0;
+  const int ni = p->node_of_op[op_id];
+  if (ni < 0 || p->nodes[ni].kind != N_GEMM || p->nodes[ni].ops[0] != op_id) return FLUID_OK;
+  // the step this node anchors (a grouped sibling launch is listed under its first node)
+  for (const Step& s : p->steps) {
+    if (s.kernel != FLUID_K_GEMM_TC || s.nodes.empty() || s.nodes[0] != ni) continue;
+    const int n_group = s.swiglu ? 2 : std::max<int>(1, (s.variant >> 20) & 15);
+    const std::vector<int> v = gemm_tc_variants(p, s.gemm, n_group);
+    *n_out = (int)v.size();
+    for (int i = 0; i < (int)v.size() && codes && i < capacity; ++i) codes[i] = v[i];
+    if (chosen) {
+      const int form = ((s.variant >> 28) & 1) ? GV_CLUSTER : (((s.variant >> 29) & 1) ? GV_PAIR : GV_SINGLE);
+      *chosen = gemm_variant_code(form, (s.variant >> 8) & 0xfff);
+    }
+    return FLUID_OK;
+  }
+  return FLUID_OK;
+}
 
 int fluid_plan_step_info(const fluid_plan_t* p, int step, fluid_step_info* info) {
   if (!p || !info || step < 0 || step >= (int)p->steps.size()) {

@@ -44,13 +44,20 @@ class LayoutCandidates(C.Structure):
 
 
 EVAL_FN = C.CFUNCTYPE(C.c_double, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32))
+EVAL_VARIANT_FN = C.CFUNCTYPE(C.c_double, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_int32)
+GV_SINGLE, GV_PAIR, GV_CLUSTER = 1, 2, 3
+
+
+def gemm_variant_code(form, tile_n):
+    return form | (tile_n << 4)
 
 
 class PlanOptions(C.Structure):
     _fields_ = [("fusion", C.c_int32), ("arena_policy", C.c_int32), ("no_reuse", C.c_int32),
                 ("force_canonical", C.c_int32), ("gemm_path", C.c_int32), ("narrow_stream", C.c_int32),
                 ("unfused_attention", C.c_int32), ("split_k", C.c_int32),
-                ("eval", EVAL_FN), ("eval_user", C.c_void_p)]
+                ("eval", EVAL_FN), ("eval_user", C.c_void_p), ("eval_variant", EVAL_VARIANT_FN),
+                ("op_variant", C.POINTER(C.c_int32)), ("n_op_variant", C.c_int32)]
 
 
 class StepInfo(C.Structure):
@@ -80,6 +87,7 @@ _SIGNATURES = {
     "fluid_plan_num_records": (C.c_int, [C.c_void_p]),
     "fluid_plan_record_info": (C.c_int, [C.c_void_p, C.c_int] + [C.POINTER(C.c_int)] * 4 + [C.POINTER(C.c_int64)] * 2 +
                                [C.POINTER(C.c_int)] * 2),
+    "fluid_plan_gemm_variants": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "fluid_plan_num_steps": (C.c_int, [C.c_void_p]),
     "fluid_plan_step_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(StepInfo)]),
     "fluid_plan_num_sequences": (C.c_int, [C.c_void_p]),
@@ -254,6 +262,15 @@ def fluid_plan_step_info(p, step) -> dict:
             "cost": s.cost, "flops": s.flops, "bytes": s.bytes}
 
 
+def fluid_plan_gemm_variants(p, op_id):
+    """(variant codes the GEMM step anchored at graph op `op_id` can run with, the one the plan runs)."""
+    n, chosen = C.c_int(), C.c_int()
+    _check(lib().fluid_plan_gemm_variants(p, op_id, None, 0, C.byref(n), C.byref(chosen)))
+    buf = (C.c_int * max(1, n.value))()
+    _check(lib().fluid_plan_gemm_variants(p, op_id, buf, n.value, C.byref(n), C.byref(chosen)))
+    return list(buf[: n.value]), chosen.value
+
+
 def fluid_plan_num_sequences(p):
     return lib().fluid_plan_num_sequences(p)
 
@@ -329,12 +346,24 @@ def graph_from_desc(desc: synth.GraphDesc):
 
 
 def make_options(**kw) -> PlanOptions:
+    """Plan options from keywords. op_variant: {graph op id: variant code} (marshalled to the C array)."""
     o = fluid_plan_default_options()
     ev = kw.pop("eval", None)
+    evv = kw.pop("eval_variant", None)
+    opv = kw.pop("op_variant", None)
     for k, v in kw.items():
         setattr(o, k, v)
     if ev is not None:
         o.eval = ev
+    if evv is not None:
+        o.eval_variant = evv
+    if opv:
+        n = max(opv) + 1
+        arr = (C.c_int32 * n)()
+        for k, v in opv.items():
+            arr[k] = v
+        o.op_variant, o.n_op_variant = arr, n
+        o._keep = arr        # alive until fluid_plan has copied it
     return o
 
 
@@ -343,7 +372,7 @@ class Plan:
 
     def __init__(self, desc: synth.GraphDesc, candidates=None, **options):
         self.desc = desc
-        self._eval_keepalive = options.get("eval")
+        self._eval_keepalive = (options.get("eval"), options.get("eval_variant"))
         self.graph = graph_from_desc(desc)
         try:
             self.handle = fluid_plan(self.graph, candidates, make_options(**options))
@@ -397,6 +426,9 @@ class Plan:
 
     def sequences(self):
         return [fluid_plan_sequence(self.handle, i) for i in range(fluid_plan_num_sequences(self.handle))]
+
+    def gemm_variants(self, op_id):
+        return fluid_plan_gemm_variants(self.handle, op_id)
 
 
 _TORCH_DTYPE = None

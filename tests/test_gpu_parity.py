@@ -433,3 +433,70 @@ def test_norm_over_many_rows_reading_the_fp32_stream():
     assert plan.tensor_info(x).bytes >= 10 * 2048 * 768 * 4     # held in fp32
     assert_close(got[y], run_oracle(g, feeds)[y], synth.BF16, "embed -> layernorm")
     plan.close()
+
+
+# ---- implementation variants of the tensor-core GEMM (the paper's "Loop Reordering": speed changes, numbers do not) ----
+@pytest.mark.parametrize("M,N,K", [(512, 768, 1024), (128, 2304, 768), (1024, 512, 256)])
+def test_every_gemm_variant_gives_the_same_numbers(M, N, K):
+    g = single_op_graph(synth.LINEAR, [[M, K], [K, N], [N]], [M, N], synth.BF16, {"contract": 1},
+                        in_kinds={1: synth.CONST, 2: synth.CONST})
+    feeds = {0: rand_feed([M, K], synth.BF16, 3), 1: rand_feed([K, N], synth.BF16, 4), 2: rand_feed([N], synth.BF16, 5)}
+    ref = run_oracle(g, feeds)[g.outputs[0]]
+    base = fluid.Plan(g, synth.default_candidates(g))
+    codes, chosen = base.gemm_variants(0)
+    base.close()
+    assert len(codes) >= 3 and chosen in codes
+    outs = {}
+    for code in codes:
+        got, plan, _ = run_gpu(g, feeds, synth.default_candidates(g), op_variant={0: code})
+        assert plan.gemm_variants(0)[1] == code
+        assert_close(got[g.outputs[0]], ref, synth.BF16, f"variant {code & 15}/{code >> 4}", tol=2 ** -7)
+        outs[code] = got[g.outputs[0]]
+        plan.close()
+    # forms that do not split k add up in the same order: bit-identical
+    whole = [outs[c] for c in codes if (c & 15) != fluid.GV_CLUSTER]
+    assert all(np.array_equal(whole[0], w) for w in whole[1:])
+
+
+def test_plan_from_measured_variant_costs():
+    """eval_variant answered by measurement: every (operator, layouts, variant) the dynamic programme asks about is
+    timed on the GPU; the node cost it sees is the fastest variant's time and that variant runs."""
+    from paper_2411_09242_b200.measure import MeasuredEval
+    cfg = synth.scaled(SMALL["gpt"], dtype=synth.BF16, L=1, H=256, F=512, S=256)
+    m = synth.build_model(cfg)
+    cands = synth.default_candidates(m.graph)
+    ev = MeasuredEval(m.graph, cands, reps=3, warmup=1, variants=True)
+    plan = fluid.Plan(m.graph, cands, eval_variant=ev.callback_variant)
+    rated = {k[2] for k in ev.table}
+    assert len(rated - {0}) >= 2 and 0 < plan.cost <= plan.canonical_cost < 1.0
+    for s in plan.steps():
+        if s["kernel_name"] == "GEMM_TC":
+            codes, chosen = plan.gemm_variants(s["ops"][0])
+            assert chosen in codes
+    ref = run_oracle(m.graph, model_feeds(m))
+    runner = fluid.Runner(plan, m.consts)
+    runner.set_inputs([m.ids])
+    runner.run()
+    assert runner.status() == 0
+    for tid, got in zip(m.graph.outputs, runner.outputs_host()):
+        assert_close(got, ref[tid], synth.BF16, f"measured-variant plan output {tid}")
+    plan.close()
+
+
+def test_step_variants_tuned_in_place():
+    """The fused steps a model really runs, each timed inside the whole plan with every variant its shape admits; the
+    fastest per step goes back into the plan. Results stay those of the oracle."""
+    from paper_2411_09242_b200.measure import tune_step_variants
+    cfg = synth.scaled(SMALL["gpt"], dtype=synth.BF16, L=2, H=256, F=1024, S=512, B=2)
+    m = synth.build_model(cfg)
+    cands = synth.default_candidates(m.graph)
+    op_variant, table = tune_step_variants(m.graph, cands, m.consts, [m.ids], reps=3, warmup=1)
+    assert op_variant and all(len(t) >= 2 and min(t, key=t.get) == op_variant[op] for op, t in table.items())
+    got, plan, _ = run_gpu(m.graph, model_feeds(m), cands, op_variant=op_variant)
+    for s in plan.steps():
+        if s["kernel_name"] == "GEMM_TC" and s["ops"][0] in op_variant:
+            assert plan.gemm_variants(s["ops"][0])[1] == op_variant[s["ops"][0]]
+    ref = run_oracle(m.graph, model_feeds(m))
+    for tid in m.graph.outputs:
+        assert_close(got[tid], ref[tid], synth.BF16, f"tuned-variant plan output {tid}")
+    plan.close()

@@ -391,3 +391,97 @@ def test_state_tensors_and_cached_attention_are_checked():
     g.op(synth.CACHED_ATTENTION, ins, [out], scale=0.125)
     with pytest.raises(fluid.FluidError):
         fluid.Plan(g, None)
+
+
+# ---- implementation variants: the dynamic programme sees the best variant's cost, the step runs it --------------
+def _mlp_graph(M=256, H=512, F=1024):
+    """x -> LINEAR(+bias) -> GELU -> LINEAR(+bias): two tensor-core GEMM nodes on one chain (bf16)."""
+    g = synth.GraphDesc()
+    x = g.tensor("x", synth.BF16, [M, H], synth.INPUT)
+    w1 = g.tensor("w1", synth.BF16, [H, F], synth.CONST)
+    w2 = g.tensor("w2", synth.BF16, [F, H], synth.CONST)
+    h = g.tensor("h", synth.BF16, [M, F], synth.ACT)
+    a = g.tensor("a", synth.BF16, [M, F], synth.ACT)
+    y = g.tensor("y", synth.BF16, [M, H], synth.OUTPUT)
+    g.op(synth.LINEAR, [x, w1], [h], contract=1)
+    g.op(synth.GELU, [h], [a])
+    g.op(synth.LINEAR, [a, w2], [y], contract=1)
+    return g
+
+
+def _decode(code):
+    return code & 15, code >> 4
+
+
+def test_every_gemm_step_lists_its_variants_and_runs_the_rated_best():
+    d = _mlp_graph()
+    plan = fluid.Plan(d, synth.default_candidates(d))
+    steps = [s for s in plan.steps() if s["kernel_name"] == "GEMM_TC"]
+    assert len(steps) == 2
+    for s in steps:
+        codes, chosen = plan.gemm_variants(s["ops"][0])
+        assert len(codes) >= 3 and chosen in codes and len(set(codes)) == len(codes)
+        form, bn = _decode(chosen)
+        assert bn == (s["variant"] >> 8) & 0xfff
+        assert form == (3 if (s["variant"] >> 28) & 1 else 2 if (s["variant"] >> 29) & 1 else 1)
+    assert plan.gemm_variants(1) == ([], 0)                # the GELU op anchors no GEMM step
+    plan.close()
+
+
+def test_a_requested_variant_is_the_one_that_runs():
+    d = _mlp_graph()
+    base = fluid.Plan(d, synth.default_candidates(d))
+    codes, chosen = base.gemm_variants(0)
+    base.close()
+    for code in codes:
+        plan = fluid.Plan(d, synth.default_candidates(d), op_variant={0: code})
+        assert plan.gemm_variants(0)[1] == code
+        plan.close()
+    # a code the shape cannot take (a CTA pair over 100 rows) is ignored
+    g = _mlp_graph(M=100)
+    plan = fluid.Plan(g, synth.default_candidates(g), op_variant={0: fluid.gemm_variant_code(fluid.GV_PAIR, 256)})
+    assert _decode(plan.gemm_variants(0)[1])[0] != fluid.GV_PAIR
+    plan.close()
+
+
+@pytest.mark.parametrize("cheap_form", [fluid.GV_SINGLE, fluid.GV_PAIR])
+def test_variant_costs_from_the_caller_decide_layouts_and_variant_with_the_oracle(cheap_form):
+    """eval_variant(node, layouts, variant) = base(node, layouts) + bump(variant). The node cost the dynamic programme
+    must see is the minimum over the node's variants (paper, Sec. "Design", "Loop Reordering"), so the oracle planner,
+    handed eval(node, layouts) = base + min over that node's variant list of bump, must arrive at the same layouts and
+    the same total cost; and the step must run the arg-min variant. Making another form cheap flips the variant."""
+    d = _mlp_graph()
+    cands = synth.default_candidates(d)
+    probe = fluid.Plan(d, cands, fusion=0)
+    variants = {op: probe.gemm_variants(op)[0] for op in range(len(d.ops))}
+    probe.close()
+    assert all(len(variants[op]) >= 3 for op in (0, 2)) and variants[1] == []
+    base = table_eval(3)
+
+    def bump(code):
+        form, bn = _decode(code)
+        return 0.0 if code == 0 else (1.0 if form == cheap_form else 5.0) + {64: 0.75, 128: 0.25, 256: 0.5}[bn]
+
+    asked, offered = set(), {}     # offered: which variants the library listed for (node, layouts): kernel knowledge
+
+    def c_eval(user, node, n, tids, lidx, variant):
+        asked.add((node, variant))
+        lay = {tids[i]: lidx[i] for i in range(n)}
+        offered.setdefault((node, tuple(sorted(lay.items()))), set()).add(variant)
+        return base(node, lay) + bump(variant)
+
+    def o_eval(op, lay):
+        listed = offered.get((op, tuple(sorted(lay.items()))), variants[op])
+        return base(op, lay) + min((bump(v) for v in listed), default=0.0)
+
+    plan = fluid.Plan(d, cands, eval_variant=fluid.EVAL_VARIANT_FN(c_eval))
+    ops, ncand, consts = _oracle_inputs(d, cands)
+    want, cost, seqs = OP.plan_layouts(ops, ncand, o_eval, consts)
+    assert {t: plan.tensor_info(t).layout_index for t in range(len(d.tensors))} == want
+    assert plan.cost == cost and plan.sequences() == seqs
+    for op in (0, 2):
+        assert {v for (n, v) in asked if n == op} >= set(variants[op])      # every variant was rated
+        codes, chosen = plan.gemm_variants(op)
+        assert chosen == min(codes, key=bump) and _decode(chosen)[0] == cheap_form
+    assert {v for (n, v) in asked if n == 1} == {0}                          # a node without variants is asked once
+    plan.close()
