@@ -307,10 +307,19 @@ def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=N
         cfg = synth.scaled(cfg, **overrides)
     m = synth.build_model(cfg)
     cands = synth.default_candidates(m.graph)
+    # the plan that runs places the arena with Algorithm 4 over several record orders (arena_policy 2, the smallest
+    # kept); the sizes the algorithm gives as printed (first fit) and by its prose (best fit) are reported beside it
+    plan_opts = dict({"arena_policy": 2}, **(plan_opts or {}))
     t0 = time.perf_counter()
-    plan = fluid.Plan(m.graph, cands, **(plan_opts or {}))
+    plan = fluid.Plan(m.graph, cands, **plan_opts)
     plan_ms = 1e3 * (time.perf_counter() - t0)
     canon = fluid.Plan(m.graph, None)
+    sizes = {}
+    for label, extra in (("first_fit", {"arena_policy": 0}), ("best_fit", {"arena_policy": 1}),
+                         ("no_inplace", {"arena_policy": 2, "no_inplace": 1})):
+        q = fluid.Plan(m.graph, cands, **dict(plan_opts, **extra))
+        sizes[label] = q.arena_bytes / 2 ** 20
+        q.close()
     runner = fluid.Runner(plan, m.consts)
     runner.set_inputs([m.ids])
     stream = torch.cuda.Stream()
@@ -319,6 +328,9 @@ def time_workload(name, steps, warmup, torch, fluid, peaks, full=True, sampler=N
     n_steps = len(steps_info)
     res = {"workload": name, "arena_mb": plan.arena_bytes / 2 ** 20, "arena_naive_mb": plan.naive_bytes / 2 ** 20,
            "arena_live_bound_mb": plan.live_bound_bytes / 2 ** 20, "arena_canonical_plan_mb": canon.arena_bytes / 2 ** 20,
+           "arena_policy": "Algorithm 4 over several record orders, smallest kept; in-place results share their operand's slice",
+           "arena_first_fit_mb": sizes["first_fit"], "arena_best_fit_mb": sizes["best_fit"],
+           "arena_without_inplace_mb": sizes["no_inplace"],
            "weights_mb": sum(a.size for a in m.consts.values()) * synth.DTYPE_BYTES[cfg.dtype] / 2 ** 20,
            "kernel_steps": n_steps, "plan_ms": plan_ms, "tokens": cfg.B * cfg.S,
            "planned_cost_ms": plan.cost * 1e3, "canonical_cost_ms": plan.canonical_cost * 1e3}
@@ -642,6 +654,8 @@ def main():
         "config": config_of(cfg, world),
         "peak_arena_mb": main_res["arena_mb"], "arena_naive_mb": main_res["arena_naive_mb"],
         "arena_live_bound_mb": main_res["arena_live_bound_mb"], "arena_canonical_plan_mb": main_res["arena_canonical_plan_mb"],
+        "arena_first_fit_mb": main_res["arena_first_fit_mb"], "arena_best_fit_mb": main_res["arena_best_fit_mb"],
+        "arena_without_inplace_mb": main_res["arena_without_inplace_mb"], "arena_policy": main_res["arena_policy"],
         "weights_mb": main_res["weights_mb"],
         "tokens_per_s": world * main_res["tokens"] / (latency_ms * 1e-3),
         "latency_eager_ms": main_res["latency_eager_ms"], "latency_min_ms": main_res["latency_min_ms"],

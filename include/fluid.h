@@ -162,6 +162,9 @@ typedef struct fluid_plan_options {
    * take is ignored. Copied by fluid_plan. */
   const int32_t* op_variant;
   int32_t n_op_variant;
+  int32_t no_inplace;       /* 0 (default): a rotary-embedding, element-wise or residual-epilogue step whose input dies
+                               with it writes its result over that input (one arena record, union lifetime);
+                               1: every result gets a slice of its own */
 } fluid_plan_options;
 
 typedef enum {

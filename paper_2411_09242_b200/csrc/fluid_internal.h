@@ -127,6 +127,7 @@ struct fluid_plan_s {
   std::vector<std::vector<int>> sequences;      // node ids
   std::vector<int> layout;                      // per tensor: candidate index
   std::vector<int> alias_root;                  // per tensor: root tensor id
+  std::vector<int> storage_root;                // per tensor: the tensor whose arena record holds it (alias root, or further the operand an in-place step wrote over)
   std::vector<int> folded;                      // per tensor: 1 if removed by fusion
   std::vector<int> op_variant;                  // per graph op: the caller's variant request (copy of opts.op_variant)
   std::vector<int> node_variant;                // per node: the variant rated best under the final layouts (0: none)

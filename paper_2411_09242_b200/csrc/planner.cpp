@@ -1358,6 +1358,61 @@ static int lower_and_place(fluid_plan_s* p) {
       p->records.push_back(w);
     }
   }
+  // In-place alias groups: a step whose every output element is written by the thread that read the same element of
+  // one input (rotary embedding, element-wise ops, the residual operand of a GEMM epilogue) may write over that input
+  // when this step is the input's last reader. Output and input then share one record whose lifetime is the union
+  // of the two ("the most suitable slot" of the paper's memory-management paragraph is, for such a tensor, the one
+  // its dying operand already holds). Same bytes, same storage dtype, same layout, no bf16 twin on either side.
+  p->storage_root.assign(nt, -1);
+  for (int t = 0; t < nt; ++t) p->storage_root[t] = p->alias_root[t];
+  if (!p->opts.no_reuse && !p->opts.no_inplace) {
+    std::vector<char> dead(p->records.size(), 0);
+    auto find = [&](int r) {
+      while (p->storage_root[r] != r) r = p->storage_root[r];
+      return r;
+    };
+    for (int si = 0; si < (int)p->steps.size(); ++si) {
+      const Step& st = p->steps[si];
+      if (st.nodes.size() != 1) continue;
+      const Node& n = p->nodes[st.node];
+      int cand[2] = {-1, -1};
+      if (n.kind == N_ROPE) cand[0] = n.a;
+      else if (n.kind == N_GEMM && n.res >= 0) cand[0] = n.res;
+      else if (n.kind == N_ELTWISE) { cand[0] = n.a; cand[1] = n.b; }
+      else continue;
+      const int rd = p->alias_root[n.out];
+      if (rd != n.out || T[rd].kind != FLUID_ACT || p->record_of[rd] < 0 || p->twin_record_of[rd] >= 0) continue;
+      for (int src : cand) {
+        if (src < 0 || T[src].kind != FLUID_ACT) continue;
+        const int ra = p->alias_root[src], rs = find(ra);
+        if (rs == rd || p->record_of[rs] < 0 || p->twin_record_of[ra] >= 0 || p->twin_record_of[rs] >= 0) continue;
+        ArenaRecord& a = p->records[p->record_of[rs]];
+        ArenaRecord& d = p->records[p->record_of[rd]];
+        if (a.bytes != d.bytes || p->wide[ra] != p->wide[rd] || a.last != si || d.first != si) continue;
+        if (T[src].rank != T[n.out].rank || !same_perm(p, src, n.out, lo)) continue;
+        bool same_dims = true;
+        for (int i = 0; i < T[src].rank; ++i) same_dims = same_dims && T[src].dims[i] == T[n.out].dims[i];
+        if (!same_dims) continue;
+        a.last = d.last;
+        dead[p->record_of[rd]] = 1;
+        p->storage_root[rd] = rs;
+        break;
+      }
+    }
+    // drop the absorbed records, resolve every tensor to the record that holds it
+    std::vector<int> remap(p->records.size(), -1);
+    std::vector<ArenaRecord> kept;
+    for (size_t i = 0; i < p->records.size(); ++i)
+      if (!dead[i]) { remap[i] = (int)kept.size(); kept.push_back(p->records[i]); }
+    p->records.swap(kept);
+    for (int t = 0; t < nt; ++t) {
+      if (p->record_of[t] >= 0) p->record_of[t] = remap[p->record_of[t]];
+      if (p->twin_record_of[t] >= 0) p->twin_record_of[t] = remap[p->twin_record_of[t]];
+    }
+    for (int t = 0; t < nt; ++t) p->storage_root[t] = find(p->alias_root[t]);
+    for (int t = 0; t < nt; ++t)
+      if (p->storage_root[t] != p->alias_root[t]) p->record_of[p->alias_root[t]] = p->record_of[p->storage_root[t]];
+  }
   // per-step scratch: split-K partial tiles of GEMM steps with too few output tiles to fill the GPU
   for (int si = 0; si < (int)p->steps.size(); ++si) {
     Step& st = p->steps[si];
@@ -1518,7 +1573,7 @@ int fluid_plan_tensor_info(const fluid_plan_t* p, int t, int* layout_index, int*
   if (layout_index) *layout_index = p->layout[t];
   if (perm)
     for (int i = 0; i < td.rank; ++i) perm[i] = p->cands[t][p->layout[t]][i];
-  const int root = p->alias_root[t];
+  const int root = p->storage_root.empty() ? p->alias_root[t] : p->storage_root[t];   // the tensor whose record holds this one (a view or an in-place result)
   const int rec = p->record_of[root];
   if (offset) *offset = rec >= 0 ? p->records[rec].offset : -1;
   if (bytes) *bytes = rec >= 0 ? p->records[rec].bytes : td.numel() * td.esize();

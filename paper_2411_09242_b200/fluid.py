@@ -57,7 +57,7 @@ class PlanOptions(C.Structure):
                 ("force_canonical", C.c_int32), ("gemm_path", C.c_int32), ("narrow_stream", C.c_int32),
                 ("unfused_attention", C.c_int32), ("split_k", C.c_int32),
                 ("eval", EVAL_FN), ("eval_user", C.c_void_p), ("eval_variant", EVAL_VARIANT_FN),
-                ("op_variant", C.POINTER(C.c_int32)), ("n_op_variant", C.c_int32)]
+                ("op_variant", C.POINTER(C.c_int32)), ("n_op_variant", C.c_int32), ("no_inplace", C.c_int32)]
 
 
 class StepInfo(C.Structure):

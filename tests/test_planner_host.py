@@ -225,7 +225,8 @@ def test_residual_stream_is_held_in_fp32():
     m = synth.build_model(synth.scaled(synth.CONFIGS["gpt2_small"], L=2), materialize=False)
     d = m.graph
     plan = fluid.Plan(d, synth.default_candidates(d))
-    by_name = {d.tensors[r["tensor"]]["name"]: r for r in plan.records() if not r["twin"]}
+    holder = {r["tensor"]: r for r in plan.records() if not r["twin"]}
+    by_name = {td["name"]: holder.get(plan.tensor_info(t).alias_of) for t, td in enumerate(d.tensors)}
     assert by_name["embed"]["dtype"] == synth.F32 and by_name["l0.res1"]["dtype"] == synth.F32
     assert by_name["l0.ln1.out"]["dtype"] == synth.BF16          # feeds GEMMs only
     assert not any(r["twin"] for r in plan.records())            # pre-LN: no tensor needs both
@@ -485,3 +486,31 @@ def test_variant_costs_from_the_caller_decide_layouts_and_variant_with_the_oracl
         assert chosen == min(codes, key=bump) and _decode(chosen)[0] == cheap_form
     assert {v for (n, v) in asked if n == 1} == {0}                          # a node without variants is asked once
     plan.close()
+
+
+def test_in_place_results_share_the_record_of_their_dying_operand():
+    """Residual epilogues and rotary embeddings write over the operand that dies with them: one record, union
+    lifetime, a smaller arena, and still a valid one (independent checker). no_inplace = 1 gives every result its own."""
+    m = synth.build_model(synth.CONFIGS["llama"], materialize=False)
+    d = m.graph
+    cands = synth.default_candidates(d)
+    plan = fluid.Plan(d, cands)
+    apart = fluid.Plan(d, cands, no_inplace=1)
+    name = {td["name"]: t for t, td in enumerate(d.tensors)}
+    root = lambda n: plan.tensor_info(name[n]).alias_of
+    # the fp32 residual stream of a pre-norm model is one buffer from the embedding to the last layer
+    assert root("l0.res1") == root("l0.res2") == root("l3.res2") == root("embed") == name["embed"]
+    assert root("l0.q_rope") == root("l0.q") and root("l2.k_rope") == root("l2.k")
+    assert root("l0.q") != root("l0.k") and root("l0.ln1.out") == name["l0.ln1.out"]
+    assert apart.tensor_info(name["l0.res1"]).alias_of == name["l0.res1"]
+    recs, offs = plan_records(plan)
+    assert OA.check_arena(recs, offs, plan.arena_bytes) == []
+    assert len(recs) < len(apart.records()) and plan.arena_bytes < apart.arena_bytes
+    assert plan.live_bound_bytes < apart.live_bound_bytes
+    # the holder's lifetime covers every tensor that lives in it
+    steps = plan.steps()
+    first, last = next((f, l) for rid, _, f, l in recs if rid == name["embed"])
+    group = [t for t in range(len(d.tensors)) if plan.tensor_info(t).alias_of == name["embed"]]
+    touched = [i for i, s in enumerate(steps) if set(group) & set(s["ins"] + s["outs"])]
+    assert (first, last) == (min(touched), max(touched)) and last > len(steps) // 2
+    plan.close(); apart.close()
