@@ -165,6 +165,10 @@ typedef struct fluid_plan_options {
   int32_t no_inplace;       /* 0 (default): a rotary-embedding, element-wise or residual-epilogue step whose input dies
                                with it writes its result over that input (one arena record, union lifetime);
                                1: every result gets a slice of its own */
+  int32_t redzone_bytes;    /* debugging aid (0 = none): every activation slice is followed by this many bytes (rounded up
+                               to 256) that no kernel may write. In a no_reuse plan the slices are disjoint, so a caller
+                               that fills the arena with a pattern before fluid_run can check the zones afterwards: an
+                               out-of-bounds store of any kernel shows up without a memory checker */
 } fluid_plan_options;
 
 typedef enum {

@@ -1344,7 +1344,8 @@ static int lower_and_place(fluid_plan_s* p) {
     ArenaRecord r;
     r.root = t;
     r.id = t;
-    r.bytes = round_up(T[t].numel() * (p->wide[t] ? 4 : T[t].esize()), FLUID_SLOT_ALIGN);
+    const int64_t zone = p->opts.redzone_bytes > 0 ? round_up(p->opts.redzone_bytes, FLUID_SLOT_ALIGN) : 0;
+    r.bytes = round_up(T[t].numel() * (p->wide[t] ? 4 : T[t].esize()), FLUID_SLOT_ALIGN) + zone;
     r.first = gfirst[t];
     r.last = glast[t];
     p->record_of[t] = (int)p->records.size();
@@ -1353,7 +1354,7 @@ static int lower_and_place(fluid_plan_s* p) {
       ArenaRecord w = r;
       w.id = t + nt;
       w.twin = 1;
-      w.bytes = round_up(T[t].numel() * T[t].esize(), FLUID_SLOT_ALIGN);
+      w.bytes = round_up(T[t].numel() * T[t].esize(), FLUID_SLOT_ALIGN) + zone;
       p->twin_record_of[t] = (int)p->records.size();
       p->records.push_back(w);
     }

@@ -57,7 +57,8 @@ class PlanOptions(C.Structure):
                 ("force_canonical", C.c_int32), ("gemm_path", C.c_int32), ("narrow_stream", C.c_int32),
                 ("unfused_attention", C.c_int32), ("split_k", C.c_int32),
                 ("eval", EVAL_FN), ("eval_user", C.c_void_p), ("eval_variant", EVAL_VARIANT_FN),
-                ("op_variant", C.POINTER(C.c_int32)), ("n_op_variant", C.c_int32), ("no_inplace", C.c_int32)]
+                ("op_variant", C.POINTER(C.c_int32)), ("n_op_variant", C.c_int32), ("no_inplace", C.c_int32),
+                ("redzone_bytes", C.c_int32)]
 
 
 class StepInfo(C.Structure):
@@ -506,6 +507,22 @@ class Runner:
     def status(self):
         torch = _torch()
         return fluid_status(self.plan.handle, self.arena.data_ptr(), torch.cuda.current_stream().cuda_stream)
+
+    def redzone_violations(self, zone_bytes):
+        """For a plan made with no_reuse = 1 and redzone_bytes = zone_bytes, run from a poisoned arena (every byte
+        0xFF): the ids of the arena records whose trailing zone no longer holds the pattern (some kernel stored
+        past the end of that slice). Empty = clean."""
+        torch = _torch()
+        torch.cuda.synchronize()
+        zone = (zone_bytes + SLOT_ALIGN - 1) // SLOT_ALIGN * SLOT_ALIGN
+        bad = []
+        for r in self.plan.records():
+            if r["tensor"] < 0:
+                continue          # per-step scratch has no zone
+            tail = self.arena[r["offset"] + r["bytes"] - zone: r["offset"] + r["bytes"]]
+            if not bool((tail == 0xFF).all()):
+                bad.append(r["id"])
+        return bad
 
     def outputs_host(self):
         torch = _torch()

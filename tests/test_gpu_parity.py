@@ -502,3 +502,52 @@ def test_step_variants_tuned_in_place():
     for tid in m.graph.outputs:
         assert_close(got[tid], ref[tid], synth.BF16, f"tuned-variant plan output {tid}")
     plan.close()
+
+
+# ---- substitutes for a memory checker ------------------------------------------------------------------------------
+@pytest.mark.parametrize("family,dtype", [("encoder", synth.F32), ("gpt", synth.BF16), ("llama", synth.BF16)])
+def test_no_kernel_writes_past_its_slice(family, dtype):
+    """Red zones: a plan with one disjoint slice per activation, each followed by 512 bytes no kernel may touch, run
+    from an arena filled with 0xFF. Every zone still holds the pattern afterwards, the outputs are the oracle's, and
+    they equal, bit for bit, those of the planned (shared-slice, in-place) arena."""
+    cfg = synth.scaled(SMALL[family], dtype=dtype)
+    m = synth.build_model(cfg)
+    cands = synth.default_candidates(m.graph)
+    got, plan, runner = run_gpu(m.graph, model_feeds(m), cands, no_reuse=1, redzone_bytes=512)
+    assert runner.redzone_violations(512) == []
+    assert all(r["bytes"] % 256 == 0 and r["bytes"] >= 768 for r in plan.records() if r["tensor"] >= 0)
+    ref = run_oracle(m.graph, model_feeds(m))
+    shared, plan2, _ = run_gpu(m.graph, model_feeds(m), cands)
+    for tid in m.graph.outputs:
+        assert_close(got[tid], ref[tid], dtype, f"{family} with red zones")
+        assert np.array_equal(got[tid], shared[tid])
+    # the check itself works: a byte scribbled into a zone is found
+    rec = next(r for r in plan.records() if r["tensor"] >= 0)
+    runner.arena[rec["offset"] + rec["bytes"] - 1] = 0
+    assert runner.redzone_violations(512) == [rec["id"]]
+    plan.close(); plan2.close()
+
+
+def test_status_word_in_the_arena_header_is_reported():
+    """The read-back path of the bounded waits, exercised from the host: a non-zero status word written into the arena
+    header (as a kernel whose wait ran out would leave it) makes fluid_status answer FLUID_ETIMEOUT with the code;
+    the next run clears it. No kernel waits on anything here."""
+    import ctypes
+    import torch
+    m = synth.build_model(synth.CONFIGS["tiny"])
+    plan = fluid.Plan(m.graph, synth.default_candidates(m.graph))
+    r = fluid.Runner(plan, m.consts)
+    r.set_inputs([m.ids])
+    r.run()
+    assert r.status() == 0
+    r.arena[:4].copy_(torch.tensor([0x04, 0x01, 0, 0], dtype=torch.uint8, device="cuda"))   # word 0x104
+    st = ctypes.c_int()
+    rc = fluid.lib().fluid_status(plan.handle, ctypes.c_void_p(r.arena.data_ptr()), None, ctypes.byref(st))
+    assert rc == fluid.FLUID_ETIMEOUT and st.value == 0x104
+    assert b"0x104" in fluid.lib().fluid_last_error()
+    r.arena[:4].copy_(torch.tensor([0x10, 0, 0, 0], dtype=torch.uint8, device="cuda"))      # position outside the cache
+    rc = fluid.lib().fluid_status(plan.handle, ctypes.c_void_p(r.arena.data_ptr()), None, ctypes.byref(st))
+    assert rc == fluid.FLUID_EINVAL and st.value == 0x10
+    r.run()                                       # the header is zeroed at the start of every run
+    assert r.status() == 0
+    plan.close()
