@@ -183,7 +183,7 @@ typedef struct fluid_step_info {
                             rating or the caller's eval_variant / op_variant: bit0 A MN-major, bit1 B MN-major, bits 8-19 tile N,
                             bits 20-23 grouped siblings, bits 24-27 split-K factor, bit 28: the split
                             runs as one thread-block cluster per output tile, bit 29: pairs of CTAs share
-                            256 x 256 tiles. GEMM_ROWS: bits 20-23 grouped siblings, bit 29: SiLU(gate) * up is
+                            256 x 256 tiles, bit 30: the rotary embedding of the first projections of the group runs in the epilogue. GEMM_ROWS: bits 20-23 grouped siblings, bit 29: SiLU(gate) * up is
                             applied in the launch, bit 30: the preceding RMS normalisation runs in the launch.
                             ATTN_DECODE: bits 0-7 head dim, bits 8-15 query heads per key/value head, bit 16:
                             the rotary embedding of query and key runs in the launch) */

@@ -101,7 +101,9 @@ __device__ __forceinline__ void rotate_row(float (&x)[V], int li, int pos, const
     const int d = li * V + i;
     const int dd = d < half ? d : d - half;
     float sn, cs;
-    rope_sincos(pos, rope_freq(freq, dd, D), sn, cs);
+    float fh, fl;
+    rope_freq(freq, dd, D, fh, fl);
+    rope_sincos(pos, fh, fl, sn, cs);
     x[i] = d < half ? x[i] * cs - partner[i] * sn : x[i] * cs + partner[i] * sn;
   }
 }

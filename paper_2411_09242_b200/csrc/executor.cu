@@ -64,7 +64,7 @@ int finalize_steps(fluid_plan_s* p) {
         }
         const GemmParams& g = s.gemm;
         // the variant the planner rated best for this node (or the caller asked for); the fused SwiGLU form exists for CTA pairs only
-        const int gv = s.swiglu ? gemm_variant_code(GV_PAIR, 256) : gemm_variant_of(p, n);
+        const int gv = (s.swiglu || s.rope_fused) ? gemm_variant_code(GV_PAIR, 256) : gemm_variant_of(p, n);
         s.kernel = gemm_tc_eligible(p, g, &s.tc, gv) ? FLUID_K_GEMM_TC : FLUID_K_GEMM_SIMT;
         if (s.kernel == FLUID_K_GEMM_TC)
           s.variant = (s.tc.cfg.a_mn_major ? 1 : 0) | (s.tc.cfg.b_mn_major ? 2 : 0) | (s.tc.cfg.bn << 8);
@@ -85,7 +85,7 @@ int finalize_steps(fluid_plan_s* p) {
         s.flops = fl;
         s.bytes = es * (a + b + (g.has_bias ? g.N : 0)) + c * (s.gemm.c_f32 ? 4.0 : es) + (g.has_res ? c * (s.gemm.r_f32 ? 4.0 : es) : 0.0);
         // SwiGLU step: the only tensor written is the product, which takes gate's place
-        const size_t n_gemm = s.swiglu ? 2 : s.nodes.size() - s.norm_fused;
+        const size_t n_gemm = s.swiglu ? 2 : s.nodes.size() - s.norm_fused - s.rope_fused;
         if (s.swiglu) {
           s.t_ptr[2] = p->nodes[s.nodes[2]].out;
           s.gemm.c_f32 = 0;
@@ -109,6 +109,17 @@ int finalize_steps(fluid_plan_s* p) {
           s.bytes += es * (b + c + (g.has_bias ? g.N : 0));
         }
         if (n_gemm > 1) s.variant |= int(n_gemm) << 20;
+        // fused rotary embeddings: the first rope_fused projections write their rotated result (the rope nodes' outputs)
+        for (int ri = 0; ri < s.rope_fused; ++ri) {
+          const Node& rn = p->nodes[s.nodes[n_gemm + ri]];
+          GemmParams& gr = ri == 0 ? s.gemm : s.gemm_x[ri - 1];
+          gr.rope = 1;
+          gr.rope_S = (int)T[rn.out].dims[1];
+          if (ri == 0) s.t_ptr[2] = rn.out; else s.x_ptr[ri - 1][1] = rn.out;
+          rope_freq_fill(s.rope_freq, rn.rope_base, (int)T[rn.out].dims[3]);
+          s.bytes -= 0.0;
+        }
+        if (s.rope_fused) s.variant |= 1 << 30;
         // a handful of rows: the weight-streaming kernel, when every GEMM of the step has k contiguous on both sides
         if (p->opts.gemm_path == 0 && s.split_k <= 1 && g.dtype == FLUID_BF16) {
           bool rows = gemm_rows_eligible(s.gemm);
@@ -407,7 +418,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       const void* b = R(s.t_ptr[1], 1);
       if (!R.ok) return FLUID_EINVAL;
       bool enc_ok = encode_tensor_map(&s.tc.map_a, a, s.tc.a) == 0 && encode_tensor_map(&s.tc.map_b, b, s.tc.b) == 0;
-      for (size_t gi = 1; enc_ok && gi < (s.swiglu ? size_t(2) : s.nodes.size()); ++gi) {
+      for (size_t gi = 1; enc_ok && gi < (s.swiglu ? size_t(2) : s.nodes.size() - s.rope_fused); ++gi) {
         const void* bx = R(s.x_ptr[gi - 1][0], 1);
         if (!R.ok) return FLUID_EINVAL;
         enc_ok = encode_tensor_map(&s.tc_x[gi - 1].map_b, bx, s.tc_x[gi - 1].b) == 0;
@@ -454,7 +465,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
         if (s.kernel == FLUID_K_GEMM_TC) {
           GemmParams gs[3] = {q, s.gemm_x[0], s.gemm_x[1]};
           GemmTcHost ts[3] = {s.tc, s.tc_x[0], s.tc_x[1]};
-          const int ng = s.swiglu ? 2 : (int)s.nodes.size();
+          const int ng = s.swiglu ? 2 : (int)s.nodes.size() - s.rope_fused;
           for (int gi = 1; gi < ng; ++gi) {
             gs[gi].A = q.A;
             gs[gi].B = R(s.x_ptr[gi - 1][0], 1);
@@ -465,7 +476,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
           float* partial = s.scratch_record >= 0
                                ? reinterpret_cast<float*>(static_cast<char*>(arena_ptr) + p->records[s.scratch_record].offset)
                                : nullptr;
-          if (R.ok) err = launch_gemm_tc(gs, ts, ng, s.split_k, s.cluster_k, partial, status, stream, s.swiglu);
+          if (R.ok) err = launch_gemm_tc(gs, ts, ng, s.split_k, s.cluster_k, partial, status, stream, s.swiglu, s.rope_fused ? &s.rope_freq : nullptr);
         } else if (R.ok) {
           err = launch_gemm_simt(q, stream);
         }

@@ -82,6 +82,8 @@ struct Step {
   int split_k = 1;          // GEMM steps with few tiles cut their k range across CTAs
   int cluster_k = 0;        // >1: the cut runs as one thread-block cluster per output tile (no scratch)
   int swiglu = 0;           // 1: nodes = {gate GEMM, up GEMM, SiLU(gate) * up}: one CTA-pair launch, gate and up never stored
+  RopeFreq rope_freq{};     // frequency table of the fused rotary embeddings
+  int rope_fused = 0;       // >0: that many trailing nodes are the rotary embeddings of this step's first projections (CTA-pair GEMM epilogue); the unrotated projections are never stored
   int norm_fused = 0;       // 1: the last node is the RMS normalisation that feeds every GEMM of the step (few-row kernel only); its output is never stored
   float norm_eps = 0.f;
   int norm_x_f32 = 0;

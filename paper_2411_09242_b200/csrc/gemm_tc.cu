@@ -56,6 +56,7 @@ struct TcParams {
   uint32_t* status;     // word 0: device status; words 8..63: per-tile arrival counters for split-K
   int scalar_turn;      // general epilogue: n is contiguous and unsplit in C (and R), so the shared-memory turn applies
   int swiglu;           // CTA-pair form: CTA 0 loads gate columns, CTA 1 up columns; the epilogue writes SiLU(gate) * up
+  RopeFreq rope_freq;   // CTA-pair form with a rotary epilogue (groups whose GemmParams has rope = 1)
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -598,7 +599,7 @@ __device__ __noinline__ void epilogue_tile_scalar(const GemmParams& g, uint32_t 
 
 // Epilogue variants (template parameter of the kernel)
 enum EpiKind { EPI_ANY = 0, EPI_PLAIN = 1, EPI_PLAIN_WIDE = 2, EPI_RES = 3, EPI_RES_WIDE = 4, EPI_GELU_ERF = 5, EPI_GELU_TANH = 6,
-               EPI_SWIGLU = 7 /* CTA-pair kernel only */ };
+               EPI_SWIGLU = 7 /* CTA-pair kernel only */, EPI_ROPE = 8 /* CTA-pair kernel only: plain, with the rotary embedding for groups that ask */ };
 
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk_c(const GemmParams& g, uint32_t taddr, const int64_t (&cbs)[8], const int64_t (&rbs)[8],
@@ -1320,6 +1321,59 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
 // SwiGLU epilogue of the CTA-pair kernel: accumulator columns [0, 128) hold the gate projection and [128, 256) the
 // up projection of the same 128 output columns; the warp writes SiLU(gate) * up for its column range, through the
 // same shared-memory turn as the other vector epilogues (bf16 output, n contiguous).
+// Rotary embedding in the epilogue of a projection (rotate-half pairing, heads of 128 columns): a warp's half of a
+// 256-wide tile is exactly one head, so columns d and d + 64 of a row sit in the same thread's accumulator row. Both
+// 32-column chunks of a pair are read, rotated by the angle of the row's position (frequency table from the host,
+// compensated fp32 angle product and reduction, as in the stand-alone kernel) and leave through the shared-memory turn of
+// the other epilogues. The unrotated projection never exists in memory and is never rounded to bf16.
+__device__ __forceinline__ void epilogue_tile_rope(const GemmParams& g, const RopeFreq& fr, uint32_t trow, int col_begin, int n_tile0,
+                                                   const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane, int pos) {
+  const int unit = lane & 7, rsub = lane >> 3;
+  const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
+  const float scale = g.scale;
+  __nv_bfloat16* const c_b16 = static_cast<__nv_bfloat16*>(g.C);
+  if (n_tile0 + col_begin >= g.N) return;   // uniform across the warp
+#pragma unroll 1
+  for (int c0 = 0; c0 < 64; c0 += 32) {
+    uint32_t ra[32], rb[32];
+    tmem_ld32(trow + uint32_t(col_begin + c0), ra);
+    tmem_ld32(trow + uint32_t(col_begin + 64 + c0), rb);
+    tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      float sn, cs;
+      rope_sincos(pos, fr.hi[c0 + j], fr.lo[c0 + j], sn, cs);
+      const float a = __uint_as_float(ra[j]) * scale, b = __uint_as_float(rb[j]) * scale;
+      ra[j] = __float_as_uint(a * cs - b * sn);
+      rb[j] = __float_as_uint(b * cs + a * sn);
+    }
+#pragma unroll
+    for (int hsel = 0; hsel < 2; ++hsel) {
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t* r = hsel ? rb : ra;
+        sts128(st_row + (uint32_t(u ^ (lane & 7)) << 4), __uint_as_float(r[4 * u]), __uint_as_float(r[4 * u + 1]),
+               __uint_as_float(r[4 * u + 2]), __uint_as_float(r[4 * u + 3]));
+      }
+      __syncwarp();
+      const int nc = n_tile0 + col_begin + hsel * 64 + c0 + unit * 4;
+      int n1, n0i;
+      split2(nc, g.N0, n1, n0i);
+      const int64_t c_col = (int64_t)n1 * g.c_s[4] + n0i;
+      const uint32_t live = nc < g.N ? ok_mask : 0u;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int row = rsub + 4 * i;
+        const float4 v = lds128(st_base + uint32_t(row * 128) + (uint32_t(unit ^ (row & 7)) << 4));
+        uint2* dst = reinterpret_cast<uint2*>(c_b16 + cbs[i] + c_col);
+        const uint2 q = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+        if ((live >> i) & 1u) *dst = q;
+      }
+      __syncwarp();   // the staging tile is rewritten by the next turn
+    }
+  }
+}
+
 __device__ __forceinline__ void epilogue_tile_swiglu(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
                                                      const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane) {
   const int unit = lane & 7, rsub = lane >> 3;
@@ -1543,7 +1597,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * PN);
       if (EPI == EPI_SWIGLU) epilogue_tile_swiglu(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
-      else epilogue_tile_c<EPI>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+      else if (EPI == EPI_ROPE) {
+        if (g.rope) epilogue_tile_rope(g, p.rope_freq, trow, col_begin, n_tile0, cbs, ok_mask, stage, lane, (mt * BM + lane_base + lane) % g.rope_S);
+        else epilogue_tile_c<EPI_PLAIN>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+      } else epilogue_tile_c<EPI>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0u));   // CTA 0 counts both CTAs' epilogue warps
@@ -1689,7 +1746,7 @@ bool gemm_pair_eligible(const GemmParams* gs, const GemmTcHost& tc, int n_group)
 }
 
 cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_group, int split_k, int cluster_k, float* partial,
-                           uint32_t* status, cudaStream_t stream, int swiglu) {
+                           uint32_t* status, cudaStream_t stream, int swiglu, const RopeFreq* rope_freq) {
   const GemmParams& g = gs[0];
   const GemmTcHost& tc = tcs[0];
   TcParams p;
@@ -1786,6 +1843,17 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
   }
   // ---- many 256-wide tiles over an even number of row tiles: pairs of CTAs share 256 x 256 tiles ----
   if (swiglu && !(tc.cfg.pair && pair_enabled() && vec && n_group == 2 && (p.tiles_m & 1) == 0)) return cudaErrorInvalidValue;
+  bool rope = false;
+  for (int i = 0; i < n_group; ++i) rope = rope || gs[i].rope;
+  if (rope) {   // the rotary epilogue exists in the CTA-pair form only, over the plain bf16 epilogue
+    if (!(tc.cfg.pair && pair_enabled() && vec && epi == EPI_PLAIN && !swiglu && rope_freq && (p.tiles_m & 1) == 0 &&
+          g.causal == CAUSAL_NONE && split_k <= 1))
+      return cudaErrorInvalidValue;
+    for (int i = 0; i < n_group; ++i)
+      if (gs[i].rope && (gs[i].N0 % 128 != 0 || gs[i].N % 128 != 0 || gs[i].rope_S < 1 || gs[i].batch != 1)) return cudaErrorInvalidValue;
+    p.rope_freq = *rope_freq;
+    epi = EPI_ROPE;
+  }
   if (tc.cfg.pair && pair_enabled() && vec && epi != EPI_ANY && split_k <= 1 && g.causal == CAUSAL_NONE && (p.tiles_m & 1) == 0 &&
       p.num_tiles > 0) {
     TcParams q = p;
@@ -1815,7 +1883,7 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 2 : 1;
-    static bool pattr_set[8] = {false, false, false, false, false, false, false, false};
+    static bool pattr_set[9] = {false, false, false, false, false, false, false, false, false};
 #define FLUID_TC_PAIR(E)                                                                                             \
   case E: {                                                                                                          \
     if (!pattr_set[E]) {                                                                                             \
@@ -1833,6 +1901,7 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
       FLUID_TC_PAIR(EPI_GELU_ERF)
       FLUID_TC_PAIR(EPI_GELU_TANH)
       FLUID_TC_PAIR(EPI_SWIGLU)
+      FLUID_TC_PAIR(EPI_ROPE)
       default: break;
     }
 #undef FLUID_TC_PAIR

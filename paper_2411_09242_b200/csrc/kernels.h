@@ -38,6 +38,8 @@ struct GemmParams {
                // CAUSAL_CLIP_K: the k loop stops after the tile holding k = m_max
   int has_bias, has_res;
   int b_const;  // B is a constant of the plan (a weight): its loads need not wait for the previous step
+  int rope;     // 1: the rotary embedding of the output (heads of 128 columns, pairs (d, d + 64), position = row % rope_S) runs in the epilogue
+  int rope_S;   // rows per sequence
 };
 
 // Host-side description of the two TMA tensor maps of a tensor-core GEMM step.
@@ -112,15 +114,19 @@ struct SoftmaxParams {
                       // multiple of zero_block past the diagonal (the consumer reads no further)
 };
 
-// Rotary frequencies base^(-2i/D) of the first 64 pairs in double, computed once on the host (head dims up to 128);
-// pairs beyond that are computed on the device from log2_base.
+// Rotary frequencies base^(-2i/D) of the first 64 pairs, computed once on the host in double and handed over as a pair of
+// floats (hi + lo carries 48 bits); pairs beyond 64 are computed on the device from log2_base (head dims above 128).
 struct RopeFreq {
   double log2_base;
-  double f[64];
+  float hi[64], lo[64];
 };
 inline void rope_freq_fill(RopeFreq& t, double base, int D) {
   t.log2_base = std::log2(base);
-  for (int i = 0; i < 64; ++i) t.f[i] = std::exp2(-2.0 * i / D * t.log2_base);
+  for (int i = 0; i < 64; ++i) {
+    const double f = std::exp2(-2.0 * i / D * t.log2_base);
+    t.hi[i] = (float)f;
+    t.lo[i] = (float)(f - (double)t.hi[i]);
+  }
 }
 
 struct RopeParams {
@@ -235,7 +241,7 @@ cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
 // swiglu (two groups, CTA-pair form only): group 0 is the gate, group 1 the up projection; the launch writes
 // SiLU(gate) * up to g[0].C and nothing else.
 cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, int split_k, int cluster_k, float* partial,
-                           uint32_t* status, cudaStream_t stream, int swiglu = 0);
+                           uint32_t* status, cudaStream_t stream, int swiglu = 0, const RopeFreq* rope_freq = nullptr);
 // Split factor a GEMM step should use (1 = none) and the scratch it then needs.
 int gemm_split_k(const GemmParams& g, const GemmTcHost& tc, int n_group, int64_t* scratch_bytes);
 // Cluster size of the cluster split-K form (CTAs of one cluster share an output tile, reduced through

@@ -724,7 +724,9 @@ __global__ void rope_kernel(RopeParams p, int64_t total) {
     const int64_t base = idx[0] * p.st[0] + idx[1] * p.st[1] + idx[2] * p.st[2];
     float sn, cs;
     const int pos0 = p.pos ? p.pos[idx[0] * p.pos_stride] : 0;
-    rope_sincos(idx[1] + pos0, rope_freq(p.freq, pr, p.dims[3]), sn, cs);
+    float fh, fl;
+    rope_freq(p.freq, pr, p.dims[3], fh, fl);
+    rope_sincos(idx[1] + pos0, fh, fl, sn, cs);
     const T* x = static_cast<const T*>(p.x);
     T* y = static_cast<T*>(p.y);
     const float a = to_f(x[base + d0 * p.st[3]]), b = to_f(x[base + d1 * p.st[3]]);
@@ -750,7 +752,9 @@ __global__ void __launch_bounds__(256) rope_vec_kernel(RopeParams p, int64_t tot
     float cs[8], sn[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      rope_sincos(s + pos0, rope_freq(p.freq, c * 8 + j, D), sn[j], cs[j]);
+      float fh, fl;
+      rope_freq(p.freq, c * 8 + j, D, fh, fl);
+      rope_sincos(s + pos0, fh, fl, sn[j], cs[j]);
     }
     const int h_end = min(p.dims[2], (hg + 1) * ROPE_HG);
     for (int h = hg * ROPE_HG; h < h_end; ++h) {

@@ -1242,6 +1242,62 @@ static int lower_and_place(fluid_plan_s* p) {
       p->steps.erase(p->steps.begin() + si + 1);
     }
   }
+  // Rotary embedding behind a grouped projection step (q, k, v): when the projections run as CTA pairs over 256-wide
+  // tiles and the heads are 128 wide, each epilogue warp holds whole heads of its rows, so the rotation of q and k
+  // runs in the epilogue and the unrotated tensors are never stored (nor rounded).
+  if (p->opts.fusion && p->opts.gemm_path == 0 && !p->opts.eval && !p->opts.eval_variant) {
+    std::vector<int> n_uses(nt, 0);
+    for (const Node& n : p->nodes)
+      for (int t : n.ins) n_uses[t]++;
+    for (int si = 0; si < (int)p->steps.size(); ++si) {
+      Step& st = p->steps[si];
+      if (st.swiglu || st.norm_fused || st.nodes.size() < 2 || p->nodes[st.node].kind != N_GEMM) continue;
+      const Node& n0 = p->nodes[st.node];
+      GemmParams g;
+      GemmTcHost tc;
+      if (n0.bias >= 0 || n0.act != ACT_NONE || !lower_gemm(p, n0, lo, &g)) continue;
+      if (!gemm_tc_eligible(p, g, &tc, gemm_variant_code(GV_PAIR, 256)) || !tc.cfg.pair) continue;
+      GemmParams gs[3] = {g, g, g};
+      if (!gemm_pair_eligible(gs, tc, (int)st.nodes.size()) || g.batch != 1 || g.N0 % 128 != 0 || g.N % 128 != 0 || g.c_s[5] != 1) continue;
+      // the rotary steps that read this step's outputs, directly behind it
+      std::vector<int> ropes;
+      std::vector<int> order;   // GEMM nodes: rotated ones first (the launch applies the rotation per group)
+      double base = 0;
+      bool ok = true;
+      for (int sj = si + 1; sj < (int)p->steps.size() && sj <= si + 2 && ok; ++sj) {
+        const Step& sr = p->steps[sj];
+        if (sr.nodes.size() != 1) break;
+        const Node& r = p->nodes[sr.node];
+        if (r.kind != N_ROPE) break;
+        int owner = -1;
+        for (int ni : st.nodes)
+          if (p->nodes[ni].out == r.a) owner = ni;
+        if (owner < 0 || r.rope_interleaved || r.pos >= 0 || n_uses[r.a] != 1 || T[r.a].kind != FLUID_ACT ||
+            p->alias_root[r.a] != r.a || p->alias_root[r.out] != r.out || T[r.out].dtype != FLUID_BF16 || T[r.out].rank != 4 ||
+            T[r.out].dims[3] != 128 || lo[r.a] != lo[r.out] || (base != 0 && base != r.rope_base))
+          break;
+        base = r.rope_base;
+        ropes.push_back(sj);
+        order.push_back(owner);
+      }
+      if (ropes.empty()) continue;
+      (void)ok;
+      for (int ni : st.nodes)
+        if (std::find(order.begin(), order.end(), ni) == order.end()) order.push_back(ni);
+      for (int sj : ropes) {
+        const Node& r = p->nodes[p->steps[sj].node];
+        st.cost += p->steps[sj].cost - kLaunch;
+        p->folded[r.a] = 1;
+      }
+      const int first_rope = p->steps[ropes[0]].node, second_rope = ropes.size() > 1 ? p->steps[ropes[1]].node : -1;
+      st.nodes = order;
+      st.node = order[0];
+      st.nodes.push_back(first_rope);
+      if (second_rope >= 0) st.nodes.push_back(second_rope);
+      st.rope_fused = (int)ropes.size();
+      for (int k = (int)ropes.size() - 1; k >= 0; --k) p->steps.erase(p->steps.begin() + ropes[k]);
+    }
+  }
   // RMSNorm or LayerNorm in front of few-row GEMMs: when every reader of the normalised tensor is a GEMM of the next step and that
   // step runs the weight-streaming kernel, the normalisation runs inside it (the gain on the way in, 1/rms in the
   // epilogue) and the normalised tensor is never stored.

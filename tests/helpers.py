@@ -255,6 +255,12 @@ def check_steps_sampled(desc, plan, runner, feeds, n_rows=48, tol=2 ** -7, seed=
             elif kind in (synth.LAYERNORM, synth.RMSNORM):
                 want = graph_exec.run_op(kind, [value(op["ins"][0])] + [np.asarray(const_value(t), np.float64) for t in op["ins"][1:]],
                                          op["attrs"])[0]
+            elif kind == synth.ROPE and first["kind"] == synth.LINEAR:
+                # a rotary embedding folded into the projection's step: the sampled rows are (batch, position) pairs,
+                # each rotated by its own position
+                x = np.asarray(value(op["ins"][0]), np.float64)
+                pos = np.asarray(index[1], dtype=np.int64)
+                want = graph_exec.run_op(kind, [x[:, None], pos], op["attrs"])[0][:, 0]
             elif kind == synth.SELECT_LAST_TOKEN:
                 want = runner.read_tensor(op["ins"][0])[:, -1, :]
             else:

@@ -102,9 +102,9 @@ def test_llama_first_layer_rounding_cascade():
             rms[name] = float(np.sqrt(np.mean(d ** 2)) / np.sqrt(np.mean(stored[t] ** 2)))
             print(f"{s['kernel_name']:10s} {name:16s} differing {frac[name]:.4f}  rms {rms[name]:.2e}  max {d.max() / np.abs(stored[t]).max():.2e}")
             assert_close(have, stored[t], synth.BF16, f"one layer, {name} vs storage-rounded oracle", tol=2 ** -7)
-    assert frac["l0.q"] < 0.01 and rms["l0.q"] < 5e-4
-    assert frac["l0.ctx_h"] > 5 * frac["l0.q"]
-    assert rms["final_norm.out"] > 5 * rms["l0.q"]
+    assert frac["l0.v"] < 0.01 and rms["l0.v"] < 5e-4 and frac["l0.q_rope"] < 0.01
+    assert frac["l0.ctx_h"] > 5 * frac["l0.v"]
+    assert rms["final_norm.out"] > 5 * rms["l0.v"]
     plan.close()
 
 
