@@ -523,6 +523,90 @@ def time_sweep(torch, fluid, peaks, reps=5):
                                            float(np.max([r["tflops"] for r in gemm_rows]))]}
 
 
+def single_cases():
+    """One-operator graphs for the captures under profiles/: the memory-bound kernels at sizes well beyond L2, the
+    decoding kernels, a few GEMM shapes. name -> (graph, algorithmic bytes or None, flops or None)."""
+    BF = synth.BF16
+
+    def one_op(kind, in_shapes, out_shape, attrs=None):
+        g = synth.GraphDesc()
+        ins = [g.tensor(f"in{i}", BF, shp, synth.INPUT) for i, shp in enumerate(in_shapes)]
+        out = g.tensor("out", BF, out_shape, synth.OUTPUT)
+        g.op(kind, ins, [out], **(attrs or {}))
+        return g
+
+    n_big = 8192 * 11008
+    out = {
+        "softmax_dense": (one_op(synth.SOFTMAX, [[1, 32, 2048, 2048]], [1, 32, 2048, 2048], {"causal": 0, "scale": 1.0}), 2.0 * 32 * 2048 * 2048 * 2, None),
+        "softmax_causal": (one_op(synth.SOFTMAX, [[1, 32, 2048, 2048]], [1, 32, 2048, 2048], {"causal": 1, "scale": 1.0}), 1.0 * 32 * 2048 * 2048 * 2, None),
+        "layernorm_65536x768": (one_op(synth.LAYERNORM, [[1, 65536, 768], [768], [768]], [1, 65536, 768], {"eps": 1e-5}), 2.0 * 65536 * 768 * 2, None),
+        "rmsnorm_16384x4096": (one_op(synth.RMSNORM, [[1, 16384, 4096], [4096]], [1, 16384, 4096], {"eps": 1e-5}), 2.0 * 16384 * 4096 * 2, None),
+        "rope_4x2048x32x128": (one_op(synth.ROPE, [[4, 2048, 32, 128]], [4, 2048, 32, 128], {"rope_base": 10000.0}), 2.0 * 4 * 2048 * 32 * 128 * 2, None),
+        "add_8192x11008": (one_op(synth.ADD, [[1, 8192, 11008]] * 2, [1, 8192, 11008]), 3.0 * n_big * 2, None),
+        "gelu_8192x11008": (one_op(synth.GELU, [[1, 8192, 11008]], [1, 8192, 11008]), 2.0 * n_big * 2, None),
+    }
+    for tgt in ("BHSD", "BHDS"):
+        for (B, S, nh, D) in ((8, 2048, 32, 128), (8, 2048, 12, 64)):
+            g, _ = synth.permute_case(B, S, nh, D, tgt)
+            out[f"permute_{tgt}_{B}x{S}x{nh}x{D}"] = (g, 2.0 * B * S * nh * D * 2, None)
+    g = synth.GraphDesc()
+    ids = g.tensor("ids", synth.I32, [16, 2048], synth.INPUT)
+    tok = g.tensor("tok", BF, [32000, 4096], synth.INPUT)
+    x = g.tensor("x", BF, [16, 2048, 4096], synth.OUTPUT)
+    g.op(synth.EMBED, [ids, tok], [x])
+    out["embed_32768x4096"] = (g, 2.0 * 32768 * 4096 * 2, None)
+    for (B_, nh, D, T) in ((4, 32, 128, 2048), (16, 32, 128, 4096)):
+        g = synth.GraphDesc()
+        q = g.tensor("q", BF, [B_, 1, nh, D], synth.INPUT)
+        k = g.tensor("k", BF, [B_, 1, nh, D], synth.INPUT)
+        v = g.tensor("v", BF, [B_, 1, nh, D], synth.INPUT)
+        kc = g.tensor("kc", BF, [B_, T, nh, D], synth.STATE)
+        vc = g.tensor("vc", BF, [B_, T, nh, D], synth.STATE)
+        pos = g.tensor("pos", synth.I32, [1], synth.INPUT)
+        o = g.tensor("ctx", BF, [B_, 1, nh, D], synth.OUTPUT)
+        g.op(synth.CACHED_ATTENTION, [q, k, v, kc, vc, pos], [o], scale=D ** -0.5)
+        out[f"decode_attention_{B_}x{nh}x{D}_cache{T}"] = (g, 2.0 * 2 * B_ * T * nh * D, None)
+    for (M, N, K) in ((8192, 8192, 8192), (4096, 2304, 768), (2048, 11008, 4096), (128, 768, 3072), (4, 32000, 4096), (4, 4096, 11008)):
+        g, _ = synth.gemm_case(M, N, K, "row", "col", materialize=False)
+        out[f"gemm_{M}x{N}x{K}"] = (g, 2.0 * (M * K + K * N + M * N) if M <= 16 else None, 2.0 * M * N * K)
+    return out
+
+
+def run_single(name, torch, fluid, peaks, reps=10):
+    """One single-operator case: planned and run through the C-ABI, timed with an event pair around `reps` back-to-back
+    runs. Operands of a few hundred MB defeat L2; the small GEMM shapes here are L2-resident and say so."""
+    cases = single_cases()
+    if name not in cases:
+        raise SystemExit("unknown case; one of: " + ", ".join(cases))
+    g, by, fl = cases[name]
+    plan = fluid.Plan(g, synth.default_candidates(g))
+    r = fluid.Runner(plan, {})
+    for b_ in r.inputs:
+        if b_.dtype == torch.int32 and b_.numel() == 1:
+            b_.fill_(g.dims(g.inputs[3])[1] - 1 if len(g.inputs) > 3 else 0)   # a decoding position: the last cache row
+        elif b_.dtype == torch.int32:
+            b_.random_(0, 32000)
+        else:
+            b_.uniform_(-2, 2)
+    for _ in range(3):
+        r.run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        r.run()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / reps
+    line = {"single": name, "kernels": [s["kernel_name"] for s in plan.steps()], "us_per_run": us, "status": r.status()}
+    if by is not None:
+        line.update({"algorithmic_mb": by / 1e6, "gbs": by / us / 1e3, "frac_measured_hbm": by / us / 1e3 / peaks["hbm_gbs"]})
+    else:
+        line.update({"gflop": fl / 1e9, "tflops": fl / us / 1e6, "frac_measured_burst": fl / us / 1e6 / peaks["bf16_tflops"]})
+    print(json.dumps(line), flush=True)
+    plan.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -539,6 +623,8 @@ def main():
     ap.add_argument("--tune-variants", action="store_true",
                     help="time every tensor-core GEMM step of the headline plan with each implementation variant, in place, "
                          "and run the plan with the fastest per step (reported beside the rated plan's latency)")
+    ap.add_argument("--single", default="", help="run one single-operator case (for the captures under profiles/) and exit; "
+                                                 "'list' prints the names")
     ap.add_argument("--layers", type=int, default=0, help="reduced copy of the workload (profiling captures only)")
     ap.add_argument("--seq", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0)
@@ -566,6 +652,13 @@ def main():
     fluid.lib()
     peaks = load_peaks()
     args.warmup = max(3, args.warmup)
+    if args.single:
+        if rank == 0:
+            if args.single == "list":
+                print("\n".join(single_cases()))
+            else:
+                run_single(args.single, torch, fluid, peaks)
+        return
 
     def barrier():
         torch.cuda.synchronize()
