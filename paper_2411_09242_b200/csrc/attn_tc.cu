@@ -585,8 +585,8 @@ __device__ __forceinline__ float ex2_poly(float x) {
   return __int_as_float(__float_as_int(q) + (__float_as_int(z) << 23));
 }
 
-template <int D>
-__global__ void __launch_bounds__(kAttnThreads, 1)
+template <int D, int TPR>
+__global__ void __launch_bounds__(256 * TPR + 64, 1)
 attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ AttnParams p) {
   constexpr int DC = D / 64;                       // 64-wide chunks of the head dim
@@ -597,6 +597,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const uint32_t q_full = bars, k_full = bars + 8, v_full = bars + 24, k_free = bars + 40, v_free = bars + 56,
                  s_full = bars + 72, p_full = bars + 88, o_done = bars + 104;
   const uint32_t tmem_slot = bars + 120;
+  float* xch = reinterpret_cast<float*>(smem_raw + (bars + 256 - raw));   // TPR = 2: [tile][parity][half][128] maxima, then [tile][half][128] sums
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
   volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
 
@@ -626,7 +627,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     mbar_init(q_full, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(k_full + 8 * i, 1); mbar_init(v_full + 8 * i, 1); mbar_init(k_free + 8 * i, 1); mbar_init(v_free + 8 * i, 1);
-      mbar_init(s_full + 8 * i, 1); mbar_init(p_full + 8 * i, 128); mbar_init(o_done + 8 * i, 1);
+      mbar_init(s_full + 8 * i, 1); mbar_init(p_full + 8 * i, 128 * TPR); mbar_init(o_done + 8 * i, 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -644,7 +645,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const uint32_t tmem_base = *tmem_slot_ptr;
   // S_t at columns 128 t (P_t over its first 64), O_t at 256 + D t
 
-  if (warp == 9) {
+  constexpr int kMmaWarp = 8 * TPR, kLoadWarp = 8 * TPR + 1;
+  if (warp == kLoadWarp) {
     // ======================= loads =======================
     const bool lead = lane == 0;
     constexpr int NB = 2 * DC;               // boxes per tile
@@ -737,7 +739,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       for (int j = max(0, k_issued - 2); j < k_issued; ++j) mbar_wait(k_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
       for (int j = max(0, v_issued - 2); j < v_issued; ++j) mbar_wait(v_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
     }
-  } else if (warp == 8) {
+  } else if (warp == kMmaWarp) {
     // ======================= MMAs =======================
     // The whole warp runs this role in lockstep and one lane's instructions carry the issue predicate. Kept
     // convergent, the descriptor arithmetic stays on the uniform datapath, where tcgen05.mma takes its operands
@@ -775,8 +777,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const uint64_t vb = dv + uint64_t(st) * (kTile >> 4);
         const uint32_t tP = tm + uint32_t(t * TK), tO = tm + 2 * TK + uint32_t(t * D);
 #pragma unroll
-        for (int kk = 0; kk < TK / 16; ++kk)   // 16 keys = 8 packed columns of P per instruction
-          umma_ts_elect(tO, tP + uint32_t(kk * 8),
+        for (int kk = 0; kk < TK / 16; ++kk)   // 16 keys = 8 packed columns of P per instruction (TPR = 2: each half row's P lies over its own 64 score columns)
+          umma_ts_elect(tO, tP + (TPR == 2 ? uint32_t((kk >> 2) * 64 + (kk & 3) * 8) : uint32_t(kk * 8)),
                         vb + (p.v_k_major ? uint64_t(((kk >> 2) * (D * 128) + (kk & 3) * 32) >> 4) : uint64_t(kk * 128)), idesc_o,
                         (j > 0 || kk > 0) ? 1u : 0u, leader);
         umma_commit_elect(o_done + 8u * t, leader);
@@ -797,6 +799,165 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       if (!ok && leader) {
         *abort_flag = 1;
         atomicOr(p.status, 0x100u | fail);
+      }
+    }
+  } else if (TPR == 2) {
+    // ======================= softmax, two threads per query row: warps 0-7 query tile 0, warps 8-15 tile 1 ===========
+    // Thread (row, half) owns score columns 64 half .. 64 half + 63 of its row and writes its probabilities over the
+    // first 32 of them, so the two threads of a row never touch each other's columns. Twice the warps per scheduler
+    // of the one-thread-per-row form: a lone softmax warp issues at about half the rate two reach together.
+    // Measured: no faster than one thread per row. Stamps in the MMA warp show why: it waits ~100 cycles per round for
+    // the probabilities and spends the rest issuing; a 128 x 128 x 16 instruction takes ~100-120 cycles here against
+    // the 64 the tensor core needs (8 KB of shared-memory operands per instruction is the whole shared-memory
+    // bandwidth of an SM at 64 cycles), so the tensor side sets the pace in either form, not the softmax.
+    // The reference point m_used of a row is the same in both threads. A pass first asks, through one reducing
+    // barrier over the tile's 256 threads, whether any half row's maximum has moved more than 2^8 above it; only
+    // then (and on the first key tile) do the halves exchange their maxima and rescale O. Every thread takes every
+    // barrier, also after a failed wait (it then only skips the work), so no barrier is left waiting.
+    const int t = warp >> 3, wq = warp & 3, half = (warp >> 2) & 1;
+    const int row = wq * 32 + lane;
+    const int qi = m0 + t * TQ + row;
+    const uint32_t lane_addr = uint32_t(wq * 32) << 16;
+    const uint32_t tS = tmem_base + lane_addr + uint32_t(t * TK + half * 64);
+    const uint32_t tO = tmem_base + lane_addr + 2 * TK + uint32_t(t * D + half * (D / 2));
+    float* xm = xch + t * 512;           // [parity][half][128]
+    float* xl = xch + 1024 + t * 256;    // [half][128]
+    const int n = n_kv[t];
+    float m_used = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    uint32_t fail = 0;
+    int slow = 0;
+    auto tile_sync = [&]() {
+      if (t == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+      else asm volatile("bar.sync 2, 256;" ::: "memory");
+    };
+    auto tile_any = [&](bool mine) -> bool {
+      uint32_t r;
+      if (t == 0)
+        asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.or.pred p, 1, 256, q;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(r) : "r"(mine ? 1u : 0u) : "memory");
+      else
+        asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.or.pred p, 2, 256, q;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(r) : "r"(mine ? 1u : 0u) : "memory");
+      return r != 0;
+    };
+    for (int j = 0; j < n; ++j) {
+      if (ok && !mbar_wait_warp(s_full + 8u * t, uint32_t(j) & 1u)) { ok = false; fail |= 0x40u; }
+      const int kv0 = j * TK + half * 64;
+      tc_fence_after();
+      const int kv_lim = (p.causal ? min(p.S, qi + 1) : p.S) - kv0;   // this thread's local columns >= kv_lim are masked
+      const bool full = __all_sync(0xffffffffu, kv_lim >= 64);
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (ok) {
+        uint32_t q[2][32];
+        tmem_ld32(tS, q[0]);
+        tmem_ld32(tS + 32, q[1]);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          if (full) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8)
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+                mx4[u] = max3(mx4[u], __uint_as_float(q[c][i + 2 * u]), __uint_as_float(q[c][i + 2 * u + 1]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i < kv_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(q[c][i]));
+          }
+        }
+      }
+      const float m_half = ceilf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2);
+      if (tile_any(ok && (j == 0 || m_half > m_used + 8.f))) {
+        float* x = xm + (slow & 1) * 256;
+        ++slow;
+        x[half * 128 + row] = ok ? m_half : -INFINITY;
+        tile_sync();
+        const float m_row = fmaxf(x[row], x[128 + row]);
+        const float m_new = (j == 0 || m_row > m_used + 8.f) ? m_row : m_used;
+        if (j > 0) {
+          // P_{j-1}.V_{j-1} must have landed in O before it is rescaled
+          if (ok && !mbar_wait_warp(o_done + 8u * t, uint32_t(j - 1) & 1u)) { ok = false; fail |= 0x80u; }
+          const float alpha = exp2f(m_used - m_new);
+          if (ok) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < D / 2; c0 += 32) {
+              uint32_t q[32];
+              tmem_ld32(tO + c0, q);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) q[i] = __float_as_uint(__uint_as_float(q[i]) * alpha);
+              tmem_st32(tO + c0, q);
+            }
+          }
+          l_run *= alpha;
+        }
+        m_used = m_new;
+      }
+      if (ok) {
+        // P = exp2(s * k - m_used) as bf16 pairs over the first 32 of this thread's 64 score columns
+        const float neg_m = -m_used;
+        const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(neg_m, neg_m);
+        uint64_t acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+        uint32_t q[2][32];
+        tmem_ld32(tS, q[0]);
+        tmem_ld32(tS + 32, q[1]);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(q[c][2 * i]), __uint_as_float(q[c][2 * i + 1])), sc2, nm2), x0, x1);
+            float a = ex2_fast(x0), bb = ex2_fast(x1);
+            if (!full) {
+              if (c * 32 + 2 * i >= kv_lim) a = 0.f;
+              if (c * 32 + 2 * i + 1 >= kv_lim) bb = 0.f;
+            }
+            w[i] = pack_bf16x2(a, bb);
+            acc[i & 1] = add2(acc[i & 1], pack2(a, bb));   // fp32 sum of the unrounded exponentials
+          }
+          tmem_st16(tS + c * 16, w);
+        }
+        float s0, s1, s2, s3;
+        unpack2(acc[0], s0, s1);
+        unpack2(acc[1], s2, s3);
+        l_run += (s0 + s1) + (s2 + s3);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        tc_fence_before();
+        mbar_arrive(p_full + 8u * t);
+      }
+    }
+    // ---- O / l -> bf16: each thread its half of the head dim ----
+    if (ok && n > 0) {
+      if (!mbar_wait_warp(o_done + 8u * t, uint32_t(n - 1) & 1u)) { ok = false; fail |= 0x80u; }
+      tc_fence_after();
+    }
+    if (fail && lane == 0) atomicOr(p.status, 0x100u | fail);
+    if (!ok) *abort_flag = 1;
+    xl[half * 128 + row] = l_run;
+    tile_sync();
+    if (ok && n > 0 && !*abort_flag) {
+      const float l_tot = xl[row] + xl[128 + row];
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.O) + (int64_t)b * p.o_s[0] + (int64_t)h * p.o_s[1] + (int64_t)qi * p.o_s[2] +
+                           half * (D / 2);
+      pdl_wait();  // O may still be read by an earlier step
+#pragma unroll 1
+      for (int c0 = 0; c0 < D / 2; c0 += 32) {
+        uint32_t q[32];
+        tmem_ld32(tO + c0, q);     // warp-collective: rows past the end take part, then skip the store
+        tmem_ld_wait();
+        if (qi < p.S) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(q[g * 8 + i]) * inv;
+            store16(out + c0 + g * 8, v);
+          }
+        }
       }
     }
   } else {
@@ -948,25 +1109,26 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 }  // namespace
 
 // Which form runs: two query tiles per CTA (probabilities in tensor memory) when the sequence has more than one query
-// tile, else the one-tile form. FLUID_ATTN_FORM=1 / 2 in the environment forces one of them (A/B timing).
+// tile (one thread per query row), else the one-tile form. FLUID_ATTN_FORM in the environment forces a form (A/B timing):
+// 1 one tile per CTA, 2 two tiles with one thread per row, 3 two tiles with two threads per row.
 static int attn_form(const AttnParams& p) {
   static const int forced = [] {
     const char* e = std::getenv("FLUID_ATTN_FORM");
     return e ? std::atoi(e) : 0;
   }();
-  if (forced == 1 || forced == 2) return forced;
+  if (forced >= 1 && forced <= 3) return forced;
   return p.S > TQ ? 2 : 1;
 }
 
 template <typename K>
-static cudaError_t launch_attn_form(K kernel, bool* attr_done, size_t smem, dim3 grid, cudaStream_t stream, const CUtensorMap* mq,
-                                    const CUtensorMap* mk, const CUtensorMap* mv, const AttnParams& p) {
+static cudaError_t launch_attn_form(K kernel, bool* attr_done, size_t smem, dim3 grid, int threads, cudaStream_t stream,
+                                    const CUtensorMap* mq, const CUtensorMap* mk, const CUtensorMap* mv, const AttnParams& p) {
   if (!*attr_done) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     *attr_done = true;
   }
-  return launch_k(kernel, grid, kAttnThreads, smem, stream, *mq, *mk, *mv, p);
+  return launch_k(kernel, grid, threads, smem, stream, *mq, *mk, *mv, p);
 }
 
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream) {
@@ -974,18 +1136,22 @@ cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream
   const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(&host.map_q);
   const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(&host.map_k);
   const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(&host.map_v);
-  static bool attr[4] = {false, false, false, false};
+  static bool attr[6] = {false, false, false, false, false, false};
   if (D != 64 && D != 128) return cudaErrorInvalidValue;
-  if (attn_form(p) == 2) {
-    const size_t smem = size_t(6) * TQ * D * 2 + 256 + 1024;
+  const int form = attn_form(p);
+  if (form >= 2) {
+    const size_t smem = size_t(6) * TQ * D * 2 + 256 + 6144 + 1024;
     const dim3 grid(((p.S + 2 * TQ - 1) / (2 * TQ)) * p.B * p.NH);
-    return D == 64 ? launch_attn_form(attn_tc2_kernel<64>, &attr[2], smem, grid, stream, mq, mk, mv, p)
-                   : launch_attn_form(attn_tc2_kernel<128>, &attr[3], smem, grid, stream, mq, mk, mv, p);
+    if (form == 3)   // two threads per query row: measured no faster (940 vs 958 TFLOP/s on 2 x 4096 x 32 x 128); kept for A/B timing
+      return D == 64 ? launch_attn_form(attn_tc2_kernel<64, 2>, &attr[4], smem, grid, 576, stream, mq, mk, mv, p)
+                     : launch_attn_form(attn_tc2_kernel<128, 2>, &attr[5], smem, grid, 576, stream, mq, mk, mv, p);
+    return D == 64 ? launch_attn_form(attn_tc2_kernel<64, 1>, &attr[2], smem, grid, 320, stream, mq, mk, mv, p)
+                   : launch_attn_form(attn_tc2_kernel<128, 1>, &attr[3], smem, grid, 320, stream, mq, mk, mv, p);
   }
   const size_t smem = size_t(5) * TQ * D * 2 + size_t(2) * TQ * TK * 2 + 128 + 2048;
   const dim3 grid(((p.S + TQ - 1) / TQ) * p.B * p.NH);
-  return D == 64 ? launch_attn_form(attn_tc_kernel<64>, &attr[0], smem, grid, stream, mq, mk, mv, p)
-                 : launch_attn_form(attn_tc_kernel<128>, &attr[1], smem, grid, stream, mq, mk, mv, p);
+  return D == 64 ? launch_attn_form(attn_tc_kernel<64>, &attr[0], smem, grid, kAttnThreads, stream, mq, mk, mv, p)
+                 : launch_attn_form(attn_tc_kernel<128>, &attr[1], smem, grid, kAttnThreads, stream, mq, mk, mv, p);
 }
 
 }  // namespace fluid
