@@ -560,6 +560,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       case FLUID_K_SELECT_LAST: {
         PermuteParams q = s.permute;
         q.x = R(s.t_ptr[0], 1); q.y = const_cast<void*>(R(s.t_ptr[1]));
+        q.status = status;
         if (R.ok) err = launch_permute(q, stream);
         break;
       }

@@ -163,6 +163,7 @@ struct PermuteParams {
   int64_t xs[5], ys[5];
   int64_t x_offset;   // elements, added to x
   int x_inner, y_inner;  // output-logical dim that is contiguous in x / in y (-1: none)
+  uint32_t* status;      // device status word for the TMA form's bounded waits (may be null)
 };
 
 struct EmbedParams {
@@ -240,6 +241,10 @@ cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
 // arrival counters (zero before the launch, left zero after it).
 // swiglu (two groups, CTA-pair form only): group 0 is the gate, group 1 the up projection; the launch writes
 // SiLU(gate) * up to g[0].C and nothing else.
+int encode_tensor_map_plain(TensorMapStorage* out, const void* base, int esize, const uint64_t* dims, const uint64_t* strides_bytes,
+                            const uint32_t* box);
+// Row-gather layout transform as TMA loads and stores; false if the transform does not qualify (nothing launched).
+bool launch_permute_rows_tma(const PermuteParams& p, uint32_t* status, cudaStream_t st, cudaError_t* err);
 cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, int split_k, int cluster_k, float* partial,
                            uint32_t* status, cudaStream_t stream, int swiglu = 0, const RopeFreq* rope_freq = nullptr);
 // Split factor a GEMM step should use (1 = none) and the scratch it then needs.

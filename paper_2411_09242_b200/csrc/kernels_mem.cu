@@ -1169,7 +1169,20 @@ static void permute_dispatch(const PermuteParams& p, cudaStream_t st) {
   launch_k(permute_tile_kernel<E>, (unsigned)blocks, 256, 0, st, x, y, t, t.dims[3], t.dims[4], tiles_i, tiles_o);
 }
 
+// FLUID_PERMUTE_TMA=0 in the environment keeps every transform on the register kernels (A/B timing).
+static bool permute_tma_enabled() {
+  static const bool on = [] {
+    const char* e = std::getenv("FLUID_PERMUTE_TMA");
+    return !(e && e[0] == '0');
+  }();
+  return on;
+}
+
 cudaError_t launch_permute(const PermuteParams& p, cudaStream_t st) {
+  if (permute_tma_enabled()) {
+    cudaError_t err = cudaSuccess;
+    if (launch_permute_rows_tma(p, p.status, st, &err)) return err;
+  }
   if (p.esize == 2) permute_dispatch<uint16_t>(p, st);
   else permute_dispatch<uint32_t>(p, st);
   return cudaGetLastError();
