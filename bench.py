@@ -548,7 +548,7 @@ def single_cases():
         "gelu_8192x11008": (one_op(synth.GELU, [[1, 8192, 11008]], [1, 8192, 11008]), 2.0 * n_big * 2, None),
     }
     for tgt in ("BHSD", "BHDS"):
-        for (B, S, nh, D) in ((8, 2048, 32, 128), (8, 2048, 12, 64)):
+        for (B, S, nh, D) in ((8, 2048, 32, 128), (32, 2048, 32, 128), (8, 2048, 12, 64)):
             g, _ = synth.permute_case(B, S, nh, D, tgt)
             out[f"permute_{tgt}_{B}x{S}x{nh}x{D}"] = (g, 2.0 * B * S * nh * D * 2, None)
     g = synth.GraphDesc()

@@ -1672,10 +1672,11 @@ int encode_tensor_map(TensorMapStorage* out, const void* base, const TmaOperand&
   return rc == CUDA_SUCCESS ? 0 : -2;
 }
 
-// A plain tiled map for copies: elements of `esize` bytes (2 or 4) moved as they are, no swizzle, dims / strides (bytes;
+// A plain tiled map for copies: elements of `esize` bytes (2 or 4) moved as they are, dims / strides (bytes;
 // strides[0] is ignored, the fastest dim is dense) / box given fastest first, padded to rank 5 by the caller.
+// swizzle128: the 128-byte swizzle (box[0] * esize must then be 128 and the shared-memory box 1024-byte aligned).
 int encode_tensor_map_plain(TensorMapStorage* out, const void* base, int esize, const uint64_t* dims, const uint64_t* strides_bytes,
-                            const uint32_t* box) {
+                            const uint32_t* box, bool swizzle128) {
   EncodeTiledFn enc = get_encode();
   if (!enc || !base || (reinterpret_cast<uintptr_t>(base) & 15) || (esize != 2 && esize != 4)) return -1;
   cuuint64_t d[5], st[4];
@@ -1687,8 +1688,8 @@ int encode_tensor_map_plain(TensorMapStorage* out, const void* base, int esize, 
     if (i > 0) st[i - 1] = strides_bytes[i];
   }
   CUresult rc = enc(reinterpret_cast<CUtensorMap*>(out), esize == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32, 5,
-                    const_cast<void*>(base), d, st, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    const_cast<void*>(base), d, st, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? 0 : -2;
 }
 

@@ -242,9 +242,11 @@ cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t stream);
 // swiglu (two groups, CTA-pair form only): group 0 is the gate, group 1 the up projection; the launch writes
 // SiLU(gate) * up to g[0].C and nothing else.
 int encode_tensor_map_plain(TensorMapStorage* out, const void* base, int esize, const uint64_t* dims, const uint64_t* strides_bytes,
-                            const uint32_t* box);
-// Row-gather layout transform as TMA loads and stores; false if the transform does not qualify (nothing launched).
-bool launch_permute_rows_tma(const PermuteParams& p, uint32_t* status, cudaStream_t st, cudaError_t* err);
+                            const uint32_t* box, bool swizzle128 = false);
+// Layout transforms as TMA loads and stores (rows gathered when both sides share the fastest dim, 64 x 64 tiles of
+// 16-bit elements transposed in shared memory when they do not); false if the transform does not qualify (nothing
+// launched).
+bool launch_permute_tma(const PermuteParams& p, uint32_t* status, cudaStream_t st, cudaError_t* err);
 cudaError_t launch_gemm_tc(const GemmParams* g, const GemmTcHost* tc, int n_group, int split_k, int cluster_k, float* partial,
                            uint32_t* status, cudaStream_t stream, int swiglu = 0, const RopeFreq* rope_freq = nullptr);
 // Split factor a GEMM step should use (1 = none) and the scratch it then needs.

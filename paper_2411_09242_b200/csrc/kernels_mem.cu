@@ -1181,7 +1181,7 @@ static bool permute_tma_enabled() {
 cudaError_t launch_permute(const PermuteParams& p, cudaStream_t st) {
   if (permute_tma_enabled()) {
     cudaError_t err = cudaSuccess;
-    if (launch_permute_rows_tma(p, p.status, st, &err)) return err;
+    if (launch_permute_tma(p, p.status, st, &err)) return err;
   }
   if (p.esize == 2) permute_dispatch<uint16_t>(p, st);
   else permute_dispatch<uint32_t>(p, st);

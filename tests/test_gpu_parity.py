@@ -216,6 +216,22 @@ def test_layout_transforms_bit_exact(dtype, case, target):
 
 
 @pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("case", [dict(B=2, S=1000, nh=5, D=72), dict(B=1, S=4104, nh=3, D=136), dict(B=3, S=520, nh=7, D=64),
+                                  dict(B=1, S=1001, nh=9, D=128), dict(B=2, S=264, nh=40, D=200)])
+@pytest.mark.parametrize("target", ["BHSD", "BHDS"])
+def test_large_ragged_layout_transforms_bit_exact(dtype, case, target):
+    """Transforms above a megabyte take the bulk-tensor (TMA) forms when their strides allow it: extents that are not
+    multiples of the 64-wide tile or of the box rows, 16- and 32-bit elements, and one case (S = 1001) whose output
+    stride is not 16-byte aligned and therefore stays on the register kernels."""
+    g, a = synth.permute_case(target=target, dtype=dtype, **case)
+    got, plan, r = run_gpu(g, {0: a})
+    ref = run_oracle(g, {0: a})[1]
+    assert np.array_equal(got[1], ref)
+    assert r.status() == 0
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
 def test_embed_and_select_last(dtype):
     g = synth.GraphDesc()
     ids = g.tensor("ids", synth.I32, [3, 17], synth.INPUT)
