@@ -1,6 +1,8 @@
 // Fused attention for sm_100a: S = Q.K^T and O = softmax(S).V on tcgen05 tensor cores with the
 // score tiles kept in tensor memory; the [S, S] score / probability tensors never reach HBM or the
-// arena. One CTA = one (batch, head, 128-query tile); 320 threads: 8 softmax warps (two threads per
+// arena. Two forms. Sequences of more than one query tile run the persistent two-tile form described further down
+// (probabilities stay in tensor memory). The one-tile form, described here, serves sequences of a single query tile
+// and A/B timing: one CTA = one (batch, head, 128-query tile); 320 threads: 8 softmax warps (two threads per
 // query row, 64 key columns each), one warp that issues the MMAs, one warp that issues the TMA loads.
 // (Sixteen softmax warps, four threads per row, were measured and are no faster: with 128 x 128 x 16 and
 // 128 x D x 16 instructions costing the same ~128 cycles as a 128 x 256 x 16 one, the tensor pipe is
@@ -494,28 +496,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 }
 
 
-// ---- two query tiles per CTA, probabilities in tensor memory ------------------------------------------------------
-// One CTA = one (batch, head) and 256 consecutive queries, as two 128-row tiles that share every K / V tile the CTA
-// loads. Warps 0-3 are the softmax of query tile 0, warps 4-7 of tile 1 (one thread per query row: the row's maximum
-// and sum never leave the thread), warp 8 (one thread) issues every tcgen05.mma, warp 9 the TMA loads. Tensor memory:
+// ---- two query tiles per work item, probabilities in tensor memory ----------------------------------------------
+// A work item = one (batch, head) and 256 consecutive queries, as two 128-row tiles ("slots") that share every K / V
+// tile loaded for the item. Warps 0-3 are the softmax of slot 0, warps 4-7 of slot 1 (one thread per query row: the
+// row's maximum and sum never leave the thread), warp 8 issues every tcgen05.mma, warp 9 the TMA loads. Tensor memory:
 // S_0, S_1 (128 fp32 columns each), O_0, O_1 (D columns each). A softmax thread reads its row of S_t, writes the bf16
 // probabilities back over the same columns (two per 32-bit column, 64 columns), and P_t.V runs with the A operand
-// taken from tensor memory: P never passes through shared memory. Per query tile the chain S = Q.K_j^T -> softmax ->
-// O += P.V_j is serial; the two tiles run half a step apart, so the tensor core works for one tile while the other
-// tile's softmax runs.
-//   q_full        both Q tiles have landed                           TMA -> MMA
-//   k_full[s], v_full[s]   K / V stage s has landed                  TMA -> MMA
-//   k_free[s], v_free[s]   every MMA that reads stage s is complete  MMA commit -> loader
-//   s_full[t]     S_t holds Q_t.K_j^T                                MMA commit -> softmax t
-//   p_full[t]     P_t is written (and S_t read)                      128 softmax threads -> MMA
-//   o_done[t]     O_t holds P_t.V_j                                  MMA commit -> softmax t (rescale, end)
-__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_c, uint32_t tmem_a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                             uint32_t acc) {
-  asm volatile(
-      "{\n .reg .pred p;\n .reg .b64 db;\n mov.b64 db, {%2, %3};\n setp.ne.b32 p, %5, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}"
-      ::"r"(tmem_c), "r"(tmem_a), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
-}
+// taken from tensor memory: P never passes through shared memory. Per slot the chain S = Q.K_j^T -> softmax ->
+// O += P.V_j is serial; the two slots run half a step apart, so the tensor core works for one while the other's
+// softmax runs.
+//   q_full        both Q tiles of the item have landed                TMA -> MMA
+//   q_free        the item's last Q.K^T has read them                 MMA commit -> loader
+//   k_full[s], v_full[s]   K / V stage s has landed                   TMA -> MMA
+//   k_free[s], v_free[s]   every MMA that reads stage s is complete   MMA commit -> loader
+//   s_full[t]     S_t holds Q_t.K_j^T                                 MMA commit -> softmax t
+//   p_full[t]     P_t is written (and S_t read)                       128 softmax threads -> MMA
+//   o_done[t]     O_t holds P_t.V_j                                   MMA commit -> softmax t (rescale, end)
+//   o_free[t]     the item's output has been read out of O_t          128 softmax threads -> MMA
+// What sets the pace (clock stamps in both roles, non-causal 2 x 4096 x 32 x 128): a slot's step is softmax ~2000
+// cycles (maximum pass 450, exponential pass 1530: 128 exponentials per thread at 4 per clock and scheduler), then
+// ~1900 cycles in which the MMA warp takes its three waits (~450) and issues the 8 + 8 instructions of P.V and the next
+// Q.K^T (~700 + ~750, i.e. ~90 cycles an instruction against 64 alone). The MMA warp serves the two slots in turn and
+// is busy throughout, so a step of both slots takes ~4050 cycles for 2 x 1024 cycles of tensor-core work.
 // Forms for a role that the whole warp runs in lockstep: every lane executes the instruction, one lane's carries a true
 // issue predicate.
 __device__ __forceinline__ void umma_ss_elect(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc,
@@ -531,6 +533,53 @@ __device__ __forceinline__ void umma_ts_elect(uint32_t tmem_c, uint32_t tmem_a, 
       "{\n .reg .pred p, q;\n setp.ne.b32 p, %4, 0;\n setp.ne.b32 q, %5, 0;\n"
       " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
       ::"r"(tmem_c), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc), "r"(leader) : "memory");
+}
+// Every MMA of one product (Q.K^T over the head dim, P.V over a key tile) in ONE asm block: the predicates are set once
+// and the descriptors advance by immediates, so an instruction costs the issuing warp two additions and itself. The
+// warp shares its scheduler with softmax warps, and every instruction it does not issue leaves the tensor cores
+// waiting less (measured alone: 64 cycles per 128 x 128 x 16 instruction either way; beside two warps issuing
+// fused multiply-adds on the same scheduler: 115 per instruction one by one, 108 in blocks, 186 when those warps
+// issue nothing else; special-function and integer instructions beside it cost nothing).
+#define FLUID_MMA_SS_1(OA, OB) \
+    " add.s64 a, %1, " #OA "; add.s64 b, %2, " #OB ";\n @q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, one;\n"
+#define FLUID_MMA_SS_HEAD \
+    "{\n .reg .pred q, one;\n .reg .b64 a, b;\n setp.ne.b32 q, %4, 0;\n setp.eq.b32 one, 0, 0;\n" \
+    " @q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, !one;\n"
+#define FLUID_MMA_SS_ARGS ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(leader) : "memory"
+// S = Q.K^T: the first instruction overwrites the accumulator. kk-th offsets: A K-major in 64-wide chunks; B likewise,
+// or MN-major (128 descriptor units per 16 keys).
+template <int D, bool B_MN>
+__device__ __forceinline__ void umma_qk_block(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t leader) {
+  if (D == 64) {
+    if (!B_MN) asm volatile(FLUID_MMA_SS_HEAD FLUID_MMA_SS_1(2, 2) FLUID_MMA_SS_1(4, 4) FLUID_MMA_SS_1(6, 6) "}" FLUID_MMA_SS_ARGS);
+    else asm volatile(FLUID_MMA_SS_HEAD FLUID_MMA_SS_1(2, 128) FLUID_MMA_SS_1(4, 256) FLUID_MMA_SS_1(6, 384) "}" FLUID_MMA_SS_ARGS);
+  } else {
+    if (!B_MN) asm volatile(FLUID_MMA_SS_HEAD FLUID_MMA_SS_1(2, 2) FLUID_MMA_SS_1(4, 4) FLUID_MMA_SS_1(6, 6) FLUID_MMA_SS_1(1024, 1024)
+                            FLUID_MMA_SS_1(1026, 1026) FLUID_MMA_SS_1(1028, 1028) FLUID_MMA_SS_1(1030, 1030) "}" FLUID_MMA_SS_ARGS);
+    else asm volatile(FLUID_MMA_SS_HEAD FLUID_MMA_SS_1(2, 128) FLUID_MMA_SS_1(4, 256) FLUID_MMA_SS_1(6, 384) FLUID_MMA_SS_1(1024, 512)
+                      FLUID_MMA_SS_1(1026, 640) FLUID_MMA_SS_1(1028, 768) FLUID_MMA_SS_1(1030, 896) "}" FLUID_MMA_SS_ARGS);
+  }
+}
+#define FLUID_MMA_TS_1(OA, OB) \
+    " add.u32 a, %1, " #OA "; add.s64 b, %2, " #OB ";\n @q tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, one;\n"
+#define FLUID_MMA_TS_HEAD \
+    "{\n .reg .pred p, q, one;\n .reg .b64 b;\n .reg .b32 a;\n setp.ne.b32 p, %4, 0;\n setp.ne.b32 q, %5, 0;\n setp.eq.b32 one, 0, 0;\n" \
+    " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+#define FLUID_MMA_TS_ARGS ::"r"(tmem_c), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc), "r"(leader) : "memory"
+// O (+)= P.V over one 128-key tile: eight instructions of 16 keys (8 packed columns of P each); acc: whether the first
+// one adds to O. B offsets: V with d contiguous (MN-major: 128 units per 16 keys) or with keys contiguous (K-major in
+// 64-key chunks of D rows).
+template <int D, bool V_K>
+__device__ __forceinline__ void umma_pv_block(uint32_t tmem_c, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc, uint32_t leader) {
+  if (!V_K)
+    asm volatile(FLUID_MMA_TS_HEAD FLUID_MMA_TS_1(8, 128) FLUID_MMA_TS_1(16, 256) FLUID_MMA_TS_1(24, 384) FLUID_MMA_TS_1(32, 512)
+                 FLUID_MMA_TS_1(40, 640) FLUID_MMA_TS_1(48, 768) FLUID_MMA_TS_1(56, 896) "}" FLUID_MMA_TS_ARGS);
+  else if (D == 64)
+    asm volatile(FLUID_MMA_TS_HEAD FLUID_MMA_TS_1(8, 2) FLUID_MMA_TS_1(16, 4) FLUID_MMA_TS_1(24, 6) FLUID_MMA_TS_1(32, 512)
+                 FLUID_MMA_TS_1(40, 514) FLUID_MMA_TS_1(48, 516) FLUID_MMA_TS_1(56, 518) "}" FLUID_MMA_TS_ARGS);
+  else
+    asm volatile(FLUID_MMA_TS_HEAD FLUID_MMA_TS_1(8, 2) FLUID_MMA_TS_1(16, 4) FLUID_MMA_TS_1(24, 6) FLUID_MMA_TS_1(32, 1024)
+                 FLUID_MMA_TS_1(40, 1026) FLUID_MMA_TS_1(48, 1028) FLUID_MMA_TS_1(56, 1030) "}" FLUID_MMA_TS_ARGS);
 }
 __device__ __forceinline__ void umma_commit_elect(uint32_t bar, uint32_t leader) {
   asm volatile(
@@ -585,8 +634,20 @@ __device__ __forceinline__ float ex2_poly(float x) {
   return __int_as_float(__float_as_int(q) + (__float_as_int(z) << 23));
 }
 
-template <int D, int TPR>
-__global__ void __launch_bounds__(256 * TPR + 64, 1)
+// Two query tiles per CTA, persistent: gridDim.x CTAs (one per SM) walk the launch's work items. A work item is a pair
+// of adjacent 128-row query tiles of one (batch, head); items are numbered heaviest first (with a causal mask the last
+// query tiles see the most key tiles) and dealt to the CTAs in a snake (round r: CTA c takes item r P + c when r is
+// even, r P + P - 1 - c when odd), which for weights that fall with the item number is the longest-first rule: the
+// CTA that drew the heaviest item of a round draws the lightest of the next. Nothing is torn down between items:
+// tensor memory and barriers stay, the key / value ring keeps running across the boundary, the next item's query
+// tiles are fetched as soon as the last Q.K^T of the current one has read them, and its first scores are computed
+// while the softmax warps still normalise and store the current output. (As one CTA per item, a second CTA on an SM
+// started 3.7 us after the first had left and spent another 3 us before its first instruction on the tensor cores;
+// the causal Llama-shaped launch of 256 items took 49.6 us for 39.4 us of its heaviest item.)
+// Barrier phases count completions over the whole launch, not per item: kc key / value tiles loaded before this item,
+// sc[t] score tiles of slot t, oc[t] items in which slot t was active.
+template <int D>
+__global__ void __launch_bounds__(320, 1)
 attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ AttnParams p) {
   constexpr int DC = D / 64;                       // 64-wide chunks of the head dim
@@ -595,29 +656,36 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t sQ = raw, sK = sQ + 2 * kTile, sV = sK + 2 * kTile, bars = sV + 2 * kTile;
   const uint32_t q_full = bars, k_full = bars + 8, v_full = bars + 24, k_free = bars + 40, v_free = bars + 56,
-                 s_full = bars + 72, p_full = bars + 88, o_done = bars + 104;
-  const uint32_t tmem_slot = bars + 120;
-  float* xch = reinterpret_cast<float*>(smem_raw + (bars + 256 - raw));   // TPR = 2: [tile][parity][half][128] maxima, then [tile][half][128] sums
+                 s_full = bars + 72, p_full = bars + 88, o_done = bars + 104, q_free = bars + 120, o_free = bars + 128;
+  const uint32_t tmem_slot = bars + 144;
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
   volatile uint32_t* abort_flag = tmem_slot_ptr + 1;
 
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // heaviest first: with a causal mask the last query tiles see the most key tiles
   const int n_bz = p.B * p.NH;
-  const int mt = (int(gridDim.x) / n_bz - 1) - int(blockIdx.x) / n_bz, bz = int(blockIdx.x) % n_bz;
-  const int h = bz % p.NH, b = bz / p.NH;
-  const int m0 = mt * 2 * TQ;
-  // key tiles each query tile needs (0: the tile lies beyond the sequence)
-  int n_kv[2];
+  const int n_mt = (p.S + 2 * TQ - 1) / (2 * TQ);
+  const int n_items = n_mt * n_bz;
+  const int n_cta = int(gridDim.x), cta = int(blockIdx.x);
+  // r-th item of this CTA, -1 past the end (a CTA without an item in round r has none in a later round either)
+  auto item_of = [&](int r) -> int {
+    const int idx = r * n_cta + ((r & 1) ? n_cta - 1 - cta : cta);
+    return idx < n_items ? idx : -1;
+  };
+  struct Item { int bz, m0, n_kv[2], n_max; };
+  auto decode = [&](int it, Item& w) {
+    w.bz = it % n_bz;
+    w.m0 = ((n_mt - 1) - it / n_bz) * 2 * TQ;
+    // key tiles each query tile needs (0: the tile lies beyond the sequence)
 #pragma unroll
-  for (int t = 0; t < 2; ++t) {
-    const int mq = m0 + t * TQ;
-    int n = mq < p.S ? (p.S + TK - 1) / TK : 0;
-    if (p.causal && n) n = min(n, (mq + TQ - 1) / TK + 1);
-    n_kv[t] = n;
-  }
-  const int n_max = max(n_kv[0], n_kv[1]);
+    for (int t = 0; t < 2; ++t) {
+      const int mq = w.m0 + t * TQ;
+      int n = mq < p.S ? (p.S + TK - 1) / TK : 0;
+      if (p.causal && n) n = min(n, (mq + TQ - 1) / TK + 1);
+      w.n_kv[t] = n;
+    }
+    w.n_max = max(w.n_kv[0], w.n_kv[1]);
+  };
   if (raw & 1023u) {   // cannot happen with the launch this file does; refuse rather than run misaligned tiles
     if (threadIdx.x == 0) atomicOr(p.status, 0x100u | 0x08u);
     return;
@@ -625,9 +693,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
+    mbar_init(q_free, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(k_full + 8 * i, 1); mbar_init(v_full + 8 * i, 1); mbar_init(k_free + 8 * i, 1); mbar_init(v_free + 8 * i, 1);
-      mbar_init(s_full + 8 * i, 1); mbar_init(p_full + 8 * i, 128 * TPR); mbar_init(o_done + 8 * i, 1);
+      mbar_init(s_full + 8 * i, 1); mbar_init(p_full + 8 * i, 128); mbar_init(o_done + 8 * i, 1); mbar_init(o_free + 8 * i, 128);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -645,7 +714,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const uint32_t tmem_base = *tmem_slot_ptr;
   // S_t at columns 128 t (P_t over its first 64), O_t at 256 + D t
 
-  constexpr int kMmaWarp = 8 * TPR, kLoadWarp = 8 * TPR + 1;
+  constexpr int kMmaWarp = 8, kLoadWarp = 9;
   if (warp == kLoadWarp) {
     // ======================= loads =======================
     const bool lead = lane == 0;
@@ -654,81 +723,96 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int bx = k_lane ? lane : lane - NB;
     int cur[5] = {0, 0, 0, 0, 0}, inc[5] = {0, 0, 0, 0, 0};
     uint32_t box_dst = 0;
-    if (k_lane) {
-      if (!p.k_mn_major) {          // [d chunk][128 keys][64 d]: box (dc, rh)
-        const int dc = bx >> 1, rh = bx & 1;
-        coords(p.k_sel, dc * 64, rh * 64, bz, p.k_b0, cur);
-        box_dst = sK + dc * 16384u + rh * 8192u;
-      } else {                      // [key chunk][D d-rows][64 keys]: box (sc, dc)
-        const int sc = bx / DC, dc = bx % DC;
-        coords(p.k_sel, dc * 64, sc * 64, bz, p.k_b0, cur);
-        box_dst = sK + sc * (D * 128u) + dc * 8192u;
+    // this lane's box of a K / V tile: where it lands, and its coordinates at key tile 0 of (batch, head) bz
+    auto start_head = [&](int bz) {
+      if (k_lane) {
+        if (!p.k_mn_major) {          // [d chunk][128 keys][64 d]: box (dc, rh)
+          const int dc = bx >> 1, rh = bx & 1;
+          coords(p.k_sel, dc * 64, rh * 64, bz, p.k_b0, cur);
+          box_dst = sK + dc * 16384u + rh * 8192u;
+        } else {                      // [key chunk][D d-rows][64 keys]: box (sc, dc)
+          const int sc = bx / DC, dc = bx % DC;
+          coords(p.k_sel, dc * 64, sc * 64, bz, p.k_b0, cur);
+          box_dst = sK + sc * (D * 128u) + dc * 8192u;
+        }
+      } else if (v_lane) {
+        if (!p.v_k_major) {           // [d chunk][128 keys][64 d]  (MN-major B of P.V): box (dc, kc)
+          const int dc = bx >> 1, kc = bx & 1;
+          coords(p.v_sel, kc * 64, dc * 64, bz, p.v_b0, cur);
+          box_dst = sV + dc * 16384u + kc * 8192u;
+        } else {                      // [key chunk][D d-rows][64 keys]  (K-major B of P.V): box (kc, dh)
+          const int kc = bx / DC, dh = bx % DC;
+          coords(p.v_sel, kc * 64, dh * 64, bz, p.v_b0, cur);
+          box_dst = sV + kc * (D * 128u) + dh * 8192u;
+        }
       }
+    };
+    if (k_lane) {
 #pragma unroll
       for (int d = 0; d < 5; ++d) inc[d] = p.k_sel[d] == 2 ? TK : 0;
     } else if (v_lane) {
-      if (!p.v_k_major) {           // [d chunk][128 keys][64 d]  (MN-major B of P.V): box (dc, kc)
-        const int dc = bx >> 1, kc = bx & 1;
-        coords(p.v_sel, kc * 64, dc * 64, bz, p.v_b0, cur);
-        box_dst = sV + dc * 16384u + kc * 8192u;
-      } else {                      // [key chunk][D d-rows][64 keys]  (K-major B of P.V): box (kc, dh)
-        const int kc = bx / DC, dh = bx % DC;
-        coords(p.v_sel, kc * 64, dh * 64, bz, p.v_b0, cur);
-        box_dst = sV + kc * (D * 128u) + dh * 8192u;
-      }
 #pragma unroll
       for (int d = 0; d < 5; ++d) inc[d] = p.v_sel[d] == 0 ? TK : 0;
     }
     uint32_t fail = 0;
-    int k_issued = 0, v_issued = 0;
-    auto load_k = [&](int j) {
-      const uint32_t bar = k_full + 8u * (j & 1);
+    int kc = 0;         // key / value tiles issued so far, over all items: tile kc lands in stage kc & 1
+    int q_issued = 0;   // items whose query tiles have been issued
+    auto load_kv = [&](bool is_k) {
+      const uint32_t bar = (is_k ? k_full : v_full) + 8u * (kc & 1);
       if (lead) mbar_expect_tx(bar, kTile);
-      if (k_lane) {
-        tma_load5(box_dst + uint32_t(j & 1) * kTile, &map_k, bar, cur);
+      if (is_k ? k_lane : v_lane) {
+        tma_load5(box_dst + uint32_t(kc & 1) * kTile, is_k ? &map_k : &map_v, bar, cur);
 #pragma unroll
         for (int d = 0; d < 5; ++d) cur[d] += inc[d];
       }
-      k_issued = j + 1;
-    };
-    auto load_v = [&](int j) {
-      const uint32_t bar = v_full + 8u * (j & 1);
-      if (lead) mbar_expect_tx(bar, kTile);
-      if (v_lane) {
-        tma_load5(box_dst + uint32_t(j & 1) * kTile, &map_v, bar, cur);
-#pragma unroll
-        for (int d = 0; d < 5; ++d) cur[d] += inc[d];
-      }
-      v_issued = j + 1;
     };
     auto all_ok = [&](bool mine) { return __shfl_sync(0xffffffffu, mine ? 1 : 0, 0) != 0; };   // lane 0 decides
 
     pdl_wait();  // Q, K, V come from the previous steps
-    if (lead) {
-      const int n_q = n_kv[1] ? 2 : 1;
-      mbar_expect_tx(q_full, uint32_t(n_q) * kTile);
-      int c[5];
-      for (int t = 0; t < n_q; ++t)
-        for (int dc = 0; dc < DC; ++dc)
-          for (int rh = 0; rh < 2; ++rh) {
-            coords(p.q_sel, dc * 64, m0 + t * TQ + rh * 64, bz, p.q_b0, c);
-            tma_load5(sQ + uint32_t(t) * kTile + dc * 16384u + rh * 8192u, &map_q, q_full, c);
-          }
-    }
-    if (n_max > 0) { load_k(0); load_v(0); }
-    if (n_max > 1) { load_k(1); load_v(1); }
     bool ok = true;
-    for (int j = 0; ok && j + 2 < n_max; ++j) {
-      const int st = j & 1;
-      const uint32_t ph = uint32_t(j >> 1) & 1u;
-      if (lead && !mbar_wait(k_free + 8u * st, ph)) { fail |= 0x40u; ok = false; }
-      ok = all_ok(ok);
-      if (!ok) break;
-      load_k(j + 2);
-      if (lead && !mbar_wait(v_free + 8u * st, ph)) { fail |= 0x80u; ok = false; }
-      ok = all_ok(ok && !*abort_flag);
-      if (!ok) break;
-      load_v(j + 2);
+    for (int r = 0; ok; ++r) {
+      const int it = item_of(r);
+      if (it < 0) break;
+      Item w;
+      decode(it, w);
+      start_head(w.bz);
+      if (r > 0) {   // the previous item's last Q.K^T has read the query tiles
+        if (lead && !mbar_wait(q_free, uint32_t(r - 1) & 1u)) { fail |= 0x10u; ok = false; }
+        ok = all_ok(ok && !*abort_flag);
+        if (!ok) break;
+      }
+      if (lead) {
+        const int n_q = w.n_kv[1] ? 2 : 1;
+        mbar_expect_tx(q_full, uint32_t(n_q) * kTile);
+        int c[5];
+        for (int t = 0; t < n_q; ++t)
+          for (int dc = 0; dc < DC; ++dc)
+            for (int rh = 0; rh < 2; ++rh) {
+              coords(p.q_sel, dc * 64, w.m0 + t * TQ + rh * 64, w.bz, p.q_b0, c);
+              tma_load5(sQ + uint32_t(t) * kTile + dc * 16384u + rh * 8192u, &map_q, q_full, c);
+            }
+      }
+      q_issued = r + 1;
+      for (int j = 0; j < w.n_max; ++j) {
+        // stage kc & 1 is free once the tile loaded two before (kc - 2) has been read: completion (kc - 2) / 2 of its barrier
+        const uint32_t ph = uint32_t((kc - 2) >> 1) & 1u;
+        if (kc >= 2) {
+          if (lead && !mbar_wait(k_free + 8u * (kc & 1), ph)) { fail |= 0x40u; ok = false; }
+          ok = all_ok(ok);
+          if (!ok) break;
+        }
+        load_kv(true);
+        if (kc >= 2) {
+          if (lead && !mbar_wait(v_free + 8u * (kc & 1), ph)) { fail |= 0x80u; ok = false; }
+          ok = all_ok(ok && !*abort_flag);
+          if (!ok) {   // the K tile of this index is in flight, its V tile is not
+            if (lead) mbar_wait(k_full + 8u * (kc & 1), uint32_t(kc >> 1) & 1u);
+            break;
+          }
+        }
+        load_kv(false);
+        ++kc;
+      }
     }
     if (!ok && lead) {
       *abort_flag = 1;
@@ -736,15 +820,21 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     if (lead && *abort_flag) {
       // let loads still in flight land before the shared memory is given up (each wait is bounded)
-      for (int j = max(0, k_issued - 2); j < k_issued; ++j) mbar_wait(k_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
-      for (int j = max(0, v_issued - 2); j < v_issued; ++j) mbar_wait(v_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
+      if (q_issued > 0) mbar_wait(q_full, uint32_t(q_issued - 1) & 1u);
+      for (int j = max(0, kc - 2); j < kc; ++j) {
+        mbar_wait(k_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
+        mbar_wait(v_full + 8u * (j & 1), uint32_t(j >> 1) & 1u);
+      }
     }
   } else if (warp == kMmaWarp) {
     // ======================= MMAs =======================
-    // The whole warp runs this role in lockstep and one lane's instructions carry the issue predicate. Kept
-    // convergent, the descriptor arithmetic stays on the uniform datapath, where tcgen05.mma takes its operands
-    // from; with the role under a one-lane branch every operand went through per-instruction register moves and a
-    // 128 x 128 x 16 instruction cost ~107 cycles to issue against the 64 the tensor core needs to run it.
+    // The whole warp runs this role in lockstep and one lane's instructions carry the issue predicate. A probe with this
+    // very issue code and nothing else on the SM runs a 128 x 128 x 16 instruction every 64 cycles (convergent or under
+    // a one-lane branch alike, also with eight warps reading and writing tensor memory beside it: 66). What slows it is
+    // arithmetic on the SAME scheduler: beside two warps there that issue fused multiply-adds back to back an
+    // instruction takes 115-186 cycles, beside warps that issue only special-function or integer instructions, or that
+    // sit on the other three schedulers, 64-77. Every scheduler carries one softmax warp of each slot (a warp reaches
+    // only the tensor-memory lanes of its own quarter), so this role cannot be moved out of their way.
     {
       const uint32_t leader = lane == 0 ? 1u : 0u;
       uint32_t fail = 0;
@@ -754,11 +844,15 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const uint64_t dk = p.k_mn_major ? make_desc(sK, D * 128u, 1024) : make_desc(sK, 16, 1024);
       const uint64_t dv = p.v_k_major ? make_desc(sV, 16, 1024) : make_desc(sV, 16384, 1024);
       auto km_off = [](int kk) { return uint64_t(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4); };   // K-major operand, 64-wide chunks
-      const int last_t = n_kv[1] ? 1 : 0;    // the tile whose MMA is the last reader of a K / V stage (n_kv[1] >= n_kv[0] when tile 1 exists)
       const uint32_t tm = __shfl_sync(0xffffffffu, tmem_base, 0);
+      Item w;
+      int kc0 = 0;              // key / value tiles of the items before this one
+      int sc[2] = {0, 0};       // score tiles of slot t before this item (= softmax passes = P.V products)
+      int oc[2] = {0, 0};       // items before this one in which slot t was active
+      int last_t = 0, qk_left = 0;
       auto issue_qk = [&](int t, int j) -> bool {   // S_t = Q_t.K_j^T
-        const int st = j & 1;
-        if (!mbar_wait_warp(k_full + 8u * st, uint32_t(j >> 1) & 1u)) { fail |= 0x20u; return false; }
+        const int kc = kc0 + j, st = kc & 1;
+        if (!mbar_wait_warp(k_full + 8u * st, uint32_t(kc >> 1) & 1u)) { fail |= 0x20u; return false; }
         tc_fence_after();
         const uint64_t kb = dk + uint64_t(st) * (kTile >> 4), qb = dq + uint64_t(t) * (kTile >> 4);
 #pragma unroll
@@ -766,34 +860,51 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           umma_ss_elect(tm + uint32_t(t * TK), qb + km_off(kk), kb + (p.k_mn_major ? uint64_t(kk * 128) : km_off(kk)), idesc_s,
                         kk > 0 ? 1u : 0u, leader);
         umma_commit_elect(s_full + 8u * t, leader);
-        if (t == last_t || j >= n_kv[1]) umma_commit_elect(k_free + 8u * st, leader);
+        if (t == last_t || j >= w.n_kv[1]) umma_commit_elect(k_free + 8u * st, leader);
+        if (--qk_left == 0) umma_commit_elect(q_free, leader);   // the item's query tiles have been read for the last time
         return true;
       };
       auto issue_pv = [&](int t, int j) -> bool {   // O_t += P_t.V_j
-        const int st = j & 1;
-        if (!mbar_wait_warp(p_full + 8u * t, uint32_t(j) & 1u)) { fail |= 0x200u; return false; }
-        if (!mbar_wait_warp(v_full + 8u * st, uint32_t(j >> 1) & 1u)) { fail |= 0x20u; return false; }
+        const int kc = kc0 + j, st = kc & 1;
+        // the first product of an item overwrites O_t: the previous item's output must have been read out of it
+        if (j == 0 && oc[t] > 0 && !mbar_wait_warp(o_free + 8u * t, uint32_t(oc[t] - 1) & 1u)) { fail |= 0x400u; return false; }
+        if (!mbar_wait_warp(p_full + 8u * t, uint32_t(sc[t] + j) & 1u)) { fail |= 0x200u; return false; }
+        if (!mbar_wait_warp(v_full + 8u * st, uint32_t(kc >> 1) & 1u)) { fail |= 0x20u; return false; }
         tc_fence_after();
         const uint64_t vb = dv + uint64_t(st) * (kTile >> 4);
         const uint32_t tP = tm + uint32_t(t * TK), tO = tm + 2 * TK + uint32_t(t * D);
 #pragma unroll
-        for (int kk = 0; kk < TK / 16; ++kk)   // 16 keys = 8 packed columns of P per instruction (TPR = 2: each half row's P lies over its own 64 score columns)
-          umma_ts_elect(tO, tP + (TPR == 2 ? uint32_t((kk >> 2) * 64 + (kk & 3) * 8) : uint32_t(kk * 8)),
+        for (int kk = 0; kk < TK / 16; ++kk)   // 16 keys = 8 packed columns of P per instruction
+          umma_ts_elect(tO, tP + uint32_t(kk * 8),
                         vb + (p.v_k_major ? uint64_t(((kk >> 2) * (D * 128) + (kk & 3) * 32) >> 4) : uint64_t(kk * 128)), idesc_o,
                         (j > 0 || kk > 0) ? 1u : 0u, leader);
         umma_commit_elect(o_done + 8u * t, leader);
-        if (t == last_t || j >= n_kv[1]) umma_commit_elect(v_free + 8u * st, leader);
+        if (t == last_t || j >= w.n_kv[1]) umma_commit_elect(v_free + 8u * st, leader);
         return true;
       };
-      bool ok = mbar_wait_warp(q_full, 0);
-      if (!ok) fail |= 0x10u;
-      for (int t = 0; ok && t < 2; ++t)
-        if (n_kv[t] > 0) ok = issue_qk(t, 0);
-      for (int j = 0; ok && j < n_max; ++j) {
-        for (int t = 0; ok && t < 2; ++t) {
-          if (j >= n_kv[t]) continue;
-          ok = issue_pv(t, j);
-          if (ok && j + 1 < n_kv[t]) ok = issue_qk(t, j + 1);   // into the S tile whose probabilities were just consumed
+      bool ok = true;
+      for (int r = 0; ok; ++r) {
+        const int it = item_of(r);
+        if (it < 0) break;
+        decode(it, w);
+        last_t = w.n_kv[1] ? 1 : 0;    // the tile whose MMA is the last reader of a K / V stage (n_kv[1] >= n_kv[0] when tile 1 exists)
+        qk_left = w.n_kv[0] + w.n_kv[1];
+        ok = mbar_wait_warp(q_full, uint32_t(r) & 1u);
+        if (!ok) fail |= 0x10u;
+        for (int t = 0; ok && t < 2; ++t)
+          if (w.n_kv[t] > 0) ok = issue_qk(t, 0);
+        for (int j = 0; ok && j < w.n_max; ++j) {
+          for (int t = 0; ok && t < 2; ++t) {
+            if (j >= w.n_kv[t]) continue;
+            ok = issue_pv(t, j);
+            if (ok && j + 1 < w.n_kv[t]) ok = issue_qk(t, j + 1);   // into the S tile whose probabilities were just consumed
+          }
+        }
+        kc0 += w.n_max;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          sc[t] += w.n_kv[t];
+          oc[t] += w.n_kv[t] > 0 ? 1 : 0;
         }
       }
       if (!ok && leader) {
@@ -801,87 +912,73 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         atomicOr(p.status, 0x100u | fail);
       }
     }
-  } else if (TPR == 2) {
-    // ======================= softmax, two threads per query row: warps 0-7 query tile 0, warps 8-15 tile 1 ===========
-    // Thread (row, half) owns score columns 64 half .. 64 half + 63 of its row and writes its probabilities over the
-    // first 32 of them, so the two threads of a row never touch each other's columns. Twice the warps per scheduler
-    // of the one-thread-per-row form: a lone softmax warp issues at about half the rate two reach together.
-    // Measured: no faster than one thread per row. Stamps in the MMA warp show why: it waits ~100 cycles per round for
-    // the probabilities and spends the rest issuing; a 128 x 128 x 16 instruction takes ~100-120 cycles here against
-    // the 64 the tensor core needs (8 KB of shared-memory operands per instruction is the whole shared-memory
-    // bandwidth of an SM at 64 cycles), so the tensor side sets the pace in either form, not the softmax.
-    // The reference point m_used of a row is the same in both threads. A pass first asks, through one reducing
-    // barrier over the tile's 256 threads, whether any half row's maximum has moved more than 2^8 above it; only
-    // then (and on the first key tile) do the halves exchange their maxima and rescale O. Every thread takes every
-    // barrier, also after a failed wait (it then only skips the work), so no barrier is left waiting.
-    const int t = warp >> 3, wq = warp & 3, half = (warp >> 2) & 1;
-    const int row = wq * 32 + lane;
-    const int qi = m0 + t * TQ + row;
-    const uint32_t lane_addr = uint32_t(wq * 32) << 16;
-    const uint32_t tS = tmem_base + lane_addr + uint32_t(t * TK + half * 64);
-    const uint32_t tO = tmem_base + lane_addr + 2 * TK + uint32_t(t * D + half * (D / 2));
-    float* xm = xch + t * 512;           // [parity][half][128]
-    float* xl = xch + 1024 + t * 256;    // [half][128]
-    const int n = n_kv[t];
-    float m_used = -INFINITY, l_run = 0.f;
+  } else {
+    // ======================= softmax: warps 0-3 query tile 0, warps 4-7 query tile 1 =======================
+    const int t = warp >> 2, row = threadIdx.x & 127;
+    const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem_base + lane_addr + uint32_t(t * TK);
+    const uint32_t tO = tmem_base + lane_addr + 2 * TK + uint32_t(t * D);
     bool ok = true;
     uint32_t fail = 0;
-    int slow = 0;
-    auto tile_sync = [&]() {
-      if (t == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
-      else asm volatile("bar.sync 2, 256;" ::: "memory");
-    };
-    auto tile_any = [&](bool mine) -> bool {
-      uint32_t r;
-      if (t == 0)
-        asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.or.pred p, 1, 256, q;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(r) : "r"(mine ? 1u : 0u) : "memory");
-      else
-        asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.or.pred p, 2, 256, q;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(r) : "r"(mine ? 1u : 0u) : "memory");
-      return r != 0;
-    };
-    for (int j = 0; j < n; ++j) {
-      if (ok && !mbar_wait_warp(s_full + 8u * t, uint32_t(j) & 1u)) { ok = false; fail |= 0x40u; }
-      const int kv0 = j * TK + half * 64;
-      tc_fence_after();
-      const int kv_lim = (p.causal ? min(p.S, qi + 1) : p.S) - kv0;   // this thread's local columns >= kv_lim are masked
-      const bool full = __all_sync(0xffffffffu, kv_lim >= 64);
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      if (ok) {
-        uint32_t q[2][32];
-        tmem_ld32(tS, q[0]);
-        tmem_ld32(tS + 32, q[1]);
-        tmem_ld_wait();
+    int sc = 0;   // score tiles of this slot before the current item
+    // (Making the two softmax groups take turns through a pair of named barriers, so that they never share the
+    // schedulers, was measured and is slower: 918 -> 876 TFLOP/s on 2 x 4096 x 32 x 128. A pass is bound by what one
+    // warp can issue alone, so two groups running together get more out of a scheduler than one at a time. Two threads
+    // per row (twice the warps) was measured no faster either, 940 vs 958 TFLOP/s: the tensor side sets the pace.)
+    for (int r = 0; ok; ++r) {
+      const int it = item_of(r);
+      if (it < 0) break;
+      Item w;
+      decode(it, w);
+      const int n = w.n_kv[t];
+      const int qi = w.m0 + t * TQ + row;
+      float m_used = -INFINITY, l_run = 0.f;
+      for (int j = 0; j < n; ++j) {
+        if (!mbar_wait_warp(s_full + 8u * t, uint32_t(sc + j) & 1u)) { ok = false; fail |= 0x40u; break; }
+        const int kv0 = j * TK;
+        tc_fence_after();
+        // Two passes over the row of S, 32 columns at a time, so that a thread holds 64 scores at most (with all 128 in
+        // registers the kernel spills at the 168 registers ten warps leave a thread). Pass 1: the row maximum.
+        const int kv_lim = (p.causal ? min(p.S, qi + 1) : p.S) - kv0;   // local columns >= kv_lim are masked
+        // one answer per warp: both branches of pass 2 issue warp-collective tensor-memory stores (on the diagonal
+        // tile the last row of a warp sees every column while the other rows do not)
+        const bool full = __all_sync(0xffffffffu, kv_lim >= TK);
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        {
+          uint32_t q[2][32];
+          tmem_ld32(tS, q[0]);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          if (full) {
+          for (int c = 0; c < TK / 32; ++c) {
+            tmem_ld_wait();
+            if (c + 1 < TK / 32) tmem_ld32(tS + (c + 1) * 32, q[(c + 1) & 1]);
+            if (full) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 8)
+              for (int i = 0; i < 32; i += 8)
 #pragma unroll
-              for (int u = 0; u < 4; ++u)
-                mx4[u] = max3(mx4[u], __uint_as_float(q[c][i + 2 * u]), __uint_as_float(q[c][i + 2 * u + 1]));
-          } else {
+                for (int u = 0; u < 4; ++u)
+                  mx4[u] = max3(mx4[u], __uint_as_float(q[c & 1][i + 2 * u]), __uint_as_float(q[c & 1][i + 2 * u + 1]));
+            } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c * 32 + i < kv_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(q[c][i]));
+              for (int i = 0; i < 32; ++i)
+                if (c * 32 + i < kv_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(q[c & 1][i]));
+            }
           }
         }
-      }
-      const float m_half = ceilf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2);
-      if (tile_any(ok && (j == 0 || m_half > m_used + 8.f))) {
-        float* x = xm + (slow & 1) * 256;
-        ++slow;
-        x[half * 128 + row] = ok ? m_half : -INFINITY;
-        tile_sync();
-        const float m_row = fmaxf(x[row], x[128 + row]);
-        const float m_new = (j == 0 || m_row > m_used + 8.f) ? m_row : m_used;
-        if (j > 0) {
-          // P_{j-1}.V_{j-1} must have landed in O before it is rescaled
-          if (ok && !mbar_wait_warp(o_done + 8u * t, uint32_t(j - 1) & 1u)) { ok = false; fail |= 0x80u; }
-          const float alpha = exp2f(m_used - m_new);
-          if (ok) {
+        // whole-number reference point (base-2 domain): P's bf16 rounding is then that of 2^t itself and the rescale
+        // factors are exact powers of two
+        const float m_tile = ceilf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2);
+        if (j == 0) {
+          m_used = m_tile;
+        } else {
+          const bool need = m_tile > m_used + 8.f;
+          if (__any_sync(0xffffffffu, need)) {
+            // P_{j-1}.V_{j-1} must have landed in O before it is rescaled
+            if (!mbar_wait_warp(o_done + 8u * t, uint32_t(sc + j - 1) & 1u)) { ok = false; fail |= 0x80u; break; }
             tc_fence_after();
+            const float m_new = need ? m_tile : m_used;
+            const float alpha = exp2f(m_used - m_new);
 #pragma unroll 1
-            for (int c0 = 0; c0 < D / 2; c0 += 32) {
+            for (int c0 = 0; c0 < D; c0 += 32) {
               uint32_t q[32];
               tmem_ld32(tO + c0, q);
               tmem_ld_wait();
@@ -889,214 +986,80 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               for (int i = 0; i < 32; ++i) q[i] = __float_as_uint(__uint_as_float(q[i]) * alpha);
               tmem_st32(tO + c0, q);
             }
+            l_run *= alpha;
+            m_used = m_new;
           }
-          l_run *= alpha;
         }
-        m_used = m_new;
-      }
-      if (ok) {
-        // P = exp2(s * k - m_used) as bf16 pairs over the first 32 of this thread's 64 score columns
+        // Pass 2: P = exp2(s * k - m_used) as bf16 pairs over S's first 64 columns. Chunk c (columns 32c..32c+31) is
+        // read before P chunk c (packed columns 16c..16c+15) is written, and the chunk read ahead lies above both.
+        float ps4[4] = {0.f, 0.f, 0.f, 0.f};
         const float neg_m = -m_used;
-        const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(neg_m, neg_m);
-        uint64_t acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
-        uint32_t q[2][32];
-        tmem_ld32(tS, q[0]);
-        tmem_ld32(tS + 32, q[1]);
-        tmem_ld_wait();
+        {
+          const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(neg_m, neg_m);
+          uint64_t acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+          uint32_t q[2][32];
+          tmem_ld32(tS, q[0]);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t w[16];
+          for (int c = 0; c < TK / 32; ++c) {
+            tmem_ld_wait();
+            if (c + 1 < TK / 32) tmem_ld32(tS + (c + 1) * 32, q[(c + 1) & 1]);
+            uint32_t wv[16];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float x0, x1;
-            unpack2(fma2(pack2(__uint_as_float(q[c][2 * i]), __uint_as_float(q[c][2 * i + 1])), sc2, nm2), x0, x1);
-            float a = ex2_fast(x0), bb = ex2_fast(x1);
-            if (!full) {
-              if (c * 32 + 2 * i >= kv_lim) a = 0.f;
-              if (c * 32 + 2 * i + 1 >= kv_lim) bb = 0.f;
+            for (int i = 0; i < 16; ++i) {
+              float x0, x1;
+              unpack2(fma2(pack2(__uint_as_float(q[c & 1][2 * i]), __uint_as_float(q[c & 1][2 * i + 1])), sc2, nm2), x0, x1);
+              float a, bb;
+              if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) { a = ex2_poly(x0); bb = ex2_poly(x1); }
+              else { a = ex2_fast(x0); bb = ex2_fast(x1); }
+              if (!full) {
+                if (c * 32 + 2 * i >= kv_lim) a = 0.f;
+                if (c * 32 + 2 * i + 1 >= kv_lim) bb = 0.f;
+              }
+              wv[i] = pack_bf16x2(a, bb);
+              acc[i & 1] = add2(acc[i & 1], pack2(a, bb));   // fp32 sum of the unrounded exponentials
             }
-            w[i] = pack_bf16x2(a, bb);
-            acc[i & 1] = add2(acc[i & 1], pack2(a, bb));   // fp32 sum of the unrounded exponentials
+            tmem_st16(tS + c * 16, wv);
           }
-          tmem_st16(tS + c * 16, w);
+          unpack2(acc[0], ps4[0], ps4[1]);
+          unpack2(acc[1], ps4[2], ps4[3]);
         }
-        float s0, s1, s2, s3;
-        unpack2(acc[0], s0, s1);
-        unpack2(acc[1], s2, s3);
-        l_run += (s0 + s1) + (s2 + s3);
+        l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         tc_fence_before();
         mbar_arrive(p_full + 8u * t);
       }
-    }
-    // ---- O / l -> bf16: each thread its half of the head dim ----
-    if (ok && n > 0) {
-      if (!mbar_wait_warp(o_done + 8u * t, uint32_t(n - 1) & 1u)) { ok = false; fail |= 0x80u; }
-      tc_fence_after();
-    }
-    if (fail && lane == 0) atomicOr(p.status, 0x100u | fail);
-    if (!ok) *abort_flag = 1;
-    xl[half * 128 + row] = l_run;
-    tile_sync();
-    if (ok && n > 0 && !*abort_flag) {
-      const float l_tot = xl[row] + xl[128 + row];
-      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.O) + (int64_t)b * p.o_s[0] + (int64_t)h * p.o_s[1] + (int64_t)qi * p.o_s[2] +
-                           half * (D / 2);
-      pdl_wait();  // O may still be read by an earlier step
+      if (!ok) break;
+      // ---- O / l -> bf16 ----
+      if (n > 0) {
+        if (!mbar_wait_warp(o_done + 8u * t, uint32_t(sc + n - 1) & 1u)) { ok = false; fail |= 0x80u; break; }
+        tc_fence_after();
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+        const int h = w.bz % p.NH, b = w.bz / p.NH;
+        __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.O) + (int64_t)b * p.o_s[0] + (int64_t)h * p.o_s[1] + (int64_t)qi * p.o_s[2];
+        pdl_wait();  // O may still be read by an earlier step
 #pragma unroll 1
-      for (int c0 = 0; c0 < D / 2; c0 += 32) {
-        uint32_t q[32];
-        tmem_ld32(tO + c0, q);     // warp-collective: rows past the end take part, then skip the store
-        tmem_ld_wait();
-        if (qi < p.S) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            float v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(q[g * 8 + i]) * inv;
-            store16(out + c0 + g * 8, v);
-          }
-        }
-      }
-    }
-  } else {
-    // ======================= softmax: warps 0-3 query tile 0, warps 4-7 query tile 1 =======================
-    const int t = warp >> 2, row = threadIdx.x & 127;
-    const int qi = m0 + t * TQ + row;
-    const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem_base + lane_addr + uint32_t(t * TK);
-    const uint32_t tO = tmem_base + lane_addr + 2 * TK + uint32_t(t * D);
-    const int n = n_kv[t];
-    float m_used = -INFINITY, l_run = 0.f;
-    bool ok = true;
-    uint32_t fail = 0;
-    // (Making the two softmax groups take turns through a pair of named barriers, so that they never share the
-    // schedulers, was measured and is slower: 918 -> 876 TFLOP/s on 2 x 4096 x 32 x 128. A pass is bound by what one
-    // warp can issue alone, so two groups running together get more out of a scheduler than one at a time.)
-    for (int j = 0; j < n; ++j) {
-      if (!mbar_wait_warp(s_full + 8u * t, uint32_t(j) & 1u)) { ok = false; fail |= 0x40u; break; }
-      const int kv0 = j * TK;
-      tc_fence_after();
-      // Two passes over the row of S, 32 columns at a time, so that a thread holds 64 scores at most (with all 128 in
-      // registers the kernel spills at the 168 registers ten warps leave a thread). Pass 1: the row maximum.
-      const int kv_lim = (p.causal ? min(p.S, qi + 1) : p.S) - kv0;   // local columns >= kv_lim are masked
-      // one answer per warp: both branches of pass 2 issue warp-collective tensor-memory stores (on the diagonal
-      // tile the last row of a warp sees every column while the other rows do not)
-      const bool full = __all_sync(0xffffffffu, kv_lim >= TK);
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      {
-        uint32_t q[2][32];
-        tmem_ld32(tS, q[0]);
-#pragma unroll
-        for (int c = 0; c < TK / 32; ++c) {
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          uint32_t q[32];
+          tmem_ld32(tO + c0, q);     // warp-collective: rows past the end take part, then skip the store
           tmem_ld_wait();
-          if (c + 1 < TK / 32) tmem_ld32(tS + (c + 1) * 32, q[(c + 1) & 1]);
-          if (full) {
+          if (qi < p.S) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 8)
+            for (int g = 0; g < 4; ++g) {
+              float v[8];
 #pragma unroll
-              for (int u = 0; u < 4; ++u)
-                mx4[u] = max3(mx4[u], __uint_as_float(q[c & 1][i + 2 * u]), __uint_as_float(q[c & 1][i + 2 * u + 1]));
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c * 32 + i < kv_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(q[c & 1][i]));
-          }
-        }
-      }
-      // whole-number reference point (base-2 domain): P's bf16 rounding is then that of 2^t itself and the rescale
-      // factors are exact powers of two
-      const float m_tile = ceilf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2);
-      if (j == 0) {
-        m_used = m_tile;
-      } else {
-        const bool need = m_tile > m_used + 8.f;
-        if (__any_sync(0xffffffffu, need)) {
-          // P_{j-1}.V_{j-1} must have landed in O before it is rescaled
-          if (!mbar_wait_warp(o_done + 8u * t, uint32_t(j - 1) & 1u)) { ok = false; fail |= 0x80u; break; }
-          tc_fence_after();
-          const float m_new = need ? m_tile : m_used;
-          const float alpha = exp2f(m_used - m_new);
-#pragma unroll 1
-          for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t q[32];
-            tmem_ld32(tO + c0, q);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) q[i] = __float_as_uint(__uint_as_float(q[i]) * alpha);
-            tmem_st32(tO + c0, q);
-          }
-          l_run *= alpha;
-          m_used = m_new;
-        }
-      }
-      // ---- P = exp2(s * k - m_used) as bf16 pairs, written over S's first 64 columns ----
-      // Pass 2: P = exp2(s * k - m_used) as bf16 pairs over S's first 64 columns. Chunk c (columns 32c..32c+31) is
-      // read before P chunk c (packed columns 16c..16c+15) is written, and the chunk read ahead lies above both.
-      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
-      const float neg_m = -m_used;
-      {
-        const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(neg_m, neg_m);
-        uint64_t acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
-        uint32_t q[2][32];
-        tmem_ld32(tS, q[0]);
-#pragma unroll
-        for (int c = 0; c < TK / 32; ++c) {
-          tmem_ld_wait();
-          if (c + 1 < TK / 32) tmem_ld32(tS + (c + 1) * 32, q[(c + 1) & 1]);
-          uint32_t w[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float x0, x1;
-            unpack2(fma2(pack2(__uint_as_float(q[c & 1][2 * i]), __uint_as_float(q[c & 1][2 * i + 1])), sc2, nm2), x0, x1);
-            float a, bb;
-            if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) { a = ex2_poly(x0); bb = ex2_poly(x1); }
-            else { a = ex2_fast(x0); bb = ex2_fast(x1); }
-            if (!full) {
-              if (c * 32 + 2 * i >= kv_lim) a = 0.f;
-              if (c * 32 + 2 * i + 1 >= kv_lim) bb = 0.f;
+              for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(q[g * 8 + i]) * inv;
+              store16(out + c0 + g * 8, v);
             }
-            w[i] = pack_bf16x2(a, bb);
-            acc[i & 1] = add2(acc[i & 1], pack2(a, bb));   // fp32 sum of the unrounded exponentials
           }
-          tmem_st16(tS + c * 16, w);
         }
-        unpack2(acc[0], ps4[0], ps4[1]);
-        unpack2(acc[1], ps4[2], ps4[3]);
+        // O_t has been read out: the next item's first P.V may overwrite it
+        tc_fence_before();
+        mbar_arrive(o_free + 8u * t);
       }
-      l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
-      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-      tc_fence_before();
-      mbar_arrive(p_full + 8u * t);
-    }
-    // ---- O / l -> bf16 ----
-    if (ok && n > 0) {
-      if (!mbar_wait_warp(o_done + 8u * t, uint32_t(n - 1) & 1u)) { ok = false; fail |= 0x80u; }
-      tc_fence_after();
+      sc += n;
     }
     if (fail && lane == 0) atomicOr(p.status, 0x100u | fail);
     if (!ok) *abort_flag = 1;
-    if (ok && n > 0) {
-      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.O) + (int64_t)b * p.o_s[0] + (int64_t)h * p.o_s[1] + (int64_t)qi * p.o_s[2];
-      pdl_wait();  // O may still be read by an earlier step
-#pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
-        uint32_t q[32];
-        tmem_ld32(tO + c0, q);     // warp-collective: rows past the end take part, then skip the store
-        tmem_ld_wait();
-        if (qi < p.S) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            float v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(q[g * 8 + i]) * inv;
-            store16(out + c0 + g * 8, v);
-          }
-        }
-      }
-    }
   }
   tc_fence_before();
   __syncthreads();
@@ -1108,16 +1071,28 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
 }  // namespace
 
-// Which form runs: two query tiles per CTA (probabilities in tensor memory) when the sequence has more than one query
-// tile (one thread per query row), else the one-tile form. FLUID_ATTN_FORM in the environment forces a form (A/B timing):
-// 1 one tile per CTA, 2 two tiles with one thread per row, 3 two tiles with two threads per row.
+// Which form runs: two query tiles per work item on persistent CTAs (probabilities in tensor memory) when the sequence
+// has more than one query tile, else the one-tile form. FLUID_ATTN_FORM in the environment forces a form (A/B timing):
+// 1 one tile per CTA, 2 the persistent two-tile form. FLUID_ATTN_CTAS caps the persistent form's grid (default: one CTA
+// per SM).
 static int attn_form(const AttnParams& p) {
   static const int forced = [] {
     const char* e = std::getenv("FLUID_ATTN_FORM");
     return e ? std::atoi(e) : 0;
   }();
-  if (forced >= 1 && forced <= 3) return forced;
+  if (forced >= 1 && forced <= 2) return forced;
   return p.S > TQ ? 2 : 1;
+}
+
+static int attn_ctas() {
+  static const int n = [] {
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const char* e = std::getenv("FLUID_ATTN_CTAS");
+    const int cap = e ? std::atoi(e) : 0;
+    return cap > 0 ? cap : sms;
+  }();
+  return n;
 }
 
 template <typename K>
@@ -1136,17 +1111,15 @@ cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream
   const CUtensorMap* mq = reinterpret_cast<const CUtensorMap*>(&host.map_q);
   const CUtensorMap* mk = reinterpret_cast<const CUtensorMap*>(&host.map_k);
   const CUtensorMap* mv = reinterpret_cast<const CUtensorMap*>(&host.map_v);
-  static bool attr[6] = {false, false, false, false, false, false};
+  static bool attr[4] = {false, false, false, false};
   if (D != 64 && D != 128) return cudaErrorInvalidValue;
   const int form = attn_form(p);
-  if (form >= 2) {
-    const size_t smem = size_t(6) * TQ * D * 2 + 256 + 6144 + 1024;
-    const dim3 grid(((p.S + 2 * TQ - 1) / (2 * TQ)) * p.B * p.NH);
-    if (form == 3)   // two threads per query row: measured no faster (940 vs 958 TFLOP/s on 2 x 4096 x 32 x 128); kept for A/B timing
-      return D == 64 ? launch_attn_form(attn_tc2_kernel<64, 2>, &attr[4], smem, grid, 576, stream, mq, mk, mv, p)
-                     : launch_attn_form(attn_tc2_kernel<128, 2>, &attr[5], smem, grid, 576, stream, mq, mk, mv, p);
-    return D == 64 ? launch_attn_form(attn_tc2_kernel<64, 1>, &attr[2], smem, grid, 320, stream, mq, mk, mv, p)
-                   : launch_attn_form(attn_tc2_kernel<128, 1>, &attr[3], smem, grid, 320, stream, mq, mk, mv, p);
+  if (form == 2) {
+    const size_t smem = size_t(6) * TQ * D * 2 + 256 + 1024;
+    const int items = ((p.S + 2 * TQ - 1) / (2 * TQ)) * p.B * p.NH;
+    const dim3 grid(std::min(items, attn_ctas()));
+    return D == 64 ? launch_attn_form(attn_tc2_kernel<64>, &attr[2], smem, grid, 320, stream, mq, mk, mv, p)
+                   : launch_attn_form(attn_tc2_kernel<128>, &attr[3], smem, grid, 320, stream, mq, mk, mv, p);
   }
   const size_t smem = size_t(5) * TQ * D * 2 + size_t(2) * TQ * TK * 2 + 128 + 2048;
   const dim3 grid(((p.S + TQ - 1) / TQ) * p.B * p.NH);
