@@ -227,6 +227,13 @@ __device__ __forceinline__ float act_t(float v) {
   if (ACT == ACT_GELU_TANH) return gelu_tanh(v);
   return v;
 }
+// the activation of two values (the erf GELU as packed instructions)
+template <int ACT>
+__device__ __forceinline__ void act2_t(float& a, float& b) {
+  if (ACT == ACT_GELU_ERF) { gelu_erf_fast2(a, b); return; }
+  a = act_t<ACT>(a);
+  b = act_t<ACT>(b);
+}
 
 __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
@@ -307,7 +314,7 @@ __device__ __forceinline__ void epilogue_chunk_vec(const GemmParams& g, uint32_t
       }
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) v[j] = act_t<ACT>(v[j]);
+    for (int j = 0; j < 8; j += 2) act2_t<ACT>(v[j], v[j + 1]);
     if (HAS_RES) {
       if (R_WIDE) {
         const uint4 a = rq[2 * q], b = rq[2 * q + 1];
@@ -404,8 +411,9 @@ __device__ __forceinline__ void epilogue_chunk_coal(const GemmParams& g, uint32_
     const int row = rsub + 4 * i;
     float4 v = *reinterpret_cast<const float4*>(stage + row * 32 + ((unit ^ (row & 7)) << 2));
     if (!col_ok || !((ok_mask >> i) & 1u)) continue;
-    v.x = act_t<ACT>(v.x + bias4[0]); v.y = act_t<ACT>(v.y + bias4[1]);
-    v.z = act_t<ACT>(v.z + bias4[2]); v.w = act_t<ACT>(v.w + bias4[3]);
+    v.x += bias4[0]; v.y += bias4[1]; v.z += bias4[2]; v.w += bias4[3];
+    act2_t<ACT>(v.x, v.y);
+    act2_t<ACT>(v.z, v.w);
     if (HAS_RES) { v.x += res[i].x; v.y += res[i].y; v.z += res[i].z; v.w += res[i].w; }
     if (C_WIDE) {
       *reinterpret_cast<float4*>(static_cast<float*>(g.C) + cbs[i] + c_col) = v;
@@ -499,8 +507,9 @@ __device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       float4& v = v8[i];
-      v.x = act_t<ACT>(v.x + bias_cur[0]); v.y = act_t<ACT>(v.y + bias_cur[1]);
-      v.z = act_t<ACT>(v.z + bias_cur[2]); v.w = act_t<ACT>(v.w + bias_cur[3]);
+      v.x += bias_cur[0]; v.y += bias_cur[1]; v.z += bias_cur[2]; v.w += bias_cur[3];
+      act2_t<ACT>(v.x, v.y);
+      act2_t<ACT>(v.z, v.w);
       if (HAS_RES) { v.x += res[i].x; v.y += res[i].y; v.z += res[i].z; v.w += res[i].w; }
     }
     const uint32_t live = col_ok ? ok_mask : 0u;
@@ -522,6 +531,80 @@ __device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t
       for (int q = 0; q < 4; ++q) bias_cur[q] = bias_nxt[q];
       c_col = c_col_nxt; col_ok = col_ok_nxt;
     }
+  }
+}
+
+// bf16 output without a residual, 64 columns at a time. A thread finishes its own row first (scale, bias, activation,
+// rounding), so the staging tile holds 32 rows of 64 bf16 (128 bytes a row, 16-byte units swizzled by the row) and a
+// row leaves as ONE 128-byte run (eight lanes x 16 bytes) where the 32-column form above writes two separate 64-byte
+// pieces. At the end of a launch every SM stores its last tile at the same moment, and it is the number of write
+// requests that reach L2, not their bytes, that sets how long this takes (clock stamps in the 32-column form: ~1200
+// cycles a chunk whatever was taken out of it, 13 bytes per cycle and SM for 64-byte pieces against 27 for the
+// 128-byte runs of the fp32 outputs). Same arithmetic, in the same order, as the 32-column form.
+template <int ACT>
+__device__ __forceinline__ void epilogue_tile_coal16(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
+                                                     const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane) {
+  const int unit = lane & 7, rsub = lane >> 3;
+  const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
+  const float scale = g.scale;
+  __nv_bfloat16* const c_b16 = static_cast<__nv_bfloat16*>(g.C);
+  const __nv_bfloat16* const bias = static_cast<const __nv_bfloat16*>(g.bias);
+  const int n_chunks = (min(col_end, g.N - n_tile0) - col_begin + 63) >> 6;   // uniform across the warp
+  if (n_chunks <= 0) return;
+  uint32_t r[32];
+  tmem_ld32(trow + uint32_t(col_begin), r);
+#pragma unroll 1
+  for (int ci = 0; ci < n_chunks; ++ci) {
+    const int c0 = col_begin + 64 * ci;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      // bias of these 32 columns, the same for every row of the warp: four 16-byte loads that every lane shares
+      uint4 b4[4];
+      const int nb = n_tile0 + c0 + 32 * h;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        b4[k] = (g.has_bias && nb + 8 * k < g.N) ? __ldg(reinterpret_cast<const uint4*>(bias + nb + 8 * k)) : make_uint4(0u, 0u, 0u, 0u);
+      tmem_ld_wait();
+      float v[32];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint32_t w[4] = {b4[k].x, b4[k].y, b4[k].z, b4[k].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          v[8 * k + 2 * q] = __uint_as_float(r[8 * k + 2 * q]) * scale + __uint_as_float(w[q] << 16);
+          v[8 * k + 2 * q + 1] = __uint_as_float(r[8 * k + 2 * q + 1]) * scale + __uint_as_float(w[q] & 0xffff0000u);
+        }
+      }
+      // the next 32 columns are on their way while these are finished (the accumulator is 64 ci + 64 columns wide at least)
+      if (h == 0 || ci + 1 < n_chunks) tmem_ld32(trow + uint32_t(c0 + 32 * (h + 1)), r);
+#pragma unroll
+      for (int k = 0; k < 16; ++k) act2_t<ACT>(v[2 * k], v[2 * k + 1]);
+#pragma unroll
+      for (int k = 0; k < 4; ++k)   // unit 4 h + k of row `lane` lives at unit (4 h + k) ^ (lane & 7)
+        sts128(st_row + (uint32_t((4 * h + k) ^ (lane & 7)) << 4), __uint_as_float(pack_bf16x2(v[8 * k], v[8 * k + 1])),
+               __uint_as_float(pack_bf16x2(v[8 * k + 2], v[8 * k + 3])), __uint_as_float(pack_bf16x2(v[8 * k + 4], v[8 * k + 5])),
+               __uint_as_float(pack_bf16x2(v[8 * k + 6], v[8 * k + 7])));
+    }
+    __syncwarp();
+    // lane (rsub, unit): rows rsub + 4 i, columns 8 unit .. 8 unit + 7 of the chunk
+    const int nc = n_tile0 + c0 + unit * 8;
+    int n1, n0i;
+    split2(nc, g.N0, n1, n0i);
+    const int64_t c_col = (int64_t)n1 * g.c_s[4] + n0i;
+    const uint32_t live = nc < g.N ? ok_mask : 0u;
+    float4 v8[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = rsub + 4 * i;
+      v8[i] = lds128(st_base + uint32_t(row * 128) + (uint32_t(unit ^ (row & 7)) << 4));
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint4* dst = reinterpret_cast<uint4*>(c_b16 + cbs[i] + c_col);
+      if ((live >> i) & 1u)
+        *dst = make_uint4(__float_as_uint(v8[i].x), __float_as_uint(v8[i].y), __float_as_uint(v8[i].z), __float_as_uint(v8[i].w));
+    }
+    __syncwarp();   // the staging tile is rewritten by the next chunk
   }
 }
 
@@ -617,7 +700,12 @@ template <int EPI>
 __device__ __forceinline__ void epilogue_tile_c(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
                                                 const int64_t (&cbs)[8], const int64_t (&rbs)[8], uint32_t ok_mask, float* stage,
                                                 int lane) {
-  if (EPI == EPI_PLAIN) epilogue_tile_coal<ACT_NONE, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+  // bf16 outputs without a residual leave in 128-byte runs when the warp's columns come in sixty-fours
+  const bool wide_runs = ((col_end - col_begin) & 63) == 0;
+  if (EPI == EPI_PLAIN && wide_runs) epilogue_tile_coal16<ACT_NONE>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
+  else if (EPI == EPI_GELU_ERF && wide_runs) epilogue_tile_coal16<ACT_GELU_ERF>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
+  else if (EPI == EPI_GELU_TANH && wide_runs) epilogue_tile_coal16<ACT_GELU_TANH>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
+  else if (EPI == EPI_PLAIN) epilogue_tile_coal<ACT_NONE, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
   else if (EPI == EPI_PLAIN_WIDE) epilogue_tile_coal<ACT_NONE, false, true, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
   else if (EPI == EPI_RES) epilogue_tile_coal<ACT_NONE, true, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
   else if (EPI == EPI_RES_WIDE) epilogue_tile_coal<ACT_NONE, true, true, true>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
@@ -992,7 +1080,8 @@ __device__ __forceinline__ void final_store4(const FinalCtx& f, float4 v, int64_
     v.x += __uint_as_float(b2.x << 16); v.y += __uint_as_float(b2.x & 0xffff0000u);
     v.z += __uint_as_float(b2.y << 16); v.w += __uint_as_float(b2.y & 0xffff0000u);
   }
-  v.x = act_t<ACT>(v.x); v.y = act_t<ACT>(v.y); v.z = act_t<ACT>(v.z); v.w = act_t<ACT>(v.w);
+  act2_t<ACT>(v.x, v.y);
+  act2_t<ACT>(v.z, v.w);
   if (HAS_RES) {
     const int64_t ro = rb + (int64_t)n1 * f.rs4 + n0i;
     if (R_WIDE) {
