@@ -768,7 +768,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     };
     auto all_ok = [&](bool mine) { return __shfl_sync(0xffffffffu, mine ? 1 : 0, 0) != 0; };   // lane 0 decides
 
-    pdl_wait();  // Q, K, V come from the previous steps
     bool ok = true;
     for (int r = 0; ok; ++r) {
       const int it = item_of(r);
@@ -776,6 +775,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       Item w;
       decode(it, w);
       start_head(w.bz);
+      if (r == 0) pdl_wait();  // Q, K, V come from the previous steps (the first item's coordinates above do not)
       if (r > 0) {   // the previous item's last Q.K^T has read the query tiles
         if (lead && !mbar_wait(q_free, uint32_t(r - 1) & 1u)) { fail |= 0x10u; ok = false; }
         ok = all_ok(ok && !*abort_flag);

@@ -812,21 +812,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // while the previous step is still finishing (its bytes may land before lane 0 posts the expected
       // count; the barrier's pending arrival keeps the phase open until then).
       const bool b_free = p.g.b_const && (p.n_group < 2 || p.gx[0].b_const) && (p.n_group < 3 || p.gx[1].b_const);
-      if (is_a || !b_free) pdl_wait();
-      for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
-        int tile, sp, k_begin, k_count;
+      // A tile's coordinates are index arithmetic only (divisions and selects, ~1 us on this one warp): the first tile's are
+      // ready before the wait for the previous step, every later tile's while its predecessor's loads are in flight
+      int c[5], ksteps = 0, k_begin = 0;
+      const CUtensorMap* map = &map_a;
+      auto prep = [&](int item) {
+        int tile, sp, k_count;
         decode_item<SPLIT>(p, item, tile, sp, k_begin, k_count);
         int grp, bz, mt, nt;
         decode_tile(p, tile, grp, bz, mt, nt);
-        const int ksteps = k_count >= 0 ? k_count : k_steps_of(p, mt);
-        int c[5];
-        {
-          int r1, r0, b1, b0;
-          split2((is_a ? mt * BM : nt * bn) + ch * box_rows, x_r0, r1, r0);
-          split2(bz, x_b0, b1, b0);
-          fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
-        }
-        const CUtensorMap* map = is_a ? &map_a : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2));
+        ksteps = k_count >= 0 ? k_count : k_steps_of(p, mt);
+        int r1, r0, b1, b0;
+        split2((is_a ? mt * BM : nt * bn) + ch * box_rows, x_r0, r1, r0);
+        split2(bz, x_b0, b1, b0);
+        fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
+        map = is_a ? &map_a : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2));
+      };
+      int item = blockIdx.x;
+      if (item < p.num_tiles) prep(item);
+      if (is_a || !b_free) pdl_wait();
+      for (; ok && item < p.num_tiles; item += gridDim.x, (item < p.num_tiles ? prep(item) : (void)0)) {
         if (k_simple) {
           const int kc = k_begin * BK;
           c[0] += i0 ? kc : 0; c[1] += i1 ? kc : 0; c[2] += i2 ? kc : 0;
@@ -922,7 +927,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     int acc = 0;
     uint32_t acc_ph = 0;
     bool ok = true;
-    pdl_wait();  // before any global read (bias, residual) or write (C)
+    bool waited = false;
     for (int item = blockIdx.x; ok && item < p.num_tiles; item += gridDim.x) {
       int tile, sp, k_begin, k_count;
       decode_item<SPLIT>(p, item, tile, sp, k_begin, k_count);
@@ -949,6 +954,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           rbs[i] = g.has_res ? rbz + (live ? split_off(mi, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
         }
       }
+      // the first tile's row and column offsets above are index arithmetic: done before the wait
+      if (!waited) { pdl_wait(); waited = true; }   // before any global read (bias, residual) or write (C)
       bool got = mbar_wait_warp(tfull_bar(acc), acc_ph);
       if (SPLIT) {
         // the eight epilogue warps meet at named barriers below: either all of them go on or none does
@@ -1575,20 +1582,26 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       uint32_t fb = map_to_rank(full_bar(0), 0u);       // the full barriers of CTA 0 collect both CTAs' bytes
       const uint32_t fb0 = fb;
       const bool b_free = p.g.b_const && (p.n_group < 2 || p.gx[0].b_const) && (p.n_group < 3 || p.gx[1].b_const);
-      if (is_a || !b_free) pdl_wait();   // weights do not wait for the previous step
-      for (int item = pair_id; ok && item < p.num_tiles; item += n_pairs) {
+      // A tile's coordinates are index arithmetic only (five divisions and the selects: ~1 us on this one warp), so the
+      // first tile's are ready before the wait for the previous step and every later tile's while its predecessor's
+      // loads are still in flight
+      int c[5], ksteps = 0;
+      const CUtensorMap* map = &map_a;
+      auto prep = [&](int item) {
         int grp, bz, pm, nt;
         decode_tile(p, item, grp, bz, pm, nt);        // p.tiles_m counts pairs of row tiles here
         const int mt = 2 * pm + int(rank);
-        const int ksteps = k_steps_of(p, mt);
-        int c[5];
-        {
-          int r1, r0, b1, b0;
-          split2((is_a ? mt * BM : (p.swiglu ? nt * 128 : nt * PN + int(rank) * 128)) + ch * box_rows, x_r0, r1, r0);
-          split2(bz, x_b0, b1, b0);
-          fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
-        }
-        const CUtensorMap* map = is_a ? &map_a : (p.swiglu ? (rank == 0 ? &map_b : &map_b1) : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2)));
+        ksteps = k_steps_of(p, mt);
+        int r1, r0, b1, b0;
+        split2((is_a ? mt * BM : (p.swiglu ? nt * 128 : nt * PN + int(rank) * 128)) + ch * box_rows, x_r0, r1, r0);
+        split2(bz, x_b0, b1, b0);
+        fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
+        map = is_a ? &map_a : (p.swiglu ? (rank == 0 ? &map_b : &map_b1) : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2)));
+      };
+      int item = pair_id;
+      if (item < p.num_tiles) prep(item);
+      if (is_a || !b_free) pdl_wait();   // weights do not wait for the previous step
+      for (; ok && item < p.num_tiles; item += n_pairs, (item < p.num_tiles ? prep(item) : (void)0)) {
         int k0 = 0, k1 = 0;
         for (int ks = 0; ks < ksteps; ++ks) {
           if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
@@ -1663,7 +1676,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     int acc = 0;
     uint32_t acc_ph = 0;
     bool ok = true;
-    pdl_wait();  // before any global read (bias, residual) or write (C)
+    bool waited = false;
     for (int item = pair_id; ok && item < p.num_tiles; item += n_pairs) {
       int grp, bz, pm, nt;
       decode_tile(p, item, grp, bz, pm, nt);
@@ -1682,6 +1695,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         cbs[i] = cbz + (live ? split_off(mi, g.M0, g.c_s[2], g.c_s[3]) : 0);
         rbs[i] = g.has_res ? rbz + (live ? split_off(mi, g.M0, g.r_s[2], g.r_s[3]) : 0) : 0;
       }
+      // the first tile's row and column offsets above are index arithmetic (sixteen divisions): done before the wait
+      if (!waited) { pdl_wait(); waited = true; }   // before any global read (bias, residual) or write (C)
       if (!mbar_wait_warp(tfull_bar(acc), acc_ph)) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * PN);
