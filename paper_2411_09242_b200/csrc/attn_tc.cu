@@ -265,15 +265,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     };
     auto all_ok = [&](bool mine) { return __shfl_sync(0xffffffffu, mine ? 1 : 0, 0) != 0; };   // lane 0 decides; also re-converges the warp
 
+    // the Q boxes' coordinates are index arithmetic: ready before the wait for the previous step
+    int qc[2 * DC][5];
+    if (lead) {
+#pragma unroll
+      for (int dc = 0; dc < DC; ++dc)
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) coords(p.q_sel, dc * 64, m0 + rh * 64, bz, p.q_b0, qc[dc * 2 + rh]);
+    }
     pdl_wait();  // Q, K, V come from the previous steps
     if (lead) {
       mbar_expect_tx(bar_q, kTile);
-      int c[5];
+#pragma unroll
       for (int dc = 0; dc < DC; ++dc)
-        for (int rh = 0; rh < 2; ++rh) {
-          coords(p.q_sel, dc * 64, m0 + rh * 64, bz, p.q_b0, c);
-          tma_load5(sQ + dc * 16384u + rh * 8192u, &map_q, bar_q, c);
-        }
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) tma_load5(sQ + dc * 16384u + rh * 8192u, &map_q, bar_q, qc[dc * 2 + rh]);
     }
     load_k(0);
     if (n_kv > 1) load_k(1);
