@@ -314,6 +314,26 @@ def test_fused_attention_shapes_and_operand_majors(D, causal, S):
         plan.close()
 
 
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("causal", [0, 1])
+def test_fused_attention_more_work_items_than_sms(D, causal):
+    """The persistent form deals its work items (a head's pair of query tiles) to one CTA per SM: with 4 x 40 heads and
+    two items per head (the second one a partial tile pair: 328 = 256 + 72 rows) every CTA walks two or three items of
+    different heads and lengths, so the barrier phases, the K / V ring and the tensor-memory tiles are carried across
+    item boundaries, including from a two-tile item to a one-tile one."""
+    B, nh, S = 4, 40, 328
+    for k_layout, v_layout in [((0, 1, 2, 3), (0, 1, 2, 3)), ((0, 3, 1, 2), (0, 2, 1, 3))]:
+        g, cands, _ = _attention_graph(B, S, nh, D, causal, k_layout, v_layout)
+        feeds = {t: rand_feed([B, S, nh, D], synth.BF16, 40 + t, -2.0, 2.0) for t in g.inputs}
+        ref = run_oracle(g, feeds)[g.outputs[0]]
+        opts = {"force_canonical": 1} if k_layout == (0, 1, 2, 3) else {}
+        got, plan, runner = run_gpu(g, feeds, cands, **opts)
+        assert "ATTN" in [s["kernel_name"] for s in plan.steps()]
+        assert runner.status() == 0
+        assert_close(got[g.outputs[0]], ref, synth.BF16, f"attention over many items D={D} causal={causal} k={k_layout}")
+        plan.close()
+
+
 @pytest.mark.parametrize("M,N,K", [(1024, 2552, 136), (512, 5120, 72), (768, 4096, 200)])
 def test_cta_pair_gemm_ragged_shapes(M, N, K):
     """Enough 256-wide tiles for the CTA-pair kernel (two CTAs per 256 x 256 tile), with a ragged last column
