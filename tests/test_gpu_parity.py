@@ -232,6 +232,26 @@ def test_large_ragged_layout_transforms_bit_exact(dtype, case, target):
 
 
 @pytest.mark.parametrize("dtype", DT)
+@pytest.mark.parametrize("dims,perm", [([6, 40, 24, 136], [2, 0, 1, 3]), ([6, 40, 24, 136], [1, 2, 0, 3]), ([6, 40, 24, 136], [0, 3, 2, 1]),
+                                       ([6, 40, 24, 136], [3, 1, 0, 2]), ([2, 3, 40, 24, 72], [0, 3, 1, 2, 4]),
+                                       ([2, 3, 40, 24, 72], [2, 1, 4, 0, 3]), ([1100, 520], [1, 0]), ([3, 520, 1096], [0, 2, 1])])
+def test_general_permutations_above_a_megabyte(dtype, dims, perm):
+    """Permutations other than the two head transposes, of rank 2 to 5, large enough for the bulk-tensor forms: the same
+    fastest dim on both sides (rows form, any order of the outer dims), a new fastest dim (tiles form: 16-bit elements
+    only, the others stay on the register kernels), extents that are no multiples of the 64-wide tile."""
+    g = synth.GraphDesc()
+    x = g.tensor("x", dtype, dims, synth.INPUT)
+    y = g.tensor("y", dtype, [dims[q] for q in perm], synth.OUTPUT)
+    g.op(synth.TRANSPOSE, [x], [y], perm=perm)
+    a = rand_feed(dims, dtype, 77)
+    got, plan, r = run_gpu(g, {x: a})
+    ref = run_oracle(g, {x: a})[y]
+    assert np.array_equal(got[y], ref)
+    assert r.status() == 0
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", DT)
 def test_embed_and_select_last(dtype):
     g = synth.GraphDesc()
     ids = g.tensor("ids", synth.I32, [3, 17], synth.INPUT)
