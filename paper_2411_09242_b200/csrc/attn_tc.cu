@@ -523,7 +523,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 // cycles (maximum pass 450, exponential pass 1530: 128 exponentials per thread at 4 per clock and scheduler), then
 // ~1900 cycles in which the MMA warp takes its three waits (~450) and issues the 8 + 8 instructions of P.V and the next
 // Q.K^T (~700 + ~750, i.e. ~90 cycles an instruction against 64 alone). The MMA warp serves the two slots in turn and
-// is busy throughout, so a step of both slots takes ~4050 cycles for 2 x 1024 cycles of tensor-core work.
+// is busy throughout, so a step of both slots takes ~4050 cycles for 2 x 1024 cycles of tensor-core work. The ~90
+// cycles are the tensor core's own pace here, not the issuing warp's: with every product's instructions split between
+// two issuing warps on two schedulers (which in a probe brings 110 cycles per instruction beside arithmetic warps back
+// to 64) the kernel ran exactly as fast (951 vs 954 TFLOP/s); and with one issuing warp per slot the slots fall into
+// step, their softmax passes share the schedulers and their products the pipe (757 TFLOP/s).
 // Forms for a role that the whole warp runs in lockstep: every lane executes the instruction, one lane's carries a true
 // issue predicate.
 __device__ __forceinline__ void umma_ss_elect(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc,
@@ -840,7 +844,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // arithmetic on the SAME scheduler: beside two warps there that issue fused multiply-adds back to back an
     // instruction takes 115-186 cycles, beside warps that issue only special-function or integer instructions, or that
     // sit on the other three schedulers, 64-77. Every scheduler carries one softmax warp of each slot (a warp reaches
-    // only the tensor-memory lanes of its own quarter), so this role cannot be moved out of their way.
+    // only the tensor-memory lanes of its own quarter), so this role cannot be moved out of their way. It does not have
+    // to be: two issuing warps (each half of every product, handed over through a named barrier and the tensor-core
+    // fences) left the kernel's time unchanged, so in the kernel the issue is not what the tensor core waits for.
     {
       const uint32_t leader = lane == 0 ? 1u : 0u;
       uint32_t fail = 0;
