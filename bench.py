@@ -568,7 +568,8 @@ def single_cases():
         o = g.tensor("ctx", BF, [B_, 1, nh, D], synth.OUTPUT)
         g.op(synth.CACHED_ATTENTION, [q, k, v, kc, vc, pos], [o], scale=D ** -0.5)
         out[f"decode_attention_{B_}x{nh}x{D}_cache{T}"] = (g, 2.0 * 2 * B_ * T * nh * D, None)
-    for (M, N, K) in ((8192, 8192, 8192), (4096, 2304, 768), (2048, 11008, 4096), (128, 768, 3072), (4, 32000, 4096), (4, 4096, 11008)):
+    for (M, N, K) in ((8192, 8192, 8192), (4096, 2304, 768), (2048, 11008, 4096), (128, 768, 3072), (4, 32000, 4096), (4, 4096, 11008),
+                      (4, 128256, 4096), (4, 4096, 4096), (4, 12288, 4096), (4, 22016, 4096), (4, 50257, 768)):
         g, _ = synth.gemm_case(M, N, K, "row", "col", materialize=False)
         out[f"gemm_{M}x{N}x{K}"] = (g, 2.0 * (M * K + K * N + M * N) if M <= 16 else None, 2.0 * M * N * K)
     return out

@@ -498,7 +498,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
           gs[gi].bias = R(s.x_ptr[gi - 1][2]);
           gs[gi].R = nullptr;
         }
-        if (R.ok) err = launch_gemm_rows(gs, ng, stream, s.swiglu, s.norm_fused ? &rn : nullptr);
+        if (R.ok) err = launch_gemm_rows(gs, ng, stream, s.swiglu, s.norm_fused ? &rn : nullptr, status);
         break;
       }
       case FLUID_K_ATTN: {

@@ -222,7 +222,8 @@ struct RowsNorm {
   int x_f32;
 };
 bool gemm_rows_eligible(const GemmParams& g);
-cudaError_t launch_gemm_rows(const GemmParams* g, int n_group, cudaStream_t stream, int swiglu = 0, const RowsNorm* norm = nullptr);
+cudaError_t launch_gemm_rows(const GemmParams* g, int n_group, cudaStream_t stream, int swiglu = 0, const RowsNorm* norm = nullptr,
+                             uint32_t* status = nullptr);
 cudaError_t launch_attn_decode(const AttnDecodeParams& p, cudaStream_t stream);
 bool attn_decode_supported(int dtype, int D);
 

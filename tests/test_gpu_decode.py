@@ -158,6 +158,7 @@ def test_decoding_steps_of_a_small_model(family, dtype, kw):
     (3, 2304, 768, True, False, False),
     (5, 97, 1032, False, True, False),
     (8, 11008, 4096, False, False, True),
+    (2, 16400, 4096, True, False, True),      # above 128 MiB of weights: the bulk-tensor form by default
 ])
 def test_few_row_linear_streams_its_weight(M, N, K, bias, act, res):
     """LINEAR with at most 8 rows: the weight-streaming kernel, with the fused bias / GELU / residual epilogue."""
@@ -411,6 +412,64 @@ def test_cached_attention_random_shapes():
         helpers.assert_close(got[out], ref[out], dtype, what)
         assert np.array_equal(runner.inputs[g.inputs.index(kc)].float().cpu().numpy(), ref[kc]), what
         assert np.array_equal(runner.inputs[g.inputs.index(vc)].float().cpu().numpy(), ref[vc]), what
+        plan.close()
+
+
+@pytest.mark.parametrize("form", ["0", "1", "1,2,1", "1,4,4", "2,2,8", "4,1,2", "2,3,16"])
+def test_few_row_linear_both_weight_paths(form, monkeypatch):
+    """The few-row GEMM brings its weights in either by per-lane asynchronous copies (form "0") or by bulk-tensor
+    boxes ("1": its own choice of boxes per stage, stages, warps per tile; else those three): every form against the oracle, on ragged N and K, 1 to 16 rows,
+    the epilogues, and one decoding step of a small Llama-shaped model (sibling projections behind a folded
+    normalisation, SwiGLU)."""
+    monkeypatch.setenv("FLUID_ROWS_TMA", form)
+    for it, (M, N, K, bias, act, res) in enumerate([(4, 1000, 136, True, True, True), (8, 4112, 4096, False, False, True),
+                                                    (13, 520, 2056, True, False, False), (16, 300, 1024, False, True, False),
+                                                    (1, 33, 8, True, False, False), (5, 2304, 768, True, False, True)]):
+        g = synth.GraphDesc()
+        x = g.tensor("x", synth.BF16, [M, K], synth.INPUT)
+        w = g.tensor("w", synth.BF16, [K, N], synth.CONST)
+        ins = [x, w]
+        feeds = {x: helpers.rand_feed([M, K], synth.BF16, 10 + it), w: synth.round_bf16(synth.normal(7, 20 + it, [K, N], 0.05))}
+        if bias:
+            b = g.tensor("b", synth.BF16, [N], synth.CONST)
+            ins.append(b)
+            feeds[b] = helpers.rand_feed([N], synth.BF16, 30 + it)
+        y = g.tensor("y", synth.BF16, [M, N], synth.ACT if (act or res) else synth.OUTPUT)
+        g.op(synth.LINEAR, ins, [y], contract=1)
+        if act:
+            a = g.tensor("a", synth.BF16, [M, N], synth.ACT if res else synth.OUTPUT)
+            g.op(synth.GELU, [y], [a], gelu_tanh=0)
+            y = a
+        if res:
+            r = g.tensor("r", synth.BF16, [M, N], synth.INPUT)
+            feeds[r] = helpers.rand_feed([M, N], synth.BF16, 40 + it)
+            o = g.tensor("o", synth.BF16, [M, N], synth.OUTPUT)
+            g.op(synth.ADD, [y, r], [o])
+            y = o
+        got, plan, _ = helpers.run_gpu(g, feeds, synth.default_candidates(g))
+        assert "GEMM_ROWS" in [s["kernel_name"] for s in plan.steps()]
+        helpers.assert_close(got[y], helpers.run_oracle(g, feeds)[y], synth.BF16, f"form {form}: {M}x{N}x{K}")
+        plan.close()
+    for family in ("llama", "gpt2_small"):
+        cfg = synth.scaled(synth.CONFIGS[family], dtype=synth.BF16, S=1, L=1, H=256, nh=4, F=640, B=3, V=777)
+        dec = synth.build_decode_model(cfg, 16)
+        g = dec.graph
+        feeds = dict(dec.consts)
+        feeds[dec.ids] = synth.token_ids(synth.TOKEN_SEED, 1, [cfg.B, 1], cfg.V)
+        feeds[dec.pos] = np.array([9], dtype=np.int32)
+        for i, pair in enumerate(dec.caches):
+            for j, t in enumerate(pair):
+                feeds[t] = synth.round_bf16(synth.uniform(3, 2 * i + j, g.dims(t)))
+        ref = helpers.run_oracle(g, feeds)
+        plan = fluid.Plan(g, synth.default_candidates(g))
+        assert [s["kernel_name"] for s in plan.steps()].count("GEMM_ROWS") >= 4
+        runner = fluid.Runner(plan, dec.consts, poison=True)
+        runner.set_inputs([feeds[t] for t in g.inputs])
+        runner.run()
+        outs = runner.outputs_host()
+        assert runner.status() == 0
+        for tid, got in zip(g.outputs, outs):
+            helpers.assert_close(got, ref[tid], synth.BF16, f"form {form} {family} {g.tensors[tid]['name']}")
         plan.close()
 
 
