@@ -254,9 +254,9 @@ def roofline_of(kernels, peaks, step_ms=None):
 
     `achieved` uses the kernel's launch durations from one event pair per step (launches serialised by the events: no
     overlap of a step's prologue with its predecessor's tail). A tensor-bound kernel is set against the measured
-    BURST bf16 rate (`frac`): the steps are milliseconds long with idle gaps between them and the SM clock stays at
-    its maximum, which is the burst measurement's regime; `frac_of_sustained` (the seconds-long power-capped figure)
-    and `frac_of_nominal` stand beside it. `in_step` is an estimate, not a measurement: the timed step (graph
+    BURST bf16 rate (`frac`), the stricter of the two measured peaks; the timed steps run back to back for seconds and
+    the clocks sampled beside them usually show the power cap active, which is the regime of the SUSTAINED figure:
+    `frac_of_sustained` stands beside it, and so does `frac_of_nominal`. `in_step` is an estimate, not a measurement: the timed step (graph
     replay, where programmatic dependent launch overlaps neighbours) times this kernel's share of the per-step
     event times."""
     name = max(kernels, key=lambda k: kernels[k]["ms"])
