@@ -383,10 +383,10 @@ gemm_rows_tma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_cons
                      const __grid_constant__ RowsTma q) {
   constexpr int MC = 8 * MT;
   constexpr int NG = SWIGLU ? 2 : 1;
-  extern __shared__ __align__(1024) unsigned char smem_raw[];
-  const uint32_t raw = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw));
+  extern __shared__ __align__(1024) unsigned char smem_boxes[];
+  const uint32_t raw = static_cast<uint32_t>(__cvta_generic_to_shared(smem_boxes));
   const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;       // boxes must sit on 1024-byte boundaries
-  unsigned char* base = smem_raw + pad;
+  unsigned char* base = smem_boxes + pad;
   const int ln = p.beta ? 1 : 0;
   const uint32_t stage_bytes = kBoxBytes * uint32_t(q.nb);
   const uint32_t ring_bytes = uint32_t(kWarps * q.stages) * stage_bytes;
