@@ -469,7 +469,9 @@ gemm_rows_tma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_cons
 #pragma unroll 1
       for (int j = 0; j < nk; ++j, ++done) {
         const int s = done % q.stages;
-        if (!mbar_wait(bars + 8u * s, uint32_t(done / q.stages) & 1u)) { ok = false; break; }
+        // one answer per warp: the lanes meet again at the __syncwarp below
+        ok = __all_sync(0xffffffffu, mbar_wait(bars + 8u * s, uint32_t(done / q.stages) & 1u));
+        if (!ok) break;
         const uint32_t wst = ring + uint32_t(s) * stage_bytes + w_lane;
         const uint32_t xst = xs_lane + uint32_t((k0 + j) * stage_k) * 2u;
         for (int b = 0; b < q.nb; ++b) {
