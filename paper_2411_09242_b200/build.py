@@ -12,7 +12,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libfluid.so")
-SOURCES = ["graph.cpp", "planner.cpp", "executor.cu", "kernels_mem.cu", "gemm_simt.cu", "gemm_tc.cu", "attn_tc.cu", "attn_decode.cu", "gemm_rows.cu", "permute_tma.cu"]
+SOURCES = ["graph.cpp", "planner.cpp", "executor.cu", "kernels_mem.cu", "gemm_simt.cu", "gemm_tc.cu", "attn_tc.cu", "attn_small.cu", "attn_decode.cu", "gemm_rows.cu", "permute_tma.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
          "-I", os.path.join(ROOT, "include"), "-I", CSRC]

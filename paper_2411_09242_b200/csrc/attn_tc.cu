@@ -1084,8 +1084,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 }  // namespace
 
 // Which form runs: two query tiles per work item on persistent CTAs (probabilities in tensor memory) when the sequence
-// has more than one query tile, else the one-tile form. FLUID_ATTN_FORM in the environment forces a form (A/B timing):
-// 1 one tile per CTA, 2 the persistent two-tile form. FLUID_ATTN_CTAS caps the persistent form's grid (default: one CTA
+// has more than one query tile; for one tile the register form of attn_small.cu when Q, K and V have d contiguous, else
+// the one-tile form. FLUID_ATTN_FORM in the environment forces a form (A/B timing): 1 one tile per CTA, 2 the
+// persistent two-tile form. FLUID_ATTN_CTAS caps the persistent form's grid (default: one CTA
 // per SM).
 static int attn_form(const AttnParams& p) {
   static const int forced = [] {
@@ -1093,6 +1094,7 @@ static int attn_form(const AttnParams& p) {
     return e ? std::atoi(e) : 0;
   }();
   if (forced >= 1 && forced <= 2) return forced;
+  if (p.S <= TQ && attn_small_eligible(p)) return 3;
   return p.S > TQ ? 2 : 1;
 }
 
@@ -1126,6 +1128,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream
   static bool attr[4] = {false, false, false, false};
   if (D != 64 && D != 128) return cudaErrorInvalidValue;
   const int form = attn_form(p);
+  if (form == 3) return launch_attn_small(p, stream);
   if (form == 2) {
     const size_t smem = size_t(6) * TQ * D * 2 + 256 + 1024;
     const int items = ((p.S + 2 * TQ - 1) / (2 * TQ)) * p.B * p.NH;

@@ -504,6 +504,7 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       case FLUID_K_ATTN: {
         AttnParams q = s.attn;
         q.O = const_cast<void*>(R(s.t_ptr[3]));
+        q.Q = R(s.t_ptr[0], 1); q.K = R(s.t_ptr[1], 1); q.V = R(s.t_ptr[2], 1);
         q.status = status;
         if (R.ok) err = launch_attn_tc(q, s.attn_host, stream);
         break;

@@ -191,6 +191,10 @@ struct AttnParams {
   int v_k_major;        // V has the sequence index contiguous
   int q_sel[5], k_sel[5], v_sel[5];   // tensor-map coordinate feeds: 0 contraction, 2 row, 4 / 5 batch split, 6 zero
   int q_b0, k_b0, v_b0;               // inner extent of each operand's (batch * head) index split
+  // plain addressing, for the short-sequence form that reads the operands without tensor maps
+  const void *Q, *K, *V;              // bound per run
+  int64_t q_s[3], k_s[3], v_s[3];     // element strides of b, h, s
+  int rows_d_contiguous;              // Q, K and V all have d contiguous and 16-byte aligned rows
 };
 
 // One decoding step against a key/value cache [B, Tmax, NKV, D] (canonical, caller-owned): the new key and
@@ -259,6 +263,9 @@ int gemm_cluster_split(const GemmParams* gs, const GemmTcHost& tc, int n_group);
 bool gemm_pair_eligible(const GemmParams* gs, const GemmTcHost& tc, int n_group);
 bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc, int variant = 0);
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream);
+// Short sequences (S <= 128) with d contiguous in Q, K and V: one warp per 16 query rows, scores in registers.
+bool attn_small_eligible(const AttnParams& p);
+cudaError_t launch_attn_small(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);
 cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t stream);
 cudaError_t launch_rope(const RopeParams& p, cudaStream_t stream);

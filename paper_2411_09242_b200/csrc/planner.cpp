@@ -375,6 +375,12 @@ bool lower_attn(const fluid_plan_s* p, const Node& n, const int* lo, AttnParams*
   a.v_k_major = h.v.mn_major ? 0 : 1;
   for (int d = 0; d < 5; ++d) { a.q_sel[d] = h.q.sel[d]; a.k_sel[d] = h.k.sel[d]; a.v_sel[d] = h.v.sel[d]; }
   a.q_b0 = h.q.b0; a.k_b0 = h.k.b0; a.v_b0 = h.v.b0;
+  // K is [B,nh,D,S] as an operand and V [B,nh,S,D]: the sequence index is dim 3 of K, dim 2 of V
+  for (int d = 0; d < 2; ++d) { a.q_s[d] = sq[d]; a.k_s[d] = sk[d]; a.v_s[d] = sv[d]; }
+  a.q_s[2] = sq[2]; a.k_s[2] = sk[3]; a.v_s[2] = sv[2];
+  a.rows_d_contiguous = sq[3] == 1 && sk[2] == 1 && sv[3] == 1;
+  for (int d = 0; d < 3; ++d)
+    if (a.q_s[d] % 8 || a.k_s[d] % 8 || a.v_s[d] % 8) a.rows_d_contiguous = 0;
   h.eligible = 1;
   *ap = a;
   *host = h;

@@ -336,6 +336,26 @@ def test_fused_attention_shapes_and_operand_majors(D, causal, S):
 
 @pytest.mark.parametrize("D", [64, 128])
 @pytest.mark.parametrize("causal", [0, 1])
+def test_short_sequence_attention_in_registers(D, causal):
+    """Sequences of at most 128 positions whose K and V have the head dim contiguous run on the register form (16
+    query rows per CTA, four warps that split the keys and then the head dim): lengths that end inside a warp's 32
+    keys, inside a 16-key step and inside a 16-row block, one key only, and the full 128; K and V rows strided
+    ([B,S,nh,D]) or dense per head ([B,nh,S,D])."""
+    B, nh = 2, 5
+    for S in (8, 16, 24, 40, 72, 120, 128):
+        for k_layout, v_layout in [((0, 3, 1, 2), (0, 2, 1, 3)), ((0, 1, 3, 2), (0, 1, 2, 3))]:
+            g, cands, _ = _attention_graph(B, S, nh, D, causal, k_layout, v_layout)
+            feeds = {t: rand_feed([B, S, nh, D], synth.BF16, 60 + t + S, -2.0, 2.0) for t in g.inputs}
+            ref = run_oracle(g, feeds)[g.outputs[0]]
+            got, plan, runner = run_gpu(g, feeds, cands)
+            assert "ATTN" in [s["kernel_name"] for s in plan.steps()]
+            assert runner.status() == 0
+            assert_close(got[g.outputs[0]], ref, synth.BF16, f"short attention D={D} S={S} causal={causal} k={k_layout}")
+            plan.close()
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("causal", [0, 1])
 def test_fused_attention_more_work_items_than_sms(D, causal):
     """The persistent form deals its work items (a head's pair of query tiles) to one CTA per SM: with 4 x 40 heads and
     two items per head (the second one a partial tile pair: 328 = 256 + 72 rows) every CTA walks two or three items of
