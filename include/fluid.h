@@ -151,7 +151,7 @@ typedef struct fluid_plan_options {
   /* Implementation variants (the paper's "Loop Reordering": the time T of a matrix-multiply-like node that the
    * dynamic programme sees is the best over its implementation variants, and that variant is the one that runs).
    * A tensor-core GEMM node has the variants listed by fluid_gemm_variants for its shape and layouts
-   * (code = form | tile_n << 4; form 1: one CTA per 128 x tile_n tile, 2: a CTA pair per 256 x 256 tile,
+   * (code = form | tile_n << 4; form 1: one CTA per 128 x tile_n tile, 2: a CTA pair per 256 x tile_n tile (tile_n 256, or 192 for single steps with a k-contiguous weight),
    * 3: a thread-block cluster per tile that splits k). With the built-in table every variant is rated by an analytic
    * model (waves of tiles, cycles per tensor-core instruction of that width, epilogue, bytes) and the cheapest is
    * kept. eval_variant, when set, replaces eval: it is called once per variant of a node (variant 0 for nodes that

@@ -64,7 +64,21 @@ int finalize_steps(fluid_plan_s* p) {
         }
         const GemmParams& g = s.gemm;
         // the variant the planner rated best for this node (or the caller asked for); the fused SwiGLU form exists for CTA pairs only
-        const int gv = (s.swiglu || s.rope_fused) ? gemm_variant_code(GV_PAIR, 256) : gemm_variant_of(p, n);
+        int gv = (s.swiglu || s.rope_fused) ? gemm_variant_code(GV_PAIR, 256) : gemm_variant_of(p, n);
+        // A node is rated on its own; siblings that share a launch multiply the tiles, which moves the wave count the
+        // rating turns on: the group is rated again as a group (unless the caller named a variant or rates them itself).
+        const int n_sib = (s.swiglu || s.rope_fused) ? 1 : int(s.nodes.size()) - s.norm_fused;
+        const int anchor = n.ops.empty() ? -1 : n.ops[0];
+        const bool asked = anchor >= 0 && anchor < (int)p->op_variant.size() && p->op_variant[anchor] != 0;
+        if (n_sib > 1 && !asked && !p->opts.eval_variant) {
+          double best = kInf;
+          for (int code : gemm_tc_variants(p, g, n_sib)) {
+            GemmTcHost tv;
+            if (!gemm_tc_describe(g, &tv, code)) continue;
+            const double c = gemm_tc_variant_cost(g, tv, n_sib);
+            if (c < best) { best = c; gv = code; }
+          }
+        }
         s.kernel = gemm_tc_eligible(p, g, &s.tc, gv) ? FLUID_K_GEMM_TC : FLUID_K_GEMM_SIMT;
         if (s.kernel == FLUID_K_GEMM_TC)
           s.variant = (s.tc.cfg.a_mn_major ? 1 : 0) | (s.tc.cfg.b_mn_major ? 2 : 0) | (s.tc.cfg.bn << 8);

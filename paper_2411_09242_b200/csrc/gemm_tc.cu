@@ -1513,9 +1513,12 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
                     const __grid_constant__ TcParams p) {
-  constexpr int PN = 256;                          // tile width of the pair (columns of the accumulator)
-  constexpr uint32_t kBHalfBytes = 128 * BK * 2;   // this CTA's 128 columns of the B tile
+  // tile width of the pair (columns of the accumulator): 256, or 192 for plain steps whose tiles then fill one wave
+  // (N = 768 over 16 row pairs: 64 tiles on 74 pairs instead of 48, each three quarters of the work)
+  const int PN = (p.swiglu || EPI == EPI_ROPE) ? 256 : p.cfg.bn;
+  constexpr uint32_t kBHalfBytes = 128 * BK * 2;   // room for this CTA's columns of the B tile (128 at most)
   constexpr uint32_t stage_bytes = kATileBytes + kBHalfBytes;
+  const uint32_t stage_tx = kATileBytes + uint32_t(PN / 2) * BK * 2;   // bytes one CTA's loads of a stage bring
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -1593,7 +1596,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const int mt = 2 * pm + int(rank);
         ksteps = k_steps_of(p, mt);
         int r1, r0, b1, b0;
-        split2((is_a ? mt * BM : (p.swiglu ? nt * 128 : nt * PN + int(rank) * 128)) + ch * box_rows, x_r0, r1, r0);
+        split2((is_a ? mt * BM : (p.swiglu ? nt * 128 : nt * PN + int(rank) * (PN / 2))) + ch * box_rows, x_r0, r1, r0);
         split2(bz, x_b0, b1, b0);
         fill_coords(sel, 5, 0, 0, r0, r1, b0, b1, c);
         map = is_a ? &map_a : (p.swiglu ? (rank == 0 ? &map_b : &map_b1) : (grp == 0 ? &map_b : (grp == 1 ? &map_b1 : &map_b2)));
@@ -1605,7 +1608,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         int k0 = 0, k1 = 0;
         for (int ks = 0; ks < ksteps; ++ks) {
           if (!mbar_wait(eb, ph ^ 1u)) { ok = false; break; }
-          if (lane == 0 && rank == 0) mbar_expect_tx(full_bar(s), 2u * stage_bytes);
+          if (lane == 0 && rank == 0) mbar_expect_tx(full_bar(s), 2u * stage_tx);
           if (k_simple) {
             tma_load_pair(dst, map, fb, c[0], c[1], c[2], c[3], c[4]);
             c[0] += i0; c[1] += i1; c[2] += i2;
@@ -2031,6 +2034,7 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
     }
 #undef FLUID_TC_PAIR
   }
+  if (tc.cfg.bn == 192) return cudaErrorInvalidValue;   // the 192-wide tile exists in the CTA-pair form only
   const int grid = std::min(p.num_tiles, sm_count());
   if (grid <= 0) return cudaSuccess;
   static bool attr_set[7] = {false, false, false, false, false, false, false};

@@ -226,8 +226,8 @@ bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc, int variant) {
   if (g.K < 8) return false;
   const int form = gemm_variant_form(variant), want_bn = gemm_variant_bn(variant);
   if (variant) {
-    if (want_bn != 64 && want_bn != 128 && want_bn != 256) return false;
-    if (form == GV_PAIR && (want_bn != 256 || g.causal != CAUSAL_NONE || g.M % 256 != 0)) return false;
+    if (want_bn != 64 && want_bn != 128 && want_bn != 256 && !(want_bn == 192 && form == GV_PAIR)) return false;
+    if (form == GV_PAIR && ((want_bn != 256 && want_bn != 192) || g.causal != CAUSAL_NONE || g.M % 256 != 0)) return false;
     if (form == GV_CLUSTER && (want_bn > 128 || g.causal != CAUSAL_NONE)) return false;
     if (form < GV_SINGLE || form > GV_CLUSTER) return false;
   }
@@ -251,13 +251,15 @@ bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc, int variant) {
   // of the B tile: its TMA box is then 128 rows, which the single-CTA kernel fetches as two boxes).
   int b_box = bn;
   while (true) {
-    b_box = (bn == 256 && g.causal == CAUSAL_NONE && g.M % 256 == 0 && form != GV_SINGLE) ? 128 : bn;
+    b_box = (bn == 256 && g.causal == CAUSAL_NONE && g.M % 256 == 0 && form != GV_SINGLE) ? 128 : (bn == 192 ? 96 : bn);
     if (build_tma_operand(g.N, g.N0, b_rs, g.K, g.K0, b_ks, g.batch, g.B0, b_bs, b_box, &h.b)) break;
     if (bn == 64 || variant) return false;   // a requested tile width is not traded for a narrower one
     bn /= 2;
   }
+  // a pair's 192-wide tile (96 columns of B per CTA: one box of a k-contiguous operand; 64-column boxes do not add up to it)
+  if (bn == 192 && h.b.mn_major) return false;
   h.cfg.b_box_rows = b_box;
-  h.cfg.pair = (bn == 256 && b_box == 128) ? 1 : 0;
+  h.cfg.pair = ((bn == 256 && b_box == 128) || (bn == 192 && b_box == 96)) ? 1 : 0;
   if (form == GV_PAIR && !h.cfg.pair) return false;
   h.cfg.no_cluster = (form == GV_SINGLE || form == GV_PAIR) ? 1 : 0;
   h.cfg.want_cluster = form == GV_CLUSTER ? 1 : 0;
@@ -287,9 +289,10 @@ std::vector<int> gemm_tc_variants(const fluid_plan_s* p, const GemmParams& g, in
   if (p->opts.gemm_path == 1) return out;
   GemmParams gs[3] = {g, g, g};
   for (int form : {GV_PAIR, GV_SINGLE, GV_CLUSTER})
-    for (int bn : {256, 128, 64}) {
+    for (int bn : {256, 192, 128, 64}) {
       GemmTcHost tc;
       const int code = gemm_variant_code(form, bn);
+      if (bn == 192 && (form != GV_PAIR || n_group != 1)) continue;   // the pair's second width: plain steps only
       if (bn > 64 && g.N <= bn / 2) continue;            // a tile more than twice as wide as the matrix
       if (!gemm_tc_describe(g, &tc, code)) continue;
       if (form == GV_PAIR && !gemm_pair_eligible(gs, tc, n_group)) continue;
@@ -319,7 +322,9 @@ double gemm_tc_variant_cost(const GemmParams& g, const GemmTcHost& tc, int n_gro
   double cycles;
   if (form == GV_PAIR) {
     const double units = sms / 2, pair_tiles = std::ceil(tiles_m / 2.0) * tiles_n * g.batch * n_group;
-    const double main = ksteps * 4.0 * 128.0, epi = (128.0 * 256.0 * out_bytes / 32.0 + 128.0 * 256.0 / 256.0 * 10.0) * act;
+    // (a 256 x 192 x 16 instruction holds 96 cycles of tensor-core work per CTA but is paced by the operand fetch:
+    // ~108 cycles, from four waves of 192-wide tiles against three of 256-wide ones on 4096 x 3072 x 768)
+    const double main = ksteps * 4.0 * (bn == 192 ? 108.0 : 128.0), epi = (128.0 * bn * out_bytes / 32.0 + 128.0 * bn / 256.0 * 10.0) * act;
     cycles = fill + std::ceil(pair_tiles / units) * std::max(main, epi) + epi;
   } else if (form == GV_SINGLE) {
     const double per = bn == 256 ? 171.0 : (bn == 128 ? 107.0 : 97.0);

@@ -461,7 +461,7 @@ def test_variant_costs_from_the_caller_decide_layouts_and_variant_with_the_oracl
 
     def bump(code):
         form, bn = _decode(code)
-        return 0.0 if code == 0 else (1.0 if form == cheap_form else 5.0) + {64: 0.75, 128: 0.25, 256: 0.5}[bn]
+        return 0.0 if code == 0 else (1.0 if form == cheap_form else 5.0) + {64: 0.75, 128: 0.25, 192: 0.625, 256: 0.5}[bn]
 
     asked, offered = set(), {}     # offered: which variants the library listed for (node, layouts): kernel knowledge
 
