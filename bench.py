@@ -259,8 +259,8 @@ def run_reference(args, rank):
 NCU_TRAFFIC = {
     "llama": {"kernel": "GEMM_TC", "bytes_per_launch": 175300000,
               "source": "profiles/launch_list_llama.md (36 GEMM_TC launches, dram read + write)"},
-    "bert_base": {"kernel": "GEMM_TC", "bytes_per_launch": 4121931,
-                  "source": "profiles/dram_traffic_bert_base.md (48 launches of one inference, dram read + write)"},
+    "bert_base": {"kernel": "GEMM_TC", "bytes_per_launch": 4122080,
+                  "source": "profiles/dram_traffic_bert_base.md (the four GEMM steps of two layers, dram read + write)"},
 }
 
 
