@@ -169,6 +169,10 @@ typedef struct fluid_plan_options {
                                to 256) that no kernel may write. In a no_reuse plan the slices are disjoint, so a caller
                                that fills the arena with a pattern before fluid_run can check the zones afterwards: an
                                out-of-bounds store of any kernel shows up without a memory checker */
+  int32_t no_norm_split;    /* 0 (default): an RMS normalisation that sits between a residual GEMM step and GEMM steps that
+                               all run as CTA pairs is split across them (the first also writes bf16(x * gain) and per-slab
+                               sums of squares, the others scale their rows by 1 / rms): no launch of its own, and the
+                               normalised tensor is never stored; 1: it stays a step */
 } fluid_plan_options;
 
 typedef enum {

@@ -64,10 +64,10 @@ int finalize_steps(fluid_plan_s* p) {
         }
         const GemmParams& g = s.gemm;
         // the variant the planner rated best for this node (or the caller asked for); the fused SwiGLU form exists for CTA pairs only
-        int gv = (s.swiglu || s.rope_fused) ? gemm_variant_code(GV_PAIR, 256) : gemm_variant_of(p, n);
+        int gv = (s.swiglu || s.rope_fused || s.nrm_emit) ? gemm_variant_code(GV_PAIR, 256) : gemm_variant_of(p, n);
         // A node is rated on its own; siblings that share a launch multiply the tiles, which moves the wave count the
         // rating turns on: the group is rated again as a group (unless the caller named a variant or rates them itself).
-        const int n_sib = (s.swiglu || s.rope_fused) ? 1 : int(s.nodes.size()) - s.norm_fused;
+        const int n_sib = (s.swiglu || s.rope_fused || s.nrm_emit) ? 1 : int(s.nodes.size()) - s.norm_fused - s.nrm_pre;
         const int anchor = n.ops.empty() ? -1 : n.ops[0];
         const bool asked = anchor >= 0 && anchor < (int)p->op_variant.size() && p->op_variant[anchor] != 0;
         if (n_sib > 1 && !asked && !p->opts.eval_variant) {
@@ -99,7 +99,7 @@ int finalize_steps(fluid_plan_s* p) {
         s.flops = fl;
         s.bytes = es * (a + b + (g.has_bias ? g.N : 0)) + c * (s.gemm.c_f32 ? 4.0 : es) + (g.has_res ? c * (s.gemm.r_f32 ? 4.0 : es) : 0.0);
         // SwiGLU step: the only tensor written is the product, which takes gate's place
-        const size_t n_gemm = s.swiglu ? 2 : s.nodes.size() - s.norm_fused - s.rope_fused;
+        const size_t n_gemm = s.swiglu ? 2 : s.nodes.size() - s.norm_fused - s.rope_fused - s.nrm_pre;
         if (s.swiglu) {
           s.t_ptr[2] = p->nodes[s.nodes[2]].out;
           s.gemm.c_f32 = 0;
@@ -428,11 +428,12 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
         continue;
       }
       if (s.kernel != FLUID_K_GEMM_TC) continue;
-      const void* a = R(s.t_ptr[0], 1);
+      // (the second half of a split normalisation reads bf16(x * gain) from the scratch slice its producer filled)
+      const void* a = s.nrm_pre ? static_cast<const void*>(static_cast<char*>(arena_ptr) + p->records[s.nrm_record].offset) : R(s.t_ptr[0], 1);
       const void* b = R(s.t_ptr[1], 1);
       if (!R.ok) return FLUID_EINVAL;
       bool enc_ok = encode_tensor_map(&s.tc.map_a, a, s.tc.a) == 0 && encode_tensor_map(&s.tc.map_b, b, s.tc.b) == 0;
-      for (size_t gi = 1; enc_ok && gi < (s.swiglu ? size_t(2) : s.nodes.size() - s.rope_fused); ++gi) {
+      for (size_t gi = 1; enc_ok && gi < (s.swiglu ? size_t(2) : s.nodes.size() - s.rope_fused - s.nrm_pre); ++gi) {
         const void* bx = R(s.x_ptr[gi - 1][0], 1);
         if (!R.ok) return FLUID_EINVAL;
         enc_ok = encode_tensor_map(&s.tc_x[gi - 1].map_b, bx, s.tc_x[gi - 1].b) == 0;
@@ -474,18 +475,39 @@ static int run_impl(fluid_plan_s* p, void* arena_ptr, const void* const* inputs,
       case FLUID_K_GEMM_SIMT:
       case FLUID_K_GEMM_TC: {
         GemmParams q = s.gemm;
-        q.A = R(s.t_ptr[0], 1); q.B = R(s.t_ptr[1], 1); q.C = const_cast<void*>(R(s.t_ptr[2]));
+        // split RMS normalisation: the scratch slice holds bf16(x * gain), then the slabs' sums of squares
+        char* nrm_base = (s.nrm_emit || s.nrm_pre) ? static_cast<char*>(arena_ptr) + p->records[s.nrm_record].offset : nullptr;
+        float* nrm_ss = nullptr;
+        int nrm_slabs = 0;
+        if (nrm_base) {
+          const TensorDesc& tn = p->graph.tensors[p->nodes[s.nrm_node].out];
+          nrm_ss = reinterpret_cast<float*>(static_cast<char*>(arena_ptr) + p->records[s.nrm_ss_record].offset);
+          nrm_slabs = int(tn.dims[tn.rank - 1] / 128);
+        }
+        q.A = s.nrm_pre ? nrm_base : R(s.t_ptr[0], 1); q.B = R(s.t_ptr[1], 1); q.C = const_cast<void*>(R(s.t_ptr[2]));
         q.bias = R(s.t_ptr[3]); q.R = R(s.t_ptr[4]);
+        if (s.nrm_emit) {
+          q.nrm_out = nrm_base;
+          q.nrm_gamma = R(p->nodes[s.nrm_node].gamma);
+          q.nrm_ss = nrm_ss;
+        }
+        if (s.nrm_pre) {
+          q.row_ss = nrm_ss;
+          q.row_slabs = nrm_slabs;
+          q.row_inv_n = 1.f / float(nrm_slabs * 128);
+          q.row_eps = float(p->nodes[s.nrm_node].eps);
+        }
         if (s.kernel == FLUID_K_GEMM_TC) {
           GemmParams gs[3] = {q, s.gemm_x[0], s.gemm_x[1]};
           GemmTcHost ts[3] = {s.tc, s.tc_x[0], s.tc_x[1]};
-          const int ng = s.swiglu ? 2 : (int)s.nodes.size() - s.rope_fused;
+          const int ng = s.swiglu ? 2 : (int)s.nodes.size() - s.rope_fused - s.nrm_pre;
           for (int gi = 1; gi < ng; ++gi) {
             gs[gi].A = q.A;
             gs[gi].B = R(s.x_ptr[gi - 1][0], 1);
             gs[gi].C = s.swiglu ? q.C : const_cast<void*>(R(s.x_ptr[gi - 1][1]));
             gs[gi].bias = R(s.x_ptr[gi - 1][2]);
             gs[gi].R = nullptr;
+            gs[gi].row_ss = q.row_ss; gs[gi].row_slabs = q.row_slabs; gs[gi].row_inv_n = q.row_inv_n; gs[gi].row_eps = q.row_eps;
           }
           float* partial = s.scratch_record >= 0
                                ? reinterpret_cast<float*>(static_cast<char*>(arena_ptr) + p->records[s.scratch_record].offset)

@@ -87,6 +87,13 @@ struct Step {
   int norm_fused = 0;       // 1: the last node is the RMS normalisation that feeds every GEMM of the step (few-row kernel only); its output is never stored
   float norm_eps = 0.f;
   int norm_x_f32 = 0;
+  // An RMS normalisation split across two CTA-pair GEMM steps: the step that writes the residual stream (nrm_emit) also
+  // writes bf16(x * gain) and per-slab sums of squares into a scratch slice that lives until the step that reads the
+  // normalised tensor (nrm_pre: its last node is the normalisation; its GEMMs take the scratch as A and scale their rows).
+  int nrm_emit = 0, nrm_pre = 0;
+  int nrm_node = -1;        // the normalisation's node (both steps)
+  int nrm_record = -1;      // the scratch slice of bf16(x * gain) (both steps)
+  int nrm_ss_record = -1;   // the scratch slice of the slabs' sums of squares (both steps)
   int64_t scratch_bytes = 0;
   int scratch_record = -1;  // arena slice holding the split-K partial tiles (alive during this step only)
   NormParams norm{};

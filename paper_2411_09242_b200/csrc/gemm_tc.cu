@@ -432,10 +432,10 @@ __device__ __forceinline__ void epilogue_chunk_coal(const GemmParams& g, uint32_
 template <int ACT, bool HAS_RES, bool C_WIDE, bool R_WIDE>
 __device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
                                                    const int64_t (&cbs)[8], const int64_t (&rbs)[8], uint32_t ok_mask,
-                                                   float* stage, int lane) {
+                                                   float* stage, int lane, float row_scale = 1.f) {
   const int unit = lane & 7, rsub = lane >> 3;
   const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
-  const float scale = g.scale;
+  const float scale = g.scale * row_scale;   // row_scale: this thread's accumulator row (1 / rms of a split normalisation)
   float* const c_f32 = static_cast<float*>(g.C);
   __nv_bfloat16* const c_b16 = static_cast<__nv_bfloat16*>(g.C);
   int n_chunks = (min(col_end, g.N - n_tile0) - col_begin + 31) >> 5;   // uniform across the warp
@@ -534,6 +534,84 @@ __device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t
   }
 }
 
+// The fp32-residual epilogue that also does the first half of an RMS normalisation of its output (the step's output x is
+// a residual stream whose only other reader is that normalisation): besides x it writes bf16(x * gain), the A operand of
+// the steps behind the normalisation, and the sum of x^2 over this warp's 128 columns of each row, one 128-column slab
+// of the row; the readers divide their accumulator rows by the rms they form from the slabs. x is added up and
+// rounded exactly as epilogue_tile_coal does it; a tile is 256 columns wide and full (N a multiple of 256), so a warp's
+// column range is one slab. row0: the row of the tile that lane 0's first staged row belongs to.
+__device__ __forceinline__ void epilogue_tile_resnorm(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
+                                                      const int64_t (&cbs)[8], const int64_t (&rbs)[8], uint32_t ok_mask,
+                                                      float* stage, int lane, int row0) {
+  const int unit = lane & 7, rsub = lane >> 3;
+  const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
+  const float scale = g.scale;
+  float* const c_f32 = static_cast<float*>(g.C);
+  __nv_bfloat16* const x_b16 = static_cast<__nv_bfloat16*>(g.nrm_out);
+  const __nv_bfloat16* const gain = static_cast<const __nv_bfloat16*>(g.nrm_gamma);
+  const int n_chunks = (min(col_end, g.N - n_tile0) - col_begin + 31) >> 5;   // uniform across the warp
+  if (n_chunks <= 0) return;
+  float ss[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+  for (int ci = 0; ci < n_chunks; ++ci) {
+    const int c0 = col_begin + 32 * ci;
+    uint32_t r[32];
+    tmem_ld32(trow + uint32_t(c0), r);
+    const int nc = n_tile0 + c0 + unit * 4;
+    const bool col_ok = nc < g.N;
+    int n1, n0i;
+    split2(nc, g.N0, n1, n0i);
+    const int64_t c_col = (int64_t)n1 * g.c_s[4] + n0i, r_col = (int64_t)n1 * g.r_s[4] + n0i;
+    float bias4[4] = {0.f, 0.f, 0.f, 0.f}, gain4[4] = {0.f, 0.f, 0.f, 0.f};
+    if (col_ok) {
+      const uint2 g2 = __ldg(reinterpret_cast<const uint2*>(gain + nc));
+      gain4[0] = __uint_as_float(g2.x << 16); gain4[1] = __uint_as_float(g2.x & 0xffff0000u);
+      gain4[2] = __uint_as_float(g2.y << 16); gain4[3] = __uint_as_float(g2.y & 0xffff0000u);
+      if (g.has_bias) {
+        const uint2 b2 = __ldg(reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.bias) + nc));
+        bias4[0] = __uint_as_float(b2.x << 16); bias4[1] = __uint_as_float(b2.x & 0xffff0000u);
+        bias4[2] = __uint_as_float(b2.y << 16); bias4[3] = __uint_as_float(b2.y & 0xffff0000u);
+      }
+    }
+    float4 res[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      res[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (col_ok && ((ok_mask >> i) & 1u)) res[i] = *reinterpret_cast<const float4*>(static_cast<const float*>(g.R) + rbs[i] + r_col);
+    }
+    tmem_ld_wait();
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      sts128(st_row + (uint32_t(u ^ (lane & 7)) << 4), __uint_as_float(r[4 * u]) * scale, __uint_as_float(r[4 * u + 1]) * scale,
+             __uint_as_float(r[4 * u + 2]) * scale, __uint_as_float(r[4 * u + 3]) * scale);
+    __syncwarp();
+    const uint32_t live = col_ok ? ok_mask : 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = rsub + 4 * i;
+      float4 v = lds128(st_base + uint32_t(row * 128) + (uint32_t(unit ^ (row & 7)) << 4));
+      v.x += bias4[0]; v.y += bias4[1]; v.z += bias4[2]; v.w += bias4[3];
+      v.x += res[i].x; v.y += res[i].y; v.z += res[i].z; v.w += res[i].w;
+      if ((live >> i) & 1u) {
+        *reinterpret_cast<float4*>(c_f32 + cbs[i] + c_col) = v;
+        *reinterpret_cast<uint2*>(x_b16 + cbs[i] + c_col) = make_uint2(pack_bf16x2(v.x * gain4[0], v.y * gain4[1]), pack_bf16x2(v.z * gain4[2], v.w * gain4[3]));
+        ss[i] += (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+      }
+    }
+    __syncwarp();   // the staging tile is rewritten by the next chunk
+  }
+  // the eight lanes that share a row add up their columns; one of them stores the slab's sum
+  const int slab = (n_tile0 + col_begin) >> 7, slabs = g.N >> 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float t = ss[i];
+    t += __shfl_xor_sync(0xffffffffu, t, 1);
+    t += __shfl_xor_sync(0xffffffffu, t, 2);
+    t += __shfl_xor_sync(0xffffffffu, t, 4);
+    if (unit == 0 && ((ok_mask >> i) & 1u)) g.nrm_ss[(int64_t)(row0 + rsub + 4 * i) * slabs + slab] = t;
+  }
+}
+
 // bf16 output without a residual, 64 columns at a time. A thread finishes its own row first (scale, bias, activation,
 // rounding), so the staging tile holds 32 rows of 64 bf16 (128 bytes a row, 16-byte units swizzled by the row) and a
 // row leaves as ONE 128-byte run (eight lanes x 16 bytes) where the 32-column form above writes two separate 64-byte
@@ -543,10 +621,11 @@ __device__ __forceinline__ void epilogue_tile_coal(const GemmParams& g, uint32_t
 // 128-byte runs of the fp32 outputs). Same arithmetic, in the same order, as the 32-column form.
 template <int ACT>
 __device__ __forceinline__ void epilogue_tile_coal16(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
-                                                     const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane) {
+                                                     const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane,
+                                                     float row_scale = 1.f) {
   const int unit = lane & 7, rsub = lane >> 3;
   const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
-  const float scale = g.scale;
+  const float scale = g.scale * row_scale;
   __nv_bfloat16* const c_b16 = static_cast<__nv_bfloat16*>(g.C);
   const __nv_bfloat16* const bias = static_cast<const __nv_bfloat16*>(g.bias);
   const int n_chunks = (min(col_end, g.N - n_tile0) - col_begin + 63) >> 6;   // uniform across the warp
@@ -682,7 +761,8 @@ __device__ __noinline__ void epilogue_tile_scalar(const GemmParams& g, uint32_t 
 
 // Epilogue variants (template parameter of the kernel)
 enum EpiKind { EPI_ANY = 0, EPI_PLAIN = 1, EPI_PLAIN_WIDE = 2, EPI_RES = 3, EPI_RES_WIDE = 4, EPI_GELU_ERF = 5, EPI_GELU_TANH = 6,
-               EPI_SWIGLU = 7 /* CTA-pair kernel only */, EPI_ROPE = 8 /* CTA-pair kernel only: plain, with the rotary embedding for groups that ask */ };
+               EPI_SWIGLU = 7 /* CTA-pair kernel only */, EPI_ROPE = 8 /* CTA-pair kernel only: plain, with the rotary embedding for groups that ask */,
+               EPI_RES_WIDE_NRM = 9 /* CTA-pair kernel only: fp32 residual in / out, plus the first half of an RMS normalisation of the output */ };
 
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk_c(const GemmParams& g, uint32_t taddr, const int64_t (&cbs)[8], const int64_t (&rbs)[8],
@@ -699,18 +779,18 @@ __device__ __forceinline__ void epilogue_chunk_c(const GemmParams& g, uint32_t t
 template <int EPI>
 __device__ __forceinline__ void epilogue_tile_c(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
                                                 const int64_t (&cbs)[8], const int64_t (&rbs)[8], uint32_t ok_mask, float* stage,
-                                                int lane) {
+                                                int lane, float row_scale = 1.f) {
   // bf16 outputs without a residual leave in 128-byte runs when the warp's columns come in sixty-fours
   const bool wide_runs = ((col_end - col_begin) & 63) == 0;
-  if (EPI == EPI_PLAIN && wide_runs) epilogue_tile_coal16<ACT_NONE>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
-  else if (EPI == EPI_GELU_ERF && wide_runs) epilogue_tile_coal16<ACT_GELU_ERF>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
-  else if (EPI == EPI_GELU_TANH && wide_runs) epilogue_tile_coal16<ACT_GELU_TANH>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
-  else if (EPI == EPI_PLAIN) epilogue_tile_coal<ACT_NONE, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
-  else if (EPI == EPI_PLAIN_WIDE) epilogue_tile_coal<ACT_NONE, false, true, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
-  else if (EPI == EPI_RES) epilogue_tile_coal<ACT_NONE, true, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
-  else if (EPI == EPI_RES_WIDE) epilogue_tile_coal<ACT_NONE, true, true, true>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
-  else if (EPI == EPI_GELU_ERF) epilogue_tile_coal<ACT_GELU_ERF, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
-  else if (EPI == EPI_GELU_TANH) epilogue_tile_coal<ACT_GELU_TANH, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+  if (EPI == EPI_PLAIN && wide_runs) epilogue_tile_coal16<ACT_NONE>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane, row_scale);
+  else if (EPI == EPI_GELU_ERF && wide_runs) epilogue_tile_coal16<ACT_GELU_ERF>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane, row_scale);
+  else if (EPI == EPI_GELU_TANH && wide_runs) epilogue_tile_coal16<ACT_GELU_TANH>(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane, row_scale);
+  else if (EPI == EPI_PLAIN) epilogue_tile_coal<ACT_NONE, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane, row_scale);
+  else if (EPI == EPI_PLAIN_WIDE) epilogue_tile_coal<ACT_NONE, false, true, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane, row_scale);
+  else if (EPI == EPI_RES) epilogue_tile_coal<ACT_NONE, true, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane, row_scale);
+  else if (EPI == EPI_RES_WIDE) epilogue_tile_coal<ACT_NONE, true, true, true>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane, row_scale);
+  else if (EPI == EPI_GELU_ERF) epilogue_tile_coal<ACT_GELU_ERF, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane, row_scale);
+  else if (EPI == EPI_GELU_TANH) epilogue_tile_coal<ACT_GELU_TANH, false, false, false>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane, row_scale);
 }
 
 template <int EPI>
@@ -1423,10 +1503,11 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
 // compensated fp32 angle product and reduction, as in the stand-alone kernel) and leave through the shared-memory turn of
 // the other epilogues. The unrotated projection never exists in memory and is never rounded to bf16.
 __device__ __forceinline__ void epilogue_tile_rope(const GemmParams& g, const RopeFreq& fr, uint32_t trow, int col_begin, int n_tile0,
-                                                   const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane, int pos) {
+                                                   const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane, int pos,
+                                                   float row_scale = 1.f) {
   const int unit = lane & 7, rsub = lane >> 3;
   const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
-  const float scale = g.scale;
+  const float scale = g.scale * row_scale;
   __nv_bfloat16* const c_b16 = static_cast<__nv_bfloat16*>(g.C);
   if (n_tile0 + col_begin >= g.N) return;   // uniform across the warp
 #pragma unroll 1
@@ -1471,10 +1552,11 @@ __device__ __forceinline__ void epilogue_tile_rope(const GemmParams& g, const Ro
 }
 
 __device__ __forceinline__ void epilogue_tile_swiglu(const GemmParams& g, uint32_t trow, int col_begin, int col_end, int n_tile0,
-                                                     const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane) {
+                                                     const int64_t (&cbs)[8], uint32_t ok_mask, float* stage, int lane,
+                                                     float row_scale = 1.f) {
   const int unit = lane & 7, rsub = lane >> 3;
   const uint32_t st_base = smem_u32(stage), st_row = st_base + uint32_t(lane) * 128u;
-  const float scale = g.scale;
+  const float scale = g.scale * row_scale;
   __nv_bfloat16* const c_b16 = static_cast<__nv_bfloat16*>(g.C);
 #pragma unroll 1
   for (int c0 = col_begin; c0 < col_end; c0 += 32) {
@@ -1700,14 +1782,30 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       }
       // the first tile's row and column offsets above are index arithmetic (sixteen divisions): done before the wait
       if (!waited) { pdl_wait(); waited = true; }   // before any global read (bias, residual) or write (C)
+      // second half of a split RMS normalisation: 1 / rms of this thread's accumulator row from the slabs its producer
+      // left, in slab order (read while the tile's MMAs still run)
+      float row_scale = 1.f;
+      if ((EPI == EPI_SWIGLU || EPI == EPI_ROPE) && g.row_ss) {
+        const int row = mt * BM + lane_base + lane;
+        if (row < g.M) {
+          const float* ssp = g.row_ss + (int64_t)row * g.row_slabs;
+          float t = 0.f;
+          for (int k = 0; k < g.row_slabs; k += 4) {
+            const float4 q4 = *reinterpret_cast<const float4*>(ssp + k);
+            t += q4.x; t += q4.y; t += q4.z; t += q4.w;
+          }
+          row_scale = rsqrtf(t * g.row_inv_n + g.row_eps);
+        }
+      }
       if (!mbar_wait_warp(tfull_bar(acc), acc_ph)) { ok = false; break; }
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t(lane_base) << 16) + uint32_t(acc * PN);
-      if (EPI == EPI_SWIGLU) epilogue_tile_swiglu(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane);
+      if (EPI == EPI_SWIGLU) epilogue_tile_swiglu(g, trow, col_begin, col_end, n_tile0, cbs, ok_mask, stage, lane, row_scale);
       else if (EPI == EPI_ROPE) {
-        if (g.rope) epilogue_tile_rope(g, p.rope_freq, trow, col_begin, n_tile0, cbs, ok_mask, stage, lane, (mt * BM + lane_base + lane) % g.rope_S);
-        else epilogue_tile_c<EPI_PLAIN>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
-      } else epilogue_tile_c<EPI>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
+        if (g.rope) epilogue_tile_rope(g, p.rope_freq, trow, col_begin, n_tile0, cbs, ok_mask, stage, lane, (mt * BM + lane_base + lane) % g.rope_S, row_scale);
+        else epilogue_tile_c<EPI_PLAIN>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane, row_scale);
+      } else if (EPI == EPI_RES_WIDE_NRM) epilogue_tile_resnorm(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane, mt * BM + lane_base);
+      else epilogue_tile_c<EPI>(g, trow, col_begin, col_end, n_tile0, cbs, rbs, ok_mask, stage, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0u));   // CTA 0 counts both CTAs' epilogue warps
@@ -2011,7 +2109,7 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 2 : 1;
-    static bool pattr_set[9] = {false, false, false, false, false, false, false, false, false};
+    static bool pattr_set[10] = {};
 #define FLUID_TC_PAIR(E)                                                                                             \
   case E: {                                                                                                          \
     if (!pattr_set[E]) {                                                                                             \
@@ -2021,11 +2119,17 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
     }                                                                                                                \
     return cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel<E>, *ma, *mb, *mb1, *mb2, q);                                \
   }
+    if (g.nrm_out) {   // first half of a split RMS normalisation: whole 256-wide tiles of one fp32 residual stream
+      if (epi != EPI_RES_WIDE || n_group != 1 || !g.nrm_gamma || !g.nrm_ss || g.N % 256 != 0 || g.N0 != g.N || tc.cfg.bn != 256)
+        return cudaErrorInvalidValue;
+      epi = EPI_RES_WIDE_NRM;
+    }
     switch (epi) {
       FLUID_TC_PAIR(EPI_PLAIN)
       FLUID_TC_PAIR(EPI_PLAIN_WIDE)
       FLUID_TC_PAIR(EPI_RES)
       FLUID_TC_PAIR(EPI_RES_WIDE)
+      FLUID_TC_PAIR(EPI_RES_WIDE_NRM)
       FLUID_TC_PAIR(EPI_GELU_ERF)
       FLUID_TC_PAIR(EPI_GELU_TANH)
       FLUID_TC_PAIR(EPI_SWIGLU)
@@ -2035,6 +2139,8 @@ cudaError_t launch_gemm_tc(const GemmParams* gs, const GemmTcHost* tcs, int n_gr
 #undef FLUID_TC_PAIR
   }
   if (tc.cfg.bn == 192) return cudaErrorInvalidValue;   // the 192-wide tile exists in the CTA-pair form only
+  for (int i = 0; i < n_group; ++i)
+    if (gs[i].nrm_out || gs[i].row_ss) return cudaErrorInvalidValue;   // so does the split normalisation
   const int grid = std::min(p.num_tiles, sm_count());
   if (grid <= 0) return cudaSuccess;
   static bool attr_set[7] = {false, false, false, false, false, false, false};

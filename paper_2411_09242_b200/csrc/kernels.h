@@ -40,6 +40,16 @@ struct GemmParams {
   int b_const;  // B is a constant of the plan (a weight): its loads need not wait for the previous step
   int rope;     // 1: the rotary embedding of the output (heads of 128 columns, pairs (d, d + 64), position = row % rope_S) runs in the epilogue
   int rope_S;   // rows per sequence
+  // An RMS normalisation split across two tensor-core steps (CTA-pair form). The step that produces the residual
+  // stream x (this GEMM's fp32 output) also writes bf16(x * gain) and, per row and 128-column slab, the sum of x^2 ...
+  void* nrm_out;          // bf16, same element offsets as C
+  const void* nrm_gamma;  // bf16 gain, indexed by n
+  float* nrm_ss;          // [M][N / 128] sums of squares
+  // ... and the steps that read the normalised tensor take bf16(x * gain) as their A operand and scale their
+  // accumulator rows by 1 / rms, formed from the slabs in slab order: (x * gain / rms) . W = ((x * gain) . W) / rms.
+  const float* row_ss;    // [M][row_slabs]
+  int row_slabs;
+  float row_inv_n, row_eps;   // 1 / (elements of a normalised row), the normalisation's epsilon
 };
 
 // Host-side description of the two TMA tensor maps of a tensor-core GEMM step.

@@ -1150,6 +1150,74 @@ static void greedy_by_size(std::vector<ArenaRecord>& recs, int policy, bool no_r
         for (size_t i = 0; i < recs.size(); ++i) best_off[i] = recs[i].offset;
       }
     }
+  // Once more, for plans in which a few large records sit among many of one common size (a 43 MB SwiGLU product among
+  // 16 MB projections): the large ones are placed as if they were a whole number of the common size, so the gaps they
+  // leave hold whole records of that size, and alternately from the bottom and from the top of the space under the
+  // largest live set, so that the common-size records around them can alternate too (a layer's scratch next to the
+  // product below it in one layer, above it in the next). Offsets found for padded sizes are valid for the true ones;
+  // the arena is measured with the true ones.
+  if (!no_reuse && !recs.empty()) {
+    std::vector<int64_t> sizes;
+    for (const ArenaRecord& r : recs) sizes.push_back(r.bytes);
+    std::sort(sizes.begin(), sizes.end());
+    int64_t quantum = 0;
+    int best_count = 0;
+    for (size_t i = 0; i < sizes.size();) {
+      size_t j = i;
+      while (j < sizes.size() && sizes[j] == sizes[i]) ++j;
+      if (int(j - i) > best_count || (int(j - i) == best_count && sizes[i] > quantum)) { best_count = int(j - i); quantum = sizes[i]; }
+      i = j;
+    }
+    int last_step = 0;
+    for (const ArenaRecord& r : recs) last_step = std::max(last_step, r.last);
+    int64_t live = 0;   // largest live set, with the padded sizes
+    std::vector<ArenaRecord> padded = recs;
+    bool any = false;
+    for (ArenaRecord& r : padded)
+      if (quantum > 0 && r.bytes > quantum && r.bytes % quantum != 0) { r.bytes = (r.bytes + quantum - 1) / quantum * quantum; any = true; }
+    for (int si = 0; si <= last_step; ++si) {
+      int64_t sum = 0;
+      for (const ArenaRecord& r : padded)
+        if (r.first <= si && si <= r.last) sum += r.bytes;
+      live = std::max(live, sum);
+    }
+    const int64_t ceiling = FLUID_ARENA_HEADER + live;
+    if (any)
+     for (const auto& ord : orders) {
+      // a padded record takes the lowest gap or the highest place under the ceiling in turn, the others the lowest gap
+      std::vector<int> placed;
+      int turn = 0;
+      for (int ri : ord) {
+        ArenaRecord& r = padded[ri];
+        std::vector<std::pair<int64_t, int64_t>> busy;
+        for (int qi : placed) {
+          const ArenaRecord& q = padded[qi];
+          if (q.first <= r.last && r.first <= q.last) busy.push_back({q.offset, q.offset + q.bytes});
+        }
+        std::sort(busy.begin(), busy.end());
+        const bool big = r.bytes != recs[ri].bytes;
+        const bool from_top = big && (turn++ & 1);
+        int64_t cursor = FLUID_ARENA_HEADER, low = -1, high = -1;
+        for (auto& b : busy) {
+          if (b.first - cursor >= r.bytes) {
+            if (low < 0) low = cursor;
+            if (b.first <= ceiling) high = b.first - r.bytes;
+          }
+          cursor = std::max(cursor, b.second);
+        }
+        if (low < 0) low = cursor;
+        if (ceiling - cursor >= r.bytes) high = ceiling - r.bytes;
+        r.offset = (from_top && high >= 0) ? high : low;
+        placed.push_back(ri);
+      }
+      int64_t a = FLUID_ARENA_HEADER;
+      for (size_t i = 0; i < recs.size(); ++i) a = std::max(a, padded[i].offset + recs[i].bytes);
+      if (a < best) {
+        best = a;
+        for (size_t i = 0; i < recs.size(); ++i) best_off[i] = padded[i].offset;
+      }
+    }
+  }
   for (size_t i = 0; i < recs.size(); ++i) recs[i].offset = best_off[i];
   *arena_bytes = (size_t)best;
 }
@@ -1349,6 +1417,59 @@ static int lower_and_place(fluid_plan_s* p) {
       p->steps.erase(p->steps.begin() + si);
     }
   }
+  // RMS normalisation between two CTA-pair steps (pre-norm decoders at prefill sizes: o-proj / down -> RMSNorm ->
+  // gate / up or q / k / v): the producer's residual epilogue holds whole 128-column slabs of the fp32 stream, so it also
+  // writes bf16(x * gain) and the slabs' sums of squares, and the readers scale their accumulator rows by 1 / rms
+  // ((x * gain / rms) . W = ((x * gain) . W) / rms): the normalisation's launch and its pass over the stream go.
+  // bf16 is applied to x * gain instead of x * gain / rms: the same relative rounding.
+  if (p->opts.fusion && p->opts.gemm_path == 0 && !p->opts.eval && !p->opts.eval_variant && !p->opts.narrow_stream &&
+      p->opts.split_k <= 0 && !p->opts.no_norm_split) {
+    std::vector<int> n_uses(nt, 0);
+    for (const Node& n : p->nodes)
+      for (int t : n.ins) n_uses[t]++;
+    for (int si = 1; si + 1 < (int)p->steps.size(); ++si) {
+      const Step& sn = p->steps[si];
+      if (sn.nodes.size() != 1) continue;
+      const Node& nn = p->nodes[sn.node];
+      if (nn.kind != N_NORM || !nn.rms || nn.res >= 0 || T[nn.out].kind != FLUID_ACT || T[nn.out].dtype != FLUID_BF16 ||
+          p->alias_root[nn.out] != nn.out || p->alias_root[nn.a] != nn.a || T[nn.gamma].kind != FLUID_CONST || lo[nn.gamma] != 0 ||
+          !is_identity(p, nn.out, lo) || !is_identity(p, nn.a, lo) || T[nn.a].kind != FLUID_ACT || T[nn.a].dtype != FLUID_BF16)
+        continue;
+      Step& sp = p->steps[si - 1];
+      Step& sc = p->steps[si + 1];
+      if (sp.nodes.size() != 1 || sp.swiglu || sp.rope_fused || sp.norm_fused || sp.nrm_emit || sp.nrm_pre) continue;
+      const Node& pn = p->nodes[sp.node];
+      if (pn.kind != N_GEMM || pn.gemm_kind != G_LINEAR || pn.res < 0 || pn.out != nn.a || pn.act != ACT_NONE) continue;
+      GemmParams g;
+      GemmTcHost tc;
+      if (!lower_gemm(p, pn, lo, &g) || !gemm_tc_eligible(p, g, &tc, gemm_variant_code(GV_PAIR, 256)) || !tc.cfg.pair) continue;
+      GemmParams gs[3] = {g, g, g};
+      bool like = true;
+      for (int d = 0; d < 6; ++d) like = like && g.r_s[d] == g.c_s[d];
+      if (!gemm_pair_eligible(gs, tc, 1) || !like || g.batch != 1 || g.N % 512 != 0 || g.N0 != g.N || g.M0 != g.M || g.c_s[5] != 1 ||
+          g.c_s[3] != g.N || g.M % 256 != 0 || T[nn.out].numel() != (int64_t)g.M * g.N || T[nn.out].dims[T[nn.out].rank - 1] != g.N)
+        continue;
+      // the readers: every GEMM of the next step, which runs as CTA pairs with an epilogue that takes a row scale
+      if (!(sc.swiglu || sc.rope_fused) || sc.nrm_pre || sc.norm_fused) continue;
+      int readers = 0;
+      bool ok = true;
+      for (int ni : sc.nodes) {
+        const Node& m = p->nodes[ni];
+        if (m.kind != N_GEMM) continue;
+        ok = ok && m.a == nn.out && m.gemm_kind == G_LINEAR;
+        ++readers;
+      }
+      if (!ok || readers == 0 || n_uses[nn.out] != readers) continue;
+      sp.nrm_emit = 1;
+      sp.nrm_node = sn.node;
+      sc.nrm_pre = 1;
+      sc.nrm_node = sn.node;
+      sc.nodes.push_back(sn.node);
+      sc.cost += sn.cost - kLaunch;
+      p->folded[nn.out] = 1;
+      p->steps.erase(p->steps.begin() + si);
+    }
+  }
   // lifetimes in step indices, per alias group
   p->first_step.assign(nt, -1);
   p->last_step.assign(nt, -1);
@@ -1505,6 +1626,28 @@ static int lower_and_place(fluid_plan_s* p) {
     r.first = r.last = si;
     st.scratch_bytes = r.bytes;
     st.scratch_record = (int)p->records.size();
+    p->records.push_back(r);
+  }
+  // scratch of a split RMS normalisation: bf16(x * gain) and the slabs' sums of squares, from the step that writes
+  // them to the step that reads them (the next one)
+  for (int si = 0; si + 1 < (int)p->steps.size(); ++si) {
+    Step& st = p->steps[si];
+    if (!st.nrm_emit) continue;
+    const Node& nn = p->nodes[st.nrm_node];
+    const int64_t n = T[nn.out].dims[T[nn.out].rank - 1], m = T[nn.out].numel() / n;
+    // (two slices: the first has exactly the size the normalised tensor's own slice would have had)
+    ArenaRecord r;
+    r.root = -1;
+    r.step = si;
+    r.id = 3 * nt + si;
+    r.bytes = round_up(m * n * 2, FLUID_SLOT_ALIGN);
+    r.first = si;
+    r.last = si + 1;
+    st.nrm_record = p->steps[si + 1].nrm_record = (int)p->records.size();
+    p->records.push_back(r);
+    r.id = 3 * nt + (int)p->steps.size() + si;
+    r.bytes = round_up(m * (n / 128) * 4, FLUID_SLOT_ALIGN);
+    st.nrm_ss_record = p->steps[si + 1].nrm_ss_record = (int)p->records.size();
     p->records.push_back(r);
   }
   greedy_by_size(p->records, p->opts.arena_policy, p->opts.no_reuse != 0, &p->arena_bytes);
@@ -1707,7 +1850,10 @@ int fluid_plan_step_info(const fluid_plan_t* p, int step, fluid_step_info* info)
   std::memset(info, 0, sizeof(*info));
   info->kernel = s.kernel;
   info->variant = s.variant;
-  for (int ni : s.nodes) {
+  // (a normalisation whose second half this step runs is listed first: its result is what the step's GEMMs read)
+  std::vector<int> order(s.nodes.begin(), s.nodes.end());
+  if (s.nrm_pre && !order.empty()) std::rotate(order.begin(), order.end() - 1, order.end());
+  for (int ni : order) {
     const Node& n = p->nodes[ni];
     for (int o : n.ops)
       if (info->n_ops < 8) info->ops[info->n_ops++] = o;

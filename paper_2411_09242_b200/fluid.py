@@ -58,7 +58,7 @@ class PlanOptions(C.Structure):
                 ("unfused_attention", C.c_int32), ("split_k", C.c_int32),
                 ("eval", EVAL_FN), ("eval_user", C.c_void_p), ("eval_variant", EVAL_VARIANT_FN),
                 ("op_variant", C.POINTER(C.c_int32)), ("n_op_variant", C.c_int32), ("no_inplace", C.c_int32),
-                ("redzone_bytes", C.c_int32)]
+                ("redzone_bytes", C.c_int32), ("no_norm_split", C.c_int32)]
 
 
 class StepInfo(C.Structure):

@@ -118,6 +118,11 @@ def storage_hooks(desc, plan):
                     probs = desc.ops[o]["ins"][0]
                     fused_p[(o, probs)] = next(d for d in desc.ops if probs in d["outs"] and d["kind"] == synth.SOFTMAX)
     scores_of = {sm["ins"][0]: None for sm in fused_p.values()}     # score tensors to hold on to until P is formed
+    # an RMS normalisation split across two tensor-core steps has no record of its own, but what its readers take as
+    # their operand is bf16(x * gain), scaled by 1 / rms afterwards: a bf16 rounding of the normalised value up to that
+    # row-wise factor, i.e. of the same relative size
+    split_norm = {desc.ops[o]["outs"][0] for s in plan.steps() if s["kernel_name"] == "GEMM_TC"
+                  for o in s["ops"] if desc.ops[o]["kind"] == synth.RMSNORM}
 
     def rb(a):
         return synth.round_bf16(np.asarray(a, dtype=np.float32)).astype(np.float64)
@@ -136,6 +141,8 @@ def storage_hooks(desc, plan):
     def store(tid, a):
         if tid in scores_of:
             scores_of[tid] = a
+        if tid in split_norm:
+            return rb(a)
         if T[tid]["kind"] == synth.OUTPUT:
             dt = T[tid]["dtype"]
         else:
@@ -255,7 +262,7 @@ def check_steps_sampled(desc, plan, runner, feeds, n_rows=48, tol=2 ** -7, seed=
             elif kind in (synth.LAYERNORM, synth.RMSNORM):
                 want = graph_exec.run_op(kind, [value(op["ins"][0])] + [np.asarray(const_value(t), np.float64) for t in op["ins"][1:]],
                                          op["attrs"])[0]
-            elif kind == synth.ROPE and first["kind"] == synth.LINEAR:
+            elif kind == synth.ROPE and first["kind"] in (synth.LINEAR, synth.RMSNORM):
                 # a rotary embedding folded into the projection's step: the sampled rows are (batch, position) pairs,
                 # each rotated by its own position
                 x = np.asarray(value(op["ins"][0]), np.float64)

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 from paper_2411_09242_b200 import fluid, synth
-from tests.helpers import assert_close, rand_feed, run_gpu, run_oracle, single_op_graph, tol_for
+from tests.helpers import assert_close, check_steps_sampled, rand_feed, run_gpu, run_oracle, single_op_graph, tol_for
 
 pytestmark = pytest.mark.gpu
 
@@ -59,6 +59,36 @@ def test_small_models_planned_and_canonical(family, dtype):
     # same kernels, different arena offsets: bit-identical outputs
     for t in m.graph.outputs:
         assert np.array_equal(results["planned"][t], results["no_reuse"][t])
+
+
+def test_rms_norm_split_across_gemm_steps():
+    """A pre-norm decoder wide enough for the CTA-pair GEMMs (hidden 1024, FFN 4096, 1024 tokens): the RMS
+    normalisations between o-proj and gate / up and between down and the next layer's q / k / v have no launch of their
+    own (the first GEMM writes bf16(x * gain) and per-slab sums of squares, the readers scale their rows by 1 / rms).
+    Whole outputs against the oracle, with the split and with no_norm_split = 1; every launch of the split plan on
+    sampled rows; a planned arena (the scratch slices among the reused ones) against one slice per tensor, bit for bit."""
+    cfg = synth.scaled(synth.CONFIGS["llama"], L=2, H=1024, nh=8, F=4096, S=1024, B=1, V=2000)
+    m = synth.build_model(cfg)
+    feeds = model_feeds(m)
+    ref = run_oracle(m.graph, feeds)
+    cands = synth.default_candidates(m.graph)
+    got, plan, runner = run_gpu(m.graph, feeds, cands, arena_policy=2)
+    split_steps = [s for s in plan.steps() if s["kernel_name"] == "GEMM_TC"
+                   and any(m.graph.ops[o]["kind"] == synth.RMSNORM for o in s["ops"])]
+    assert len(split_steps) == 3                                   # layer 0: gate / up; layer 1: q / k / v and gate / up
+    assert [s["kernel_name"] for s in plan.steps()].count("NORM") == 2   # the first and the last one stay
+    assert runner.status() == 0
+    for t in m.graph.outputs:
+        assert_close(got[t], ref[t], synth.BF16, "split RMS normalisation")
+    apart, plan_apart, _ = run_gpu(m.graph, feeds, cands, arena_policy=2, no_norm_split=1)
+    assert [s["kernel_name"] for s in plan_apart.steps()].count("NORM") == 5
+    for t in m.graph.outputs:
+        assert_close(apart[t], ref[t], synth.BF16, "RMS normalisation as its own step")
+    alone, plan_alone, runner_alone = run_gpu(m.graph, feeds, cands, no_reuse=1)
+    for t in m.graph.outputs:
+        assert np.array_equal(alone[t], got[t])
+    assert check_steps_sampled(m.graph, plan_alone, runner_alone, feeds) >= len(plan_alone.steps())
+    plan.close(); plan_apart.close(); plan_alone.close()
 
 
 @pytest.mark.parametrize("family", ["gpt", "llama"])

@@ -119,6 +119,13 @@ def test_arena_matches_greedy_by_size_oracle(name, policy):
     steps = plan.steps()
     nt = len(m.graph.tensors)
     for rid, _, first, last in recs:
+        if rid >= 3 * nt:
+            # the scratch of a split RMS normalisation: from the GEMM step that fills it to the next step, which
+            # lists the normalisation among its ops and reads the scratch instead of the normalised tensor
+            assert (first, last) in ((rid - 3 * nt, rid - 3 * nt + 1), (rid - 3 * nt - len(steps), rid - 3 * nt - len(steps) + 1))
+            assert steps[first]["kernel_name"] == steps[last]["kernel_name"] == "GEMM_TC"
+            assert any(m.graph.ops[o]["kind"] == synth.RMSNORM for o in steps[last]["ops"])
+            continue
         if rid >= 2 * nt:
             assert first == last == rid - 2 * nt      # per-step scratch lives during its step only
             continue
@@ -145,7 +152,17 @@ def test_arena_over_several_orders_is_valid_and_never_larger(name):
         sizes[policy] = (plan.arena_bytes, plan.live_bound_bytes)
         plan.close()
     assert sizes[2][0] <= min(sizes[0][0], sizes[1][0])
-    assert sizes[2][0] == sizes[2][1]
+    if name == "llama":
+        # with the RMS normalisations split across their neighbouring GEMM steps the 16 MB operand of the readers
+        # lives one step longer than the normalised tensor did; the packing that meets the largest live set then
+        # alternates from layer to layer (found by placing the 43 MB products from the bottom and the top in turn):
+        # 96.5 MB against 96.25 MB (no_norm_split = 1: 96 = 96)
+        assert sizes[2][0] <= 1.005 * sizes[2][1]
+        plan = fluid.Plan(m.graph, cands, arena_policy=2, no_norm_split=1)
+        assert plan.arena_bytes == plan.live_bound_bytes
+        plan.close()
+    else:
+        assert sizes[2][0] == sizes[2][1]
 
 
 def test_no_reuse_plan_is_the_naive_sum():
@@ -211,11 +228,17 @@ def test_sibling_projections_share_one_launch():
     lp = fluid.Plan(ll.graph, synth.default_candidates(ll.graph))
     groups = sorted(((s["variant"] >> 20) & 15) for s in lp.steps() if s["kernel_name"] == "GEMM_TC" and ((s["variant"] >> 20) & 15))
     assert groups == [2, 3]                      # gate/up and q/k/v
-    # the gate/up launch also applies SiLU(gate) * up: four graph ops, one output, no slice for gate or up
-    fused = [s for s in lp.steps() if s["kernel_name"] == "GEMM_TC" and len(s["ops"]) == 4]
-    assert len(fused) == 1 and len(fused[0]["outs"]) == 1
+    # the gate/up launch also applies SiLU(gate) * up and runs the second half of the RMS normalisation in front of
+    # it (the o-proj step did the first half): five graph ops, one output, no slice for the normalised tensor, gate or up
+    fused = [s for s in lp.steps() if s["kernel_name"] == "GEMM_TC" and any(ll.graph.ops[o]["kind"] == synth.SILU for o in s["ops"])]
+    assert len(fused) == 1 and len(fused[0]["outs"]) == 1 and len(fused[0]["ops"]) == 5
     kinds = sorted(ll.graph.ops[o]["kind"] for o in fused[0]["ops"])
-    assert kinds == sorted([synth.LINEAR, synth.LINEAR, synth.SILU, synth.MUL])
+    assert kinds == sorted([synth.RMSNORM, synth.LINEAR, synth.LINEAR, synth.SILU, synth.MUL])
+    assert ll.graph.ops[fused[0]["ops"][0]]["kind"] == synth.RMSNORM     # listed first: the GEMMs read its result
+    apart = fluid.Plan(ll.graph, synth.default_candidates(ll.graph), no_norm_split=1)
+    four = [s for s in apart.steps() if s["kernel_name"] == "GEMM_TC" and any(ll.graph.ops[o]["kind"] == synth.SILU for o in s["ops"])]
+    assert len(four) == 1 and len(four[0]["ops"]) == 4 and len(apart.steps()) == len(lp.steps()) + 1
+    apart.close()
     unfused = fluid.Plan(ll.graph, synth.default_candidates(ll.graph), fusion=0)
     assert all(((s["variant"] >> 20) & 15) == 0 for s in unfused.steps())
     plan.close(); lp.close(); unfused.close()
