@@ -98,6 +98,9 @@ int finalize_steps(fluid_plan_s* p) {
         }
         s.flops = fl;
         s.bytes = es * (a + b + (g.has_bias ? g.N : 0)) + c * (s.gemm.c_f32 ? 4.0 : es) + (g.has_res ? c * (s.gemm.r_f32 ? 4.0 : es) : 0.0);
+        // split RMS normalisation: bf16(x * gain) and the slabs' sums of squares, written by one side, read by the other
+        if (s.nrm_emit) s.bytes += es * c + 4.0 * g.M * (g.N / 128);
+        if (s.nrm_pre) s.bytes += 4.0 * g.M * (g.K / 128);
         // SwiGLU step: the only tensor written is the product, which takes gate's place
         const size_t n_gemm = s.swiglu ? 2 : s.nodes.size() - s.norm_fused - s.rope_fused - s.nrm_pre;
         if (s.swiglu) {
