@@ -165,6 +165,51 @@ def test_arena_over_several_orders_is_valid_and_never_larger(name):
         assert sizes[2][0] == sizes[2][1]
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_arena_over_several_orders_on_records_of_mixed_sizes(seed):
+    """Random layered graphs whose tensors have a common width and a few odd, larger ones (what sets off the padded,
+    alternating-ends placement of arena_policy 2): every policy's placement passes the independent checker, and the
+    several-orders policy is never larger than first or best fit."""
+    rng = np.random.default_rng(100 + seed)
+    g = synth.GraphDesc()
+    M, common = 64, 64
+    x = g.tensor("in", synth.F32, [M, common], synth.INPUT)
+    avail = [(x, common)]
+    n_ops = 14 + seed % 5
+    for i in range(n_ops):
+        last = i == n_ops - 1
+        kind = synth.OUTPUT if last else synth.ACT
+        a, wa = avail[int(rng.integers(max(0, len(avail) - 4), len(avail)))]
+        r = rng.random()
+        same = [t for t in avail if t[1] == wa and t[0] != a]
+        if r < 0.45:
+            wb = common if rng.random() < 0.6 else int(rng.choice([112, 176, 200, 328]))
+            w = g.tensor(f"w{i}", synth.F32, [wa, wb], synth.CONST)
+            out = g.tensor(f"t{i}", synth.F32, [M, wb], kind)
+            g.op(synth.LINEAR, [a, w], [out], contract=1)
+            avail.append((out, wb))
+        elif r < 0.75 and same:
+            b, _ = same[int(rng.integers(len(same)))]
+            out = g.tensor(f"t{i}", synth.F32, [M, wa], kind)
+            g.op(synth.ADD, [a, b], [out])
+            avail.append((out, wa))
+        else:
+            out = g.tensor(f"t{i}", synth.F32, [M, wa], kind)
+            g.op(synth.GELU, [a], [out])
+            avail.append((out, wa))
+    sizes = {}
+    for policy in (0, 1, 2):
+        for extra in ({}, {"fusion": 0}):
+            plan = fluid.Plan(g, None, arena_policy=policy, **extra)
+            recs, offs = plan_records(plan)
+            assert OA.check_arena(recs, offs, plan.arena_bytes) == []
+            assert plan.live_bound_bytes <= plan.arena_bytes <= plan.naive_bytes
+            sizes[(policy, bool(extra))] = plan.arena_bytes
+            plan.close()
+    for unfused in (False, True):
+        assert sizes[(2, unfused)] <= min(sizes[(0, unfused)], sizes[(1, unfused)])
+
+
 def test_no_reuse_plan_is_the_naive_sum():
     m = synth.build_model(synth.CONFIGS["tiny"], materialize=False)
     plan = fluid.Plan(m.graph, None, no_reuse=1)
