@@ -2180,7 +2180,7 @@ namespace fluid {
 namespace {
 constexpr size_t kStaticHeaderBytes = 256;                 // status word + arrival counters
 constexpr size_t kStaticPartialBytes = size_t(8) << 20;    // 8 MiB of fp32 partial tiles
-__device__ __align__(256) unsigned char g_static_scratch[kStaticHeaderBytes + kStaticPartialBytes];
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticHeaderBytes + kStaticPartialBytes];
 // g_static_scratch is only a host-side handle here; the device address is looked up once per device.
 std::mutex g_static_mu;
 void* g_static_addr[64] = {};
