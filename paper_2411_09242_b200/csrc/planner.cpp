@@ -1311,7 +1311,10 @@ static int lower_and_place(fluid_plan_s* p) {
       GemmParams gu;
       // a handful of rows: the weight-streaming kernel keeps the same tiles of gate and up in one CTA
       const bool rows = gemm_rows_eligible(g) && lower_gemm(p, un, lo, &gu) && gemm_rows_eligible(gu);
-      if (!rows && (!tc.cfg.pair || g.batch != 1 || g.N % 128 != 0 || g.N0 % 128 != 0 || ((g.M + 127) / 128) % 2 != 0 || g.c_s[5] != 1))
+      GemmParams gpair[3] = {g, g, g};
+      // (gemm_pair_eligible also answers no when the pair form is switched off in the environment)
+      if (!rows && (!tc.cfg.pair || !gemm_pair_eligible(gpair, tc, 2) || g.batch != 1 || g.N % 128 != 0 || g.N0 % 128 != 0 ||
+                    ((g.M + 127) / 128) % 2 != 0 || g.c_s[5] != 1))
         continue;
       st.nodes = {gi, ui, p->steps[si + 1].node};
       st.node = gi;
