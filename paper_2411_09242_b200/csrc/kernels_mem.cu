@@ -460,7 +460,11 @@ static cudaError_t norm_t(const NormParams& p, cudaStream_t st) {
   const int nch = p.width / (vec ? V : 1);
   if (vec && nch <= 32 * 8 * 4) {
     // warps per row so that a lane owns at most 4 chunks
-    const int wpr = nch <= 128 ? 1 : (nch <= 256 ? 2 : (nch <= 512 ? 4 : 8));
+    int wpr = nch <= 128 ? 1 : (nch <= 256 ? 2 : (nch <= 512 ? 4 : 8));
+    // few rows (a 128-token encoder): the launch is one dependent chain of latencies, and a row spread over more warps
+    // and the rows over more SMs shortens it (128 x 768: 2.7 us a launch with one warp per row on 16 SMs, 1.9 us with a
+    // CTA per row on 128), as long as the grid stays one CTA per SM and a warp still has a quarter of its lanes busy
+    while (wpr < 8 && (int64_t)p.rows * (2 * wpr) <= 148 * 8 && nch >= 8 * (2 * wpr)) wpr *= 2;
     const int per_lane = (nch + 32 * wpr - 1) / (32 * wpr);
     const unsigned grid = (unsigned)((p.rows + 8 / wpr - 1) / (8 / wpr));
     const bool early = grid <= 148u * 2u;
