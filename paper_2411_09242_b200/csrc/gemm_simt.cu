@@ -115,8 +115,68 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmParams p, int a_k_fa
   }
 }
 
+// Small products (the fp32 toy configuration: 32 rows, 128-512 columns): the tiled kernel above would run as two to
+// eight CTAs, each a serial loop of load -> shared memory -> barrier -> FFMA over k with one slab in flight (15-26 us a
+// launch). Here a CTA owns one output row and 32 columns: its eight warps split the k range (lane = column: A's element
+// is one broadcast load, B's row of 32 a coalesced one, eight of each in flight per thread), the partial sums meet in
+// shared memory and are added in warp order. A hundred CTAs or more, one barrier.
+template <typename T>
+__global__ void __launch_bounds__(256) gemm_simt_small_kernel(GemmParams p) {
+  __shared__ float part[8][32];
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n = blockIdx.x * 32 + lane, m = blockIdx.y, bz = blockIdx.z;
+  const bool col_ok = n < p.N && !(p.causal == CAUSAL_SKIP_UPPER && n > (m / BM) * BM + BM - 1);
+  int kend = p.K;
+  if (p.causal == CAUSAL_CLIP_K) kend = min(p.K, (m / BM) * BM + BM);
+  const int per = ((kend + 7) / 8 + 7) & ~7;          // k elements per warp, a multiple of the unroll
+  const int k0 = warp * per, k1 = min(kend, k0 + per);
+  const T* A = static_cast<const T*>(p.A) + split_off(bz, p.B0, p.a_s[0], p.a_s[1]) + split_off(m, p.M0, p.a_s[2], p.a_s[3]);
+  const T* B = static_cast<const T*>(p.B) + split_off(bz, p.B0, p.b_s[0], p.b_s[1]) + (col_ok ? split_off(n, p.N0, p.b_s[4], p.b_s[5]) : 0);
+  pdl_wait();
+  float acc = 0.f;
+  if (col_ok) {
+    int k = k0;
+    for (; k + 8 <= k1; k += 8) {
+      float a[8], b[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        a[u] = to_f(__ldg(A + split_off(k + u, p.K0, p.a_s[4], p.a_s[5])));
+        b[u] = to_f(__ldg(B + split_off(k + u, p.K0, p.b_s[2], p.b_s[3])));
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc = fmaf(a[u], b[u], acc);
+    }
+    for (; k < k1; ++k)
+      acc = fmaf(to_f(__ldg(A + split_off(k, p.K0, p.a_s[4], p.a_s[5]))), to_f(__ldg(B + split_off(k, p.K0, p.b_s[2], p.b_s[3]))), acc);
+  }
+  part[warp][lane] = acc;
+  __syncthreads();
+  if (warp != 0 || !col_ok) return;
+  float v = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) v += part[w][lane];
+  v *= p.scale;
+  if (p.has_bias) v += to_f(static_cast<const T*>(p.bias)[n]);
+  if (p.act == ACT_GELU_ERF) v = gelu_erf(v);
+  else if (p.act == ACT_GELU_TANH) v = gelu_tanh(v);
+  if (p.has_res) {
+    const int64_t ro = split_off(bz, p.B0, p.r_s[0], p.r_s[1]) + split_off(m, p.M0, p.r_s[2], p.r_s[3]) + split_off(n, p.N0, p.r_s[4], p.r_s[5]);
+    v += (p.r_f32 && sizeof(T) == 2) ? static_cast<const float*>(p.R)[ro] : to_f(static_cast<const T*>(p.R)[ro]);
+  }
+  const int64_t co = split_off(bz, p.B0, p.c_s[0], p.c_s[1]) + split_off(m, p.M0, p.c_s[2], p.c_s[3]) + split_off(n, p.N0, p.c_s[4], p.c_s[5]);
+  if (p.c_f32 && sizeof(T) == 2) static_cast<float*>(p.C)[co] = v;
+  else static_cast<T*>(p.C)[co] = from_f<T>(v);
+}
+
 cudaError_t launch_gemm_simt(const GemmParams& p, cudaStream_t st) {
   dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, p.batch);
+  // few tiles (and few enough rows for a CTA per row and 32 columns to stay a modest grid): the small form
+  if ((int64_t)grid.x * grid.y * grid.z <= 32 && (int64_t)p.M * ((p.N + 31) / 32) * p.batch <= 4096) {
+    dim3 small((p.N + 31) / 32, p.M, p.batch);
+    return p.dtype == FLUID_BF16 ? launch_k(gemm_simt_small_kernel<__nv_bfloat16>, small, 256, 0, st, p)
+                                 : launch_k(gemm_simt_small_kernel<float>, small, 256, 0, st, p);
+  }
   const int a_k_fast = p.a_s[5] == 1 || p.a_s[3] != 1;
   const int b_n_fast = p.b_s[5] == 1 || p.b_s[3] != 1;
   return p.dtype == FLUID_BF16 ? launch_k(gemm_simt_kernel<__nv_bfloat16>, grid, 256, 0, st, p, a_k_fast, b_n_fast)
