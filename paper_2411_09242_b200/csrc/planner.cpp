@@ -334,9 +334,15 @@ double gemm_tc_variant_cost(const GemmParams& g, const GemmTcHost& tc, int n_gro
     GemmParams gs[3] = {g, g, g};
     const int sk = std::max(2, gemm_cluster_split(gs, tc, n_group));
     const double per = bn == 128 ? 107.0 : 97.0;
-    const double main = std::ceil(ksteps / sk) * 4.0 * per, exchange = 128.0 * bn * 4.0 * (sk - 1) / sk / 21.0;
+    // Measured on the 128-token encoder shape (per-step event pairs and graph replays with each form forced): with 12
+    // k-steps a tile the cluster form is no faster than one CTA per 128 x 64 tile (q / k / v 14.9 vs 13.3 us, FFN1 14.5 vs
+    // 14.3, o-proj 12.5 vs 12.5), with 48 it is (FFN2 12.4 vs 22.5): besides the bytes, the exchange costs a round of
+    // shared-memory staging and remote completion (~1800 cycles), and a cluster launch, its two barriers and its
+    // CTAs' lock-step ~1500 more than the rating's other terms account for (the o-proj, whose fp32-residual epilogue the
+    // cluster divides among its CTAs, stays on the cluster form: 13.1 vs 13.3 us).
+    const double main = std::ceil(ksteps / sk) * 4.0 * per, exchange = 1800.0 + 128.0 * bn * 4.0 * (sk - 1) / sk / 21.0;
     const double epi = (128.0 * bn * out_bytes / 32.0 + 128.0 * bn / 256.0 * 10.0) * act / sk;
-    cycles = fill + main + exchange + epi + 600.0;     // two cluster barriers
+    cycles = fill + main + exchange + epi + 600.0 + 1500.0;
   }
   return cycles / clk;
 }
@@ -434,6 +440,9 @@ double node_cost(const fluid_plan_s* p, const Node& n, const int* lo) {
         const double c_pen = g.c_s[5] == 1 ? 1.0 : (g.c_s[3] == 1 ? 1.3 : 1.6);
         // T of the node = the best over its implementation variants (tile width, CTA pair, cluster split-K)
         double best = kInf;
+        // (a residual step's output and addend are residual-stream tensors, which a bf16 plan holds in fp32 unless told
+        // otherwise: the epilogue's bytes, which the forms divide differently among their CTAs, are rated as such)
+        if (n.res >= 0 && !p->opts.narrow_stream && g.dtype == FLUID_BF16) g.c_f32 = g.r_f32 = 1;
         // (a caller's op_variant request does not enter the rating: it swaps the variant of a step, not the plan)
         for (int code : gemm_tc_variants(p, g, 1)) {
           GemmTcHost tv;
@@ -539,6 +548,7 @@ struct Evaluator {
     GemmParams g;
     GemmTcHost tc;
     if (n.kind != N_GEMM || !lower_gemm(p, n, lo.data(), &g) || !gemm_tc_eligible(p, g, &tc)) return 0;
+    if (n.res >= 0 && !p->opts.narrow_stream && g.dtype == FLUID_BF16) g.c_f32 = g.r_f32 = 1;   // as node_cost rates it
     double best = kInf;
     int arg = 0;
     for (int code : gemm_tc_variants(p, g, 1)) {
