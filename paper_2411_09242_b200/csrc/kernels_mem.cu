@@ -467,7 +467,9 @@ static cudaError_t norm_t(const NormParams& p, cudaStream_t st) {
     while (wpr < 8 && (int64_t)p.rows * (2 * wpr) <= 148 * 8 && nch >= 8 * (2 * wpr)) wpr *= 2;
     const int per_lane = (nch + 32 * wpr - 1) / (32 * wpr);
     const unsigned grid = (unsigned)((p.rows + 8 / wpr - 1) / (8 / wpr));
-    const bool early = grid <= 148u * 2u;
+    // (up to four CTAs' worth of rows per SM: 4096 x 768 runs 0.4 us a launch shorter inside a plan with the constants
+    // fetched ahead, although its 112 registers make it two waves where the late form is one)
+    const bool early = grid <= 148u * 4u;
     // many more rows than resident warps, no second addend: the persistent ring kernel
     // (with fewer rows per warp the ring never fills: measured slower on the 2048- and 4096-row norms of the model steps)
     if (!p.res && (int64_t)p.rows * wpr >= 148 * 2 * 8 * 8 && (sizeof(T) == 2 || !p.x_f32)) {
