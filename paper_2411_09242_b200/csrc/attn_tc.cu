@@ -1128,7 +1128,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream
   static bool attr[4] = {false, false, false, false};
   if (D != 64 && D != 128) return cudaErrorInvalidValue;
   const int form = attn_form(p);
-  if (form == 3) return launch_attn_small(p, stream);
+  if (form == 3) return launch_attn_small(p, &host, stream);
   if (form == 2) {
     const size_t smem = size_t(6) * TQ * D * 2 + 256 + 1024;
     const int items = ((p.S + 2 * TQ - 1) / (2 * TQ)) * p.B * p.NH;

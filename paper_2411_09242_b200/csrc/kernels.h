@@ -275,7 +275,7 @@ bool gemm_tc_describe(const GemmParams& g, GemmTcHost* tc, int variant = 0);
 cudaError_t launch_attn_tc(const AttnParams& p, const AttnHost& host, cudaStream_t stream);
 // Short sequences (S <= 128) with d contiguous in Q, K and V: one warp per 16 query rows, scores in registers.
 bool attn_small_eligible(const AttnParams& p);
-cudaError_t launch_attn_small(const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_attn_small(const AttnParams& p, const AttnHost* host, cudaStream_t stream);
 cudaError_t launch_norm(const NormParams& p, cudaStream_t stream);
 cudaError_t launch_softmax(const SoftmaxParams& p, cudaStream_t stream);
 cudaError_t launch_rope(const RopeParams& p, cudaStream_t stream);
